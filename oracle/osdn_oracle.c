@@ -1,0 +1,361 @@
+/*
+ * OSDN oracle -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, double-precision, token-by-token CPU statement of the
+ * online-scaled gated delta rule and of its reverse-mode derivative.  It is
+ * the definition the CUDA library is checked against; it shares no code with
+ * that library and must never be called from it.  Only the tests, the smoke
+ * check and the CPU-baseline leg of the benchmark may use it.
+ *
+ * What is computed, per (sequence, head) chain, for t = 1..L:
+ *
+ *   phase 1 (Algorithm 1; Eq. "dt_update_apf"; beta-aware form of the
+ *   backbone-extension appendix, Eq. "extension_beta_aware_phase1"):
+ *       ktil_t = d_t (.) k_t                       write key from PRE-update d
+ *       kap    = k_t (.) k_t ,  n = max(sum kap, eps)
+ *       a      = <d_t, kap> ,   b = beta_aware ? beta_t : 1
+ *       c      = eta * b * (1 - b a) / n
+ *       rho    = 1 | exp(g_t) | exp(l_t)           (no APF | aliased | separate)
+ *       dbar   = rho d_t + c kap ;  d_{t+1} = clip(dbar, d_min, d_max)
+ *
+ *   phase 2 (gated, online-scaled delta rule of the backbone-extension
+ *   appendix, post-gate residual):
+ *       Sbar = exp(g_t) S_{t-1}
+ *       u    = v_t - Sbar k_t                      read with the unscaled key
+ *       S_t  = Sbar + beta_t u ktil_t^T            write with the scaled key
+ *       o_t  = scale * S_t q_t                     read after the write
+ *
+ * The backward pass is the hand-derived adjoint of exactly these lines
+ * (Section 3.5 only states its factorisation); it is validated against
+ * central finite differences in the tests.
+ *
+ * Pins (tests/test_oracle_pins.py): Lemma 1 residual identity, the monotone
+ * descent corollary, reduction to the gated delta rule / DeltaNet for d == 1,
+ * beta == 0 no-op, exact overwrite for orthonormal keys, the one-hot closed
+ * form of the preconditioner recurrence, the K=V=1 alternating example, the
+ * WY product identity and the chunkwise form (an independent numpy program),
+ * APF with unit retention, split-sequence carry, finite differences.
+ * Absolute output values for random inputs have no printed example in the
+ * paper: beyond those pins they are "parity unpinned".
+ *
+ * Layout: packed tokens [T_total, H, *]; sequences given by cu_seqlens
+ * (nseq + 1 entries).  States S are [nseq, H, V, K], preconditioners
+ * [nseq, H, K].  Everything is double.
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    double eta, d_min, d_max, eps, scale;
+    int beta_aware, apf_mode, clamp;
+} oracle_hyper;
+
+int osdn_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* One phase-1 step.  Reads d (length K) and overwrites it with d_{t+1}.
+ * Optionally reports ktil, the scalar c and the pass-through mask. */
+static void phase1_step(const oracle_hyper *hp, int K, const double *k, double beta,
+                        double g, double lret, double *d, double *ktil,
+                        double *c_out, double *rho_out, double *a_out, double *n_out,
+                        int *raw_norm_above_eps, unsigned char *mask)
+{
+    double sumk = 0.0, a = 0.0;
+    for (int i = 0; i < K; ++i) {
+        double kap = k[i] * k[i];
+        if (ktil) ktil[i] = d[i] * k[i];
+        sumk += kap;
+        a += d[i] * kap;
+    }
+    double n = sumk > hp->eps ? sumk : hp->eps;
+    double b = hp->beta_aware ? beta : 1.0;
+    double c = hp->eta * b * (1.0 - b * a) / n;
+    double rho = 1.0;
+    if (hp->apf_mode == 1) rho = exp(g);
+    else if (hp->apf_mode == 2) rho = exp(lret);
+    for (int i = 0; i < K; ++i) {
+        double dbar = rho * d[i] + c * k[i] * k[i];
+        unsigned char m = 1;
+        if (hp->clamp) {
+            if (dbar < hp->d_min) { dbar = hp->d_min; m = 0; }
+            else if (dbar > hp->d_max) { dbar = hp->d_max; m = 0; }
+        }
+        d[i] = dbar;
+        if (mask) mask[i] = m;
+    }
+    if (c_out) *c_out = c;
+    if (rho_out) *rho_out = rho;
+    if (a_out) *a_out = a;
+    if (n_out) *n_out = n;
+    if (raw_norm_above_eps) *raw_norm_above_eps = sumk > hp->eps;
+}
+
+/* One phase-2 step on S (V x K, row-major).  u_out (length V) receives the
+ * post-gate residual v - Sbar k; S is overwritten by S_t. */
+static void phase2_step(int K, int V, const double *k, const double *ktil, const double *v,
+                        double beta, double g, double *S, double *u_out)
+{
+    double alpha = exp(g);
+    for (int r = 0; r < V; ++r) {
+        double *row = S + (size_t)r * K;
+        double acc = 0.0;
+        for (int i = 0; i < K; ++i) {
+            row[i] *= alpha;
+            acc += row[i] * k[i];
+        }
+        double u = v[r] - acc;
+        if (u_out) u_out[r] = u;
+        double bu = beta * u;
+        for (int i = 0; i < K; ++i) row[i] += bu * ktil[i];
+    }
+}
+
+/*
+ * Forward.  Nullable: log_ret (unless apf_mode 2), S0 (zeros), d0 (ones),
+ * ktil_out, d_traj_out ([T_total, H, K], the PRE-update d_t of every token).
+ */
+void osdn_oracle_fwd(int nseq, const int *cu, int H, int K, int V, const oracle_hyper *hp,
+                     const double *q, const double *k, const double *v,
+                     const double *beta, const double *gate, const double *log_ret,
+                     const double *S0, const double *d0,
+                     double *out, double *S_final, double *d_final,
+                     double *ktil_out, double *d_traj_out)
+{
+    int nchain = nseq * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int ch = 0; ch < nchain; ++ch) {
+        int s = ch / H, h = ch % H;
+        int t0 = cu[s], t1 = cu[s + 1];
+        double *S = (double *)malloc(sizeof(double) * V * K);
+        double *d = (double *)malloc(sizeof(double) * K);
+        double *ktil = (double *)malloc(sizeof(double) * K);
+        if (S0) memcpy(S, S0 + ((size_t)s * H + h) * V * K, sizeof(double) * V * K);
+        else memset(S, 0, sizeof(double) * V * K);
+        for (int i = 0; i < K; ++i) d[i] = d0 ? d0[((size_t)s * H + h) * K + i] : 1.0;
+        for (int t = t0; t < t1; ++t) {
+            size_t th = (size_t)t * H + h;
+            const double *kt = k + th * K, *qt = q + th * K, *vt = v + th * V;
+            if (d_traj_out) memcpy(d_traj_out + th * K, d, sizeof(double) * K);
+            phase1_step(hp, K, kt, beta[th], gate[th], log_ret ? log_ret[th] : 0.0, d, ktil,
+                        0, 0, 0, 0, 0, 0);
+            if (ktil_out) memcpy(ktil_out + th * K, ktil, sizeof(double) * K);
+            phase2_step(K, V, kt, ktil, vt, beta[th], gate[th], S, 0);
+            for (int r = 0; r < V; ++r) {
+                double acc = 0.0;
+                for (int i = 0; i < K; ++i) acc += S[(size_t)r * K + i] * qt[i];
+                out[th * V + r] = hp->scale * acc;
+            }
+        }
+        if (S_final) memcpy(S_final + ((size_t)s * H + h) * V * K, S, sizeof(double) * V * K);
+        if (d_final) memcpy(d_final + ((size_t)s * H + h) * K, d, sizeof(double) * K);
+        free(S); free(d); free(ktil);
+    }
+}
+
+/* Phase 1 alone (the stand-alone preconditioner update). */
+void osdn_oracle_precond_update(int nseq, const int *cu, int H, int K, const oracle_hyper *hp,
+                                const double *k, const double *beta, const double *gate,
+                                const double *log_ret, const double *d0,
+                                double *ktil_out, double *d_final)
+{
+    int nchain = nseq * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int ch = 0; ch < nchain; ++ch) {
+        int s = ch / H, h = ch % H;
+        double *d = (double *)malloc(sizeof(double) * K);
+        double *ktil = (double *)malloc(sizeof(double) * K);
+        for (int i = 0; i < K; ++i) d[i] = d0 ? d0[((size_t)s * H + h) * K + i] : 1.0;
+        for (int t = cu[s]; t < cu[s + 1]; ++t) {
+            size_t th = (size_t)t * H + h;
+            phase1_step(hp, K, k + th * K, beta[th], gate ? gate[th] : 0.0,
+                        log_ret ? log_ret[th] : 0.0, d, ktil, 0, 0, 0, 0, 0, 0);
+            if (ktil_out) memcpy(ktil_out + th * K, ktil, sizeof(double) * K);
+        }
+        memcpy(d_final + ((size_t)s * H + h) * K, d, sizeof(double) * K);
+        free(d); free(ktil);
+    }
+}
+
+/*
+ * Backward: reverse sweep over the same recurrence.
+ *
+ * Cotangents in: dout [T,H,V]; dS_final, dd_final nullable (zeros).
+ * Gradients out: dq, dk [T,H,K], dv [T,H,V], dbeta, dgate [T,H],
+ * dlog_ret [T,H] (nullable; written only for apf_mode 2), dS0, dd0 (nullable).
+ *
+ * S_{t-1} and d_t are needed in reverse order.  Each chain keeps S and d at
+ * every SEG-token boundary during a forward sweep, then walks the segments
+ * backwards, re-running each segment forward with a full per-token history.
+ *
+ * Conventions where the paper is silent: the box projection passes gradient
+ * iff d_min <= dbar <= d_max; max(|k|^2, eps) passes gradient iff |k|^2 > eps.
+ */
+#define SEG 64
+
+void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_hyper *hp,
+                     const double *q, const double *k, const double *v,
+                     const double *beta, const double *gate, const double *log_ret,
+                     const double *S0, const double *d0,
+                     const double *dout, const double *dS_final, const double *dd_final,
+                     double *dq, double *dk, double *dv, double *dbeta, double *dgate,
+                     double *dlog_ret, double *dS0, double *dd0)
+{
+    int nchain = nseq * H;
+    size_t VK = (size_t)V * K;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int ch = 0; ch < nchain; ++ch) {
+        int s = ch / H, h = ch % H;
+        int t0 = cu[s], t1 = cu[s + 1];
+        int L = t1 - t0;
+        int nseg = (L + SEG - 1) / SEG;
+        double *Sck = (double *)malloc(sizeof(double) * VK * (nseg > 0 ? nseg : 1));
+        double *dck = (double *)malloc(sizeof(double) * K * (nseg > 0 ? nseg : 1));
+        double *Shist = (double *)malloc(sizeof(double) * VK * (SEG + 1)); /* S before each token */
+        double *dhist = (double *)malloc(sizeof(double) * K * (SEG + 1));  /* d before each token */
+        double *S = (double *)malloc(sizeof(double) * VK);
+        double *d = (double *)malloc(sizeof(double) * K);
+        double *ktil = (double *)malloc(sizeof(double) * K);
+        double *Shat = (double *)malloc(sizeof(double) * VK);   /* dL/dS_t */
+        double *lam = (double *)malloc(sizeof(double) * K);     /* dL/dd_{t+1} */
+        double *Sbar = (double *)malloc(sizeof(double) * VK);
+        double *u = (double *)malloc(sizeof(double) * V);
+        double *w = (double *)malloc(sizeof(double) * V);
+        double *du = (double *)malloc(sizeof(double) * V);
+        double *dktil = (double *)malloc(sizeof(double) * K);
+        double *dnew = (double *)malloc(sizeof(double) * K);
+        unsigned char *mask = (unsigned char *)malloc(K);
+
+        if (S0) memcpy(S, S0 + ((size_t)s * H + h) * VK, sizeof(double) * VK);
+        else memset(S, 0, sizeof(double) * VK);
+        for (int i = 0; i < K; ++i) d[i] = d0 ? d0[((size_t)s * H + h) * K + i] : 1.0;
+
+        /* forward sweep keeping segment-boundary checkpoints */
+        for (int sg = 0; sg < nseg; ++sg) {
+            memcpy(Sck + (size_t)sg * VK, S, sizeof(double) * VK);
+            memcpy(dck + (size_t)sg * K, d, sizeof(double) * K);
+            int a0 = t0 + sg * SEG, a1 = a0 + SEG < t1 ? a0 + SEG : t1;
+            for (int t = a0; t < a1; ++t) {
+                size_t th = (size_t)t * H + h;
+                phase1_step(hp, K, k + th * K, beta[th], gate[th], log_ret ? log_ret[th] : 0.0,
+                            d, ktil, 0, 0, 0, 0, 0, 0);
+                phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
+            }
+        }
+
+        if (dS_final) memcpy(Shat, dS_final + ((size_t)s * H + h) * VK, sizeof(double) * VK);
+        else memset(Shat, 0, sizeof(double) * VK);
+        for (int i = 0; i < K; ++i) lam[i] = dd_final ? dd_final[((size_t)s * H + h) * K + i] : 0.0;
+
+        for (int sg = nseg - 1; sg >= 0; --sg) {
+            int a0 = t0 + sg * SEG, a1 = a0 + SEG < t1 ? a0 + SEG : t1;
+            /* replay the segment, recording S_{t-1} and d_t for every token */
+            memcpy(S, Sck + (size_t)sg * VK, sizeof(double) * VK);
+            memcpy(d, dck + (size_t)sg * K, sizeof(double) * K);
+            for (int t = a0; t < a1; ++t) {
+                size_t th = (size_t)t * H + h;
+                memcpy(Shist + (size_t)(t - a0) * VK, S, sizeof(double) * VK);
+                memcpy(dhist + (size_t)(t - a0) * K, d, sizeof(double) * K);
+                phase1_step(hp, K, k + th * K, beta[th], gate[th], log_ret ? log_ret[th] : 0.0,
+                            d, ktil, 0, 0, 0, 0, 0, 0);
+                phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
+            }
+            for (int t = a1 - 1; t >= a0; --t) {
+                size_t th = (size_t)t * H + h;
+                const double *kt = k + th * K, *qt = q + th * K, *vt = v + th * V;
+                const double *dot = dout + th * V;
+                const double *Sprev = Shist + (size_t)(t - a0) * VK;
+                const double *dt = dhist + (size_t)(t - a0) * K;
+                double bt = beta[th], gt = gate[th], lt = log_ret ? log_ret[th] : 0.0;
+                double alpha = exp(gt);
+
+                /* recompute this token's forward quantities */
+                double c, rho, a, n; int above;
+                memcpy(dnew, dt, sizeof(double) * K);
+                phase1_step(hp, K, kt, bt, gt, lt, dnew, ktil, &c, &rho, &a, &n, &above, mask);
+                for (int r = 0; r < V; ++r) {
+                    double acc = 0.0;
+                    for (int i = 0; i < K; ++i) {
+                        Sbar[(size_t)r * K + i] = alpha * Sprev[(size_t)r * K + i];
+                        acc += Sbar[(size_t)r * K + i] * kt[i];
+                    }
+                    u[r] = vt[r] - acc;
+                }
+                /* o_t = scale S_t q_t with S_t = Sbar + beta u ktil^T */
+                {
+                    for (int i = 0; i < K; ++i) dq[th * K + i] = 0.0;
+                    for (int r = 0; r < V; ++r) {
+                        double sdo = hp->scale * dot[r];
+                        for (int i = 0; i < K; ++i) {
+                            double St = Sbar[(size_t)r * K + i] + bt * u[r] * ktil[i];
+                            dq[th * K + i] += sdo * St;
+                            Shat[(size_t)r * K + i] += sdo * qt[i];
+                        }
+                    }
+                }
+                /* S_t = Sbar + beta u ktil^T */
+                double dbeta_t = 0.0;
+                for (int i = 0; i < K; ++i) dktil[i] = 0.0;
+                for (int r = 0; r < V; ++r) {
+                    double acc = 0.0;
+                    for (int i = 0; i < K; ++i) acc += Shat[(size_t)r * K + i] * ktil[i];
+                    w[r] = acc;
+                    dbeta_t += u[r] * acc;
+                    du[r] = bt * acc;
+                    for (int i = 0; i < K; ++i) dktil[i] += bt * u[r] * Shat[(size_t)r * K + i];
+                }
+                /* u = v - Sbar k ; Sbar = alpha S_{t-1} */
+                double dg_t = 0.0;
+                for (int i = 0; i < K; ++i) dk[th * K + i] = 0.0;
+                for (int r = 0; r < V; ++r) {
+                    dv[th * V + r] = du[r];
+                    for (int i = 0; i < K; ++i) {
+                        size_t id = (size_t)r * K + i;
+                        dk[th * K + i] -= Sbar[id] * du[r];
+                        double dSbar = Shat[id] - du[r] * kt[i];
+                        dg_t += dSbar * Sbar[id];
+                        Shat[id] = alpha * dSbar;          /* now dL/dS_{t-1} */
+                    }
+                }
+                /* phase-1 adjoint of this step; lam holds dL/dd_{t+1} */
+                double drho = 0.0, dc = 0.0;
+                for (int i = 0; i < K; ++i) {
+                    double lb = mask[i] ? lam[i] : 0.0;
+                    lam[i] = lb;
+                    drho += lb * dt[i];
+                    dc += lb * kt[i] * kt[i];
+                }
+                double b = hp->beta_aware ? bt : 1.0;
+                double da = -hp->eta * b * b / n * dc;
+                double db = hp->eta * (1.0 - 2.0 * b * a) / n * dc;
+                double dn = above ? -c / n * dc : 0.0;
+                if (hp->beta_aware) dbeta_t += db;
+                for (int i = 0; i < K; ++i) {
+                    double kap = kt[i] * kt[i];
+                    double dkap = c * lam[i] + da * dt[i] + dn;
+                    dk[th * K + i] += dt[i] * dktil[i] + 2.0 * kt[i] * dkap;
+                    lam[i] = rho * lam[i] + da * kap + kt[i] * dktil[i];   /* dL/dd_t */
+                }
+                if (hp->apf_mode == 1) dg_t += rho * drho;
+                if (dlog_ret) dlog_ret[th] = hp->apf_mode == 2 ? rho * drho : 0.0;
+                dbeta[th] = dbeta_t;
+                dgate[th] = dg_t;
+            }
+        }
+        if (dS0) memcpy(dS0 + ((size_t)s * H + h) * VK, Shat, sizeof(double) * VK);
+        if (dd0) memcpy(dd0 + ((size_t)s * H + h) * K, lam, sizeof(double) * K);
+
+        free(Sck); free(dck); free(Shist); free(dhist); free(S); free(d); free(ktil);
+        free(Shat); free(lam); free(Sbar); free(u); free(w); free(du); free(dktil);
+        free(dnew); free(mask);
+    }
+}

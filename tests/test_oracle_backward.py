@@ -1,0 +1,161 @@
+"""Pins of the oracle's reverse sweep: central finite differences of the oracle
+forward, and agreement with an independently derived chunk-level reverse pass."""
+import numpy as np
+import pytest
+
+import oracle
+import chunkwise_np as cw
+from paper_2605_13473_b200.synth import OsdnHyper
+
+
+def _unit(x):
+    return x / np.linalg.norm(x, axis=-1, keepdims=True)
+
+
+def _case(seed, hy, L=11, H=2, K=5, V=4, lens=None, unit=False):
+    r = np.random.default_rng(seed)
+    lens = lens or [L]
+    T = sum(lens)
+    ns = len(lens)
+    k = r.standard_normal((T, H, K)) * 0.6
+    if unit:
+        k = _unit(k)
+    x = dict(
+        q=_unit(r.standard_normal((T, H, K))), k=k, v=r.standard_normal((T, H, V)),
+        beta=1 / (1 + np.exp(-r.standard_normal((T, H)))),
+        gate=-0.4 * np.abs(r.standard_normal((T, H))),
+        log_ret=-0.2 * np.abs(r.standard_normal((T, H))),
+        init_state=0.5 * r.standard_normal((ns, H, V, K)),
+        precond_in=hy.d_min + (hy.d_max - hy.d_min) * r.random((ns, H, K)),
+    )
+    cot = dict(out=r.standard_normal((T, H, V)), final_state=r.standard_normal((ns, H, V, K)),
+               precond_out=r.standard_normal((ns, H, K)))
+    return lens, x, cot
+
+
+def _loss(hy, lens, x, cot):
+    res = oracle.fwd(hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], x["log_ret"],
+                     x["init_state"], x["precond_in"])
+    return sum(float(np.sum(res[n] * cot[n])) for n in cot)
+
+
+def _min_margin(hy, lens, x):
+    """Smallest distance of any pre-projection value to a box face (kink of the clamp)."""
+    if not hy.clamp:
+        return np.inf, 0.0
+    m = np.inf
+    frac_clamped = []
+    off = 0
+    for s, n in enumerate(lens):
+        for h in range(x["k"].shape[1]):
+            sl = slice(off, off + n)
+            _, dtr, dfin, cs, rhos, mask, *_ = cw.phase1_np(x["k"][sl, h], x["beta"][sl, h], x["gate"][sl, h],
+                                                        x["log_ret"][sl, h], x["precond_in"][s, h], hy)
+            dbar = rhos[:, None] * dtr + cs[:, None] * x["k"][sl, h] ** 2
+            m = min(m, np.abs(dbar - hy.d_min).min(), np.abs(dbar - hy.d_max).min())
+            frac_clamped.append(1.0 - mask.mean())
+        off += n
+    return m, float(np.mean(frac_clamped))
+
+
+HYPERS = [
+    ("alias_clamped", OsdnHyper(eta=0.5, apf_mode=1)),
+    ("separate_ret", OsdnHyper(eta=0.5, apf_mode=2)),
+    ("no_apf", OsdnHyper(eta=0.8, apf_mode=0)),
+    ("no_clamp", OsdnHyper(eta=0.3, apf_mode=1, clamp=0)),
+    ("not_beta_aware", OsdnHyper(eta=0.5, apf_mode=2, beta_aware=0)),
+]
+
+
+@pytest.mark.parametrize("name,hy", HYPERS, ids=[h[0] for h in HYPERS])
+def test_backward_matches_finite_differences(name, hy):
+    # pick a seed whose trajectory is partly clamped yet stays 1e-4 away from every kink
+    for seed in range(200, 260):
+        lens, x, cot = _case(seed, hy, lens=[7, 5])
+        margin, frac = _min_margin(hy, lens, x)
+        if margin > 1e-4 and (not hy.clamp or 0.02 < frac < 0.98):
+            break
+    else:
+        pytest.fail("no usable seed")
+    g = oracle.bwd(hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], cot["out"], x["log_ret"],
+                   x["init_state"], x["precond_in"], cot["final_state"], cot["precond_out"])
+    names = dict(q="dq", k="dk", v="dv", beta="dbeta", gate="dgate", init_state="dinit_state",
+                 precond_in="dprecond_in")
+    if hy.apf_mode == 2:
+        names["log_ret"] = "dlog_ret"
+    h = 1e-6
+    r = np.random.default_rng(7)
+    for inp, gname in names.items():
+        arr = x[inp]
+        flat = arr.reshape(-1)
+        idxs = r.choice(flat.size, size=min(flat.size, 25), replace=False)
+        for i in idxs:
+            old = flat[i]
+            flat[i] = old + h
+            lp = _loss(hy, lens, x, cot)
+            flat[i] = old - h
+            lm = _loss(hy, lens, x, cot)
+            flat[i] = old
+            fd = (lp - lm) / (2 * h)
+            an = g[gname].reshape(-1)[i]
+            assert abs(fd - an) <= 2e-6 * max(1.0, abs(an)), (name, inp, i, fd, an)
+    if hy.apf_mode != 2:
+        assert np.all(g["dlog_ret"] == 0.0)
+
+
+@pytest.mark.parametrize("name,hy", HYPERS, ids=[h[0] for h in HYPERS])
+def test_backward_directional_derivative(name, hy):
+    """<grad, direction> equals the directional finite difference (all inputs at once)."""
+    lens, x, cot = _case(300, hy, lens=[9, 4, 6])
+    for seed in range(300, 360):
+        lens, x, cot = _case(seed, hy, lens=[9, 4, 6])
+        if _min_margin(hy, lens, x)[0] > 1e-4:
+            break
+    g = oracle.bwd(hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], cot["out"], x["log_ret"],
+                   x["init_state"], x["precond_in"], cot["final_state"], cot["precond_out"])
+    r = np.random.default_rng(11)
+    names = dict(q="dq", k="dk", v="dv", beta="dbeta", gate="dgate", log_ret="dlog_ret",
+                 init_state="dinit_state", precond_in="dprecond_in")
+    dirs = {n: r.standard_normal(x[n].shape) for n in names}
+    dirs["precond_in"] *= 0.1
+    an = sum(float(np.sum(g[names[n]] * dirs[n])) for n in names)
+    h = 1e-6
+    xp = {n: x[n] + h * dirs[n] for n in names}
+    xm = {n: x[n] - h * dirs[n] for n in names}
+    fd = (_loss(hy, lens, xp, cot) - _loss(hy, lens, xm, cot)) / (2 * h)
+    assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (fd, an)
+
+
+@pytest.mark.parametrize("name,hy", HYPERS, ids=[h[0] for h in HYPERS])
+@pytest.mark.parametrize("L", [3, 64, 150])
+def test_chunk_level_reverse_pass_equals_token_level(name, hy, L):
+    lens, x, cot = _case(400 + L, hy, H=2, K=8, V=6, lens=[L, 17], unit=True)
+    a = oracle.bwd(hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], cot["out"], x["log_ret"],
+                   x["init_state"], x["precond_in"], cot["final_state"], cot["precond_out"])
+    b = cw.layer_bwd(hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], cot["out"], x["log_ret"],
+                     x["init_state"], x["precond_in"], cot["final_state"], cot["precond_out"])
+    for key in a:
+        scale = max(1.0, np.abs(a[key]).max())
+        np.testing.assert_allclose(a[key], b[key], atol=1e-9 * scale, rtol=0, err_msg=key)
+
+
+def test_backward_segment_checkpointing_is_transparent():
+    """Gradients of a 150-token chain (three replay segments) equal those of the same chain
+    split in two calls with the state cotangents handed across the split."""
+    hy = OsdnHyper(eta=0.5, apf_mode=1)
+    lens, x, cot = _case(500, hy, H=1, K=6, V=4, lens=[150], unit=True)
+    full = oracle.bwd(hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], cot["out"], None,
+                      x["init_state"], x["precond_in"], cot["final_state"], cot["precond_out"])
+    n1 = 70
+    f1 = oracle.fwd(hy, [n1], x["q"][:n1], x["k"][:n1], x["v"][:n1], x["beta"][:n1], x["gate"][:n1],
+                    None, x["init_state"], x["precond_in"])
+    b2 = oracle.bwd(hy, [150 - n1], x["q"][n1:], x["k"][n1:], x["v"][n1:], x["beta"][n1:], x["gate"][n1:],
+                    cot["out"][n1:], None, f1["final_state"], f1["precond_out"],
+                    cot["final_state"], cot["precond_out"])
+    b1 = oracle.bwd(hy, [n1], x["q"][:n1], x["k"][:n1], x["v"][:n1], x["beta"][:n1], x["gate"][:n1],
+                    cot["out"][:n1], None, x["init_state"], x["precond_in"],
+                    b2["dinit_state"], b2["dprecond_in"])
+    for key in ("dq", "dk", "dv", "dbeta", "dgate"):
+        np.testing.assert_allclose(np.concatenate([b1[key], b2[key]]), full[key], atol=1e-12)
+    np.testing.assert_allclose(b1["dinit_state"], full["dinit_state"], atol=1e-12)
+    np.testing.assert_allclose(b1["dprecond_in"], full["dprecond_in"], atol=1e-12)
