@@ -1,0 +1,163 @@
+/*
+ * osdn.h -- C ABI of the B200 (sm_100a) OSDN layer library.
+ *
+ * The library computes the chunkwise-parallel, gated, online-scaled delta-rule
+ * sequence layer (OSDN / OSGDN with Adaptive Preconditioner Forgetting):
+ *
+ *   phase 1  (Algorithm 1; Eq. "dt_update_apf"; beta-aware form
+ *             Eq. "extension_beta_aware_phase1"), per (sequence, head), t = 1..L:
+ *       ktil_t  = d_t (.) k_t                          (write key, pre-update d)
+ *       c_t     = eta * b_t * (1 - b_t <d_t, k_t^2>) / max(|k_t|^2, eps),  b_t = beta_t or 1
+ *       d_{t+1} = clip(rho_t d_t + c_t k_t^2, d_min, d_max),  rho_t = 1 | exp(g_t) | exp(l_t)
+ *   phase 2  (Eq. "recurrent_form" with the gate of the backbone-extension appendix):
+ *       S_t = exp(g_t) S_{t-1} + beta_t (v_t - exp(g_t) S_{t-1} k_t) ktil_t^T ,  o_t = scale * S_t q_t
+ *
+ * evaluated chunk by chunk (chunk = 64 tokens) through the UT / WY transform of the
+ * chunkwise-WY appendix and its gated form (decay-ratio Gram, unit-triangular inverse,
+ * pseudo keys W and values U, suffix-gated state advance), and the reverse-mode
+ * derivative of all of it (Section 3.5: phase 2 yields dL/dktil, the gradient through d
+ * is a reverse sweep over the projected affine recurrence).
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer unless the name ends in _host.  The caller
+ *     owns all buffers; the library allocates no device memory and keeps no state
+ *     between calls.  Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = default stream) and return without synchronising.
+ *   - Token tensors are packed [T_total, H, D] row-major (a dense [B, T, H, D] batch is
+ *     the same memory).  q, k, v, out, dout, dq, dk, dv are `io_dtype` (fp32 or bf16);
+ *     beta, gate (log-decay g <= 0), log-retention, states, preconditioners and their
+ *     gradients are fp32.  States are [S, H, V, K], preconditioners [S, H, K], where
+ *     S = B (dense) or nseq (var-len).  All pointers must be 16-byte aligned.
+ *   - Sequences: dense (nseq == 0): B sequences of T tokens.  Var-len (nseq > 0): B must
+ *     be 1, T is the packed token count and cu_seqlens (device, int32, nseq+1 entries,
+ *     non-decreasing, cu[0] = 0, cu[nseq] = T) gives the boundaries; state and
+ *     preconditioner restart at every boundary and chunks never straddle sequences.
+ *   - Return value: 0 on success, a negative osdn_status otherwise.  Arguments are
+ *     validated before anything is launched; on error nothing has been enqueued.
+ *     Errors detected on the device (a bounded wait that ran out) are recorded in the
+ *     first 4 bytes of the workspace, readable with osdn_read_device_status after the
+ *     stream has been synchronised.
+ */
+#ifndef OSDN_H_
+#define OSDN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum osdn_status {
+    OSDN_OK = 0,
+    OSDN_INVALID_ARG = -1,        /* null required pointer, bad enum, inconsistent sizes   */
+    OSDN_UNSUPPORTED_SHAPE = -2,  /* K or V not in {64, 128}, chunk != 64, T <= 0, ...      */
+    OSDN_MISALIGNED = -3,         /* a pointer is not 16-byte aligned                      */
+    OSDN_WORKSPACE_TOO_SMALL = -4,
+    OSDN_CUDA_ERROR = -5          /* a CUDA runtime call or launch failed                  */
+} osdn_status;
+
+enum { OSDN_FP32 = 0, OSDN_BF16 = 1 };
+enum { OSDN_APF_NONE = 0, OSDN_APF_ALIAS_GATE = 1, OSDN_APF_SEPARATE = 2 };
+enum {
+    OSDN_FLAG_SAVE_RESIDUALS = 1,  /* osdn_fwd: keep chunk residuals in the workspace for osdn_bwd */
+    OSDN_FLAG_RESIDUALS_VALID = 2, /* osdn_bwd: the workspace holds the residuals of the matching
+                                      osdn_fwd call (same params, same inputs); otherwise osdn_bwd
+                                      recomputes the forward itself                              */
+    OSDN_FLAG_FORCE_SIMT = 4       /* use the fp32 CUDA-core kernels even for bf16 I/O          */
+};
+
+typedef struct osdn_params {
+    int32_t B, T, H, K, V;      /* dense: [B,T,H,*]; var-len: B = 1, T = packed tokens          */
+    int32_t chunk;              /* 64                                                            */
+    int32_t io_dtype;           /* OSDN_FP32 | OSDN_BF16                                         */
+    float   eta, d_min, d_max;  /* step size and box of the preconditioner (0.003, 0.5, 2.0)     */
+    float   eps;                /* floor of |k|^2 (1e-6)                                         */
+    float   scale;              /* output scale on q; <= 0 selects K^-1/2                        */
+    int32_t beta_aware;         /* 1: b_t = beta_t ; 0: b_t = 1                                  */
+    int32_t apf_mode;           /* OSDN_APF_*                                                    */
+    int32_t clamp;              /* 1: project onto the box after every token ; 0: never          */
+    int32_t nseq;               /* 0 = dense                                                     */
+    const int32_t* cu_seqlens;  /* device pointer, nseq+1 entries (var-len only)                 */
+    int32_t flags;              /* OSDN_FLAG_*                                                   */
+} osdn_params;
+
+/* Bytes of device scratch the calls below need for these params (need_bwd != 0: enough
+ * for osdn_fwd with OSDN_FLAG_SAVE_RESIDUALS followed by osdn_bwd).  0 on invalid params. */
+size_t osdn_workspace_bytes(const osdn_params* p, int need_bwd);
+
+/*
+ * Forward (Algorithm 1 + the gated chunk form).
+ *   in : q,k [T,H,K], v [T,H,V] io_dtype; beta, gate [T,H] fp32;
+ *        apf_log_ret [T,H] fp32 (required iff apf_mode == SEPARATE, else may be NULL);
+ *        init_state [S,H,V,K] (NULL = zeros); precond_in [S,H,K] (NULL = ones).
+ *   out: out [T,H,V] io_dtype; final_state [S,H,V,K] and precond_out [S,H,K] fp32 (either may
+ *        be NULL; precond_out may alias precond_in).
+ *   workspace: >= osdn_workspace_bytes(p, flags & SAVE_RESIDUALS) bytes, 256-byte aligned.
+ */
+int osdn_fwd(const osdn_params* p, const void* q, const void* k, const void* v,
+             const float* beta, const float* gate, const float* apf_log_ret,
+             const float* init_state, const float* precond_in,
+             void* out, float* final_state, float* precond_out,
+             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward (Section 3.5): gradients of sum(out*dout) + sum(final_state*dfinal_state) +
+ * sum(precond_out*dprecond_out) with respect to every forward input.
+ *   in : the forward inputs; dout [T,H,V] io_dtype; dfinal_state, dprecond_out (NULL = zeros).
+ *   out: dq, dk [T,H,K], dv [T,H,V] io_dtype; dbeta, dgate [T,H] fp32;
+ *        dapf_log_ret [T,H] (written iff apf_mode == SEPARATE; may be NULL otherwise);
+ *        dinit_state [S,H,V,K], dprecond_in [S,H,K] (either may be NULL).
+ *   The projection passes gradient where d_min <= pre-projection value <= d_max;
+ *   max(|k|^2, eps) passes gradient where |k|^2 > eps.
+ *   workspace: >= osdn_workspace_bytes(p, 1) bytes.
+ */
+int osdn_bwd(const osdn_params* p, const void* q, const void* k, const void* v,
+             const float* beta, const float* gate, const float* apf_log_ret,
+             const float* init_state, const float* precond_in,
+             const void* dout, const float* dfinal_state, const float* dprecond_out,
+             void* dq, void* dk, void* dv, float* dbeta, float* dgate, float* dapf_log_ret,
+             float* dinit_state, float* dprecond_in,
+             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Phase 1 alone (Algorithm 1 as its own pass; Section 3.5 "Phase 1"): advances the
+ * preconditioner over the given tokens and optionally emits the write keys.
+ *   in : k [T,H,K] io_dtype; beta [T,H]; gate_or_log_ret [T,H] (the log-retention source:
+ *        the gate for ALIAS_GATE, the separate log-retention for SEPARATE; may be NULL for
+ *        APF_NONE); precond_in [S,H,K] (NULL = ones).
+ *   out: k_tilde_out [T,H,K] io_dtype (may be NULL); precond_out [S,H,K] (required; may alias
+ *        precond_in).  Needs no workspace for dense batches; var-len reads cu_seqlens directly.
+ */
+int osdn_precond_update(const osdn_params* p, const void* k, const float* beta,
+                        const float* gate_or_log_ret, const float* precond_in,
+                        void* k_tilde_out, float* precond_out, void* cuda_stream);
+
+/*
+ * Host-buffer convenience for end-to-end measurements: copies the inputs (HOST pointers,
+ * ideally pinned) into `staging` (device scratch of osdn_host_staging_bytes bytes), runs
+ * osdn_fwd (and osdn_bwd when dout_host != NULL) and copies out / the gradients back to the
+ * host buffers, all on `cuda_stream`, without synchronising.  Same layouts as above; NULL
+ * optional inputs as above.  Nothing is allocated.
+ */
+size_t osdn_host_staging_bytes(const osdn_params* p, int with_bwd);
+int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host, const void* v_host,
+                   const float* beta_host, const float* gate_host, const void* dout_host,
+                   void* out_host, void* dq_host, void* dk_host, void* dv_host,
+                   float* dbeta_host, float* dgate_host,
+                   void* staging, size_t staging_bytes, void* cuda_stream);
+
+/* Reads the device status word at the head of a workspace (synchronous 4-byte copy).
+ * 0 = no device-side error recorded. */
+int osdn_read_device_status(const void* workspace, int32_t* status_host);
+
+const char* osdn_status_string(int status);
+
+/* Number of kernel launches the most recent osdn_fwd / osdn_bwd / osdn_precond_update call of
+ * this thread enqueued (for launch accounting in benchmarks). */
+int osdn_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OSDN_H_ */

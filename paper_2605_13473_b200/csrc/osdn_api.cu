@@ -1,0 +1,282 @@
+// C ABI of the OSDN library: argument validation, workspace carving, launch plans.
+// No device memory is allocated here and no state survives a call (apart from a
+// thread-local launch counter used for benchmark accounting).
+#include <cmath>
+#include <cstring>
+
+#include "osdn_common.cuh"
+
+namespace osdn {
+int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+               bool save, cudaStream_t st);
+int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                cudaStream_t st);
+bool tc_supported(const osdn_params& p);
+}  // namespace osdn
+
+using namespace osdn;
+
+namespace {
+
+thread_local int g_last_launches = 0;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate(const osdn_params* p)
+{
+    if (!p) return OSDN_INVALID_ARG;
+    if (p->io_dtype != OSDN_FP32 && p->io_dtype != OSDN_BF16) return OSDN_INVALID_ARG;
+    if (p->apf_mode < 0 || p->apf_mode > 2) return OSDN_INVALID_ARG;
+    if (p->B <= 0 || p->H <= 0) return OSDN_INVALID_ARG;
+    if (p->T <= 0) return OSDN_UNSUPPORTED_SHAPE;
+    if (p->chunk != CH) return OSDN_UNSUPPORTED_SHAPE;
+    if ((p->K != 64 && p->K != 128) || (p->V != 64 && p->V != 128)) return OSDN_UNSUPPORTED_SHAPE;
+    if (p->nseq < 0) return OSDN_INVALID_ARG;
+    if (p->nseq > 0 && (p->B != 1 || !p->cu_seqlens)) return OSDN_INVALID_ARG;
+    if (!(p->d_min <= p->d_max) || !(p->eps > 0.f) || !std::isfinite(p->eta)) return OSDN_INVALID_ARG;
+    const double tokens = (double)p->B * p->T;
+    if (tokens * p->H * (p->K > p->V ? p->K : p->V) > 2.0e10) return OSDN_UNSUPPORTED_SHAPE;
+    if (tokens > 1.0e9) return OSDN_UNSUPPORTED_SHAPE;
+    return OSDN_OK;
+}
+
+Hyper make_hyper(const osdn_params& p)
+{
+    Hyper h;
+    h.eta = p.eta; h.d_min = p.d_min; h.d_max = p.d_max; h.eps = p.eps;
+    h.scale = p.scale > 0.f ? p.scale : 1.0f / std::sqrt((float)p.K);
+    h.beta_aware = p.beta_aware ? 1 : 0; h.apf_mode = p.apf_mode; h.clamp = p.clamp ? 1 : 0;
+    return h;
+}
+
+bool use_tc(const osdn_params& p)
+{
+    return p.io_dtype == OSDN_BF16 && !(p.flags & OSDN_FLAG_FORCE_SIMT) && tc_supported(p);
+}
+
+int run_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                bool save, cudaStream_t st)
+{
+    int n0 = launch_build_table(p, L, ws, st);
+    if (n0 < 0) return -1;
+    int n1 = use_tc(p) ? tc_forward(p, hy, L, ws, a, save, st) : simt_forward(p, hy, L, ws, a, save, st);
+    if (n1 < 0) return -1;
+    return n0 + n1;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t osdn_workspace_bytes(const osdn_params* p, int need_bwd)
+{
+    if (validate(p) != OSDN_OK) return 0;
+    return make_layout(*p, need_bwd != 0).total;
+}
+
+int osdn_fwd(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+             const float* gate, const float* apf_log_ret, const float* init_state, const float* precond_in,
+             void* out, float* final_state, float* precond_out, void* workspace, size_t workspace_bytes,
+             void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (!q || !k || !v || !beta || !gate || !out || !workspace) return OSDN_INVALID_ARG;
+    if (p->apf_mode == OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, init_state, precond_in, out, final_state,
+                          precond_out};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return OSDN_MISALIGNED;
+    const bool save = (p->flags & OSDN_FLAG_SAVE_RESIDUALS) != 0;
+    const WsLayout L = make_layout(*p, save);
+    if (workspace_bytes < L.total) return OSDN_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(static_cast<char*>(workspace) + L.status, 0, 256, st) != cudaSuccess)
+        return OSDN_CUDA_ERROR;
+    Pointers a{};
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.gate = gate; a.log_ret = apf_log_ret;
+    a.init_state = init_state; a.precond_in = precond_in; a.out = out; a.final_state = final_state;
+    a.precond_out = precond_out;
+    const int n = run_forward(*p, make_hyper(*p), L, workspace, a, save, st);
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = n;
+    return OSDN_OK;
+}
+
+int osdn_bwd(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+             const float* gate, const float* apf_log_ret, const float* init_state, const float* precond_in,
+             const void* dout, const float* dfinal_state, const float* dprecond_out, void* dq, void* dk,
+             void* dv, float* dbeta, float* dgate, float* dapf_log_ret, float* dinit_state,
+             float* dprecond_in, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (!q || !k || !v || !beta || !gate || !dout || !dq || !dk || !dv || !dbeta || !dgate || !workspace)
+        return OSDN_INVALID_ARG;
+    if (p->apf_mode == OSDN_APF_SEPARATE && (!apf_log_ret || !dapf_log_ret)) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, init_state, precond_in, dout, dfinal_state,
+                          dprecond_out, dq, dk, dv, dbeta, dgate, dapf_log_ret, dinit_state, dprecond_in};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return OSDN_MISALIGNED;
+    const WsLayout L = make_layout(*p, true);
+    if (workspace_bytes < L.total) return OSDN_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Hyper hy = make_hyper(*p);
+    Pointers a{};
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.gate = gate; a.log_ret = apf_log_ret;
+    a.init_state = init_state; a.precond_in = precond_in;
+    a.dout = dout; a.dfinal_state = dfinal_state; a.dprecond_out = dprecond_out;
+    a.dq = dq; a.dk = dk; a.dv = dv; a.dbeta = dbeta; a.dgate = dgate; a.dlog_ret = dapf_log_ret;
+    a.dinit_state = dinit_state; a.dprecond_in = dprecond_in;
+    int total = 0;
+    if (!(p->flags & OSDN_FLAG_RESIDUALS_VALID)) {
+        // Recompute the forward residuals; the forward output itself lands in scratch.
+        if (cudaMemsetAsync(static_cast<char*>(workspace) + L.status, 0, 256, st) != cudaSuccess)
+            return OSDN_CUDA_ERROR;
+        Pointers f = a;
+        f.out = static_cast<char*>(workspace) + L.out_scratch;
+        f.final_state = nullptr;
+        f.precond_out = nullptr;
+        const int n = run_forward(*p, hy, L, workspace, f, true, st);
+        if (n < 0) return OSDN_CUDA_ERROR;
+        total += n;
+    }
+    const int n = use_tc(*p) ? tc_backward(*p, hy, L, workspace, a, st) : simt_backward(*p, hy, L, workspace, a, st);
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = total + n;
+    return OSDN_OK;
+}
+
+int osdn_precond_update(const osdn_params* p, const void* k, const float* beta, const float* gate_or_log_ret,
+                        const float* precond_in, void* k_tilde_out, float* precond_out, void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (!k || !beta || !precond_out) return OSDN_INVALID_ARG;
+    if (p->apf_mode != OSDN_APF_NONE && !gate_or_log_ret) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {k, beta, gate_or_log_ret, precond_in, k_tilde_out, precond_out};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    const int n = simt_precond_update(*p, make_hyper(*p), k, beta, gate_or_log_ret, precond_in, k_tilde_out,
+                                      precond_out, static_cast<cudaStream_t>(cuda_stream));
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = n;
+    return OSDN_OK;
+}
+
+// ---- host-buffer convenience --------------------------------------------------------------
+namespace {
+struct Staging {
+    size_t q, k, v, beta, gate, out, dout, dq, dk, dv, dbeta, dgate, ws, total, ws_bytes;
+};
+Staging make_staging(const osdn_params& p, bool bwd)
+{
+    Staging s{};
+    const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
+    const size_t es = p.io_dtype == OSDN_BF16 ? 2 : 4;
+    size_t off = 0;
+    auto take = [&](size_t b) { size_t o = off; off = align_up(off + b, 256); return o; };
+    s.q = take(Ttot * p.H * p.K * es); s.k = take(Ttot * p.H * p.K * es); s.v = take(Ttot * p.H * p.V * es);
+    s.beta = take(Ttot * p.H * 4); s.gate = take(Ttot * p.H * 4); s.out = take(Ttot * p.H * p.V * es);
+    if (bwd) {
+        s.dout = take(Ttot * p.H * p.V * es); s.dq = take(Ttot * p.H * p.K * es);
+        s.dk = take(Ttot * p.H * p.K * es); s.dv = take(Ttot * p.H * p.V * es);
+        s.dbeta = take(Ttot * p.H * 4); s.dgate = take(Ttot * p.H * 4);
+    }
+    s.ws_bytes = make_layout(p, bwd).total;
+    s.ws = take(s.ws_bytes);
+    s.total = off;
+    return s;
+}
+}  // namespace
+
+size_t osdn_host_staging_bytes(const osdn_params* p, int with_bwd)
+{
+    if (validate(p) != OSDN_OK) return 0;
+    return make_staging(*p, with_bwd != 0).total;
+}
+
+int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host, const void* v_host,
+                   const float* beta_host, const float* gate_host, const void* dout_host, void* out_host,
+                   void* dq_host, void* dk_host, void* dv_host, float* dbeta_host, float* dgate_host,
+                   void* staging, size_t staging_bytes, void* cuda_stream)
+{
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    const bool bwd = dout_host != nullptr;
+    if (!q_host || !k_host || !v_host || !beta_host || !gate_host || !out_host || !staging) return OSDN_INVALID_ARG;
+    if (bwd && (!dq_host || !dk_host || !dv_host || !dbeta_host || !dgate_host)) return OSDN_INVALID_ARG;
+    if (p->apf_mode == OSDN_APF_SEPARATE) return OSDN_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(staging) & 255u) return OSDN_MISALIGNED;
+    const Staging s = make_staging(*p, bwd);
+    if (staging_bytes < s.total) return OSDN_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* d = static_cast<char*>(staging);
+    const size_t Ttot = p->nseq > 0 ? (size_t)p->T : (size_t)p->B * p->T;
+    const size_t es = p->io_dtype == OSDN_BF16 ? 2 : 4;
+    const size_t nk = Ttot * p->H * p->K * es, nv = Ttot * p->H * p->V * es, ns = Ttot * p->H * 4;
+    bool ok = true;
+    auto h2d = [&](size_t off, const void* src, size_t n) {
+        ok = ok && cudaMemcpyAsync(d + off, src, n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    };
+    auto d2h = [&](void* dst, size_t off, size_t n) {
+        ok = ok && cudaMemcpyAsync(dst, d + off, n, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    };
+    h2d(s.q, q_host, nk); h2d(s.k, k_host, nk); h2d(s.v, v_host, nv);
+    h2d(s.beta, beta_host, ns); h2d(s.gate, gate_host, ns);
+    if (bwd) h2d(s.dout, dout_host, nv);
+    if (!ok) return OSDN_CUDA_ERROR;
+    osdn_params pp = *p;
+    pp.flags = (p->flags & OSDN_FLAG_FORCE_SIMT) | (bwd ? OSDN_FLAG_SAVE_RESIDUALS : 0);
+    rc = osdn_fwd(&pp, d + s.q, d + s.k, d + s.v, reinterpret_cast<float*>(d + s.beta),
+                  reinterpret_cast<float*>(d + s.gate), nullptr, nullptr, nullptr, d + s.out, nullptr, nullptr,
+                  d + s.ws, s.ws_bytes, cuda_stream);
+    if (rc != OSDN_OK) return rc;
+    int launches = g_last_launches;
+    if (bwd) {
+        pp.flags |= OSDN_FLAG_RESIDUALS_VALID;
+        rc = osdn_bwd(&pp, d + s.q, d + s.k, d + s.v, reinterpret_cast<float*>(d + s.beta),
+                      reinterpret_cast<float*>(d + s.gate), nullptr, nullptr, nullptr, d + s.dout, nullptr,
+                      nullptr, d + s.dq, d + s.dk, d + s.dv, reinterpret_cast<float*>(d + s.dbeta),
+                      reinterpret_cast<float*>(d + s.dgate), nullptr, nullptr, nullptr, d + s.ws, s.ws_bytes,
+                      cuda_stream);
+        if (rc != OSDN_OK) return rc;
+        launches += g_last_launches;
+    }
+    d2h(out_host, s.out, nv);
+    if (bwd) {
+        d2h(dq_host, s.dq, nk); d2h(dk_host, s.dk, nk); d2h(dv_host, s.dv, nv);
+        d2h(dbeta_host, s.dbeta, ns); d2h(dgate_host, s.dgate, ns);
+    }
+    g_last_launches = launches;
+    return ok ? OSDN_OK : OSDN_CUDA_ERROR;
+}
+
+int osdn_read_device_status(const void* workspace, int32_t* status_host)
+{
+    if (!workspace || !status_host) return OSDN_INVALID_ARG;
+    return cudaMemcpy(status_host, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess
+               ? OSDN_OK : OSDN_CUDA_ERROR;
+}
+
+const char* osdn_status_string(int status)
+{
+    switch (status) {
+        case OSDN_OK: return "ok";
+        case OSDN_INVALID_ARG: return "invalid argument";
+        case OSDN_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case OSDN_MISALIGNED: return "pointer not sufficiently aligned";
+        case OSDN_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case OSDN_CUDA_ERROR: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+int osdn_last_launch_count(void) { return g_last_launches; }
+
+}  // extern "C"

@@ -1,0 +1,142 @@
+// Shared declarations of the OSDN CUDA library: workspace layout, chunk table, launch
+// arguments.  Device-side helpers for the two kernel families (CUDA-core fp32 kernels and
+// tcgen05 bf16 kernels) live in their own files.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/osdn.h"
+
+namespace osdn {
+
+constexpr int CH = 64;  // chunk length (tokens)
+
+// Scalar settings broadcast to every kernel.
+struct Hyper {
+    float eta, d_min, d_max, eps, scale;
+    int beta_aware, apf_mode, clamp;
+};
+
+// Sequence / chunk table built on the device from cu_seqlens (or from B, T for dense input).
+// Chunks never straddle sequences; chunk_len < 64 marks a ragged tail; entries beyond the
+// realised chunk count have chunk_len == 0.
+struct Table {
+    int* seq_tok0;    // [S]    first packed token of the sequence
+    int* seq_len;     // [S]
+    int* seq_chunk0;  // [S+1]  first chunk of the sequence; [S] = number of chunks
+    int* chunk_tok0;  // [NTmax]
+    int* chunk_len;   // [NTmax]
+    int* chunk_seq;   // [NTmax]
+};
+
+// Byte offsets of every region inside the caller's workspace.
+struct WsLayout {
+    size_t status;      // int32 device status word (+ padding)
+    size_t table;       // ints, see carve_table
+    size_t ktil;        // [T,H,K]        f32   write keys
+    size_t dbound;      // [NT,H,K]       f32   preconditioner at chunk starts
+    size_t Tm;          // [NT,H,64,64]   f32   UT inverse
+    size_t P;           // [NT,H,64,64]   f32   masked, decayed q.ktil scores
+    size_t W;           // [NT,H,64,K]    f32
+    size_t U;           // [NT,H,64,V]    f32
+    size_t dU;          // [NT,H,64,V]    f32   chunk update (new values)
+    size_t Sn;          // [NT,H,V,K]     f32   state at chunk start
+    // backward only
+    size_t ddU;         // [NT,H,64,V]    f32
+    size_t dSn;         // [NT,H,V,K]     f32   state cotangent at chunk end
+    size_t dktil;       // [T,H,K]        f32
+    size_t dkread;      // [T,H,K]        f32
+    size_t scr;         // [NT,H,5,64,max(K,V)] f32 scratch of the chunk-local backward
+    size_t out_scratch; // [T,H,V]        f32   forward output when the backward recomputes the forward
+    size_t total;
+    int S, NTmax;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline WsLayout make_layout(const osdn_params& p, bool need_bwd)
+{
+    WsLayout L{};
+    const int S = p.nseq > 0 ? p.nseq : p.B;
+    const size_t Ttot = (size_t)(p.nseq > 0 ? p.T : (size_t)p.B * p.T);
+    const int NTmax = p.nseq > 0 ? (int)(Ttot / CH) + S : p.B * ((p.T + CH - 1) / CH);
+    L.S = S;
+    L.NTmax = NTmax;
+    const size_t H = p.H, K = p.K, V = p.V, NT = NTmax;
+    const size_t D = K > V ? K : V;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.status = take(256);
+    L.table = take(sizeof(int) * (3 * (size_t)S + 1 + 3 * NT));
+    L.ktil = take(4 * Ttot * H * K);
+    L.dbound = take(4 * NT * H * K);
+    L.Tm = take(4 * NT * H * CH * CH);
+    L.P = take(4 * NT * H * CH * CH);
+    L.W = take(4 * NT * H * CH * K);
+    L.U = take(4 * NT * H * CH * V);
+    L.dU = take(4 * NT * H * CH * V);
+    L.Sn = take(4 * NT * H * V * K);
+    if (need_bwd) {
+        L.ddU = take(4 * NT * H * CH * V);
+        L.dSn = take(4 * NT * H * V * K);
+        L.dktil = take(4 * Ttot * H * K);
+        L.dkread = take(4 * Ttot * H * K);
+        L.scr = take(4 * NT * H * 5 * CH * D);
+        L.out_scratch = take(4 * Ttot * H * V);
+    }
+    L.total = off;
+    return L;
+}
+
+inline Table carve_table(void* ws, const WsLayout& L)
+{
+    int* base = reinterpret_cast<int*>(static_cast<char*>(ws) + L.table);
+    Table t;
+    t.seq_tok0 = base;
+    t.seq_len = base + L.S;
+    t.seq_chunk0 = base + 2 * L.S;
+    t.chunk_tok0 = base + 3 * L.S + 1;
+    t.chunk_len = t.chunk_tok0 + L.NTmax;
+    t.chunk_seq = t.chunk_len + L.NTmax;
+    return t;
+}
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p);
+template <> __device__ __forceinline__ float ldf<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p)
+{
+    return __bfloat162float(*p);
+}
+template <typename T> __device__ __forceinline__ void stf(T* p, float x);
+template <> __device__ __forceinline__ void stf<float>(float* p, float x) { *p = x; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, float x)
+{
+    *p = __float2bfloat16_rn(x);
+}
+
+// Everything a forward / backward launch sequence needs.
+struct Pointers {
+    const void *q, *k, *v;
+    const float *beta, *gate, *log_ret, *init_state, *precond_in;
+    void* out;
+    float *final_state, *precond_out;
+    // backward
+    const void* dout;
+    const float *dfinal_state, *dprecond_out;
+    void *dq, *dk, *dv;
+    float *dbeta, *dgate, *dlog_ret, *dinit_state, *dprecond_in;
+};
+
+// CUDA-core fp32 kernels (osdn_simt.cu).  Return the number of launches, or -1 on a launch error.
+int simt_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
+                 const Pointers& a, bool save, cudaStream_t st);
+int simt_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
+                  const Pointers& a, cudaStream_t st);
+int simt_precond_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta,
+                        const float* retsrc, const float* precond_in, void* ktil_out,
+                        float* precond_out, cudaStream_t st);
+int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st);
+
+}  // namespace osdn

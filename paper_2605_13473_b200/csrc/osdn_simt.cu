@@ -1,0 +1,937 @@
+// CUDA-core (fp32 FMA) kernels of the OSDN layer.
+//
+// This family is the fp32 mode of the library (fp32 I/O needs better than TF32 accuracy)
+// and the reference-quality path for bf16 I/O when OSDN_FLAG_FORCE_SIMT is set.  Every
+// step of the chunkwise algorithm runs here in fp32:
+//
+//   phase1_fwd      Algorithm 1 with APF and the box projection, one warp per chain
+//   chunk_local_fwd decay-ratio Gram A, UT inverse T, W = T diag(beta gamma) K,
+//                   U = T diag(beta) V, local scores P           (gated chunk form)
+//   chain_fwd       dU = U - W S^T ; O = scale[(gamma Q) S^T + P dU] ;
+//                   S <- gamma_C S + dU^T (rho Ktil)              (state recurrence)
+//   chain_bwd       reverse state chain: ddU, dS
+//   chunk_local_bwd all chunk-local gradients (through P, W, U, T, A and the gate prefix)
+//   phase1_bwd      reverse sweep over the projected affine recurrence (Section 3.5)
+//
+// Notation follows the paper: G_i in-chunk inclusive prefix of the log gate,
+// gamma_i = exp(G_i), Gamma_ij = exp(G_i - G_j), rho_i = exp(G_C - G_i).
+#include "osdn_common.cuh"
+
+namespace osdn {
+
+namespace {
+
+constexpr int NTH = 256;
+
+// ---------------------------------------------------------------------------------------
+// chunk table
+// ---------------------------------------------------------------------------------------
+__global__ void build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Table t)
+{
+    __shared__ int s_total;
+    if (threadIdx.x == 0) {
+        int c = 0;
+        for (int s = 0; s < S; ++s) {
+            int t0 = cu ? cu[s] : s * T_dense;
+            int len = cu ? cu[s + 1] - cu[s] : T_dense;
+            if (len < 0) len = 0;
+            t.seq_tok0[s] = t0;
+            t.seq_len[s] = len;
+            t.seq_chunk0[s] = c < NTmax ? c : NTmax;
+            c += (len + CH - 1) / CH;
+        }
+        if (c > NTmax) c = NTmax;
+        t.seq_chunk0[S] = c;
+        s_total = c;
+    }
+    __syncthreads();
+    for (int s = 0; s < S; ++s) {
+        int c0 = t.seq_chunk0[s], c1 = t.seq_chunk0[s + 1];
+        int t0 = t.seq_tok0[s], len = t.seq_len[s];
+        for (int j = threadIdx.x; j < c1 - c0; j += blockDim.x) {
+            t.chunk_tok0[c0 + j] = t0 + j * CH;
+            int rem = len - j * CH;
+            t.chunk_len[c0 + j] = rem < CH ? rem : CH;
+            t.chunk_seq[c0 + j] = s;
+        }
+    }
+    for (int j = s_total + threadIdx.x; j < NTmax; j += blockDim.x) {
+        t.chunk_tok0[j] = 0;
+        t.chunk_len[j] = 0;
+        t.chunk_seq[j] = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// phase 1 forward: one warp per (sequence, head) chain, lanes own K/32 coordinates each
+// ---------------------------------------------------------------------------------------
+struct P1Args {
+    int S, H, T_dense;
+    const int* cu;           // nullable (dense)
+    const int* seq_chunk0;   // nullable (needed only with dbound)
+    const void* k;
+    const float *beta, *retsrc, *d0;
+    void* ktil;              // nullable
+    float *d_final, *dbound; // nullable
+    Hyper hy;
+};
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+template <typename TI, typename TO, int K>
+__global__ void __launch_bounds__(128) phase1_fwd_kernel(P1Args a)
+{
+    constexpr int R = K / 32;
+    const int lane = threadIdx.x & 31;
+    const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (chain >= a.S * a.H) return;
+    const int s = chain / a.H, h = chain % a.H;
+    const int t0 = a.cu ? a.cu[s] : s * a.T_dense;
+    const int len = a.cu ? max(a.cu[s + 1] - a.cu[s], 0) : a.T_dense;
+    const TI* kp = static_cast<const TI*>(a.k);
+    TO* kt = static_cast<TO*>(a.ktil);
+    float d[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) d[r] = a.d0 ? a.d0[((size_t)s * a.H + h) * K + lane + 32 * r] : 1.0f;
+    const Hyper hy = a.hy;
+    for (int i = 0; i < len; ++i) {
+        const size_t th = (size_t)(t0 + i) * a.H + h;
+        if (a.dbound && (i % CH) == 0) {
+            float* db = a.dbound + ((size_t)(a.seq_chunk0[s] + i / CH) * a.H + h) * K;
+#pragma unroll
+            for (int r = 0; r < R; ++r) db[lane + 32 * r] = d[r];
+        }
+        float kk[R], kap[R], sumk = 0.f, al = 0.f;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            kk[r] = ldf(kp + th * K + lane + 32 * r);
+            kap[r] = kk[r] * kk[r];
+            sumk += kap[r];
+            al += d[r] * kap[r];
+            if (kt) stf(kt + th * K + lane + 32 * r, d[r] * kk[r]);
+        }
+        sumk = warp_sum(sumk);
+        al = warp_sum(al);
+        const float n = fmaxf(sumk, hy.eps);
+        const float b = hy.beta_aware ? a.beta[th] : 1.0f;
+        const float c = hy.eta * b * (1.0f - b * al) / n;
+        const float rho = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            float x = rho * d[r] + c * kap[r];
+            if (hy.clamp) x = fminf(fmaxf(x, hy.d_min), hy.d_max);
+            d[r] = x;
+        }
+    }
+    if (a.d_final) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) a.d_final[((size_t)s * a.H + h) * K + lane + 32 * r] = d[r];
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// CTA-wide small matrix product with operand access through functors:
+//   acc(m, n) = sum_{k < K1} a1(m,k) b1(k,n) + sum_{k < K2} a2(m,k) b2(k,n);  epi(m, n, acc)
+// Thread tiles are TM x TN; columns of a tile are strided by N/TN so that neighbouring
+// threads touch neighbouring columns.
+// ---------------------------------------------------------------------------------------
+template <int M, int N, int TM, int TN, class A1, class B1, class A2, class B2, class E>
+__device__ __forceinline__ void cta_mm2(int K1, A1 a1, B1 b1, int K2, A2 a2, B2 b2, E epi)
+{
+    constexpr int TN_CNT = N / TN, TM_CNT = M / TM;
+    for (int tile = threadIdx.x; tile < TN_CNT * TM_CNT; tile += NTH) {
+        const int tn = tile % TN_CNT, tm = tile / TN_CNT;
+        float acc[TM][TN];
+#pragma unroll
+        for (int i = 0; i < TM; ++i)
+#pragma unroll
+            for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+        for (int k = 0; k < K1; ++k) {
+            float av[TM], bv[TN];
+#pragma unroll
+            for (int i = 0; i < TM; ++i) av[i] = a1(tm * TM + i, k);
+#pragma unroll
+            for (int j = 0; j < TN; ++j) bv[j] = b1(k, tn + j * TN_CNT);
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        for (int k = 0; k < K2; ++k) {
+            float av[TM], bv[TN];
+#pragma unroll
+            for (int i = 0; i < TM; ++i) av[i] = a2(tm * TM + i, k);
+#pragma unroll
+            for (int j = 0; j < TN; ++j) bv[j] = b2(k, tn + j * TN_CNT);
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < TM; ++i)
+#pragma unroll
+            for (int j = 0; j < TN; ++j) epi(tm * TM + i, tn + j * TN_CNT, acc[i][j]);
+    }
+}
+
+struct ZeroOp {
+    __device__ __forceinline__ float operator()(int, int) const { return 0.f; }
+};
+
+template <int M, int N, int TM, int TN, class A1, class B1, class E>
+__device__ __forceinline__ void cta_mm(int K1, A1 a1, B1 b1, E epi)
+{
+    cta_mm2<M, N, TM, TN>(K1, a1, b1, 0, ZeroOp(), ZeroOp(), epi);
+}
+
+// In-chunk gate prefix and the factors derived from it (thread 0 does the 64-term prefix).
+struct GateVecs {
+    float G[CH], gam[CH], rho[CH], beta[CH];
+    float gC;
+};
+
+__device__ __forceinline__ void load_gates(GateVecs& gv, const float* __restrict__ gate,
+                                           const float* __restrict__ beta, int tok0, int len, int H, int h)
+{
+    if (threadIdx.x < CH) {
+        const int i = threadIdx.x;
+        gv.G[i] = i < len ? gate[(size_t)(tok0 + i) * H + h] : 0.f;
+        gv.beta[i] = i < len ? beta[(size_t)(tok0 + i) * H + h] : 0.f;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float acc = 0.f;
+        for (int i = 0; i < CH; ++i) { acc += gv.G[i]; gv.G[i] = acc; }
+        gv.gC = expf(acc);
+    }
+    __syncthreads();
+    if (threadIdx.x < CH) {
+        const int i = threadIdx.x;
+        gv.gam[i] = expf(gv.G[i]);
+        gv.rho[i] = expf(gv.G[CH - 1] - gv.G[i]);
+    }
+    __syncthreads();
+}
+
+// Load a [64 x D] token tile (rows beyond len are zero) from a packed [T,H,D] tensor.
+template <typename T, int D>
+__device__ __forceinline__ void load_tile(float* dst, int ld, const T* __restrict__ src, int tok0, int len,
+                                          int H, int h)
+{
+    for (int e = threadIdx.x; e < CH * D; e += NTH) {
+        const int i = e / D, c = e % D;
+        dst[i * ld + c] = i < len ? ldf(src + ((size_t)(tok0 + i) * H + h) * D + c) : 0.f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// chunk-local forward: A, T = (I + A)^-1, W, U, P
+// ---------------------------------------------------------------------------------------
+struct ChunkArgs {
+    int H;
+    Table tab;
+    const void *q, *k, *v;
+    const float *beta, *gate;
+    const float* ktil;
+    float *Tm, *P, *W, *U;
+    // backward extras
+    const void* dout;
+    const float *Sn, *dSn, *dU, *ddU;
+    float *scr, *dktil, *dkread;
+    void *dq, *dv;
+    float *dbeta, *dgate;
+    Hyper hy;
+};
+
+template <typename T, int K, int V>
+__global__ void __launch_bounds__(NTH) chunk_local_fwd_kernel(ChunkArgs a)
+{
+    extern __shared__ float sm[];
+    constexpr int LD = K + 1, LC = CH + 1;
+    float* sK = sm;
+    float* sKt = sK + CH * LD;
+    float* sQ = sKt + CH * LD;
+    float* sT = sQ + CH * LD;
+    float* sA = sT + CH * LC;
+    __shared__ GateVecs gv;
+
+    const int c = blockIdx.x, h = blockIdx.y, H = a.H;
+    const int len = a.tab.chunk_len[c];
+    if (len == 0) return;
+    const int tok0 = a.tab.chunk_tok0[c];
+    const size_t tile = (size_t)c * H + h;
+
+    load_tile<T, K>(sK, LD, static_cast<const T*>(a.k), tok0, len, H, h);
+    load_tile<float, K>(sKt, LD, a.ktil, tok0, len, H, h);
+    load_tile<T, K>(sQ, LD, static_cast<const T*>(a.q), tok0, len, H, h);
+    load_gates(gv, a.gate, a.beta, tok0, len, H, h);
+
+    // A_ij = 1[j<i] beta_i Gamma_ij <k_i, ktil_j>
+    cta_mm<CH, CH, 4, 4>(
+        K, [&](int m, int k) { return sK[m * LD + k]; }, [&](int k, int n) { return sKt[n * LD + k]; },
+        [&](int i, int j, float acc) {
+            sA[i * LC + j] = j < i ? gv.beta[i] * expf(gv.G[i] - gv.G[j]) * acc : 0.f;
+        });
+    // P_ij = 1[j<=i] Gamma_ij <q_i, ktil_j>
+    float* Pg = a.P + tile * CH * CH;
+    cta_mm<CH, CH, 4, 4>(
+        K, [&](int m, int k) { return sQ[m * LD + k]; }, [&](int k, int n) { return sKt[n * LD + k]; },
+        [&](int i, int j, float acc) { Pg[i * CH + j] = j <= i ? expf(gv.G[i] - gv.G[j]) * acc : 0.f; });
+    __syncthreads();
+
+    // T = (I + A)^-1 by forward substitution; column `col` of T solves (I + A) x = e_col.
+    // Four lanes share a column and split the inner sum.
+    {
+        const int col = threadIdx.x >> 2, part = threadIdx.x & 3;
+        for (int i = 0; i < CH; ++i) {
+            float sum = 0.f;   // empty for i <= col; the shuffles stay outside any divergent branch
+            for (int j = col + part; j < i; j += 4) sum = fmaf(sA[i * LC + j], sT[j * LC + col], sum);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            const float x = i < col ? 0.f : (i == col ? 1.f : -sum);
+            if (part == 0) sT[i * LC + col] = x;
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    float* Tg = a.Tm + tile * CH * CH;
+    for (int e = threadIdx.x; e < CH * CH; e += NTH) Tg[e] = sT[(e / CH) * LC + (e % CH)];
+
+    // W = T diag(beta gamma) K ; U = T diag(beta) V
+    float* Wg = a.W + tile * CH * K;
+    cta_mm<CH, K, 4, K / 16>(
+        CH, [&](int m, int j) { return sT[m * LC + j] * gv.beta[j] * gv.gam[j]; },
+        [&](int j, int n) { return sK[j * LD + n]; }, [&](int m, int n, float acc) { Wg[m * K + n] = acc; });
+    float* Ug = a.U + tile * CH * V;
+    const T* vp = static_cast<const T*>(a.v);
+    cta_mm<CH, V, 4, V / 16>(
+        CH, [&](int m, int j) { return sT[m * LC + j] * gv.beta[j]; },
+        [&](int j, int n) { return j < len ? ldf(vp + ((size_t)(tok0 + j) * H + h) * V + n) : 0.f; },
+        [&](int m, int n, float acc) { Ug[m * V + n] = acc; });
+}
+
+// ---------------------------------------------------------------------------------------
+// state chain, forward.  One CTA per (chain, slice of VS state rows).
+// ---------------------------------------------------------------------------------------
+struct ChainArgs {
+    int S, H;
+    Table tab;
+    const void* q;
+    const float *gate, *beta, *ktil, *W, *U, *P, *init_state;
+    void* out;
+    float *final_state, *Sn, *dU;
+    int save;
+    // backward
+    const void* dout;
+    const float* dfinal_state;
+    float *ddU, *dSn, *dinit_state;
+    Hyper hy;
+};
+
+template <typename T, int K, int V, int VS>
+__global__ void __launch_bounds__(NTH) chain_fwd_kernel(ChainArgs a)
+{
+    extern __shared__ float sm[];
+    constexpr int LD = K + 1, LC = CH + 1, LV = VS + 1;
+    float* sS = sm;                 // [VS][LD]
+    float* sW = sS + VS * LD;       // [64][LD]
+    float* sKt = sW + CH * LD;
+    float* sQ = sKt + CH * LD;
+    float* sP = sQ + CH * LD;       // [64][LC]
+    float* sU = sP + CH * LC;       // [64][LV]  U slice, then dU
+    float* sO = sU + CH * LV;       // [64][LV]
+    __shared__ GateVecs gv;
+
+    const int chain = blockIdx.x, H = a.H;
+    const int s = chain / H, h = chain % H;
+    const int v0 = blockIdx.y * VS;
+    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const float scale = a.hy.scale;
+
+    for (int e = threadIdx.x; e < VS * K; e += NTH) {
+        const int r = e / K, k = e % K;
+        sS[r * LD + k] = a.init_state ? a.init_state[(((size_t)s * H + h) * V + v0 + r) * K + k] : 0.f;
+    }
+    T* outp = static_cast<T*>(a.out);
+    for (int c = c0; c < c1; ++c) {
+        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+        const size_t tile = (size_t)c * H + h;
+        __syncthreads();
+        for (int e = threadIdx.x; e < CH * K; e += NTH) sW[(e / K) * LD + e % K] = a.W[tile * CH * K + e];
+        load_tile<float, K>(sKt, LD, a.ktil, tok0, len, H, h);
+        load_tile<T, K>(sQ, LD, static_cast<const T*>(a.q), tok0, len, H, h);
+        for (int e = threadIdx.x; e < CH * CH; e += NTH) sP[(e / CH) * LC + e % CH] = a.P[tile * CH * CH + e];
+        for (int e = threadIdx.x; e < CH * VS; e += NTH)
+            sU[(e / VS) * LV + e % VS] = a.U[tile * CH * V + (size_t)(e / VS) * V + v0 + e % VS];
+        if (a.save)
+            for (int e = threadIdx.x; e < VS * K; e += NTH)
+                a.Sn[(tile * V + v0 + e / K) * K + e % K] = sS[(e / K) * LD + e % K];
+        load_gates(gv, a.gate, a.beta, tok0, len, H, h);
+
+        // dU = U - W S^T
+        cta_mm<CH, VS, 2, VS / 8>(
+            K, [&](int m, int k) { return sW[m * LD + k]; }, [&](int k, int n) { return sS[n * LD + k]; },
+            [&](int m, int n, float acc) { sU[m * LV + n] -= acc; });
+        __syncthreads();
+        if (a.save)
+            for (int e = threadIdx.x; e < CH * VS; e += NTH)
+                a.dU[tile * CH * V + (size_t)(e / VS) * V + v0 + e % VS] = sU[(e / VS) * LV + e % VS];
+        // O = scale [ (gamma Q) S^T + P dU ]
+        cta_mm2<CH, VS, 2, VS / 8>(
+            K, [&](int m, int k) { return gv.gam[m] * sQ[m * LD + k]; },
+            [&](int k, int n) { return sS[n * LD + k]; }, CH, [&](int m, int j) { return sP[m * LC + j]; },
+            [&](int j, int n) { return sU[j * LV + n]; },
+            [&](int m, int n, float acc) { sO[m * LV + n] = scale * acc; });
+        __syncthreads();
+        for (int e = threadIdx.x; e < CH * VS; e += NTH) {
+            const int i = e / VS, n = e % VS;
+            if (i < len) stf(outp + ((size_t)(tok0 + i) * H + h) * V + v0 + n, sO[i * LV + n]);
+        }
+        // S <- gamma_C S + dU^T (rho Ktil)
+        cta_mm<VS, K, 2, K / 16>(
+            CH, [&](int m, int i) { return sU[i * LV + m]; },
+            [&](int i, int n) { return gv.rho[i] * sKt[i * LD + n]; },
+            [&](int m, int n, float acc) { sS[m * LD + n] = gv.gC * sS[m * LD + n] + acc; });
+    }
+    __syncthreads();
+    if (a.final_state)
+        for (int e = threadIdx.x; e < VS * K; e += NTH)
+            a.final_state[(((size_t)s * H + h) * V + v0 + e / K) * K + e % K] = sS[(e / K) * LD + e % K];
+}
+
+// ---------------------------------------------------------------------------------------
+// state chain, backward (reverse over chunks)
+//   ddU = scale P^T dO + (rho Ktil) dS^T ;  dS <- gamma_C dS + scale dO^T (gamma Q) - ddU^T W
+// ---------------------------------------------------------------------------------------
+template <typename T, int K, int V, int VS>
+__global__ void __launch_bounds__(NTH) chain_bwd_kernel(ChainArgs a)
+{
+    extern __shared__ float sm[];
+    constexpr int LD = K + 1, LC = CH + 1, LV = VS + 1;
+    float* sdS = sm;                // [VS][LD]
+    float* sW = sdS + VS * LD;
+    float* sKt = sW + CH * LD;
+    float* sQ = sKt + CH * LD;
+    float* sP = sQ + CH * LD;       // [64][LC]
+    float* sdO = sP + CH * LC;      // [64][LV]
+    float* sddU = sdO + CH * LV;    // [64][LV]
+    __shared__ GateVecs gv;
+
+    const int chain = blockIdx.x, H = a.H;
+    const int s = chain / H, h = chain % H;
+    const int v0 = blockIdx.y * VS;
+    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const float scale = a.hy.scale;
+
+    for (int e = threadIdx.x; e < VS * K; e += NTH) {
+        const int r = e / K, k = e % K;
+        sdS[r * LD + k] = a.dfinal_state ? a.dfinal_state[(((size_t)s * H + h) * V + v0 + r) * K + k] : 0.f;
+    }
+    const T* dop = static_cast<const T*>(a.dout);
+    for (int c = c1 - 1; c >= c0; --c) {
+        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+        const size_t tile = (size_t)c * H + h;
+        __syncthreads();
+        for (int e = threadIdx.x; e < CH * K; e += NTH) sW[(e / K) * LD + e % K] = a.W[tile * CH * K + e];
+        load_tile<float, K>(sKt, LD, a.ktil, tok0, len, H, h);
+        load_tile<T, K>(sQ, LD, static_cast<const T*>(a.q), tok0, len, H, h);
+        for (int e = threadIdx.x; e < CH * CH; e += NTH) sP[(e / CH) * LC + e % CH] = a.P[tile * CH * CH + e];
+        for (int e = threadIdx.x; e < CH * VS; e += NTH) {
+            const int i = e / VS, n = e % VS;
+            sdO[i * LV + n] = i < len ? ldf(dop + ((size_t)(tok0 + i) * H + h) * V + v0 + n) : 0.f;
+        }
+        for (int e = threadIdx.x; e < VS * K; e += NTH)
+            a.dSn[(tile * V + v0 + e / K) * K + e % K] = sdS[(e / K) * LD + e % K];
+        load_gates(gv, a.gate, a.beta, tok0, len, H, h);
+
+        cta_mm2<CH, VS, 2, VS / 8>(
+            CH, [&](int i, int j) { return scale * sP[j * LC + i]; }, [&](int j, int n) { return sdO[j * LV + n]; },
+            K, [&](int i, int k) { return gv.rho[i] * sKt[i * LD + k]; },
+            [&](int k, int n) { return sdS[n * LD + k]; },
+            [&](int i, int n, float acc) { sddU[i * LV + n] = acc; });
+        __syncthreads();
+        for (int e = threadIdx.x; e < CH * VS; e += NTH)
+            a.ddU[tile * CH * V + (size_t)(e / VS) * V + v0 + e % VS] = sddU[(e / VS) * LV + e % VS];
+        cta_mm2<VS, K, 2, K / 16>(
+            CH, [&](int m, int i) { return scale * sdO[i * LV + m]; },
+            [&](int i, int n) { return gv.gam[i] * sQ[i * LD + n]; }, CH,
+            [&](int m, int i) { return -sddU[i * LV + m]; }, [&](int i, int n) { return sW[i * LD + n]; },
+            [&](int m, int n, float acc) { sdS[m * LD + n] = gv.gC * sdS[m * LD + n] + acc; });
+    }
+    __syncthreads();
+    if (a.dinit_state)
+        for (int e = threadIdx.x; e < VS * K; e += NTH)
+            a.dinit_state[(((size_t)s * H + h) * V + v0 + e / K) * K + e % K] = sdS[(e / K) * LD + e % K];
+}
+
+// ---------------------------------------------------------------------------------------
+// chunk-local backward: gradients through P, the state-advance factors, W, U, T, A, gates
+// ---------------------------------------------------------------------------------------
+template <typename T, int K, int V>
+__global__ void __launch_bounds__(NTH) chunk_local_bwd_kernel(ChunkArgs a)
+{
+    extern __shared__ float sm[];
+    constexpr int LD = K + 1, LC = CH + 1;
+    constexpr int D = K > V ? K : V;
+    float* sK = sm;
+    float* sKt = sK + CH * LD;
+    float* sQ = sKt + CH * LD;
+    float* sT = sQ + CH * LD;       // [64][LC]
+    float* sX = sT + CH * LC;       // dT, later dA * beta_i * Gamma_ij
+    float* sY = sX + CH * LC;       // scratch
+    float* sDP = sY + CH * LC;      // dP * Gamma
+    __shared__ GateVecs gv;
+    __shared__ float sdG[CH], sdB[CH], sR[CH], sRed[NTH / 32];
+
+    const int c = blockIdx.x, h = blockIdx.y, H = a.H;
+    const int len = a.tab.chunk_len[c];
+    if (len == 0) return;
+    const int tok0 = a.tab.chunk_tok0[c];
+    const size_t tile = (size_t)c * H + h;
+    const float scale = a.hy.scale;
+
+    const T* vp = static_cast<const T*>(a.v);
+    const T* dop = static_cast<const T*>(a.dout);
+    const float* Sg = a.Sn + tile * V * K;
+    const float* dSg = a.dSn + tile * V * K;
+    const float* dUg = a.dU + tile * CH * V;
+    const float* ddUg = a.ddU + tile * CH * V;
+    const float* Pg = a.P + tile * CH * CH;
+    float* scr = a.scr + tile * 5 * CH * D;
+    float* gdQ = scr;                 // gamma_i * dQg
+    float* gdKt = scr + CH * D;       // rho_j * dKtr
+    float* gdW = scr + 2 * CH * D;
+    float* gdK = scr + 3 * CH * D;    // beta gamma dKb
+    auto vld = [&](int j, int n) { return j < len ? ldf(vp + ((size_t)(tok0 + j) * H + h) * V + n) : 0.f; };
+    auto dold = [&](int i, int n) { return i < len ? ldf(dop + ((size_t)(tok0 + i) * H + h) * V + n) : 0.f; };
+
+    load_tile<T, K>(sK, LD, static_cast<const T*>(a.k), tok0, len, H, h);
+    load_tile<float, K>(sKt, LD, a.ktil, tok0, len, H, h);
+    load_tile<T, K>(sQ, LD, static_cast<const T*>(a.q), tok0, len, H, h);
+    for (int e = threadIdx.x; e < CH * CH; e += NTH) sT[(e / CH) * LC + e % CH] = a.Tm[tile * CH * CH + e];
+    if (threadIdx.x < CH) { sdG[threadIdx.x] = 0.f; sdB[threadIdx.x] = 0.f; sR[threadIdx.x] = 0.f; }
+    load_gates(gv, a.gate, a.beta, tok0, len, H, h);
+
+    // <dS, S>_F (for the gradient of the chunk-level decay gamma_C)
+    {
+        float part = 0.f;
+        for (int e = threadIdx.x; e < V * K; e += NTH) part = fmaf(Sg[e], dSg[e], part);
+        part = warp_sum(part);
+        if ((threadIdx.x & 31) == 0) sRed[threadIdx.x >> 5] = part;
+    }
+
+    // (1) dP = 1[j<=i] scale dO dU^T ;  sDP = dP * Gamma ;  sY = dP * P
+    cta_mm<CH, CH, 4, 4>(
+        V, [&](int i, int n) { return scale * dold(i, n); }, [&](int n, int j) { return dUg[j * V + n]; },
+        [&](int i, int j, float acc) {
+            const float dp = j <= i ? acc : 0.f;
+            sDP[i * LC + j] = dp * expf(fminf(gv.G[i] - gv.G[j], 0.f));
+            sY[i * LC + j] = dp * Pg[i * CH + j];
+        });
+    __syncthreads();
+    if (threadIdx.x < CH) {
+        const int i = threadIdx.x;
+        float r = 0.f, cs = 0.f;
+        for (int j = 0; j < CH; ++j) { r += sY[i * LC + j]; cs += sY[j * LC + i]; }
+        sdG[i] += r - cs;   // only this thread touches sdG[i] here
+    }
+    __syncthreads();
+
+    // (2) gamma_i * dQg = gamma_i scale dO S ; dq = that + (dP Gamma) Ktil
+    cta_mm<CH, K, 4, K / 16>(
+        V, [&](int i, int n) { return scale * gv.gam[i] * dold(i, n); }, [&](int n, int k) { return Sg[n * K + k]; },
+        [&](int i, int k, float acc) {
+            gdQ[i * K + k] = acc;
+            atomicAdd(&sdG[i], acc * sQ[i * LD + k]);
+        });
+    T* dqp = static_cast<T*>(a.dq);
+    cta_mm<CH, K, 4, K / 16>(
+        CH, [&](int i, int j) { return sDP[i * LC + j]; }, [&](int j, int k) { return sKt[j * LD + k]; },
+        [&](int i, int k, float acc) {
+            if (i < len) stf(dqp + ((size_t)(tok0 + i) * H + h) * K + k, gdQ[i * K + k] + acc);
+        });
+
+    // (3) rho_j * dKtr = rho_j dU dS ; r_j = <rho_j dKtr_j, ktil_j>
+    cta_mm<CH, K, 4, K / 16>(
+        V, [&](int j, int n) { return gv.rho[j] * dUg[j * V + n]; }, [&](int n, int k) { return dSg[n * K + k]; },
+        [&](int j, int k, float acc) {
+            gdKt[j * K + k] = acc;
+            atomicAdd(&sR[j], acc * sKt[j * LD + k]);
+        });
+
+    // (4) dW = -ddU S
+    cta_mm<CH, K, 4, K / 16>(
+        V, [&](int i, int n) { return -ddUg[i * V + n]; }, [&](int n, int k) { return Sg[n * K + k]; },
+        [&](int i, int k, float acc) { gdW[i * K + k] = acc; });
+    __syncthreads();
+    //     dT = dW Kb^T + ddU Vb^T
+    cta_mm2<CH, CH, 4, 4>(
+        K, [&](int i, int k) { return gdW[i * K + k]; },
+        [&](int k, int j) { return gv.beta[j] * gv.gam[j] * sK[j * LD + k]; }, V,
+        [&](int i, int n) { return ddUg[i * V + n]; }, [&](int n, int j) { return gv.beta[j] * vld(j, n); },
+        [&](int i, int j, float acc) { sX[i * LC + j] = acc; });
+
+    // (5) dKb = T^T dW ; dVb = T^T ddU
+    cta_mm<CH, K, 4, K / 16>(
+        CH, [&](int j, int i) { return sT[i * LC + j]; }, [&](int i, int k) { return gdW[i * K + k]; },
+        [&](int j, int k, float acc) {
+            const float gk = gv.gam[j] * sK[j * LD + k];
+            gdK[j * K + k] = gv.beta[j] * gv.gam[j] * acc;
+            atomicAdd(&sdB[j], acc * gk);
+            atomicAdd(&sdG[j], acc * gv.beta[j] * gk);
+        });
+    T* dvp = static_cast<T*>(a.dv);
+    cta_mm<CH, V, 4, V / 16>(
+        CH, [&](int j, int i) { return sT[i * LC + j]; }, [&](int i, int n) { return ddUg[i * V + n]; },
+        [&](int j, int n, float acc) {
+            if (j < len) stf(dvp + ((size_t)(tok0 + j) * H + h) * V + n, gv.beta[j] * acc);
+            atomicAdd(&sdB[j], acc * vld(j, n));
+        });
+    __syncthreads();
+
+    // (6) dA = -strictLower(T^T dT T^T)
+    cta_mm<CH, CH, 4, 4>(
+        CH, [&](int x, int i) { return sT[i * LC + x]; }, [&](int i, int y) { return sX[i * LC + y]; },
+        [&](int x, int y, float acc) { sY[x * LC + y] = acc; });
+    __syncthreads();
+    cta_mm<CH, CH, 4, 4>(
+        CH, [&](int x, int z) { return sY[x * LC + z]; }, [&](int z, int y) { return sT[y * LC + z]; },
+        [&](int x, int y, float acc) { sX[x * LC + y] = y < x ? -acc : 0.f; });
+    __syncthreads();
+    //     raw Gram once more: dbeta_i += dA_ij Gamma_ij <k_i,ktil_j>; dG from dA (.) A; sX <- dA beta_i Gamma_ij
+    cta_mm<CH, CH, 4, 4>(
+        K, [&](int i, int k) { return sK[i * LD + k]; }, [&](int k, int j) { return sKt[j * LD + k]; },
+        [&](int i, int j, float raw) {
+            const float da = sX[i * LC + j];
+            const float gm = j < i ? expf(gv.G[i] - gv.G[j]) : 0.f;
+            const float t = da * gm * raw;
+            if (j < i) {
+                atomicAdd(&sdB[i], t);
+                atomicAdd(&sdG[i], t * gv.beta[i]);
+                atomicAdd(&sdG[j], -t * gv.beta[i]);
+            }
+            sX[i * LC + j] = da * gv.beta[i] * gm;
+        });
+    __syncthreads();
+
+    // (7) dk (read side) and dktil
+    float* dkr = a.dkread;
+    cta_mm<CH, K, 4, K / 16>(
+        CH, [&](int i, int j) { return sX[i * LC + j]; }, [&](int j, int k) { return sKt[j * LD + k]; },
+        [&](int i, int k, float acc) {
+            if (i < len) dkr[((size_t)(tok0 + i) * H + h) * K + k] = gdK[i * K + k] + acc;
+        });
+    float* dkt = a.dktil;
+    cta_mm2<CH, K, 4, K / 16>(
+        CH, [&](int j, int i) { return sDP[i * LC + j]; }, [&](int i, int k) { return sQ[i * LD + k]; }, CH,
+        [&](int j, int i) { return sX[i * LC + j]; }, [&](int i, int k) { return sK[i * LD + k]; },
+        [&](int j, int k, float acc) {
+            if (j < len) dkt[((size_t)(tok0 + j) * H + h) * K + k] = gdKt[j * K + k] + acc;
+        });
+    __syncthreads();
+
+    // (8) gate gradients: reverse in-chunk prefix of dG; phase-2 part of dbeta
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < NTH / 32; ++w) tot += sRed[w];
+        float rsum = 0.f;
+        for (int j = 0; j < CH; ++j) { rsum += sR[j]; sdG[j] -= sR[j]; }
+        sdG[CH - 1] += rsum + gv.gC * tot;
+        float acc = 0.f;
+        for (int i = CH - 1; i >= 0; --i) { acc += sdG[i]; sdG[i] = acc; }
+    }
+    __syncthreads();
+    if (threadIdx.x < len) {
+        const size_t th = (size_t)(tok0 + threadIdx.x) * H + h;
+        a.dgate[th] = sdG[threadIdx.x];
+        a.dbeta[th] = sdB[threadIdx.x];
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// phase 1 backward: reverse sweep over the projected affine recurrence, one warp per chain.
+// Per chunk the forward scan is replayed from the saved chunk-start d.
+// ---------------------------------------------------------------------------------------
+struct P1BwdArgs {
+    int S, H;
+    Table tab;
+    const void* k;
+    const float *beta, *retsrc, *dbound, *dktil, *dkread, *dprecond_out;
+    void* dk;
+    float *dbeta, *dgate, *dlog_ret, *dprecond_in;
+    Hyper hy;
+};
+
+template <typename T, int K>
+__global__ void __launch_bounds__(64) phase1_bwd_kernel(P1BwdArgs a)
+{
+    constexpr int R = K / 32;
+    extern __shared__ float sm[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* sd = sm + (size_t)warp * (CH * K + 4 * CH);   // d_t for the chunk [64][K]
+    float* sc = sd + CH * K;                              // c_t
+    float* sa = sc + CH;                                  // <d_t, kap_t>
+    float* sn = sa + CH;                                  // n_t (negative when the floor eps is active)
+    float* srho = sn + CH;
+    const int chain = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (chain >= a.S * a.H) return;
+    const int s = chain / a.H, h = chain % a.H, H = a.H;
+    const Hyper hy = a.hy;
+    const T* kp = static_cast<const T*>(a.k);
+    T* dkp = static_cast<T*>(a.dk);
+    float lam[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+        lam[r] = a.dprecond_out ? a.dprecond_out[((size_t)s * H + h) * K + lane + 32 * r] : 0.f;
+    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    for (int c = c1 - 1; c >= c0; --c) {
+        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+        float d[R];
+        unsigned long long mb[R];  // bit i: the projection passes gradient at token i
+#pragma unroll
+        for (int r = 0; r < R; ++r) d[r] = a.dbound[((size_t)c * H + h) * K + lane + 32 * r];
+#pragma unroll
+        for (int r = 0; r < R; ++r) mb[r] = 0ull;
+        for (int i = 0; i < len; ++i) {
+            const size_t th = (size_t)(tok0 + i) * H + h;
+            float kap[R], sumk = 0.f, al = 0.f;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float kk = ldf(kp + th * K + lane + 32 * r);
+                kap[r] = kk * kk;
+                sumk += kap[r];
+                al += d[r] * kap[r];
+                sd[i * K + lane + 32 * r] = d[r];
+            }
+            sumk = warp_sum(sumk);
+            al = warp_sum(al);
+            const float n = fmaxf(sumk, hy.eps);
+            const float b = hy.beta_aware ? a.beta[th] : 1.0f;
+            const float cc = hy.eta * b * (1.0f - b * al) / n;
+            const float rho = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
+            if (lane == 0) { sc[i] = cc; sa[i] = al; sn[i] = sumk > hy.eps ? n : -n; srho[i] = rho; }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float x = rho * d[r] + cc * kap[r];
+                bool pass = true;
+                if (hy.clamp) {
+                    pass = (x >= hy.d_min) && (x <= hy.d_max);
+                    x = fminf(fmaxf(x, hy.d_min), hy.d_max);
+                }
+                if (pass) mb[r] |= 1ull << i;
+                d[r] = x;
+            }
+        }
+        __syncwarp();
+        for (int i = len - 1; i >= 0; --i) {
+            const size_t th = (size_t)(tok0 + i) * H + h;
+            float kk[R], kap[R], dt[R], dkt[R], drho = 0.f, dc = 0.f;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                kk[r] = ldf(kp + th * K + lane + 32 * r);
+                kap[r] = kk[r] * kk[r];
+                dt[r] = sd[i * K + lane + 32 * r];
+                dkt[r] = a.dktil[th * K + lane + 32 * r];
+                if (!((mb[r] >> i) & 1ull)) lam[r] = 0.f;
+                drho += lam[r] * dt[r];
+                dc += lam[r] * kap[r];
+            }
+            drho = warp_sum(drho);
+            dc = warp_sum(dc);
+            const float nn = sn[i], n = fabsf(nn), cc = sc[i], al = sa[i], rho = srho[i];
+            const float b = hy.beta_aware ? a.beta[th] : 1.0f;
+            const float da = -hy.eta * b * b / n * dc;
+            const float db = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
+            const float dn = nn > 0.f ? -cc / n * dc : 0.f;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float dkap = cc * lam[r] + da * dt[r] + dn;
+                const float dkv = a.dkread[th * K + lane + 32 * r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
+                stf(dkp + th * K + lane + 32 * r, dkv);
+                lam[r] = rho * lam[r] + da * kap[r] + kk[r] * dkt[r];
+            }
+            if (lane == 0) {
+                if (hy.beta_aware) a.dbeta[th] += db;
+                if (hy.apf_mode == 1) a.dgate[th] += rho * drho;
+                if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
+            }
+        }
+        __syncwarp();
+    }
+    if (a.dprecond_in) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) a.dprecond_in[((size_t)s * H + h) * K + lane + 32 * r] = lam[r];
+    }
+}
+
+template <typename F> bool set_smem(F* kernel, size_t bytes)
+{
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
+constexpr int VSL = 32;  // state rows per chain CTA
+
+template <typename T, int K, int V>
+int fwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+             bool save, cudaStream_t st)
+{
+    char* w = static_cast<char*>(ws);
+    Table tab = carve_table(ws, L);
+    int launches = 0;
+    const int S = L.S, H = p.H;
+    {
+        P1Args pa{};
+        pa.S = S; pa.H = H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
+        pa.seq_chunk0 = tab.seq_chunk0;
+        pa.k = a.k; pa.beta = a.beta;
+        pa.retsrc = p.apf_mode == 2 ? a.log_ret : a.gate;
+        pa.d0 = a.precond_in; pa.ktil = w + L.ktil; pa.d_final = a.precond_out;
+        pa.dbound = reinterpret_cast<float*>(w + L.dbound);
+        pa.hy = hy;
+        const int chains = S * H;
+        phase1_fwd_kernel<T, float, K><<<(chains + 3) / 4, 128, 0, st>>>(pa);
+        ++launches;
+    }
+    {
+        ChunkArgs ca{};
+        ca.H = H; ca.tab = tab; ca.q = a.q; ca.k = a.k; ca.v = a.v; ca.beta = a.beta; ca.gate = a.gate;
+        ca.ktil = reinterpret_cast<float*>(w + L.ktil);
+        ca.Tm = reinterpret_cast<float*>(w + L.Tm); ca.P = reinterpret_cast<float*>(w + L.P);
+        ca.W = reinterpret_cast<float*>(w + L.W); ca.U = reinterpret_cast<float*>(w + L.U);
+        ca.hy = hy;
+        const size_t smem = sizeof(float) * (3 * CH * (K + 1) + 2 * CH * (CH + 1));
+        if (!set_smem(chunk_local_fwd_kernel<T, K, V>, smem)) return -1;
+        chunk_local_fwd_kernel<T, K, V><<<dim3(L.NTmax, H), NTH, smem, st>>>(ca);
+        ++launches;
+    }
+    {
+        ChainArgs ch{};
+        ch.S = S; ch.H = H; ch.tab = tab; ch.q = a.q; ch.gate = a.gate; ch.beta = a.beta;
+        ch.ktil = reinterpret_cast<float*>(w + L.ktil);
+        ch.W = reinterpret_cast<float*>(w + L.W); ch.U = reinterpret_cast<float*>(w + L.U);
+        ch.P = reinterpret_cast<float*>(w + L.P);
+        ch.init_state = a.init_state; ch.out = a.out; ch.final_state = a.final_state;
+        ch.Sn = reinterpret_cast<float*>(w + L.Sn); ch.dU = reinterpret_cast<float*>(w + L.dU);
+        ch.save = save ? 1 : 0; ch.hy = hy;
+        const size_t smem = sizeof(float) * (VSL * (K + 1) + 3 * CH * (K + 1) + CH * (CH + 1) + 2 * CH * (VSL + 1));
+        if (!set_smem(chain_fwd_kernel<T, K, V, VSL>, smem)) return -1;
+        chain_fwd_kernel<T, K, V, VSL><<<dim3(S * H, V / VSL), NTH, smem, st>>>(ch);
+        ++launches;
+    }
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+template <typename T, int K, int V>
+int bwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+             cudaStream_t st)
+{
+    char* w = static_cast<char*>(ws);
+    Table tab = carve_table(ws, L);
+    int launches = 0;
+    const int S = L.S, H = p.H;
+    auto F = [&](size_t off) { return reinterpret_cast<float*>(w + off); };
+    {
+        ChainArgs ch{};
+        ch.S = S; ch.H = H; ch.tab = tab; ch.q = a.q; ch.gate = a.gate; ch.beta = a.beta;
+        ch.ktil = F(L.ktil); ch.W = F(L.W); ch.P = F(L.P);
+        ch.dout = a.dout; ch.dfinal_state = a.dfinal_state; ch.ddU = F(L.ddU); ch.dSn = F(L.dSn);
+        ch.dinit_state = a.dinit_state; ch.hy = hy;
+        const size_t smem = sizeof(float) * (VSL * (K + 1) + 3 * CH * (K + 1) + CH * (CH + 1) + 2 * CH * (VSL + 1));
+        if (!set_smem(chain_bwd_kernel<T, K, V, VSL>, smem)) return -1;
+        chain_bwd_kernel<T, K, V, VSL><<<dim3(S * H, V / VSL), NTH, smem, st>>>(ch);
+        ++launches;
+    }
+    {
+        ChunkArgs ca{};
+        ca.H = H; ca.tab = tab; ca.q = a.q; ca.k = a.k; ca.v = a.v; ca.beta = a.beta; ca.gate = a.gate;
+        ca.ktil = F(L.ktil); ca.Tm = F(L.Tm); ca.P = F(L.P); ca.W = F(L.W); ca.U = F(L.U);
+        ca.dout = a.dout; ca.Sn = F(L.Sn); ca.dSn = F(L.dSn); ca.dU = F(L.dU); ca.ddU = F(L.ddU);
+        ca.scr = F(L.scr); ca.dktil = F(L.dktil); ca.dkread = F(L.dkread);
+        ca.dq = a.dq; ca.dv = a.dv; ca.dbeta = a.dbeta; ca.dgate = a.dgate; ca.hy = hy;
+        const size_t smem = sizeof(float) * (3 * CH * (K + 1) + 4 * CH * (CH + 1));
+        if (!set_smem(chunk_local_bwd_kernel<T, K, V>, smem)) return -1;
+        chunk_local_bwd_kernel<T, K, V><<<dim3(L.NTmax, H), NTH, smem, st>>>(ca);
+        ++launches;
+    }
+    {
+        P1BwdArgs pb{};
+        pb.S = S; pb.H = H; pb.tab = tab; pb.k = a.k; pb.beta = a.beta;
+        pb.retsrc = p.apf_mode == 2 ? a.log_ret : a.gate;
+        pb.dbound = F(L.dbound); pb.dktil = F(L.dktil); pb.dkread = F(L.dkread);
+        pb.dprecond_out = a.dprecond_out; pb.dk = a.dk; pb.dbeta = a.dbeta; pb.dgate = a.dgate;
+        pb.dlog_ret = a.dlog_ret; pb.dprecond_in = a.dprecond_in; pb.hy = hy;
+        const size_t smem = sizeof(float) * 2 * (CH * K + 4 * CH);
+        if (!set_smem(phase1_bwd_kernel<T, K>, smem)) return -1;
+        const int chains = S * H;
+        phase1_bwd_kernel<T, K><<<(chains + 1) / 2, 64, smem, st>>>(pb);
+        ++launches;
+    }
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+template <typename TI, typename TO>
+int p1_dispatch(int K, const P1Args& pa, cudaStream_t st)
+{
+    const int chains = pa.S * pa.H;
+    if (K == 64) phase1_fwd_kernel<TI, TO, 64><<<(chains + 3) / 4, 128, 0, st>>>(pa);
+    else phase1_fwd_kernel<TI, TO, 128><<<(chains + 3) / 4, 128, 0, st>>>(pa);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace
+
+int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st)
+{
+    Table tab = carve_table(ws, L);
+    build_table_kernel<<<1, 256, 0, st>>>(L.S, p.T, p.nseq > 0 ? p.cu_seqlens : nullptr, L.NTmax, tab);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+#define OSDN_DISPATCH(FN, ...)                                                              \
+    do {                                                                                    \
+        if (p.io_dtype == OSDN_FP32) {                                                      \
+            if (p.K == 64 && p.V == 64) return FN<float, 64, 64>(__VA_ARGS__);              \
+            if (p.K == 128 && p.V == 128) return FN<float, 128, 128>(__VA_ARGS__);          \
+            if (p.K == 64 && p.V == 128) return FN<float, 64, 128>(__VA_ARGS__);            \
+            if (p.K == 128 && p.V == 64) return FN<float, 128, 64>(__VA_ARGS__);            \
+        } else {                                                                            \
+            if (p.K == 64 && p.V == 64) return FN<__nv_bfloat16, 64, 64>(__VA_ARGS__);      \
+            if (p.K == 128 && p.V == 128) return FN<__nv_bfloat16, 128, 128>(__VA_ARGS__);  \
+            if (p.K == 64 && p.V == 128) return FN<__nv_bfloat16, 64, 128>(__VA_ARGS__);    \
+            if (p.K == 128 && p.V == 64) return FN<__nv_bfloat16, 128, 64>(__VA_ARGS__);    \
+        }                                                                                   \
+        return -1;                                                                          \
+    } while (0)
+
+int simt_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                 bool save, cudaStream_t st)
+{
+    OSDN_DISPATCH(fwd_impl, p, hy, L, ws, a, save, st);
+}
+
+int simt_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                  cudaStream_t st)
+{
+    OSDN_DISPATCH(bwd_impl, p, hy, L, ws, a, st);
+}
+
+int simt_precond_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta,
+                        const float* retsrc, const float* precond_in, void* ktil_out, float* precond_out,
+                        cudaStream_t st)
+{
+    P1Args pa{};
+    pa.S = p.nseq > 0 ? p.nseq : p.B;
+    pa.H = p.H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
+    pa.k = k; pa.beta = beta; pa.retsrc = retsrc; pa.d0 = precond_in; pa.ktil = ktil_out;
+    pa.d_final = precond_out; pa.hy = hy;
+    if (p.io_dtype == OSDN_FP32) return p1_dispatch<float, float>(p.K, pa, st);
+    return p1_dispatch<__nv_bfloat16, __nv_bfloat16>(p.K, pa, st);
+}
+
+}  // namespace osdn

@@ -1,0 +1,152 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by element."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from paper_2605_13473_b200 import binding, run_inputs_bwd, run_inputs_fwd
+from paper_2605_13473_b200.synth import OsdnHyper, config, draw, lively
+
+pytestmark = pytest.mark.gpu
+
+REPORT = {}
+
+
+def teardown_module(module):
+    out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
+    try:
+        os.makedirs(out, exist_ok=True)
+        with open(os.path.join(out, "parity_report.json"), "w") as f:
+            json.dump(REPORT, f, indent=1)
+    except OSError:
+        pass
+
+
+def _check(inp, bwd, label, flags=0, tol=None):
+    got = run_inputs_bwd(inp, flags=flags) if bwd else run_inputs_fwd(inp, flags=flags)
+    ref = parity.oracle_all(inp, bwd)
+    keys = parity.FWD_KEYS + (parity.BWD_KEYS if bwd else ())
+    return parity.compare(got, ref, inp.io_dtype, keys, label, tol=tol, report=REPORT)
+
+
+PATHS = [("simt", binding.FLAG_FORCE_SIMT), ("auto", 0)]
+
+
+def test_cfg0_tiny_forward_fp32():
+    _check(config(0), False, "cfg0")
+
+
+def test_cfg0_shape_backward_fp32():
+    inp = draw("cfg0_bwd", 10, [256], 1, 64, 64, "fp32", dense_B=1, with_dout=True,
+               with_state=True, with_state_cotangents=True)
+    _check(inp, True, "cfg0_bwd")
+
+
+@pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])
+@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+def test_benchmark_configs_reduced(idx, path, flags):
+    shrink = {1: dict(B=2, T=320, H=2), 2: dict(B=2, T=320, H=2), 3: dict(B=1, T=448, H=3),
+              4: dict(nseq=5, lo=40, hi=700, total=1500, H=2)}[idx]
+    inp = config(idx, shrink=shrink)
+    _check(inp, idx >= 2, f"cfg{idx}_reduced_{path}", flags=flags)
+
+
+@pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])
+@pytest.mark.parametrize("io", ["fp32", "bf16"])
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_lively_sets(idx, io, path, flags):
+    if io == "fp32" and path == "auto":
+        pytest.skip("fp32 I/O always runs the CUDA-core kernels")
+    inp = lively(idx, T=200, B=2, H=2, D=128, io_dtype=io)
+    _check(inp, True, f"lively{idx}_{io}_{path}", flags=flags)
+
+
+@pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])
+@pytest.mark.parametrize("K,V", [(64, 64), (64, 128), (128, 64)])
+@pytest.mark.parametrize("T", [1, 63, 65, 200])
+def test_shapes_and_ragged_tails(T, K, V, path, flags):
+    hy = OsdnHyper(eta=0.3, apf_mode=1)
+    inp = draw(f"shape_{T}_{K}_{V}", 700 + T + K + V, [T, T], 2, K, V, "bf16", dense_B=2, hyper=hy,
+               with_dout=True, with_state=True, with_state_cotangents=True)
+    _check(inp, True, f"shape_T{T}_K{K}_V{V}_{path}", flags=flags)
+
+
+@pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])
+def test_degenerate_inputs(path, flags):
+    hy = OsdnHyper(eta=0.3, apf_mode=1)
+    inp = draw("degenerate", 900, [130, 0, 70, 3], 2, 128, 128, "bf16", hyper=hy, with_dout=True,
+               with_state=True, with_state_cotangents=True)
+    inp.beta[:40] = 0.0          # no-op writes
+    inp.beta[40:60] = 1.0        # full-step writes
+    inp.k[100:110] = 0.0         # zero keys: the eps floor of the normaliser
+    inp.gate[120:125] = -20.0    # near-total forgetting
+    _check(inp, True, f"degenerate_{path}", flags=flags)
+
+
+def test_precond_update_alone():
+    hy = OsdnHyper(eta=0.3, apf_mode=2)
+    inp = draw("pu", 950, [150, 64, 7], 3, 128, 128, "bf16", hyper=hy, with_log_ret=True, with_state=True)
+    dev = torch.device("cuda:0")
+    b = binding.DeviceBundle(inp, dev, need_bwd=False)
+    ktil = torch.empty_like(b.k)
+    dout = torch.empty_like(b.precond_in)
+    binding.osdn_precond_update(b.params, b.k, b.beta, b.log_ret, b.precond_in, ktil, dout)
+    torch.cuda.synchronize()
+    ref = oracle.precond_update(hy, inp.seq_lens, inp.k, inp.beta, None, inp.log_ret, inp.precond_in)
+    assert parity.err(dout.cpu().numpy(), ref["precond_out"], "fp32") <= 1e-5
+    assert parity.err(ktil.float().cpu().numpy(), ref["ktil"], "bf16") <= 2e-2
+    # streaming: two calls with the preconditioner carried equal one call (dense, fp32)
+    inp2 = draw("pu2", 951, [90], 2, 64, 64, "fp32", dense_B=1, hyper=OsdnHyper(eta=0.3, apf_mode=1))
+    b2 = binding.DeviceBundle(inp2, dev, need_bwd=False)
+    d_all = torch.empty(1, 2, 64, device=dev)
+    binding.osdn_precond_update(b2.params, b2.k, b2.beta, b2.gate, None, None, d_all)
+    p1 = binding.make_params(B=1, T=50, H=2, K=64, V=64, io_dtype="fp32", hyper=inp2.hyper)
+    p2 = binding.make_params(B=1, T=40, H=2, K=64, V=64, io_dtype="fp32", hyper=inp2.hyper)
+    d_mid = torch.empty(1, 2, 64, device=dev)
+    binding.osdn_precond_update(p1, b2.k[:50].contiguous(), b2.beta[:50].contiguous(), b2.gate[:50].contiguous(),
+                                None, None, d_mid)
+    binding.osdn_precond_update(p2, b2.k[50:].contiguous(), b2.beta[50:].contiguous(), b2.gate[50:].contiguous(),
+                                d_mid, None, d_mid)
+    torch.cuda.synchronize()
+    assert torch.equal(d_mid, d_all)
+
+
+def test_split_sequence_state_carry_on_gpu():
+    hy = OsdnHyper(eta=0.3, apf_mode=1)
+    inp = draw("carry", 960, [192], 2, 128, 128, "fp32", dense_B=1, hyper=hy)
+    full = run_inputs_fwd(inp)
+    a, _, _ = parity.subset(inp, [0], [0, 1])
+    first = draw("carry", 960, [192], 2, 128, 128, "fp32", dense_B=1, hyper=hy)
+    for name in ("q", "k", "v", "beta", "gate"):
+        setattr(first, name, getattr(inp, name)[:128].contiguous())
+    first.seq_lens = [128]
+    r1 = run_inputs_fwd(first)
+    second = draw("carry", 960, [192], 2, 128, 128, "fp32", dense_B=1, hyper=hy)
+    for name in ("q", "k", "v", "beta", "gate"):
+        setattr(second, name, getattr(inp, name)[128:].contiguous())
+    second.seq_lens = [64]
+    second.init_state, second.precond_in = r1["final_state"], r1["precond_out"]
+    r2 = run_inputs_fwd(second)
+    assert parity.err(torch.cat([r1["out"], r2["out"]]).numpy(), full["out"].numpy(), "fp32") <= 1e-5
+    assert parity.err(r2["final_state"].numpy(), full["final_state"].numpy(), "fp32") <= 1e-5
+    assert parity.err(r2["precond_out"].numpy(), full["precond_out"].numpy(), "fp32") <= 1e-6
+
+
+def test_backward_with_and_without_saved_residuals_agree():
+    inp = lively(1, T=150, B=1, H=2, D=128, io_dtype="bf16")
+    a = run_inputs_bwd(inp, reuse_residuals=True)
+    b = run_inputs_bwd(inp, reuse_residuals=False)
+    for k in parity.BWD_KEYS:
+        assert torch.equal(a[k], b[k]), k
+
+
+def test_run_to_run_determinism():
+    inp = config(2, shrink=dict(B=1, T=256, H=2))
+    a = run_inputs_bwd(inp)
+    b = run_inputs_bwd(inp)
+    for k in ("out", "final_state", "dq", "dv", "dinit_state"):
+        assert torch.equal(a[k], b[k]), k
