@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the OSDN layer hot path: forward + backward tokens/s per layer on B200.
+
+    python bench.py --gpus 1 --steps 20 --warmup 5
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference            # the fp64 CPU oracle, timed on the host cores
+
+One step = one pass of the whole hot path (osdn_fwd with saved residuals + osdn_bwd) over one
+synthetic batch of the 340M-model layer shape (B=8, T=2048, H=8, dk=dv=128, bf16).  Inputs are
+resident in HBM for `value`; `e2e` goes through osdn_step_host with pinned host buffers.  With N
+GPUs every rank runs its own batch (weak scaling, no data-path collective: chains are independent).
+Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    "cfg1": dict(idx=1, bwd=False, desc="cfg1 340M layer forward: B=8 T=2048 H=8 dk=dv=128 bf16"),
+    "cfg2": dict(idx=2, bwd=True, desc="cfg2 340M layer train step (fwd+bwd): B=8 T=2048 H=8 dk=dv=128 bf16"),
+    "cfg3": dict(idx=3, bwd=True, desc="cfg3 1.3B layer fwd+bwd: B=4 T=4096 H=16 dk=dv=128 bf16, mixture gates"),
+    "cfg4": dict(idx=4, bwd=True, desc="cfg4 varlen fwd+bwd: 8 packed sequences, 131072 tokens, H=8 dk=dv=128 bf16"),
+    "cfg2_lively": dict(idx=-2, bwd=True, desc="cfg2 shape with a moving preconditioner (eta=0.3, sparse keys, "
+                                               "separate retention): B=8 T=2048 H=8 dk=dv=128 bf16"),
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def make_inputs(name):
+    from paper_2605_13473_b200.synth import OsdnHyper, config, draw
+    w = WORKLOADS[name]
+    if w["idx"] >= 0:
+        return config(w["idx"])
+    hy = OsdnHyper(eta=0.3, apf_mode=2)
+    return draw("cfg2_lively", 12, [2048] * 8, 8, 128, 128, "bf16", dense_B=8, hyper=hy, key_kind="sparse",
+                with_dout=True, with_log_ret=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# Algorithmic work of each kernel per launch (bytes it must read + write given the data flow of
+# the design, and tensor flops), as a function of the workload.  Stated in the design doc.
+# ---------------------------------------------------------------------------------------------
+def kernel_model(name, inp, NT):
+    """returns (bytes, flops, bound) for one launch; NT = number of 64-token chunks (all heads excluded)."""
+    H, K, V = inp.H, inp.K, inp.V
+    T = inp.T_total
+    es = 2 if inp.io_dtype == "bf16" else 4
+    tiles = NT * H               # (chunk, head) tiles
+    tokh = T * H                 # token-heads
+    C = 64
+    f = lambda m, n, k: 2.0 * m * n * k
+    m = {}
+    # CUDA-core (fp32 workspace) family
+    m["phase1_fwd"] = (tokh * (K * es + 8 + K * 4) + tiles * K * 4, tokh * 9.0 * K, "hbm")
+    m["simt_chunk_local_fwd"] = (tokh * (2 * K * es + K * 4 + V * es + 8) + tiles * 4 * (2 * C * C + C * K + C * V),
+                                 tiles * (2 * f(C, C, K) + f(C, K, C) + f(C, V, C)), "alu")
+    m["simt_chain_fwd"] = (tokh * (K * es + K * 4 + V * es + 8) + tiles * 4 * (C * K + 2 * C * V + C * C + V * K),
+                           tiles * (2 * f(C, V, K) + f(C, V, C) + f(V, K, C)), "alu")
+    m["simt_chain_bwd"] = (tokh * (K * es + K * 4 + V * es + 8) + tiles * 4 * (C * K + C * V + C * C + V * K),
+                           tiles * (f(C, V, C) + f(C, V, K) + 2 * f(V, K, C)), "alu")
+    m["simt_chunk_local_bwd"] = (tokh * (3 * K * es + K * 4 + 3 * V * es + 2 * K * 4 + 16)
+                                 + tiles * 4 * (2 * C * C + 2 * C * V + 2 * V * K + 10 * C * K),
+                                 tiles * (f(C, C, V) + 5 * f(C, K, V) + f(C, C, K) * 2 + f(C, C, V)
+                                          + f(C, K, C) * 5 + f(C, V, C) + 2 * f(C, C, C)), "alu")
+    m["phase1_bwd"] = (tokh * (K * es * 2 + 2 * K * 4 + 24) + tiles * K * 4, tokh * 30.0 * K, "hbm")
+    m["build_table"] = (NT * 12, 0.0, "hbm")
+    return m.get(name)
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for r in self.rows:
+            c = [x.strip() for x in r.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2])); power.append(float(c[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    power_w_max=max(power) if power else None, samples=len(sm), reasons=sorted(reasons))
+
+
+def run_reference(args):
+    """The oracle as it stands, timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import oracle
+    inp = make_inputs(args.workload)
+    w = WORKLOADS[args.workload]
+    tokens = inp.T_total
+
+    def step():
+        oracle.fwd_inputs(inp)
+        if w["bwd"]:
+            oracle.bwd_inputs(inp)
+
+    oracle.build()
+    for _ in range(args.warmup if args.warmup is not None else 1):
+        step()
+    steps = args.steps if args.steps is not None else 5
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = time.perf_counter() - t0
+    val = tokens * steps / dt
+    cores = oracle.threads()
+    line = {
+        "impl": "reference", "metric": "fwd+bwd tokens/s per layer", "value": val, "unit": "tokens/s",
+        "n_gpus": 0, "steps": steps, "warmup": args.warmup if args.warmup is not None else 1,
+        "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w["desc"], "note": "fp64 token-by-token CPU oracle, OpenMP over chains"},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": f"whole workload ({tokens} tokens x {inp.H} heads) per step"},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=list(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--simt", action="store_true", help="force the CUDA-core fp32 kernels")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    steps = args.steps if args.steps is not None else 20
+    warmup = max(args.warmup if args.warmup is not None else 5, 3)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2605_13473_b200 import binding
+    from paper_2605_13473_b200.build import build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    binding.load_library()
+
+    w = WORKLOADS[args.workload]
+    inp = make_inputs(args.workload)
+    flags = binding.FLAG_FORCE_SIMT if args.simt else 0
+    b = binding.DeviceBundle(inp, dev, need_bwd=w["bwd"], flags=flags)
+    tokens = inp.T_total
+
+    def step():
+        if w["bwd"]:
+            b.fwd(save=True)
+            n = binding.osdn_last_launch_count()
+            b.bwd(residuals_valid=True)
+            return n + binding.osdn_last_launch_count()
+        b.fwd(save=False)
+        return binding.osdn_last_launch_count()
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    assert b.device_status() == 0, "device-side error recorded during warm-up"
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    binding.stage_timing_enable(True)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches = 0
+    e0.record()
+    for _ in range(steps):
+        launches += step()
+    e1.record()
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    stages = binding.stage_timing_collect()
+    binding.stage_timing_enable(False)
+    clocks = sampler.stop()
+    assert b.device_status() == 0, "device-side error recorded during the timed region"
+
+    # ---- end to end through the host-buffer entry point --------------------------------------
+    e2e = None
+    if inp.log_ret is None:
+        pin = lambda t: None if t is None else t.contiguous().pin_memory()
+        io_dt = torch.bfloat16 if inp.io_dtype == "bf16" else torch.float32
+        hq, hk, hv = (pin(x.to(io_dt)) for x in (inp.q, inp.k, inp.v))
+        hb, hg = pin(inp.beta), pin(inp.gate)
+        hdo = pin(inp.dout.to(io_dt)) if w["bwd"] else None
+        hout = torch.empty(tokens, inp.H, inp.V, dtype=io_dt).pin_memory()
+        if w["bwd"]:
+            hdq, hdk = (torch.empty(tokens, inp.H, inp.K, dtype=io_dt).pin_memory() for _ in range(2))
+            hdv = torch.empty(tokens, inp.H, inp.V, dtype=io_dt).pin_memory()
+            hdb, hdg = (torch.empty(tokens, inp.H, dtype=torch.float32).pin_memory() for _ in range(2))
+        else:
+            hdq = hdk = hdv = hdb = hdg = None
+        staging = torch.empty(binding.osdn_host_staging_bytes(b.params, w["bwd"]), device=dev, dtype=torch.uint8)
+        b.params.flags = flags
+
+        def host_step():
+            binding.osdn_step_host(b.params, hq, hk, hv, hb, hg, hdo, hout, hdq, hdk, hdv, hdb, hdg, staging)
+
+        for _ in range(2):
+            host_step()
+        sync_all()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record()
+        for _ in range(steps):
+            host_step()
+        h1.record()
+        sync_all()
+        ms_host = h0.elapsed_time(h1)
+        nb = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts if t is not None))
+        e2e = dict(ms=ms_host, h2d=nb(hq, hk, hv, hb, hg, hdo), d2h=nb(hout, hdq, hdk, hdv, hdb, hdg))
+
+    # ---- max over ranks ----------------------------------------------------------------------
+    if world > 1:
+        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t[0])
+        if e2e:
+            e2e["ms"] = float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    value = tokens * world * steps / (ms_total * 1e-3)
+    # dominant kernel and its roofline
+    totals = {k: sum(v) for k, v in stages.items()}
+    NT = sum((L + 63) // 64 for L in inp.seq_lens)
+    roofline = None
+    kernel_table = {}
+    if totals:
+        all_ms = sum(totals.values())
+        for k, v in sorted(totals.items(), key=lambda kv: -kv[1]):
+            kernel_table[k] = dict(launches=len(stages[k]), avg_us=1e3 * v / len(stages[k]), share=v / all_ms)
+        dom = max(totals, key=totals.get)
+        avg_s = totals[dom] / len(stages[dom]) * 1e-3
+        model = kernel_model(dom, inp, NT)
+        if model:
+            nbytes, flops, bound = model
+            if bound == "tensor":
+                ach, peak, unit = flops / avg_s / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
+            elif bound == "alu":
+                # fp32 FMA peak of the chip: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
+                ach, peak, unit = flops / avg_s / 1e12, 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
+            else:
+                ach, peak, unit = nbytes / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
+            roofline = dict(kernel=dom, bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak,
+                            traffic=None, peak_source=peaks["source"], avg_us=avg_s * 1e6,
+                            algorithmic_bytes=nbytes, algorithmic_flops=flops)
+    # whole-step roofline (the slower of the step's flops at tensor peak and its bytes at HBM peak)
+    es = 2 if inp.io_dtype == "bf16" else 4
+    tokh = tokens * inp.H
+    if w["bwd"]:
+        step_bytes = tokh * ((2 * inp.K + inp.V) * es * 2 + inp.V * es * 2 + 16 + 16) + 0.0
+        step_flops = tokh * 0.67e6 * (inp.K * inp.V) / (128 * 128)
+    else:
+        step_bytes = tokh * ((2 * inp.K + 2 * inp.V) * es + 8)
+        step_flops = tokh * 139264.0 * (inp.K * inp.V) / (128 * 128)
+    t_roof = max(step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (peaks["bf16_tflops"] * 1e12))
+    step_roof = dict(roofline_us=t_roof * 1e6, measured_us=ms_total / steps * 1e3,
+                     frac=t_roof / (ms_total / steps * 1e-3), min_bytes=step_bytes, flops=step_flops)
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import oracle
+        oracle.build()
+        t0 = time.perf_counter()
+        reps = 0
+        while True:
+            oracle.fwd_inputs(inp)
+            if w["bwd"]:
+                oracle.bwd_inputs(inp)
+            reps += 1
+            if time.perf_counter() - t0 > 10.0 or reps >= 50:
+                break
+        dt = time.perf_counter() - t0
+        cpu_baseline = dict(value=tokens * reps / dt, unit="tokens/s", cores=oracle.threads(), kind="oracle",
+                            sample=f"whole workload ({tokens} tokens x {inp.H} heads), {reps} repetitions, {dt:.1f} s")
+
+    line = {
+        "metric": "fwd+bwd tokens/s per layer" if w["bwd"] else "fwd tokens/s per layer",
+        "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if inp.io_dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w["desc"], "l2": "inputs + workspace exceed L2 (no flush)",
+                   "path": "simt" if args.simt else "auto", "tokens_per_step_per_gpu": tokens},
+        "clocks": clocks, "gpu_launches": launches,
+        "e2e": ({"value": tokens * world * steps / (e2e["ms"] * 1e-3), "unit": "tokens/s",
+                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"]} if e2e else None),
+        "roofline": roofline, "step_roofline": step_roof, "kernels": kernel_table, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

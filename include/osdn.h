@@ -157,6 +157,17 @@ const char* osdn_status_string(int status);
  * this thread enqueued (for launch accounting in benchmarks). */
 int osdn_last_launch_count(void);
 
+/*
+ * Optional per-kernel timing for benchmarks (not part of the method).  While enabled, the library
+ * records a CUDA event on the launching stream before each of its kernels (at most 2048 marks
+ * since the last enable; later launches go unrecorded).  After synchronising the stream,
+ * osdn_stage_timing_read(i, &name, &ms) yields the name and duration of the i-th recorded kernel
+ * (name == NULL for separators between calls) and returns the number of marks.  Process-wide, not
+ * thread safe; enable(0) switches it off again.
+ */
+void osdn_stage_timing_enable(int on);
+int osdn_stage_timing_read(int index, const char** name, float* ms);
+
 #ifdef __cplusplus
 }
 #endif

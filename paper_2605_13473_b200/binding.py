@@ -18,6 +18,7 @@ FLAG_FORCE_SIMT = 4
 EXPORTS = [
     "osdn_workspace_bytes", "osdn_fwd", "osdn_bwd", "osdn_precond_update", "osdn_host_staging_bytes",
     "osdn_step_host", "osdn_read_device_status", "osdn_status_string", "osdn_last_launch_count",
+    "osdn_stage_timing_enable", "osdn_stage_timing_read",
 ]
 
 
@@ -62,6 +63,10 @@ def load_library(path: Optional[str] = None):
     lib.osdn_status_string.argtypes = [ci]
     lib.osdn_last_launch_count.restype = ci
     lib.osdn_last_launch_count.argtypes = []
+    lib.osdn_stage_timing_enable.restype = None
+    lib.osdn_stage_timing_enable.argtypes = [ci]
+    lib.osdn_stage_timing_read.restype = ci
+    lib.osdn_stage_timing_read.argtypes = [ci, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)]
     if path == _LIB_PATH:
         _lib = lib
     return lib
@@ -124,6 +129,23 @@ def osdn_host_staging_bytes(p: OsdnParams, with_bwd: bool) -> int:
 
 def osdn_last_launch_count() -> int:
     return int(load_library().osdn_last_launch_count())
+
+
+def stage_timing_enable(on: bool):
+    load_library().osdn_stage_timing_enable(int(on))
+
+
+def stage_timing_collect() -> dict:
+    """{kernel name: [durations in ms]} of the marks recorded since the last enable (sync first)."""
+    lib = load_library()
+    name, ms = ctypes.c_char_p(), ctypes.c_float()
+    n = lib.osdn_stage_timing_read(-1, None, None)
+    out = {}
+    for i in range(max(n - 1, 0)):
+        lib.osdn_stage_timing_read(i, ctypes.byref(name), ctypes.byref(ms))
+        if name.value is not None:
+            out.setdefault(name.value.decode(), []).append(float(ms.value))
+    return out
 
 
 def osdn_read_device_status(workspace: torch.Tensor) -> int:

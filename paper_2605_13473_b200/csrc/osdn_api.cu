@@ -20,6 +20,30 @@ namespace {
 
 thread_local int g_last_launches = 0;
 
+// ---- optional stage timing ------------------------------------------------------------------
+constexpr int MAX_MARKS = 2048;
+struct StageTimer {
+    bool enabled = false;
+    int count = 0;
+    cudaEvent_t ev[MAX_MARKS] = {};
+    const char* name[MAX_MARKS] = {};   // nullptr marks the end of a kernel sequence
+    int created = 0;
+};
+StageTimer g_timer;
+
+void timer_push(cudaStream_t st, const char* name)
+{
+    if (!g_timer.enabled || g_timer.count >= MAX_MARKS) return;
+    const int i = g_timer.count;
+    if (i >= g_timer.created) {
+        if (cudaEventCreate(&g_timer.ev[i]) != cudaSuccess) return;
+        g_timer.created = i + 1;
+    }
+    if (cudaEventRecord(g_timer.ev[i], st) != cudaSuccess) return;
+    g_timer.name[i] = name;
+    g_timer.count = i + 1;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int validate(const osdn_params* p)
@@ -66,7 +90,32 @@ int run_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
 
 }  // namespace
 
+namespace osdn {
+void stage_mark(cudaStream_t st, const char* name) { timer_push(st, name); }
+void stage_end(cudaStream_t st) { timer_push(st, nullptr); }
+}  // namespace osdn
+
 extern "C" {
+
+void osdn_stage_timing_enable(int on)
+{
+    g_timer.enabled = on != 0;
+    g_timer.count = 0;
+}
+
+int osdn_stage_timing_read(int index, const char** name, float* ms)
+{
+    if (index < 0 || index + 1 >= g_timer.count || !g_timer.name[index]) {
+        if (name) *name = nullptr;
+        if (ms) *ms = 0.f;
+        return g_timer.count;
+    }
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, g_timer.ev[index], g_timer.ev[index + 1]) != cudaSuccess) t = -1.f;
+    if (name) *name = g_timer.name[index];
+    if (ms) *ms = t;
+    return g_timer.count;
+}
 
 size_t osdn_workspace_bytes(const osdn_params* p, int need_bwd)
 {

@@ -139,4 +139,10 @@ int simt_precond_update(const osdn_params& p, const Hyper& hy, const void* k, co
                         float* precond_out, cudaStream_t st);
 int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st);
 
+// Optional per-kernel timing (off by default): when enabled through osdn_stage_timing_enable, every
+// launch site records a CUDA event on the launching stream before its kernel; stage_end closes the
+// last one.  Durations are read back with osdn_stage_timing_read after a synchronise.
+void stage_mark(cudaStream_t st, const char* name);
+void stage_end(cudaStream_t st);
+
 }  // namespace osdn

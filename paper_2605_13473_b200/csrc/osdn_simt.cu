@@ -795,6 +795,7 @@ int fwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
         pa.dbound = reinterpret_cast<float*>(w + L.dbound);
         pa.hy = hy;
         const int chains = S * H;
+        stage_mark(st, "phase1_fwd");
         phase1_fwd_kernel<T, float, K><<<(chains + 3) / 4, 128, 0, st>>>(pa);
         ++launches;
     }
@@ -807,6 +808,7 @@ int fwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
         ca.hy = hy;
         const size_t smem = sizeof(float) * (3 * CH * (K + 1) + 2 * CH * (CH + 1));
         if (!set_smem(chunk_local_fwd_kernel<T, K, V>, smem)) return -1;
+        stage_mark(st, "simt_chunk_local_fwd");
         chunk_local_fwd_kernel<T, K, V><<<dim3(L.NTmax, H), NTH, smem, st>>>(ca);
         ++launches;
     }
@@ -821,9 +823,11 @@ int fwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
         ch.save = save ? 1 : 0; ch.hy = hy;
         const size_t smem = sizeof(float) * (VSL * (K + 1) + 3 * CH * (K + 1) + CH * (CH + 1) + 2 * CH * (VSL + 1));
         if (!set_smem(chain_fwd_kernel<T, K, V, VSL>, smem)) return -1;
+        stage_mark(st, "simt_chain_fwd");
         chain_fwd_kernel<T, K, V, VSL><<<dim3(S * H, V / VSL), NTH, smem, st>>>(ch);
         ++launches;
     }
+    stage_end(st);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
@@ -844,6 +848,7 @@ int bwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
         ch.dinit_state = a.dinit_state; ch.hy = hy;
         const size_t smem = sizeof(float) * (VSL * (K + 1) + 3 * CH * (K + 1) + CH * (CH + 1) + 2 * CH * (VSL + 1));
         if (!set_smem(chain_bwd_kernel<T, K, V, VSL>, smem)) return -1;
+        stage_mark(st, "simt_chain_bwd");
         chain_bwd_kernel<T, K, V, VSL><<<dim3(S * H, V / VSL), NTH, smem, st>>>(ch);
         ++launches;
     }
@@ -856,6 +861,7 @@ int bwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
         ca.dq = a.dq; ca.dv = a.dv; ca.dbeta = a.dbeta; ca.dgate = a.dgate; ca.hy = hy;
         const size_t smem = sizeof(float) * (3 * CH * (K + 1) + 4 * CH * (CH + 1));
         if (!set_smem(chunk_local_bwd_kernel<T, K, V>, smem)) return -1;
+        stage_mark(st, "simt_chunk_local_bwd");
         chunk_local_bwd_kernel<T, K, V><<<dim3(L.NTmax, H), NTH, smem, st>>>(ca);
         ++launches;
     }
@@ -869,9 +875,11 @@ int bwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
         const size_t smem = sizeof(float) * 2 * (CH * K + 4 * CH);
         if (!set_smem(phase1_bwd_kernel<T, K>, smem)) return -1;
         const int chains = S * H;
+        stage_mark(st, "phase1_bwd");
         phase1_bwd_kernel<T, K><<<(chains + 1) / 2, 64, smem, st>>>(pb);
         ++launches;
     }
+    stage_end(st);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
@@ -889,6 +897,7 @@ int p1_dispatch(int K, const P1Args& pa, cudaStream_t st)
 int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st)
 {
     Table tab = carve_table(ws, L);
+    stage_mark(st, "build_table");
     build_table_kernel<<<1, 256, 0, st>>>(L.S, p.T, p.nseq > 0 ? p.cu_seqlens : nullptr, L.NTmax, tab);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

@@ -98,7 +98,7 @@ def test_precond_update_alone():
     torch.cuda.synchronize()
     ref = oracle.precond_update(hy, inp.seq_lens, inp.k, inp.beta, None, inp.log_ret, inp.precond_in)
     assert parity.err(dout.cpu().numpy(), ref["precond_out"], "fp32") <= 1e-5
-    assert parity.err(ktil.float().cpu().numpy(), ref["ktil"], "bf16") <= 2e-2
+    assert parity.err(ktil.float().cpu().numpy(), ref["ktil"], "bf16", True) <= 2e-2
     # streaming: two calls with the preconditioner carried equal one call (dense, fp32)
     inp2 = draw("pu2", 951, [90], 2, 64, 64, "fp32", dense_B=1, hyper=OsdnHyper(eta=0.3, apf_mode=1))
     b2 = binding.DeviceBundle(inp2, dev, need_bwd=False)
@@ -119,7 +119,6 @@ def test_split_sequence_state_carry_on_gpu():
     hy = OsdnHyper(eta=0.3, apf_mode=1)
     inp = draw("carry", 960, [192], 2, 128, 128, "fp32", dense_B=1, hyper=hy)
     full = run_inputs_fwd(inp)
-    a, _, _ = parity.subset(inp, [0], [0, 1])
     first = draw("carry", 960, [192], 2, 128, 128, "fp32", dense_B=1, hyper=hy)
     for name in ("q", "k", "v", "beta", "gate"):
         setattr(first, name, getattr(inp, name)[:128].contiguous())
@@ -141,7 +140,7 @@ def test_backward_with_and_without_saved_residuals_agree():
     a = run_inputs_bwd(inp, reuse_residuals=True)
     b = run_inputs_bwd(inp, reuse_residuals=False)
     for k in parity.BWD_KEYS:
-        assert torch.equal(a[k], b[k]), k
+        assert parity.err(a[k].numpy(), b[k].numpy(), "fp32") <= 1e-5, k
 
 
 def test_run_to_run_determinism():
