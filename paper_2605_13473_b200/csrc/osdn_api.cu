@@ -12,6 +12,7 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
 int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
                 cudaStream_t st);
 bool tc_supported(const osdn_params& p);
+bool tc_backward_supported(const osdn_params& p);
 }  // namespace osdn
 
 using namespace osdn;
@@ -73,9 +74,12 @@ Hyper make_hyper(const osdn_params& p)
     return h;
 }
 
-bool use_tc(const osdn_params& p)
+// The tensor-core kernels serve bf16 I/O.  A forward that saves residuals and the backward that
+// consumes them must use the same kernel family, so both follow tc_backward_supported.
+bool use_tc(const osdn_params& p, bool with_residuals)
 {
-    return p.io_dtype == OSDN_BF16 && !(p.flags & OSDN_FLAG_FORCE_SIMT) && tc_supported(p);
+    if (p.io_dtype != OSDN_BF16 || (p.flags & OSDN_FLAG_FORCE_SIMT) || !tc_supported(p)) return false;
+    return with_residuals ? tc_backward_supported(p) : true;
 }
 
 int run_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
@@ -83,7 +87,7 @@ int run_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
 {
     int n0 = launch_build_table(p, L, ws, st);
     if (n0 < 0) return -1;
-    int n1 = use_tc(p) ? tc_forward(p, hy, L, ws, a, save, st) : simt_forward(p, hy, L, ws, a, save, st);
+    int n1 = use_tc(p, save) ? tc_forward(p, hy, L, ws, a, save, st) : simt_forward(p, hy, L, ws, a, save, st);
     if (n1 < 0) return -1;
     return n0 + n1;
 }
@@ -194,7 +198,7 @@ int osdn_bwd(const osdn_params* p, const void* q, const void* k, const void* v, 
         if (n < 0) return OSDN_CUDA_ERROR;
         total += n;
     }
-    const int n = use_tc(*p) ? tc_backward(*p, hy, L, workspace, a, st) : simt_backward(*p, hy, L, workspace, a, st);
+    const int n = use_tc(*p, true) ? tc_backward(*p, hy, L, workspace, a, st) : simt_backward(*p, hy, L, workspace, a, st);
     if (n < 0) return OSDN_CUDA_ERROR;
     g_last_launches = total + n;
     return OSDN_OK;

@@ -137,6 +137,9 @@ int simt_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void
 int simt_precond_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta,
                         const float* retsrc, const float* precond_in, void* ktil_out,
                         float* precond_out, cudaStream_t st);
+// Phase 1 alone with bf16 write keys in the packed [T,H,K] layout (used by the tensor-core path).
+int simt_phase1(const osdn_params& p, const Hyper& hy, const Pointers& a, const int* seq_chunk0,
+                void* ktil_bf16, float* dbound, cudaStream_t st);
 int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st);
 
 // Optional per-kernel timing (off by default): when enabled through osdn_stage_timing_enable, every

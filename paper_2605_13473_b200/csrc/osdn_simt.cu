@@ -930,6 +930,19 @@ int simt_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void
     OSDN_DISPATCH(bwd_impl, p, hy, L, ws, a, st);
 }
 
+int simt_phase1(const osdn_params& p, const Hyper& hy, const Pointers& a, const int* seq_chunk0,
+                void* ktil_bf16, float* dbound, cudaStream_t st)
+{
+    P1Args pa{};
+    pa.S = p.nseq > 0 ? p.nseq : p.B;
+    pa.H = p.H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
+    pa.seq_chunk0 = seq_chunk0;
+    pa.k = a.k; pa.beta = a.beta; pa.retsrc = p.apf_mode == 2 ? a.log_ret : a.gate;
+    pa.d0 = a.precond_in; pa.ktil = ktil_bf16; pa.d_final = a.precond_out; pa.dbound = dbound; pa.hy = hy;
+    stage_mark(st, "phase1_fwd");
+    return p1_dispatch<__nv_bfloat16, __nv_bfloat16>(p.K, pa, st);
+}
+
 int simt_precond_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta,
                         const float* retsrc, const float* precond_in, void* ktil_out, float* precond_out,
                         cudaStream_t st)

@@ -1,14 +1,675 @@
-// tcgen05 / TMA kernels of the OSDN layer for bf16 I/O (sm_100a).
+// tcgen05 / TMA kernels of the OSDN layer for bf16 I/O, K = V = 128, chunk = 64 (sm_100a).
+//
+// Data flow of the forward pass (gated chunk form; G_i in-chunk gate prefix, gamma = exp(G),
+// Gamma_ij = exp(G_i - G_j), rho_i = exp(G_C - G_i)):
+//
+//   phase1_fwd (CUDA cores)      ktil = d (.) k in bf16, preconditioner at chunk starts
+//   tc_chunk_fwd  per (chunk, head), parallel:
+//        [K;Q] Ktil^T  -> A = strictLower(beta_i Gamma_ij <k_i,ktil_j>),  P' = scale * Lower(Gamma_ij <q_i,ktil_j>)
+//        T = (I + A)^-1 (fp32 forward substitution), Tb = T diag(beta), Tbg = T diag(beta gamma)
+//        W^T = K^T Tbg^T                               (tensor memory: lane = feature, column = token)
+//   tc_chain_fwd  per chain, sequential over chunks, state S (V x K, fp32) resident in tensor memory:
+//        dU^T = V^T Tb^T - S W^T ;  O1^T = S Q^T
+//        O2^T = dU^T P'^T ;         S <- gamma_C S + (rho dU)^T Ktil
+//        O^T  = scale gamma_i O1^T + O2^T
+//
+// Work tiles that travel between kernels are stored in HBM as ready-made images of the
+// 128-byte-swizzled shared-memory layout (see umma.cuh), so that the consumer fetches them with a
+// plain bulk copy; user tensors (q, k, ktil, v, dout) are fetched with TMA tensor maps.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include "osdn_common.cuh"
+#include "umma.cuh"
 
 namespace osdn {
 
-bool tc_supported(const osdn_params&) { return false; }
+using namespace umma;
 
-int tc_forward(const osdn_params&, const Hyper&, const WsLayout&, void*, const Pointers&, bool, cudaStream_t)
+namespace {
+
+constexpr int KD = 128;  // K = V = 128 on this path
+constexpr uint32_t BOX = 8192;   // one [64 rows x 128 B] box
+
+// device status codes of bounded waits
+enum { ERR_TMA = 101, ERR_MMA1 = 102, ERR_MMA2 = 103, ERR_CHAIN_TMA = 111, ERR_CHAIN_MMA1 = 112, ERR_CHAIN_MMA2 = 113 };
+
+struct TcLayout {
+    size_t ktil, dbound, WT, Tb, Tm, P, Qg, Sn, dUT, ddUT, dSn, dktil, dkread, total;
+};
+
+TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
 {
-    return -1;
+    TcLayout t{};
+    const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
+    const size_t H = p.H, NT = L.NTmax;
+    size_t off = L.ktil;
+    auto take = [&](size_t b) { size_t o = off; off = align_up(off + b, 1024); return o; };
+    off = align_up(off, 1024);
+    t.ktil = take(Ttot * H * KD * 2);
+    t.dbound = take(NT * H * KD * 4);
+    t.WT = take(NT * H * 16384);
+    t.Tb = take(NT * H * 8192);
+    t.Tm = take(NT * H * 8192);
+    t.P = take(NT * H * 8192);
+    t.Qg = take(NT * H * 16384);
+    t.Sn = take(NT * H * 32768);
+    t.dUT = take(NT * H * 16384);
+    if (need_bwd) {
+        t.ddUT = take(NT * H * 16384);
+        t.dSn = take(NT * H * 32768);
+        t.dktil = take(Ttot * H * KD * 4);
+        t.dkread = take(Ttot * H * KD * 4);
+    }
+    t.total = off;
+    return t;
 }
+
+// ---------------------------------------------------------------------------------------------
+// tensor maps
+// ---------------------------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled get_encoder()
+{
+    static PFN_cuTensorMapEncodeTiled fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(ptr);
+    }
+    return fn;
+}
+
+// Map over a packed [rows, H * 128] bf16 tensor; boxes of 64 rows x 64 columns, 128-byte swizzle,
+// out-of-range rows read as zero.
+bool make_token_map(CUtensorMap* m, const void* base, size_t rows, int H)
+{
+    PFN_cuTensorMapEncodeTiled enc = get_encoder();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)H * KD, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)H * KD * 2};
+    cuuint32_t box[2] = {64, 64};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__device__ __forceinline__ uint8_t* align1024(uint8_t* p)
+{
+    return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
+}
+
+// Zero rows [len, 64) of a box (tail chunks only).
+__device__ __forceinline__ void zero_tail_rows(uint8_t* box, int len, int tid, int nthreads)
+{
+    const int rows = CH - len;
+    for (int e = tid; e < rows * 8; e += nthreads)
+        *reinterpret_cast<uint4*>(box + (len + e / 8) * 128 + (e % 8) * 16) = make_uint4(0, 0, 0, 0);
+}
+
+// ---------------------------------------------------------------------------------------------
+// chunk-local forward
+// ---------------------------------------------------------------------------------------------
+struct TcChunkArgs {
+    int H;
+    Table tab;
+    const float *beta, *gate;
+    float scale;
+    uint8_t *WT, *Tb, *Tm, *P, *Qg;
+    int save;
+    int* status;
+};
+
+constexpr int CL_THREADS = 128;
+constexpr int LC = CH + 1;
+constexpr size_t CL_SMEM = 32768 + 16384 + 8192 + 2 * CH * LC * 4 + 1024;
+
+__global__ void __launch_bounds__(CL_THREADS)
+tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
+                    const __grid_constant__ CUtensorMap tmKt, TcChunkArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sm = align1024(smem_raw);
+    uint8_t* sKQ = sm;                 // per k-half h: [K rows 0-63 | Q rows 64-127], 16 KB each
+    uint8_t* sKt = sKQ + 32768;        // per k-half: 8 KB
+    uint8_t* sTb = sKt + 16384;        // T diag(beta gamma), K-major [i][j]
+    float* sA = reinterpret_cast<float*>(sTb + 8192);
+    float* sT = sA + CH * LC;
+    __shared__ uint64_t bar_tma, bar_mma1, bar_mma2;
+    __shared__ uint32_t tmem_base;
+    __shared__ float sG[CH], sBeta[CH], sg[CH];
+
+    const int c = blockIdx.x, h = blockIdx.y, H = a.H;
+    const int len = a.tab.chunk_len[c];
+    if (len == 0) return;
+    const int tok0 = a.tab.chunk_tok0[c];
+    const size_t tile = (size_t)c * H + h;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        mbar_init(&bar_tma, 1);
+        mbar_init(&bar_mma1, 1);
+        mbar_init(&bar_mma2, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(&tmem_base, 128);
+    if (tid < CH) {
+        const bool in = tid < len;
+        sg[tid] = in ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
+        sBeta[tid] = in ? a.beta[(size_t)(tok0 + tid) * H + h] : 0.f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+
+    if (tid == 0) {
+        mbar_expect_tx(&bar_tma, 6 * BOX);
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_load_2d(sKQ + hf * 16384, &tmK, h * KD + hf * 64, tok0, &bar_tma);
+            tma_load_2d(sKQ + hf * 16384 + BOX, &tmQ, h * KD + hf * 64, tok0, &bar_tma);
+            tma_load_2d(sKt + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_tma);
+        }
+    }
+    if (tid < CH) {
+        float acc = 0.f;
+        for (int j = 0; j <= tid; ++j) acc += sg[j];
+        sG[tid] = acc;
+    }
+    bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
+    if (len < CH) {
+        for (int hf = 0; hf < 2; ++hf) {
+            zero_tail_rows(sKQ + hf * 16384, len, tid, CL_THREADS);
+            zero_tail_rows(sKQ + hf * 16384 + BOX, len, tid, CL_THREADS);
+            zero_tail_rows(sKt + hf * BOX, len, tid, CL_THREADS);
+        }
+        fence_proxy_async();
+    }
+    __syncthreads();
+
+    // ---- D1[128 x 64] = [K;Q] Ktil^T ---------------------------------------------------------
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        const uint32_t idesc = make_idesc(128, 64);
+        for (int s = 0; s < 8; ++s) {
+            const uint64_t da = desc_advance(desc_kmajor(sKQ + (s >> 2) * 16384), 32 * (s & 3));
+            const uint64_t db = desc_advance(desc_kmajor(sKt + (s >> 2) * BOX), 32 * (s & 3));
+            mma_ss(tb, da, db, idesc, s > 0);
+        }
+        mma_commit(&bar_mma1);
+    }
+    ok = ok && mbar_wait(&bar_mma1, 0, a.status, ERR_MMA1);
+    tc_fence_after();
+    if (ok) {
+        const int L = warp * 32 + lane;
+        const uint32_t taddr = tb + ((uint32_t)(warp * 32) << 16);
+        if (L < CH) {
+            const int i = L;
+            const float bi = sBeta[i], Gi = sG[i];
+            for (int cb = 0; cb < 4; ++cb) {
+                uint32_t r[16];
+                tmem_ld16(taddr + cb * 16, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const int j = cb * 16 + x;
+                    sA[i * LC + j] = j < i ? bi * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+                }
+            }
+        } else {
+            const int i = L - CH;
+            const float Gi = sG[i];
+            uint8_t* Pg = a.P + tile * 8192;
+            for (int cb = 0; cb < 4; ++cb) {
+                uint32_t r[16];
+                tmem_ld16(taddr + cb * 16, r);
+                tmem_ld_wait();
+                float pv[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const int j = cb * 16 + x;
+                    pv[x] = j <= i ? a.scale * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+                }
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    uint4 w;
+                    w.x = pack_bf16(pv[c2 * 8 + 0], pv[c2 * 8 + 1]);
+                    w.y = pack_bf16(pv[c2 * 8 + 2], pv[c2 * 8 + 3]);
+                    w.z = pack_bf16(pv[c2 * 8 + 4], pv[c2 * 8 + 5]);
+                    w.w = pack_bf16(pv[c2 * 8 + 6], pv[c2 * 8 + 7]);
+                    *reinterpret_cast<uint4*>(Pg + sw128_chunk(i, cb * 2 + c2)) = w;
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- T = (I + A)^-1, column by column (two lanes per column split the inner sum) -----------
+    {
+        const int col = tid >> 1, part = tid & 1;
+        for (int i = 0; i < CH; ++i) {
+            float sum = 0.f;
+            for (int j = col + part; j < i; j += 2) sum = fmaf(sA[i * LC + j], sT[j * LC + col], sum);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            const float x = i < col ? 0.f : (i == col ? 1.f : -sum);
+            if (part == 0) sT[i * LC + col] = x;
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+
+    // ---- operand images: Tbg (shared), Tb and T (HBM) -----------------------------------------
+    for (int e = tid; e < CH * 8; e += CL_THREADS) {
+        const int i = e >> 3, ch = e & 7;
+        float t[8], tb8[8], tbg[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            const int j = ch * 8 + x;
+            t[x] = sT[i * LC + j];
+            tb8[x] = t[x] * sBeta[j];
+            tbg[x] = tb8[x] * __expf(sG[j]);
+        }
+        const uint32_t off = sw128_chunk(i, ch);
+        *reinterpret_cast<uint4*>(sTb + off) = make_uint4(pack_bf16(tbg[0], tbg[1]), pack_bf16(tbg[2], tbg[3]),
+                                                         pack_bf16(tbg[4], tbg[5]), pack_bf16(tbg[6], tbg[7]));
+        *reinterpret_cast<uint4*>(a.Tb + tile * 8192 + off) =
+            make_uint4(pack_bf16(tb8[0], tb8[1]), pack_bf16(tb8[2], tb8[3]), pack_bf16(tb8[4], tb8[5]),
+                       pack_bf16(tb8[6], tb8[7]));
+        if (a.save)
+            *reinterpret_cast<uint4*>(a.Tm + tile * 8192 + off) =
+                make_uint4(pack_bf16(t[0], t[1]), pack_bf16(t[2], t[3]), pack_bf16(t[4], t[5]), pack_bf16(t[6], t[7]));
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- D2[128 x 64] = K^T Tbg^T  (W^T) -----------------------------------------------------
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
+        const uint64_t da0 = desc_mnmajor(sKQ, 16384);
+        const uint64_t db0 = desc_kmajor(sTb);
+        for (int s = 0; s < 4; ++s) mma_ss(tb + 64, desc_advance(da0, 2048 * s), desc_advance(db0, 32 * s), idesc, s > 0);
+        mma_commit(&bar_mma2);
+    }
+    // gated, scaled queries for the backward state chain: Qg = scale gamma_i Q (same image layout as Q)
+    if (a.save) {
+        for (int e = tid; e < 2 * CH * 8; e += CL_THREADS) {
+            const int hf = e >> 9, i = (e >> 3) & 63, ch = e & 7;
+            const uint32_t off = sw128_chunk(i, ch);
+            const uint4 w = *reinterpret_cast<const uint4*>(sKQ + hf * 16384 + BOX + off);
+            const float f = a.scale * __expf(sG[i]);
+            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&w);
+            uint32_t o[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const float2 v = __bfloat1622float2(p2[x]);
+                o[x] = pack_bf16(v.x * f, v.y * f);
+            }
+            *reinterpret_cast<uint4*>(a.Qg + tile * 16384 + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+    ok = ok && mbar_wait(&bar_mma2, 0, a.status, ERR_MMA2);
+    tc_fence_after();
+    if (ok) {
+        const int k = warp * 32 + lane;
+        const uint32_t taddr = tb + ((uint32_t)(warp * 32) << 16) + 64;
+        uint8_t* Wg = a.WT + tile * 16384;
+        for (int cb = 0; cb < 4; ++cb) {
+            uint32_t r[16];
+            tmem_ld16(taddr + cb * 16, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c2 = 0; c2 < 2; ++c2) {
+                uint4 w;
+                w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
+                w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
+                w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
+                w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
+                *reinterpret_cast<uint4*>(Wg + sw128_chunk(k, cb * 2 + c2)) = w;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tb, 128);
+}
+
+// ---------------------------------------------------------------------------------------------
+// state chain, forward
+// ---------------------------------------------------------------------------------------------
+struct TcChainArgs {
+    int H;
+    Table tab;
+    const float *gate, *init_state;
+    __nv_bfloat16* out;
+    float* final_state;
+    const uint8_t *WT, *Tb, *P;
+    uint8_t *Sn, *dUT;
+    float scale;
+    int save;
+    int* status;
+};
+
+constexpr int CF_THREADS = 256;
+constexpr uint32_t STAGE_BYTES = 16384 + 8192 + 8192 + 3 * 16384;   // WT, Tb, P, V, Q, Ktil = 81920
+constexpr uint32_t ST_WT = 0, ST_TB = 16384, ST_P = 24576, ST_V = 32768, ST_Q = 49152, ST_KT = 65536;
+constexpr size_t CF_SMEM = 2 * STAGE_BYTES + 32768 + 2 * 16384 + 1024;
+
+__global__ void __launch_bounds__(CF_THREADS, 1)
+tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
+                    const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sm = align1024(smem_raw);
+    uint8_t* sStage = sm;                       // 2 stages
+    uint8_t* sS = sm + 2 * STAGE_BYTES;         // S as bf16, K-major: 2 k-halves x [128 rows x 128 B]
+    uint8_t* sDU1 = sS + 32768;                 // dU^T, K-major [v][i]
+    uint8_t* sDU2 = sDU1 + 16384;               // (rho dU)^T
+    __shared__ uint64_t bar_full[2], bar_mma1, bar_mma2;
+    __shared__ uint32_t tmem_base;
+    __shared__ float sGam[2][CH], sRho[2][CH], sGC[2], sgraw[CH];
+
+    const int chain = blockIdx.x, H = a.H;
+    const int s = chain / H, h = chain % H;
+    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int quad = warp & 3, colhalf = warp >> 2;
+    const int v = quad * 32 + lane;             // state row owned by this thread
+    float* fin = a.final_state ? a.final_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
+    const float* ini = a.init_state ? a.init_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
+    if (c1 <= c0) {   // empty sequence: the state passes through
+        if (fin)
+            for (int x = 0; x < 64; ++x) fin[x] = ini ? ini[x] : 0.f;
+        return;
+    }
+
+    if (tid == 0) {
+        mbar_init(&bar_full[0], 1);
+        mbar_init(&bar_full[1], 1);
+        mbar_init(&bar_mma1, 1);
+        mbar_init(&bar_mma2, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(&tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t tS = tb, tDU = tb + 128, tO1 = tb + 192, tO2 = tb + 256;
+
+    auto issue_loads = [&](int c, int st) {
+        const int tok0 = a.tab.chunk_tok0[c];
+        const size_t tile = (size_t)c * H + h;
+        uint8_t* d = sStage + st * STAGE_BYTES;
+        mbar_expect_tx(&bar_full[st], STAGE_BYTES);
+        bulk_load(d + ST_WT, a.WT + tile * 16384, 16384, &bar_full[st]);
+        bulk_load(d + ST_TB, a.Tb + tile * 8192, 8192, &bar_full[st]);
+        bulk_load(d + ST_P, a.P + tile * 8192, 8192, &bar_full[st]);
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_load_2d(d + ST_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_full[st]);
+            tma_load_2d(d + ST_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_full[st]);
+            tma_load_2d(d + ST_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
+        }
+    };
+    // gate vectors of chunk c into slot st (threads 0..63, then a barrier by the caller)
+    auto gate_vectors = [&](int c, int st) {
+        if (tid < CH) {
+            const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+            sgraw[tid] = tid < len ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
+        }
+        __syncthreads();
+        if (tid < CH) {
+            float G = 0.f, tot = 0.f;
+            for (int j = 0; j < CH; ++j) {
+                const float g = sgraw[j];
+                tot += g;
+                if (j <= tid) G += g;
+            }
+            sGam[st][tid] = __expf(G);
+            sRho[st][tid] = __expf(tot - G);
+            if (tid == 0) sGC[st] = __expf(tot);
+        }
+    };
+
+    if (tid == 0) issue_loads(c0, 0);
+    // initial state into tensor memory
+    for (int cb = 0; cb < 4; ++cb) {
+        uint32_t r[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(ini ? ini[cb * 16 + x] : 0.f);
+        tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+    }
+    tmem_st_wait();
+    gate_vectors(c0, 0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    bool ok = true;
+    for (int c = c0; c < c1; ++c) {
+        const int n = c - c0, st = n & 1;
+        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+        const size_t tile = (size_t)c * H + h;
+        uint8_t* d = sStage + st * STAGE_BYTES;
+        if (tid == 0 && c + 1 < c1) issue_loads(c + 1, st ^ 1);
+
+        // ---- E0: S -> bf16 operand (+ saved copy), decay the accumulator -----------------------
+        {
+            const float gC = sGC[st];
+            uint8_t* Sg = a.Sn + tile * 32768 + colhalf * 16384;
+            for (int cb = 0; cb < 4; ++cb) {
+                uint32_t r[16];
+                tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
+                    w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
+                    w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
+                    w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
+                    const uint32_t off = sw128_chunk(v, cb * 2 + c2);
+                    *reinterpret_cast<uint4*>(sS + colhalf * 16384 + off) = w;
+                    if (a.save) *reinterpret_cast<uint4*>(Sg + off) = w;
+                }
+#pragma unroll
+                for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
+                tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+            }
+            tmem_st_wait();
+        }
+        ok = ok && mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
+        if (len < CH) {
+            for (int hf = 0; hf < 2; ++hf) {
+                zero_tail_rows(d + ST_V + hf * BOX, len, tid, CF_THREADS);
+                zero_tail_rows(d + ST_Q + hf * BOX, len, tid, CF_THREADS);
+                zero_tail_rows(d + ST_KT + hf * BOX, len, tid, CF_THREADS);
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+
+        // ---- MMA group 1 -----------------------------------------------------------------------
+        if (tid == 0 && ok) {
+            tc_fence_after();
+            {   // dU^T = V^T Tb^T
+                const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
+                const uint64_t da0 = desc_mnmajor(d + ST_V, BOX), db0 = desc_kmajor(d + ST_TB);
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tDU, desc_advance(da0, 2048 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+            }
+            {   // dU^T -= S W^T
+                const uint32_t idesc = make_idesc(128, 64, IDESC_A_NEG | IDESC_B_MN);
+                const uint64_t db0 = desc_mnmajor(d + ST_WT, 0);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tDU, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
+                           desc_advance(db0, 2048 * k), idesc, 1);
+            }
+            {   // O1^T = S Q^T
+                const uint32_t idesc = make_idesc(128, 64);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tO1, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
+                           desc_advance(desc_kmajor(d + ST_Q + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
+            }
+            mma_commit(&bar_mma1);
+        }
+        ok = ok && mbar_wait(&bar_mma1, n & 1, a.status, ERR_CHAIN_MMA1);
+        tc_fence_after();
+
+        // ---- E1: dU^T -> bf16 operands ---------------------------------------------------------
+        {
+            uint8_t* dUg = a.dUT + tile * 16384;
+            for (int cb = 0; cb < 2; ++cb) {
+                uint32_t r[16];
+                tmem_ld16(tDU + lane_addr + colhalf * 32 + cb * 16, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    float f[8], g[8];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        f[x] = __uint_as_float(r[c2 * 8 + x]);
+                        g[x] = f[x] * sRho[st][colhalf * 32 + cb * 16 + c2 * 8 + x];
+                    }
+                    const uint32_t off = sw128_chunk(v, colhalf * 4 + cb * 2 + c2);
+                    const uint4 w1 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                                                pack_bf16(f[6], f[7]));
+                    *reinterpret_cast<uint4*>(sDU1 + off) = w1;
+                    *reinterpret_cast<uint4*>(sDU2 + off) = make_uint4(pack_bf16(g[0], g[1]), pack_bf16(g[2], g[3]),
+                                                                      pack_bf16(g[4], g[5]), pack_bf16(g[6], g[7]));
+                    if (a.save) *reinterpret_cast<uint4*>(dUg + off) = w1;
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+
+        // ---- MMA group 2 -----------------------------------------------------------------------
+        if (tid == 0 && ok) {
+            tc_fence_after();
+            {   // O2^T = dU^T P'^T
+                const uint32_t idesc = make_idesc(128, 64);
+                const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tO2, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+            }
+            {   // S += (rho dU)^T Ktil
+                const uint32_t idesc = make_idesc(128, 128, IDESC_B_MN);
+                const uint64_t da0 = desc_kmajor(sDU2), db0 = desc_mnmajor(d + ST_KT, BOX);
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k), idesc, 1);
+            }
+            mma_commit(&bar_mma2);
+        }
+        // gate vectors of the next chunk while the tensor core works
+        if (c + 1 < c1) gate_vectors(c + 1, st ^ 1);
+        ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
+        tc_fence_after();
+
+        // ---- E2: O^T = scale gamma_i O1^T + O2^T -> out ----------------------------------------
+        if (ok) {
+            __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
+            for (int cb = 0; cb < 2; ++cb) {
+                uint32_t r1[16], r2[16];
+                tmem_ld16(tO1 + lane_addr + colhalf * 32 + cb * 16, r1);
+                tmem_ld16(tO2 + lane_addr + colhalf * 32 + cb * 16, r2);
+                tmem_ld_wait();
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const int i = colhalf * 32 + cb * 16 + x;
+                    if (i < len)
+                        op[(size_t)i * H * KD] = __float2bfloat16_rn(
+                            a.scale * sGam[st][i] * __uint_as_float(r1[x]) + __uint_as_float(r2[x]));
+                }
+            }
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+
+    if (fin && ok) {
+        for (int cb = 0; cb < 4; ++cb) {
+            uint32_t r[16];
+            tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 16; ++x) fin[cb * 16 + x] = __uint_as_float(r[x]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+template <typename F> bool set_smem(F* kernel, size_t bytes)
+{
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
+}  // namespace
+
+bool tc_supported(const osdn_params& p)
+{
+    return p.io_dtype == OSDN_BF16 && p.K == KD && p.V == KD && get_encoder() != nullptr;
+}
+
+int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a, bool save,
+               cudaStream_t st)
+{
+    char* w = static_cast<char*>(ws);
+    const TcLayout t = make_tc_layout(p, L, save);
+    if (t.total > L.total) return -1;
+    Table tab = carve_table(ws, L);
+    const int S = L.S, H = p.H;
+    const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
+    int* status = reinterpret_cast<int*>(w + L.status);
+    int launches = 0;
+
+    // phase 1 on CUDA cores: bf16 write keys, chunk-start preconditioners
+    const int n1 = simt_phase1(p, hy, a, tab.seq_chunk0, w + t.ktil, reinterpret_cast<float*>(w + t.dbound), st);
+    if (n1 < 0) return -1;
+    launches += n1;
+
+    CUtensorMap tmK, tmQ, tmKt, tmV;
+    if (!make_token_map(&tmK, a.k, Ttot, H) || !make_token_map(&tmQ, a.q, Ttot, H) ||
+        !make_token_map(&tmKt, w + t.ktil, Ttot, H) || !make_token_map(&tmV, a.v, Ttot, H))
+        return -1;
+    {
+        TcChunkArgs ca{};
+        ca.H = H; ca.tab = tab; ca.beta = a.beta; ca.gate = a.gate; ca.scale = hy.scale;
+        ca.WT = reinterpret_cast<uint8_t*>(w + t.WT); ca.Tb = reinterpret_cast<uint8_t*>(w + t.Tb);
+        ca.Tm = reinterpret_cast<uint8_t*>(w + t.Tm); ca.P = reinterpret_cast<uint8_t*>(w + t.P);
+        ca.Qg = reinterpret_cast<uint8_t*>(w + t.Qg); ca.save = save ? 1 : 0; ca.status = status;
+        if (!set_smem(tc_chunk_fwd_kernel, CL_SMEM)) return -1;
+        stage_mark(st, "tc_chunk_fwd");
+        tc_chunk_fwd_kernel<<<dim3(L.NTmax, H), CL_THREADS, CL_SMEM, st>>>(tmK, tmQ, tmKt, ca);
+        ++launches;
+    }
+    {
+        TcChainArgs ch{};
+        ch.H = H; ch.tab = tab; ch.gate = a.gate; ch.init_state = a.init_state;
+        ch.out = static_cast<__nv_bfloat16*>(a.out); ch.final_state = a.final_state;
+        ch.WT = reinterpret_cast<uint8_t*>(w + t.WT); ch.Tb = reinterpret_cast<uint8_t*>(w + t.Tb);
+        ch.P = reinterpret_cast<uint8_t*>(w + t.P); ch.Sn = reinterpret_cast<uint8_t*>(w + t.Sn);
+        ch.dUT = reinterpret_cast<uint8_t*>(w + t.dUT); ch.scale = hy.scale; ch.save = save ? 1 : 0;
+        ch.status = status;
+        if (!set_smem(tc_chain_fwd_kernel, CF_SMEM)) return -1;
+        stage_mark(st, "tc_chain_fwd");
+        tc_chain_fwd_kernel<<<S * H, CF_THREADS, CF_SMEM, st>>>(tmV, tmQ, tmKt, ch);
+        ++launches;
+    }
+    stage_end(st);
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+bool tc_backward_supported(const osdn_params&) { return false; }
 
 int tc_backward(const osdn_params&, const Hyper&, const WsLayout&, void*, const Pointers&, cudaStream_t)
 {
