@@ -71,7 +71,7 @@ def _cu(seq_lens: Sequence[int]) -> np.ndarray:
 
 
 def fwd(hy, seq_lens, q, k, v, beta, gate, log_ret=None, init_state=None, precond_in=None,
-        want_ktil: bool = False, want_dtraj: bool = False) -> dict:
+        want_ktil: bool = False, want_dtraj: bool = False, want_margin: bool = False) -> dict:
     """Token-by-token forward.  Returns dict(out, final_state, precond_out[, ktil, d_traj])."""
     lib = _load()
     q, k, v, beta, gate = map(_f64, (q, k, v, beta, gate))
@@ -88,12 +88,17 @@ def fwd(hy, seq_lens, q, k, v, beta, gate, log_ret=None, init_state=None, precon
     d = np.zeros((nseq, H, K))
     ktil = np.zeros((T, H, K)) if want_ktil else None
     dtraj = np.zeros((T, H, K)) if want_dtraj else None
+    margin = np.zeros((T, H, K)) if want_margin else None
+    mask = np.zeros((T, H, K), dtype=np.uint8) if want_margin else None
     hp = _hyper(hy, K)
     lib.osdn_oracle_fwd(ctypes.c_int(nseq), _p(cu), ctypes.c_int(H), ctypes.c_int(K),
                         ctypes.c_int(V), ctypes.byref(hp), _p(q), _p(k), _p(v), _p(beta), _p(gate),
                         _p(log_ret), _p(init_state), _p(precond_in), _p(out), _p(S), _p(d),
-                        _p(ktil), _p(dtraj))
+                        _p(ktil), _p(dtraj), _p(margin), _p(mask))
     res = dict(out=out, final_state=S, precond_out=d)
+    if want_margin:
+        res["margin"] = margin
+        res["mask"] = mask
     if want_ktil:
         res["ktil"] = ktil
     if want_dtraj:
@@ -117,8 +122,9 @@ def precond_update(hy, seq_lens, k, beta, gate=None, log_ret=None, precond_in=No
 
 
 def bwd(hy, seq_lens, q, k, v, beta, gate, dout, log_ret=None, init_state=None, precond_in=None,
-        dfinal_state=None, dprecond_out=None) -> dict:
-    """Reverse sweep.  Returns dict(dq, dk, dv, dbeta, dgate, dlog_ret, dinit_state, dprecond_in)."""
+        dfinal_state=None, dprecond_out=None, mask_override=None) -> dict:
+    """Reverse sweep.  mask_override: uint8 [T,H,K], 0/1 force a projection pass decision, 255 = default.
+  Returns dict(dq, dk, dv, dbeta, dgate, dlog_ret, dinit_state, dprecond_in)."""
     lib = _load()
     q, k, v, beta, gate, dout = map(_f64, (q, k, v, beta, gate, dout))
     log_ret, init_state, precond_in = map(_f64, (log_ret, init_state, precond_in))
@@ -131,10 +137,11 @@ def bwd(hy, seq_lens, q, k, v, beta, gate, dout, log_ret=None, init_state=None, 
     dbeta, dgate, dlr = np.zeros((T, H)), np.zeros((T, H)), np.zeros((T, H))
     dS0, dd0 = np.zeros((nseq, H, V, K)), np.zeros((nseq, H, K))
     hp = _hyper(hy, K)
+    mo = None if mask_override is None else np.ascontiguousarray(mask_override, dtype=np.uint8)
     lib.osdn_oracle_bwd(ctypes.c_int(nseq), _p(cu), ctypes.c_int(H), ctypes.c_int(K),
                         ctypes.c_int(V), ctypes.byref(hp), _p(q), _p(k), _p(v), _p(beta), _p(gate),
                         _p(log_ret), _p(init_state), _p(precond_in), _p(dout), _p(dfinal_state),
-                        _p(dprecond_out), _p(dq), _p(dk), _p(dv), _p(dbeta), _p(dgate), _p(dlr),
+                        _p(dprecond_out), _p(mo), _p(dq), _p(dk), _p(dv), _p(dbeta), _p(dgate), _p(dlr),
                         _p(dS0), _p(dd0))
     return dict(dq=dq, dk=dk, dv=dv, dbeta=dbeta, dgate=dgate, dlog_ret=dlr,
                 dinit_state=dS0, dprecond_in=dd0)
@@ -146,6 +153,7 @@ def fwd_inputs(inp, **kw) -> dict:
                inp.init_state, inp.precond_in, **kw)
 
 
-def bwd_inputs(inp) -> dict:
+def bwd_inputs(inp, mask_override=None) -> dict:
     return bwd(inp.hyper, inp.seq_lens, inp.q, inp.k, inp.v, inp.beta, inp.gate, inp.dout,
-               inp.log_ret, inp.init_state, inp.precond_in, inp.dfinal_state, inp.dprecond_out)
+               inp.log_ret, inp.init_state, inp.precond_in, inp.dfinal_state, inp.dprecond_out,
+               mask_override=mask_override)

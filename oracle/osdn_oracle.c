@@ -68,7 +68,7 @@ int osdn_oracle_threads(void)
 static void phase1_step(const oracle_hyper *hp, int K, const double *k, double beta,
                         double g, double lret, double *d, double *ktil,
                         double *c_out, double *rho_out, double *a_out, double *n_out,
-                        int *raw_norm_above_eps, unsigned char *mask)
+                        int *raw_norm_above_eps, unsigned char *mask, double *margin)
 {
     double sumk = 0.0, a = 0.0;
     for (int i = 0; i < K; ++i) {
@@ -86,6 +86,10 @@ static void phase1_step(const oracle_hyper *hp, int K, const double *k, double b
     for (int i = 0; i < K; ++i) {
         double dbar = rho * d[i] + c * k[i] * k[i];
         unsigned char m = 1;
+        if (margin) {
+            double lo = fabs(dbar - hp->d_min), hi = fabs(dbar - hp->d_max);
+            margin[i] = hp->clamp ? (lo < hi ? lo : hi) : 1e300;
+        }
         if (hp->clamp) {
             if (dbar < hp->d_min) { dbar = hp->d_min; m = 0; }
             else if (dbar > hp->d_max) { dbar = hp->d_max; m = 0; }
@@ -129,7 +133,7 @@ void osdn_oracle_fwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                      const double *beta, const double *gate, const double *log_ret,
                      const double *S0, const double *d0,
                      double *out, double *S_final, double *d_final,
-                     double *ktil_out, double *d_traj_out)
+                     double *ktil_out, double *d_traj_out, double *margin_out, unsigned char *mask_out)
 {
     int nchain = nseq * H;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -147,7 +151,7 @@ void osdn_oracle_fwd(int nseq, const int *cu, int H, int K, int V, const oracle_
             const double *kt = k + th * K, *qt = q + th * K, *vt = v + th * V;
             if (d_traj_out) memcpy(d_traj_out + th * K, d, sizeof(double) * K);
             phase1_step(hp, K, kt, beta[th], gate[th], log_ret ? log_ret[th] : 0.0, d, ktil,
-                        0, 0, 0, 0, 0, 0);
+                        0, 0, 0, 0, 0, mask_out ? mask_out + th * K : 0, margin_out ? margin_out + th * K : 0);
             if (ktil_out) memcpy(ktil_out + th * K, ktil, sizeof(double) * K);
             phase2_step(K, V, kt, ktil, vt, beta[th], gate[th], S, 0);
             for (int r = 0; r < V; ++r) {
@@ -178,7 +182,7 @@ void osdn_oracle_precond_update(int nseq, const int *cu, int H, int K, const ora
         for (int t = cu[s]; t < cu[s + 1]; ++t) {
             size_t th = (size_t)t * H + h;
             phase1_step(hp, K, k + th * K, beta[th], gate ? gate[th] : 0.0,
-                        log_ret ? log_ret[th] : 0.0, d, ktil, 0, 0, 0, 0, 0, 0);
+                        log_ret ? log_ret[th] : 0.0, d, ktil, 0, 0, 0, 0, 0, 0, 0);
             if (ktil_out) memcpy(ktil_out + th * K, ktil, sizeof(double) * K);
         }
         memcpy(d_final + ((size_t)s * H + h) * K, d, sizeof(double) * K);
@@ -199,6 +203,12 @@ void osdn_oracle_precond_update(int nseq, const int *cu, int H, int K, const ora
  *
  * Conventions where the paper is silent: the box projection passes gradient
  * iff d_min <= dbar <= d_max; max(|k|^2, eps) passes gradient iff |k|^2 > eps.
+ *
+ * mask_override ([T_total, H, K], nullable): 0 / 1 force the pass decision of
+ * one coordinate of one step, 255 leaves it to the rule above.  The gradient is
+ * discontinuous where dbar touches a face; a caller comparing against an fp32
+ * implementation uses this to take near-tie decisions (|dbar - face| within
+ * fp32 rounding) in that implementation's precision, and only those.
  */
 #define SEG 64
 
@@ -207,6 +217,7 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                      const double *beta, const double *gate, const double *log_ret,
                      const double *S0, const double *d0,
                      const double *dout, const double *dS_final, const double *dd_final,
+                     const unsigned char *mask_override,
                      double *dq, double *dk, double *dv, double *dbeta, double *dgate,
                      double *dlog_ret, double *dS0, double *dd0)
 {
@@ -247,7 +258,7 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
             for (int t = a0; t < a1; ++t) {
                 size_t th = (size_t)t * H + h;
                 phase1_step(hp, K, k + th * K, beta[th], gate[th], log_ret ? log_ret[th] : 0.0,
-                            d, ktil, 0, 0, 0, 0, 0, 0);
+                            d, ktil, 0, 0, 0, 0, 0, 0, 0);
                 phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
             }
         }
@@ -266,7 +277,7 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 memcpy(Shist + (size_t)(t - a0) * VK, S, sizeof(double) * VK);
                 memcpy(dhist + (size_t)(t - a0) * K, d, sizeof(double) * K);
                 phase1_step(hp, K, k + th * K, beta[th], gate[th], log_ret ? log_ret[th] : 0.0,
-                            d, ktil, 0, 0, 0, 0, 0, 0);
+                            d, ktil, 0, 0, 0, 0, 0, 0, 0);
                 phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
             }
             for (int t = a1 - 1; t >= a0; --t) {
@@ -281,7 +292,10 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 /* recompute this token's forward quantities */
                 double c, rho, a, n; int above;
                 memcpy(dnew, dt, sizeof(double) * K);
-                phase1_step(hp, K, kt, bt, gt, lt, dnew, ktil, &c, &rho, &a, &n, &above, mask);
+                phase1_step(hp, K, kt, bt, gt, lt, dnew, ktil, &c, &rho, &a, &n, &above, mask, 0);
+                if (mask_override)
+                    for (int i = 0; i < K; ++i)
+                        if (mask_override[th * K + i] != 255) mask[i] = mask_override[th * K + i];
                 for (int r = 0; r < V; ++r) {
                     double acc = 0.0;
                     for (int i = 0; i < K; ++i) {

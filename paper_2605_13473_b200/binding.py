@@ -18,7 +18,7 @@ FLAG_FORCE_SIMT = 4
 EXPORTS = [
     "osdn_workspace_bytes", "osdn_fwd", "osdn_bwd", "osdn_precond_update", "osdn_host_staging_bytes",
     "osdn_step_host", "osdn_read_device_status", "osdn_status_string", "osdn_last_launch_count",
-    "osdn_stage_timing_enable", "osdn_stage_timing_read",
+    "osdn_stage_timing_enable", "osdn_stage_timing_read", "osdn_workspace_region",
 ]
 
 
@@ -67,6 +67,8 @@ def load_library(path: Optional[str] = None):
     lib.osdn_stage_timing_enable.argtypes = [ci]
     lib.osdn_stage_timing_read.restype = ci
     lib.osdn_stage_timing_read.argtypes = [ci, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)]
+    lib.osdn_workspace_region.restype = ci
+    lib.osdn_workspace_region.argtypes = [pp, ci, ctypes.c_char_p, ctypes.POINTER(sz), ctypes.POINTER(sz)]
     if path == _LIB_PATH:
         _lib = lib
     return lib
@@ -146,6 +148,14 @@ def stage_timing_collect() -> dict:
         if name.value is not None:
             out.setdefault(name.value.decode(), []).append(float(ms.value))
     return out
+
+
+def workspace_region(p: OsdnParams, name: str):
+    """(offset, bytes) of a named region of a backward-capable workspace."""
+    off, nb = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(load_library().osdn_workspace_region(ctypes.byref(p), 1, name.encode(), ctypes.byref(off),
+                                                ctypes.byref(nb)), "osdn_workspace_region")
+    return int(off.value), int(nb.value)
 
 
 def osdn_read_device_status(workspace: torch.Tensor) -> int:
@@ -263,6 +273,33 @@ class DeviceBundle:
     def device_status(self) -> int:
         return osdn_read_device_status(self.workspace)
 
+    def projection_masks(self) -> torch.Tensor:
+        """uint8 [T,H,K] pass masks of the projection as the forward (with saved residuals) took them."""
+        inp = self.inp
+        T, H, K = inp.T_total, inp.H, inp.K
+        o1, n1 = workspace_region(self.params, "p1_skip")
+        o2, n2 = workspace_region(self.params, "p1_mask")
+        skip = self.workspace[o1:o1 + n1].view(torch.int32).cpu().numpy().astype("uint32").reshape(-1, H, 2)
+        words = self.workspace[o2:o2 + n2].view(torch.int32).cpu().numpy().astype("uint32").reshape(T, H, K // 32)
+        import numpy as np
+        bits = ((words[..., None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8).reshape(T, H, K)
+        skipped = np.zeros((T, H), dtype=bool)
+        c = 0
+        t0 = 0
+        for L in inp.seq_lens:
+            for j in range((L + 63) // 64):
+                n = min(64, L - 64 * j)
+                w = skip[c].astype(np.uint64)
+                pair = w[:, 0] | (w[:, 1] << np.uint64(32))
+                sk = ((pair[None, :] >> np.arange(n, dtype=np.uint64)[:, None]) & np.uint64(1)).astype(bool)
+                skipped[t0 + 64 * j:t0 + 64 * j + n] = sk
+                c += 1
+            t0 += L
+        bits[skipped] = 0
+        if not inp.hyper.clamp:
+            bits[:] = 1
+        return torch.from_numpy(bits)
+
 
 def run_inputs_fwd(inp, device="cuda:0", flags: int = 0) -> dict:
     b = DeviceBundle(inp, device, need_bwd=False, flags=flags)
@@ -278,7 +315,8 @@ def run_inputs_bwd(inp, device="cuda:0", flags: int = 0, reuse_residuals: bool =
     b.bwd(residuals_valid=reuse_residuals)
     torch.cuda.synchronize()
     assert b.device_status() == 0
+    masks = b.projection_masks() if reuse_residuals else None
     return dict(out=b.out.float().cpu(), final_state=b.final_state.cpu(), precond_out=b.precond_out.cpu(),
-                dq=b.dq.float().cpu(), dk=b.dk.float().cpu(), dv=b.dv.float().cpu(), dbeta=b.dbeta.cpu(),
+                projection_masks=masks, dq=b.dq.float().cpu(), dk=b.dk.float().cpu(), dv=b.dv.float().cpu(), dbeta=b.dbeta.cpu(),
                 dgate=b.dgate.cpu(), dlog_ret=b.dlog_ret.cpu(), dinit_state=b.dinit_state.cpu(),
                 dprecond_in=b.dprecond_in.cpu())

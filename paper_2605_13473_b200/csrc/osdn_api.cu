@@ -215,7 +215,7 @@ int osdn_precond_update(const osdn_params* p, const void* k, const float* beta, 
     const void* ptrs[] = {k, beta, gate_or_log_ret, precond_in, k_tilde_out, precond_out};
     for (const void* x : ptrs)
         if (x && !aligned16(x)) return OSDN_MISALIGNED;
-    const int n = simt_precond_update(*p, make_hyper(*p), k, beta, gate_or_log_ret, precond_in, k_tilde_out,
+    const int n = phase1_update(*p, make_hyper(*p), k, beta, gate_or_log_ret, precond_in, k_tilde_out,
                                       precond_out, static_cast<cudaStream_t>(cuda_stream));
     if (n < 0) return OSDN_CUDA_ERROR;
     g_last_launches = n;
@@ -308,6 +308,24 @@ int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host,
     }
     g_last_launches = launches;
     return ok ? OSDN_OK : OSDN_CUDA_ERROR;
+}
+
+int osdn_workspace_region(const osdn_params* p, int need_bwd, const char* name, size_t* offset, size_t* bytes)
+{
+    if (validate(p) != OSDN_OK || !name || !offset || !bytes || !need_bwd) return OSDN_INVALID_ARG;
+    const WsLayout L = make_layout(*p, true);
+    const size_t Ttot = p->nseq > 0 ? (size_t)p->T : (size_t)p->B * p->T;
+    if (!std::strcmp(name, "p1_skip")) {
+        *offset = L.p1skip;
+        *bytes = 4 * (size_t)L.NTmax * p->H * 2;
+        return OSDN_OK;
+    }
+    if (!std::strcmp(name, "p1_mask")) {
+        *offset = L.pmask;
+        *bytes = 4 * Ttot * p->H * (p->K / 32);
+        return OSDN_OK;
+    }
+    return OSDN_INVALID_ARG;
 }
 
 int osdn_read_device_status(const void* workspace, int32_t* status_host)

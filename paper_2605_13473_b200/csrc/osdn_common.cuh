@@ -35,8 +35,15 @@ struct Table {
 struct WsLayout {
     size_t status;      // int32 device status word (+ padding)
     size_t table;       // ints, see carve_table
+    // phase 1 (shared by both kernel families)
+    size_t p1n;         // [T,H]          f32   max(|k|^2, eps), negated where the floor is active
+    size_t p1rho;       // [T,H]          f32   retention of the preconditioner
+    size_t p1flags;     // [NT,H,2]       u32   per token: the step maps d_min*1 to d_min*1, mask all zero
+    size_t dbound;      // [NT,H,K]       f32   preconditioner at chunk starts              (save only)
+    size_t p1skip;      // [NT,H,2]       u32   tokens the sequential pass skipped           (save only)
+    size_t pmask;       // [T,H,K/32]     u32   projection pass masks of processed tokens    (save only)
+    size_t dtraj;       // [T,H,K]        f32   d_t of processed tokens                      (save only)
     size_t ktil;        // [T,H,K]        f32   write keys
-    size_t dbound;      // [NT,H,K]       f32   preconditioner at chunk starts
     size_t Tm;          // [NT,H,64,64]   f32   UT inverse
     size_t P;           // [NT,H,64,64]   f32   masked, decayed q.ktil scores
     size_t W;           // [NT,H,64,K]    f32
@@ -70,8 +77,16 @@ inline WsLayout make_layout(const osdn_params& p, bool need_bwd)
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     L.status = take(256);
     L.table = take(sizeof(int) * (3 * (size_t)S + 1 + 3 * NT));
+    L.p1n = take(4 * Ttot * H);
+    L.p1rho = take(4 * Ttot * H);
+    L.p1flags = take(4 * NT * H * 2);
+    if (need_bwd) {
+        L.dbound = take(4 * NT * H * K);
+        L.p1skip = take(4 * NT * H * 2);
+        L.pmask = take(4 * Ttot * H * (K / 32));
+        L.dtraj = take(4 * Ttot * H * K);
+    }
     L.ktil = take(4 * Ttot * H * K);
-    L.dbound = take(4 * NT * H * K);
     L.Tm = take(4 * NT * H * CH * CH);
     L.P = take(4 * NT * H * CH * CH);
     L.W = take(4 * NT * H * CH * K);
@@ -101,6 +116,25 @@ inline Table carve_table(void* ws, const WsLayout& L)
     t.chunk_len = t.chunk_tok0 + L.NTmax;
     t.chunk_seq = t.chunk_len + L.NTmax;
     return t;
+}
+
+struct P1Regions {
+    float *n, *rho, *dbound, *dtraj;
+    unsigned *flags, *skipw, *pmask;
+};
+
+inline P1Regions carve_p1(void* ws, const WsLayout& L)
+{
+    char* w = static_cast<char*>(ws);
+    P1Regions r;
+    r.n = reinterpret_cast<float*>(w + L.p1n);
+    r.rho = reinterpret_cast<float*>(w + L.p1rho);
+    r.flags = reinterpret_cast<unsigned*>(w + L.p1flags);
+    r.dbound = reinterpret_cast<float*>(w + L.dbound);
+    r.skipw = reinterpret_cast<unsigned*>(w + L.p1skip);
+    r.pmask = reinterpret_cast<unsigned*>(w + L.pmask);
+    r.dtraj = reinterpret_cast<float*>(w + L.dtraj);
+    return r;
 }
 
 template <typename T> __device__ __forceinline__ float ldf(const T* p);
@@ -134,12 +168,15 @@ int simt_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void*
                  const Pointers& a, bool save, cudaStream_t st);
 int simt_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
                   const Pointers& a, cudaStream_t st);
-int simt_precond_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta,
-                        const float* retsrc, const float* precond_in, void* ktil_out,
-                        float* precond_out, cudaStream_t st);
-// Phase 1 alone with bf16 write keys in the packed [T,H,K] layout (used by the tensor-core path).
-int simt_phase1(const osdn_params& p, const Hyper& hy, const Pointers& a, const int* seq_chunk0,
-                void* ktil_bf16, float* dbound, cudaStream_t st);
+// Phase 1 (osdn_phase1.cu).  ktil: packed [T,H,K] write keys, fp32 or bf16.  `save` records what
+// the backward needs.  `bulk`: also finalise dk of skipped tokens (the tensor-core chunk kernel does
+// that itself).
+int phase1_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                   void* ktil, bool ktil_bf16, bool save, cudaStream_t st);
+int phase1_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                    const float* dktil, const float* dkread, bool bulk, cudaStream_t st);
+int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta, const float* retsrc,
+                  const float* precond_in, void* ktil_out, float* precond_out, cudaStream_t st);
 int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st);
 
 // Optional per-kernel timing (off by default): when enabled through osdn_stage_timing_enable, every

@@ -62,76 +62,11 @@ __global__ void build_table_kernel(int S, int T_dense, const int* __restrict__ c
     }
 }
 
-// ---------------------------------------------------------------------------------------
-// phase 1 forward: one warp per (sequence, head) chain, lanes own K/32 coordinates each
-// ---------------------------------------------------------------------------------------
-struct P1Args {
-    int S, H, T_dense;
-    const int* cu;           // nullable (dense)
-    const int* seq_chunk0;   // nullable (needed only with dbound)
-    const void* k;
-    const float *beta, *retsrc, *d0;
-    void* ktil;              // nullable
-    float *d_final, *dbound; // nullable
-    Hyper hy;
-};
-
 __device__ __forceinline__ float warp_sum(float x)
 {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
     return x;
-}
-
-template <typename TI, typename TO, int K>
-__global__ void __launch_bounds__(128) phase1_fwd_kernel(P1Args a)
-{
-    constexpr int R = K / 32;
-    const int lane = threadIdx.x & 31;
-    const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (chain >= a.S * a.H) return;
-    const int s = chain / a.H, h = chain % a.H;
-    const int t0 = a.cu ? a.cu[s] : s * a.T_dense;
-    const int len = a.cu ? max(a.cu[s + 1] - a.cu[s], 0) : a.T_dense;
-    const TI* kp = static_cast<const TI*>(a.k);
-    TO* kt = static_cast<TO*>(a.ktil);
-    float d[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) d[r] = a.d0 ? a.d0[((size_t)s * a.H + h) * K + lane + 32 * r] : 1.0f;
-    const Hyper hy = a.hy;
-    for (int i = 0; i < len; ++i) {
-        const size_t th = (size_t)(t0 + i) * a.H + h;
-        if (a.dbound && (i % CH) == 0) {
-            float* db = a.dbound + ((size_t)(a.seq_chunk0[s] + i / CH) * a.H + h) * K;
-#pragma unroll
-            for (int r = 0; r < R; ++r) db[lane + 32 * r] = d[r];
-        }
-        float kk[R], kap[R], sumk = 0.f, al = 0.f;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            kk[r] = ldf(kp + th * K + lane + 32 * r);
-            kap[r] = kk[r] * kk[r];
-            sumk += kap[r];
-            al += d[r] * kap[r];
-            if (kt) stf(kt + th * K + lane + 32 * r, d[r] * kk[r]);
-        }
-        sumk = warp_sum(sumk);
-        al = warp_sum(al);
-        const float n = fmaxf(sumk, hy.eps);
-        const float b = hy.beta_aware ? a.beta[th] : 1.0f;
-        const float c = hy.eta * b * (1.0f - b * al) / n;
-        const float rho = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float x = rho * d[r] + c * kap[r];
-            if (hy.clamp) x = fminf(fmaxf(x, hy.d_min), hy.d_max);
-            d[r] = x;
-        }
-    }
-    if (a.d_final) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) a.d_final[((size_t)s * a.H + h) * K + lane + 32 * r] = d[r];
-    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -654,122 +589,6 @@ __global__ void __launch_bounds__(NTH) chunk_local_bwd_kernel(ChunkArgs a)
     }
 }
 
-// ---------------------------------------------------------------------------------------
-// phase 1 backward: reverse sweep over the projected affine recurrence, one warp per chain.
-// Per chunk the forward scan is replayed from the saved chunk-start d.
-// ---------------------------------------------------------------------------------------
-struct P1BwdArgs {
-    int S, H;
-    Table tab;
-    const void* k;
-    const float *beta, *retsrc, *dbound, *dktil, *dkread, *dprecond_out;
-    void* dk;
-    float *dbeta, *dgate, *dlog_ret, *dprecond_in;
-    Hyper hy;
-};
-
-template <typename T, int K>
-__global__ void __launch_bounds__(64) phase1_bwd_kernel(P1BwdArgs a)
-{
-    constexpr int R = K / 32;
-    extern __shared__ float sm[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float* sd = sm + (size_t)warp * (CH * K + 4 * CH);   // d_t for the chunk [64][K]
-    float* sc = sd + CH * K;                              // c_t
-    float* sa = sc + CH;                                  // <d_t, kap_t>
-    float* sn = sa + CH;                                  // n_t (negative when the floor eps is active)
-    float* srho = sn + CH;
-    const int chain = blockIdx.x * (blockDim.x >> 5) + warp;
-    if (chain >= a.S * a.H) return;
-    const int s = chain / a.H, h = chain % a.H, H = a.H;
-    const Hyper hy = a.hy;
-    const T* kp = static_cast<const T*>(a.k);
-    T* dkp = static_cast<T*>(a.dk);
-    float lam[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-        lam[r] = a.dprecond_out ? a.dprecond_out[((size_t)s * H + h) * K + lane + 32 * r] : 0.f;
-    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
-    for (int c = c1 - 1; c >= c0; --c) {
-        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
-        float d[R];
-        unsigned long long mb[R];  // bit i: the projection passes gradient at token i
-#pragma unroll
-        for (int r = 0; r < R; ++r) d[r] = a.dbound[((size_t)c * H + h) * K + lane + 32 * r];
-#pragma unroll
-        for (int r = 0; r < R; ++r) mb[r] = 0ull;
-        for (int i = 0; i < len; ++i) {
-            const size_t th = (size_t)(tok0 + i) * H + h;
-            float kap[R], sumk = 0.f, al = 0.f;
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const float kk = ldf(kp + th * K + lane + 32 * r);
-                kap[r] = kk * kk;
-                sumk += kap[r];
-                al += d[r] * kap[r];
-                sd[i * K + lane + 32 * r] = d[r];
-            }
-            sumk = warp_sum(sumk);
-            al = warp_sum(al);
-            const float n = fmaxf(sumk, hy.eps);
-            const float b = hy.beta_aware ? a.beta[th] : 1.0f;
-            const float cc = hy.eta * b * (1.0f - b * al) / n;
-            const float rho = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
-            if (lane == 0) { sc[i] = cc; sa[i] = al; sn[i] = sumk > hy.eps ? n : -n; srho[i] = rho; }
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float x = rho * d[r] + cc * kap[r];
-                bool pass = true;
-                if (hy.clamp) {
-                    pass = (x >= hy.d_min) && (x <= hy.d_max);
-                    x = fminf(fmaxf(x, hy.d_min), hy.d_max);
-                }
-                if (pass) mb[r] |= 1ull << i;
-                d[r] = x;
-            }
-        }
-        __syncwarp();
-        for (int i = len - 1; i >= 0; --i) {
-            const size_t th = (size_t)(tok0 + i) * H + h;
-            float kk[R], kap[R], dt[R], dkt[R], drho = 0.f, dc = 0.f;
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                kk[r] = ldf(kp + th * K + lane + 32 * r);
-                kap[r] = kk[r] * kk[r];
-                dt[r] = sd[i * K + lane + 32 * r];
-                dkt[r] = a.dktil[th * K + lane + 32 * r];
-                if (!((mb[r] >> i) & 1ull)) lam[r] = 0.f;
-                drho += lam[r] * dt[r];
-                dc += lam[r] * kap[r];
-            }
-            drho = warp_sum(drho);
-            dc = warp_sum(dc);
-            const float nn = sn[i], n = fabsf(nn), cc = sc[i], al = sa[i], rho = srho[i];
-            const float b = hy.beta_aware ? a.beta[th] : 1.0f;
-            const float da = -hy.eta * b * b / n * dc;
-            const float db = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
-            const float dn = nn > 0.f ? -cc / n * dc : 0.f;
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const float dkap = cc * lam[r] + da * dt[r] + dn;
-                const float dkv = a.dkread[th * K + lane + 32 * r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
-                stf(dkp + th * K + lane + 32 * r, dkv);
-                lam[r] = rho * lam[r] + da * kap[r] + kk[r] * dkt[r];
-            }
-            if (lane == 0) {
-                if (hy.beta_aware) a.dbeta[th] += db;
-                if (hy.apf_mode == 1) a.dgate[th] += rho * drho;
-                if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
-            }
-        }
-        __syncwarp();
-    }
-    if (a.dprecond_in) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) a.dprecond_in[((size_t)s * H + h) * K + lane + 32 * r] = lam[r];
-    }
-}
-
 template <typename F> bool set_smem(F* kernel, size_t bytes)
 {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
@@ -786,18 +605,9 @@ int fwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
     int launches = 0;
     const int S = L.S, H = p.H;
     {
-        P1Args pa{};
-        pa.S = S; pa.H = H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
-        pa.seq_chunk0 = tab.seq_chunk0;
-        pa.k = a.k; pa.beta = a.beta;
-        pa.retsrc = p.apf_mode == 2 ? a.log_ret : a.gate;
-        pa.d0 = a.precond_in; pa.ktil = w + L.ktil; pa.d_final = a.precond_out;
-        pa.dbound = reinterpret_cast<float*>(w + L.dbound);
-        pa.hy = hy;
-        const int chains = S * H;
-        stage_mark(st, "phase1_fwd");
-        phase1_fwd_kernel<T, float, K><<<(chains + 3) / 4, 128, 0, st>>>(pa);
-        ++launches;
+        const int n1 = phase1_forward(p, hy, L, ws, a, w + L.ktil, false, save, st);
+        if (n1 < 0) return -1;
+        launches += n1;
     }
     {
         ChunkArgs ca{};
@@ -866,30 +676,12 @@ int bwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
         ++launches;
     }
     {
-        P1BwdArgs pb{};
-        pb.S = S; pb.H = H; pb.tab = tab; pb.k = a.k; pb.beta = a.beta;
-        pb.retsrc = p.apf_mode == 2 ? a.log_ret : a.gate;
-        pb.dbound = F(L.dbound); pb.dktil = F(L.dktil); pb.dkread = F(L.dkread);
-        pb.dprecond_out = a.dprecond_out; pb.dk = a.dk; pb.dbeta = a.dbeta; pb.dgate = a.dgate;
-        pb.dlog_ret = a.dlog_ret; pb.dprecond_in = a.dprecond_in; pb.hy = hy;
-        const size_t smem = sizeof(float) * 2 * (CH * K + 4 * CH);
-        if (!set_smem(phase1_bwd_kernel<T, K>, smem)) return -1;
-        const int chains = S * H;
-        stage_mark(st, "phase1_bwd");
-        phase1_bwd_kernel<T, K><<<(chains + 1) / 2, 64, smem, st>>>(pb);
-        ++launches;
+        const int n1 = phase1_backward(p, hy, L, ws, a, F(L.dktil), F(L.dkread), true, st);
+        if (n1 < 0) return -1;
+        launches += n1;
     }
     stage_end(st);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
-}
-
-template <typename TI, typename TO>
-int p1_dispatch(int K, const P1Args& pa, cudaStream_t st)
-{
-    const int chains = pa.S * pa.H;
-    if (K == 64) phase1_fwd_kernel<TI, TO, 64><<<(chains + 3) / 4, 128, 0, st>>>(pa);
-    else phase1_fwd_kernel<TI, TO, 128><<<(chains + 3) / 4, 128, 0, st>>>(pa);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace
@@ -928,32 +720,6 @@ int simt_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void
                   cudaStream_t st)
 {
     OSDN_DISPATCH(bwd_impl, p, hy, L, ws, a, st);
-}
-
-int simt_phase1(const osdn_params& p, const Hyper& hy, const Pointers& a, const int* seq_chunk0,
-                void* ktil_bf16, float* dbound, cudaStream_t st)
-{
-    P1Args pa{};
-    pa.S = p.nseq > 0 ? p.nseq : p.B;
-    pa.H = p.H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
-    pa.seq_chunk0 = seq_chunk0;
-    pa.k = a.k; pa.beta = a.beta; pa.retsrc = p.apf_mode == 2 ? a.log_ret : a.gate;
-    pa.d0 = a.precond_in; pa.ktil = ktil_bf16; pa.d_final = a.precond_out; pa.dbound = dbound; pa.hy = hy;
-    stage_mark(st, "phase1_fwd");
-    return p1_dispatch<__nv_bfloat16, __nv_bfloat16>(p.K, pa, st);
-}
-
-int simt_precond_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta,
-                        const float* retsrc, const float* precond_in, void* ktil_out, float* precond_out,
-                        cudaStream_t st)
-{
-    P1Args pa{};
-    pa.S = p.nseq > 0 ? p.nseq : p.B;
-    pa.H = p.H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
-    pa.k = k; pa.beta = beta; pa.retsrc = retsrc; pa.d0 = precond_in; pa.ktil = ktil_out;
-    pa.d_final = precond_out; pa.hy = hy;
-    if (p.io_dtype == OSDN_FP32) return p1_dispatch<float, float>(p.K, pa, st);
-    return p1_dispatch<__nv_bfloat16, __nv_bfloat16>(p.K, pa, st);
 }
 
 }  // namespace osdn

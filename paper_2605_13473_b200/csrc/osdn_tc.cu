@@ -35,7 +35,7 @@ constexpr uint32_t BOX = 8192;   // one [64 rows x 128 B] box
 enum { ERR_TMA = 101, ERR_MMA1 = 102, ERR_MMA2 = 103, ERR_CHAIN_TMA = 111, ERR_CHAIN_MMA1 = 112, ERR_CHAIN_MMA2 = 113 };
 
 struct TcLayout {
-    size_t ktil, dbound, WT, Tb, Tm, P, Qg, Sn, dUT, ddUT, dSn, dktil, dkread, total;
+    size_t ktil, WT, Tb, Tm, P, Qg, Sn, dUT, ddUT, dSn, dktil, dkread, total;
 };
 
 TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
@@ -47,7 +47,6 @@ TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
     auto take = [&](size_t b) { size_t o = off; off = align_up(off + b, 1024); return o; };
     off = align_up(off, 1024);
     t.ktil = take(Ttot * H * KD * 2);
-    t.dbound = take(NT * H * KD * 4);
     t.WT = take(NT * H * 16384);
     t.Tb = take(NT * H * 8192);
     t.Tm = take(NT * H * 8192);
@@ -633,7 +632,7 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
     int launches = 0;
 
     // phase 1 on CUDA cores: bf16 write keys, chunk-start preconditioners
-    const int n1 = simt_phase1(p, hy, a, tab.seq_chunk0, w + t.ktil, reinterpret_cast<float*>(w + t.dbound), st);
+    const int n1 = phase1_forward(p, hy, L, ws, a, w + t.ktil, true, save, st);
     if (n1 < 0) return -1;
     launches += n1;
 

@@ -62,6 +62,8 @@ def subset_result(res, seqs, heads, tok_t, hd):
     sq = torch.as_tensor(list(seqs))
     out = {}
     for k, v in res.items():
+        if v is None:
+            continue
         v = torch.as_tensor(v)
         if k in ("final_state", "precond_out", "dinit_state", "dprecond_in"):
             out[k] = v.index_select(0, sq).index_select(1, hd).numpy()
@@ -70,10 +72,26 @@ def subset_result(res, seqs, heads, tok_t, hd):
     return out
 
 
-def oracle_all(inp, bwd: bool):
-    ref = oracle.fwd_inputs(inp)
-    if bwd:
-        ref.update(oracle.bwd_inputs(inp))
+TIE = 2e-6   # |pre-projection value - box face| below which fp32 and fp64 may decide differently
+
+
+def oracle_all(inp, bwd: bool, gpu_masks=None):
+    """Oracle forward (and backward).  The gradient is discontinuous where a pre-projection value of
+    the preconditioner touches a face of the box.  Where the oracle's fp64 value is within TIE of a
+    face the decision is not unique at fp32 resolution: there (and only there) the oracle's reverse
+    sweep takes the decision the CUDA path took (`gpu_masks`); everywhere else the two must agree."""
+    if not bwd:
+        return oracle.fwd_inputs(inp)
+    ref = oracle.fwd_inputs(inp, want_margin=True)
+    override = None
+    if gpu_masks is not None and inp.hyper.clamp:
+        gm = np.asarray(gpu_masks, dtype=np.uint8)
+        near = ref["margin"] <= TIE
+        disagree = (gm != ref["mask"]) & ~near
+        assert not disagree.any(), f"{int(disagree.sum())} projection decisions differ away from any tie"
+        override = np.where(near, gm, 255).astype(np.uint8)
+        ref["near_ties"] = int(near.sum())
+    ref.update(oracle.bwd_inputs(inp, mask_override=override))
     return ref
 
 

@@ -15,8 +15,8 @@ REPORT = {}
 def _sampled(inp, bwd, seqs, heads, label):
     got = run_inputs_bwd(inp) if bwd else run_inputs_fwd(inp)
     sub, tok_t, hd = parity.subset(inp, seqs, heads)
-    ref = parity.oracle_all(sub, bwd)
     got_sub = parity.subset_result(got, seqs, heads, tok_t, hd)
+    ref = parity.oracle_all(sub, bwd, got_sub.get("projection_masks"))
     keys = parity.FWD_KEYS + (parity.BWD_KEYS if bwd else ())
     parity.compare(got_sub, ref, inp.io_dtype, keys, label, report=REPORT)
 

@@ -28,7 +28,7 @@ def teardown_module(module):
 
 def _check(inp, bwd, label, flags=0, tol=None):
     got = run_inputs_bwd(inp, flags=flags) if bwd else run_inputs_fwd(inp, flags=flags)
-    ref = parity.oracle_all(inp, bwd)
+    ref = parity.oracle_all(inp, bwd, got.get("projection_masks"))
     keys = parity.FWD_KEYS + (parity.BWD_KEYS if bwd else ())
     return parity.compare(got, ref, inp.io_dtype, keys, label, tol=tol, report=REPORT)
 

@@ -159,3 +159,26 @@ def test_backward_segment_checkpointing_is_transparent():
         np.testing.assert_allclose(np.concatenate([b1[key], b2[key]]), full[key], atol=1e-12)
     np.testing.assert_allclose(b1["dinit_state"], full["dinit_state"], atol=1e-12)
     np.testing.assert_allclose(b1["dprecond_in"], full["dprecond_in"], atol=1e-12)
+
+
+def test_mask_override_only_changes_what_it_forces():
+    hy = OsdnHyper(eta=0.5, apf_mode=1)
+    lens, x, cot = _case(600, hy, H=1, K=6, V=4, lens=[20], unit=True)
+    args = (hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], cot["out"], None, x["init_state"],
+            x["precond_in"], cot["final_state"], cot["precond_out"])
+    base = oracle.bwd(*args)
+    f = oracle.fwd(hy, lens, x["q"], x["k"], x["v"], x["beta"], x["gate"], None, x["init_state"],
+                   x["precond_in"], want_margin=True)
+    same = oracle.bwd(*args, mask_override=f["mask"])
+    for key in base:
+        np.testing.assert_allclose(base[key], same[key], atol=0)
+    none = oracle.bwd(*args, mask_override=np.full(f["mask"].shape, 255, np.uint8))
+    for key in base:
+        np.testing.assert_allclose(base[key], none[key], atol=0)
+    flipped = f["mask"].copy()
+    flipped[10, 0, 2] ^= 1
+    other = oracle.bwd(*args, mask_override=flipped)
+    assert np.abs(other["dk"] - base["dk"]).max() > 0
+    np.testing.assert_allclose(other["dq"], base["dq"], atol=0)      # phase 2 is untouched
+    np.testing.assert_allclose(other["dk"][11:], base["dk"][11:], atol=0)  # later tokens too
+    assert f["margin"].min() >= 0 and f["mask"].mean() < 1.0
