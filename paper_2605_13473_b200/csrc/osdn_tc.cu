@@ -607,6 +607,691 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     if (warp == 0) tmem_dealloc(tb, 512);
 }
 
+// ---------------------------------------------------------------------------------------------
+// state chain, backward (reverse over chunks); dS (V x K, fp32) resident in tensor memory
+//   ddU^T = dO^T P' + rho_i (dS Ktil^T) ;   dS <- gamma_C dS + dO^T Qg - ddU^T W
+// ---------------------------------------------------------------------------------------------
+struct TcChainBwdArgs {
+    int H;
+    Table tab;
+    const float *gate, *dfinal_state;
+    float* dinit_state;
+    const uint8_t *WT, *P, *Qg;
+    uint8_t *dSn, *ddUT;
+    int* status;
+};
+
+constexpr uint32_t BS_DO = 0, BS_KT = 16384, BS_P = 32768, BS_QG = 40960, BS_WT = 57344;
+constexpr uint32_t BSTAGE_BYTES = 73728;
+constexpr size_t CB_SMEM = 2 * BSTAGE_BYTES + 32768 + 16384 + 1024;
+
+__global__ void __launch_bounds__(CF_THREADS, 1)
+tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_constant__ CUtensorMap tmKt,
+                    TcChainBwdArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sm = align1024(smem_raw);
+    uint8_t* sStage = sm;
+    uint8_t* sdS = sm + 2 * BSTAGE_BYTES;       // dS as bf16, K-major, 2 k-halves x [128 x 128 B]
+    uint8_t* sddU = sdS + 32768;                // ddU^T, K-major [v][i]
+    __shared__ uint64_t bar_full[2], bar_mma1, bar_mma2;
+    __shared__ uint32_t tmem_base;
+    __shared__ float sRho[2][CH], sGC[2], sgraw[CH];
+
+    const int chain = blockIdx.x, H = a.H;
+    const int s = chain / H, h = chain % H;
+    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int quad = warp & 3, colhalf = warp >> 2;
+    const int v = quad * 32 + lane;
+    float* dini = a.dinit_state ? a.dinit_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
+    const float* dfin = a.dfinal_state ? a.dfinal_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
+    if (c1 <= c0) {
+        if (dini)
+            for (int x = 0; x < 64; ++x) dini[x] = dfin ? dfin[x] : 0.f;
+        return;
+    }
+    if (tid == 0) {
+        mbar_init(&bar_full[0], 1);
+        mbar_init(&bar_full[1], 1);
+        mbar_init(&bar_mma1, 1);
+        mbar_init(&bar_mma2, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(&tmem_base, 256);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t tS = tb, tA1 = tb + 128, tA2 = tb + 192;
+
+    auto issue_loads = [&](int c, int st) {
+        const int tok0 = a.tab.chunk_tok0[c];
+        const size_t tile = (size_t)c * H + h;
+        uint8_t* d = sStage + st * BSTAGE_BYTES;
+        mbar_expect_tx(&bar_full[st], BSTAGE_BYTES);
+        bulk_load(d + BS_P, a.P + tile * 8192, 8192, &bar_full[st]);
+        bulk_load(d + BS_QG, a.Qg + tile * 16384, 16384, &bar_full[st]);
+        bulk_load(d + BS_WT, a.WT + tile * 16384, 16384, &bar_full[st]);
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_load_2d(d + BS_DO + hf * BOX, &tmDO, h * KD + hf * 64, tok0, &bar_full[st]);
+            tma_load_2d(d + BS_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
+        }
+    };
+    auto gate_vectors = [&](int c, int st) {
+        if (tid < CH) {
+            const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+            sgraw[tid] = tid < len ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
+        }
+        __syncthreads();
+        if (tid < CH) {
+            float G = 0.f, tot = 0.f;
+            for (int j = 0; j < CH; ++j) {
+                const float g = sgraw[j];
+                tot += g;
+                if (j <= tid) G += g;
+            }
+            sRho[st][tid] = __expf(tot - G);
+            if (tid == 0) sGC[st] = __expf(tot);
+        }
+    };
+
+    if (tid == 0) issue_loads(c1 - 1, 0);
+    for (int cb = 0; cb < 4; ++cb) {
+        uint32_t r[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(dfin ? dfin[cb * 16 + x] : 0.f);
+        tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+    }
+    tmem_st_wait();
+    gate_vectors(c1 - 1, 0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    bool ok = true;
+    for (int c = c1 - 1; c >= c0; --c) {
+        const int n = c1 - 1 - c, st = n & 1;
+        const int len = a.tab.chunk_len[c];
+        const size_t tile = (size_t)c * H + h;
+        uint8_t* d = sStage + st * BSTAGE_BYTES;
+        if (tid == 0 && c > c0) issue_loads(c - 1, st ^ 1);
+
+        // ---- E0: dS (cotangent at the chunk end) -> bf16 operand + saved copy; decay -----------
+        {
+            const float gC = sGC[st];
+            uint8_t* Sg = a.dSn + tile * 32768 + colhalf * 16384;
+            for (int cb = 0; cb < 4; ++cb) {
+                uint32_t r[16];
+                tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
+                    w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
+                    w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
+                    w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
+                    const uint32_t off = sw128_chunk(v, cb * 2 + c2);
+                    *reinterpret_cast<uint4*>(sdS + colhalf * 16384 + off) = w;
+                    *reinterpret_cast<uint4*>(Sg + off) = w;
+                }
+#pragma unroll
+                for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
+                tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+            }
+            tmem_st_wait();
+        }
+        ok = ok && mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
+        if (len < CH) {
+            for (int hf = 0; hf < 2; ++hf) {
+                zero_tail_rows(d + BS_DO + hf * BOX, len, tid, CF_THREADS);
+                zero_tail_rows(d + BS_KT + hf * BOX, len, tid, CF_THREADS);
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+
+        if (tid == 0 && ok) {
+            tc_fence_after();
+            {   // acc1 = dO^T P'
+                const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN);
+                const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_P, 0);
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tA1, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k), idesc, k > 0);
+            }
+            {   // acc2 = dS Ktil^T
+                const uint32_t idesc = make_idesc(128, 64);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tA2, desc_advance(desc_kmajor(sdS + (k >> 2) * 16384), 32 * (k & 3)),
+                           desc_advance(desc_kmajor(d + BS_KT + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
+            }
+            mma_commit(&bar_mma1);
+        }
+        ok = ok && mbar_wait(&bar_mma1, n & 1, a.status, ERR_CHAIN_MMA1);
+        tc_fence_after();
+
+        // ---- E1: ddU^T = acc1 + rho_i acc2 ---------------------------------------------------
+        {
+            uint8_t* dg = a.ddUT + tile * 16384;
+            for (int cb = 0; cb < 2; ++cb) {
+                uint32_t r1[16], r2[16];
+                tmem_ld16(tA1 + lane_addr + colhalf * 32 + cb * 16, r1);
+                tmem_ld16(tA2 + lane_addr + colhalf * 32 + cb * 16, r2);
+                tmem_ld_wait();
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    float f[8];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x)
+                        f[x] = __uint_as_float(r1[c2 * 8 + x]) +
+                               sRho[st][colhalf * 32 + cb * 16 + c2 * 8 + x] * __uint_as_float(r2[c2 * 8 + x]);
+                    const uint32_t off = sw128_chunk(v, colhalf * 4 + cb * 2 + c2);
+                    const uint4 w = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                                               pack_bf16(f[6], f[7]));
+                    *reinterpret_cast<uint4*>(sddU + off) = w;
+                    *reinterpret_cast<uint4*>(dg + off) = w;
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+
+        if (tid == 0 && ok) {
+            tc_fence_after();
+            {   // dS += dO^T Qg
+                const uint32_t idesc = make_idesc(128, 128, IDESC_A_MN | IDESC_B_MN);
+                const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_QG, BOX);
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tS, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k), idesc, 1);
+            }
+            {   // dS -= ddU^T W
+                const uint32_t idesc = make_idesc(128, 128, IDESC_A_NEG);
+                const uint64_t da0 = desc_kmajor(sddU), db0 = desc_kmajor(d + BS_WT);
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, 1);
+            }
+            mma_commit(&bar_mma2);
+        }
+        if (c > c0) gate_vectors(c - 1, st ^ 1);
+        ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
+        tc_fence_after();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+    if (dini && ok) {
+        for (int cb = 0; cb < 4; ++cb) {
+            uint32_t r[16];
+            tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 16; ++x) dini[cb * 16 + x] = __uint_as_float(r[x]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tb, 256);
+}
+
+// ---------------------------------------------------------------------------------------------
+// chunk-local backward.  Feature-major ("transposed") accumulators: lane = feature, column = token.
+//   phase A : rawkk = K Ktil^T ; dP' = dO dU^T ; dQ1^T = S^T dO^T ; dKtr^T = dS^T dU ; dW^T = -S^T ddU
+//   phase B : dT = (dW K^T) beta gamma + (ddU V^T) beta ; dKb^T = dW^T T ; dVb^T = ddU^T T ;
+//             dq2^T = Ktil^T M1^T ; dktil^T = Q^T M1            (M1 = scale Gamma (.) lower(dP'))
+//   phase C : Y = T^T dT        phase D : Z = Y T^T, dA = -strictLower(Z), M2 = dA beta_i Gamma_ij
+//   phase E : dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T
+//   final   : dq = scale gamma dQ1 + dq2 ; dktil += rho dKtr ; dk_read = dkr + beta gamma dKb ;
+//             dv = beta dVb ; dbeta, dgate from the products of the gradients with their inputs
+// ---------------------------------------------------------------------------------------------
+struct TcChunkBwdArgs {
+    int H;
+    Table tab;
+    const float *beta, *gate;
+    float scale, d_min;
+    const uint8_t *Tm, *Sn, *dSn, *dUT, *ddUT;
+    const unsigned* skipw;
+    __nv_bfloat16 *dq, *dk, *dv;
+    float *dbeta, *dgate, *dktil, *dkread;
+    int* status;
+};
+
+constexpr int CBW_THREADS = 256;
+constexpr uint32_t R_Q = 0, R_K = 16384, R_KT = 32768, R_V = 49152, R_DO = 65536, R_DU = 81920, R_DDU = 98304,
+                   R_T = 114688, R_S = 122880, R_DS = 155648, R_RAW = 188416;
+constexpr uint32_t R_DWT = R_DO;                 // dW^T image replaces dO after phase A
+constexpr uint32_t R_M1 = R_S, R_M2 = R_S + 8192, R_DT = R_S + 16384, R_Y = R_S + 24576;
+constexpr size_t CBW_SMEM = R_RAW + CH * LC * 4 + 1024;
+
+__global__ void __launch_bounds__(CBW_THREADS, 1)
+tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmV,
+                    const __grid_constant__ CUtensorMap tmDO, TcChunkBwdArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sm = align1024(smem_raw);
+    float* sRaw = reinterpret_cast<float*>(sm + R_RAW);       // Gamma_ij <k_i, ktil_j>, j < i
+    __shared__ uint64_t bar_tma, bar_mma[5];
+    __shared__ uint32_t tmem_base;
+    __shared__ float sG[CH], sBeta[CH], sg[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
+    __shared__ float sRsum;
+
+    const int c = blockIdx.x, h = blockIdx.y, H = a.H;
+    const int len = a.tab.chunk_len[c];
+    if (len == 0) return;
+    const int tok0 = a.tab.chunk_tok0[c];
+    const size_t tile = (size_t)c * H + h;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int quad = warp & 3, colhalf = warp >> 2;
+    const int f = quad * 32 + lane;                 // feature (k or v) owned in 128-lane accumulators
+    const int row64 = quad * 16 + (lane & 15);      // token row owned in 64-row accumulators (lanes 0-15)
+    const bool row_active = lane < 16;
+
+    if (tid == 0) {
+        mbar_init(&bar_tma, 1);
+        for (int i = 0; i < 5; ++i) mbar_init(&bar_mma[i], 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(&tmem_base, 512);
+    if (tid < CH) {
+        const bool in = tid < len;
+        sg[tid] = in ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
+        sBeta[tid] = in ? a.beta[(size_t)(tok0 + tid) * H + h] : 0.f;
+        sdB[tid] = 0.f;
+        sdG[tid] = 0.f;
+    }
+    if (tid == 0) sRsum = 0.f;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+
+    if (tid == 0) {
+        mbar_expect_tx(&bar_tma, 10 * BOX + 16384 + 16384 + 8192 + 32768 + 32768);
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_load_2d(sm + R_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_tma);
+            tma_load_2d(sm + R_K + hf * BOX, &tmK, h * KD + hf * 64, tok0, &bar_tma);
+            tma_load_2d(sm + R_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_tma);
+            tma_load_2d(sm + R_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_tma);
+            tma_load_2d(sm + R_DO + hf * BOX, &tmDO, h * KD + hf * 64, tok0, &bar_tma);
+        }
+        bulk_load(sm + R_DU, a.dUT + tile * 16384, 16384, &bar_tma);
+        bulk_load(sm + R_DDU, a.ddUT + tile * 16384, 16384, &bar_tma);
+        bulk_load(sm + R_T, a.Tm + tile * 8192, 8192, &bar_tma);
+        bulk_load(sm + R_S, a.Sn + tile * 32768, 32768, &bar_tma);
+        bulk_load(sm + R_DS, a.dSn + tile * 32768, 32768, &bar_tma);
+    }
+    if (tid < CH) {
+        float acc = 0.f, tot = 0.f;
+        for (int j = 0; j < CH; ++j) {
+            tot += sg[j];
+            if (j <= tid) acc += sg[j];
+        }
+        sG[tid] = acc;
+        sGam[tid] = __expf(acc);
+        sRho[tid] = __expf(tot - acc);
+    }
+    bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
+    if (len < CH) {
+        for (int hf = 0; hf < 2; ++hf) {
+            zero_tail_rows(sm + R_Q + hf * BOX, len, tid, CBW_THREADS);
+            zero_tail_rows(sm + R_K + hf * BOX, len, tid, CBW_THREADS);
+            zero_tail_rows(sm + R_KT + hf * BOX, len, tid, CBW_THREADS);
+            zero_tail_rows(sm + R_V + hf * BOX, len, tid, CBW_THREADS);
+            zero_tail_rows(sm + R_DO + hf * BOX, len, tid, CBW_THREADS);
+        }
+        fence_proxy_async();
+    }
+    __syncthreads();
+
+    // tensor memory columns
+    const uint32_t cRAW = 0, cDP = 64, cDQ1 = 128, cDKTR = 192, cDW = 256, cDTA = 320, cDTB = 384, cDKT = 448;
+    const uint32_t cDKB = 256, cDVB = 64, cDQ2 = 0, cY = 320, cZ = 384, cDKR = 320;
+
+    // ---- phase A -------------------------------------------------------------------------------
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        for (int k = 0; k < 8; ++k) {   // rawkk[i][j] = <k_i, ktil_j>          (M = 64)
+            mma_ss(tb + cRAW, desc_advance(desc_kmajor(sm + R_K + (k >> 2) * BOX), 32 * (k & 3)),
+                   desc_advance(desc_kmajor(sm + R_KT + (k >> 2) * BOX), 32 * (k & 3)), make_idesc(64, 64), k > 0);
+        }
+        {   // dP'[i][j] = sum_v dO[i][v] dU[j][v]                               (M = 64)
+            const uint64_t db0 = desc_mnmajor(sm + R_DU, 0);
+            for (int k = 0; k < 8; ++k)
+                mma_ss(tb + cDP, desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
+                       desc_advance(db0, 2048 * k), make_idesc(64, 64, IDESC_B_MN), k > 0);
+        }
+        {   // dQ1^T[k][i] = sum_v S[v][k] dO[i][v]
+            const uint64_t da0 = desc_mnmajor(sm + R_S, 16384);
+            for (int k = 0; k < 8; ++k)
+                mma_ss(tb + cDQ1, desc_advance(da0, 2048 * k),
+                       desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
+                       make_idesc(128, 64, IDESC_A_MN), k > 0);
+        }
+        {   // dKtr^T[k][j] = sum_v dS[v][k] dU[j][v]
+            const uint64_t da0 = desc_mnmajor(sm + R_DS, 16384), db0 = desc_mnmajor(sm + R_DU, 0);
+            for (int k = 0; k < 8; ++k)
+                mma_ss(tb + cDKTR, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
+                       make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
+        }
+        {   // dW^T[k][i] = -sum_v S[v][k] ddU[i][v]
+            const uint64_t da0 = desc_mnmajor(sm + R_S, 16384), db0 = desc_mnmajor(sm + R_DDU, 0);
+            for (int k = 0; k < 8; ++k)
+                mma_ss(tb + cDW, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
+                       make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN | IDESC_A_NEG), k > 0);
+        }
+        mma_commit(&bar_mma[0]);
+    }
+    // <dS, S>_F while the tensor core works (both images share the same layout)
+    {
+        float part = 0.f;
+        for (int e = tid; e < 2048; e += CBW_THREADS) {
+            const uint4 x = *reinterpret_cast<const uint4*>(sm + R_S + e * 16);
+            const uint4 y = *reinterpret_cast<const uint4*>(sm + R_DS + e * 16);
+            const __nv_bfloat162* px = reinterpret_cast<const __nv_bfloat162*>(&x);
+            const __nv_bfloat162* py = reinterpret_cast<const __nv_bfloat162*>(&y);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 fx = __bfloat1622float2(px[q]), fy = __bfloat1622float2(py[q]);
+                part = fmaf(fx.x, fy.x, part);
+                part = fmaf(fx.y, fy.y, part);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        if (lane == 0) sRed[warp] = part;
+    }
+    ok = ok && mbar_wait(&bar_mma[0], 0, a.status, ERR_MMA1);
+    tc_fence_after();
+    __syncthreads();   // every thread is done reading S / dS before their space is reused
+    // epilogue A
+    {
+        // rawkk, dP' (64-row accumulators: rows in lanes 0-15 of each quadrant)
+        const int i = row64;
+        const float Gi = sG[i];
+        for (int cb = 0; cb < 2; ++cb) {
+            uint32_t r1[16], r2[16];
+            const int j0 = colhalf * 32 + cb * 16;
+            tmem_ld16(tb + cRAW + lane_addr + j0, r1);
+            tmem_ld16(tb + cDP + lane_addr + j0, r2);
+            tmem_ld_wait();
+            if (row_active) {
+                float m1[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const int j = j0 + x;
+                    const float gm = j <= i ? __expf(Gi - sG[j]) : 0.f;
+                    sRaw[i * LC + j] = j < i ? gm * __uint_as_float(r1[x]) : 0.f;
+                    m1[x] = a.scale * gm * __uint_as_float(r2[x]);
+                }
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2)
+                    *reinterpret_cast<uint4*>(sm + R_M1 + sw128_chunk(i, (j0 >> 3) + c2)) =
+                        make_uint4(pack_bf16(m1[c2 * 8 + 0], m1[c2 * 8 + 1]), pack_bf16(m1[c2 * 8 + 2], m1[c2 * 8 + 3]),
+                                   pack_bf16(m1[c2 * 8 + 4], m1[c2 * 8 + 5]), pack_bf16(m1[c2 * 8 + 6], m1[c2 * 8 + 7]));
+            }
+        }
+        // dW^T -> bf16 image [rows k][cols i]
+        for (int cb = 0; cb < 2; ++cb) {
+            uint32_t r[16];
+            tmem_ld16(tb + cDW + lane_addr + colhalf * 32 + cb * 16, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c2 = 0; c2 < 2; ++c2)
+                *reinterpret_cast<uint4*>(sm + R_DWT + sw128_chunk(f, colhalf * 4 + cb * 2 + c2)) = make_uint4(
+                    pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1])),
+                    pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3])),
+                    pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5])),
+                    pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7])));
+        }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- phase B -------------------------------------------------------------------------------
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        {   // dT_a[i][j] = sum_k dW[i][k] K[j][k]                               (M = 64)
+            const uint64_t da0 = desc_mnmajor(sm + R_DWT, 0);
+            for (int k = 0; k < 8; ++k)
+                mma_ss(tb + cDTA, desc_advance(da0, 2048 * k),
+                       desc_advance(desc_kmajor(sm + R_K + (k >> 2) * BOX), 32 * (k & 3)),
+                       make_idesc(64, 64, IDESC_A_MN), k > 0);
+        }
+        {   // dT_b[i][j] = sum_v ddU[i][v] V[j][v]                              (M = 64)
+            const uint64_t da0 = desc_mnmajor(sm + R_DDU, 0);
+            for (int k = 0; k < 8; ++k)
+                mma_ss(tb + cDTB, desc_advance(da0, 2048 * k),
+                       desc_advance(desc_kmajor(sm + R_V + (k >> 2) * BOX), 32 * (k & 3)),
+                       make_idesc(64, 64, IDESC_A_MN), k > 0);
+        }
+        {   // dKb^T[k][j] = sum_i dW^T[k][i] T[i][j] ;  dVb^T[v][j] = sum_i ddU^T[v][i] T[i][j]
+            const uint64_t db0 = desc_mnmajor(sm + R_T, 0);
+            const uint64_t da0 = desc_kmajor(sm + R_DWT), da1 = desc_kmajor(sm + R_DDU);
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tb + cDKB, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k),
+                       make_idesc(128, 64, IDESC_B_MN), k > 0);
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tb + cDVB, desc_advance(da1, 32 * k), desc_advance(db0, 2048 * k),
+                       make_idesc(128, 64, IDESC_B_MN), k > 0);
+        }
+        {   // dq2^T[k][i] = sum_j Ktil[j][k] M1[i][j] ;  dktil^T[k][j] = sum_i Q[i][k] M1[i][j]
+            const uint64_t da0 = desc_mnmajor(sm + R_KT, BOX), da1 = desc_mnmajor(sm + R_Q, BOX);
+            const uint64_t dbk = desc_kmajor(sm + R_M1), dbm = desc_mnmajor(sm + R_M1, 0);
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tb + cDQ2, desc_advance(da0, 2048 * k), desc_advance(dbk, 32 * k),
+                       make_idesc(128, 64, IDESC_A_MN), k > 0);
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tb + cDKT, desc_advance(da1, 2048 * k), desc_advance(dbm, 2048 * k),
+                       make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
+        }
+        mma_commit(&bar_mma[1]);
+    }
+    ok = ok && mbar_wait(&bar_mma[1], 0, a.status, ERR_MMA2);
+    tc_fence_after();
+    {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j]
+        const int i = row64;
+        for (int cb = 0; cb < 2; ++cb) {
+            uint32_t r1[16], r2[16];
+            const int j0 = colhalf * 32 + cb * 16;
+            tmem_ld16(tb + cDTA + lane_addr + j0, r1);
+            tmem_ld16(tb + cDTB + lane_addr + j0, r2);
+            tmem_ld_wait();
+            if (row_active) {
+                float t[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const int j = j0 + x;
+                    t[x] = sBeta[j] * (sGam[j] * __uint_as_float(r1[x]) + __uint_as_float(r2[x]));
+                }
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2)
+                    *reinterpret_cast<uint4*>(sm + R_DT + sw128_chunk(i, (j0 >> 3) + c2)) =
+                        make_uint4(pack_bf16(t[c2 * 8 + 0], t[c2 * 8 + 1]), pack_bf16(t[c2 * 8 + 2], t[c2 * 8 + 3]),
+                                   pack_bf16(t[c2 * 8 + 4], t[c2 * 8 + 5]), pack_bf16(t[c2 * 8 + 6], t[c2 * 8 + 7]));
+            }
+        }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] -----------------------------------------------
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        const uint64_t da0 = desc_mnmajor(sm + R_T, 0), db0 = desc_mnmajor(sm + R_DT, 0);
+        for (int k = 0; k < 4; ++k)
+            mma_ss(tb + cY, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
+                   make_idesc(64, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
+        mma_commit(&bar_mma[2]);
+    }
+    ok = ok && mbar_wait(&bar_mma[2], 0, a.status, ERR_MMA2);
+    tc_fence_after();
+    {
+        const int i = row64;
+        for (int cb = 0; cb < 2; ++cb) {
+            uint32_t r[16];
+            const int j0 = colhalf * 32 + cb * 16;
+            tmem_ld16(tb + cY + lane_addr + j0, r);
+            tmem_ld_wait();
+            if (row_active) {
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2)
+                    *reinterpret_cast<uint4*>(sm + R_Y + sw128_chunk(i, (j0 >> 3) + c2)) = make_uint4(
+                        pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1])),
+                        pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3])),
+                        pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5])),
+                        pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7])));
+            }
+        }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- phase D: Z[a][b] = sum_c Y[a][c] T[b][c] ; dA = -strictLower(Z) --------------------------
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        const uint64_t da0 = desc_kmajor(sm + R_Y), db0 = desc_kmajor(sm + R_T);
+        for (int k = 0; k < 4; ++k)
+            mma_ss(tb + cZ, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), make_idesc(64, 64), k > 0);
+        mma_commit(&bar_mma[3]);
+    }
+    ok = ok && mbar_wait(&bar_mma[3], 0, a.status, ERR_MMA2);
+    tc_fence_after();
+    {
+        const int i = row64;
+        const float bi = sBeta[i], Gi = sG[i];
+        float db = 0.f;
+        for (int cb = 0; cb < 2; ++cb) {
+            uint32_t r[16];
+            const int j0 = colhalf * 32 + cb * 16;
+            tmem_ld16(tb + cZ + lane_addr + j0, r);
+            tmem_ld_wait();
+            if (row_active) {
+                float m2[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const int j = j0 + x;
+                    const float da = j < i ? -__uint_as_float(r[x]) : 0.f;
+                    db = fmaf(da, sRaw[i * LC + j], db);
+                    m2[x] = j < i ? da * bi * __expf(Gi - sG[j]) : 0.f;
+                }
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2)
+                    *reinterpret_cast<uint4*>(sm + R_M2 + sw128_chunk(i, (j0 >> 3) + c2)) =
+                        make_uint4(pack_bf16(m2[c2 * 8 + 0], m2[c2 * 8 + 1]), pack_bf16(m2[c2 * 8 + 2], m2[c2 * 8 + 3]),
+                                   pack_bf16(m2[c2 * 8 + 4], m2[c2 * 8 + 5]), pack_bf16(m2[c2 * 8 + 6], m2[c2 * 8 + 7]));
+            }
+        }
+        if (row_active) atomicAdd(&sdB[i], db);
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- phase E: dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T -----------------------------------------
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        const uint64_t da0 = desc_mnmajor(sm + R_K, BOX), da1 = desc_mnmajor(sm + R_KT, BOX);
+        const uint64_t dbm = desc_mnmajor(sm + R_M2, 0), dbk = desc_kmajor(sm + R_M2);
+        for (int k = 0; k < 4; ++k)
+            mma_ss(tb + cDKT, desc_advance(da0, 2048 * k), desc_advance(dbm, 2048 * k),
+                   make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), 1);
+        for (int k = 0; k < 4; ++k)
+            mma_ss(tb + cDKR, desc_advance(da1, 2048 * k), desc_advance(dbk, 32 * k),
+                   make_idesc(128, 64, IDESC_A_MN), k > 0);
+        mma_commit(&bar_mma[4]);
+    }
+    ok = ok && mbar_wait(&bar_mma[4], 0, a.status, ERR_MMA2);
+    tc_fence_after();
+
+    // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
+    if (ok) {
+        const unsigned long long sk =
+            (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
+        const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
+        const uint32_t fc = f & 63;
+        float rsum = 0.f;
+        for (int cb = 0; cb < 4; ++cb) {
+            const int j0 = colhalf * 32 + cb * 8;
+            uint32_t rq1[8], rq2[8], rkt[8], rdk[8], rkb[8], rkr[8], rvb[8];
+            tmem_ld8(tb + cDQ1 + lane_addr + j0, rq1);
+            tmem_ld8(tb + cDQ2 + lane_addr + j0, rq2);
+            tmem_ld8(tb + cDKTR + lane_addr + j0, rkt);
+            tmem_ld8(tb + cDKT + lane_addr + j0, rdk);
+            tmem_ld8(tb + cDKB + lane_addr + j0, rkb);
+            tmem_ld8(tb + cDKR + lane_addr + j0, rkr);
+            tmem_ld8(tb + cDVB + lane_addr + j0, rvb);
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                const int j = j0 + x;
+                const uint32_t eo = boxf + sw128_elem(j, fc);
+                const float qv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_Q + eo));
+                const float kv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_K + eo));
+                const float ktv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_KT + eo));
+                const float vv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_V + eo));
+                const float bj = sBeta[j], gj = sGam[j], rj = sRho[j];
+                const float dq = a.scale * gj * __uint_as_float(rq1[x]) + __uint_as_float(rq2[x]);
+                const float dktr = rj * __uint_as_float(rkt[x]);
+                const float dkt = dktr + __uint_as_float(rdk[x]);
+                const float dkb = __uint_as_float(rkb[x]);
+                const float dkr = bj * gj * dkb + __uint_as_float(rkr[x]);
+                const float dvb = __uint_as_float(rvb[x]);
+                float gval = dq * qv + dkr * kv - dkt * ktv;
+                float bval = gj * dkb * kv + dvb * vv;
+                float rval = dktr * ktv;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    gval += __shfl_xor_sync(0xffffffffu, gval, o);
+                    bval += __shfl_xor_sync(0xffffffffu, bval, o);
+                    rval += __shfl_xor_sync(0xffffffffu, rval, o);
+                }
+                if (lane == 0) {
+                    atomicAdd(&sdG[j], gval);
+                    atomicAdd(&sdB[j], bval);
+                    rsum += rval;
+                }
+                if (j < len) {
+                    const size_t g = ((size_t)(tok0 + j) * H + h) * KD + f;
+                    a.dq[g] = __float2bfloat16_rn(dq);
+                    a.dv[g] = __float2bfloat16_rn(bj * dvb);
+                    const bool skipped = (sk >> j) & 1ull;
+                    if (skipped) a.dk[g] = __float2bfloat16_rn(dkr + a.d_min * dkt);
+                    else a.dkread[g] = dkr;
+                    if (!skipped || j == 0 || !((sk >> (j - 1)) & 1ull)) a.dktil[g] = dkt;
+                }
+            }
+        }
+        if (lane == 0) atomicAdd(&sRsum, rsum);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < CBW_THREADS / 32; ++w) tot += sRed[w];
+        float gl = 0.f;
+        for (int j = 0; j < CH; ++j) gl += sg[j];
+        sdG[CH - 1] += sRsum + __expf(gl) * tot;
+        float acc = 0.f;
+        for (int i = CH - 1; i >= 0; --i) { acc += sdG[i]; sdG[i] = acc; }
+    }
+    __syncthreads();
+    if (tid < len) {
+        const size_t th = (size_t)(tok0 + tid) * H + h;
+        a.dgate[th] = sdG[tid];
+        a.dbeta[th] = sdB[tid];
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tb, 512);
+}
+
 template <typename F> bool set_smem(F* kernel, size_t bytes)
 {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
@@ -668,11 +1353,55 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
-bool tc_backward_supported(const osdn_params&) { return false; }
+bool tc_backward_supported(const osdn_params& p) { return tc_supported(p); }
 
-int tc_backward(const osdn_params&, const Hyper&, const WsLayout&, void*, const Pointers&, cudaStream_t)
+int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                cudaStream_t st)
 {
-    return -1;
+    char* w = static_cast<char*>(ws);
+    const TcLayout t = make_tc_layout(p, L, true);
+    if (t.total > L.total) return -1;
+    Table tab = carve_table(ws, L);
+    const int S = L.S, H = p.H;
+    const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
+    int* status = reinterpret_cast<int*>(w + L.status);
+    int launches = 0;
+    auto U8 = [&](size_t off) { return reinterpret_cast<uint8_t*>(w + off); };
+    CUtensorMap tmK, tmQ, tmKt, tmV, tmDO;
+    if (!make_token_map(&tmK, a.k, Ttot, H) || !make_token_map(&tmQ, a.q, Ttot, H) ||
+        !make_token_map(&tmKt, w + t.ktil, Ttot, H) || !make_token_map(&tmV, a.v, Ttot, H) ||
+        !make_token_map(&tmDO, a.dout, Ttot, H))
+        return -1;
+    {
+        TcChainBwdArgs ch{};
+        ch.H = H; ch.tab = tab; ch.gate = a.gate; ch.dfinal_state = a.dfinal_state; ch.dinit_state = a.dinit_state;
+        ch.WT = U8(t.WT); ch.P = U8(t.P); ch.Qg = U8(t.Qg); ch.dSn = U8(t.dSn); ch.ddUT = U8(t.ddUT);
+        ch.status = status;
+        if (!set_smem(tc_chain_bwd_kernel, CB_SMEM)) return -1;
+        stage_mark(st, "tc_chain_bwd");
+        tc_chain_bwd_kernel<<<S * H, CF_THREADS, CB_SMEM, st>>>(tmDO, tmKt, ch);
+        ++launches;
+    }
+    {
+        TcChunkBwdArgs cb{};
+        cb.H = H; cb.tab = tab; cb.beta = a.beta; cb.gate = a.gate; cb.scale = hy.scale; cb.d_min = hy.d_min;
+        cb.Tm = U8(t.Tm); cb.Sn = U8(t.Sn); cb.dSn = U8(t.dSn); cb.dUT = U8(t.dUT); cb.ddUT = U8(t.ddUT);
+        cb.skipw = carve_p1(ws, L).skipw;
+        cb.dq = static_cast<__nv_bfloat16*>(a.dq); cb.dk = static_cast<__nv_bfloat16*>(a.dk);
+        cb.dv = static_cast<__nv_bfloat16*>(a.dv); cb.dbeta = a.dbeta; cb.dgate = a.dgate;
+        cb.dktil = reinterpret_cast<float*>(w + t.dktil); cb.dkread = reinterpret_cast<float*>(w + t.dkread);
+        cb.status = status;
+        if (!set_smem(tc_chunk_bwd_kernel, CBW_SMEM)) return -1;
+        stage_mark(st, "tc_chunk_bwd");
+        tc_chunk_bwd_kernel<<<dim3(L.NTmax, H), CBW_THREADS, CBW_SMEM, st>>>(tmQ, tmK, tmKt, tmV, tmDO, cb);
+        ++launches;
+    }
+    const int n1 = phase1_backward(p, hy, L, ws, a, reinterpret_cast<float*>(w + t.dktil),
+                                   reinterpret_cast<float*>(w + t.dkread), false, st);
+    if (n1 < 0) return -1;
+    launches += n1;
+    stage_end(st);
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 }  // namespace osdn
