@@ -214,7 +214,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {
                     const int j = cb * 16 + x;
-                    sA[i * LC + j] = j < i ? bi * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+                    sA[j * CH + i] = j < i ? bi * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
                 }
             }
         } else {
@@ -245,16 +245,38 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     __syncthreads();
 
-    // ---- T = (I + A)^-1, column by column (two lanes per column split the inner sum) -----------
-    {
-        const int col = tid >> 1, part = tid & 1;
-        for (int i = 0; i < CH; ++i) {
-            float sum = 0.f;
-            for (int j = col + part; j < i; j += 2) sum = fmaf(sA[i * LC + j], sT[j * LC + col], sum);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-            const float x = i < col ? 0.f : (i == col ? 1.f : -sum);
-            if (part == 0) sT[i * LC + col] = x;
-            __syncwarp();
+    // ---- T = (I + A)^-1 --------------------------------------------------------------------------
+    // Thread `col` (warps 0-1) solves (I + A) x = e_col with the whole column in registers: after x_j is
+    // final, every later partial sum is updated at once (independent FMAs, broadcast reads of A).
+    // Warps 2-3 meanwhile emit the gated, scaled queries for the backward state chain:
+    // Qg = scale gamma_i Q, same image layout as Q.
+    if (tid < CH) {
+        const int col = tid;
+        float x[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) x[i] = i == col ? 1.f : 0.f;
+#pragma unroll
+        for (int j = 0; j < CH - 1; ++j) {
+            const float xj = x[j];
+#pragma unroll
+            for (int i = j + 1; i < CH; ++i) x[i] = fmaf(-sA[j * CH + i], xj, x[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < CH; ++i) sT[i * LC + col] = x[i];
+    } else if (a.save) {
+        for (int e = tid - CH; e < 2 * CH * 8; e += CL_THREADS - CH) {
+            const int hf = e >> 9, i = (e >> 3) & 63, ch = e & 7;
+            const uint32_t off = sw128_chunk(i, ch);
+            const uint4 w = *reinterpret_cast<const uint4*>(sKQ + hf * 16384 + BOX + off);
+            const float f = a.scale * __expf(sG[i]);
+            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&w);
+            uint32_t o[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const float2 v = __bfloat1622float2(p2[x]);
+                o[x] = pack_bf16(v.x * f, v.y * f);
+            }
+            *reinterpret_cast<uint4*>(a.Qg + tile * 16384 + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
     __syncthreads();
@@ -292,23 +314,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint64_t db0 = desc_kmajor(sTb);
         for (int s = 0; s < 4; ++s) mma_ss(tb + 64, desc_advance(da0, 2048 * s), desc_advance(db0, 32 * s), idesc, s > 0);
         mma_commit(&bar_mma2);
-    }
-    // gated, scaled queries for the backward state chain: Qg = scale gamma_i Q (same image layout as Q)
-    if (a.save) {
-        for (int e = tid; e < 2 * CH * 8; e += CL_THREADS) {
-            const int hf = e >> 9, i = (e >> 3) & 63, ch = e & 7;
-            const uint32_t off = sw128_chunk(i, ch);
-            const uint4 w = *reinterpret_cast<const uint4*>(sKQ + hf * 16384 + BOX + off);
-            const float f = a.scale * __expf(sG[i]);
-            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&w);
-            uint32_t o[4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const float2 v = __bfloat1622float2(p2[x]);
-                o[x] = pack_bf16(v.x * f, v.y * f);
-            }
-            *reinterpret_cast<uint4*>(a.Qg + tile * 16384 + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
-        }
     }
     ok = ok && mbar_wait(&bar_mma2, 0, a.status, ERR_MMA2);
     tc_fence_after();
@@ -460,10 +465,13 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         {
             const float gC = sGC[st];
             uint8_t* Sg = a.Sn + tile * 32768 + colhalf * 16384;
+            uint32_t rr[4][16];
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb) tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, rr[cb]);
+            tmem_ld_wait();
+#pragma unroll
             for (int cb = 0; cb < 4; ++cb) {
-                uint32_t r[16];
-                tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
-                tmem_ld_wait();
+                uint32_t* r = rr[cb];
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     uint4 w;
@@ -523,10 +531,13 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         // ---- E1: dU^T -> bf16 operands ---------------------------------------------------------
         {
             uint8_t* dUg = a.dUT + tile * 16384;
+            uint32_t rr[2][16];
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) tmem_ld16(tDU + lane_addr + colhalf * 32 + cb * 16, rr[cb]);
+            tmem_ld_wait();
+#pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
-                uint32_t r[16];
-                tmem_ld16(tDU + lane_addr + colhalf * 32 + cb * 16, r);
-                tmem_ld_wait();
+                uint32_t* r = rr[cb];
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     float f[8], g[8];
@@ -574,11 +585,16 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         // ---- E2: O^T = scale gamma_i O1^T + O2^T -> out ----------------------------------------
         if (ok) {
             __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
+            uint32_t ra[2][16], rb[2][16];
+#pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
-                uint32_t r1[16], r2[16];
-                tmem_ld16(tO1 + lane_addr + colhalf * 32 + cb * 16, r1);
-                tmem_ld16(tO2 + lane_addr + colhalf * 32 + cb * 16, r2);
-                tmem_ld_wait();
+                tmem_ld16(tO1 + lane_addr + colhalf * 32 + cb * 16, ra[cb]);
+                tmem_ld16(tO2 + lane_addr + colhalf * 32 + cb * 16, rb[cb]);
+            }
+            tmem_ld_wait();
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                const uint32_t *r1 = ra[cb], *r2 = rb[cb];
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {
                     const int i = colhalf * 32 + cb * 16 + x;
@@ -722,10 +738,13 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         {
             const float gC = sGC[st];
             uint8_t* Sg = a.dSn + tile * 32768 + colhalf * 16384;
+            uint32_t rr[4][16];
+#pragma unroll
+            for (int cb = 0; cb < 4; ++cb) tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, rr[cb]);
+            tmem_ld_wait();
+#pragma unroll
             for (int cb = 0; cb < 4; ++cb) {
-                uint32_t r[16];
-                tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
-                tmem_ld_wait();
+                uint32_t* r = rr[cb];
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     uint4 w;
@@ -776,11 +795,16 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         // ---- E1: ddU^T = acc1 + rho_i acc2 ---------------------------------------------------
         {
             uint8_t* dg = a.ddUT + tile * 16384;
+            uint32_t ra[2][16], rb[2][16];
+#pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
-                uint32_t r1[16], r2[16];
-                tmem_ld16(tA1 + lane_addr + colhalf * 32 + cb * 16, r1);
-                tmem_ld16(tA2 + lane_addr + colhalf * 32 + cb * 16, r2);
-                tmem_ld_wait();
+                tmem_ld16(tA1 + lane_addr + colhalf * 32 + cb * 16, ra[cb]);
+                tmem_ld16(tA2 + lane_addr + colhalf * 32 + cb * 16, rb[cb]);
+            }
+            tmem_ld_wait();
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                const uint32_t *r1 = ra[cb], *r2 = rb[cb];
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     float f[8];
