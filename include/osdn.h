@@ -54,7 +54,8 @@ typedef enum osdn_status {
     OSDN_UNSUPPORTED_SHAPE = -2,  /* K or V not in {64, 128}, chunk != 64, T <= 0, ...      */
     OSDN_MISALIGNED = -3,         /* a pointer is not 16-byte aligned                      */
     OSDN_WORKSPACE_TOO_SMALL = -4,
-    OSDN_CUDA_ERROR = -5          /* a CUDA runtime call or launch failed                  */
+    OSDN_CUDA_ERROR = -5,         /* a CUDA runtime call or launch failed                  */
+    OSDN_STATIC_SCRATCH_TOO_SMALL = -6 /* osdn_fwd_static: problem larger than the built-in scratch */
 } osdn_status;
 
 enum { OSDN_FP32 = 0, OSDN_BF16 = 1 };
@@ -132,6 +133,37 @@ int osdn_bwd(const osdn_params* p, const void* q, const void* k, const void* v,
 int osdn_precond_update(const osdn_params* p, const void* k, const float* beta,
                         const float* gate_or_log_ret, const float* precond_in,
                         void* k_tilde_out, float* precond_out, void* cuda_stream);
+
+/*
+ * Forward pass for callers that cannot provide a workspace.  (The paper has no counterpart to
+ * this call; it exists for deployment reasons only.)
+ *
+ * Some callers are not able to allocate device memory at the point where they need the layer:
+ * code running inside a serving loop whose memory pool is fixed at start-up, plugins that are
+ * handed input and output buffers by a host framework but no allocator, and code that must not
+ * call cudaMalloc because that call synchronises the device.  osdn_fwd_static computes exactly
+ * what osdn_fwd computes (same kernels, same results) but takes its scratch space from a fixed
+ * array of OSDN_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
+ * library holds that array until the process exits.  The call allocates nothing, neither with
+ * cudaMalloc nor through any library.
+ *
+ *   - Inputs and outputs are passed exactly as for osdn_fwd (flags other than
+ *     OSDN_FLAG_FORCE_SIMT are ignored: residuals for a backward pass are not kept).
+ *   - Problems whose forward workspace (osdn_workspace_bytes(p, 0)) exceeds
+ *     OSDN_STATIC_SCRATCH_BYTES are rejected with OSDN_STATIC_SCRATCH_TOO_SMALL before anything is
+ *     launched; use osdn_fwd with a caller-owned workspace for those.
+ *   - The first call on each device looks up the device address of the array (with that device
+ *     current) and remembers it; make that first call before starting any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it;
+ *     the call clears the part that has to start at zero itself.  Two calls that overlap on the
+ *     GPU (different streams, or different host threads without ordering) race on the array and
+ *     give undefined results: serialise them.
+ */
+#define OSDN_STATIC_SCRATCH_BYTES (32u << 20)
+int osdn_fwd_static(const osdn_params* p, const void* q, const void* k, const void* v,
+                    const float* beta, const float* gate, const float* apf_log_ret,
+                    const float* init_state, const float* precond_in,
+                    void* out, float* final_state, float* precond_out, void* cuda_stream);
 
 /*
  * Host-buffer convenience for end-to-end measurements: copies the inputs (HOST pointers,

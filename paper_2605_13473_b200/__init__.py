@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     make_params,
     osdn_bwd,
     osdn_fwd,
+    osdn_fwd_static,
     osdn_precond_update,
     osdn_step_host,
     osdn_workspace_bytes,

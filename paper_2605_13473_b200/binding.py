@@ -19,6 +19,7 @@ EXPORTS = [
     "osdn_workspace_bytes", "osdn_fwd", "osdn_bwd", "osdn_precond_update", "osdn_host_staging_bytes",
     "osdn_step_host", "osdn_read_device_status", "osdn_status_string", "osdn_last_launch_count",
     "osdn_stage_timing_enable", "osdn_stage_timing_read", "osdn_workspace_region",
+    "osdn_fwd_static",
 ]
 
 
@@ -51,6 +52,8 @@ def load_library(path: Optional[str] = None):
     lib.osdn_host_staging_bytes.argtypes = [pp, ci]
     lib.osdn_fwd.restype = ci
     lib.osdn_fwd.argtypes = [pp] + [vp] * 11 + [vp, sz, vp]
+    lib.osdn_fwd_static.restype = ci
+    lib.osdn_fwd_static.argtypes = [pp] + [vp] * 11 + [vp]
     lib.osdn_bwd.restype = ci
     lib.osdn_bwd.argtypes = [pp] + [vp] * 19 + [vp, sz, vp]
     lib.osdn_precond_update.restype = ci
@@ -172,6 +175,20 @@ def osdn_fwd(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, init_state, precon
                       _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                       _stream_ptr())
     _check(rc, "osdn_fwd")
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def osdn_fwd_static(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, init_state, precond_in, out, final_state,
+                    precond_out) -> int:
+    """Forward pass on the library's built-in scratch array: for callers that cannot allocate a
+    workspace.  Returns the status code (0 = ok, -6 = the problem does not fit the built-in scratch)
+    instead of raising, so that a caller can fall back to ``osdn_fwd`` with its own workspace."""
+    lib = load_library()
+    return int(lib.osdn_fwd_static(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gate),
+                                   _ptr(apf_log_ret), _ptr(init_state), _ptr(precond_in), _ptr(out),
+                                   _ptr(final_state), _ptr(precond_out), _stream_ptr()))
 
 
 def osdn_bwd(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, init_state, precond_in, dout, dfinal_state,

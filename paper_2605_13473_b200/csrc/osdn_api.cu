@@ -3,6 +3,7 @@
 // thread-local launch counter used for benchmark accounting).
 #include <cmath>
 #include <cstring>
+#include <mutex>
 
 #include "osdn_common.cuh"
 
@@ -310,6 +311,63 @@ int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host,
     return ok ? OSDN_OK : OSDN_CUDA_ERROR;
 }
 
+// ---- forward without a caller workspace ----------------------------------------------------
+// Scratch for osdn_fwd_static.  In host code the name below is only a handle for the symbol, not a
+// device address: the address is looked up once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[OSDN_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[MAX_DEVICES] = {};
+
+// Device address of g_static_scratch on the current device (looked up on first use).
+void* static_scratch_address()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
+        g_static_ptr[dev] = ptr;
+    }
+    return g_static_ptr[dev];
+}
+}  // namespace
+
+int osdn_fwd_static(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                    const float* gate, const float* apf_log_ret, const float* init_state, const float* precond_in,
+                    void* out, float* final_state, float* precond_out, void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (!q || !k || !v || !beta || !gate || !out) return OSDN_INVALID_ARG;
+    if (p->apf_mode == OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, init_state, precond_in, out, final_state,
+                          precond_out};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    osdn_params pp = *p;
+    pp.flags = p->flags & OSDN_FLAG_FORCE_SIMT;
+    const WsLayout L = make_layout(pp, false);
+    if (L.total > (size_t)OSDN_STATIC_SCRATCH_BYTES) return OSDN_STATIC_SCRATCH_TOO_SMALL;
+    void* scratch = static_scratch_address();
+    if (!scratch) return OSDN_CUDA_ERROR;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // the device status word is the only part that must start at zero
+    if (cudaMemsetAsync(static_cast<char*>(scratch) + L.status, 0, 256, st) != cudaSuccess) return OSDN_CUDA_ERROR;
+    Pointers a{};
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.gate = gate; a.log_ret = apf_log_ret;
+    a.init_state = init_state; a.precond_in = precond_in; a.out = out; a.final_state = final_state;
+    a.precond_out = precond_out;
+    const int n = run_forward(pp, make_hyper(pp), L, scratch, a, false, st);
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = n;
+    return OSDN_OK;
+}
+
 int osdn_workspace_region(const osdn_params* p, int need_bwd, const char* name, size_t* offset, size_t* bytes)
 {
     if (validate(p) != OSDN_OK || !name || !offset || !bytes || !need_bwd) return OSDN_INVALID_ARG;
@@ -344,6 +402,8 @@ const char* osdn_status_string(int status)
         case OSDN_MISALIGNED: return "pointer not sufficiently aligned";
         case OSDN_WORKSPACE_TOO_SMALL: return "workspace too small";
         case OSDN_CUDA_ERROR: return "CUDA error";
+        case OSDN_STATIC_SCRATCH_TOO_SMALL:
+            return "problem too large for the built-in scratch of osdn_fwd_static (use osdn_fwd with a workspace)";
         default: return "unknown status";
     }
 }
