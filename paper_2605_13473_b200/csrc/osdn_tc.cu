@@ -26,6 +26,18 @@ namespace osdn {
 
 using namespace umma;
 
+// Developer aid (compiled only with -DOSDN_PHASE_CLOCKS): clock64 stamps of one CTA at the phase
+// boundaries of each tensor-core kernel, read back with osdn_debug_clocks.
+#ifdef OSDN_PHASE_CLOCKS
+__device__ long long g_clk[4][32];
+#define OSDN_CLK(k, i, cond)                                          \
+    do {                                                              \
+        if ((cond) && threadIdx.x == 0) g_clk[k][i] = clock64();      \
+    } while (0)
+#else
+#define OSDN_CLK(k, i, cond)
+#endif
+
 namespace {
 
 constexpr int KD = 128;  // K = V = 128 on this path
@@ -161,6 +173,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(0, 0, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     const uint32_t tb = tmem_base;
 
@@ -178,6 +191,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         sG[tid] = acc;
     }
     bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
+    OSDN_CLK(0, 1, blockIdx.x == 5 && blockIdx.y == 0);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sKQ + hf * 16384, len, tid, CL_THREADS);
@@ -187,6 +201,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         fence_proxy_async();
     }
     __syncthreads();
+    OSDN_CLK(0, 2, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- D1[128 x 64] = [K;Q] Ktil^T ---------------------------------------------------------
     if (tid == 0 && ok) {
@@ -200,6 +215,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mma_commit(&bar_mma1);
     }
     ok = ok && mbar_wait(&bar_mma1, 0, a.status, ERR_MMA1);
+    OSDN_CLK(0, 3, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
         const int L = warp * 32 + lane;
@@ -244,6 +260,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
     }
     __syncthreads();
+    OSDN_CLK(0, 4, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- T = (I + A)^-1 --------------------------------------------------------------------------
     // Thread `col` (warps 0-1) solves (I + A) x = e_col with the whole column in registers: after x_j is
@@ -280,6 +297,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
     }
     __syncthreads();
+    OSDN_CLK(0, 5, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- operand images: Tbg (shared), Tb and T (HBM) -----------------------------------------
     for (int e = tid; e < CH * 8; e += CL_THREADS) {
@@ -305,6 +323,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(0, 6, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- D2[128 x 64] = K^T Tbg^T  (W^T) -----------------------------------------------------
     if (tid == 0 && ok) {
@@ -316,6 +335,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mma_commit(&bar_mma2);
     }
     ok = ok && mbar_wait(&bar_mma2, 0, a.status, ERR_MMA2);
+    OSDN_CLK(0, 7, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
         const int k = warp * 32 + lane;
@@ -338,6 +358,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(0, 8, blockIdx.x == 5 && blockIdx.y == 0);
     if (warp == 0) tmem_dealloc(tb, 128);
 }
 
@@ -362,6 +383,25 @@ constexpr uint32_t STAGE_BYTES = 16384 + 8192 + 8192 + 3 * 16384;   // WT, Tb, P
 constexpr uint32_t ST_WT = 0, ST_TB = 16384, ST_P = 24576, ST_V = 32768, ST_Q = 49152, ST_KT = 65536;
 constexpr size_t CF_SMEM = 2 * STAGE_BYTES + 32768 + 2 * 16384 + 1024;
 
+// In-chunk gate prefix by one warp: lane l holds g_l and g_{l+32}.  Writes gamma_i = exp(G_i),
+// rho_i = exp(G_C - G_i) and gamma_C into the given slot.
+__device__ __forceinline__ void warp_gate_vectors(float ga, float gb, int lane, float* gam, float* rho, float* gC)
+{
+    float sa = ga, sb = gb;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float ua = __shfl_up_sync(0xffffffffu, sa, o), ub = __shfl_up_sync(0xffffffffu, sb, o);
+        if (lane >= o) { sa += ua; sb += ub; }
+    }
+    const float ta = __shfl_sync(0xffffffffu, sa, 31);
+    sb += ta;
+    const float tot = __shfl_sync(0xffffffffu, sb, 31);
+    if (gam) { gam[lane] = __expf(sa); gam[lane + 32] = __expf(sb); }
+    rho[lane] = __expf(tot - sa);
+    rho[lane + 32] = __expf(tot - sb);
+    if (lane == 0) *gC = __expf(tot);
+}
+
 __global__ void __launch_bounds__(CF_THREADS, 1)
 tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
                     const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
@@ -374,11 +414,12 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     uint8_t* sDU2 = sDU1 + 16384;               // (rho dU)^T
     __shared__ uint64_t bar_full[2], bar_mma1, bar_mma2;
     __shared__ uint32_t tmem_base;
-    __shared__ float sGam[2][CH], sRho[2][CH], sGC[2], sgraw[CH];
+    __shared__ float sGam[3][CH], sRho[3][CH], sGC[3];   // slot = chunk % 3
 
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
     const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, colhalf = warp >> 2;
     const int v = quad * 32 + lane;             // state row owned by this thread
@@ -389,6 +430,9 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             for (int x = 0; x < 64; ++x) fin[x] = ini ? ini[x] : 0.f;
         return;
     }
+    const int nchunks = c1 - c0;
+    auto chunk_tok0 = [&](int n) { return seq_t0 + n * CH; };
+    auto chunk_len = [&](int n) { return min(CH, seq_len - n * CH); };
 
     if (tid == 0) {
         mbar_init(&bar_full[0], 1);
@@ -403,11 +447,11 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     tc_fence_after();
     const uint32_t tb = tmem_base;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t tS = tb, tDU = tb + 128, tO1 = tb + 192, tO2 = tb + 256;
+    const uint32_t tS = tb, tDU = tb + 128, tO1 = tb + 192, tO2 = tb + 320;   // O1, O2: two buffers of 64
 
-    auto issue_loads = [&](int c, int st) {
-        const int tok0 = a.tab.chunk_tok0[c];
-        const size_t tile = (size_t)c * H + h;
+    auto issue_loads = [&](int n, int st) {
+        const int tok0 = chunk_tok0(n);
+        const size_t tile = (size_t)(c0 + n) * H + h;
         uint8_t* d = sStage + st * STAGE_BYTES;
         mbar_expect_tx(&bar_full[st], STAGE_BYTES);
         bulk_load(d + ST_WT, a.WT + tile * 16384, 16384, &bar_full[st]);
@@ -419,27 +463,41 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             tma_load_2d(d + ST_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
         }
     };
-    // gate vectors of chunk c into slot st (threads 0..63, then a barrier by the caller)
-    auto gate_vectors = [&](int c, int st) {
-        if (tid < CH) {
-            const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
-            sgraw[tid] = tid < len ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
+    // raw gates of chunk n for the gate warp (lane l: tokens l and l + 32)
+    auto load_gates = [&](int n, float& ga, float& gb) {
+        const int tok0 = chunk_tok0(n), len = chunk_len(n);
+        ga = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
+        gb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+    };
+    // output of chunk n from its O1 / O2 accumulators
+    auto store_out = [&](int n) {
+        const int tok0 = chunk_tok0(n), len = chunk_len(n), st = n & 1, gs = n % 3;
+        __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
+        uint32_t ra[2][16], rb[2][16];
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+            tmem_ld16(tO1 + st * 64 + lane_addr + colhalf * 32 + cb * 16, ra[cb]);
+            tmem_ld16(tO2 + st * 64 + lane_addr + colhalf * 32 + cb * 16, rb[cb]);
         }
-        __syncthreads();
-        if (tid < CH) {
-            float G = 0.f, tot = 0.f;
-            for (int j = 0; j < CH; ++j) {
-                const float g = sgraw[j];
-                tot += g;
-                if (j <= tid) G += g;
+        tmem_ld_wait();
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+#pragma unroll
+            for (int x = 0; x < 16; ++x) {
+                const int i = colhalf * 32 + cb * 16 + x;
+                if (i < len)
+                    op[(size_t)i * H * KD] = __float2bfloat16_rn(
+                        a.scale * sGam[gs][i] * __uint_as_float(ra[cb][x]) + __uint_as_float(rb[cb][x]));
             }
-            sGam[st][tid] = __expf(G);
-            sRho[st][tid] = __expf(tot - G);
-            if (tid == 0) sGC[st] = __expf(tot);
         }
     };
 
-    if (tid == 0) issue_loads(c0, 0);
+    if (tid == 0) issue_loads(0, 0);
+    float ga = 0.f, gb = 0.f;
+    if (warp == 7) {
+        load_gates(0, ga, gb);
+        warp_gate_vectors(ga, gb, lane, sGam[0], sRho[0], &sGC[0]);
+    }
     // initial state into tensor memory
     for (int cb = 0; cb < 4; ++cb) {
         uint32_t r[16];
@@ -448,22 +506,23 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
     }
     tmem_st_wait();
-    gate_vectors(c0, 0);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
 
     bool ok = true;
-    for (int c = c0; c < c1; ++c) {
-        const int n = c - c0, st = n & 1;
-        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
-        const size_t tile = (size_t)c * H + h;
+    for (int n = 0; n < nchunks; ++n) {
+        const int st = n & 1, gs = n % 3;
+        const int len = chunk_len(n);
+        const size_t tile = (size_t)(c0 + n) * H + h;
         uint8_t* d = sStage + st * STAGE_BYTES;
-        if (tid == 0 && c + 1 < c1) issue_loads(c + 1, st ^ 1);
+        if (tid == 0 && n + 1 < nchunks) issue_loads(n + 1, st ^ 1);
+        if (warp == 7 && n + 1 < nchunks) load_gates(n + 1, ga, gb);   // consumed after MMA group 2 is issued
+    OSDN_CLK(1, 0, blockIdx.x == 0 && n == 3);
 
         // ---- E0: S -> bf16 operand (+ saved copy), decay the accumulator -----------------------
         {
-            const float gC = sGC[st];
+            const float gC = sGC[gs];
             uint8_t* Sg = a.Sn + tile * 32768 + colhalf * 16384;
             uint32_t rr[4][16];
 #pragma unroll
@@ -489,7 +548,9 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             }
             tmem_st_wait();
         }
+    OSDN_CLK(1, 1, blockIdx.x == 0 && n == 3);
         ok = ok && mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
+    OSDN_CLK(1, 2, blockIdx.x == 0 && n == 3);
         if (len < CH) {
             for (int hf = 0; hf < 2; ++hf) {
                 zero_tail_rows(d + ST_V + hf * BOX, len, tid, CF_THREADS);
@@ -500,6 +561,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+    OSDN_CLK(1, 3, blockIdx.x == 0 && n == 3);
 
         // ---- MMA group 1 -----------------------------------------------------------------------
         if (tid == 0 && ok) {
@@ -517,16 +579,17 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                     mma_ss(tDU, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
                            desc_advance(db0, 2048 * k), idesc, 1);
             }
-            {   // O1^T = S Q^T
+            mma_commit(&bar_mma1);
+            {   // O1^T = S Q^T  (not needed before the output is assembled: rides on the next commit)
                 const uint32_t idesc = make_idesc(128, 64);
                 for (int k = 0; k < 8; ++k)
-                    mma_ss(tO1, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
+                    mma_ss(tO1 + st * 64, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
                            desc_advance(desc_kmajor(d + ST_Q + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
             }
-            mma_commit(&bar_mma1);
         }
         ok = ok && mbar_wait(&bar_mma1, n & 1, a.status, ERR_CHAIN_MMA1);
         tc_fence_after();
+    OSDN_CLK(1, 4, blockIdx.x == 0 && n == 3);
 
         // ---- E1: dU^T -> bf16 operands ---------------------------------------------------------
         {
@@ -544,7 +607,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 #pragma unroll
                     for (int x = 0; x < 8; ++x) {
                         f[x] = __uint_as_float(r[c2 * 8 + x]);
-                        g[x] = f[x] * sRho[st][colhalf * 32 + cb * 16 + c2 * 8 + x];
+                        g[x] = f[x] * sRho[gs][colhalf * 32 + cb * 16 + c2 * 8 + x];
                     }
                     const uint32_t off = sw128_chunk(v, colhalf * 4 + cb * 2 + c2);
                     const uint4 w1 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
@@ -559,55 +622,47 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+    OSDN_CLK(1, 5, blockIdx.x == 0 && n == 3);
 
         // ---- MMA group 2 -----------------------------------------------------------------------
         if (tid == 0 && ok) {
             tc_fence_after();
-            {   // O2^T = dU^T P'^T
-                const uint32_t idesc = make_idesc(128, 64);
-                const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
-                for (int k = 0; k < 4; ++k)
-                    mma_ss(tO2, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, k > 0);
-            }
-            {   // S += (rho dU)^T Ktil
+            {   // S += (rho dU)^T Ktil   (on the critical path: first)
                 const uint32_t idesc = make_idesc(128, 128, IDESC_B_MN);
                 const uint64_t da0 = desc_kmajor(sDU2), db0 = desc_mnmajor(d + ST_KT, BOX);
                 for (int k = 0; k < 4; ++k)
                     mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k), idesc, 1);
             }
             mma_commit(&bar_mma2);
+            {   // O2^T = dU^T P'^T   (completes before the next commit, which the output waits for)
+                const uint32_t idesc = make_idesc(128, 64);
+                const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tO2 + st * 64, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+            }
         }
-        // gate vectors of the next chunk while the tensor core works
-        if (c + 1 < c1) gate_vectors(c + 1, st ^ 1);
+        // while the tensor core works: gate vectors of the next chunk, output of the previous chunk
+        // (its O2 accumulator was issued after the previous chunk's last commit and is covered by
+        // this chunk's first commit, which has been waited for above)
+        if (warp == 7 && n + 1 < nchunks)
+            warp_gate_vectors(ga, gb, lane, sGam[(n + 1) % 3], sRho[(n + 1) % 3], &sGC[(n + 1) % 3]);
+        if (n > 0 && ok) store_out(n - 1);
         ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
         tc_fence_after();
-
-        // ---- E2: O^T = scale gamma_i O1^T + O2^T -> out ----------------------------------------
-        if (ok) {
-            __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
-            uint32_t ra[2][16], rb[2][16];
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                tmem_ld16(tO1 + lane_addr + colhalf * 32 + cb * 16, ra[cb]);
-                tmem_ld16(tO2 + lane_addr + colhalf * 32 + cb * 16, rb[cb]);
-            }
-            tmem_ld_wait();
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                const uint32_t *r1 = ra[cb], *r2 = rb[cb];
-#pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const int i = colhalf * 32 + cb * 16 + x;
-                    if (i < len)
-                        op[(size_t)i * H * KD] = __float2bfloat16_rn(
-                            a.scale * sGam[st][i] * __uint_as_float(r1[x]) + __uint_as_float(r2[x]));
-                }
-            }
-        }
+    OSDN_CLK(1, 6, blockIdx.x == 0 && n == 3);
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
+    OSDN_CLK(1, 7, blockIdx.x == 0 && n == 3);
     }
+
+    // the last chunk's output accumulators were issued after the last commits: close them
+    if (tid == 0 && ok) {
+        mma_commit(&bar_mma1);
+    }
+    ok = ok && mbar_wait(&bar_mma1, nchunks & 1, a.status, ERR_CHAIN_MMA1);
+    tc_fence_after();
+    if (ok) store_out(nchunks - 1);
 
     if (fin && ok) {
         for (int cb = 0; cb < 4; ++cb) {
@@ -762,7 +817,9 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
             }
             tmem_st_wait();
         }
+    OSDN_CLK(2, 1, blockIdx.x == 0 && n == 3);
         ok = ok && mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
+    OSDN_CLK(2, 2, blockIdx.x == 0 && n == 3);
         if (len < CH) {
             for (int hf = 0; hf < 2; ++hf) {
                 zero_tail_rows(d + BS_DO + hf * BOX, len, tid, CF_THREADS);
@@ -772,6 +829,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+    OSDN_CLK(2, 3, blockIdx.x == 0 && n == 3);
 
         if (tid == 0 && ok) {
             tc_fence_after();
@@ -790,6 +848,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
             mma_commit(&bar_mma1);
         }
         ok = ok && mbar_wait(&bar_mma1, n & 1, a.status, ERR_CHAIN_MMA1);
+    OSDN_CLK(2, 4, blockIdx.x == 0 && n == 3);
         tc_fence_after();
 
         // ---- E1: ddU^T = acc1 + rho_i acc2 ---------------------------------------------------
@@ -823,6 +882,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+    OSDN_CLK(2, 5, blockIdx.x == 0 && n == 3);
 
         if (tid == 0 && ok) {
             tc_fence_after();
@@ -842,9 +902,11 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         }
         if (c > c0) gate_vectors(c - 1, st ^ 1);
         ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
+    OSDN_CLK(2, 6, blockIdx.x == 0 && n == 3);
         tc_fence_after();
         tc_fence_before();
         __syncthreads();
+    OSDN_CLK(2, 7, blockIdx.x == 0 && n == 3);
         tc_fence_after();
     }
     if (dini && ok) {
@@ -930,6 +992,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (tid == 0) sRsum = 0.f;
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(3, 0, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     const uint32_t tb = tmem_base;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
@@ -960,6 +1023,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sRho[tid] = __expf(tot - acc);
     }
     bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
+    OSDN_CLK(3, 1, blockIdx.x == 5 && blockIdx.y == 0);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sm + R_Q + hf * BOX, len, tid, CBW_THREADS);
@@ -971,6 +1035,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fence_proxy_async();
     }
     __syncthreads();
+    OSDN_CLK(3, 2, blockIdx.x == 5 && blockIdx.y == 0);
 
     // tensor memory columns
     const uint32_t cRAW = 0, cDP = 64, cDQ1 = 128, cDKTR = 192, cDW = 256, cDTA = 320, cDTB = 384, cDKT = 448;
@@ -1030,6 +1095,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (lane == 0) sRed[warp] = part;
     }
     ok = ok && mbar_wait(&bar_mma[0], 0, a.status, ERR_MMA1);
+    OSDN_CLK(3, 3, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     __syncthreads();   // every thread is done reading S / dS before their space is reused
     // epilogue A
@@ -1076,6 +1142,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(3, 4, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- phase B -------------------------------------------------------------------------------
     if (tid == 0 && ok) {
@@ -1117,6 +1184,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[1]);
     }
     ok = ok && mbar_wait(&bar_mma[1], 0, a.status, ERR_MMA2);
+    OSDN_CLK(3, 5, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j]
         const int i = row64;
@@ -1144,6 +1212,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(3, 6, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] -----------------------------------------------
     if (tid == 0 && ok) {
@@ -1155,6 +1224,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[2]);
     }
     ok = ok && mbar_wait(&bar_mma[2], 0, a.status, ERR_MMA2);
+    OSDN_CLK(3, 7, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     {
         const int i = row64;
@@ -1177,6 +1247,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(3, 8, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- phase D: Z[a][b] = sum_c Y[a][c] T[b][c] ; dA = -strictLower(Z) --------------------------
     if (tid == 0 && ok) {
@@ -1187,6 +1258,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[3]);
     }
     ok = ok && mbar_wait(&bar_mma[3], 0, a.status, ERR_MMA2);
+    OSDN_CLK(3, 9, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     {
         const int i = row64;
@@ -1218,6 +1290,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(3, 10, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- phase E: dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T -----------------------------------------
     if (tid == 0 && ok) {
@@ -1233,6 +1306,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[4]);
     }
     ok = ok && mbar_wait(&bar_mma[4], 0, a.status, ERR_MMA2);
+    OSDN_CLK(3, 11, blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
@@ -1242,6 +1316,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
         const uint32_t fc = f & 63;
         float rsum = 0.f;
+        float gv[32], bv[32];   // per column: gate and beta contributions of this feature
+#pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
             const int j0 = colhalf * 32 + cb * 8;
             uint32_t rq1[8], rq2[8], rkt[8], rdk[8], rkb[8], rkr[8], rvb[8];
@@ -1268,20 +1344,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const float dkb = __uint_as_float(rkb[x]);
                 const float dkr = bj * gj * dkb + __uint_as_float(rkr[x]);
                 const float dvb = __uint_as_float(rvb[x]);
-                float gval = dq * qv + dkr * kv - dkt * ktv;
-                float bval = gj * dkb * kv + dvb * vv;
-                float rval = dktr * ktv;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    gval += __shfl_xor_sync(0xffffffffu, gval, o);
-                    bval += __shfl_xor_sync(0xffffffffu, bval, o);
-                    rval += __shfl_xor_sync(0xffffffffu, rval, o);
-                }
-                if (lane == 0) {
-                    atomicAdd(&sdG[j], gval);
-                    atomicAdd(&sdB[j], bval);
-                    rsum += rval;
-                }
+                gv[cb * 8 + x] = dq * qv + dkr * kv - dkt * ktv;
+                bv[cb * 8 + x] = gj * dkb * kv + dvb * vv;
+                rsum = fmaf(dktr, ktv, rsum);
                 if (j < len) {
                     const size_t g = ((size_t)(tok0 + j) * H + h) * KD + f;
                     a.dq[g] = __float2bfloat16_rn(dq);
@@ -1293,9 +1358,29 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
             }
         }
+        // Sum over the 32 features of the warp for all 32 columns at once: in each of five steps a
+        // lane keeps one half of its columns and hands the other half to its partner (31 shuffles per
+        // quantity); afterwards lane l holds the warp total of column l.
+#pragma unroll
+        for (int step = 0; step < 5; ++step) {
+            const int off = 16 >> step, n = 16 >> step;   // n = columns kept after this step
+            const bool upper = (lane & off) != 0;
+#pragma unroll
+            for (int i = 0; i < n; ++i) {
+                const float gs = upper ? gv[i] : gv[i + n], gk = upper ? gv[i + n] : gv[i];
+                const float bs = upper ? bv[i] : bv[i + n], bk = upper ? bv[i + n] : bv[i];
+                gv[i] = gk + __shfl_xor_sync(0xffffffffu, gs, off);
+                bv[i] = bk + __shfl_xor_sync(0xffffffffu, bs, off);
+            }
+        }
+        atomicAdd(&sdG[colhalf * 32 + lane], gv[0]);
+        atomicAdd(&sdB[colhalf * 32 + lane], bv[0]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
         if (lane == 0) atomicAdd(&sRsum, rsum);
     }
     __syncthreads();
+    OSDN_CLK(3, 12, blockIdx.x == 5 && blockIdx.y == 0);
     if (tid == 0) {
         float tot = 0.f;
         for (int w = 0; w < CBW_THREADS / 32; ++w) tot += sRed[w];
@@ -1313,6 +1398,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
+    OSDN_CLK(3, 13, blockIdx.x == 5 && blockIdx.y == 0);
     if (warp == 0) tmem_dealloc(tb, 512);
 }
 
@@ -1429,3 +1515,10 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
 }
 
 }  // namespace osdn
+
+#ifdef OSDN_PHASE_CLOCKS
+extern "C" int osdn_debug_clocks(long long* out)
+{
+    return (int)cudaMemcpyFromSymbol(out, osdn::g_clk, sizeof(osdn::g_clk));
+}
+#endif
