@@ -950,6 +950,9 @@ constexpr uint32_t R_Q = 0, R_K = 16384, R_KT = 32768, R_V = 49152, R_DO = 65536
                    R_T = 114688, R_S = 122880, R_DS = 155648, R_RAW = 188416;
 constexpr uint32_t R_DWT = R_DO;                 // dW^T image replaces dO after phase A
 constexpr uint32_t R_M1 = R_S, R_M2 = R_S + 8192, R_DT = R_S + 16384, R_Y = R_S + 24576;
+// output staging after the last product ([token][feature] tiles over the dead operand space)
+constexpr uint32_t ST_DQ = 65536, ST_DV = 81920, ST_DK = 98304, ST_DKR = 114688, ST_DKT = 147456;
+static_assert(ST_DKT + 32768 <= R_RAW, "staging tiles must fit below the fp32 scratch");
 constexpr size_t CBW_SMEM = R_RAW + CH * LC * 4 + 1024;
 
 __global__ void __launch_bounds__(CBW_THREADS, 1)
@@ -1311,12 +1314,17 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
     if (ok) {
-        const unsigned long long sk =
-            (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
         const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
         const uint32_t fc = f & 63;
         float rsum = 0.f;
         float gv[32], bv[32];   // per column: gate and beta contributions of this feature
+        // Results are staged in shared memory as [token][feature] tiles (the operand tiles of the
+        // finished products are dead by now) and written out with 16-byte stores afterwards.
+        __nv_bfloat16* stq = reinterpret_cast<__nv_bfloat16*>(sm + ST_DQ);
+        __nv_bfloat16* stv = reinterpret_cast<__nv_bfloat16*>(sm + ST_DV);
+        __nv_bfloat16* stk = reinterpret_cast<__nv_bfloat16*>(sm + ST_DK);
+        float* stkr = reinterpret_cast<float*>(sm + ST_DKR);
+        float* stkt = reinterpret_cast<float*>(sm + ST_DKT);
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
             const int j0 = colhalf * 32 + cb * 8;
@@ -1328,34 +1336,37 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tmem_ld8(tb + cDKB + lane_addr + j0, rkb);
             tmem_ld8(tb + cDKR + lane_addr + j0, rkr);
             tmem_ld8(tb + cDVB + lane_addr + j0, rvb);
-            tmem_ld_wait();
+            float qv[8], kv[8], ktv[8], vv[8], bj[8], gj[8], rj[8];
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
                 const int j = j0 + x;
                 const uint32_t eo = boxf + sw128_elem(j, fc);
-                const float qv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_Q + eo));
-                const float kv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_K + eo));
-                const float ktv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_KT + eo));
-                const float vv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_V + eo));
-                const float bj = sBeta[j], gj = sGam[j], rj = sRho[j];
-                const float dq = a.scale * gj * __uint_as_float(rq1[x]) + __uint_as_float(rq2[x]);
-                const float dktr = rj * __uint_as_float(rkt[x]);
+                qv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_Q + eo));
+                kv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_K + eo));
+                ktv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_KT + eo));
+                vv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_V + eo));
+                bj[x] = sBeta[j];
+                gj[x] = sGam[j];
+                rj[x] = sRho[j];
+            }
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                const int j = j0 + x;
+                const float dq = a.scale * gj[x] * __uint_as_float(rq1[x]) + __uint_as_float(rq2[x]);
+                const float dktr = rj[x] * __uint_as_float(rkt[x]);
                 const float dkt = dktr + __uint_as_float(rdk[x]);
                 const float dkb = __uint_as_float(rkb[x]);
-                const float dkr = bj * gj * dkb + __uint_as_float(rkr[x]);
+                const float dkr = bj[x] * gj[x] * dkb + __uint_as_float(rkr[x]);
                 const float dvb = __uint_as_float(rvb[x]);
-                gv[cb * 8 + x] = dq * qv + dkr * kv - dkt * ktv;
-                bv[cb * 8 + x] = gj * dkb * kv + dvb * vv;
-                rsum = fmaf(dktr, ktv, rsum);
-                if (j < len) {
-                    const size_t g = ((size_t)(tok0 + j) * H + h) * KD + f;
-                    a.dq[g] = __float2bfloat16_rn(dq);
-                    a.dv[g] = __float2bfloat16_rn(bj * dvb);
-                    const bool skipped = (sk >> j) & 1ull;
-                    if (skipped) a.dk[g] = __float2bfloat16_rn(dkr + a.d_min * dkt);
-                    else a.dkread[g] = dkr;
-                    if (!skipped || j == 0 || !((sk >> (j - 1)) & 1ull)) a.dktil[g] = dkt;
-                }
+                gv[cb * 8 + x] = dq * qv[x] + dkr * kv[x] - dkt * ktv[x];
+                bv[cb * 8 + x] = gj[x] * dkb * kv[x] + dvb * vv[x];
+                rsum = fmaf(dktr, ktv[x], rsum);
+                stq[j * KD + f] = __float2bfloat16_rn(dq);
+                stv[j * KD + f] = __float2bfloat16_rn(bj[x] * dvb);
+                stk[j * KD + f] = __float2bfloat16_rn(dkr + a.d_min * dkt);
+                stkr[j * KD + f] = dkr;
+                stkt[j * KD + f] = dkt;
             }
         }
         // Sum over the 32 features of the warp for all 32 columns at once: in each of five steps a
@@ -1380,6 +1391,28 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (lane == 0) atomicAdd(&sRsum, rsum);
     }
     __syncthreads();
+    if (ok) {
+        // copy-out: 16-byte stores, one 256-byte (bf16) or 512-byte (fp32) token row after another
+        const unsigned long long sk =
+            (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
+        for (int e = tid; e < len * 16; e += CBW_THREADS) {
+            const int j = e >> 4, ch = e & 15;
+            const size_t g = ((size_t)(tok0 + j) * H + h) * KD + ch * 8;
+            *reinterpret_cast<uint4*>(a.dq + g) = *reinterpret_cast<const uint4*>(sm + ST_DQ + j * 256 + ch * 16);
+            *reinterpret_cast<uint4*>(a.dv + g) = *reinterpret_cast<const uint4*>(sm + ST_DV + j * 256 + ch * 16);
+            if ((sk >> j) & 1ull)
+                *reinterpret_cast<uint4*>(a.dk + g) = *reinterpret_cast<const uint4*>(sm + ST_DK + j * 256 + ch * 16);
+        }
+        for (int e = tid; e < len * 32; e += CBW_THREADS) {
+            const int j = e >> 5, ch = e & 31;
+            const size_t g = ((size_t)(tok0 + j) * H + h) * KD + ch * 4;
+            const bool skipped = (sk >> j) & 1ull;
+            if (!skipped)
+                *reinterpret_cast<uint4*>(a.dkread + g) = *reinterpret_cast<const uint4*>(sm + ST_DKR + j * 512 + ch * 16);
+            if (!skipped || j == 0 || !((sk >> (j - 1)) & 1ull))
+                *reinterpret_cast<uint4*>(a.dktil + g) = *reinterpret_cast<const uint4*>(sm + ST_DKT + j * 512 + ch * 16);
+        }
+    }
     OSDN_CLK(3, 12, blockIdx.x == 5 && blockIdx.y == 0);
     if (tid == 0) {
         float tot = 0.f;
