@@ -121,6 +121,66 @@ __device__ __forceinline__ void zero_tail_rows(uint8_t* box, int len, int tid, i
 }
 
 // ---------------------------------------------------------------------------------------------
+// T = (I + A)^-1 for a 64 x 64 strictly lower triangular A (fp32, shared memory, row stride LC),
+// by 16 x 16 blocks: the four diagonal blocks by forward substitution with a column per thread in
+// registers, then block by block away from the diagonal,
+//     T_bc = -T_bb sum_{m=c}^{b-1} A_bm T_mc            (b > c).
+// The inner sums are parked in the unused upper triangle of A (block (c, b)).  Called by all 128
+// threads of the CTA; ends with a barrier.
+// ---------------------------------------------------------------------------------------------
+constexpr int LC = CH + 1;
+
+__device__ __forceinline__ void ut_inverse_64(float* sA, float* sT, int tid)
+{
+    for (int e = tid; e < CH * CH; e += 128) sT[(e >> 6) * LC + (e & 63)] = 0.f;
+    __syncthreads();
+    if (tid < CH) {
+        const int b = tid >> 4, col = tid & 15;
+        const float* Ab = sA + (16 * b) * LC + 16 * b;
+        float x[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] = i == col ? 1.f : 0.f;
+#pragma unroll
+        for (int j = 0; j < 15; ++j) {
+#pragma unroll
+            for (int i = j + 1; i < 16; ++i) x[i] = fmaf(-Ab[i * LC + j], x[j], x[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sT[(16 * b + i) * LC + 16 * b + col] = x[i];
+    }
+    __syncthreads();
+    for (int d = 1; d < 4; ++d) {
+        const int nblk = 4 - d;   // blocks (b, b - d), b = d .. 3
+        // X_bc = sum_m A_bm T_mc  -> upper triangle of A, block (c, b)
+        for (int e = tid; e < nblk * 256; e += 128) {
+            const int p = e >> 8, r = (e >> 4) & 15, cc = e & 15;
+            const int b = d + p, c = p;
+            float acc = 0.f;
+            for (int m = c; m < b; ++m) {
+                const float* Am = sA + (16 * b + r) * LC + 16 * m;
+                const float* Tm = sT + (16 * m) * LC + 16 * c + cc;
+#pragma unroll 4
+                for (int k = 0; k < 16; ++k) acc = fmaf(Am[k], Tm[k * LC], acc);
+            }
+            sA[(16 * c + r) * LC + 16 * b + cc] = acc;
+        }
+        __syncthreads();
+        // T_bc = -T_bb X_bc
+        for (int e = tid; e < nblk * 256; e += 128) {
+            const int p = e >> 8, r = (e >> 4) & 15, cc = e & 15;
+            const int b = d + p, c = p;
+            const float* Tb = sT + (16 * b + r) * LC + 16 * b;
+            const float* X = sA + (16 * c) * LC + 16 * b + cc;
+            float acc = 0.f;
+#pragma unroll 4
+            for (int k = 0; k < 16; ++k) acc = fmaf(Tb[k], X[k * LC], acc);
+            sT[(16 * b + r) * LC + 16 * c + cc] = -acc;
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // chunk-local forward
 // ---------------------------------------------------------------------------------------------
 struct TcChunkArgs {
@@ -134,7 +194,6 @@ struct TcChunkArgs {
 };
 
 constexpr int CL_THREADS = 128;
-constexpr int LC = CH + 1;
 constexpr size_t CL_SMEM = 32768 + 16384 + 8192 + 2 * CH * LC * 4 + 1024;
 
 __global__ void __launch_bounds__(CL_THREADS)
@@ -230,7 +289,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {
                     const int j = cb * 16 + x;
-                    sA[j * CH + i] = j < i ? bi * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+                    sA[i * LC + j] = j < i ? bi * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
                 }
             }
         } else {
@@ -262,26 +321,11 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     __syncthreads();
     OSDN_CLK(0, 4, blockIdx.x == 5 && blockIdx.y == 0);
 
-    // ---- T = (I + A)^-1 --------------------------------------------------------------------------
-    // Thread `col` (warps 0-1) solves (I + A) x = e_col with the whole column in registers: after x_j is
-    // final, every later partial sum is updated at once (independent FMAs, broadcast reads of A).
-    // Warps 2-3 meanwhile emit the gated, scaled queries for the backward state chain:
-    // Qg = scale gamma_i Q, same image layout as Q.
-    if (tid < CH) {
-        const int col = tid;
-        float x[CH];
-#pragma unroll
-        for (int i = 0; i < CH; ++i) x[i] = i == col ? 1.f : 0.f;
-#pragma unroll
-        for (int j = 0; j < CH - 1; ++j) {
-            const float xj = x[j];
-#pragma unroll
-            for (int i = j + 1; i < CH; ++i) x[i] = fmaf(-sA[j * CH + i], xj, x[i]);
-        }
-#pragma unroll
-        for (int i = 0; i < CH; ++i) sT[i * LC + col] = x[i];
-    } else if (a.save) {
-        for (int e = tid - CH; e < 2 * CH * 8; e += CL_THREADS - CH) {
+    // ---- T = (I + A)^-1, blocked --------------------------------------------------------------------
+    ut_inverse_64(sA, sT, tid);
+    // gated, scaled queries for the backward state chain: Qg = scale gamma_i Q (same image layout as Q)
+    if (a.save) {
+        for (int e = tid; e < 2 * CH * 8; e += CL_THREADS) {
             const int hf = e >> 9, i = (e >> 3) & 63, ch = e & 7;
             const uint32_t off = sw128_chunk(i, ch);
             const uint4 w = *reinterpret_cast<const uint4*>(sKQ + hf * 16384 + BOX + off);
@@ -296,8 +340,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             *reinterpret_cast<uint4*>(a.Qg + tile * 16384 + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
-    __syncthreads();
-    OSDN_CLK(0, 5, blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- operand images: Tbg (shared), Tb and T (HBM) -----------------------------------------
     for (int e = tid; e < CH * 8; e += CL_THREADS) {
