@@ -299,7 +299,9 @@ class DeviceBundle:
         skip = self.workspace[o1:o1 + n1].view(torch.int32).cpu().numpy().astype("uint32").reshape(-1, H, 2)
         words = self.workspace[o2:o2 + n2].view(torch.int32).cpu().numpy().astype("uint32").reshape(T, H, K // 32)
         import numpy as np
-        bits = ((words[..., None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8).reshape(T, H, K)
+        R = K // 32   # bit l of word r <-> coordinate R * l + r
+        bits = ((words[..., None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8)   # [T,H,R,32]
+        bits = np.ascontiguousarray(bits.transpose(0, 1, 3, 2)).reshape(T, H, K)
         skipped = np.zeros((T, H), dtype=bool)
         c = 0
         t0 = 0

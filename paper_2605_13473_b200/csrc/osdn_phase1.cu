@@ -32,7 +32,7 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
-// One step of the recurrence on the warp-distributed vector d (lane owns coordinates lane + 32 r).
+// One step of the recurrence on the warp-distributed vector d (lane l owns coordinates R l + r).
 //   c = eta b (1 - b <d, kap>) / n ;  x = rho d + c kap ;  d <- clip(x)
 // n_signed: max(sum kap, eps), negated when the floor eps is active.  pass[r]: ballot of the
 // coordinates whose projection passes gradient; all_low: every x strictly below d_min.
@@ -66,13 +66,55 @@ __device__ __forceinline__ void p1_step(float (&d)[R], const float (&kap)[R], fl
     al_out = al;
 }
 
-template <typename T, int R>
-__device__ __forceinline__ float load_key(const T* kp, size_t th, int lane, float (&kk)[R], float (&kap)[R])
+// Lane l of the warp owns the R = K / 32 consecutive coordinates R l .. R l + R - 1, so that a
+// row of K values is one vector access per lane.
+template <int R> __device__ __forceinline__ void load_row(const float* p, int lane, float (&x)[R])
+{
+    if constexpr (R == 4) {
+        const float4 v = *reinterpret_cast<const float4*>(p + 4 * lane);
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    } else {
+        const float2 v = *reinterpret_cast<const float2*>(p + 2 * lane);
+        x[0] = v.x; x[1] = v.y;
+    }
+}
+template <int R> __device__ __forceinline__ void load_row(const __nv_bfloat16* p, int lane, float (&x)[R])
+{
+    if constexpr (R == 4) {
+        const uint2 v = *reinterpret_cast<const uint2*>(p + 4 * lane);
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
+        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
+        x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+    } else {
+        const uint32_t v = *reinterpret_cast<const uint32_t*>(p + 2 * lane);
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
+        x[0] = a.x; x[1] = a.y;
+    }
+}
+template <int R> __device__ __forceinline__ void store_row(float* p, int lane, const float (&x)[R])
+{
+    if constexpr (R == 4) *reinterpret_cast<float4*>(p + 4 * lane) = make_float4(x[0], x[1], x[2], x[3]);
+    else *reinterpret_cast<float2*>(p + 2 * lane) = make_float2(x[0], x[1]);
+}
+template <int R> __device__ __forceinline__ void store_row(__nv_bfloat16* p, int lane, const float (&x)[R])
+{
+    if constexpr (R == 4) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]), b = __floats2bfloat162_rn(x[2], x[3]);
+        uint2 v;
+        v.x = *reinterpret_cast<uint32_t*>(&a);
+        v.y = *reinterpret_cast<uint32_t*>(&b);
+        *reinterpret_cast<uint2*>(p + 4 * lane) = v;
+    } else {
+        __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]);
+        *reinterpret_cast<uint32_t*>(p + 2 * lane) = *reinterpret_cast<uint32_t*>(&a);
+    }
+}
+
+template <int R> __device__ __forceinline__ float square_sum(const float (&kk)[R], float (&kap)[R])
 {
     float sumk = 0.f;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        kk[r] = ldf(kp + th * (32 * R) + lane + 32 * r);
         kap[r] = kk[r] * kk[r];
         sumk += kap[r];
     }
@@ -105,16 +147,21 @@ __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
     const TI* kp = static_cast<const TI*>(a.k);
     TO* kt = static_cast<TO*>(a.ktil);
     float d[R];
+    if (a.d0) load_row<R>(a.d0 + ((size_t)s * a.H + h) * K, lane, d);
+    else {
 #pragma unroll
-    for (int r = 0; r < R; ++r) d[r] = a.d0 ? a.d0[((size_t)s * a.H + h) * K + lane + 32 * r] : 1.0f;
+        for (int r = 0; r < R; ++r) d[r] = 1.0f;
+    }
     const Hyper hy = a.hy;
     for (int i = 0; i < len; ++i) {
         const size_t th = (size_t)(t0 + i) * a.H + h;
-        float kk[R], kap[R];
-        const float sumk = load_key<TI, R>(kp, th, lane, kk, kap);
+        float kk[R], kap[R], w[R];
+        load_row<R>(kp + th * K, lane, kk);
+        const float sumk = square_sum<R>(kk, kap);
         if (kt) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) stf(kt + th * K + lane + 32 * r, d[r] * kk[r]);
+            for (int r = 0; r < R; ++r) w[r] = d[r] * kk[r];
+            store_row<R>(kt + th * K, lane, w);
         }
         const float n = fmaxf(sumk, hy.eps);
         const float b = hy.beta_aware ? a.beta[th] : 1.0f;
@@ -124,8 +171,7 @@ __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
         float c, al;
         p1_step<R>(d, kap, n, b, rho, hy, pass, low, c, al);
     }
-#pragma unroll
-    for (int r = 0; r < R; ++r) a.d_final[((size_t)s * a.H + h) * K + lane + 32 * r] = d[r];
+    store_row<R>(a.d_final + ((size_t)s * a.H + h) * K, lane, d);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -143,7 +189,8 @@ struct P1Fwd {
     Hyper hy;
 };
 
-// one warp per (chunk, head, 32-token half)
+// one warp per (chunk, head, 32-token half); tokens in batches of eight so that eight row loads
+// are in flight at a time
 template <typename TI, typename TO, int K>
 __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
 {
@@ -159,33 +206,55 @@ __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
     TO* kt = static_cast<TO*>(a.ktil);
     const Hyper hy = a.hy;
     unsigned word = 0;
-    for (int j = 0; j < 32; ++j) {
-        const int i = half * 32 + j;
-        if (i >= len) break;
-        const size_t th = (size_t)(tok0 + i) * a.H + h;
-        float kk[R], kap[R];
-        const float sumk = load_key<TI, R>(kp, th, lane, kk, kap);
-        const float n = fmaxf(sumk, hy.eps);
-        const float rho = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
-        if (lane == 0) {
-            a.r.n[th] = sumk > hy.eps ? n : -n;
-            a.r.rho[th] = rho;
+    // per-token scalars: lane j of the warp fetches those of token half*32 + j
+    const int mine = half * 32 + lane;
+    const size_t th_mine = (size_t)(tok0 + min(mine, max(len - 1, 0))) * a.H + h;
+    const float beta_l = (mine < len && hy.beta_aware) ? a.beta[th_mine] : 1.0f;
+    const float ret_l = (mine < len && hy.apf_mode != 0) ? a.retsrc[th_mine] : 0.f;
+    float n_l = 0.f, rho_l = 1.f;
+    for (int j0 = 0; j0 < 32; j0 += 8) {
+        if (half * 32 + j0 >= len) break;
+        float kk[8][R];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = min(half * 32 + j0 + u, len - 1);
+            load_row<R>(kp + ((size_t)(tok0 + i) * a.H + h) * K, lane, kk[u]);
         }
-        if (hy.clamp) {
-            const float b = hy.beta_aware ? a.beta[th] : 1.0f;
-            float d[R];
 #pragma unroll
-            for (int r = 0; r < R; ++r) d[r] = hy.d_min;
-            unsigned pass[R];
-            bool low;
-            float cc, al;
-            p1_step<R>(d, kap, n, b, rho, hy, pass, low, cc, al);
-            if (low) {
-                word |= 1u << j;
+        for (int u = 0; u < 8; ++u) {
+            const int j = j0 + u, i = half * 32 + j;
+            if (i >= len) break;
+            const size_t th = (size_t)(tok0 + i) * a.H + h;
+            float kap[R];
+            const float sumk = square_sum<R>(kk[u], kap);
+            const float n = fmaxf(sumk, hy.eps);
+            const float rho = hy.apf_mode == 0 ? 1.0f : expf(__shfl_sync(0xffffffffu, ret_l, j));
+            const float b = __shfl_sync(0xffffffffu, beta_l, j);
+            if (lane == j) {
+                n_l = sumk > hy.eps ? n : -n;
+                rho_l = rho;
+            }
+            if (hy.clamp) {
+                float d[R];
 #pragma unroll
-                for (int r = 0; r < R; ++r) stf(kt + th * K + lane + 32 * r, hy.d_min * kk[r]);
+                for (int r = 0; r < R; ++r) d[r] = hy.d_min;
+                unsigned pass[R];
+                bool low;
+                float cc, al;
+                p1_step<R>(d, kap, n, b, rho, hy, pass, low, cc, al);
+                if (low) {
+                    word |= 1u << j;
+                    float wk[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) wk[r] = hy.d_min * kk[u][r];
+                    store_row<R>(kt + th * K, lane, wk);
+                }
             }
         }
+    }
+    if (mine < len) {
+        a.r.n[th_mine] = n_l;
+        a.r.rho[th_mine] = rho_l;
     }
     if (lane == 0) a.r.flags[tile * 2 + half] = word;
 }
@@ -198,11 +267,13 @@ template <int R> __device__ __forceinline__ bool on_lower_face(const float (&d)[
     return __all_sync(0xffffffffu, f);
 }
 
-// one warp per chain
+// one warp per chain.  Flag words are fetched for 32 chunks at a time (one chunk per lane); the
+// rows of the tokens that are really processed are prefetched a few tokens ahead.
 template <typename TI, typename TO, int K>
 __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
 {
     constexpr int R = K / 32;
+    constexpr int PF = 8;   // prefetch distance in tokens
     const int lane = threadIdx.x & 31;
     const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (chain >= a.S * a.H) return;
@@ -211,67 +282,104 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
     TO* kt = static_cast<TO*>(a.ktil);
     const Hyper hy = a.hy;
     float d[R];
+    if (a.d0) load_row<R>(a.d0 + ((size_t)s * H + h) * K, lane, d);
+    else {
 #pragma unroll
-    for (int r = 0; r < R; ++r) d[r] = a.d0 ? a.d0[((size_t)s * H + h) * K + lane + 32 * r] : 1.0f;
+        for (int r = 0; r < R; ++r) d[r] = 1.0f;
+    }
     bool face = on_lower_face<R>(d, hy);
     const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
-    for (int c = c0; c < c1; ++c) {
-        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
-        const size_t tile = (size_t)c * H + h;
-        const unsigned long long bits =
-            (unsigned long long)a.r.flags[tile * 2] | ((unsigned long long)a.r.flags[tile * 2 + 1] << 32);
-        const unsigned long long valid = len >= 64 ? ~0ull : ((1ull << len) - 1ull);
-        if (a.save) {
-#pragma unroll
-            for (int r = 0; r < R; ++r) a.r.dbound[tile * K + lane + 32 * r] = d[r];
+    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
+    for (int cbase = c0; cbase < c1; cbase += 32) {
+        unsigned w0 = 0, w1 = 0;
+        if (cbase + lane < c1) {
+            const size_t tl = (size_t)(cbase + lane) * H + h;
+            w0 = a.r.flags[tl * 2];
+            w1 = a.r.flags[tl * 2 + 1];
         }
-        unsigned long long skipped = 0ull;
-        if (face && (bits & valid) == valid) {
-            skipped = valid;
-        } else {
-            for (int i = 0; i < len; ++i) {
-                if (face && ((bits >> i) & 1ull)) {
-                    skipped |= 1ull << i;
-                    continue;
-                }
-                const size_t th = (size_t)(tok0 + i) * H + h;
-                float kk[R], kap[R];
+        const int cend = min(cbase + 32, c1);
+        for (int c = cbase; c < cend; ++c) {
+            const int nrel = c - c0;
+            const int tok0 = seq_t0 + nrel * CH, len = min(CH, seq_len - nrel * CH);
+            const size_t tile = (size_t)c * H + h;
+            const unsigned long long bits = (unsigned long long)__shfl_sync(0xffffffffu, w0, c - cbase) |
+                                            ((unsigned long long)__shfl_sync(0xffffffffu, w1, c - cbase) << 32);
+            const unsigned long long valid = len >= 64 ? ~0ull : ((1ull << len) - 1ull);
+            if (a.save) store_row<R>(a.r.dbound + tile * K, lane, d);
+            unsigned long long skipped = 0ull;
+            if (face && (bits & valid) == valid) {
+                skipped = valid;
+            } else {
+                // ring of prefetched rows and scalars
+                float kbuf[PF][R], nbuf[PF], rbuf[PF], bbuf[PF];
+                auto fetch = [&](int i, int slot) {
+                    const int ii = min(i, len - 1);
+                    const size_t th = (size_t)(tok0 + ii) * H + h;
+                    load_row<R>(kp + th * K, lane, kbuf[slot]);
+                    nbuf[slot] = a.r.n[th];
+                    rbuf[slot] = a.r.rho[th];
+                    bbuf[slot] = hy.beta_aware ? a.beta[th] : 1.0f;
+                };
+                int i = 0;
+                while (i < len) {
+                    if (face) {
+                        // jump over the flagged tokens that follow while d stays on the face
+                        const unsigned long long rest = (~bits & valid) >> i;
+                        const int run = rest ? __ffsll((long long)rest) - 1 : len - i;
+                        if (run > 0) {
+                            skipped |= (run >= 64 ? ~0ull : ((1ull << run) - 1ull)) << i;
+                            i += run;
+                            continue;
+                        }
+                    }
+                    // process tokens i, i+1, ... until d is back on the face (or the chunk ends)
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    kk[r] = ldf(kp + th * K + lane + 32 * r);
-                    kap[r] = kk[r] * kk[r];
-                }
-                const float n = fabsf(a.r.n[th]);
-                const float rho = a.r.rho[th];
-                const float b = hy.beta_aware ? a.beta[th] : 1.0f;
+                    for (int u = 0; u < PF; ++u) fetch(i + u, u);
+                    bool stop = false;
+                    while (i < len && !stop) {
 #pragma unroll
-                for (int r = 0; r < R; ++r) stf(kt + th * K + lane + 32 * r, d[r] * kk[r]);
-                if (a.save) {
+                        for (int u = 0; u < PF; ++u) {
+                            if (i < len && !stop) {
+                                float kk[R];
 #pragma unroll
-                    for (int r = 0; r < R; ++r) a.r.dtraj[th * K + lane + 32 * r] = d[r];
-                }
-                unsigned pass[R];
-                bool low;
-                float cc, al;
-                p1_step<R>(d, kap, n, b, rho, hy, pass, low, cc, al);
-                if (a.save && lane < R) {
-                    unsigned wv = 0;
+                                for (int r = 0; r < R; ++r) kk[r] = kbuf[u][r];
+                                const float n = fabsf(nbuf[u]), rho = rbuf[u], b = bbuf[u];
+                                fetch(i + PF, u);
+                                const size_t th = (size_t)(tok0 + i) * H + h;
+                                float kap[R], wk[R];
 #pragma unroll
-                    for (int r = 0; r < R; ++r) wv = lane == r ? pass[r] : wv;
-                    a.r.pmask[th * R + lane] = wv;
+                                for (int r = 0; r < R; ++r) {
+                                    kap[r] = kk[r] * kk[r];
+                                    wk[r] = d[r] * kk[r];
+                                }
+                                store_row<R>(kt + th * K, lane, wk);
+                                if (a.save) store_row<R>(a.r.dtraj + th * K, lane, d);
+                                unsigned pass[R];
+                                bool low;
+                                float cc, al;
+                                p1_step<R>(d, kap, n, b, rho, hy, pass, low, cc, al);
+                                if (a.save && lane < R) {
+                                    unsigned wv = 0;
+#pragma unroll
+                                    for (int r = 0; r < R; ++r) wv = lane == r ? pass[r] : wv;
+                                    a.r.pmask[th * R + lane] = wv;
+                                }
+                                face = on_lower_face<R>(d, hy);
+                                ++i;
+                                // back on the face with a flagged token next: leave the run
+                                stop = face && i < len && ((bits >> i) & 1ull);
+                            }
+                        }
+                    }
                 }
-                face = on_lower_face<R>(d, hy);
+            }
+            if (a.save && lane == 0) {
+                a.r.skipw[tile * 2] = (unsigned)(skipped & 0xffffffffull);
+                a.r.skipw[tile * 2 + 1] = (unsigned)(skipped >> 32);
             }
         }
-        if (a.save && lane == 0) {
-            a.r.skipw[tile * 2] = (unsigned)(skipped & 0xffffffffull);
-            a.r.skipw[tile * 2 + 1] = (unsigned)(skipped >> 32);
-        }
     }
-    if (a.d_final) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) a.d_final[((size_t)s * H + h) * K + lane + 32 * r] = d[r];
-    }
+    if (a.d_final) store_row<R>(a.d_final + ((size_t)s * H + h) * K, lane, d);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -307,15 +415,16 @@ __global__ void __launch_bounds__(128) phase1_bwd_bulk_kernel(P1Bwd a)
         if (i >= len) break;
         if (!((word >> j) & 1u)) continue;
         const size_t th = (size_t)(tok0 + i) * a.H + h;
+        float x[R], y[R];
+        load_row<R>(a.dkread + th * K, lane, x);
+        load_row<R>(a.dktil + th * K, lane, y);
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const size_t e = th * K + lane + 32 * r;
-            stf(dkp + e, a.dkread[e] + a.hy.d_min * a.dktil[e]);
-        }
+        for (int r = 0; r < R; ++r) x[r] = fmaf(a.hy.d_min, y[r], x[r]);
+        store_row<R>(dkp + th * K, lane, x);
     }
 }
 
-// processed tokens, in reverse; one warp per chain
+// processed tokens, in reverse; one warp per chain.  Skip words are fetched for 32 chunks at a time.
 template <typename T, int K>
 __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
 {
@@ -328,84 +437,133 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
     const T* kp = static_cast<const T*>(a.k);
     T* dkp = static_cast<T*>(a.dk);
     float lam[R];
+    if (a.dprecond_out) load_row<R>(a.dprecond_out + ((size_t)s * H + h) * K, lane, lam);
+    else {
 #pragma unroll
-    for (int r = 0; r < R; ++r)
-        lam[r] = a.dprecond_out ? a.dprecond_out[((size_t)s * H + h) * K + lane + 32 * r] : 0.f;
+        for (int r = 0; r < R; ++r) lam[r] = 0.f;
+    }
     bool lam_valid = true;     // lam holds dL/dd_{t+1} for the token about to be processed
     long src = -1;             // otherwise it is k (.) dktil of this (skipped) token
+    auto restart = [&](long tsrc) {
+        const size_t ts = (size_t)tsrc * H + h;
+        float kk[R], dk[R];
+        load_row<R>(kp + ts * K, lane, kk);
+        load_row<R>(a.dktil + ts * K, lane, dk);
+#pragma unroll
+        for (int r = 0; r < R; ++r) lam[r] = kk[r] * dk[r];
+    };
     const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
-    for (int c = c1 - 1; c >= c0; --c) {
-        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
-        const size_t tile = (size_t)c * H + h;
-        const unsigned long long sk =
-            (unsigned long long)a.r.skipw[tile * 2] | ((unsigned long long)a.r.skipw[tile * 2 + 1] << 32);
-        const unsigned long long valid = len >= 64 ? ~0ull : ((1ull << len) - 1ull);
-        if ((sk & valid) == valid) {
-            lam_valid = false;
-            src = tok0;
-            continue;
+    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
+    for (int ctop = c1; ctop > c0; ctop -= 32) {
+        // lane j holds the words of chunk ctop - 1 - j
+        unsigned w0 = 0, w1 = 0;
+        if (ctop - 1 - lane >= c0) {
+            const size_t tl = (size_t)(ctop - 1 - lane) * H + h;
+            w0 = a.r.skipw[tl * 2];
+            w1 = a.r.skipw[tl * 2 + 1];
         }
-        for (int i = len - 1; i >= 0; --i) {
-            if ((sk >> i) & 1ull) {
+        const int cbot = max(ctop - 32, c0);
+        for (int c = ctop - 1; c >= cbot; --c) {
+            const int nrel = c - c0;
+            const int tok0 = seq_t0 + nrel * CH, len = min(CH, seq_len - nrel * CH);
+            const unsigned long long sk = (unsigned long long)__shfl_sync(0xffffffffu, w0, ctop - 1 - c) |
+                                          ((unsigned long long)__shfl_sync(0xffffffffu, w1, ctop - 1 - c) << 32);
+            const unsigned long long valid = len >= 64 ? ~0ull : ((1ull << len) - 1ull);
+            if ((sk & valid) == valid) {
                 lam_valid = false;
-                src = tok0 + i;
+                src = tok0;
                 continue;
             }
-            if (!lam_valid) {
-                const size_t ts = (size_t)src * H + h;
+            constexpr int PF = 4;
+            float kb[PF][R], db[PF][R], tb[PF][R], rb[PF][R], nb[PF], hb[PF], bb[PF];
+            unsigned mb[PF];
+            auto fetch = [&](int i, int slot) {
+                const int ii = max(i, 0);
+                const size_t th = (size_t)(tok0 + ii) * H + h;
+                load_row<R>(kp + th * K, lane, kb[slot]);
+                load_row<R>(a.r.dtraj + th * K, lane, db[slot]);
+                load_row<R>(a.dktil + th * K, lane, tb[slot]);
+                load_row<R>(a.dkread + th * K, lane, rb[slot]);
+                mb[slot] = lane < R ? a.r.pmask[th * R + lane] : 0u;
+                nb[slot] = a.r.n[th];
+                hb[slot] = a.r.rho[th];
+                bb[slot] = hy.beta_aware ? a.beta[th] : 1.0f;
+            };
+            int i = len - 1;
+            while (i >= 0) {
+                if ((sk >> i) & 1ull) {
+                    // run of skipped tokens: the recurrence restarts at its lowest token
+                    const unsigned long long below = i >= 63 ? ~0ull : ((1ull << (i + 1)) - 1ull);
+                    const unsigned long long real = ~sk & valid & below;
+                    lam_valid = false;
+                    if (!real) {
+                        src = tok0;
+                        break;
+                    }
+                    const int j = 63 - __clzll((long long)real);
+                    src = tok0 + j + 1;
+                    i = j;
+                }
 #pragma unroll
-                for (int r = 0; r < R; ++r)
-                    lam[r] = ldf(kp + ts * K + lane + 32 * r) * a.dktil[ts * K + lane + 32 * r];
-                lam_valid = true;
-            }
-            const size_t th = (size_t)(tok0 + i) * H + h;
-            float kk[R], kap[R], dt[R], dkt[R], drho = 0.f, dc = 0.f, al = 0.f;
-            unsigned mw = lane < R ? a.r.pmask[th * R + lane] : 0u;
+                for (int u = 0; u < PF; ++u) fetch(i - u, u);
+                bool stop = false;
+                while (i >= 0 && !stop) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const size_t e = th * K + lane + 32 * r;
-                kk[r] = ldf(kp + e);
-                kap[r] = kk[r] * kk[r];
-                dt[r] = a.r.dtraj[e];
-                dkt[r] = a.dktil[e];
-                const unsigned wr = __shfl_sync(0xffffffffu, mw, r);
-                if (!((wr >> lane) & 1u)) lam[r] = 0.f;
-                drho = fmaf(lam[r], dt[r], drho);
-                dc = fmaf(lam[r], kap[r], dc);
-                al = fmaf(dt[r], kap[r], al);
-            }
-            drho = warp_sum(drho);
-            dc = warp_sum(dc);
-            al = warp_sum(al);
-            const float ns = a.r.n[th], n = fabsf(ns), rho = a.r.rho[th];
-            const float b = hy.beta_aware ? a.beta[th] : 1.0f;
-            const float cc = hy.eta * b * (1.0f - b * al) / n;
-            const float da = -hy.eta * b * b / n * dc;
-            const float db = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
-            const float dn = ns > 0.f ? -cc / n * dc : 0.f;
+                    for (int u = 0; u < PF; ++u) {
+                        if (i >= 0 && !stop) {
+                            float kk[R], kap[R], dt[R], dkt[R], dkr[R], drho = 0.f, dc = 0.f, al = 0.f;
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const size_t e = th * K + lane + 32 * r;
-                const float dkap = cc * lam[r] + da * dt[r] + dn;
-                stf(dkp + e, a.dkread[e] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap);
-                lam[r] = rho * lam[r] + da * kap[r] + kk[r] * dkt[r];
-            }
-            if (lane == 0) {
-                if (hy.beta_aware) a.dbeta[th] += db;
-                if (hy.apf_mode == 1) a.dgate[th] += rho * drho;
-                if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
+                            for (int r = 0; r < R; ++r) {
+                                kk[r] = kb[u][r]; dt[r] = db[u][r]; dkt[r] = tb[u][r]; dkr[r] = rb[u][r];
+                            }
+                            const unsigned mw = mb[u];
+                            const float ns = nb[u], n = fabsf(ns), rho = hb[u], b = bb[u];
+                            fetch(i - PF, u);
+                            if (!lam_valid) {
+                                restart(src);
+                                lam_valid = true;
+                            }
+                            const size_t th = (size_t)(tok0 + i) * H + h;
+#pragma unroll
+                            for (int r = 0; r < R; ++r) {
+                                kap[r] = kk[r] * kk[r];
+                                const unsigned wr = __shfl_sync(0xffffffffu, mw, r);
+                                if (!((wr >> lane) & 1u)) lam[r] = 0.f;
+                                drho = fmaf(lam[r], dt[r], drho);
+                                dc = fmaf(lam[r], kap[r], dc);
+                                al = fmaf(dt[r], kap[r], al);
+                            }
+                            drho = warp_sum(drho);
+                            dc = warp_sum(dc);
+                            al = warp_sum(al);
+                            const float cc = hy.eta * b * (1.0f - b * al) / n;
+                            const float da = -hy.eta * b * b / n * dc;
+                            const float dbt = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
+                            const float dn = ns > 0.f ? -cc / n * dc : 0.f;
+                            float out[R];
+#pragma unroll
+                            for (int r = 0; r < R; ++r) {
+                                const float dkap = cc * lam[r] + da * dt[r] + dn;
+                                out[r] = dkr[r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
+                                lam[r] = rho * lam[r] + da * kap[r] + kk[r] * dkt[r];
+                            }
+                            store_row<R>(dkp + th * K, lane, out);
+                            if (lane == 0) {
+                                if (hy.beta_aware) a.dbeta[th] += dbt;
+                                if (hy.apf_mode == 1) a.dgate[th] += rho * drho;
+                                if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
+                            }
+                            --i;
+                            stop = i >= 0 && ((sk >> i) & 1ull);
+                        }
+                    }
+                }
             }
         }
     }
     if (a.dprecond_in) {
-        if (!lam_valid) {
-            const size_t ts = (size_t)src * H + h;
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                lam[r] = ldf(kp + ts * K + lane + 32 * r) * a.dktil[ts * K + lane + 32 * r];
-        }
-#pragma unroll
-        for (int r = 0; r < R; ++r) a.dprecond_in[((size_t)s * H + h) * K + lane + 32 * r] = lam[r];
+        if (!lam_valid) restart(src);
+        store_row<R>(a.dprecond_in + ((size_t)s * H + h) * K, lane, lam);
     }
 }
 

@@ -421,6 +421,7 @@ struct TcChainArgs {
 };
 
 constexpr int CF_THREADS = 256;
+constexpr int CF2_THREADS = 512;   // forward chain: 16 warps = 4 lane quadrants x 4 column groups
 constexpr uint32_t STAGE_BYTES = 16384 + 8192 + 8192 + 3 * 16384;   // WT, Tb, P, V, Q, Ktil = 81920
 constexpr uint32_t ST_WT = 0, ST_TB = 16384, ST_P = 24576, ST_V = 32768, ST_Q = 49152, ST_KT = 65536;
 constexpr size_t CF_SMEM = 2 * STAGE_BYTES + 32768 + 2 * 16384 + 1024;
@@ -444,7 +445,7 @@ __device__ __forceinline__ void warp_gate_vectors(float ga, float gb, int lane, 
     if (lane == 0) *gC = __expf(tot);
 }
 
-__global__ void __launch_bounds__(CF_THREADS, 1)
+__global__ void __launch_bounds__(CF2_THREADS, 1)
 tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
                     const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
 {
@@ -463,13 +464,13 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
     const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int quad = warp & 3, colhalf = warp >> 2;
+    const int quad = warp & 3, colq = warp >> 2;   // lane quadrant, column group (4 groups)
     const int v = quad * 32 + lane;             // state row owned by this thread
-    float* fin = a.final_state ? a.final_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
-    const float* ini = a.init_state ? a.init_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
+    float* fin = a.final_state ? a.final_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
+    const float* ini = a.init_state ? a.init_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
     if (c1 <= c0) {   // empty sequence: the state passes through
         if (fin)
-            for (int x = 0; x < 64; ++x) fin[x] = ini ? ini[x] : 0.f;
+            for (int x = 0; x < 32; ++x) fin[x] = ini ? ini[x] : 0.f;
         return;
     }
     const int nchunks = c1 - c0;
@@ -515,37 +516,31 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     auto store_out = [&](int n) {
         const int tok0 = chunk_tok0(n), len = chunk_len(n), st = n & 1, gs = n % 3;
         __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
-        uint32_t ra[2][16], rb[2][16];
-#pragma unroll
-        for (int cb = 0; cb < 2; ++cb) {
-            tmem_ld16(tO1 + st * 64 + lane_addr + colhalf * 32 + cb * 16, ra[cb]);
-            tmem_ld16(tO2 + st * 64 + lane_addr + colhalf * 32 + cb * 16, rb[cb]);
-        }
+        uint32_t ra[16], rb[16];
+        tmem_ld16(tO1 + st * 64 + lane_addr + colq * 16, ra);
+        tmem_ld16(tO2 + st * 64 + lane_addr + colq * 16, rb);
         tmem_ld_wait();
 #pragma unroll
-        for (int cb = 0; cb < 2; ++cb) {
-#pragma unroll
-            for (int x = 0; x < 16; ++x) {
-                const int i = colhalf * 32 + cb * 16 + x;
-                if (i < len)
-                    op[(size_t)i * H * KD] = __float2bfloat16_rn(
-                        a.scale * sGam[gs][i] * __uint_as_float(ra[cb][x]) + __uint_as_float(rb[cb][x]));
-            }
+        for (int x = 0; x < 16; ++x) {
+            const int i = colq * 16 + x;
+            if (i < len)
+                op[(size_t)i * H * KD] = __float2bfloat16_rn(a.scale * sGam[gs][i] * __uint_as_float(ra[x]) +
+                                                             __uint_as_float(rb[x]));
         }
     };
 
     if (tid == 0) issue_loads(0, 0);
     float ga = 0.f, gb = 0.f;
-    if (warp == 7) {
+    if (warp == 15) {
         load_gates(0, ga, gb);
         warp_gate_vectors(ga, gb, lane, sGam[0], sRho[0], &sGC[0]);
     }
     // initial state into tensor memory
-    for (int cb = 0; cb < 4; ++cb) {
+    for (int cb = 0; cb < 2; ++cb) {
         uint32_t r[16];
 #pragma unroll
         for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(ini ? ini[cb * 16 + x] : 0.f);
-        tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+        tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
     }
     tmem_st_wait();
     tc_fence_before();
@@ -559,19 +554,19 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         const size_t tile = (size_t)(c0 + n) * H + h;
         uint8_t* d = sStage + st * STAGE_BYTES;
         if (tid == 0 && n + 1 < nchunks) issue_loads(n + 1, st ^ 1);
-        if (warp == 7 && n + 1 < nchunks) load_gates(n + 1, ga, gb);   // consumed after MMA group 2 is issued
+        if (warp == 15 && n + 1 < nchunks) load_gates(n + 1, ga, gb);   // consumed after MMA group 2 is issued
     OSDN_CLK(1, 0, blockIdx.x == 0 && n == 3);
 
         // ---- E0: S -> bf16 operand (+ saved copy), decay the accumulator -----------------------
         {
             const float gC = sGC[gs];
-            uint8_t* Sg = a.Sn + tile * 32768 + colhalf * 16384;
-            uint32_t rr[4][16];
+            uint8_t* Sg = a.Sn + tile * 32768 + (colq >> 1) * 16384;
+            uint32_t rr[2][16];
 #pragma unroll
-            for (int cb = 0; cb < 4; ++cb) tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, rr[cb]);
+            for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
             tmem_ld_wait();
 #pragma unroll
-            for (int cb = 0; cb < 4; ++cb) {
+            for (int cb = 0; cb < 2; ++cb) {
                 uint32_t* r = rr[cb];
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
@@ -580,13 +575,13 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                     w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
                     w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
                     w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
-                    const uint32_t off = sw128_chunk(v, cb * 2 + c2);
-                    *reinterpret_cast<uint4*>(sS + colhalf * 16384 + off) = w;
+                    const uint32_t off = sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2);
+                    *reinterpret_cast<uint4*>(sS + (colq >> 1) * 16384 + off) = w;
                     if (a.save) *reinterpret_cast<uint4*>(Sg + off) = w;
                 }
 #pragma unroll
                 for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
-                tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+                tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
             }
             tmem_st_wait();
         }
@@ -595,9 +590,9 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     OSDN_CLK(1, 2, blockIdx.x == 0 && n == 3);
         if (len < CH) {
             for (int hf = 0; hf < 2; ++hf) {
-                zero_tail_rows(d + ST_V + hf * BOX, len, tid, CF_THREADS);
-                zero_tail_rows(d + ST_Q + hf * BOX, len, tid, CF_THREADS);
-                zero_tail_rows(d + ST_KT + hf * BOX, len, tid, CF_THREADS);
+                zero_tail_rows(d + ST_V + hf * BOX, len, tid, CF2_THREADS);
+                zero_tail_rows(d + ST_Q + hf * BOX, len, tid, CF2_THREADS);
+                zero_tail_rows(d + ST_KT + hf * BOX, len, tid, CF2_THREADS);
             }
         }
         fence_proxy_async();
@@ -636,22 +631,19 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         // ---- E1: dU^T -> bf16 operands ---------------------------------------------------------
         {
             uint8_t* dUg = a.dUT + tile * 16384;
-            uint32_t rr[2][16];
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) tmem_ld16(tDU + lane_addr + colhalf * 32 + cb * 16, rr[cb]);
+            uint32_t r[16];
+            tmem_ld16(tDU + lane_addr + colq * 16, r);
             tmem_ld_wait();
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                uint32_t* r = rr[cb];
+            {
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     float f[8], g[8];
 #pragma unroll
                     for (int x = 0; x < 8; ++x) {
                         f[x] = __uint_as_float(r[c2 * 8 + x]);
-                        g[x] = f[x] * sRho[gs][colhalf * 32 + cb * 16 + c2 * 8 + x];
+                        g[x] = f[x] * sRho[gs][colq * 16 + c2 * 8 + x];
                     }
-                    const uint32_t off = sw128_chunk(v, colhalf * 4 + cb * 2 + c2);
+                    const uint32_t off = sw128_chunk(v, colq * 2 + c2);
                     const uint4 w1 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
                                                 pack_bf16(f[6], f[7]));
                     *reinterpret_cast<uint4*>(sDU1 + off) = w1;
@@ -686,7 +678,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         // while the tensor core works: gate vectors of the next chunk, output of the previous chunk
         // (its O2 accumulator was issued after the previous chunk's last commit and is covered by
         // this chunk's first commit, which has been waited for above)
-        if (warp == 7 && n + 1 < nchunks)
+        if (warp == 15 && n + 1 < nchunks)
             warp_gate_vectors(ga, gb, lane, sGam[(n + 1) % 3], sRho[(n + 1) % 3], &sGC[(n + 1) % 3]);
         if (n > 0 && ok) store_out(n - 1);
         ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
@@ -707,9 +699,9 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     if (ok) store_out(nchunks - 1);
 
     if (fin && ok) {
-        for (int cb = 0; cb < 4; ++cb) {
+        for (int cb = 0; cb < 2; ++cb) {
             uint32_t r[16];
-            tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
+            tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, r);
             tmem_ld_wait();
 #pragma unroll
             for (int x = 0; x < 16; ++x) fin[cb * 16 + x] = __uint_as_float(r[x]);
@@ -1531,7 +1523,7 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
         ch.status = status;
         if (!set_smem(tc_chain_fwd_kernel, CF_SMEM)) return -1;
         stage_mark(st, "tc_chain_fwd");
-        tc_chain_fwd_kernel<<<S * H, CF_THREADS, CF_SMEM, st>>>(tmV, tmQ, tmKt, ch);
+        tc_chain_fwd_kernel<<<S * H, CF2_THREADS, CF_SMEM, st>>>(tmV, tmQ, tmKt, ch);
         ++launches;
     }
     stage_end(st);
