@@ -80,8 +80,23 @@ def kernel_model(name, inp, NT):
                                  + tiles * 4 * (2 * C * C + 2 * C * V + 2 * V * K + 10 * C * K),
                                  tiles * (f(C, C, V) + 5 * f(C, K, V) + f(C, C, K) * 2 + f(C, C, V)
                                           + f(C, K, C) * 5 + f(C, V, C) + 2 * f(C, C, C)), "alu")
-    m["phase1_bwd"] = (tokh * (K * es * 2 + 2 * K * 4 + 24) + tiles * K * 4, tokh * 30.0 * K, "hbm")
     m["build_table"] = (NT * 12, 0.0, "hbm")
+    # phase 1 (both families)
+    m["phase1_spec"] = (tokh * (2 * K * es + 16), tokh * 12.0 * K, "hbm")
+    m["phase1_seq"] = (tiles * (16 + K * 4), 0.0, "hbm")          # pinned regime: flag words + chunk-start d
+    m["phase1_bwd_seq"] = (tiles * 8, 0.0, "hbm")
+    m["phase1_bwd_bulk"] = (tokh * (2 * K * 4 + K * es), tokh * 2.0 * K, "hbm")
+    # tensor-core family: bytes of the tiles each kernel must read and write (bf16 images)
+    raw = C * K * es                                               # one [64 x 128] user tile
+    m["tc_chunk_fwd"] = (tiles * (3 * raw + 16384 + 8192 + 8192 + 8192 + 16384) + tokh * 8,
+                         tiles * (f(128, 64, K) + f(128, 64, C)), "hbm")
+    m["tc_chain_fwd"] = (tiles * (16384 + 8192 + 8192 + 3 * raw + raw + 32768 + 16384) + tokh * 4,
+                         tiles * (f(128, 64, C) + 2 * f(128, 64, K) + f(128, 64, C) + f(128, 128, C)), "hbm")
+    m["tc_chain_bwd"] = (tiles * (2 * raw + 8192 + 16384 + 16384 + 32768 + 16384) + tokh * 4,
+                         tiles * (f(128, 64, C) + f(128, 64, K) + 2 * f(128, 128, C)), "hbm")
+    m["tc_chunk_bwd"] = (tiles * (5 * raw + 16384 + 16384 + 8192 + 32768 + 32768 + 3 * raw) + tokh * 24,
+                         tiles * (2 * f(64, 64, K) + 3 * f(128, 64, K) + 2 * f(64, 64, K) + 2 * f(128, 64, C)
+                                  + 2 * f(64, 64, C) + 4 * f(128, 64, C)), "hbm")
     return m.get(name)
 
 
@@ -286,20 +301,18 @@ def main():
         nb = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts if t is not None))
         e2e = dict(ms=ms_host, h2d=nb(hq, hk, hv, hb, hg, hdo), d2h=nb(hout, hdq, hdk, hdv, hdb, hdg))
 
-    # ---- max over ranks ----------------------------------------------------------------------
-    if world > 1:
-        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t[0])
-        if e2e:
-            e2e["ms"] = float(t[1])
+    # ---- whole-job numbers: units summed over ranks, time = max over ranks ----------------------
+    from paper_2605_13473_b200.sharding import aggregate_throughput
+    total_tokens, ms_total, _ = aggregate_throughput(tokens * steps, ms_total, dev)
+    if e2e:
+        _, e2e["ms"], _ = aggregate_throughput(tokens * steps, e2e["ms"], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     peaks = load_peaks()
-    value = tokens * world * steps / (ms_total * 1e-3)
+    value = total_tokens / (ms_total * 1e-3)
     # dominant kernel and its roofline
     totals = {k: sum(v) for k, v in stages.items()}
     NT = sum((L + 63) // 64 for L in inp.seq_lens)
@@ -363,7 +376,7 @@ def main():
         "config": {"workload": w["desc"], "l2": "inputs + workspace exceed L2 (no flush)",
                    "path": "simt" if args.simt else "auto", "tokens_per_step_per_gpu": tokens},
         "clocks": clocks, "gpu_launches": launches,
-        "e2e": ({"value": tokens * world * steps / (e2e["ms"] * 1e-3), "unit": "tokens/s",
+        "e2e": ({"value": total_tokens / (e2e["ms"] * 1e-3), "unit": "tokens/s",
                  "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"]} if e2e else None),
         "roofline": roofline, "step_roofline": step_roof, "kernels": kernel_table, "cpu_baseline": cpu_baseline,
     }
