@@ -130,8 +130,70 @@ __device__ __forceinline__ void zero_tail_rows(uint8_t* box, int len, int tid, i
 // ---------------------------------------------------------------------------------------------
 constexpr int LC = CH + 1;
 
+// fp32 value as a TF32 operand (round to nearest)
+__device__ __forceinline__ uint32_t to_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+
+// Warp-level 16x8x8 TF32 MMA (fp32 accumulate).  The 16 x 16 blocks of the triangular solve are
+// below the smallest tcgen05 tile (M = 64), so they use the warp-level tensor path.
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// acc (16 x 16, two 16 x 8 fragments) += A (16 x 16) * B (16 x 16), fp32 in shared memory with row
+// stride LC, evaluated as three TF32 products (hi*hi + hi*lo + lo*hi) to keep fp32 accuracy.  One warp.
+__device__ __forceinline__ void block16_mma(float (&acc)[2][4], const float* A, const float* B, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int kt = 0; kt < 2; ++kt) {
+        float af[4] = {A[g * LC + 8 * kt + t], A[(g + 8) * LC + 8 * kt + t], A[g * LC + 8 * kt + t + 4],
+                       A[(g + 8) * LC + 8 * kt + t + 4]};
+        uint32_t ah[4], al[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            ah[x] = to_tf32(af[x]);
+            al[x] = to_tf32(af[x] - __uint_as_float(ah[x]));
+        }
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            float bf[2] = {B[(8 * kt + t) * LC + 8 * nt + g], B[(8 * kt + t + 4) * LC + 8 * nt + g]};
+            uint32_t bh[2], bl[2];
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                bh[x] = to_tf32(bf[x]);
+                bl[x] = to_tf32(bf[x] - __uint_as_float(bh[x]));
+            }
+            mma_tf32(acc[nt], al, bh);
+            mma_tf32(acc[nt], ah, bl);
+            mma_tf32(acc[nt], ah, bh);
+        }
+    }
+}
+
+// store a 16 x 16 accumulator (optionally negated) to shared memory
+__device__ __forceinline__ void block16_store(float* C, const float (&acc)[2][4], float sign, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+        C[g * LC + 8 * nt + 2 * t] = sign * acc[nt][0];
+        C[g * LC + 8 * nt + 2 * t + 1] = sign * acc[nt][1];
+        C[(g + 8) * LC + 8 * nt + 2 * t] = sign * acc[nt][2];
+        C[(g + 8) * LC + 8 * nt + 2 * t + 1] = sign * acc[nt][3];
+    }
+}
+
 __device__ __forceinline__ void ut_inverse_64(float* sA, float* sT, int tid)
 {
+    const int warp = tid >> 5, lane = tid & 31;
     for (int e = tid; e < CH * CH; e += 128) sT[(e >> 6) * LC + (e & 63)] = 0.f;
     __syncthreads();
     if (tid < CH) {
@@ -150,31 +212,19 @@ __device__ __forceinline__ void ut_inverse_64(float* sA, float* sT, int tid)
     }
     __syncthreads();
     for (int d = 1; d < 4; ++d) {
-        const int nblk = 4 - d;   // blocks (b, b - d), b = d .. 3
-        // X_bc = sum_m A_bm T_mc  -> upper triangle of A, block (c, b)
-        for (int e = tid; e < nblk * 256; e += 128) {
-            const int p = e >> 8, r = (e >> 4) & 15, cc = e & 15;
-            const int b = d + p, c = p;
-            float acc = 0.f;
-            for (int m = c; m < b; ++m) {
-                const float* Am = sA + (16 * b + r) * LC + 16 * m;
-                const float* Tm = sT + (16 * m) * LC + 16 * c + cc;
-#pragma unroll 4
-                for (int k = 0; k < 16; ++k) acc = fmaf(Am[k], Tm[k * LC], acc);
-            }
-            sA[(16 * c + r) * LC + 16 * b + cc] = acc;
-        }
-        __syncthreads();
-        // T_bc = -T_bb X_bc
-        for (int e = tid; e < nblk * 256; e += 128) {
-            const int p = e >> 8, r = (e >> 4) & 15, cc = e & 15;
-            const int b = d + p, c = p;
-            const float* Tb = sT + (16 * b + r) * LC + 16 * b;
-            const float* X = sA + (16 * c) * LC + 16 * b + cc;
-            float acc = 0.f;
-#pragma unroll 4
-            for (int k = 0; k < 16; ++k) acc = fmaf(Tb[k], X[k * LC], acc);
-            sT[(16 * b + r) * LC + 16 * c + cc] = -acc;
+        // warp p handles block (b, c) = (d + p, p): X = sum_m A_bm T_mc, parked in the upper triangle
+        // of A (block (c, b)), then T_bc = -T_bb X
+        if (warp < 4 - d) {
+            const int b = d + warp, c = warp;
+            float acc[2][4] = {};
+            for (int m = c; m < b; ++m)
+                block16_mma(acc, sA + (16 * b) * LC + 16 * m, sT + (16 * m) * LC + 16 * c, lane);
+            float* X = sA + (16 * c) * LC + 16 * b;
+            block16_store(X, acc, 1.f, lane);
+            __syncwarp();
+            float acc2[2][4] = {};
+            block16_mma(acc2, sT + (16 * b) * LC + 16 * b, X, lane);
+            block16_store(sT + (16 * b) * LC + 16 * c, acc2, -1.f, lane);
         }
         __syncthreads();
     }
@@ -194,7 +244,7 @@ struct TcChunkArgs {
 };
 
 constexpr int CL_THREADS = 128;
-constexpr size_t CL_SMEM = 32768 + 16384 + 8192 + 2 * CH * LC * 4 + 1024;
+constexpr size_t CL_SMEM = 32768 + 16384 + 8192 + CH * LC * 4 + 1024;
 
 __global__ void __launch_bounds__(CL_THREADS)
 tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
@@ -205,8 +255,10 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     uint8_t* sKQ = sm;                 // per k-half h: [K rows 0-63 | Q rows 64-127], 16 KB each
     uint8_t* sKt = sKQ + 32768;        // per k-half: 8 KB
     uint8_t* sTb = sKt + 16384;        // T diag(beta gamma), K-major [i][j]
-    float* sA = reinterpret_cast<float*>(sTb + 8192);
-    float* sT = sA + CH * LC;
+    // A (fp32) takes over the space of Ktil once the first product has consumed it (and the first
+    // 256 bytes of the Tbg image, which is written only after the inversion)
+    float* sA = reinterpret_cast<float*>(sKt);
+    float* sT = reinterpret_cast<float*>(sTb + 8192);
     __shared__ uint64_t bar_tma, bar_mma1, bar_mma2;
     __shared__ uint32_t tmem_base;
     __shared__ float sG[CH], sBeta[CH], sg[CH];
