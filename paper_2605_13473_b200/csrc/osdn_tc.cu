@@ -1031,7 +1031,7 @@ struct TcChunkBwdArgs {
     int* status;
 };
 
-constexpr int CBW_THREADS = 256;
+constexpr int CBW_THREADS = 512;   // 16 warps = 4 lane quadrants x 4 column groups
 constexpr uint32_t R_Q = 0, R_K = 16384, R_KT = 32768, R_V = 49152, R_DO = 65536, R_DU = 81920, R_DDU = 98304,
                    R_T = 114688, R_S = 122880, R_DS = 155648, R_RAW = 188416;
 constexpr uint32_t R_DWT = R_DO;                 // dW^T image replaces dO after phase A
@@ -1060,7 +1060,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int tok0 = a.tab.chunk_tok0[c];
     const size_t tile = (size_t)c * H + h;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int quad = warp & 3, colhalf = warp >> 2;
+    const int quad = warp & 3, colq = warp >> 2;   // lane quadrant, column group (16 columns each)
     const int f = quad * 32 + lane;                 // feature (k or v) owned in 128-lane accumulators
     const int row64 = quad * 16 + (lane & 15);      // token row owned in 64-row accumulators (lanes 0-15)
     const bool row_active = lane < 16;
@@ -1192,9 +1192,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // rawkk, dP' (64-row accumulators: rows in lanes 0-15 of each quadrant)
         const int i = row64;
         const float Gi = sG[i];
-        for (int cb = 0; cb < 2; ++cb) {
+        {
             uint32_t r1[16], r2[16];
-            const int j0 = colhalf * 32 + cb * 16;
+            const int j0 = colq * 16;
             tmem_ld16(tb + cRAW + lane_addr + j0, r1);
             tmem_ld16(tb + cDP + lane_addr + j0, r2);
             tmem_ld_wait();
@@ -1215,13 +1215,13 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
         }
         // dW^T -> bf16 image [rows k][cols i]
-        for (int cb = 0; cb < 2; ++cb) {
+        {
             uint32_t r[16];
-            tmem_ld16(tb + cDW + lane_addr + colhalf * 32 + cb * 16, r);
+            tmem_ld16(tb + cDW + lane_addr + colq * 16, r);
             tmem_ld_wait();
 #pragma unroll
             for (int c2 = 0; c2 < 2; ++c2)
-                *reinterpret_cast<uint4*>(sm + R_DWT + sw128_chunk(f, colhalf * 4 + cb * 2 + c2)) = make_uint4(
+                *reinterpret_cast<uint4*>(sm + R_DWT + sw128_chunk(f, colq * 2 + c2)) = make_uint4(
                     pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1])),
                     pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3])),
                     pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5])),
@@ -1277,9 +1277,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_after();
     {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j]
         const int i = row64;
-        for (int cb = 0; cb < 2; ++cb) {
+        {
             uint32_t r1[16], r2[16];
-            const int j0 = colhalf * 32 + cb * 16;
+            const int j0 = colq * 16;
             tmem_ld16(tb + cDTA + lane_addr + j0, r1);
             tmem_ld16(tb + cDTB + lane_addr + j0, r2);
             tmem_ld_wait();
@@ -1317,9 +1317,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_after();
     {
         const int i = row64;
-        for (int cb = 0; cb < 2; ++cb) {
+        {
             uint32_t r[16];
-            const int j0 = colhalf * 32 + cb * 16;
+            const int j0 = colq * 16;
             tmem_ld16(tb + cY + lane_addr + j0, r);
             tmem_ld_wait();
             if (row_active) {
@@ -1353,9 +1353,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int i = row64;
         const float bi = sBeta[i], Gi = sG[i];
         float db = 0.f;
-        for (int cb = 0; cb < 2; ++cb) {
+        {
             uint32_t r[16];
-            const int j0 = colhalf * 32 + cb * 16;
+            const int j0 = colq * 16;
             tmem_ld16(tb + cZ + lane_addr + j0, r);
             tmem_ld_wait();
             if (row_active) {
@@ -1403,7 +1403,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
         const uint32_t fc = f & 63;
         float rsum = 0.f;
-        float gv[32], bv[32];   // per column: gate and beta contributions of this feature
+        float gv[16], bv[16];   // per column: gate and beta contributions of this feature
         // Results are staged in shared memory as [token][feature] tiles (the operand tiles of the
         // finished products are dead by now) and written out with 16-byte stores afterwards.
         __nv_bfloat16* stq = reinterpret_cast<__nv_bfloat16*>(sm + ST_DQ);
@@ -1412,8 +1412,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         float* stkr = reinterpret_cast<float*>(sm + ST_DKR);
         float* stkt = reinterpret_cast<float*>(sm + ST_DKT);
 #pragma unroll
-        for (int cb = 0; cb < 4; ++cb) {
-            const int j0 = colhalf * 32 + cb * 8;
+        for (int cb = 0; cb < 2; ++cb) {
+            const int j0 = colq * 16 + cb * 8;
             uint32_t rq1[8], rq2[8], rkt[8], rdk[8], rkb[8], rkr[8], rvb[8];
             tmem_ld8(tb + cDQ1 + lane_addr + j0, rq1);
             tmem_ld8(tb + cDQ2 + lane_addr + j0, rq2);
@@ -1455,12 +1455,12 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 stkt[j * KD + f] = dkt;
             }
         }
-        // Sum over the 32 features of the warp for all 32 columns at once: in each of five steps a
-        // lane keeps one half of its columns and hands the other half to its partner (31 shuffles per
-        // quantity); afterwards lane l holds the warp total of column l.
+        // Sum over the 32 features of the warp for all 16 columns at once: in each of four steps a
+        // lane keeps one half of its columns and hands the other half to its partner; a last exchange
+        // joins the two lanes that end up with the same column (16 shuffles per quantity).
 #pragma unroll
-        for (int step = 0; step < 5; ++step) {
-            const int off = 16 >> step, n = 16 >> step;   // n = columns kept after this step
+        for (int step = 0; step < 4; ++step) {
+            const int off = 16 >> step, n = 8 >> step;   // n = columns kept after this step
             const bool upper = (lane & off) != 0;
 #pragma unroll
             for (int i = 0; i < n; ++i) {
@@ -1470,8 +1470,12 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 bv[i] = bk + __shfl_xor_sync(0xffffffffu, bs, off);
             }
         }
-        atomicAdd(&sdG[colhalf * 32 + lane], gv[0]);
-        atomicAdd(&sdB[colhalf * 32 + lane], bv[0]);
+        gv[0] += __shfl_xor_sync(0xffffffffu, gv[0], 1);
+        bv[0] += __shfl_xor_sync(0xffffffffu, bv[0], 1);
+        if ((lane & 1) == 0) {
+            atomicAdd(&sdG[colq * 16 + (lane >> 1)], gv[0]);
+            atomicAdd(&sdB[colq * 16 + (lane >> 1)], bv[0]);
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
         if (lane == 0) atomicAdd(&sRsum, rsum);
