@@ -612,7 +612,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         // ---- E0: S -> bf16 operand (+ saved copy), decay the accumulator -----------------------
         {
             const float gC = sGC[gs];
-            uint8_t* Sg = a.Sn + tile * 32768 + (colq >> 1) * 16384;
             uint32_t rr[2][16];
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
@@ -629,7 +628,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                     w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
                     const uint32_t off = sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2);
                     *reinterpret_cast<uint4*>(sS + (colq >> 1) * 16384 + off) = w;
-                    if (a.save) *reinterpret_cast<uint4*>(Sg + off) = w;
                 }
 #pragma unroll
                 for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
@@ -655,6 +653,10 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         // ---- MMA group 1 -----------------------------------------------------------------------
         if (tid == 0 && ok) {
             tc_fence_after();
+            if (a.save) {   // the state of this chunk, as the bf16 image just written
+                bulk_store(a.Sn + tile * 32768, sS, 32768);
+                bulk_commit();
+            }
             {   // dU^T = V^T Tb^T
                 const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
                 const uint64_t da0 = desc_mnmajor(d + ST_V, BOX), db0 = desc_kmajor(d + ST_TB);
@@ -682,7 +684,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 
         // ---- E1: dU^T -> bf16 operands ---------------------------------------------------------
         {
-            uint8_t* dUg = a.dUT + tile * 16384;
             uint32_t r[16];
             tmem_ld16(tDU + lane_addr + colq * 16, r);
             tmem_ld_wait();
@@ -701,7 +702,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                     *reinterpret_cast<uint4*>(sDU1 + off) = w1;
                     *reinterpret_cast<uint4*>(sDU2 + off) = make_uint4(pack_bf16(g[0], g[1]), pack_bf16(g[2], g[3]),
                                                                       pack_bf16(g[4], g[5]), pack_bf16(g[6], g[7]));
-                    if (a.save) *reinterpret_cast<uint4*>(dUg + off) = w1;
                 }
             }
         }
@@ -713,6 +713,10 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         // ---- MMA group 2 -----------------------------------------------------------------------
         if (tid == 0 && ok) {
             tc_fence_after();
+            if (a.save) {
+                bulk_store(a.dUT + tile * 16384, sDU1, 16384);
+                bulk_commit();
+            }
             {   // S += (rho dU)^T Ktil   (on the critical path: first)
                 const uint32_t idesc = make_idesc(128, 128, IDESC_B_MN);
                 const uint64_t da0 = desc_kmajor(sDU2), db0 = desc_mnmajor(d + ST_KT, BOX);
@@ -736,6 +740,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
         tc_fence_after();
     OSDN_CLK(1, 6, blockIdx.x == 0 && n == 3);
+        if (tid == 0) bulk_wait_read();   // the saved images have left shared memory before it is rewritten
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
@@ -759,6 +764,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             for (int x = 0; x < 16; ++x) fin[cb * 16 + x] = __uint_as_float(r[x]);
         }
     }
+    if (tid == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tb, 512);
@@ -878,7 +884,6 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         // ---- E0: dS (cotangent at the chunk end) -> bf16 operand + saved copy; decay -----------
         {
             const float gC = sGC[st];
-            uint8_t* Sg = a.dSn + tile * 32768 + colhalf * 16384;
             uint32_t rr[4][16];
 #pragma unroll
             for (int cb = 0; cb < 4; ++cb) tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, rr[cb]);
@@ -895,7 +900,6 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
                     w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
                     const uint32_t off = sw128_chunk(v, cb * 2 + c2);
                     *reinterpret_cast<uint4*>(sdS + colhalf * 16384 + off) = w;
-                    *reinterpret_cast<uint4*>(Sg + off) = w;
                 }
 #pragma unroll
                 for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
@@ -919,6 +923,8 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
 
         if (tid == 0 && ok) {
             tc_fence_after();
+            bulk_store(a.dSn + tile * 32768, sdS, 32768);   // cotangent at the end of this chunk
+            bulk_commit();
             {   // acc1 = dO^T P'
                 const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN);
                 const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_P, 0);
@@ -939,7 +945,6 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
 
         // ---- E1: ddU^T = acc1 + rho_i acc2 ---------------------------------------------------
         {
-            uint8_t* dg = a.ddUT + tile * 16384;
             uint32_t ra[2][16], rb[2][16];
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
@@ -961,7 +966,6 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
                     const uint4 w = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
                                                pack_bf16(f[6], f[7]));
                     *reinterpret_cast<uint4*>(sddU + off) = w;
-                    *reinterpret_cast<uint4*>(dg + off) = w;
                 }
             }
         }
@@ -972,6 +976,8 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
 
         if (tid == 0 && ok) {
             tc_fence_after();
+            bulk_store(a.ddUT + tile * 16384, sddU, 16384);
+            bulk_commit();
             {   // dS += dO^T Qg
                 const uint32_t idesc = make_idesc(128, 128, IDESC_A_MN | IDESC_B_MN);
                 const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_QG, BOX);
@@ -990,6 +996,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
     OSDN_CLK(2, 6, blockIdx.x == 0 && n == 3);
         tc_fence_after();
+        if (tid == 0) bulk_wait_read();
         tc_fence_before();
         __syncthreads();
     OSDN_CLK(2, 7, blockIdx.x == 0 && n == 3);
@@ -1004,6 +1011,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
             for (int x = 0; x < 16; ++x) dini[cb * 16 + x] = __uint_as_float(r[x]);
         }
     }
+    if (tid == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tb, 256);
