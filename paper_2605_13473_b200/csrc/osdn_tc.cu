@@ -107,6 +107,20 @@ bool make_token_map(CUtensorMap* m, const void* base, size_t rows, int H)
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Map over the same kind of tensor for storing dense [64 tokens x 128 features] tiles (no swizzle).
+bool make_store_map(CUtensorMap* m, void* base, size_t rows, int H)
+{
+    PFN_cuTensorMapEncodeTiled enc = get_encoder();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)H * KD, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)H * KD * 2};
+    cuuint32_t box[2] = {KD, 64};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
 __device__ __forceinline__ uint8_t* align1024(uint8_t* p)
 {
     return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
@@ -1052,7 +1066,9 @@ constexpr size_t CBW_SMEM = R_RAW + CH * LC * 4 + 1024;
 __global__ void __launch_bounds__(CBW_THREADS, 1)
 tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmV,
-                    const __grid_constant__ CUtensorMap tmDO, TcChunkBwdArgs a)
+                    const __grid_constant__ CUtensorMap tmDO, const __grid_constant__ CUtensorMap tmDQ,
+                    const __grid_constant__ CUtensorMap tmDK, const __grid_constant__ CUtensorMap tmDV,
+                    TcChunkBwdArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* sm = align1024(smem_raw);
@@ -1488,28 +1504,61 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
         if (lane == 0) atomicAdd(&sRsum, rsum);
     }
-    __syncthreads();
+    ok = __syncthreads_and(ok);   // block-uniform from here on (the copy-out contains a barrier)
     if (ok) {
-        // copy-out: 16-byte stores, one 256-byte (bf16) or 512-byte (fp32) token row after another
         const unsigned long long sk =
             (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
-        for (int e = tid; e < len * 16; e += CBW_THREADS) {
-            const int j = e >> 4, ch = e & 15;
-            const size_t g = ((size_t)(tok0 + j) * H + h) * KD + ch * 8;
-            *reinterpret_cast<uint4*>(a.dq + g) = *reinterpret_cast<const uint4*>(sm + ST_DQ + j * 256 + ch * 16);
-            *reinterpret_cast<uint4*>(a.dv + g) = *reinterpret_cast<const uint4*>(sm + ST_DV + j * 256 + ch * 16);
-            if ((sk >> j) & 1ull)
-                *reinterpret_cast<uint4*>(a.dk + g) = *reinterpret_cast<const uint4*>(sm + ST_DK + j * 256 + ch * 16);
+        // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's
+        // preconditioner step was skipped); ragged or mixed chunks are copied row by row.
+        const bool full = len == CH;
+        const bool dk_tile = full && sk == ~0ull;
+        if (full) {
+            fence_proxy_async();
         }
-        for (int e = tid; e < len * 32; e += CBW_THREADS) {
-            const int j = e >> 5, ch = e & 31;
-            const size_t g = ((size_t)(tok0 + j) * H + h) * KD + ch * 4;
-            const bool skipped = (sk >> j) & 1ull;
-            if (!skipped)
-                *reinterpret_cast<uint4*>(a.dkread + g) = *reinterpret_cast<const uint4*>(sm + ST_DKR + j * 512 + ch * 16);
-            if (!skipped || j == 0 || !((sk >> (j - 1)) & 1ull))
-                *reinterpret_cast<uint4*>(a.dktil + g) = *reinterpret_cast<const uint4*>(sm + ST_DKT + j * 512 + ch * 16);
+        __syncthreads();
+        if (full && tid == 0) {
+            tma_store_2d(&tmDQ, h * KD, tok0, sm + ST_DQ);
+            tma_store_2d(&tmDV, h * KD, tok0, sm + ST_DV);
+            if (dk_tile) tma_store_2d(&tmDK, h * KD, tok0, sm + ST_DK);
+            bulk_commit();
         }
+        if (!full) {
+            for (int e = tid; e < len * 16; e += CBW_THREADS) {
+                const int j = e >> 4, ch = e & 15;
+                const size_t g = ((size_t)(tok0 + j) * H + h) * KD + ch * 8;
+                *reinterpret_cast<uint4*>(a.dq + g) = *reinterpret_cast<const uint4*>(sm + ST_DQ + j * 256 + ch * 16);
+                *reinterpret_cast<uint4*>(a.dv + g) = *reinterpret_cast<const uint4*>(sm + ST_DV + j * 256 + ch * 16);
+            }
+        }
+        if (!dk_tile) {
+            for (int e = tid; e < len * 16; e += CBW_THREADS) {
+                const int j = e >> 4, ch = e & 15;
+                const size_t g = ((size_t)(tok0 + j) * H + h) * KD + ch * 8;
+                if ((sk >> j) & 1ull)
+                    *reinterpret_cast<uint4*>(a.dk + g) =
+                        *reinterpret_cast<const uint4*>(sm + ST_DK + j * 256 + ch * 16);
+            }
+        }
+        if (dk_tile) {
+            // only the first token's dL/dktil is needed (a reverse recurrence may restart there)
+            for (int e = tid; e < 32; e += CBW_THREADS) {
+                const size_t g = ((size_t)tok0 * H + h) * KD + e * 4;
+                *reinterpret_cast<uint4*>(a.dktil + g) = *reinterpret_cast<const uint4*>(sm + ST_DKT + e * 16);
+            }
+        } else {
+            for (int e = tid; e < len * 32; e += CBW_THREADS) {
+                const int j = e >> 5, ch = e & 31;
+                const size_t g = ((size_t)(tok0 + j) * H + h) * KD + ch * 4;
+                const bool skipped = (sk >> j) & 1ull;
+                if (!skipped)
+                    *reinterpret_cast<uint4*>(a.dkread + g) =
+                        *reinterpret_cast<const uint4*>(sm + ST_DKR + j * 512 + ch * 16);
+                if (!skipped || j == 0 || !((sk >> (j - 1)) & 1ull))
+                    *reinterpret_cast<uint4*>(a.dktil + g) =
+                        *reinterpret_cast<const uint4*>(sm + ST_DKT + j * 512 + ch * 16);
+            }
+        }
+        if (full && tid == 0) bulk_wait_all();
     }
     OSDN_CLK(3, 12, blockIdx.x == 5 && blockIdx.y == 0);
     if (tid == 0) {
@@ -1632,9 +1681,14 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
         cb.dv = static_cast<__nv_bfloat16*>(a.dv); cb.dbeta = a.dbeta; cb.dgate = a.dgate;
         cb.dktil = reinterpret_cast<float*>(w + t.dktil); cb.dkread = reinterpret_cast<float*>(w + t.dkread);
         cb.status = status;
+        CUtensorMap tmDQ, tmDK, tmDV;
+        if (!make_store_map(&tmDQ, a.dq, Ttot, H) || !make_store_map(&tmDK, a.dk, Ttot, H) ||
+            !make_store_map(&tmDV, a.dv, Ttot, H))
+            return -1;
         if (!set_smem(tc_chunk_bwd_kernel, CBW_SMEM)) return -1;
         stage_mark(st, "tc_chunk_bwd");
-        tc_chunk_bwd_kernel<<<dim3(L.NTmax, H), CBW_THREADS, CBW_SMEM, st>>>(tmQ, tmK, tmKt, tmV, tmDO, cb);
+        tc_chunk_bwd_kernel<<<dim3(L.NTmax, H), CBW_THREADS, CBW_SMEM, st>>>(tmQ, tmK, tmKt, tmV, tmDO, tmDQ, tmDK,
+                                                                                tmDV, cb);
         ++launches;
     }
     const int n1 = phase1_backward(p, hy, L, ws, a, reinterpret_cast<float*>(w + t.dktil),
