@@ -16,6 +16,8 @@
 // Work tiles that travel between kernels are stored in HBM as ready-made images of the
 // 128-byte-swizzled shared-memory layout (see umma.cuh), so that the consumer fetches them with a
 // plain bulk copy; user tensors (q, k, ktil, v, dout) are fetched with TMA tensor maps.
+#include <algorithm>
+
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
@@ -1042,7 +1044,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
 //             dv = beta dVb ; dbeta, dgate from the products of the gradients with their inputs
 // ---------------------------------------------------------------------------------------------
 struct TcChunkBwdArgs {
-    int H;
+    int H, ntiles;
     Table tab;
     const float *beta, *gate;
     float scale, d_min;
@@ -1078,11 +1080,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __shared__ float sG[CH], sBeta[CH], sg[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
     __shared__ float sRsum;
 
-    const int c = blockIdx.x, h = blockIdx.y, H = a.H;
-    const int len = a.tab.chunk_len[c];
-    if (len == 0) return;
-    const int tok0 = a.tab.chunk_tok0[c];
-    const size_t tile = (size_t)c * H + h;
+    const int H = a.H;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, colq = warp >> 2;   // lane quadrant, column group (16 columns each)
     const int f = quad * 32 + lane;                 // feature (k or v) owned in 128-lane accumulators
@@ -1095,6 +1093,22 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(&tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+
+    // persistent: one CTA per SM walks over the (chunk, head) tiles
+    uint32_t ph = 0;   // barrier phase parity: number of tiles processed so far, mod 2
+    for (long tile_l = blockIdx.x; tile_l < a.ntiles; tile_l += gridDim.x) {
+    const size_t tile = (size_t)tile_l;
+    const int c = (int)(tile_l / H), h = (int)(tile_l % H);
+    const bool clk = tile_l == 1603;
+    (void)clk;
+    const int len = a.tab.chunk_len[c];
+    if (len == 0) continue;
+    const int tok0 = a.tab.chunk_tok0[c];
     if (tid < CH) {
         const bool in = tid < len;
         sg[tid] = in ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
@@ -1103,12 +1117,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sdG[tid] = 0.f;
     }
     if (tid == 0) sRsum = 0.f;
-    tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 0, blockIdx.x == 5 && blockIdx.y == 0);
-    tc_fence_after();
-    const uint32_t tb = tmem_base;
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    OSDN_CLK(3, 0, clk);
 
     if (tid == 0) {
         mbar_expect_tx(&bar_tma, 10 * BOX + 16384 + 16384 + 8192 + 32768 + 32768);
@@ -1135,8 +1145,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sGam[tid] = __expf(acc);
         sRho[tid] = __expf(tot - acc);
     }
-    bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
-    OSDN_CLK(3, 1, blockIdx.x == 5 && blockIdx.y == 0);
+    bool ok = mbar_wait(&bar_tma, ph, a.status, ERR_TMA);
+    OSDN_CLK(3, 1, clk);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sm + R_Q + hf * BOX, len, tid, CBW_THREADS);
@@ -1148,7 +1158,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fence_proxy_async();
     }
     __syncthreads();
-    OSDN_CLK(3, 2, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLK(3, 2, clk);
 
     // tensor memory columns
     const uint32_t cRAW = 0, cDP = 64, cDQ1 = 128, cDKTR = 192, cDW = 256, cDTA = 320, cDTB = 384, cDKT = 448;
@@ -1207,8 +1217,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
         if (lane == 0) sRed[warp] = part;
     }
-    ok = ok && mbar_wait(&bar_mma[0], 0, a.status, ERR_MMA1);
-    OSDN_CLK(3, 3, blockIdx.x == 5 && blockIdx.y == 0);
+    ok = ok && mbar_wait(&bar_mma[0], ph, a.status, ERR_MMA1);
+    OSDN_CLK(3, 3, clk);
     tc_fence_after();
     __syncthreads();   // every thread is done reading S / dS before their space is reused
     // epilogue A
@@ -1255,7 +1265,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 4, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLK(3, 4, clk);
 
     // ---- phase B -------------------------------------------------------------------------------
     if (tid == 0 && ok) {
@@ -1296,8 +1306,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         mma_commit(&bar_mma[1]);
     }
-    ok = ok && mbar_wait(&bar_mma[1], 0, a.status, ERR_MMA2);
-    OSDN_CLK(3, 5, blockIdx.x == 5 && blockIdx.y == 0);
+    ok = ok && mbar_wait(&bar_mma[1], ph, a.status, ERR_MMA2);
+    OSDN_CLK(3, 5, clk);
     tc_fence_after();
     {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j]
         const int i = row64;
@@ -1325,7 +1335,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 6, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLK(3, 6, clk);
 
     // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] -----------------------------------------------
     if (tid == 0 && ok) {
@@ -1336,8 +1346,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                    make_idesc(64, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
         mma_commit(&bar_mma[2]);
     }
-    ok = ok && mbar_wait(&bar_mma[2], 0, a.status, ERR_MMA2);
-    OSDN_CLK(3, 7, blockIdx.x == 5 && blockIdx.y == 0);
+    ok = ok && mbar_wait(&bar_mma[2], ph, a.status, ERR_MMA2);
+    OSDN_CLK(3, 7, clk);
     tc_fence_after();
     {
         const int i = row64;
@@ -1360,7 +1370,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 8, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLK(3, 8, clk);
 
     // ---- phase D: Z[a][b] = sum_c Y[a][c] T[b][c] ; dA = -strictLower(Z) --------------------------
     if (tid == 0 && ok) {
@@ -1370,8 +1380,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mma_ss(tb + cZ, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), make_idesc(64, 64), k > 0);
         mma_commit(&bar_mma[3]);
     }
-    ok = ok && mbar_wait(&bar_mma[3], 0, a.status, ERR_MMA2);
-    OSDN_CLK(3, 9, blockIdx.x == 5 && blockIdx.y == 0);
+    ok = ok && mbar_wait(&bar_mma[3], ph, a.status, ERR_MMA2);
+    OSDN_CLK(3, 9, clk);
     tc_fence_after();
     {
         const int i = row64;
@@ -1403,7 +1413,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 10, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLK(3, 10, clk);
 
     // ---- phase E: dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T -----------------------------------------
     if (tid == 0 && ok) {
@@ -1418,8 +1428,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                    make_idesc(128, 64, IDESC_A_MN), k > 0);
         mma_commit(&bar_mma[4]);
     }
-    ok = ok && mbar_wait(&bar_mma[4], 0, a.status, ERR_MMA2);
-    OSDN_CLK(3, 11, blockIdx.x == 5 && blockIdx.y == 0);
+    ok = ok && mbar_wait(&bar_mma[4], ph, a.status, ERR_MMA2);
+    OSDN_CLK(3, 11, clk);
     tc_fence_after();
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
@@ -1558,9 +1568,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         *reinterpret_cast<const uint4*>(sm + ST_DKT + j * 512 + ch * 16);
             }
         }
-        if (full && tid == 0) bulk_wait_all();
+        if (full && tid == 0) bulk_wait_read();   // the staging tiles may be overwritten by the next tile
     }
-    OSDN_CLK(3, 12, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLK(3, 12, clk);
     if (tid == 0) {
         float tot = 0.f;
         for (int w = 0; w < CBW_THREADS / 32; ++w) tot += sRed[w];
@@ -1578,8 +1588,25 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 13, blockIdx.x == 5 && blockIdx.y == 0);
+    tc_fence_after();
+    OSDN_CLK(3, 13, clk);
+    ph ^= 1u;
+    }   // tile loop
+    if (tid == 0) bulk_wait_all();
+    tc_fence_before();
+    __syncthreads();
     if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+int num_sms()
+{
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
 }
 
 template <typename F> bool set_smem(F* kernel, size_t bytes)
@@ -1674,7 +1701,7 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
     }
     {
         TcChunkBwdArgs cb{};
-        cb.H = H; cb.tab = tab; cb.beta = a.beta; cb.gate = a.gate; cb.scale = hy.scale; cb.d_min = hy.d_min;
+        cb.H = H; cb.ntiles = L.NTmax * H; cb.tab = tab; cb.beta = a.beta; cb.gate = a.gate; cb.scale = hy.scale; cb.d_min = hy.d_min;
         cb.Tm = U8(t.Tm); cb.Sn = U8(t.Sn); cb.dSn = U8(t.dSn); cb.dUT = U8(t.dUT); cb.ddUT = U8(t.ddUT);
         cb.skipw = carve_p1(ws, L).skipw;
         cb.dq = static_cast<__nv_bfloat16*>(a.dq); cb.dk = static_cast<__nv_bfloat16*>(a.dk);
@@ -1687,7 +1714,7 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
             return -1;
         if (!set_smem(tc_chunk_bwd_kernel, CBW_SMEM)) return -1;
         stage_mark(st, "tc_chunk_bwd");
-        tc_chunk_bwd_kernel<<<dim3(L.NTmax, H), CBW_THREADS, CBW_SMEM, st>>>(tmQ, tmK, tmKt, tmV, tmDO, tmDQ, tmDK,
+        tc_chunk_bwd_kernel<<<std::min(cb.ntiles, num_sms()), CBW_THREADS, CBW_SMEM, st>>>(tmQ, tmK, tmKt, tmV, tmDO, tmDQ, tmDK,
                                                                                 tmDV, cb);
         ++launches;
     }
