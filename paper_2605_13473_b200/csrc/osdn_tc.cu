@@ -1099,42 +1099,75 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t tb = tmem_base;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
 
-    // persistent: one CTA per SM walks over the (chunk, head) tiles
+    // persistent: one CTA per SM walks over the (chunk, head) tiles.  The operands of the next tile
+    // are requested in two batches as soon as the shared-memory regions they land in are dead, and
+    // its per-token scalars are fetched into registers one tile ahead.
+    auto next_tile = [&](long t) {   // first non-empty tile of this CTA at or after t
+        while (t < a.ntiles && a.tab.chunk_len[(int)(t / H)] == 0) t += gridDim.x;
+        return t;
+    };
+    auto issue_first = [&](long t, int t0) {   // q, k, ktil, v
+        const int hh = (int)(t % H);
+        mbar_expect_tx(&bar_tma, 10 * BOX + 16384 + 16384 + 8192 + 32768 + 32768);
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_load_2d(sm + R_Q + hf * BOX, &tmQ, hh * KD + hf * 64, t0, &bar_tma);
+            tma_load_2d(sm + R_K + hf * BOX, &tmK, hh * KD + hf * 64, t0, &bar_tma);
+            tma_load_2d(sm + R_KT + hf * BOX, &tmKt, hh * KD + hf * 64, t0, &bar_tma);
+            tma_load_2d(sm + R_V + hf * BOX, &tmV, hh * KD + hf * 64, t0, &bar_tma);
+        }
+    };
+    auto issue_second = [&](long t, int t0) {   // dout and the chain tiles
+        const int hh = (int)(t % H);
+        for (int hf = 0; hf < 2; ++hf) tma_load_2d(sm + R_DO + hf * BOX, &tmDO, hh * KD + hf * 64, t0, &bar_tma);
+        bulk_load(sm + R_DU, a.dUT + (size_t)t * 16384, 16384, &bar_tma);
+        bulk_load(sm + R_DDU, a.ddUT + (size_t)t * 16384, 16384, &bar_tma);
+        bulk_load(sm + R_T, a.Tm + (size_t)t * 8192, 8192, &bar_tma);
+        bulk_load(sm + R_S, a.Sn + (size_t)t * 32768, 32768, &bar_tma);
+        bulk_load(sm + R_DS, a.dSn + (size_t)t * 32768, 32768, &bar_tma);
+    };
+    auto fetch_scalars = [&](long t, int t0, int ln, float& g, float& b) {
+        const int hh = (int)(t % H);
+        const bool in = tid < ln;
+        g = (tid < CH && in) ? a.gate[(size_t)(t0 + tid) * H + hh] : 0.f;
+        b = (tid < CH && in) ? a.beta[(size_t)(t0 + tid) * H + hh] : 0.f;
+    };
     uint32_t ph = 0;   // barrier phase parity: number of tiles processed so far, mod 2
-    for (long tile_l = blockIdx.x; tile_l < a.ntiles; tile_l += gridDim.x) {
+    long tile_l = next_tile(blockIdx.x);
+    int tok0 = 0, len = 0;
+    float g_cur = 0.f, b_cur = 0.f;
+    if (tile_l < a.ntiles) {
+        tok0 = a.tab.chunk_tok0[(int)(tile_l / H)];
+        len = a.tab.chunk_len[(int)(tile_l / H)];
+        if (tid == 0) {
+            issue_first(tile_l, tok0);
+            issue_second(tile_l, tok0);
+        }
+        fetch_scalars(tile_l, tok0, len, g_cur, b_cur);
+    }
+    while (tile_l < a.ntiles) {
     const size_t tile = (size_t)tile_l;
-    const int c = (int)(tile_l / H), h = (int)(tile_l % H);
+    const int h = (int)(tile_l % H);
     const bool clk = tile_l == 1603;
     (void)clk;
-    const int len = a.tab.chunk_len[c];
-    if (len == 0) continue;
-    const int tok0 = a.tab.chunk_tok0[c];
     if (tid < CH) {
-        const bool in = tid < len;
-        sg[tid] = in ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
-        sBeta[tid] = in ? a.beta[(size_t)(tok0 + tid) * H + h] : 0.f;
+        sg[tid] = g_cur;
+        sBeta[tid] = b_cur;
         sdB[tid] = 0.f;
         sdG[tid] = 0.f;
     }
     if (tid == 0) sRsum = 0.f;
     __syncthreads();
     OSDN_CLK(3, 0, clk);
-
-    if (tid == 0) {
-        mbar_expect_tx(&bar_tma, 10 * BOX + 16384 + 16384 + 8192 + 32768 + 32768);
-        for (int hf = 0; hf < 2; ++hf) {
-            tma_load_2d(sm + R_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_tma);
-            tma_load_2d(sm + R_K + hf * BOX, &tmK, h * KD + hf * 64, tok0, &bar_tma);
-            tma_load_2d(sm + R_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_tma);
-            tma_load_2d(sm + R_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_tma);
-            tma_load_2d(sm + R_DO + hf * BOX, &tmDO, h * KD + hf * 64, tok0, &bar_tma);
-        }
-        bulk_load(sm + R_DU, a.dUT + tile * 16384, 16384, &bar_tma);
-        bulk_load(sm + R_DDU, a.ddUT + tile * 16384, 16384, &bar_tma);
-        bulk_load(sm + R_T, a.Tm + tile * 8192, 8192, &bar_tma);
-        bulk_load(sm + R_S, a.Sn + tile * 32768, 32768, &bar_tma);
-        bulk_load(sm + R_DS, a.dSn + tile * 32768, 32768, &bar_tma);
+    // table entries and scalars of the next tile, one tile ahead
+    const long tile_next = next_tile(tile_l + gridDim.x);
+    int tok0_next = 0, len_next = 0;
+    float g_next = 0.f, b_next = 0.f;
+    if (tile_next < a.ntiles) {
+        tok0_next = a.tab.chunk_tok0[(int)(tile_next / H)];
+        len_next = a.tab.chunk_len[(int)(tile_next / H)];
+        fetch_scalars(tile_next, tok0_next, len_next, g_next, b_next);
     }
+
     if (tid < CH) {
         float acc = 0.f, tot = 0.f;
         for (int j = 0; j < CH; ++j) {
@@ -1515,6 +1548,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (lane == 0) atomicAdd(&sRsum, rsum);
     }
     ok = __syncthreads_and(ok);   // block-uniform from here on (the copy-out contains a barrier)
+    if (tid == 0 && tile_next < a.ntiles) issue_first(tile_next, tok0_next);   // q, k, ktil, v are dead
     if (ok) {
         const unsigned long long sk =
             (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
@@ -1570,6 +1604,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         if (full && tid == 0) bulk_wait_read();   // the staging tiles may be overwritten by the next tile
     }
+    __syncthreads();   // every copy-out read of the staging tiles is done
+    if (tid == 0 && tile_next < a.ntiles) issue_second(tile_next, tok0_next);
     OSDN_CLK(3, 12, clk);
     if (tid == 0) {
         float tot = 0.f;
@@ -1591,6 +1627,11 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_after();
     OSDN_CLK(3, 13, clk);
     ph ^= 1u;
+    tile_l = tile_next;
+    tok0 = tok0_next;
+    len = len_next;
+    g_cur = g_next;
+    b_cur = b_next;
     }   // tile loop
     if (tid == 0) bulk_wait_all();
     tc_fence_before();
