@@ -513,7 +513,21 @@ __device__ __forceinline__ void warp_gate_vectors(float ga, float gb, int lane, 
     if (lane == 0) *gC = __expf(tot);
 }
 
-__global__ void __launch_bounds__(CF2_THREADS, 1)
+// Warp roles of the forward chain: 16 epilogue warps (4 lane quadrants x 4 column groups), one warp
+// that issues the tensor-core work, one warp that issues the loads and prepares the gate vectors.
+// The roles run decoupled and meet only at mbarriers:
+//   full[st]   loads of a chunk have landed (and its gate vectors are written)      producer -> all
+//   empty[st]  every product reading the stage has finished                         tensor core -> producer
+//   s_ready    S is in shared memory as a bf16 operand, the accumulator is decayed  epilogue -> issuer
+//   du_done    dU^T accumulator complete                                            tensor core -> epilogue
+//   du_ready   dU^T operands are in shared memory                                   epilogue -> issuer
+//   s_done     the state update of the chunk is complete                            tensor core -> epilogue
+//   o_done     both output accumulators of the chunk are complete                   tensor core -> epilogue
+constexpr int CFW_EPI_WARPS = 16;
+constexpr int CFW_MMA_WARP = 16, CFW_TMA_WARP = 17;
+constexpr int CFW_THREADS = 18 * 32;
+
+__global__ void __launch_bounds__(CFW_THREADS, 1)
 tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
                     const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
 {
@@ -523,21 +537,21 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     uint8_t* sS = sm + 2 * STAGE_BYTES;         // S as bf16, K-major: 2 k-halves x [128 rows x 128 B]
     uint8_t* sDU1 = sS + 32768;                 // dU^T, K-major [v][i]
     uint8_t* sDU2 = sDU1 + 16384;               // (rho dU)^T
-    __shared__ uint64_t bar_full[2], bar_mma1, bar_mma2;
+    __shared__ uint64_t bar_full[2], bar_empty[2], bar_s_ready, bar_du_done, bar_du_ready, bar_s_done, bar_o_done;
     __shared__ uint32_t tmem_base;
-    __shared__ float sGam[3][CH], sRho[3][CH], sGC[3];   // slot = chunk % 3
+    __shared__ float sGam[2][CH], sRho[2][CH], sGC[2];   // slot = chunk % 2 (read only before du_ready)
 
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
     const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
     const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int quad = warp & 3, colq = warp >> 2;   // lane quadrant, column group (4 groups)
-    const int v = quad * 32 + lane;             // state row owned by this thread
+    const int quad = warp & 3, colq = (warp >> 2) & 3;
+    const int v = quad * 32 + lane;             // state row owned by an epilogue thread
     float* fin = a.final_state ? a.final_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
     const float* ini = a.init_state ? a.init_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
     if (c1 <= c0) {   // empty sequence: the state passes through
-        if (fin)
+        if (fin && warp < CFW_EPI_WARPS)
             for (int x = 0; x < 32; ++x) fin[x] = ini ? ini[x] : 0.f;
         return;
     }
@@ -548,8 +562,13 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     if (tid == 0) {
         mbar_init(&bar_full[0], 1);
         mbar_init(&bar_full[1], 1);
-        mbar_init(&bar_mma1, 1);
-        mbar_init(&bar_mma2, 1);
+        mbar_init(&bar_empty[0], 1);
+        mbar_init(&bar_empty[1], 1);
+        mbar_init(&bar_s_ready, CFW_EPI_WARPS);
+        mbar_init(&bar_du_done, 1);
+        mbar_init(&bar_du_ready, CFW_EPI_WARPS);
+        mbar_init(&bar_s_done, 1);
+        mbar_init(&bar_o_done, 1);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(&tmem_base, 512);
@@ -557,153 +576,184 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base;
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t tS = tb, tDU = tb + 128, tO1 = tb + 192, tO2 = tb + 320;   // O1, O2: two buffers of 64
 
-    auto issue_loads = [&](int n, int st) {
-        const int tok0 = chunk_tok0(n);
-        const size_t tile = (size_t)(c0 + n) * H + h;
-        uint8_t* d = sStage + st * STAGE_BYTES;
-        mbar_expect_tx(&bar_full[st], STAGE_BYTES);
-        bulk_load(d + ST_WT, a.WT + tile * 16384, 16384, &bar_full[st]);
-        bulk_load(d + ST_TB, a.Tb + tile * 8192, 8192, &bar_full[st]);
-        bulk_load(d + ST_P, a.P + tile * 8192, 8192, &bar_full[st]);
-        for (int hf = 0; hf < 2; ++hf) {
-            tma_load_2d(d + ST_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_full[st]);
-            tma_load_2d(d + ST_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_full[st]);
-            tma_load_2d(d + ST_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
-        }
-    };
-    // raw gates of chunk n for the gate warp (lane l: tokens l and l + 32)
-    auto load_gates = [&](int n, float& ga, float& gb) {
-        const int tok0 = chunk_tok0(n), len = chunk_len(n);
-        ga = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
-        gb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
-    };
-    // output of chunk n from its O1 / O2 accumulators
-    auto store_out = [&](int n) {
-        const int tok0 = chunk_tok0(n), len = chunk_len(n), st = n & 1, gs = n % 3;
-        __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
-        uint32_t ra[16], rb[16];
-        tmem_ld16(tO1 + st * 64 + lane_addr + colq * 16, ra);
-        tmem_ld16(tO2 + st * 64 + lane_addr + colq * 16, rb);
-        tmem_ld_wait();
-#pragma unroll
-        for (int x = 0; x < 16; ++x) {
-            const int i = colq * 16 + x;
-            if (i < len)
-                op[(size_t)i * H * KD] = __float2bfloat16_rn(a.scale * sGam[gs][i] * __uint_as_float(ra[x]) +
-                                                             __uint_as_float(rb[x]));
-        }
-    };
-
-    if (tid == 0) issue_loads(0, 0);
-    float ga = 0.f, gb = 0.f;
-    if (warp == 15) {
-        load_gates(0, ga, gb);
-        warp_gate_vectors(ga, gb, lane, sGam[0], sRho[0], &sGC[0]);
-    }
-    // initial state into tensor memory
-    for (int cb = 0; cb < 2; ++cb) {
-        uint32_t r[16];
-#pragma unroll
-        for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(ini ? ini[cb * 16 + x] : 0.f);
-        tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
-    }
-    tmem_st_wait();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-
-    bool ok = true;
-    for (int n = 0; n < nchunks; ++n) {
-        const int st = n & 1, gs = n % 3;
-        const int len = chunk_len(n);
-        const size_t tile = (size_t)(c0 + n) * H + h;
-        uint8_t* d = sStage + st * STAGE_BYTES;
-        if (tid == 0 && n + 1 < nchunks) issue_loads(n + 1, st ^ 1);
-        if (warp == 15 && n + 1 < nchunks) load_gates(n + 1, ga, gb);   // consumed after MMA group 2 is issued
-    OSDN_CLK(1, 0, blockIdx.x == 0 && n == 3);
-
-        // ---- E0: S -> bf16 operand (+ saved copy), decay the accumulator -----------------------
-        {
-            const float gC = sGC[gs];
-            uint32_t rr[2][16];
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
-            tmem_ld_wait();
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                uint32_t* r = rr[cb];
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
-                    w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
-                    w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
-                    w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
-                    const uint32_t off = sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2);
-                    *reinterpret_cast<uint4*>(sS + (colq >> 1) * 16384 + off) = w;
+    if (warp == CFW_TMA_WARP) {
+        // ------------------------------------------------------------------ producer
+        bool ok = true;
+        for (int n = 0; n < nchunks && ok; ++n) {
+            const int st = n & 1, gs = n & 1;
+            const int tok0 = chunk_tok0(n), len = chunk_len(n);
+            const float ga = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
+            const float gb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+            if (n >= 2) ok = mbar_wait(&bar_empty[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_TMA);
+            if (!ok) break;
+            warp_gate_vectors(ga, gb, lane, sGam[gs], sRho[gs], &sGC[gs]);
+            __syncwarp();
+            if (lane == 0) {
+                const size_t tile = (size_t)(c0 + n) * H + h;
+                uint8_t* d = sStage + st * STAGE_BYTES;
+                mbar_expect_tx(&bar_full[st], STAGE_BYTES);
+                bulk_load(d + ST_WT, a.WT + tile * 16384, 16384, &bar_full[st]);
+                bulk_load(d + ST_TB, a.Tb + tile * 8192, 8192, &bar_full[st]);
+                bulk_load(d + ST_P, a.P + tile * 8192, 8192, &bar_full[st]);
+                for (int hf = 0; hf < 2; ++hf) {
+                    tma_load_2d(d + ST_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_full[st]);
+                    tma_load_2d(d + ST_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_full[st]);
+                    tma_load_2d(d + ST_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
                 }
-#pragma unroll
-                for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
-                tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
             }
-            tmem_st_wait();
+            __syncwarp();
         }
-    OSDN_CLK(1, 1, blockIdx.x == 0 && n == 3);
-        ok = ok && mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
-    OSDN_CLK(1, 2, blockIdx.x == 0 && n == 3);
-        if (len < CH) {
-            for (int hf = 0; hf < 2; ++hf) {
-                zero_tail_rows(d + ST_V + hf * BOX, len, tid, CF2_THREADS);
-                zero_tail_rows(d + ST_Q + hf * BOX, len, tid, CF2_THREADS);
-                zero_tail_rows(d + ST_KT + hf * BOX, len, tid, CF2_THREADS);
-            }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-    OSDN_CLK(1, 3, blockIdx.x == 0 && n == 3);
-
-        // ---- MMA group 1 -----------------------------------------------------------------------
-        if (tid == 0 && ok) {
+    } else if (warp == CFW_MMA_WARP) {
+        // ------------------------------------------------------------------ tensor-core issuer
+        bool ok = true;
+        for (int n = 0; n < nchunks && ok; ++n) {
+            const int st = n & 1;
+            const size_t tile = (size_t)(c0 + n) * H + h;
+            uint8_t* d = sStage + st * STAGE_BYTES;
+            ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
+            ok = ok && mbar_wait(&bar_s_ready, n & 1, a.status, ERR_CHAIN_MMA1);
+            if (!ok) break;
             tc_fence_after();
-            if (a.save) {   // the state of this chunk, as the bf16 image just written
-                bulk_store(a.Sn + tile * 32768, sS, 32768);
-                bulk_commit();
+            if (lane == 0) {
+                bulk_wait_read();   // saved images of the previous chunk have left shared memory
+                if (a.save) {
+                    bulk_store(a.Sn + tile * 32768, sS, 32768);
+                    bulk_commit();
+                }
+                {   // dU^T = V^T Tb^T
+                    const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
+                    const uint64_t da0 = desc_mnmajor(d + ST_V, BOX), db0 = desc_kmajor(d + ST_TB);
+                    for (int k = 0; k < 4; ++k)
+                        mma_ss(tDU, desc_advance(da0, 2048 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+                }
+                {   // dU^T -= S W^T
+                    const uint32_t idesc = make_idesc(128, 64, IDESC_A_NEG | IDESC_B_MN);
+                    const uint64_t db0 = desc_mnmajor(d + ST_WT, 0);
+                    for (int k = 0; k < 8; ++k)
+                        mma_ss(tDU, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
+                               desc_advance(db0, 2048 * k), idesc, 1);
+                }
+                mma_commit(&bar_du_done);
+                {   // O1^T = S Q^T
+                    const uint32_t idesc = make_idesc(128, 64);
+                    for (int k = 0; k < 8; ++k)
+                        mma_ss(tO1 + st * 64, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
+                               desc_advance(desc_kmajor(d + ST_Q + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
+                }
             }
-            {   // dU^T = V^T Tb^T
-                const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
-                const uint64_t da0 = desc_mnmajor(d + ST_V, BOX), db0 = desc_kmajor(d + ST_TB);
-                for (int k = 0; k < 4; ++k)
-                    mma_ss(tDU, desc_advance(da0, 2048 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+            __syncwarp();
+            ok = mbar_wait(&bar_du_ready, n & 1, a.status, ERR_CHAIN_MMA2);
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0) {
+                if (a.save) {
+                    bulk_store(a.dUT + tile * 16384, sDU1, 16384);
+                    bulk_commit();
+                }
+                {   // S += (rho dU)^T Ktil
+                    const uint32_t idesc = make_idesc(128, 128, IDESC_B_MN);
+                    const uint64_t da0 = desc_kmajor(sDU2), db0 = desc_mnmajor(d + ST_KT, BOX);
+                    for (int k = 0; k < 4; ++k)
+                        mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k), idesc, 1);
+                }
+                mma_commit(&bar_s_done);
+                {   // O2^T = dU^T P'^T
+                    const uint32_t idesc = make_idesc(128, 64);
+                    const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
+                    for (int k = 0; k < 4; ++k)
+                        mma_ss(tO2 + st * 64, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+                }
+                mma_commit(&bar_o_done);
+                mma_commit(&bar_empty[st]);
             }
-            {   // dU^T -= S W^T
-                const uint32_t idesc = make_idesc(128, 64, IDESC_A_NEG | IDESC_B_MN);
-                const uint64_t db0 = desc_mnmajor(d + ST_WT, 0);
-                for (int k = 0; k < 8; ++k)
-                    mma_ss(tDU, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
-                           desc_advance(db0, 2048 * k), idesc, 1);
-            }
-            mma_commit(&bar_mma1);
-            {   // O1^T = S Q^T  (not needed before the output is assembled: rides on the next commit)
-                const uint32_t idesc = make_idesc(128, 64);
-                for (int k = 0; k < 8; ++k)
-                    mma_ss(tO1 + st * 64, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
-                           desc_advance(desc_kmajor(d + ST_Q + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
-            }
+            __syncwarp();
         }
-        ok = ok && mbar_wait(&bar_mma1, n & 1, a.status, ERR_CHAIN_MMA1);
-        tc_fence_after();
-    OSDN_CLK(1, 4, blockIdx.x == 0 && n == 3);
-
-        // ---- E1: dU^T -> bf16 operands ---------------------------------------------------------
-        {
-            uint32_t r[16];
-            tmem_ld16(tDU + lane_addr + colq * 16, r);
+        if (lane == 0) bulk_wait_all();
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const int etid = tid;   // 0 .. 511
+        float gkeep[16];   // scale * gamma_i of the chunk whose output is still to be written
+        auto store_out = [&](int n) {
+            const int tok0 = chunk_tok0(n), len = chunk_len(n), st = n & 1;
+            __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
+            uint32_t ra[16], rb[16];
+            tmem_ld16(tO1 + st * 64 + lane_addr + colq * 16, ra);
+            tmem_ld16(tO2 + st * 64 + lane_addr + colq * 16, rb);
             tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 16; ++x) {
+                const int i = colq * 16 + x;
+                if (i < len)
+                    op[(size_t)i * H * KD] = __float2bfloat16_rn(gkeep[x] * __uint_as_float(ra[x]) +
+                                                                 __uint_as_float(rb[x]));
+            }
+        };
+        // initial state into tensor memory
+        for (int cb = 0; cb < 2; ++cb) {
+            uint32_t r[16];
+#pragma unroll
+            for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(ini ? ini[cb * 16 + x] : 0.f);
+            tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
+        }
+        tmem_st_wait();
+
+        bool ok = true;
+        for (int n = 0; n < nchunks && ok; ++n) {
+            const int st = n & 1, gs = n & 1;
+            const int len = chunk_len(n);
+            uint8_t* d = sStage + st * STAGE_BYTES;
+            ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);   // gate vectors, tail rows
+            if (n > 0) ok = ok && mbar_wait(&bar_s_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2);
+            if (!ok) break;
+            tc_fence_after();
+            // ---- E0: S -> bf16 operand, decay the accumulator
             {
+                const float gC = sGC[gs];
+                uint32_t rr[2][16];
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    uint32_t* r = rr[cb];
+#pragma unroll
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
+                        w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
+                        w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
+                        w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
+                        *reinterpret_cast<uint4*>(sS + (colq >> 1) * 16384 + sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2)) = w;
+                    }
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
+                    tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
+                }
+                tmem_st_wait();
+            }
+            if (len < CH) {
+                for (int hf = 0; hf < 2; ++hf) {
+                    zero_tail_rows(d + ST_V + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
+                    zero_tail_rows(d + ST_Q + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
+                    zero_tail_rows(d + ST_KT + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
+                }
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_s_ready);
+
+            // ---- E1: dU^T -> bf16 operands
+            ok = mbar_wait(&bar_du_done, n & 1, a.status, ERR_CHAIN_MMA1);
+            if (!ok) break;
+            tc_fence_after();
+            {
+                uint32_t r[16];
+                tmem_ld16(tDU + lane_addr + colq * 16, r);
+                tmem_ld_wait();
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     float f[8], g[8];
@@ -713,74 +763,50 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                         g[x] = f[x] * sRho[gs][colq * 16 + c2 * 8 + x];
                     }
                     const uint32_t off = sw128_chunk(v, colq * 2 + c2);
-                    const uint4 w1 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
-                                                pack_bf16(f[6], f[7]));
-                    *reinterpret_cast<uint4*>(sDU1 + off) = w1;
+                    *reinterpret_cast<uint4*>(sDU1 + off) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
+                                                                      pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
                     *reinterpret_cast<uint4*>(sDU2 + off) = make_uint4(pack_bf16(g[0], g[1]), pack_bf16(g[2], g[3]),
                                                                       pack_bf16(g[4], g[5]), pack_bf16(g[6], g[7]));
                 }
             }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-    OSDN_CLK(1, 5, blockIdx.x == 0 && n == 3);
-
-        // ---- MMA group 2 -----------------------------------------------------------------------
-        if (tid == 0 && ok) {
-            tc_fence_after();
-            if (a.save) {
-                bulk_store(a.dUT + tile * 16384, sDU1, 16384);
-                bulk_commit();
-            }
-            {   // S += (rho dU)^T Ktil   (on the critical path: first)
-                const uint32_t idesc = make_idesc(128, 128, IDESC_B_MN);
-                const uint64_t da0 = desc_kmajor(sDU2), db0 = desc_mnmajor(d + ST_KT, BOX);
-                for (int k = 0; k < 4; ++k)
-                    mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k), idesc, 1);
-            }
-            mma_commit(&bar_mma2);
-            {   // O2^T = dU^T P'^T   (completes before the next commit, which the output waits for)
-                const uint32_t idesc = make_idesc(128, 64);
-                const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
-                for (int k = 0; k < 4; ++k)
-                    mma_ss(tO2 + st * 64, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, k > 0);
-            }
-        }
-        // while the tensor core works: gate vectors of the next chunk, output of the previous chunk
-        // (its O2 accumulator was issued after the previous chunk's last commit and is covered by
-        // this chunk's first commit, which has been waited for above)
-        if (warp == 15 && n + 1 < nchunks)
-            warp_gate_vectors(ga, gb, lane, sGam[(n + 1) % 3], sRho[(n + 1) % 3], &sGC[(n + 1) % 3]);
-        if (n > 0 && ok) store_out(n - 1);
-        ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
-        tc_fence_after();
-    OSDN_CLK(1, 6, blockIdx.x == 0 && n == 3);
-        if (tid == 0) bulk_wait_read();   // the saved images have left shared memory before it is rewritten
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-    OSDN_CLK(1, 7, blockIdx.x == 0 && n == 3);
-    }
-
-    // the last chunk's output accumulators were issued after the last commits: close them
-    if (tid == 0 && ok) {
-        mma_commit(&bar_mma1);
-    }
-    ok = ok && mbar_wait(&bar_mma1, nchunks & 1, a.status, ERR_CHAIN_MMA1);
-    tc_fence_after();
-    if (ok) store_out(nchunks - 1);
-
-    if (fin && ok) {
-        for (int cb = 0; cb < 2; ++cb) {
-            uint32_t r[16];
-            tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, r);
-            tmem_ld_wait();
+            float gnew[16];   // this chunk's output factors, read while the gate slot is still valid
 #pragma unroll
-            for (int x = 0; x < 16; ++x) fin[cb * 16 + x] = __uint_as_float(r[x]);
+            for (int x = 0; x < 16; ++x) gnew[x] = a.scale * sGam[gs][colq * 16 + x];
+            // The previous chunk's output accumulators: observed complete BEFORE this warp releases the
+            // products of this chunk, so that the barrier cannot run two phases ahead of a waiter.
+            if (n > 0) {
+                ok = mbar_wait(&bar_o_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2);
+                if (!ok) break;
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_du_ready);
+
+            // ---- output of the previous chunk, in the shadow of this chunk's state update
+            if (n > 0) {
+                tc_fence_after();
+                store_out(n - 1);
+            }
+#pragma unroll
+            for (int x = 0; x < 16; ++x) gkeep[x] = gnew[x];
+        }
+        if (ok) ok = mbar_wait(&bar_o_done, (nchunks - 1) & 1, a.status, ERR_CHAIN_MMA2);
+        if (ok) ok = mbar_wait(&bar_s_done, (nchunks - 1) & 1, a.status, ERR_CHAIN_MMA2);
+        tc_fence_after();
+        if (ok) {
+            store_out(nchunks - 1);
+            if (fin) {
+                for (int cb = 0; cb < 2; ++cb) {
+                    uint32_t r[16];
+                    tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) fin[cb * 16 + x] = __uint_as_float(r[x]);
+                }
+            }
         }
     }
-    if (tid == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tb, 512);
@@ -1704,7 +1730,7 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
         ch.status = status;
         if (!set_smem(tc_chain_fwd_kernel, CF_SMEM)) return -1;
         stage_mark(st, "tc_chain_fwd");
-        tc_chain_fwd_kernel<<<S * H, CF2_THREADS, CF_SMEM, st>>>(tmV, tmQ, tmKt, ch);
+        tc_chain_fwd_kernel<<<S * H, CFW_THREADS, CF_SMEM, st>>>(tmV, tmQ, tmKt, ch);
         ++launches;
     }
     stage_end(st);
