@@ -36,8 +36,39 @@ __device__ long long g_clk[4][32];
     do {                                                              \
         if ((cond) && threadIdx.x == 0) g_clk[k][i] = clock64();      \
     } while (0)
+#ifndef OSDN_CLK_MASK
+#define OSDN_CLK_MASK 0xffffffffu
+#endif
+#define OSDN_CLKW(k, i, cond)                                         \
+    do {                                                              \
+        if (((OSDN_CLK_MASK >> (i)) & 1u) && (cond)) g_clk[k][i] = clock64(); \
+    } while (0)
+// stamps kept in shared memory until the kernel ends (a global store in the loop would itself stall
+// the tensor-memory loads that follow it)
+#define OSDN_CLKS(i, cond)                                            \
+    do {                                                              \
+        if (((OSDN_CLK_MASK >> (i)) & 1u) && (cond)) s_clk[i] = clock64(); \
+    } while (0)
+// accumulated waiting time of one thread: OSDN_ACC_DECL once, then OSDN_ACC(slot, statement)
+#define OSDN_ACC_DECL long long acc_clk[6] = {0, 0, 0, 0, 0, 0}
+#define OSDN_ACC(slot, stmt)                                          \
+    do {                                                              \
+        const long long t_acc0 = clock64();                           \
+        stmt;                                                         \
+        acc_clk[slot] += clock64() - t_acc0;                          \
+    } while (0)
+#define OSDN_ACC_DUMP(base, count, cond)                              \
+    do {                                                              \
+        if (cond)                                                     \
+            for (int i_acc = 0; i_acc < (count); ++i_acc) s_clk[(base) + i_acc] = acc_clk[i_acc]; \
+    } while (0)
 #else
 #define OSDN_CLK(k, i, cond)
+#define OSDN_CLKW(k, i, cond)
+#define OSDN_CLKS(i, cond)
+#define OSDN_ACC_DECL
+#define OSDN_ACC(slot, stmt) stmt
+#define OSDN_ACC_DUMP(base, count, cond)
 #endif
 
 namespace {
@@ -47,6 +78,8 @@ constexpr uint32_t BOX = 8192;   // one [64 rows x 128 B] box
 
 // device status codes of bounded waits
 enum { ERR_TMA = 101, ERR_MMA1 = 102, ERR_MMA2 = 103, ERR_CHAIN_TMA = 111, ERR_CHAIN_MMA1 = 112, ERR_CHAIN_MMA2 = 113 };
+
+constexpr uint32_t REC_BYTES = 49152;   // stride of the Tb | W^T | P' | Qg record of a tile
 
 struct TcLayout {
     size_t ktil, WT, Tb, Tm, P, Qg, Sn, dUT, ddUT, dSn, dktil, dkread, total;
@@ -61,11 +94,14 @@ TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
     auto take = [&](size_t b) { size_t o = off; off = align_up(off + b, 1024); return o; };
     off = align_up(off, 1024);
     t.ktil = take(Ttot * H * KD * 2);
-    t.WT = take(NT * H * 16384);
-    t.Tb = take(NT * H * 8192);
+    // One record per (chunk, head) tile, Tb | W^T | P' | Qg, so that either chain kernel fetches the
+    // tiles it needs (the first three forward, the last three backward) with a single bulk copy.
+    const size_t rec = take(NT * H * (size_t)REC_BYTES);
+    t.Tb = rec;
+    t.WT = rec + 8192;
+    t.P = rec + 24576;
+    t.Qg = rec + 32768;
     t.Tm = take(NT * H * 8192);
-    t.P = take(NT * H * 8192);
-    t.Qg = take(NT * H * 16384);
     t.Sn = take(NT * H * 32768);
     t.dUT = take(NT * H * 16384);
     if (need_bwd) {
@@ -363,7 +399,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         } else {
             const int i = L - CH;
             const float Gi = sG[i];
-            uint8_t* Pg = a.P + tile * 8192;
+            uint8_t* Pg = a.P + tile * REC_BYTES;
             for (int cb = 0; cb < 4; ++cb) {
                 uint32_t r[16];
                 tmem_ld16(taddr + cb * 16, r);
@@ -405,7 +441,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const float2 v = __bfloat1622float2(p2[x]);
                 o[x] = pack_bf16(v.x * f, v.y * f);
             }
-            *reinterpret_cast<uint4*>(a.Qg + tile * 16384 + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(a.Qg + tile * REC_BYTES + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
 
@@ -423,7 +459,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t off = sw128_chunk(i, ch);
         *reinterpret_cast<uint4*>(sTb + off) = make_uint4(pack_bf16(tbg[0], tbg[1]), pack_bf16(tbg[2], tbg[3]),
                                                          pack_bf16(tbg[4], tbg[5]), pack_bf16(tbg[6], tbg[7]));
-        *reinterpret_cast<uint4*>(a.Tb + tile * 8192 + off) =
+        *reinterpret_cast<uint4*>(a.Tb + tile * REC_BYTES + off) =
             make_uint4(pack_bf16(tb8[0], tb8[1]), pack_bf16(tb8[2], tb8[3]), pack_bf16(tb8[4], tb8[5]),
                        pack_bf16(tb8[6], tb8[7]));
         if (a.save)
@@ -450,7 +486,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (ok) {
         const int k = warp * 32 + lane;
         const uint32_t taddr = tb + ((uint32_t)(warp * 32) << 16) + 64;
-        uint8_t* Wg = a.WT + tile * 16384;
+        uint8_t* Wg = a.WT + tile * REC_BYTES;
         for (int cb = 0; cb < 4; ++cb) {
             uint32_t r[16];
             tmem_ld16(taddr + cb * 16, r);
@@ -491,7 +527,7 @@ struct TcChainArgs {
 constexpr int CF_THREADS = 256;
 constexpr int CF2_THREADS = 512;   // forward chain: 16 warps = 4 lane quadrants x 4 column groups
 constexpr uint32_t STAGE_BYTES = 16384 + 8192 + 8192 + 3 * 16384;   // WT, Tb, P, V, Q, Ktil = 81920
-constexpr uint32_t ST_WT = 0, ST_TB = 16384, ST_P = 24576, ST_V = 32768, ST_Q = 49152, ST_KT = 65536;
+constexpr uint32_t ST_TB = 0, ST_WT = 8192, ST_P = 24576, ST_V = 32768, ST_Q = 49152, ST_KT = 65536;
 constexpr size_t CF_SMEM = 2 * STAGE_BYTES + 32768 + 2 * 16384 + 1024;
 
 // In-chunk gate prefix by one warp: lane l holds g_l and g_{l+32}.  Writes gamma_i = exp(G_i),
@@ -513,19 +549,23 @@ __device__ __forceinline__ void warp_gate_vectors(float ga, float gb, int lane, 
     if (lane == 0) *gC = __expf(tot);
 }
 
-// Warp roles of the forward chain: 16 epilogue warps (4 lane quadrants x 4 column groups), one warp
-// that issues the tensor-core work, one warp that issues the loads and prepares the gate vectors.
-// The roles run decoupled and meet only at mbarriers:
-//   full[st]   loads of a chunk have landed (and its gate vectors are written)      producer -> all
-//   empty[st]  every product reading the stage has finished                         tensor core -> producer
-//   s_ready    S is in shared memory as a bf16 operand, the accumulator is decayed  epilogue -> issuer
-//   du_done    dU^T accumulator complete                                            tensor core -> epilogue
-//   du_ready   dU^T operands are in shared memory                                   epilogue -> issuer
-//   s_done     the state update of the chunk is complete                            tensor core -> epilogue
-//   o_done     both output accumulators of the chunk are complete                   tensor core -> epilogue
-constexpr int CFW_EPI_WARPS = 16;
-constexpr int CFW_MMA_WARP = 16, CFW_TMA_WARP = 17;
-constexpr int CFW_THREADS = 18 * 32;
+// Warp roles of the forward chain: 16 state warps (4 lane quadrants x 4 column groups), 4 output warps
+// (one per lane quadrant), one warp that issues the tensor-core work, one warp that issues the loads
+// and prepares the gate vectors.  The roles run decoupled and meet only at mbarriers:
+//   full[st]    loads of a chunk have landed (and its gate vectors are written)      producer -> all
+//   empty[st]   every product reading the stage has finished                         tensor core -> producer
+//   s_ready     S is in shared memory as a bf16 operand, the accumulator is decayed  state warps -> issuer
+//   du_done     dU^T accumulator complete                                            tensor core -> state warps
+//   du_ready    dU^T operands are in shared memory                                   state warps -> issuer
+//   s_done      the state update of the chunk is complete                            tensor core -> state warps
+//   o_done[st]  both output accumulators of the chunk are complete                   tensor core -> output warps
+//   o_free[st]  the output accumulators have been read                               output warps -> issuer
+// The state warps carry the recurrence and never store to global memory inside the loop: a warp's
+// tensor-memory load does not return while its earlier global stores are outstanding, which would
+// put the latency of the output stores on the chunk-to-chunk path.
+constexpr int CFW_EPI_WARPS = 16, CFW_OUT_WARPS = 4;
+constexpr int CFW_OUT_WARP0 = 16, CFW_MMA_WARP = 20, CFW_TMA_WARP = 21;
+constexpr int CFW_THREADS = 22 * 32;
 
 __global__ void __launch_bounds__(CFW_THREADS, 1)
 tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
@@ -537,9 +577,16 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     uint8_t* sS = sm + 2 * STAGE_BYTES;         // S as bf16, K-major: 2 k-halves x [128 rows x 128 B]
     uint8_t* sDU1 = sS + 32768;                 // dU^T, K-major [v][i]
     uint8_t* sDU2 = sDU1 + 16384;               // (rho dU)^T
-    __shared__ uint64_t bar_full[2], bar_empty[2], bar_s_ready, bar_du_done, bar_du_ready, bar_s_done, bar_o_done;
+    __shared__ uint64_t bar_full[2], bar_empty[2], bar_s_ready, bar_du_done, bar_du_ready, bar_s_done;
+    __shared__ uint64_t bar_o_done[2], bar_o_free[2];
     __shared__ uint32_t tmem_base;
-    __shared__ float sGam[2][CH], sRho[2][CH], sGC[2];   // slot = chunk % 2 (read only before du_ready)
+    __shared__ float sRho[2][CH], sGC[2];              // slot = chunk % 2
+    __shared__ float sOutGam[CFW_OUT_WARPS][CH];       // scale * gamma_i, private to each output warp
+#ifdef OSDN_PHASE_CLOCKS
+    __shared__ long long s_clk[32];
+    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
+    __syncthreads();
+#endif
 
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
@@ -547,7 +594,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, colq = (warp >> 2) & 3;
-    const int v = quad * 32 + lane;             // state row owned by an epilogue thread
+    const int v = quad * 32 + lane;             // state row owned by a state-warp thread
     float* fin = a.final_state ? a.final_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
     const float* ini = a.init_state ? a.init_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
     if (c1 <= c0) {   // empty sequence: the state passes through
@@ -558,17 +605,21 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     const int nchunks = c1 - c0;
     auto chunk_tok0 = [&](int n) { return seq_t0 + n * CH; };
     auto chunk_len = [&](int n) { return min(CH, seq_len - n * CH); };
+    OSDN_CLKS(15, blockIdx.x == 0 && tid == 0);
 
     if (tid == 0) {
-        mbar_init(&bar_full[0], 1);
-        mbar_init(&bar_full[1], 1);
+        mbar_init(&bar_full[0], 2);
+        mbar_init(&bar_full[1], 2);
         mbar_init(&bar_empty[0], 1);
         mbar_init(&bar_empty[1], 1);
         mbar_init(&bar_s_ready, CFW_EPI_WARPS);
         mbar_init(&bar_du_done, 1);
         mbar_init(&bar_du_ready, CFW_EPI_WARPS);
         mbar_init(&bar_s_done, 1);
-        mbar_init(&bar_o_done, 1);
+        mbar_init(&bar_o_done[0], 1);
+        mbar_init(&bar_o_done[1], 1);
+        mbar_init(&bar_o_free[0], CFW_OUT_WARPS);
+        mbar_init(&bar_o_free[1], CFW_OUT_WARPS);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(&tmem_base, 512);
@@ -580,54 +631,66 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 
     if (warp == CFW_TMA_WARP) {
         // ------------------------------------------------------------------ producer
+        // A stage is complete when its copies have landed (transaction count, first arrival) and the
+        // gate vectors of the chunk are written (second arrival).  The gates are read a chunk ahead.
         bool ok = true;
+        auto load_gates = [&](int n, float& ga, float& gb) {
+            const int tok0 = chunk_tok0(n), len = chunk_len(n);
+            ga = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
+            gb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+        };
+        float ga, gb;
+        load_gates(0, ga, gb);
         for (int n = 0; n < nchunks && ok; ++n) {
             const int st = n & 1, gs = n & 1;
-            const int tok0 = chunk_tok0(n), len = chunk_len(n);
-            const float ga = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
-            const float gb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+            const int tok0 = chunk_tok0(n);
+            float ga_next = 0.f, gb_next = 0.f;
+            if (n + 1 < nchunks) load_gates(n + 1, ga_next, gb_next);
             if (n >= 2) ok = mbar_wait(&bar_empty[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_TMA);
             if (!ok) break;
-            warp_gate_vectors(ga, gb, lane, sGam[gs], sRho[gs], &sGC[gs]);
-            __syncwarp();
             if (lane == 0) {
                 const size_t tile = (size_t)(c0 + n) * H + h;
                 uint8_t* d = sStage + st * STAGE_BYTES;
                 mbar_expect_tx(&bar_full[st], STAGE_BYTES);
-                bulk_load(d + ST_WT, a.WT + tile * 16384, 16384, &bar_full[st]);
-                bulk_load(d + ST_TB, a.Tb + tile * 8192, 8192, &bar_full[st]);
-                bulk_load(d + ST_P, a.P + tile * 8192, 8192, &bar_full[st]);
-                for (int hf = 0; hf < 2; ++hf) {
-                    tma_load_2d(d + ST_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_full[st]);
-                    tma_load_2d(d + ST_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_full[st]);
-                    tma_load_2d(d + ST_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
-                }
+                bulk_load(d + ST_TB, a.Tb + tile * REC_BYTES, 32768, &bar_full[st]);   // Tb, W^T, P'
+                for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + ST_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_full[st]);
+                for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + ST_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_full[st]);
+                for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + ST_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
             }
             __syncwarp();
+            warp_gate_vectors(ga, gb, lane, nullptr, sRho[gs], &sGC[gs]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_full[st]);
+            ga = ga_next;
+            gb = gb_next;
         }
     } else if (warp == CFW_MMA_WARP) {
         // ------------------------------------------------------------------ tensor-core issuer
         bool ok = true;
+        OSDN_ACC_DECL;
+        bool ut_issued = false;   // V^T Tb^T of the coming chunk is already in the dU^T accumulator
+        auto issue_ut = [&](uint8_t* d) {   // dU^T = V^T Tb^T
+            const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
+            const uint64_t da0 = desc_mnmajor(d + ST_V, BOX), db0 = desc_kmajor(d + ST_TB);
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tDU, desc_advance(da0, 2048 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+        };
         for (int n = 0; n < nchunks && ok; ++n) {
             const int st = n & 1;
             const size_t tile = (size_t)(c0 + n) * H + h;
             uint8_t* d = sStage + st * STAGE_BYTES;
-            ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
-            ok = ok && mbar_wait(&bar_s_ready, n & 1, a.status, ERR_CHAIN_MMA1);
+            if (!ut_issued) OSDN_ACC(0, ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA));
+            OSDN_ACC(1, ok = ok && mbar_wait(&bar_s_ready, n & 1, a.status, ERR_CHAIN_MMA1));
             if (!ok) break;
             tc_fence_after();
+            OSDN_CLKS(10, blockIdx.x == 0 && n == 10 && lane == 0);
             if (lane == 0) {
                 bulk_wait_read();   // saved images of the previous chunk have left shared memory
                 if (a.save) {
                     bulk_store(a.Sn + tile * 32768, sS, 32768);
                     bulk_commit();
                 }
-                {   // dU^T = V^T Tb^T
-                    const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
-                    const uint64_t da0 = desc_mnmajor(d + ST_V, BOX), db0 = desc_kmajor(d + ST_TB);
-                    for (int k = 0; k < 4; ++k)
-                        mma_ss(tDU, desc_advance(da0, 2048 * k), desc_advance(db0, 32 * k), idesc, k > 0);
-                }
+                if (!ut_issued) issue_ut(d);
                 {   // dU^T -= S W^T
                     const uint32_t idesc = make_idesc(128, 64, IDESC_A_NEG | IDESC_B_MN);
                     const uint64_t db0 = desc_mnmajor(d + ST_WT, 0);
@@ -636,18 +699,28 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                                desc_advance(db0, 2048 * k), idesc, 1);
                 }
                 mma_commit(&bar_du_done);
-                {   // O1^T = S Q^T
-                    const uint32_t idesc = make_idesc(128, 64);
-                    for (int k = 0; k < 8; ++k)
-                        mma_ss(tO1 + st * 64, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
-                               desc_advance(desc_kmajor(d + ST_Q + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
-                }
+                OSDN_CLKS(11, blockIdx.x == 0 && n == 10);
             }
             __syncwarp();
-            ok = mbar_wait(&bar_du_ready, n & 1, a.status, ERR_CHAIN_MMA2);
+            // the output accumulators of chunk n - 2 (same buffers) have been read
+            if (n >= 2) OSDN_ACC(2, ok = mbar_wait(&bar_o_free[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_MMA2));
             if (!ok) break;
             tc_fence_after();
+            if (lane == 0) {   // O1^T = S Q^T
+                const uint32_t idesc = make_idesc(128, 64);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tO1 + st * 64, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
+                           desc_advance(desc_kmajor(d + ST_Q + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
+            }
+            __syncwarp();
+            OSDN_ACC(3, ok = mbar_wait(&bar_du_ready, n & 1, a.status, ERR_CHAIN_MMA2));
+            if (!ok) break;
+            tc_fence_after();
+            OSDN_CLKS(12, blockIdx.x == 0 && n == 10 && lane == 0);
             if (lane == 0) {
+                // The image of S sent off at the start of this chunk must have left shared memory before
+                // the state update is released: its completion lets the state warps overwrite that image.
+                bulk_wait_read();
                 if (a.save) {
                     bulk_store(a.dUT + tile * 16384, sDU1, 16384);
                     bulk_commit();
@@ -659,56 +732,160 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                         mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k), idesc, 1);
                 }
                 mma_commit(&bar_s_done);
+                OSDN_CLKS(13, blockIdx.x == 0 && n == 10);
                 {   // O2^T = dU^T P'^T
                     const uint32_t idesc = make_idesc(128, 64);
                     const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
                     for (int k = 0; k < 4; ++k)
                         mma_ss(tO2 + st * 64, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, k > 0);
                 }
-                mma_commit(&bar_o_done);
+                mma_commit(&bar_o_done[st]);
                 mma_commit(&bar_empty[st]);
             }
             __syncwarp();
+            // The part of the next chunk's dU^T that does not depend on the state goes in now, while the
+            // state warps convert S (full chunks only: a ragged chunk has its tail rows cleared first).
+            ut_issued = false;
+            if (n + 1 < nchunks && chunk_len(n + 1) == CH) {
+                OSDN_ACC(4, ok = mbar_wait(&bar_full[st ^ 1], ((n + 1) >> 1) & 1, a.status, ERR_CHAIN_TMA));
+                if (!ok) break;
+                if (lane == 0) issue_ut(sStage + (st ^ 1) * STAGE_BYTES);
+                __syncwarp();
+                ut_issued = true;
+            }
         }
         if (lane == 0) bulk_wait_all();
+        OSDN_ACC_DUMP(0, 5, blockIdx.x == 0 && lane == 0);
+    } else if (warp >= CFW_OUT_WARP0) {
+        // ------------------------------------------------------------------ output warps
+        // o_i = scale gamma_i (S q_i) + (P' dU)_i : lane = feature, 16 token columns per load
+        const int ow = warp - CFW_OUT_WARP0;   // == lane quadrant
+        const uint32_t lane_addr = (uint32_t)(ow * 32) << 16;
+        float* og = sOutGam[ow];
+        bool ok = true;
+        OSDN_ACC_DECL;
+        for (int n = 0; n < nchunks && ok; ++n) {
+            const int st = n & 1;
+            const int tok0 = chunk_tok0(n), len = chunk_len(n);
+            {   // in-chunk gate prefix, kept private to this warp
+                float sa = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
+                float sb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const float ua = __shfl_up_sync(0xffffffffu, sa, o), ub = __shfl_up_sync(0xffffffffu, sb, o);
+                    if (lane >= o) { sa += ua; sb += ub; }
+                }
+                sb += __shfl_sync(0xffffffffu, sa, 31);
+                __syncwarp();   // the previous chunk's factors are no longer read
+                og[lane] = a.scale * __expf(sa);
+                og[lane + 32] = a.scale * __expf(sb);
+                __syncwarp();
+            }
+            // Warm L2 with the operands of chunk n + 2 (the stage copies can only run one chunk ahead);
+            // each output warp asks for one operand.
+            if (lane == 0 && n + 2 < nchunks) {
+                const int t2 = chunk_tok0(n + 2);
+                if (ow == 0) bulk_prefetch(a.Tb + ((size_t)(c0 + n + 2) * H + h) * REC_BYTES, 32768);
+                const CUtensorMap* tm = ow == 1 ? &tmV : ow == 2 ? &tmQ : &tmKt;
+                if (ow > 0)
+                    for (int hf = 0; hf < 2; ++hf) tma_prefetch_2d(tm, h * KD + hf * 64, t2);
+            }
+            OSDN_ACC(0, ok = mbar_wait(&bar_o_done[st], (n >> 1) & 1, a.status, ERR_CHAIN_MMA2));
+            if (!ok) break;
+            tc_fence_after();
+            // Results leave as 16-byte stores: three shuffle rounds turn "lane = feature, 16 tokens" into
+            // "lane = 8 consecutive features of 2 tokens" (lane bit 0 picks the token half, bits 1-2 the
+            // token pair inside it, bits 3-4 the feature octet).
+            const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4;
+            const int tsub = (b0 ? 8 : 0) + ((lane >> 1) & 3) * 2;
+            __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + ow * 32 + (lane >> 3) * 8;
+#pragma unroll
+            for (int cg = 0; cg < 4; ++cg) {
+                uint32_t ra[16], rb[16];
+                tmem_ld16(tO1 + st * 64 + lane_addr + cg * 16, ra);
+                tmem_ld16(tO2 + st * 64 + lane_addr + cg * 16, rb);
+                tmem_ld_wait();
+                if (cg == 3) {   // everything is in registers: the buffers may be overwritten
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bar_o_free[st]);
+                }
+                float o[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x)
+                    o[x] = og[cg * 16 + x] * __uint_as_float(ra[x]) + __uint_as_float(rb[x]);
+                uint32_t w[8];    // feature pair (lane >> 1), token (b0 ? 8 : 0) + i
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float recv = __shfl_xor_sync(0xffffffffu, b0 ? o[i] : o[i + 8], 1);
+                    w[i] = b0 ? pack_bf16(recv, o[i + 8]) : pack_bf16(o[i], recv);
+                }
+                uint32_t wa[2][2][2];   // [token-pair bit 1][token parity][feature pair 0 / 1]
+#pragma unroll
+                for (int th = 0; th < 2; ++th)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const uint32_t w0 = w[(th * 2 + 0) * 2 + e], w1 = w[(th * 2 + 1) * 2 + e];
+                        const uint32_t keep = b1 ? w1 : w0;
+                        const uint32_t recv = __shfl_xor_sync(0xffffffffu, b1 ? w0 : w1, 2);
+                        wa[th][e][0] = b1 ? recv : keep;
+                        wa[th][e][1] = b1 ? keep : recv;
+                    }
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    uint32_t q4[4];
+#pragma unroll
+                    for (int sp = 0; sp < 2; ++sp) {
+                        const uint32_t keep = b2 ? wa[1][e][sp] : wa[0][e][sp];
+                        const uint32_t recv = __shfl_xor_sync(0xffffffffu, b2 ? wa[0][e][sp] : wa[1][e][sp], 4);
+                        q4[sp] = b2 ? recv : keep;
+                        q4[2 + sp] = b2 ? keep : recv;
+                    }
+                    const int i = cg * 16 + tsub + e;
+                    if (i < len)
+                        *reinterpret_cast<uint4*>(op + (size_t)i * H * KD) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
+                }
+            }
+        }
+        OSDN_ACC_DUMP(12, 1, blockIdx.x == 0 && ow == 0 && lane == 0);
     } else {
-        // ------------------------------------------------------------------ epilogue warps
+        // ------------------------------------------------------------------ state warps
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const int etid = tid;   // 0 .. 511
-        float gkeep[16];   // scale * gamma_i of the chunk whose output is still to be written
-        auto store_out = [&](int n) {
-            const int tok0 = chunk_tok0(n), len = chunk_len(n), st = n & 1;
-            __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + v;
-            uint32_t ra[16], rb[16];
-            tmem_ld16(tO1 + st * 64 + lane_addr + colq * 16, ra);
-            tmem_ld16(tO2 + st * 64 + lane_addr + colq * 16, rb);
-            tmem_ld_wait();
-#pragma unroll
-            for (int x = 0; x < 16; ++x) {
-                const int i = colq * 16 + x;
-                if (i < len)
-                    op[(size_t)i * H * KD] = __float2bfloat16_rn(gkeep[x] * __uint_as_float(ra[x]) +
-                                                                 __uint_as_float(rb[x]));
-            }
-        };
         // initial state into tensor memory
         for (int cb = 0; cb < 2; ++cb) {
             uint32_t r[16];
 #pragma unroll
-            for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(ini ? ini[cb * 16 + x] : 0.f);
+            for (int x4 = 0; x4 < 4; ++x4) {
+                const float4 f4 = ini ? *reinterpret_cast<const float4*>(ini + cb * 16 + x4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                r[x4 * 4 + 0] = __float_as_uint(f4.x);
+                r[x4 * 4 + 1] = __float_as_uint(f4.y);
+                r[x4 * 4 + 2] = __float_as_uint(f4.z);
+                r[x4 * 4 + 3] = __float_as_uint(f4.w);
+            }
             tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
         }
         tmem_st_wait();
 
         bool ok = true;
+        OSDN_ACC_DECL;
         for (int n = 0; n < nchunks && ok; ++n) {
             const int st = n & 1, gs = n & 1;
             const int len = chunk_len(n);
             uint8_t* d = sStage + st * STAGE_BYTES;
-            ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);   // gate vectors, tail rows
-            if (n > 0) ok = ok && mbar_wait(&bar_s_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2);
+            OSDN_ACC(0, ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA));   // gate vectors, tail rows
+#ifdef OSDN_PHASE_CLOCKS
+            acc_clk[3] += clock64() - s_clk[20 + st];
+#endif
+            if (n > 0) OSDN_ACC(1, ok = ok && mbar_wait(&bar_s_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2));
             if (!ok) break;
             tc_fence_after();
+            OSDN_CLKS(0, blockIdx.x == 0 && n == 10 && tid == 0);
+            OSDN_CLKS(8, blockIdx.x == 0 && n == 11 && tid == 0);
+            OSDN_CLKS(17, blockIdx.x == 0 && n == 0 && tid == 0);
+            OSDN_CLKS(18, blockIdx.x == 0 && n == 1 && tid == 0);
+            OSDN_CLKS(19, blockIdx.x == 0 && n == 20 && tid == 0);
+            OSDN_CLKS(24, blockIdx.x == 0 && n == 31 && tid == 0);
             // ---- E0: S -> bf16 operand, decay the accumulator
             {
                 const float gC = sGC[gs];
@@ -716,6 +893,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 #pragma unroll
                 for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
                 tmem_ld_wait();
+                OSDN_CLKS(1, blockIdx.x == 0 && n == 10 && tid == 0);
 #pragma unroll
                 for (int cb = 0; cb < 2; ++cb) {
                     uint32_t* r = rr[cb];
@@ -734,6 +912,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                 }
                 tmem_st_wait();
             }
+            OSDN_CLKS(2, blockIdx.x == 0 && n == 10 && tid == 0);
             if (len < CH) {
                 for (int hf = 0; hf < 2; ++hf) {
                     zero_tail_rows(d + ST_V + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
@@ -745,70 +924,65 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_s_ready);
+            OSDN_CLKS(3, blockIdx.x == 0 && n == 10 && tid == 0);
 
             // ---- E1: dU^T -> bf16 operands
-            ok = mbar_wait(&bar_du_done, n & 1, a.status, ERR_CHAIN_MMA1);
+            float rho[16];
+#pragma unroll
+            for (int x = 0; x < 16; ++x) rho[x] = sRho[gs][colq * 16 + x];
+            OSDN_ACC(2, ok = mbar_wait(&bar_du_done, n & 1, a.status, ERR_CHAIN_MMA1));
             if (!ok) break;
             tc_fence_after();
+            OSDN_CLKS(4, blockIdx.x == 0 && n == 10 && tid == 0);
             {
                 uint32_t r[16];
                 tmem_ld16(tDU + lane_addr + colq * 16, r);
                 tmem_ld_wait();
+                OSDN_CLKS(5, blockIdx.x == 0 && n == 10 && tid == 0);
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     float f[8], g[8];
 #pragma unroll
                     for (int x = 0; x < 8; ++x) {
                         f[x] = __uint_as_float(r[c2 * 8 + x]);
-                        g[x] = f[x] * sRho[gs][colq * 16 + c2 * 8 + x];
+                        g[x] = f[x] * rho[c2 * 8 + x];
                     }
                     const uint32_t off = sw128_chunk(v, colq * 2 + c2);
-                    *reinterpret_cast<uint4*>(sDU1 + off) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
-                                                                      pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
                     *reinterpret_cast<uint4*>(sDU2 + off) = make_uint4(pack_bf16(g[0], g[1]), pack_bf16(g[2], g[3]),
                                                                       pack_bf16(g[4], g[5]), pack_bf16(g[6], g[7]));
+                    *reinterpret_cast<uint4*>(sDU1 + off) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
+                                                                      pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
                 }
-            }
-            float gnew[16];   // this chunk's output factors, read while the gate slot is still valid
-#pragma unroll
-            for (int x = 0; x < 16; ++x) gnew[x] = a.scale * sGam[gs][colq * 16 + x];
-            // The previous chunk's output accumulators: observed complete BEFORE this warp releases the
-            // products of this chunk, so that the barrier cannot run two phases ahead of a waiter.
-            if (n > 0) {
-                ok = mbar_wait(&bar_o_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2);
-                if (!ok) break;
             }
             fence_proxy_async();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_du_ready);
-
-            // ---- output of the previous chunk, in the shadow of this chunk's state update
-            if (n > 0) {
-                tc_fence_after();
-                store_out(n - 1);
-            }
-#pragma unroll
-            for (int x = 0; x < 16; ++x) gkeep[x] = gnew[x];
+            OSDN_CLKS(6, blockIdx.x == 0 && n == 10 && tid == 0);
         }
-        if (ok) ok = mbar_wait(&bar_o_done, (nchunks - 1) & 1, a.status, ERR_CHAIN_MMA2);
+        OSDN_ACC_DUMP(6, 4, blockIdx.x == 0 && tid == 0);
         if (ok) ok = mbar_wait(&bar_s_done, (nchunks - 1) & 1, a.status, ERR_CHAIN_MMA2);
         tc_fence_after();
-        if (ok) {
-            store_out(nchunks - 1);
-            if (fin) {
-                for (int cb = 0; cb < 2; ++cb) {
-                    uint32_t r[16];
-                    tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, r);
-                    tmem_ld_wait();
+        if (ok && fin) {
+            for (int cb = 0; cb < 2; ++cb) {
+                uint32_t r[16];
+                tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, r);
+                tmem_ld_wait();
 #pragma unroll
-                    for (int x = 0; x < 16; ++x) fin[cb * 16 + x] = __uint_as_float(r[x]);
-                }
+                for (int x4 = 0; x4 < 4; ++x4)
+                    *reinterpret_cast<float4*>(fin + cb * 16 + x4 * 4) =
+                        make_float4(__uint_as_float(r[x4 * 4 + 0]), __uint_as_float(r[x4 * 4 + 1]),
+                                    __uint_as_float(r[x4 * 4 + 2]), __uint_as_float(r[x4 * 4 + 3]));
             }
         }
     }
     tc_fence_before();
     __syncthreads();
+    OSDN_CLKS(16, blockIdx.x == 0 && tid == 0);
+#ifdef OSDN_PHASE_CLOCKS
+    __syncthreads();
+    if (blockIdx.x == 0 && tid < 32) g_clk[1][tid] = s_clk[tid];
+#endif
     if (warp == 0) tmem_dealloc(tb, 512);
 }
 
@@ -826,7 +1000,7 @@ struct TcChainBwdArgs {
     int* status;
 };
 
-constexpr uint32_t BS_DO = 0, BS_KT = 16384, BS_P = 32768, BS_QG = 40960, BS_WT = 57344;
+constexpr uint32_t BS_DO = 0, BS_KT = 16384, BS_WT = 32768, BS_P = 49152, BS_QG = 57344;
 constexpr uint32_t BSTAGE_BYTES = 73728;
 constexpr size_t CB_SMEM = 2 * BSTAGE_BYTES + 32768 + 16384 + 1024;
 
@@ -876,9 +1050,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         const size_t tile = (size_t)c * H + h;
         uint8_t* d = sStage + st * BSTAGE_BYTES;
         mbar_expect_tx(&bar_full[st], BSTAGE_BYTES);
-        bulk_load(d + BS_P, a.P + tile * 8192, 8192, &bar_full[st]);
-        bulk_load(d + BS_QG, a.Qg + tile * 16384, 16384, &bar_full[st]);
-        bulk_load(d + BS_WT, a.WT + tile * 16384, 16384, &bar_full[st]);
+        bulk_load(d + BS_WT, a.WT + tile * REC_BYTES, 40960, &bar_full[st]);   // W^T, P', Qg
         for (int hf = 0; hf < 2; ++hf) {
             tma_load_2d(d + BS_DO + hf * BOX, &tmDO, h * KD + hf * 64, tok0, &bar_full[st]);
             tma_load_2d(d + BS_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);

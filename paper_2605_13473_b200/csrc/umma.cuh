@@ -71,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
         const long long t0 = clock64();
         uint32_t it = 0;
         while (!(done = mbar_try_wait(bar, parity))) {
-            if ((++it & 63u) == 0u) {
+            if ((++it & 1023u) == 0u) {
                 if (clock64() - t0 > 4000000000ll) break;
                 if (status && *reinterpret_cast<volatile int*>(status) != 0) break;
             }
@@ -135,6 +135,17 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // ... and have completed
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Requests that only warm the L2 cache (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_2d(const void* tmap, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_prefetch(const void* gsrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gsrc), "r"(bytes) : "memory");
+}
 
 __device__ __forceinline__ void prefetch_tmap(const void* tmap)
 {
