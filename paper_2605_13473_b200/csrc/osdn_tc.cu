@@ -303,6 +303,11 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     const __grid_constant__ CUtensorMap tmKt, TcChunkArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
+#ifdef OSDN_PHASE_CLOCKS
+    __shared__ long long s_clk[32];
+    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
+    __syncthreads();
+#endif
     uint8_t* sm = align1024(smem_raw);
     uint8_t* sKQ = sm;                 // per k-half h: [K rows 0-63 | Q rows 64-127], 16 KB each
     uint8_t* sKt = sKQ + 32768;        // per k-half: 8 KB
@@ -336,7 +341,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(0, 0, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(0, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     const uint32_t tb = tmem_base;
 
@@ -354,7 +359,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         sG[tid] = acc;
     }
     bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
-    OSDN_CLK(0, 1, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(1, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sKQ + hf * 16384, len, tid, CL_THREADS);
@@ -364,7 +369,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         fence_proxy_async();
     }
     __syncthreads();
-    OSDN_CLK(0, 2, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(2, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- D1[128 x 64] = [K;Q] Ktil^T ---------------------------------------------------------
     if (tid == 0 && ok) {
@@ -378,7 +383,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mma_commit(&bar_mma1);
     }
     ok = ok && mbar_wait(&bar_mma1, 0, a.status, ERR_MMA1);
-    OSDN_CLK(0, 3, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(3, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
         const int L = warp * 32 + lane;
@@ -423,7 +428,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
     }
     __syncthreads();
-    OSDN_CLK(0, 4, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(4, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- T = (I + A)^-1, blocked --------------------------------------------------------------------
     ut_inverse_64(sA, sT, tid);
@@ -469,7 +474,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(0, 6, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(6, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- D2[128 x 64] = K^T Tbg^T  (W^T) -----------------------------------------------------
     if (tid == 0 && ok) {
@@ -481,7 +486,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mma_commit(&bar_mma2);
     }
     ok = ok && mbar_wait(&bar_mma2, 0, a.status, ERR_MMA2);
-    OSDN_CLK(0, 7, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(7, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
         const int k = warp * 32 + lane;
@@ -504,7 +509,11 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(0, 8, blockIdx.x == 5 && blockIdx.y == 0);
+    OSDN_CLKS(8, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
+#ifdef OSDN_PHASE_CLOCKS
+    __syncthreads();
+    if ((blockIdx.x == 5 && blockIdx.y == 0) && threadIdx.x < 32) g_clk[0][threadIdx.x] = s_clk[threadIdx.x];
+#endif
     if (warp == 0) tmem_dealloc(tb, 128);
 }
 
@@ -524,8 +533,6 @@ struct TcChainArgs {
     int* status;
 };
 
-constexpr int CF_THREADS = 256;
-constexpr int CF2_THREADS = 512;   // forward chain: 16 warps = 4 lane quadrants x 4 column groups
 constexpr uint32_t STAGE_BYTES = 16384 + 8192 + 8192 + 3 * 16384;   // WT, Tb, P, V, Q, Ktil = 81920
 constexpr uint32_t ST_TB = 0, ST_WT = 8192, ST_P = 24576, ST_V = 32768, ST_Q = 49152, ST_KT = 65536;
 constexpr size_t CF_SMEM = 2 * STAGE_BYTES + 32768 + 2 * 16384 + 1024;
@@ -1004,37 +1011,66 @@ constexpr uint32_t BS_DO = 0, BS_KT = 16384, BS_WT = 32768, BS_P = 49152, BS_QG 
 constexpr uint32_t BSTAGE_BYTES = 73728;
 constexpr size_t CB_SMEM = 2 * BSTAGE_BYTES + 32768 + 16384 + 1024;
 
-__global__ void __launch_bounds__(CF_THREADS, 1)
+// Warp roles as in the forward chain: 16 state warps (4 lane quadrants x 4 column groups), one warp
+// issuing the tensor-core work, one producer warp.  Barriers:
+//   full[st]   copies of a chunk have landed and its gate vectors are written          producer -> all
+//   empty[st]  every product reading the stage has finished                           tensor core -> producer
+//   s_ready    dS is in shared memory as a bf16 operand, the accumulator is decayed    state warps -> issuer
+//   a_done     both parts of ddU^T are complete                                        tensor core -> state warps
+//   a_ready    ddU^T is in shared memory as a bf16 operand                             state warps -> issuer
+//   s_done     the cotangent update of the chunk is complete                           tensor core -> state warps
+constexpr int CBK_EPI_WARPS = 16, CBK_MMA_WARP = 16, CBK_TMA_WARP = 17;
+constexpr int CBK_THREADS = 18 * 32;
+
+__global__ void __launch_bounds__(CBK_THREADS, 1)
 tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_constant__ CUtensorMap tmKt,
                     TcChainBwdArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
+#ifdef OSDN_PHASE_CLOCKS
+    __shared__ long long s_clk[32];
+    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
+    __syncthreads();
+#endif
     uint8_t* sm = align1024(smem_raw);
     uint8_t* sStage = sm;
     uint8_t* sdS = sm + 2 * BSTAGE_BYTES;       // dS as bf16, K-major, 2 k-halves x [128 x 128 B]
     uint8_t* sddU = sdS + 32768;                // ddU^T, K-major [v][i]
-    __shared__ uint64_t bar_full[2], bar_mma1, bar_mma2;
+    __shared__ uint64_t bar_full[2], bar_empty[2], bar_s_ready, bar_a_done, bar_a_ready, bar_s_done;
     __shared__ uint32_t tmem_base;
-    __shared__ float sRho[2][CH], sGC[2], sgraw[CH];
+    __shared__ float sRho[2][CH], sGC[2];
 
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
     const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int quad = warp & 3, colhalf = warp >> 2;
+    const int quad = warp & 3, colq = (warp >> 2) & 3;
     const int v = quad * 32 + lane;
-    float* dini = a.dinit_state ? a.dinit_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
-    const float* dfin = a.dfinal_state ? a.dfinal_state + (((size_t)s * H + h) * KD + v) * KD + colhalf * 64 : nullptr;
+    float* dini = a.dinit_state ? a.dinit_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
+    const float* dfin = a.dfinal_state ? a.dfinal_state + (((size_t)s * H + h) * KD + v) * KD + colq * 32 : nullptr;
     if (c1 <= c0) {
-        if (dini)
-            for (int x = 0; x < 64; ++x) dini[x] = dfin ? dfin[x] : 0.f;
+        if (dini && warp < CBK_EPI_WARPS)
+            for (int x = 0; x < 32; ++x) dini[x] = dfin ? dfin[x] : 0.f;
         return;
     }
+    const int nchunks = c1 - c0;
+    // step n of the reverse walk handles chunk c1 - 1 - n of the sequence
+    auto chunk_rel = [&](int n) { return nchunks - 1 - n; };
+    auto chunk_tok0 = [&](int n) { return seq_t0 + chunk_rel(n) * CH; };
+    auto chunk_len = [&](int n) { return min(CH, seq_len - chunk_rel(n) * CH); };
+    auto chunk_tile = [&](int n) { return (size_t)(c0 + chunk_rel(n)) * H + h; };
+    OSDN_CLKS(15, blockIdx.x == 0 && tid == 0);
+
     if (tid == 0) {
-        mbar_init(&bar_full[0], 1);
-        mbar_init(&bar_full[1], 1);
-        mbar_init(&bar_mma1, 1);
-        mbar_init(&bar_mma2, 1);
+        mbar_init(&bar_full[0], 2);
+        mbar_init(&bar_full[1], 2);
+        mbar_init(&bar_empty[0], 1);
+        mbar_init(&bar_empty[1], 1);
+        mbar_init(&bar_s_ready, CBK_EPI_WARPS);
+        mbar_init(&bar_a_done, 1);
+        mbar_init(&bar_a_ready, CBK_EPI_WARPS);
+        mbar_init(&bar_s_done, 1);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(&tmem_base, 256);
@@ -1042,192 +1078,229 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base;
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t tS = tb, tA1 = tb + 128, tA2 = tb + 192;
 
-    auto issue_loads = [&](int c, int st) {
-        const int tok0 = a.tab.chunk_tok0[c];
-        const size_t tile = (size_t)c * H + h;
-        uint8_t* d = sStage + st * BSTAGE_BYTES;
-        mbar_expect_tx(&bar_full[st], BSTAGE_BYTES);
-        bulk_load(d + BS_WT, a.WT + tile * REC_BYTES, 40960, &bar_full[st]);   // W^T, P', Qg
-        for (int hf = 0; hf < 2; ++hf) {
-            tma_load_2d(d + BS_DO + hf * BOX, &tmDO, h * KD + hf * 64, tok0, &bar_full[st]);
-            tma_load_2d(d + BS_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
-        }
-    };
-    auto gate_vectors = [&](int c, int st) {
-        if (tid < CH) {
-            const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
-            sgraw[tid] = tid < len ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
-        }
-        __syncthreads();
-        if (tid < CH) {
-            float G = 0.f, tot = 0.f;
-            for (int j = 0; j < CH; ++j) {
-                const float g = sgraw[j];
-                tot += g;
-                if (j <= tid) G += g;
+    if (warp == CBK_TMA_WARP) {
+        // ------------------------------------------------------------------ producer
+        bool ok = true;
+        auto load_gates = [&](int n, float& ga, float& gb) {
+            const int tok0 = chunk_tok0(n), len = chunk_len(n);
+            ga = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
+            gb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+        };
+        float ga, gb;
+        load_gates(0, ga, gb);
+        for (int n = 0; n < nchunks && ok; ++n) {
+            const int st = n & 1;
+            float ga_next = 0.f, gb_next = 0.f;
+            if (n + 1 < nchunks) load_gates(n + 1, ga_next, gb_next);
+            if (n >= 2) ok = mbar_wait(&bar_empty[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_TMA);
+            if (!ok) break;
+            if (lane == 0) {
+                const int tok0 = chunk_tok0(n);
+                uint8_t* d = sStage + st * BSTAGE_BYTES;
+                mbar_expect_tx(&bar_full[st], BSTAGE_BYTES);
+                bulk_load(d + BS_WT, a.WT + chunk_tile(n) * REC_BYTES, 40960, &bar_full[st]);   // W^T, P', Qg
+                for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + BS_DO + hf * BOX, &tmDO, h * KD + hf * 64, tok0, &bar_full[st]);
+                for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + BS_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
             }
-            sRho[st][tid] = __expf(tot - G);
-            if (tid == 0) sGC[st] = __expf(tot);
-        }
-    };
-
-    if (tid == 0) issue_loads(c1 - 1, 0);
-    for (int cb = 0; cb < 4; ++cb) {
-        uint32_t r[16];
-#pragma unroll
-        for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(dfin ? dfin[cb * 16 + x] : 0.f);
-        tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
-    }
-    tmem_st_wait();
-    gate_vectors(c1 - 1, 0);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-
-    bool ok = true;
-    for (int c = c1 - 1; c >= c0; --c) {
-        const int n = c1 - 1 - c, st = n & 1;
-        const int len = a.tab.chunk_len[c];
-        const size_t tile = (size_t)c * H + h;
-        uint8_t* d = sStage + st * BSTAGE_BYTES;
-        if (tid == 0 && c > c0) issue_loads(c - 1, st ^ 1);
-
-        // ---- E0: dS (cotangent at the chunk end) -> bf16 operand + saved copy; decay -----------
-        {
-            const float gC = sGC[st];
-            uint32_t rr[4][16];
-#pragma unroll
-            for (int cb = 0; cb < 4; ++cb) tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, rr[cb]);
-            tmem_ld_wait();
-#pragma unroll
-            for (int cb = 0; cb < 4; ++cb) {
-                uint32_t* r = rr[cb];
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
-                    w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
-                    w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
-                    w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
-                    const uint32_t off = sw128_chunk(v, cb * 2 + c2);
-                    *reinterpret_cast<uint4*>(sdS + colhalf * 16384 + off) = w;
+            __syncwarp();
+            warp_gate_vectors(ga, gb, lane, nullptr, sRho[st], &sGC[st]);
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&bar_full[st]);
+                // warm L2 two chunks ahead: the stage copies can only run one chunk ahead
+                if (n + 2 < nchunks) {
+                    const int t2 = chunk_tok0(n + 2);
+                    bulk_prefetch(a.WT + chunk_tile(n + 2) * REC_BYTES, 40960);
+                    for (int hf = 0; hf < 2; ++hf) {
+                        tma_prefetch_2d(&tmDO, h * KD + hf * 64, t2);
+                        tma_prefetch_2d(&tmKt, h * KD + hf * 64, t2);
+                    }
                 }
-#pragma unroll
-                for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
-                tmem_st16(tS + lane_addr + colhalf * 64 + cb * 16, r);
             }
-            tmem_st_wait();
+            ga = ga_next;
+            gb = gb_next;
         }
-    OSDN_CLK(2, 1, blockIdx.x == 0 && n == 3);
-        ok = ok && mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
-    OSDN_CLK(2, 2, blockIdx.x == 0 && n == 3);
-        if (len < CH) {
-            for (int hf = 0; hf < 2; ++hf) {
-                zero_tail_rows(d + BS_DO + hf * BOX, len, tid, CF_THREADS);
-                zero_tail_rows(d + BS_KT + hf * BOX, len, tid, CF_THREADS);
-            }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-    OSDN_CLK(2, 3, blockIdx.x == 0 && n == 3);
-
-        if (tid == 0 && ok) {
+    } else if (warp == CBK_MMA_WARP) {
+        // ------------------------------------------------------------------ tensor-core issuer
+        bool ok = true;
+        bool a1_issued = false;   // dO^T P' of the coming chunk is already in its accumulator
+        auto issue_a1 = [&](uint8_t* d) {   // acc1 = dO^T P'
+            const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN);
+            const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_P, 0);
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tA1, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k), idesc, k > 0);
+        };
+        for (int n = 0; n < nchunks && ok; ++n) {
+            const int st = n & 1;
+            const size_t tile = chunk_tile(n);
+            uint8_t* d = sStage + st * BSTAGE_BYTES;
+            if (!a1_issued) ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
+            ok = ok && mbar_wait(&bar_s_ready, n & 1, a.status, ERR_CHAIN_MMA1);
+            if (!ok) break;
             tc_fence_after();
-            bulk_store(a.dSn + tile * 32768, sdS, 32768);   // cotangent at the end of this chunk
-            bulk_commit();
-            {   // acc1 = dO^T P'
-                const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN);
-                const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_P, 0);
-                for (int k = 0; k < 4; ++k)
-                    mma_ss(tA1, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k), idesc, k > 0);
+            if (lane == 0) {
+                bulk_wait_read();   // the ddU^T image of the previous chunk has left shared memory
+                bulk_store(a.dSn + tile * 32768, sdS, 32768);   // cotangent at the end of this chunk
+                bulk_commit();
+                if (!a1_issued) issue_a1(d);
+                {   // acc2 = dS Ktil^T
+                    const uint32_t idesc = make_idesc(128, 64);
+                    for (int k = 0; k < 8; ++k)
+                        mma_ss(tA2, desc_advance(desc_kmajor(sdS + (k >> 2) * 16384), 32 * (k & 3)),
+                               desc_advance(desc_kmajor(d + BS_KT + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
+                }
+                mma_commit(&bar_a_done);
+                {   // dS += dO^T Qg (the accumulator has been decayed before s_ready)
+                    const uint32_t idesc = make_idesc(128, 128, IDESC_A_MN | IDESC_B_MN);
+                    const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_QG, BOX);
+                    for (int k = 0; k < 4; ++k)
+                        mma_ss(tS, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k), idesc, 1);
+                }
             }
-            {   // acc2 = dS Ktil^T
-                const uint32_t idesc = make_idesc(128, 64);
-                for (int k = 0; k < 8; ++k)
-                    mma_ss(tA2, desc_advance(desc_kmajor(sdS + (k >> 2) * 16384), 32 * (k & 3)),
-                           desc_advance(desc_kmajor(d + BS_KT + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
+            __syncwarp();
+            ok = mbar_wait(&bar_a_ready, n & 1, a.status, ERR_CHAIN_MMA2);
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0) {
+                // The dS image sent off above must have left shared memory before the update is
+                // released: its completion lets the state warps overwrite that image.
+                bulk_wait_read();
+                bulk_store(a.ddUT + tile * 16384, sddU, 16384);
+                bulk_commit();
+                {   // dS -= ddU^T W
+                    const uint32_t idesc = make_idesc(128, 128, IDESC_A_NEG);
+                    const uint64_t da0 = desc_kmajor(sddU), db0 = desc_kmajor(d + BS_WT);
+                    for (int k = 0; k < 4; ++k)
+                        mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, 1);
+                }
+                mma_commit(&bar_s_done);
+                mma_commit(&bar_empty[st]);
             }
-            mma_commit(&bar_mma1);
+            __syncwarp();
+            // the state-independent part of the next chunk's ddU^T, while the state warps convert dS
+            a1_issued = false;
+            if (n + 1 < nchunks && chunk_len(n + 1) == CH) {
+                ok = mbar_wait(&bar_full[st ^ 1], ((n + 1) >> 1) & 1, a.status, ERR_CHAIN_TMA);
+                if (!ok) break;
+                if (lane == 0) issue_a1(sStage + (st ^ 1) * BSTAGE_BYTES);
+                __syncwarp();
+                a1_issued = true;
+            }
         }
-        ok = ok && mbar_wait(&bar_mma1, n & 1, a.status, ERR_CHAIN_MMA1);
-    OSDN_CLK(2, 4, blockIdx.x == 0 && n == 3);
-        tc_fence_after();
-
-        // ---- E1: ddU^T = acc1 + rho_i acc2 ---------------------------------------------------
-        {
-            uint32_t ra[2][16], rb[2][16];
+        if (lane == 0) bulk_wait_all();
+    } else {
+        // ------------------------------------------------------------------ state warps
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        for (int cb = 0; cb < 2; ++cb) {
+            uint32_t r[16];
 #pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                tmem_ld16(tA1 + lane_addr + colhalf * 32 + cb * 16, ra[cb]);
-                tmem_ld16(tA2 + lane_addr + colhalf * 32 + cb * 16, rb[cb]);
+            for (int x4 = 0; x4 < 4; ++x4) {
+                const float4 f4 = dfin ? *reinterpret_cast<const float4*>(dfin + cb * 16 + x4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                r[x4 * 4 + 0] = __float_as_uint(f4.x);
+                r[x4 * 4 + 1] = __float_as_uint(f4.y);
+                r[x4 * 4 + 2] = __float_as_uint(f4.z);
+                r[x4 * 4 + 3] = __float_as_uint(f4.w);
             }
-            tmem_ld_wait();
+            tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
+        }
+        tmem_st_wait();
+
+        bool ok = true;
+        for (int n = 0; n < nchunks && ok; ++n) {
+            const int st = n & 1;
+            const int len = chunk_len(n);
+            uint8_t* d = sStage + st * BSTAGE_BYTES;
+            ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);   // gate vectors, tail rows
+            if (n > 0) ok = ok && mbar_wait(&bar_s_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2);
+            if (!ok) break;
+            tc_fence_after();
+            // ---- E0: dS (cotangent at the chunk end) -> bf16 operand; decay the accumulator
+            {
+                const float gC = sGC[st];
+                uint32_t rr[2][16];
 #pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                const uint32_t *r1 = ra[cb], *r2 = rb[cb];
+                for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    uint32_t* r = rr[cb];
+#pragma unroll
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
+                        w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
+                        w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
+                        w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
+                        *reinterpret_cast<uint4*>(sdS + (colq >> 1) * 16384 + sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2)) = w;
+                    }
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
+                    tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
+                }
+                tmem_st_wait();
+            }
+            if (len < CH) {
+                for (int hf = 0; hf < 2; ++hf) {
+                    zero_tail_rows(d + BS_DO + hf * BOX, len, tid, CBK_EPI_WARPS * 32);
+                    zero_tail_rows(d + BS_KT + hf * BOX, len, tid, CBK_EPI_WARPS * 32);
+                }
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_s_ready);
+
+            // ---- E1: ddU^T = acc1 + rho_i acc2 -> bf16 operand
+            float rho[16];
+#pragma unroll
+            for (int x = 0; x < 16; ++x) rho[x] = sRho[st][colq * 16 + x];
+            ok = mbar_wait(&bar_a_done, n & 1, a.status, ERR_CHAIN_MMA1);
+            if (!ok) break;
+            tc_fence_after();
+            {
+                uint32_t r1[16], r2[16];
+                tmem_ld16(tA1 + lane_addr + colq * 16, r1);
+                tmem_ld16(tA2 + lane_addr + colq * 16, r2);
+                tmem_ld_wait();
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     float f[8];
 #pragma unroll
                     for (int x = 0; x < 8; ++x)
-                        f[x] = __uint_as_float(r1[c2 * 8 + x]) +
-                               sRho[st][colhalf * 32 + cb * 16 + c2 * 8 + x] * __uint_as_float(r2[c2 * 8 + x]);
-                    const uint32_t off = sw128_chunk(v, colhalf * 4 + cb * 2 + c2);
-                    const uint4 w = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
-                                               pack_bf16(f[6], f[7]));
-                    *reinterpret_cast<uint4*>(sddU + off) = w;
+                        f[x] = __uint_as_float(r1[c2 * 8 + x]) + rho[c2 * 8 + x] * __uint_as_float(r2[c2 * 8 + x]);
+                    *reinterpret_cast<uint4*>(sddU + sw128_chunk(v, colq * 2 + c2)) =
+                        make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
                 }
             }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_a_ready);
         }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-    OSDN_CLK(2, 5, blockIdx.x == 0 && n == 3);
-
-        if (tid == 0 && ok) {
-            tc_fence_after();
-            bulk_store(a.ddUT + tile * 16384, sddU, 16384);
-            bulk_commit();
-            {   // dS += dO^T Qg
-                const uint32_t idesc = make_idesc(128, 128, IDESC_A_MN | IDESC_B_MN);
-                const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_QG, BOX);
-                for (int k = 0; k < 4; ++k)
-                    mma_ss(tS, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k), idesc, 1);
-            }
-            {   // dS -= ddU^T W
-                const uint32_t idesc = make_idesc(128, 128, IDESC_A_NEG);
-                const uint64_t da0 = desc_kmajor(sddU), db0 = desc_kmajor(d + BS_WT);
-                for (int k = 0; k < 4; ++k)
-                    mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, 1);
-            }
-            mma_commit(&bar_mma2);
-        }
-        if (c > c0) gate_vectors(c - 1, st ^ 1);
-        ok = ok && mbar_wait(&bar_mma2, n & 1, a.status, ERR_CHAIN_MMA2);
-    OSDN_CLK(2, 6, blockIdx.x == 0 && n == 3);
+        if (ok) ok = mbar_wait(&bar_s_done, (nchunks - 1) & 1, a.status, ERR_CHAIN_MMA2);
         tc_fence_after();
-        if (tid == 0) bulk_wait_read();
-        tc_fence_before();
-        __syncthreads();
-    OSDN_CLK(2, 7, blockIdx.x == 0 && n == 3);
-        tc_fence_after();
-    }
-    if (dini && ok) {
-        for (int cb = 0; cb < 4; ++cb) {
-            uint32_t r[16];
-            tmem_ld16(tS + lane_addr + colhalf * 64 + cb * 16, r);
-            tmem_ld_wait();
+        if (ok && dini) {
+            for (int cb = 0; cb < 2; ++cb) {
+                uint32_t r[16];
+                tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, r);
+                tmem_ld_wait();
 #pragma unroll
-            for (int x = 0; x < 16; ++x) dini[cb * 16 + x] = __uint_as_float(r[x]);
+                for (int x4 = 0; x4 < 4; ++x4)
+                    *reinterpret_cast<float4*>(dini + cb * 16 + x4 * 4) =
+                        make_float4(__uint_as_float(r[x4 * 4 + 0]), __uint_as_float(r[x4 * 4 + 1]),
+                                    __uint_as_float(r[x4 * 4 + 2]), __uint_as_float(r[x4 * 4 + 3]));
+            }
         }
     }
-    if (tid == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
+    OSDN_CLKS(16, blockIdx.x == 0 && tid == 0);
+#ifdef OSDN_PHASE_CLOCKS
+    __syncthreads();
+    if ((blockIdx.x == 0) && threadIdx.x < 32) g_clk[2][threadIdx.x] = s_clk[threadIdx.x];
+#endif
     if (warp == 0) tmem_dealloc(tb, 256);
 }
 
@@ -1271,6 +1344,11 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     TcChunkBwdArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
+#ifdef OSDN_PHASE_CLOCKS
+    __shared__ long long s_clk[32];
+    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
+    __syncthreads();
+#endif
     uint8_t* sm = align1024(smem_raw);
     float* sRaw = reinterpret_cast<float*>(sm + R_RAW);       // Gamma_ij <k_i, ktil_j>, j < i
     __shared__ uint64_t bar_tma, bar_mma[5];
@@ -1355,7 +1433,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     if (tid == 0) sRsum = 0.f;
     __syncthreads();
-    OSDN_CLK(3, 0, clk);
+    OSDN_CLKS(0, threadIdx.x == 0 && clk);
     // table entries and scalars of the next tile, one tile ahead
     const long tile_next = next_tile(tile_l + gridDim.x);
     int tok0_next = 0, len_next = 0;
@@ -1377,7 +1455,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sRho[tid] = __expf(tot - acc);
     }
     bool ok = mbar_wait(&bar_tma, ph, a.status, ERR_TMA);
-    OSDN_CLK(3, 1, clk);
+    OSDN_CLKS(1, threadIdx.x == 0 && clk);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sm + R_Q + hf * BOX, len, tid, CBW_THREADS);
@@ -1389,7 +1467,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fence_proxy_async();
     }
     __syncthreads();
-    OSDN_CLK(3, 2, clk);
+    OSDN_CLKS(2, threadIdx.x == 0 && clk);
 
     // tensor memory columns
     const uint32_t cRAW = 0, cDP = 64, cDQ1 = 128, cDKTR = 192, cDW = 256, cDTA = 320, cDTB = 384, cDKT = 448;
@@ -1449,7 +1527,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (lane == 0) sRed[warp] = part;
     }
     ok = ok && mbar_wait(&bar_mma[0], ph, a.status, ERR_MMA1);
-    OSDN_CLK(3, 3, clk);
+    OSDN_CLKS(3, threadIdx.x == 0 && clk);
     tc_fence_after();
     __syncthreads();   // every thread is done reading S / dS before their space is reused
     // epilogue A
@@ -1496,7 +1574,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 4, clk);
+    OSDN_CLKS(4, threadIdx.x == 0 && clk);
 
     // ---- phase B -------------------------------------------------------------------------------
     if (tid == 0 && ok) {
@@ -1538,7 +1616,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[1]);
     }
     ok = ok && mbar_wait(&bar_mma[1], ph, a.status, ERR_MMA2);
-    OSDN_CLK(3, 5, clk);
+    OSDN_CLKS(5, threadIdx.x == 0 && clk);
     tc_fence_after();
     {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j]
         const int i = row64;
@@ -1566,7 +1644,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 6, clk);
+    OSDN_CLKS(6, threadIdx.x == 0 && clk);
 
     // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] -----------------------------------------------
     if (tid == 0 && ok) {
@@ -1578,7 +1656,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[2]);
     }
     ok = ok && mbar_wait(&bar_mma[2], ph, a.status, ERR_MMA2);
-    OSDN_CLK(3, 7, clk);
+    OSDN_CLKS(7, threadIdx.x == 0 && clk);
     tc_fence_after();
     {
         const int i = row64;
@@ -1601,7 +1679,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 8, clk);
+    OSDN_CLKS(8, threadIdx.x == 0 && clk);
 
     // ---- phase D: Z[a][b] = sum_c Y[a][c] T[b][c] ; dA = -strictLower(Z) --------------------------
     if (tid == 0 && ok) {
@@ -1612,7 +1690,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[3]);
     }
     ok = ok && mbar_wait(&bar_mma[3], ph, a.status, ERR_MMA2);
-    OSDN_CLK(3, 9, clk);
+    OSDN_CLKS(9, threadIdx.x == 0 && clk);
     tc_fence_after();
     {
         const int i = row64;
@@ -1644,7 +1722,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLK(3, 10, clk);
+    OSDN_CLKS(10, threadIdx.x == 0 && clk);
 
     // ---- phase E: dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T -----------------------------------------
     if (tid == 0 && ok) {
@@ -1660,7 +1738,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[4]);
     }
     ok = ok && mbar_wait(&bar_mma[4], ph, a.status, ERR_MMA2);
-    OSDN_CLK(3, 11, clk);
+    OSDN_CLKS(11, threadIdx.x == 0 && clk);
     tc_fence_after();
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
@@ -1804,7 +1882,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     __syncthreads();   // every copy-out read of the staging tiles is done
     if (tid == 0 && tile_next < a.ntiles) issue_second(tile_next, tok0_next);
-    OSDN_CLK(3, 12, clk);
+    OSDN_CLKS(12, threadIdx.x == 0 && clk);
     if (tid == 0) {
         float tot = 0.f;
         for (int w = 0; w < CBW_THREADS / 32; ++w) tot += sRed[w];
@@ -1823,7 +1901,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    OSDN_CLK(3, 13, clk);
+    OSDN_CLKS(13, threadIdx.x == 0 && clk);
     ph ^= 1u;
     tile_l = tile_next;
     tok0 = tok0_next;
@@ -1834,6 +1912,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (tid == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
+#ifdef OSDN_PHASE_CLOCKS
+    __syncthreads();
+    if (blockIdx.x == 1603 % gridDim.x && threadIdx.x < 32) g_clk[3][threadIdx.x] = s_clk[threadIdx.x];
+#endif
     if (warp == 0) tmem_dealloc(tb, 512);
 }
 
@@ -1935,7 +2017,7 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
         ch.status = status;
         if (!set_smem(tc_chain_bwd_kernel, CB_SMEM)) return -1;
         stage_mark(st, "tc_chain_bwd");
-        tc_chain_bwd_kernel<<<S * H, CF_THREADS, CB_SMEM, st>>>(tmDO, tmKt, ch);
+        tc_chain_bwd_kernel<<<S * H, CBK_THREADS, CB_SMEM, st>>>(tmDO, tmKt, ch);
         ++launches;
     }
     {
