@@ -432,8 +432,8 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
     // ---- T = (I + A)^-1, blocked --------------------------------------------------------------------
     ut_inverse_64(sA, sT, tid);
-    // gated, scaled queries for the backward state chain: Qg = scale gamma_i Q (same image layout as Q)
-    if (a.save) {
+    // gated, scaled queries for both state chains: Qg = scale gamma_i Q (same image layout as Q)
+    {
         for (int e = tid; e < 2 * CH * 8; e += CL_THREADS) {
             const int hf = e >> 9, i = (e >> 3) & 63, ch = e & 7;
             const uint32_t off = sw128_chunk(i, ch);
@@ -533,8 +533,8 @@ struct TcChainArgs {
     int* status;
 };
 
-constexpr uint32_t STAGE_BYTES = 16384 + 8192 + 8192 + 3 * 16384;   // WT, Tb, P, V, Q, Ktil = 81920
-constexpr uint32_t ST_TB = 0, ST_WT = 8192, ST_P = 24576, ST_V = 32768, ST_Q = 49152, ST_KT = 65536;
+constexpr uint32_t STAGE_BYTES = 8192 + 16384 + 8192 + 3 * 16384;   // Tb, WT, P, Qg, V, Ktil = 81920
+constexpr uint32_t ST_TB = 0, ST_WT = 8192, ST_P = 24576, ST_QG = 32768, ST_V = 49152, ST_KT = 65536;
 constexpr size_t CF_SMEM = 2 * STAGE_BYTES + 32768 + 2 * 16384 + 1024;
 
 // In-chunk gate prefix by one warp: lane l holds g_l and g_{l+32}.  Writes gamma_i = exp(G_i),
@@ -575,8 +575,7 @@ constexpr int CFW_OUT_WARP0 = 16, CFW_MMA_WARP = 20, CFW_TMA_WARP = 21;
 constexpr int CFW_THREADS = 22 * 32;
 
 __global__ void __launch_bounds__(CFW_THREADS, 1)
-tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
-                    const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
+tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* sm = align1024(smem_raw);
@@ -588,7 +587,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     __shared__ uint64_t bar_o_done[2], bar_o_free[2];
     __shared__ uint32_t tmem_base;
     __shared__ float sRho[2][CH], sGC[2];              // slot = chunk % 2
-    __shared__ float sOutGam[CFW_OUT_WARPS][CH];       // scale * gamma_i, private to each output warp
 #ifdef OSDN_PHASE_CLOCKS
     __shared__ long long s_clk[32];
     if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
@@ -634,7 +632,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base;
-    const uint32_t tS = tb, tDU = tb + 128, tO1 = tb + 192, tO2 = tb + 320;   // O1, O2: two buffers of 64
+    const uint32_t tS = tb, tDU = tb + 128, tO = tb + 192;   // O^T: two buffers of 64 columns
 
     if (warp == CFW_TMA_WARP) {
         // ------------------------------------------------------------------ producer
@@ -659,9 +657,8 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                 const size_t tile = (size_t)(c0 + n) * H + h;
                 uint8_t* d = sStage + st * STAGE_BYTES;
                 mbar_expect_tx(&bar_full[st], STAGE_BYTES);
-                bulk_load(d + ST_TB, a.Tb + tile * REC_BYTES, 32768, &bar_full[st]);   // Tb, W^T, P'
+                bulk_load(d + ST_TB, a.Tb + tile * REC_BYTES, REC_BYTES, &bar_full[st]);   // Tb, W^T, P', Qg
                 for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + ST_V + hf * BOX, &tmV, h * KD + hf * 64, tok0, &bar_full[st]);
-                for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + ST_Q + hf * BOX, &tmQ, h * KD + hf * 64, tok0, &bar_full[st]);
                 for (int hf = 0; hf < 2; ++hf) tma_load_2d(d + ST_KT + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_full[st]);
             }
             __syncwarp();
@@ -713,11 +710,11 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             if (n >= 2) OSDN_ACC(2, ok = mbar_wait(&bar_o_free[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_MMA2));
             if (!ok) break;
             tc_fence_after();
-            if (lane == 0) {   // O1^T = S Q^T
+            if (lane == 0) {   // O^T = S Qg^T
                 const uint32_t idesc = make_idesc(128, 64);
                 for (int k = 0; k < 8; ++k)
-                    mma_ss(tO1 + st * 64, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
-                           desc_advance(desc_kmajor(d + ST_Q + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
+                    mma_ss(tO + st * 64, desc_advance(desc_kmajor(sS + (k >> 2) * 16384), 32 * (k & 3)),
+                           desc_advance(desc_kmajor(d + ST_QG + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
             }
             __syncwarp();
             OSDN_ACC(3, ok = mbar_wait(&bar_du_ready, n & 1, a.status, ERR_CHAIN_MMA2));
@@ -740,11 +737,11 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                 }
                 mma_commit(&bar_s_done);
                 OSDN_CLKS(13, blockIdx.x == 0 && n == 10);
-                {   // O2^T = dU^T P'^T
+                {   // O^T += dU^T P'^T
                     const uint32_t idesc = make_idesc(128, 64);
                     const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
                     for (int k = 0; k < 4; ++k)
-                        mma_ss(tO2 + st * 64, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, k > 0);
+                        mma_ss(tO + st * 64, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), idesc, 1);
                 }
                 mma_commit(&bar_o_done[st]);
                 mma_commit(&bar_empty[st]);
@@ -765,67 +762,48 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         OSDN_ACC_DUMP(0, 5, blockIdx.x == 0 && lane == 0);
     } else if (warp >= CFW_OUT_WARP0) {
         // ------------------------------------------------------------------ output warps
-        // o_i = scale gamma_i (S q_i) + (P' dU)_i : lane = feature, 16 token columns per load
+        // o_i = (S Qg^T + dU^T P'^T)_i is complete in the accumulator: lane = feature, 16 token columns
+        // per load.  Results leave as 16-byte stores: three shuffle rounds turn "lane = feature, 16
+        // tokens" into "lane = 8 consecutive features of 2 tokens" (lane bit 0 picks the token half,
+        // bits 1-2 the token pair inside it, bits 3-4 the feature octet).
         const int ow = warp - CFW_OUT_WARP0;   // == lane quadrant
         const uint32_t lane_addr = (uint32_t)(ow * 32) << 16;
-        float* og = sOutGam[ow];
+        const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4;
+        const int tsub = (b0 ? 8 : 0) + ((lane >> 1) & 3) * 2;
         bool ok = true;
         OSDN_ACC_DECL;
         for (int n = 0; n < nchunks && ok; ++n) {
             const int st = n & 1;
             const int tok0 = chunk_tok0(n), len = chunk_len(n);
-            {   // in-chunk gate prefix, kept private to this warp
-                float sa = lane < len ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
-                float sb = lane + 32 < len ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const float ua = __shfl_up_sync(0xffffffffu, sa, o), ub = __shfl_up_sync(0xffffffffu, sb, o);
-                    if (lane >= o) { sa += ua; sb += ub; }
-                }
-                sb += __shfl_sync(0xffffffffu, sa, 31);
-                __syncwarp();   // the previous chunk's factors are no longer read
-                og[lane] = a.scale * __expf(sa);
-                og[lane + 32] = a.scale * __expf(sb);
-                __syncwarp();
-            }
-            // Warm L2 with the operands of chunk n + 2 (the stage copies can only run one chunk ahead);
-            // each output warp asks for one operand.
+            // Warm L2 with the operands of chunk n + 2 (the stage copies can only run one chunk ahead).
             if (lane == 0 && n + 2 < nchunks) {
                 const int t2 = chunk_tok0(n + 2);
-                if (ow == 0) bulk_prefetch(a.Tb + ((size_t)(c0 + n + 2) * H + h) * REC_BYTES, 32768);
-                const CUtensorMap* tm = ow == 1 ? &tmV : ow == 2 ? &tmQ : &tmKt;
-                if (ow > 0)
-                    for (int hf = 0; hf < 2; ++hf) tma_prefetch_2d(tm, h * KD + hf * 64, t2);
+                if (ow == 0) bulk_prefetch(a.Tb + ((size_t)(c0 + n + 2) * H + h) * REC_BYTES, REC_BYTES);
+                if (ow == 1)
+                    for (int hf = 0; hf < 2; ++hf) tma_prefetch_2d(&tmV, h * KD + hf * 64, t2);
+                if (ow == 2)
+                    for (int hf = 0; hf < 2; ++hf) tma_prefetch_2d(&tmKt, h * KD + hf * 64, t2);
             }
             OSDN_ACC(0, ok = mbar_wait(&bar_o_done[st], (n >> 1) & 1, a.status, ERR_CHAIN_MMA2));
             if (!ok) break;
             tc_fence_after();
-            // Results leave as 16-byte stores: three shuffle rounds turn "lane = feature, 16 tokens" into
-            // "lane = 8 consecutive features of 2 tokens" (lane bit 0 picks the token half, bits 1-2 the
-            // token pair inside it, bits 3-4 the feature octet).
-            const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4;
-            const int tsub = (b0 ? 8 : 0) + ((lane >> 1) & 3) * 2;
             __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + ow * 32 + (lane >> 3) * 8;
 #pragma unroll
             for (int cg = 0; cg < 4; ++cg) {
-                uint32_t ra[16], rb[16];
-                tmem_ld16(tO1 + st * 64 + lane_addr + cg * 16, ra);
-                tmem_ld16(tO2 + st * 64 + lane_addr + cg * 16, rb);
+                uint32_t ra[16];
+                tmem_ld16(tO + st * 64 + lane_addr + cg * 16, ra);
                 tmem_ld_wait();
-                if (cg == 3) {   // everything is in registers: the buffers may be overwritten
+                if (cg == 3) {   // everything is in registers: the buffer may be overwritten
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bar_o_free[st]);
                 }
-                float o[16];
-#pragma unroll
-                for (int x = 0; x < 16; ++x)
-                    o[x] = og[cg * 16 + x] * __uint_as_float(ra[x]) + __uint_as_float(rb[x]);
                 uint32_t w[8];    // feature pair (lane >> 1), token (b0 ? 8 : 0) + i
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const float recv = __shfl_xor_sync(0xffffffffu, b0 ? o[i] : o[i + 8], 1);
-                    w[i] = b0 ? pack_bf16(recv, o[i + 8]) : pack_bf16(o[i], recv);
+                    const float lo = __uint_as_float(ra[i]), hi = __uint_as_float(ra[i + 8]);
+                    const float recv = __shfl_xor_sync(0xffffffffu, b0 ? lo : hi, 1);
+                    w[i] = b0 ? pack_bf16(recv, hi) : pack_bf16(lo, recv);
                 }
                 uint32_t wa[2][2][2];   // [token-pair bit 1][token parity][feature pair 0 / 1]
 #pragma unroll
@@ -923,7 +901,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             if (len < CH) {
                 for (int hf = 0; hf < 2; ++hf) {
                     zero_tail_rows(d + ST_V + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
-                    zero_tail_rows(d + ST_Q + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
                     zero_tail_rows(d + ST_KT + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
                 }
             }
@@ -1984,7 +1961,7 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
         ch.status = status;
         if (!set_smem(tc_chain_fwd_kernel, CF_SMEM)) return -1;
         stage_mark(st, "tc_chain_fwd");
-        tc_chain_fwd_kernel<<<S * H, CFW_THREADS, CF_SMEM, st>>>(tmV, tmQ, tmKt, ch);
+        tc_chain_fwd_kernel<<<S * H, CFW_THREADS, CF_SMEM, st>>>(tmV, tmKt, ch);
         ++launches;
     }
     stage_end(st);
