@@ -173,12 +173,7 @@ __device__ __forceinline__ void zero_tail_rows(uint8_t* box, int len, int tid, i
 }
 
 // ---------------------------------------------------------------------------------------------
-// T = (I + A)^-1 for a 64 x 64 strictly lower triangular A (fp32, shared memory, row stride LC),
-// by 16 x 16 blocks: the four diagonal blocks by forward substitution with a column per thread in
-// registers, then block by block away from the diagonal,
-//     T_bc = -T_bb sum_{m=c}^{b-1} A_bm T_mc            (b > c).
-// The inner sums are parked in the unused upper triangle of A (block (c, b)).  Called by all 128
-// threads of the CTA; ends with a barrier.
+// fp32 scratch rows of the chunk-local backward: odd stride, one row per lane without bank conflicts
 // ---------------------------------------------------------------------------------------------
 constexpr int LC = CH + 1;
 
@@ -199,15 +194,27 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], 
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 
+// ---------------------------------------------------------------------------------------------
+// T = (I + A)^-1 for a 64 x 64 strictly lower triangular A, in place (fp32, shared memory, row
+// stride LCF), by 16 x 16 blocks: the four diagonal blocks by forward substitution with a column
+// per thread in registers, then block row by block row,
+//     T_bc = -T_bb sum_{m=c}^{b-1} A_bm T_mc            (c < b),
+// where row b of A is still untouched and the rows above already hold T.  The inner sums are
+// parked in the upper triangle (block (c, b)), so on return only entries with j <= i are meaningful.
+// Called by all threads of the CTA (at least 96); ends with a barrier.
+// ---------------------------------------------------------------------------------------------
+constexpr int LCF = CH + 4;   // stride = 4 mod 32 words: conflict-free 16-byte row stores and A fragments
+
 // acc (16 x 16, two 16 x 8 fragments) += A (16 x 16) * B (16 x 16), fp32 in shared memory with row
-// stride LC, evaluated as three TF32 products (hi*hi + hi*lo + lo*hi) to keep fp32 accuracy.  One warp.
-__device__ __forceinline__ void block16_mma(float (&acc)[2][4], const float* A, const float* B, int lane)
+// stride LD, evaluated as three TF32 products (hi*hi + hi*lo + lo*hi) to keep fp32 accuracy.  One warp.
+template <int LD>
+__device__ __forceinline__ void block16_mma_ld(float (&acc)[2][4], const float* A, const float* B, int lane)
 {
     const int g = lane >> 2, t = lane & 3;
 #pragma unroll
     for (int kt = 0; kt < 2; ++kt) {
-        float af[4] = {A[g * LC + 8 * kt + t], A[(g + 8) * LC + 8 * kt + t], A[g * LC + 8 * kt + t + 4],
-                       A[(g + 8) * LC + 8 * kt + t + 4]};
+        float af[4] = {A[g * LD + 8 * kt + t], A[(g + 8) * LD + 8 * kt + t], A[g * LD + 8 * kt + t + 4],
+                       A[(g + 8) * LD + 8 * kt + t + 4]};
         uint32_t ah[4], al[4];
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -216,7 +223,7 @@ __device__ __forceinline__ void block16_mma(float (&acc)[2][4], const float* A, 
         }
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
-            float bf[2] = {B[(8 * kt + t) * LC + 8 * nt + g], B[(8 * kt + t + 4) * LC + 8 * nt + g]};
+            float bf[2] = {B[(8 * kt + t) * LD + 8 * nt + g], B[(8 * kt + t + 4) * LD + 8 * nt + g]};
             uint32_t bh[2], bl[2];
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
@@ -231,53 +238,55 @@ __device__ __forceinline__ void block16_mma(float (&acc)[2][4], const float* A, 
 }
 
 // store a 16 x 16 accumulator (optionally negated) to shared memory
-__device__ __forceinline__ void block16_store(float* C, const float (&acc)[2][4], float sign, int lane)
+template <int LD>
+__device__ __forceinline__ void block16_store_ld(float* C, const float (&acc)[2][4], float sign, int lane)
 {
     const int g = lane >> 2, t = lane & 3;
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt) {
-        C[g * LC + 8 * nt + 2 * t] = sign * acc[nt][0];
-        C[g * LC + 8 * nt + 2 * t + 1] = sign * acc[nt][1];
-        C[(g + 8) * LC + 8 * nt + 2 * t] = sign * acc[nt][2];
-        C[(g + 8) * LC + 8 * nt + 2 * t + 1] = sign * acc[nt][3];
+        *reinterpret_cast<float2*>(C + g * LD + 8 * nt + 2 * t) = make_float2(sign * acc[nt][0], sign * acc[nt][1]);
+        *reinterpret_cast<float2*>(C + (g + 8) * LD + 8 * nt + 2 * t) = make_float2(sign * acc[nt][2], sign * acc[nt][3]);
     }
 }
 
-__device__ __forceinline__ void ut_inverse_64(float* sA, float* sT, int tid)
+__device__ __forceinline__ void ut_inverse_64_inplace(float* sA, int tid)
 {
     const int warp = tid >> 5, lane = tid & 31;
-    for (int e = tid; e < CH * CH; e += 128) sT[(e >> 6) * LC + (e & 63)] = 0.f;
-    __syncthreads();
-    if (tid < CH) {
-        const int b = tid >> 4, col = tid & 15;
-        const float* Ab = sA + (16 * b) * LC + 16 * b;
+    {
         float x[16];
+        const int b = (tid >> 4) & 3, col = tid & 15;
+        float* Ab = sA + (16 * b) * LCF + 16 * b;
+        if (tid < CH) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) x[i] = i == col ? 1.f : 0.f;
+            for (int i = 0; i < 16; ++i) x[i] = i == col ? 1.f : 0.f;
 #pragma unroll
-        for (int j = 0; j < 15; ++j) {
+            for (int j = 0; j < 15; ++j) {
 #pragma unroll
-            for (int i = j + 1; i < 16; ++i) x[i] = fmaf(-Ab[i * LC + j], x[j], x[i]);
+                for (int i = j + 1; i < 16; ++i) x[i] = fmaf(-Ab[i * LCF + j], x[j], x[i]);
+            }
         }
+        __syncthreads();   // every column has read the block before anyone overwrites it
+        if (tid < CH) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) sT[(16 * b + i) * LC + 16 * b + col] = x[i];
+            for (int i = 0; i < 16; ++i) Ab[i * LCF + col] = x[i];
+        }
     }
     __syncthreads();
-    for (int d = 1; d < 4; ++d) {
-        // warp p handles block (b, c) = (d + p, p): X = sum_m A_bm T_mc, parked in the upper triangle
-        // of A (block (c, b)), then T_bc = -T_bb X
-        if (warp < 4 - d) {
-            const int b = d + warp, c = warp;
+    for (int b = 1; b < 4; ++b) {
+        // warp c < b: X = sum_m A_bm T_mc, parked in block (c, b); then T_bc = -T_bb X
+        float acc2[2][4] = {};
+        if (warp < b) {
+            const int c = warp;
             float acc[2][4] = {};
             for (int m = c; m < b; ++m)
-                block16_mma(acc, sA + (16 * b) * LC + 16 * m, sT + (16 * m) * LC + 16 * c, lane);
-            float* X = sA + (16 * c) * LC + 16 * b;
-            block16_store(X, acc, 1.f, lane);
+                block16_mma_ld<LCF>(acc, sA + (16 * b) * LCF + 16 * m, sA + (16 * m) * LCF + 16 * c, lane);
+            float* X = sA + (16 * c) * LCF + 16 * b;
+            block16_store_ld<LCF>(X, acc, 1.f, lane);
             __syncwarp();
-            float acc2[2][4] = {};
-            block16_mma(acc2, sT + (16 * b) * LC + 16 * b, X, lane);
-            block16_store(sT + (16 * b) * LC + 16 * c, acc2, -1.f, lane);
+            block16_mma_ld<LCF>(acc2, sA + (16 * b) * LCF + 16 * b, X, lane);
         }
+        __syncthreads();   // row b of A has been read by every warp that needs it
+        if (warp < b) block16_store_ld<LCF>(sA + (16 * b) * LCF + 16 * warp, acc2, -1.f, lane);
         __syncthreads();
     }
 }
@@ -295,10 +304,12 @@ struct TcChunkArgs {
     int* status;
 };
 
-constexpr int CL_THREADS = 128;
-constexpr size_t CL_SMEM = 32768 + 16384 + 8192 + CH * LC * 4 + 1024;
+// 8 warps = 4 lane quadrants x 2 column halves; 50 KB of shared memory and 128 tensor-memory columns,
+// so that four CTAs share an SM and hide each other's waits.
+constexpr int CL_THREADS = 256;
+constexpr size_t CL_SMEM = 32768 + CH * LCF * 4 + 1024;
 
-__global__ void __launch_bounds__(CL_THREADS)
+__global__ void __launch_bounds__(CL_THREADS, 4)
 tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
                     const __grid_constant__ CUtensorMap tmKt, TcChunkArgs a)
 {
@@ -311,14 +322,13 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     uint8_t* sm = align1024(smem_raw);
     uint8_t* sKQ = sm;                 // per k-half h: [K rows 0-63 | Q rows 64-127], 16 KB each
     uint8_t* sKt = sKQ + 32768;        // per k-half: 8 KB
-    uint8_t* sTb = sKt + 16384;        // T diag(beta gamma), K-major [i][j]
-    // A (fp32) takes over the space of Ktil once the first product has consumed it (and the first
-    // 256 bytes of the Tbg image, which is written only after the inversion)
+    // A, then T (fp32, in place) take over the space of Ktil once the first product has consumed it;
+    // the T diag(beta gamma) operand image takes over the first Q box once Qg has been written.
     float* sA = reinterpret_cast<float*>(sKt);
-    float* sT = reinterpret_cast<float*>(sTb + 8192);
+    uint8_t* sTb = sKQ + BOX;          // K-major [i][j]
     __shared__ uint64_t bar_tma, bar_mma1, bar_mma2;
     __shared__ uint32_t tmem_base;
-    __shared__ float sG[CH], sBeta[CH], sg[CH];
+    __shared__ __align__(16) float sG[CH], sBeta[CH];
 
     const int c = blockIdx.x, h = blockIdx.y, H = a.H;
     const int len = a.tab.chunk_len[c];
@@ -326,26 +336,13 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int tok0 = a.tab.chunk_tok0[c];
     const size_t tile = (size_t)c * H + h;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int quad = warp & 3, half = warp >> 2;
 
     if (tid == 0) {
         mbar_init(&bar_tma, 1);
         mbar_init(&bar_mma1, 1);
         mbar_init(&bar_mma2, 1);
         fence_mbar_init();
-    }
-    if (warp == 0) tmem_alloc(&tmem_base, 128);
-    if (tid < CH) {
-        const bool in = tid < len;
-        sg[tid] = in ? a.gate[(size_t)(tok0 + tid) * H + h] : 0.f;
-        sBeta[tid] = in ? a.beta[(size_t)(tok0 + tid) * H + h] : 0.f;
-    }
-    tc_fence_before();
-    __syncthreads();
-    OSDN_CLKS(0, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
-    tc_fence_after();
-    const uint32_t tb = tmem_base;
-
-    if (tid == 0) {
         mbar_expect_tx(&bar_tma, 6 * BOX);
         for (int hf = 0; hf < 2; ++hf) {
             tma_load_2d(sKQ + hf * 16384, &tmK, h * KD + hf * 64, tok0, &bar_tma);
@@ -353,11 +350,28 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             tma_load_2d(sKt + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_tma);
         }
     }
-    if (tid < CH) {
-        float acc = 0.f;
-        for (int j = 0; j <= tid; ++j) acc += sg[j];
-        sG[tid] = acc;
+    if (warp == 1) tmem_alloc(&tmem_base, 128);
+    if (warp == 2) {   // per-token scalars and the in-chunk gate prefix G_i
+        const bool in0 = lane < len, in1 = lane + 32 < len;
+        float sa = in0 ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
+        float sb = in1 ? a.gate[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+        sBeta[lane] = in0 ? a.beta[(size_t)(tok0 + lane) * H + h] : 0.f;
+        sBeta[lane + 32] = in1 ? a.beta[(size_t)(tok0 + lane + 32) * H + h] : 0.f;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float ua = __shfl_up_sync(0xffffffffu, sa, o), ub = __shfl_up_sync(0xffffffffu, sb, o);
+            if (lane >= o) { sa += ua; sb += ub; }
+        }
+        sb += __shfl_sync(0xffffffffu, sa, 31);
+        sG[lane] = sa;
+        sG[lane + 32] = sb;
     }
+    tc_fence_before();
+    __syncthreads();
+    OSDN_CLKS(0, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+
     bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
     OSDN_CLKS(1, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     if (len < CH) {
@@ -367,13 +381,12 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             zero_tail_rows(sKt + hf * BOX, len, tid, CL_THREADS);
         }
         fence_proxy_async();
+        __syncthreads();
     }
-    __syncthreads();
     OSDN_CLKS(2, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- D1[128 x 64] = [K;Q] Ktil^T ---------------------------------------------------------
     if (tid == 0 && ok) {
-        tc_fence_after();
         const uint32_t idesc = make_idesc(128, 64);
         for (int s = 0; s < 8; ++s) {
             const uint64_t da = desc_advance(desc_kmajor(sKQ + (s >> 2) * 16384), 32 * (s & 3));
@@ -382,38 +395,73 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
         mma_commit(&bar_mma1);
     }
+    // gated, scaled queries for both state chains, while the product runs: Qg = scale gamma_i Q
+    // (same image layout as Q)
+    for (int e = tid; e < 2 * CH * 8; e += CL_THREADS) {
+        const int hf = e >> 9, i = (e >> 3) & 63, ch = e & 7;
+        const uint32_t off = sw128_chunk(i, ch);
+        const uint4 w = *reinterpret_cast<const uint4*>(sKQ + hf * 16384 + BOX + off);
+        const float f = a.scale * __expf(sG[i]);
+        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&w);
+        uint32_t o[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const float2 v = __bfloat1622float2(p2[x]);
+            o[x] = pack_bf16(v.x * f, v.y * f);
+        }
+        *reinterpret_cast<uint4*>(a.Qg + tile * REC_BYTES + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
     ok = ok && mbar_wait(&bar_mma1, 0, a.status, ERR_MMA1);
     OSDN_CLKS(3, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
-        const int L = warp * 32 + lane;
-        const uint32_t taddr = tb + ((uint32_t)(warp * 32) << 16);
-        if (L < CH) {
+        const int L = quad * 32 + lane;
+        const uint32_t taddr = tb + ((uint32_t)(quad * 32) << 16) + half * 32;
+        if (L < CH) {   // A_ij = beta_i Gamma_ij <k_i, ktil_j>, j < i
             const int i = L;
             const float bi = sBeta[i], Gi = sG[i];
-            for (int cb = 0; cb < 4; ++cb) {
-                uint32_t r[16];
-                tmem_ld16(taddr + cb * 16, r);
-                tmem_ld_wait();
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const int j = cb * 16 + x;
-                    sA[i * LC + j] = j < i ? bi * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+            for (int cb = 0; cb < 2; ++cb) {
+                const int j0 = half * 32 + cb * 16;
+                float av[16];
+                if (j0 <= (quad & 1) * 32 + 31) {   // warp-uniform: some row of this warp reaches the block
+                    uint32_t r[16];
+                    tmem_ld16(taddr + cb * 16, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        const int j = j0 + x;
+                        av[x] = j < i ? bi * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+                    }
+                } else {
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) av[x] = 0.f;
                 }
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    *reinterpret_cast<float4*>(sA + i * LCF + j0 + q4 * 4) =
+                        make_float4(av[q4 * 4 + 0], av[q4 * 4 + 1], av[q4 * 4 + 2], av[q4 * 4 + 3]);
             }
-        } else {
+        } else {        // P'_ij = scale Gamma_ij <q_i, ktil_j>, j <= i
             const int i = L - CH;
             const float Gi = sG[i];
             uint8_t* Pg = a.P + tile * REC_BYTES;
-            for (int cb = 0; cb < 4; ++cb) {
-                uint32_t r[16];
-                tmem_ld16(taddr + cb * 16, r);
-                tmem_ld_wait();
-                float pv[16];
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const int j = cb * 16 + x;
-                    pv[x] = j <= i ? a.scale * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+            for (int cb = 0; cb < 2; ++cb) {
+                const int j0 = half * 32 + cb * 16;
+                float pv[16];
+                if (j0 <= (quad & 1) * 32 + 31) {   // warp-uniform
+                    uint32_t r[16];
+                    tmem_ld16(taddr + cb * 16, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        const int j = j0 + x;
+                        pv[x] = j <= i ? a.scale * __expf(Gi - sG[j]) * __uint_as_float(r[x]) : 0.f;
+                    }
+                } else {
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) pv[x] = 0.f;
                 }
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
@@ -422,7 +470,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     w.y = pack_bf16(pv[c2 * 8 + 2], pv[c2 * 8 + 3]);
                     w.z = pack_bf16(pv[c2 * 8 + 4], pv[c2 * 8 + 5]);
                     w.w = pack_bf16(pv[c2 * 8 + 6], pv[c2 * 8 + 7]);
-                    *reinterpret_cast<uint4*>(Pg + sw128_chunk(i, cb * 2 + c2)) = w;
+                    *reinterpret_cast<uint4*>(Pg + sw128_chunk(i, (j0 >> 3) + c2)) = w;
                 }
             }
         }
@@ -430,34 +478,20 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     __syncthreads();
     OSDN_CLKS(4, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
-    // ---- T = (I + A)^-1, blocked --------------------------------------------------------------------
-    ut_inverse_64(sA, sT, tid);
-    // gated, scaled queries for both state chains: Qg = scale gamma_i Q (same image layout as Q)
-    {
-        for (int e = tid; e < 2 * CH * 8; e += CL_THREADS) {
-            const int hf = e >> 9, i = (e >> 3) & 63, ch = e & 7;
-            const uint32_t off = sw128_chunk(i, ch);
-            const uint4 w = *reinterpret_cast<const uint4*>(sKQ + hf * 16384 + BOX + off);
-            const float f = a.scale * __expf(sG[i]);
-            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&w);
-            uint32_t o[4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const float2 v = __bfloat1622float2(p2[x]);
-                o[x] = pack_bf16(v.x * f, v.y * f);
-            }
-            *reinterpret_cast<uint4*>(a.Qg + tile * REC_BYTES + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
-        }
-    }
+    // ---- T = (I + A)^-1, blocked, in place ---------------------------------------------------------
+    ut_inverse_64_inplace(sA, tid);
 
     // ---- operand images: Tbg (shared), Tb and T (HBM) -----------------------------------------
     for (int e = tid; e < CH * 8; e += CL_THREADS) {
         const int i = e >> 3, ch = e & 7;
+        const float4 t0 = *reinterpret_cast<const float4*>(sA + i * LCF + ch * 8);
+        const float4 t1 = *reinterpret_cast<const float4*>(sA + i * LCF + ch * 8 + 4);
+        const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
         float t[8], tb8[8], tbg[8];
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
             const int j = ch * 8 + x;
-            t[x] = sT[i * LC + j];
+            t[x] = j <= i ? tv[x] : 0.f;   // above the diagonal the array holds scratch
             tb8[x] = t[x] * sBeta[j];
             tbg[x] = tb8[x] * __expf(sG[j]);
         }
@@ -489,23 +523,24 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     OSDN_CLKS(7, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
-        const int k = warp * 32 + lane;
-        const uint32_t taddr = tb + ((uint32_t)(warp * 32) << 16) + 64;
+        const int k = quad * 32 + lane;
+        const uint32_t taddr = tb + ((uint32_t)(quad * 32) << 16) + 64 + half * 32;
         uint8_t* Wg = a.WT + tile * REC_BYTES;
-        for (int cb = 0; cb < 4; ++cb) {
-            uint32_t r[16];
-            tmem_ld16(taddr + cb * 16, r);
-            tmem_ld_wait();
+        uint32_t r[2][16];
+        tmem_ld16(taddr, r[0]);
+        tmem_ld16(taddr + 16, r[1]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb)
 #pragma unroll
             for (int c2 = 0; c2 < 2; ++c2) {
                 uint4 w;
-                w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
-                w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
-                w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
-                w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
-                *reinterpret_cast<uint4*>(Wg + sw128_chunk(k, cb * 2 + c2)) = w;
+                w.x = pack_bf16(__uint_as_float(r[cb][c2 * 8 + 0]), __uint_as_float(r[cb][c2 * 8 + 1]));
+                w.y = pack_bf16(__uint_as_float(r[cb][c2 * 8 + 2]), __uint_as_float(r[cb][c2 * 8 + 3]));
+                w.z = pack_bf16(__uint_as_float(r[cb][c2 * 8 + 4]), __uint_as_float(r[cb][c2 * 8 + 5]));
+                w.w = pack_bf16(__uint_as_float(r[cb][c2 * 8 + 6]), __uint_as_float(r[cb][c2 * 8 + 7]));
+                *reinterpret_cast<uint4*>(Wg + sw128_chunk(k, half * 4 + cb * 2 + c2)) = w;
             }
-        }
     }
     tc_fence_before();
     __syncthreads();
@@ -514,7 +549,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     __syncthreads();
     if ((blockIdx.x == 5 && blockIdx.y == 0) && threadIdx.x < 32) g_clk[0][threadIdx.x] = s_clk[threadIdx.x];
 #endif
-    if (warp == 0) tmem_dealloc(tb, 128);
+    if (warp == 1) tmem_dealloc(tb, 128);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1330,7 +1365,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     float* sRaw = reinterpret_cast<float*>(sm + R_RAW);       // Gamma_ij <k_i, ktil_j>, j < i
     __shared__ uint64_t bar_tma, bar_mma[5];
     __shared__ uint32_t tmem_base;
-    __shared__ float sG[CH], sBeta[CH], sg[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
+    __shared__ __align__(16) float sG[CH], sBeta[CH], sg[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
     __shared__ float sRsum;
 
     const int H = a.H;
@@ -1421,6 +1456,24 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fetch_scalars(tile_next, tok0_next, len_next, g_next, b_next);
     }
 
+    // skip words of this tile (every thread reads the same two words; used in the final epilogue)
+    const unsigned long long sk =
+        (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
+    if (tid == 64 && tile_next < a.ntiles) {   // warm L2 with everything the next tile will ask for
+        const int hh = (int)(tile_next % H);
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_prefetch_2d(&tmQ, hh * KD + hf * 64, tok0_next);
+            tma_prefetch_2d(&tmK, hh * KD + hf * 64, tok0_next);
+            tma_prefetch_2d(&tmKt, hh * KD + hf * 64, tok0_next);
+            tma_prefetch_2d(&tmV, hh * KD + hf * 64, tok0_next);
+            tma_prefetch_2d(&tmDO, hh * KD + hf * 64, tok0_next);
+        }
+        bulk_prefetch(a.dUT + (size_t)tile_next * 16384, 16384);
+        bulk_prefetch(a.ddUT + (size_t)tile_next * 16384, 16384);
+        bulk_prefetch(a.Tm + (size_t)tile_next * 8192, 8192);
+        bulk_prefetch(a.Sn + (size_t)tile_next * 32768, 32768);
+        bulk_prefetch(a.dSn + (size_t)tile_next * 32768, 32768);
+    }
     if (tid < CH) {
         float acc = 0.f, tot = 0.f;
         for (int j = 0; j < CH; ++j) {
@@ -1719,6 +1772,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_after();
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
+    // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's preconditioner
+    // step was skipped); ragged or mixed chunks are copied row by row.
+    const bool full = len == CH;
+    const bool dk_tile = full && sk == ~0ull;
     if (ok) {
         const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
         const uint32_t fc = f & 63;
@@ -1743,6 +1800,12 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tmem_ld8(tb + cDKR + lane_addr + j0, rkr);
             tmem_ld8(tb + cDVB + lane_addr + j0, rvb);
             float qv[8], kv[8], ktv[8], vv[8], bj[8], gj[8], rj[8];
+            *reinterpret_cast<float4*>(&bj[0]) = *reinterpret_cast<const float4*>(&sBeta[j0]);
+            *reinterpret_cast<float4*>(&bj[4]) = *reinterpret_cast<const float4*>(&sBeta[j0 + 4]);
+            *reinterpret_cast<float4*>(&gj[0]) = *reinterpret_cast<const float4*>(&sGam[j0]);
+            *reinterpret_cast<float4*>(&gj[4]) = *reinterpret_cast<const float4*>(&sGam[j0 + 4]);
+            *reinterpret_cast<float4*>(&rj[0]) = *reinterpret_cast<const float4*>(&sRho[j0]);
+            *reinterpret_cast<float4*>(&rj[4]) = *reinterpret_cast<const float4*>(&sRho[j0 + 4]);
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
                 const int j = j0 + x;
@@ -1751,9 +1814,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 kv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_K + eo));
                 ktv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_KT + eo));
                 vv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_V + eo));
-                bj[x] = sBeta[j];
-                gj[x] = sGam[j];
-                rj[x] = sRho[j];
             }
             tmem_ld_wait();
 #pragma unroll
@@ -1771,10 +1831,13 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 stq[j * KD + f] = __float2bfloat16_rn(dq);
                 stv[j * KD + f] = __float2bfloat16_rn(bj[x] * dvb);
                 stk[j * KD + f] = __float2bfloat16_rn(dkr + a.d_min * dkt);
-                stkr[j * KD + f] = dkr;
-                stkt[j * KD + f] = dkt;
+                if (!dk_tile || j == 0) {   // fp32 copies feed the preconditioner's reverse pass only
+                    stkr[j * KD + f] = dkr;
+                    stkt[j * KD + f] = dkt;
+                }
             }
         }
+        OSDN_CLKS(14, threadIdx.x == 0 && clk);
         // Sum over the 32 features of the warp for all 16 columns at once: in each of four steps a
         // lane keeps one half of its columns and hands the other half to its partner; a last exchange
         // joins the two lanes that end up with the same column (16 shuffles per quantity).
@@ -1800,15 +1863,39 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
         if (lane == 0) atomicAdd(&sRsum, rsum);
     }
+    OSDN_CLKS(15, threadIdx.x == 0 && clk);
     ok = __syncthreads_and(ok);   // block-uniform from here on (the copy-out contains a barrier)
+    OSDN_CLKS(16, threadIdx.x == 0 && clk);
     if (tid == 0 && tile_next < a.ntiles) issue_first(tile_next, tok0_next);   // q, k, ktil, v are dead
+    if (ok && warp == 1) {
+        // gate and beta gradients of the chunk: dgate_j is the suffix sum of the per-token terms (the
+        // in-chunk prefix G_i collects every g_j with j <= i), by one warp while the tiles are sent off
+        float s0 = sdG[lane], s1 = sdG[lane + 32];
+        float gl = sg[lane] + sg[lane + 32], tot = lane < CBW_THREADS / 32 ? sRed[lane] : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            gl += __shfl_xor_sync(0xffffffffu, gl, o);
+            tot += __shfl_xor_sync(0xffffffffu, tot, o);
+        }
+        if (lane == 31) s1 += sRsum + __expf(gl) * tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float u0 = __shfl_down_sync(0xffffffffu, s0, o), u1 = __shfl_down_sync(0xffffffffu, s1, o);
+            if (lane + o < 32) { s0 += u0; s1 += u1; }
+        }
+        s0 += __shfl_sync(0xffffffffu, s1, 0);
+        if (lane < len) {
+            const size_t th = (size_t)(tok0 + lane) * H + h;
+            a.dgate[th] = s0;
+            a.dbeta[th] = sdB[lane];
+        }
+        if (lane + 32 < len) {
+            const size_t th = (size_t)(tok0 + lane + 32) * H + h;
+            a.dgate[th] = s1;
+            a.dbeta[th] = sdB[lane + 32];
+        }
+    }
     if (ok) {
-        const unsigned long long sk =
-            (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
-        // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's
-        // preconditioner step was skipped); ragged or mixed chunks are copied row by row.
-        const bool full = len == CH;
-        const bool dk_tile = full && sk == ~0ull;
         if (full) {
             fence_proxy_async();
         }
@@ -1855,26 +1942,12 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         *reinterpret_cast<const uint4*>(sm + ST_DKT + j * 512 + ch * 16);
             }
         }
+        OSDN_CLKS(17, threadIdx.x == 0 && clk);
         if (full && tid == 0) bulk_wait_read();   // the staging tiles may be overwritten by the next tile
     }
     __syncthreads();   // every copy-out read of the staging tiles is done
     if (tid == 0 && tile_next < a.ntiles) issue_second(tile_next, tok0_next);
     OSDN_CLKS(12, threadIdx.x == 0 && clk);
-    if (tid == 0) {
-        float tot = 0.f;
-        for (int w = 0; w < CBW_THREADS / 32; ++w) tot += sRed[w];
-        float gl = 0.f;
-        for (int j = 0; j < CH; ++j) gl += sg[j];
-        sdG[CH - 1] += sRsum + __expf(gl) * tot;
-        float acc = 0.f;
-        for (int i = CH - 1; i >= 0; --i) { acc += sdG[i]; sdG[i] = acc; }
-    }
-    __syncthreads();
-    if (tid < len) {
-        const size_t th = (size_t)(tok0 + tid) * H + h;
-        a.dgate[th] = sdG[tid];
-        a.dbeta[th] = sdB[tid];
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
