@@ -22,6 +22,8 @@
 #include <cudaTypedefs.h>
 
 #include "osdn_common.cuh"
+#include <type_traits>
+
 #include "umma.cuh"
 
 namespace osdn {
@@ -1343,10 +1345,15 @@ constexpr uint32_t R_Q = 0, R_K = 16384, R_KT = 32768, R_V = 49152, R_DO = 65536
                    R_T = 114688, R_S = 122880, R_DS = 155648, R_RAW = 188416;
 constexpr uint32_t R_DWT = R_DO;                 // dW^T image replaces dO after phase A
 constexpr uint32_t R_M1 = R_S, R_M2 = R_S + 8192, R_DT = R_S + 16384, R_Y = R_S + 24576;
-// output staging after the last product ([token][feature] tiles over the dead operand space)
-constexpr uint32_t ST_DQ = 65536, ST_DV = 81920, ST_DK = 98304, ST_DKR = 114688, ST_DKT = 147456;
-static_assert(ST_DKT + 32768 <= R_RAW, "staging tiles must fit below the fp32 scratch");
-constexpr size_t CBW_SMEM = R_RAW + CH * LC * 4 + 1024;
+// Output staging after the last product ([token][feature] tiles over dead space): dq and dv over the
+// fp32 scratch (dead after phase D), dk over dO / dW^T; the fp32 copies of dk_read and dL/dktil, needed
+// only when some token's preconditioner step was really taken, over T, S and dS.  When every token of a
+// full chunk was skipped, the space of dU, ddU, T, S and dS is therefore free during the final epilogue
+// and the next tile's copies of them start there.
+constexpr uint32_t ST_DQ = R_RAW, ST_DV = R_RAW + 16384, ST_DK = R_DO, ST_DKR = 114688, ST_DKT = 147456;
+static_assert(ST_DKT + 32768 <= R_RAW, "fp32 staging tiles must fit below the fp32 scratch");
+constexpr size_t CBW_SMEM = R_RAW + 32768 + 1024;
+static_assert(CH * LC * 4 <= 32768, "fp32 scratch must fit in its region");
 
 __global__ void __launch_bounds__(CBW_THREADS, 1)
 tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -1367,6 +1374,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __shared__ uint32_t tmem_base;
     __shared__ __align__(16) float sG[CH], sBeta[CH], sg[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
     __shared__ float sRsum;
+    __shared__ __align__(16) float sFirstKt[KD];
 
     const int H = a.H;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1390,13 +1398,16 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // persistent: one CTA per SM walks over the (chunk, head) tiles.  The operands of the next tile
     // are requested in two batches as soon as the shared-memory regions they land in are dead, and
     // its per-token scalars are fetched into registers one tile ahead.
-    auto next_tile = [&](long t) {   // first non-empty tile of this CTA at or after t
-        while (t < a.ntiles && a.tab.chunk_len[(int)(t / H)] == 0) t += gridDim.x;
+    auto next_tile = [&](int t) {   // first non-empty tile of this CTA at or after t
+        while (t < a.ntiles && a.tab.chunk_len[(int)(t / H)] == 0) t += (int)gridDim.x;
         return t;
     };
-    auto issue_first = [&](long t, int t0) {   // q, k, ktil, v
+    // The copies of a tile arrive on one barrier phase; the transaction count is announced with the
+    // first group that is issued (expect_all), whichever that is.
+    constexpr uint32_t TILE_TX = 10 * BOX + 16384 + 16384 + 8192 + 32768 + 32768;
+    auto expect_all = [&]() { mbar_expect_tx(&bar_tma, TILE_TX); };
+    auto issue_first = [&](int t, int t0) {   // q, k, ktil, v
         const int hh = (int)(t % H);
-        mbar_expect_tx(&bar_tma, 10 * BOX + 16384 + 16384 + 8192 + 32768 + 32768);
         for (int hf = 0; hf < 2; ++hf) {
             tma_load_2d(sm + R_Q + hf * BOX, &tmQ, hh * KD + hf * 64, t0, &bar_tma);
             tma_load_2d(sm + R_K + hf * BOX, &tmK, hh * KD + hf * 64, t0, &bar_tma);
@@ -1404,31 +1415,35 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tma_load_2d(sm + R_V + hf * BOX, &tmV, hh * KD + hf * 64, t0, &bar_tma);
         }
     };
-    auto issue_second = [&](long t, int t0) {   // dout and the chain tiles
+    auto issue_dout = [&](int t, int t0) {
         const int hh = (int)(t % H);
         for (int hf = 0; hf < 2; ++hf) tma_load_2d(sm + R_DO + hf * BOX, &tmDO, hh * KD + hf * 64, t0, &bar_tma);
+    };
+    auto issue_chain_tiles = [&](int t) {   // dU, ddU, T, S, dS
         bulk_load(sm + R_DU, a.dUT + (size_t)t * 16384, 16384, &bar_tma);
         bulk_load(sm + R_DDU, a.ddUT + (size_t)t * 16384, 16384, &bar_tma);
         bulk_load(sm + R_T, a.Tm + (size_t)t * 8192, 8192, &bar_tma);
         bulk_load(sm + R_S, a.Sn + (size_t)t * 32768, 32768, &bar_tma);
         bulk_load(sm + R_DS, a.dSn + (size_t)t * 32768, 32768, &bar_tma);
     };
-    auto fetch_scalars = [&](long t, int t0, int ln, float& g, float& b) {
+    auto fetch_scalars = [&](int t, int t0, int ln, float& g, float& b) {
         const int hh = (int)(t % H);
         const bool in = tid < ln;
         g = (tid < CH && in) ? a.gate[(size_t)(t0 + tid) * H + hh] : 0.f;
         b = (tid < CH && in) ? a.beta[(size_t)(t0 + tid) * H + hh] : 0.f;
     };
     uint32_t ph = 0;   // barrier phase parity: number of tiles processed so far, mod 2
-    long tile_l = next_tile(blockIdx.x);
+    int tile_l = next_tile((int)blockIdx.x);
     int tok0 = 0, len = 0;
     float g_cur = 0.f, b_cur = 0.f;
     if (tile_l < a.ntiles) {
         tok0 = a.tab.chunk_tok0[(int)(tile_l / H)];
         len = a.tab.chunk_len[(int)(tile_l / H)];
         if (tid == 0) {
+            expect_all();
             issue_first(tile_l, tok0);
-            issue_second(tile_l, tok0);
+            issue_dout(tile_l, tok0);
+            issue_chain_tiles(tile_l);
         }
         fetch_scalars(tile_l, tok0, len, g_cur, b_cur);
     }
@@ -1447,7 +1462,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     OSDN_CLKS(0, threadIdx.x == 0 && clk);
     // table entries and scalars of the next tile, one tile ahead
-    const long tile_next = next_tile(tile_l + gridDim.x);
+    const int tile_next = next_tile(tile_l + (int)gridDim.x);
     int tok0_next = 0, len_next = 0;
     float g_next = 0.f, b_next = 0.f;
     if (tile_next < a.ntiles) {
@@ -1459,6 +1474,13 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // skip words of this tile (every thread reads the same two words; used in the final epilogue)
     const unsigned long long sk =
         (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
+    // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's preconditioner
+    // step was skipped); ragged or mixed chunks are copied row by row.  In the all-skipped case the
+    // space of each chain tile is not reused by the output staging, so the next tile's copy of it
+    // starts as soon as the last product reading it has finished (thread 0, below).
+    const bool full = len == CH;
+    const bool dk_tile = full && sk == ~0ull;
+    const bool early = dk_tile && tile_next < a.ntiles;
     if (tid == 64 && tile_next < a.ntiles) {   // warm L2 with everything the next tile will ask for
         const int hh = (int)(tile_next % H);
         for (int hf = 0; hf < 2; ++hf) {
@@ -1644,6 +1666,11 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                        make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
         }
         mma_commit(&bar_mma[1]);
+        if (early) {   // phase A has finished: dU and dS are dead
+            expect_all();
+            bulk_load(sm + R_DU, a.dUT + (size_t)tile_next * 16384, 16384, &bar_tma);
+            bulk_load(sm + R_DS, a.dSn + (size_t)tile_next * 32768, 32768, &bar_tma);
+        }
     }
     ok = ok && mbar_wait(&bar_mma[1], ph, a.status, ERR_MMA2);
     OSDN_CLKS(5, threadIdx.x == 0 && clk);
@@ -1684,6 +1711,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mma_ss(tb + cY, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
                    make_idesc(64, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
         mma_commit(&bar_mma[2]);
+        if (early) bulk_load(sm + R_DDU, a.ddUT + (size_t)tile_next * 16384, 16384, &bar_tma);   // phase B done
     }
     ok = ok && mbar_wait(&bar_mma[2], ph, a.status, ERR_MMA2);
     OSDN_CLKS(7, threadIdx.x == 0 && clk);
@@ -1766,16 +1794,17 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mma_ss(tb + cDKR, desc_advance(da1, 2048 * k), desc_advance(dbk, 32 * k),
                    make_idesc(128, 64, IDESC_A_MN), k > 0);
         mma_commit(&bar_mma[4]);
+        if (early) bulk_load(sm + R_T, a.Tm + (size_t)tile_next * 8192, 8192, &bar_tma);   // phase D done
     }
     ok = ok && mbar_wait(&bar_mma[4], ph, a.status, ERR_MMA2);
     OSDN_CLKS(11, threadIdx.x == 0 && clk);
     tc_fence_after();
+    // every product has finished: the images in the space of S are dead
+    if (early && tid == 0 && ok) bulk_load(sm + R_S, a.Sn + (size_t)tile_next * 32768, 32768, &bar_tma);
+    OSDN_CLKS(19, threadIdx.x == 0 && clk);
+    OSDN_CLKS(20, threadIdx.x == 32 && clk);
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
-    // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's preconditioner
-    // step was skipped); ragged or mixed chunks are copied row by row.
-    const bool full = len == CH;
-    const bool dk_tile = full && sk == ~0ull;
     if (ok) {
         const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
         const uint32_t fc = f & 63;
@@ -1788,28 +1817,27 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         __nv_bfloat16* stk = reinterpret_cast<__nv_bfloat16*>(sm + ST_DK);
         float* stkr = reinterpret_cast<float*>(sm + ST_DKR);
         float* stkt = reinterpret_cast<float*>(sm + ST_DKT);
+        // four token columns at a time: few enough live registers for the whole loop to stay in them
 #pragma unroll
-        for (int cb = 0; cb < 2; ++cb) {
-            const int j0 = colq * 16 + cb * 8;
-            uint32_t rq1[8], rq2[8], rkt[8], rdk[8], rkb[8], rkr[8], rvb[8];
-            tmem_ld8(tb + cDQ1 + lane_addr + j0, rq1);
-            tmem_ld8(tb + cDQ2 + lane_addr + j0, rq2);
-            tmem_ld8(tb + cDKTR + lane_addr + j0, rkt);
-            tmem_ld8(tb + cDKT + lane_addr + j0, rdk);
-            tmem_ld8(tb + cDKB + lane_addr + j0, rkb);
-            tmem_ld8(tb + cDKR + lane_addr + j0, rkr);
-            tmem_ld8(tb + cDVB + lane_addr + j0, rvb);
-            float qv[8], kv[8], ktv[8], vv[8], bj[8], gj[8], rj[8];
-            *reinterpret_cast<float4*>(&bj[0]) = *reinterpret_cast<const float4*>(&sBeta[j0]);
-            *reinterpret_cast<float4*>(&bj[4]) = *reinterpret_cast<const float4*>(&sBeta[j0 + 4]);
-            *reinterpret_cast<float4*>(&gj[0]) = *reinterpret_cast<const float4*>(&sGam[j0]);
-            *reinterpret_cast<float4*>(&gj[4]) = *reinterpret_cast<const float4*>(&sGam[j0 + 4]);
-            *reinterpret_cast<float4*>(&rj[0]) = *reinterpret_cast<const float4*>(&sRho[j0]);
-            *reinterpret_cast<float4*>(&rj[4]) = *reinterpret_cast<const float4*>(&sRho[j0 + 4]);
+        for (int cb = 0; cb < 4; ++cb) {
+            const int j0 = colq * 16 + cb * 4;
+            uint32_t rq1[4], rq2[4], rkt[4], rdk[4], rkb[4], rkr[4], rvb[4];
+            tmem_ld4(tb + cDQ1 + lane_addr + j0, rq1);
+            tmem_ld4(tb + cDQ2 + lane_addr + j0, rq2);
+            tmem_ld4(tb + cDVB + lane_addr + j0, rvb);
+            tmem_ld4(tb + cDKTR + lane_addr + j0, rkt);
+            tmem_ld4(tb + cDKT + lane_addr + j0, rdk);
+            tmem_ld4(tb + cDKB + lane_addr + j0, rkb);
+            tmem_ld4(tb + cDKR + lane_addr + j0, rkr);
+            float qv[4], kv[4], ktv[4], vv[4];
+            const float4 b4 = *reinterpret_cast<const float4*>(&sBeta[j0]);
+            const float4 g4 = *reinterpret_cast<const float4*>(&sGam[j0]);
+            const float4 r4 = *reinterpret_cast<const float4*>(&sRho[j0]);
+            const float bj[4] = {b4.x, b4.y, b4.z, b4.w}, gj[4] = {g4.x, g4.y, g4.z, g4.w};
+            const float rj[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
-            for (int x = 0; x < 8; ++x) {
-                const int j = j0 + x;
-                const uint32_t eo = boxf + sw128_elem(j, fc);
+            for (int x = 0; x < 4; ++x) {
+                const uint32_t eo = boxf + sw128_elem(j0 + x, fc);
                 qv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_Q + eo));
                 kv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_K + eo));
                 ktv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_KT + eo));
@@ -1817,7 +1845,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
             tmem_ld_wait();
 #pragma unroll
-            for (int x = 0; x < 8; ++x) {
+            for (int x = 0; x < 4; ++x) {
                 const int j = j0 + x;
                 const float dq = a.scale * gj[x] * __uint_as_float(rq1[x]) + __uint_as_float(rq2[x]);
                 const float dktr = rj[x] * __uint_as_float(rkt[x]);
@@ -1825,19 +1853,22 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const float dkb = __uint_as_float(rkb[x]);
                 const float dkr = bj[x] * gj[x] * dkb + __uint_as_float(rkr[x]);
                 const float dvb = __uint_as_float(rvb[x]);
-                gv[cb * 8 + x] = dq * qv[x] + dkr * kv[x] - dkt * ktv[x];
-                bv[cb * 8 + x] = gj[x] * dkb * kv[x] + dvb * vv[x];
+                gv[cb * 4 + x] = dq * qv[x] + dkr * kv[x] - dkt * ktv[x];
+                bv[cb * 4 + x] = gj[x] * dkb * kv[x] + dvb * vv[x];
                 rsum = fmaf(dktr, ktv[x], rsum);
                 stq[j * KD + f] = __float2bfloat16_rn(dq);
                 stv[j * KD + f] = __float2bfloat16_rn(bj[x] * dvb);
                 stk[j * KD + f] = __float2bfloat16_rn(dkr + a.d_min * dkt);
-                if (!dk_tile || j == 0) {   // fp32 copies feed the preconditioner's reverse pass only
+                if (!dk_tile) {   // fp32 copies feed the preconditioner's reverse pass only
                     stkr[j * KD + f] = dkr;
                     stkt[j * KD + f] = dkt;
+                } else if (j == 0) {
+                    sFirstKt[f] = dkt;   // a reverse pass may restart at the first token
                 }
             }
         }
         OSDN_CLKS(14, threadIdx.x == 0 && clk);
+        OSDN_CLKS(21, threadIdx.x == 32 && clk);
         // Sum over the 32 features of the warp for all 16 columns at once: in each of four steps a
         // lane keeps one half of its columns and hands the other half to its partner; a last exchange
         // joins the two lanes that end up with the same column (16 shuffles per quantity).
@@ -1866,7 +1897,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     OSDN_CLKS(15, threadIdx.x == 0 && clk);
     ok = __syncthreads_and(ok);   // block-uniform from here on (the copy-out contains a barrier)
     OSDN_CLKS(16, threadIdx.x == 0 && clk);
-    if (tid == 0 && tile_next < a.ntiles) issue_first(tile_next, tok0_next);   // q, k, ktil, v are dead
+    if (tid == 0 && tile_next < a.ntiles) {   // q, k, ktil, v are dead
+        if (!early) expect_all();
+        issue_first(tile_next, tok0_next);
+    }
     if (ok && warp == 1) {
         // gate and beta gradients of the chunk: dgate_j is the suffix sum of the per-token terms (the
         // in-chunk prefix G_i collects every g_j with j <= i), by one warp while the tiles are sent off
@@ -1927,7 +1961,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             // only the first token's dL/dktil is needed (a reverse recurrence may restart there)
             for (int e = tid; e < 32; e += CBW_THREADS) {
                 const size_t g = ((size_t)tok0 * H + h) * KD + e * 4;
-                *reinterpret_cast<uint4*>(a.dktil + g) = *reinterpret_cast<const uint4*>(sm + ST_DKT + e * 16);
+                *reinterpret_cast<uint4*>(a.dktil + g) = *reinterpret_cast<const uint4*>(&sFirstKt[e * 4]);
             }
         } else {
             for (int e = tid; e < len * 32; e += CBW_THREADS) {
@@ -1946,7 +1980,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (full && tid == 0) bulk_wait_read();   // the staging tiles may be overwritten by the next tile
     }
     __syncthreads();   // every copy-out read of the staging tiles is done
-    if (tid == 0 && tile_next < a.ntiles) issue_second(tile_next, tok0_next);
+    if (tid == 0 && tile_next < a.ntiles) {
+        issue_dout(tile_next, tok0_next);
+        if (!early) issue_chain_tiles(tile_next);
+    }
     OSDN_CLKS(12, threadIdx.x == 0 && clk);
     tc_fence_before();
     __syncthreads();
