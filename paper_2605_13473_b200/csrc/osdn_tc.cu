@@ -1805,11 +1805,11 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     OSDN_CLKS(20, threadIdx.x == 32 && clk);
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
+    float rsum = 0.f;
+    float gv[16], bv[16];   // per column: gate and beta contributions of this feature
     if (ok) {
         const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
         const uint32_t fc = f & 63;
-        float rsum = 0.f;
-        float gv[16], bv[16];   // per column: gate and beta contributions of this feature
         // Results are staged in shared memory as [token][feature] tiles (the operand tiles of the
         // finished products are dead by now) and written out with 16-byte stores afterwards.
         __nv_bfloat16* stq = reinterpret_cast<__nv_bfloat16*>(sm + ST_DQ);
@@ -1869,6 +1869,24 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         OSDN_CLKS(14, threadIdx.x == 0 && clk);
         OSDN_CLKS(21, threadIdx.x == 32 && clk);
+    }
+    OSDN_CLKS(15, threadIdx.x == 0 && clk);
+    fence_proxy_async();
+    ok = __syncthreads_and(ok);   // block-uniform from here on; staging complete, q, k, ktil, v dead
+    OSDN_CLKS(16, threadIdx.x == 0 && clk);
+    if (tid == 0) {
+        if (tile_next < a.ntiles) {
+            if (!early) expect_all();
+            issue_first(tile_next, tok0_next);
+        }
+        if (ok && full) {   // the tiles leave while the per-token sums below are formed
+            tma_store_2d(&tmDQ, h * KD, tok0, sm + ST_DQ);
+            tma_store_2d(&tmDV, h * KD, tok0, sm + ST_DV);
+            if (dk_tile) tma_store_2d(&tmDK, h * KD, tok0, sm + ST_DK);
+            bulk_commit();
+        }
+    }
+    if (ok) {
         // Sum over the 32 features of the warp for all 16 columns at once: in each of four steps a
         // lane keeps one half of its columns and hands the other half to its partner; a last exchange
         // joins the two lanes that end up with the same column (16 shuffles per quantity).
@@ -1894,13 +1912,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
         if (lane == 0) atomicAdd(&sRsum, rsum);
     }
-    OSDN_CLKS(15, threadIdx.x == 0 && clk);
-    ok = __syncthreads_and(ok);   // block-uniform from here on (the copy-out contains a barrier)
-    OSDN_CLKS(16, threadIdx.x == 0 && clk);
-    if (tid == 0 && tile_next < a.ntiles) {   // q, k, ktil, v are dead
-        if (!early) expect_all();
-        issue_first(tile_next, tok0_next);
-    }
+    __syncthreads();   // the per-token sums are complete
     if (ok && warp == 1) {
         // gate and beta gradients of the chunk: dgate_j is the suffix sum of the per-token terms (the
         // in-chunk prefix G_i collects every g_j with j <= i), by one warp while the tiles are sent off
@@ -1930,16 +1942,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     }
     if (ok) {
-        if (full) {
-            fence_proxy_async();
-        }
-        __syncthreads();
-        if (full && tid == 0) {
-            tma_store_2d(&tmDQ, h * KD, tok0, sm + ST_DQ);
-            tma_store_2d(&tmDV, h * KD, tok0, sm + ST_DV);
-            if (dk_tile) tma_store_2d(&tmDK, h * KD, tok0, sm + ST_DK);
-            bulk_commit();
-        }
         if (!full) {
             for (int e = tid; e < len * 16; e += CBW_THREADS) {
                 const int j = e >> 4, ch = e & 15;
