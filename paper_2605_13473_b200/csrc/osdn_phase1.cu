@@ -8,8 +8,8 @@
 //    all tokens in parallel first (phase1_spec).
 //  * Once every coordinate of d sits on the lower face of the box, the step for token t maps
 //    d_min*1 to d_min*1 again iff every pre-projection value rho_t d_min + c_t k_t^2 is below d_min,
-//    a condition that involves token t alone.  phase1_spec evaluates exactly that step for every
-//    token ("flag" bit) with the same arithmetic as the sequential kernel.  The sequential kernel
+//    a condition that involves token t alone.  phase1_spec evaluates that step for every token
+//    ("flag" bit), one thread per token; from the face the step has a closed form.  The sequential kernel
 //    (phase1_seq) then only walks tokens where d is not on the face or the flag is clear; flagged
 //    tokens entered on the face are skipped (their write key d_min*k was already emitted, their
 //    projection mask is all zero).  On the benchmark distributions with the retention aliased to
@@ -189,72 +189,106 @@ struct P1Fwd {
     Hyper hy;
 };
 
-// one warp per (chunk, head, 32-token half); tokens in batches of eight so that eight row loads
-// are in flight at a time
+// Eight consecutive values of a row as floats (one 16-byte load for bf16, two for fp32).
+__device__ __forceinline__ void load8(const float* p, float (&x)[8])
+{
+    const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&x)[8])
+{
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float2 f = __bfloat1622float2(h[q]);
+        x[2 * q] = f.x;
+        x[2 * q + 1] = f.y;
+    }
+}
+__device__ __forceinline__ void store8(float* p, const float (&x)[8])
+{
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+    *reinterpret_cast<float4*>(p + 4) = make_float4(x[4], x[5], x[6], x[7]);
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&x)[8])
+{
+    uint4 v;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) h[q] = __floats2bfloat162_rn(x[2 * q], x[2 * q + 1]);
+    *reinterpret_cast<uint4*>(p) = v;
+}
+
+// One warp per (chunk, head, 32-token half), eight lanes per token (four tokens at a time): a row is
+// read in full 128-byte lines and the sums need three shuffle rounds.  The step is taken from
+// d = d_min 1: then <d, k^2> = d_min sum k^2, and since x_r = rho d_min + c k_r^2 is monotone in k_r^2
+// for a fixed c, "every x_r below d_min" is decided by the largest (c >= 0) or smallest (c < 0) k_r^2.
 template <typename TI, typename TO, int K>
 __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
 {
-    constexpr int R = K / 32;
+    constexpr int NV = K / 64;   // 8-value vectors per lane
     const int lane = threadIdx.x & 31;
+    const int grp = lane >> 3, l8 = lane & 7;
     const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const long tile = w >> 1;
     const int half = (int)(w & 1);
     if (tile >= (long)a.NT * a.H) return;
     const int c = (int)(tile / a.H), h = (int)(tile % a.H);
     const int len = a.tab.chunk_len[c], tok0 = a.tab.chunk_tok0[c];
-    const TI* kp = static_cast<const TI*>(a.k);
-    TO* kt = static_cast<TO*>(a.ktil);
     const Hyper hy = a.hy;
+    const TI* kbase = static_cast<const TI*>(a.k);
+    TO* tbase = static_cast<TO*>(a.ktil);
     unsigned word = 0;
-    // per-token scalars: lane j of the warp fetches those of token half*32 + j
-    const int mine = half * 32 + lane;
-    const size_t th_mine = (size_t)(tok0 + min(mine, max(len - 1, 0))) * a.H + h;
-    const float beta_l = (mine < len && hy.beta_aware) ? a.beta[th_mine] : 1.0f;
-    const float ret_l = (mine < len && hy.apf_mode != 0) ? a.retsrc[th_mine] : 0.f;
-    float n_l = 0.f, rho_l = 1.f;
-    for (int j0 = 0; j0 < 32; j0 += 8) {
-        if (half * 32 + j0 >= len) break;
-        float kk[8][R];
+#pragma unroll 2
+    for (int it = 0; it < 8; ++it) {
+        const int i = half * 32 + it * 4 + grp;
+        const bool in = i < len;
+        const size_t th = (size_t)(tok0 + (in ? i : 0)) * a.H + h;
+        float x[NV][8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = min(half * 32 + j0 + u, len - 1);
-            load_row<R>(kp + ((size_t)(tok0 + i) * a.H + h) * K, lane, kk[u]);
-        }
+        for (int v = 0; v < NV; ++v) load8(kbase + th * K + v * 64 + l8 * 8, x[v]);
+        const float ret = (in && hy.apf_mode != 0) ? a.retsrc[th] : 0.f;
+        const float b = (in && hy.beta_aware) ? a.beta[th] : 1.0f;
+        float sumk = 0.f, kmax = 0.f, kmin = 3.0e38f;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int j = j0 + u, i = half * 32 + j;
-            if (i >= len) break;
-            const size_t th = (size_t)(tok0 + i) * a.H + h;
-            float kap[R];
-            const float sumk = square_sum<R>(kk[u], kap);
-            const float n = fmaxf(sumk, hy.eps);
-            const float rho = hy.apf_mode == 0 ? 1.0f : expf(__shfl_sync(0xffffffffu, ret_l, j));
-            const float b = __shfl_sync(0xffffffffu, beta_l, j);
-            if (lane == j) {
-                n_l = sumk > hy.eps ? n : -n;
-                rho_l = rho;
+        for (int v = 0; v < NV; ++v)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float kap = x[v][e] * x[v][e];
+                sumk += kap;
+                kmax = fmaxf(kmax, kap);
+                kmin = fminf(kmin, kap);
             }
-            if (hy.clamp) {
-                float d[R];
 #pragma unroll
-                for (int r = 0; r < R; ++r) d[r] = hy.d_min;
-                unsigned pass[R];
-                bool low;
-                float cc, al;
-                p1_step<R>(d, kap, n, b, rho, hy, pass, low, cc, al);
-                if (low) {
-                    word |= 1u << j;
-                    float wk[R];
+        for (int o = 4; o > 0; o >>= 1) {
+            sumk += __shfl_xor_sync(0xffffffffu, sumk, o);
+            kmax = fmaxf(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+            kmin = fminf(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+        }
+        const float n = fmaxf(sumk, hy.eps);
+        const float rho = hy.apf_mode == 0 ? 1.0f : expf(ret);
+        bool low = false;
+        if (hy.clamp) {
+            const float al = hy.d_min * sumk;
+            const float cc = hy.eta * b * (1.0f - b * al) / n;
+            const float xtop = fmaf(cc, cc >= 0.f ? kmax : kmin, rho * hy.d_min);
+            low = in && xtop < hy.d_min;
+        }
+        if (in && l8 == 0) {
+            a.r.n[th] = sumk > hy.eps ? n : -n;
+            a.r.rho[th] = rho;
+        }
+        if (low) {   // the write key of a token entered on the face: d_min k
 #pragma unroll
-                    for (int r = 0; r < R; ++r) wk[r] = hy.d_min * kk[u][r];
-                    store_row<R>(kt + th * K, lane, wk);
-                }
+            for (int v = 0; v < NV; ++v) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) x[v][e] *= hy.d_min;
+                store8(tbase + th * K + v * 64 + l8 * 8, x[v]);
             }
         }
-    }
-    if (mine < len) {
-        a.r.n[th_mine] = n_l;
-        a.r.rho[th_mine] = rho_l;
+        const unsigned bal = __ballot_sync(0xffffffffu, low);
+        word |= ((bal & 1u) | ((bal >> 7) & 2u) | ((bal >> 14) & 4u) | ((bal >> 21) & 8u)) << (it * 4);
     }
     if (lane == 0) a.r.flags[tile * 2 + half] = word;
 }
