@@ -39,7 +39,6 @@ struct WsLayout {
     size_t p1n;         // [T,H]          f32   max(|k|^2, eps), negated where the floor is active
     size_t p1rho;       // [T,H]          f32   retention of the preconditioner
     size_t p1flags;     // [NT,H,2]       u32   per token: the step maps d_min*1 to d_min*1, mask all zero
-    size_t dbound;      // [NT,H,K]       f32   preconditioner at chunk starts              (save only)
     size_t p1skip;      // [NT,H,2]       u32   tokens the sequential pass skipped           (save only)
     size_t pmask;       // [T,H,K/32]     u32   projection pass masks of processed tokens    (save only)
     size_t dtraj;       // [T,H,K]        f32   d_t of processed tokens                      (save only)
@@ -81,7 +80,6 @@ inline WsLayout make_layout(const osdn_params& p, bool need_bwd)
     L.p1rho = take(4 * Ttot * H);
     L.p1flags = take(4 * NT * H * 2);
     if (need_bwd) {
-        L.dbound = take(4 * NT * H * K);
         L.p1skip = take(4 * NT * H * 2);
         L.pmask = take(4 * Ttot * H * (K / 32));
         L.dtraj = take(4 * Ttot * H * K);
@@ -119,7 +117,7 @@ inline Table carve_table(void* ws, const WsLayout& L)
 }
 
 struct P1Regions {
-    float *n, *rho, *dbound, *dtraj;
+    float *n, *rho, *dtraj;
     unsigned *flags, *skipw, *pmask;
 };
 
@@ -130,7 +128,6 @@ inline P1Regions carve_p1(void* ws, const WsLayout& L)
     r.n = reinterpret_cast<float*>(w + L.p1n);
     r.rho = reinterpret_cast<float*>(w + L.p1rho);
     r.flags = reinterpret_cast<unsigned*>(w + L.p1flags);
-    r.dbound = reinterpret_cast<float*>(w + L.dbound);
     r.skipw = reinterpret_cast<unsigned*>(w + L.p1skip);
     r.pmask = reinterpret_cast<unsigned*>(w + L.pmask);
     r.dtraj = reinterpret_cast<float*>(w + L.dtraj);

@@ -332,14 +332,39 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
             w1 = a.r.flags[tl * 2 + 1];
         }
         const int cend = min(cbase + 32, c1);
+        // chunks of this group whose every token is flagged (lane = chunk)
+        unsigned allflag;
+        {
+            const int cl = cbase + lane;
+            const int lenl = cl < c1 ? min(CH, seq_len - (cl - c0) * CH) : 0;
+            const unsigned long long bl = (unsigned long long)w0 | ((unsigned long long)w1 << 32);
+            const unsigned long long vl = lenl >= 64 ? ~0ull : ((1ull << lenl) - 1ull);
+            allflag = __ballot_sync(0xffffffffu, cl < c1 && (bl & vl) == vl);
+        }
         for (int c = cbase; c < cend; ++c) {
+            if (face) {
+                // a run of fully flagged chunks entered on the face is skipped in one go
+                const unsigned rest = ~allflag >> (c - cbase);
+                const int run = min(rest ? __ffs((int)rest) - 1 : 32, cend - c);
+                if (run > 0) {
+                    if (a.save && lane < run) {
+                        const int cl = c + lane;
+                        const int lenl = min(CH, seq_len - (cl - c0) * CH);
+                        const unsigned long long vl = lenl >= 64 ? ~0ull : ((1ull << lenl) - 1ull);
+                        const size_t tl = (size_t)cl * H + h;
+                        a.r.skipw[tl * 2] = (unsigned)(vl & 0xffffffffull);
+                        a.r.skipw[tl * 2 + 1] = (unsigned)(vl >> 32);
+                    }
+                    c += run - 1;
+                    continue;
+                }
+            }
             const int nrel = c - c0;
             const int tok0 = seq_t0 + nrel * CH, len = min(CH, seq_len - nrel * CH);
             const size_t tile = (size_t)c * H + h;
             const unsigned long long bits = (unsigned long long)__shfl_sync(0xffffffffu, w0, c - cbase) |
                                             ((unsigned long long)__shfl_sync(0xffffffffu, w1, c - cbase) << 32);
             const unsigned long long valid = len >= 64 ? ~0ull : ((1ull << len) - 1ull);
-            if (a.save) store_row<R>(a.r.dbound + tile * K, lane, d);
             unsigned long long skipped = 0ull;
             if (face && (bits & valid) == valid) {
                 skipped = valid;
