@@ -26,39 +26,78 @@ constexpr int NTH = 256;
 // ---------------------------------------------------------------------------------------
 // chunk table
 // ---------------------------------------------------------------------------------------
-__global__ void build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Table t)
+// One CTA.  Chunk counts per sequence are scanned 256 sequences at a time; every chunk then finds
+// its sequence by bisection over the chunk offsets (kept in shared memory while they fit).
+constexpr int TBL_THREADS = 256, TBL_SMEM_SEQ = 2048;
+
+__global__ void __launch_bounds__(TBL_THREADS)
+build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Table t)
 {
-    __shared__ int s_total;
-    if (threadIdx.x == 0) {
-        int c = 0;
-        for (int s = 0; s < S; ++s) {
-            int t0 = cu ? cu[s] : s * T_dense;
-            int len = cu ? cu[s + 1] - cu[s] : T_dense;
+    __shared__ int s_c0[TBL_SMEM_SEQ + 1];
+    __shared__ int s_scan[TBL_THREADS];
+    __shared__ int s_carry;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (int base = 0; base < S; base += TBL_THREADS) {
+        const int s = base + tid;
+        int t0 = 0, len = 0;
+        if (s < S) {
+            t0 = cu ? cu[s] : s * T_dense;
+            len = cu ? cu[s + 1] - cu[s] : T_dense;
             if (len < 0) len = 0;
+        }
+        const int nc = (len + CH - 1) / CH;
+        s_scan[tid] = nc;
+        __syncthreads();
+        for (int o = 1; o < TBL_THREADS; o <<= 1) {   // inclusive scan
+            const int v = tid >= o ? s_scan[tid - o] : 0;
+            __syncthreads();
+            s_scan[tid] += v;
+            __syncthreads();
+        }
+        const int carry = s_carry;
+        if (s < S) {
+            const int c = min(carry + s_scan[tid] - nc, NTmax);
             t.seq_tok0[s] = t0;
             t.seq_len[s] = len;
-            t.seq_chunk0[s] = c < NTmax ? c : NTmax;
-            c += (len + CH - 1) / CH;
+            t.seq_chunk0[s] = c;
+            if (s <= TBL_SMEM_SEQ) s_c0[s] = c;
         }
-        if (c > NTmax) c = NTmax;
-        t.seq_chunk0[S] = c;
-        s_total = c;
+        __syncthreads();
+        if (tid == TBL_THREADS - 1) s_carry = carry + s_scan[tid];
+        __syncthreads();
+    }
+    const int total = min(s_carry, NTmax);
+    if (tid == 0) {
+        t.seq_chunk0[S] = total;
+        if (S <= TBL_SMEM_SEQ) s_c0[S] = total;
     }
     __syncthreads();
-    for (int s = 0; s < S; ++s) {
-        int c0 = t.seq_chunk0[s], c1 = t.seq_chunk0[s + 1];
-        int t0 = t.seq_tok0[s], len = t.seq_len[s];
-        for (int j = threadIdx.x; j < c1 - c0; j += blockDim.x) {
-            t.chunk_tok0[c0 + j] = t0 + j * CH;
-            int rem = len - j * CH;
-            t.chunk_len[c0 + j] = rem < CH ? rem : CH;
-            t.chunk_seq[c0 + j] = s;
+    const bool in_smem = S <= TBL_SMEM_SEQ;
+    for (int j = tid; j < NTmax; j += TBL_THREADS) {
+        if (j >= total) {
+            t.chunk_tok0[j] = 0;
+            t.chunk_len[j] = 0;
+            t.chunk_seq[j] = 0;
+            continue;
         }
-    }
-    for (int j = s_total + threadIdx.x; j < NTmax; j += blockDim.x) {
-        t.chunk_tok0[j] = 0;
-        t.chunk_len[j] = 0;
-        t.chunk_seq[j] = 0;
+        int lo = 0, hi = S - 1;   // last sequence whose first chunk is <= j (empty sequences share an offset)
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            const int c = in_smem ? s_c0[mid] : t.seq_chunk0[mid];
+            if (c <= j) lo = mid;
+            else hi = mid - 1;
+        }
+        const int s = lo;
+        const int c0 = in_smem ? s_c0[s] : t.seq_chunk0[s];
+        const int t0 = cu ? cu[s] : s * T_dense;
+        int len = cu ? cu[s + 1] - cu[s] : T_dense;
+        if (len < 0) len = 0;
+        const int rem = len - (j - c0) * CH;
+        t.chunk_tok0[j] = t0 + (j - c0) * CH;
+        t.chunk_len[j] = rem < CH ? rem : CH;
+        t.chunk_seq[j] = s;
     }
 }
 
@@ -690,7 +729,7 @@ int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaSt
 {
     Table tab = carve_table(ws, L);
     stage_mark(st, "build_table");
-    build_table_kernel<<<1, 256, 0, st>>>(L.S, p.T, p.nseq > 0 ? p.cu_seqlens : nullptr, L.NTmax, tab);
+    build_table_kernel<<<1, TBL_THREADS, 0, st>>>(L.S, p.T, p.nseq > 0 ? p.cu_seqlens : nullptr, L.NTmax, tab);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
