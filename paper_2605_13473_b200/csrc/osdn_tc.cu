@@ -908,31 +908,24 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             OSDN_CLKS(18, blockIdx.x == 0 && n == 1 && tid == 0);
             OSDN_CLKS(19, blockIdx.x == 0 && n == 20 && tid == 0);
             OSDN_CLKS(24, blockIdx.x == 0 && n == 31 && tid == 0);
-            // ---- E0: S -> bf16 operand, decay the accumulator
-            {
-                const float gC = sGC[gs];
-                uint32_t rr[2][16];
+            // ---- E0: S -> bf16 operand (what the next products wait for), then decay the accumulator
+            uint32_t rr[2][16];
 #pragma unroll
-                for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
-                tmem_ld_wait();
-                OSDN_CLKS(1, blockIdx.x == 0 && n == 10 && tid == 0);
+            for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
+            tmem_ld_wait();
+            OSDN_CLKS(1, blockIdx.x == 0 && n == 10 && tid == 0);
 #pragma unroll
-                for (int cb = 0; cb < 2; ++cb) {
-                    uint32_t* r = rr[cb];
+            for (int cb = 0; cb < 2; ++cb) {
+                const uint32_t* r = rr[cb];
 #pragma unroll
-                    for (int c2 = 0; c2 < 2; ++c2) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
-                        w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
-                        w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
-                        w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
-                        *reinterpret_cast<uint4*>(sS + (colq >> 1) * 16384 + sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2)) = w;
-                    }
-#pragma unroll
-                    for (int x = 0; x < 16; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * gC);
-                    tmem_st16(tS + lane_addr + colq * 32 + cb * 16, r);
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1]));
+                    w.y = pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3]));
+                    w.z = pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5]));
+                    w.w = pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7]));
+                    *reinterpret_cast<uint4*>(sS + (colq >> 1) * 16384 + sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2)) = w;
                 }
-                tmem_st_wait();
             }
             OSDN_CLKS(2, blockIdx.x == 0 && n == 10 && tid == 0);
             if (len < CH) {
@@ -946,6 +939,15 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_s_ready);
             OSDN_CLKS(3, blockIdx.x == 0 && n == 10 && tid == 0);
+            {   // gamma_C S back into the accumulator: only the state update (after du_ready) reads it
+                const float gC = sGC[gs];
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) rr[cb][x] = __float_as_uint(__uint_as_float(rr[cb][x]) * gC);
+                    tmem_st16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
+                }
+            }
 
             // ---- E1: dU^T -> bf16 operands
             float rho[16];
@@ -975,6 +977,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                                                                       pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
                 }
             }
+            tmem_st_wait();   // the decayed accumulator is in place
             fence_proxy_async();
             tc_fence_before();
             __syncwarp();
