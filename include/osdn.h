@@ -169,8 +169,14 @@ int osdn_fwd_static(const osdn_params* p, const void* q, const void* k, const vo
  * Host-buffer convenience for end-to-end measurements: copies the inputs (HOST pointers,
  * ideally pinned) into `staging` (device scratch of osdn_host_staging_bytes bytes), runs
  * osdn_fwd (and osdn_bwd when dout_host != NULL) and copies out / the gradients back to the
- * host buffers, all on `cuda_stream`, without synchronising.  Same layouts as above; NULL
- * optional inputs as above.  Nothing is allocated.
+ * host buffers, without synchronising: when the call returns everything is enqueued and ordered
+ * before whatever is enqueued on `cuda_stream` next.  Same layouts as above.
+ *
+ * A dense batch with B > 1 is cut into its B sequences (independent problems): the inputs of
+ * sequence b + 1 arrive and the results of sequence b - 1 leave while sequence b is computed.  The
+ * copies run on two internal streams that fork from and join `cuda_stream`; the streams and the
+ * events between them are created on the first such call on a device and kept.  Packed batches
+ * (nseq > 0) and B = 1 run in one piece on `cuda_stream` alone and create nothing.
  */
 size_t osdn_host_staging_bytes(const osdn_params* p, int with_bwd);
 int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host, const void* v_host,

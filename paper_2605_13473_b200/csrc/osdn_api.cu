@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "osdn_common.cuh"
 
@@ -255,6 +256,38 @@ size_t osdn_host_staging_bytes(const osdn_params* p, int with_bwd)
     return make_staging(*p, with_bwd != 0).total;
 }
 
+namespace {
+// Copy streams and events of the pipelined host step, created once per device.
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    std::vector<cudaEvent_t> arrived, computed;
+};
+std::mutex g_pipe_mutex;
+HostPipe* host_pipe(int nseq)
+{
+    static HostPipe pipes[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe& hp = pipes[dev];
+    if (!hp.in) {
+        if (cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&hp.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&hp.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    while ((int)hp.arrived.size() < nseq) {
+        cudaEvent_t e1, e2;
+        if (cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&e2, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        hp.arrived.push_back(e1);
+        hp.computed.push_back(e2);
+    }
+    return &hp;
+}
+}  // namespace
+
 int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host, const void* v_host,
                    const float* beta_host, const float* gate_host, const void* dout_host, void* out_host,
                    void* dq_host, void* dk_host, void* dv_host, float* dbeta_host, float* dgate_host,
@@ -271,41 +304,79 @@ int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host,
     if (staging_bytes < s.total) return OSDN_WORKSPACE_TOO_SMALL;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* d = static_cast<char*>(staging);
-    const size_t Ttot = p->nseq > 0 ? (size_t)p->T : (size_t)p->B * p->T;
     const size_t es = p->io_dtype == OSDN_BF16 ? 2 : 4;
-    const size_t nk = Ttot * p->H * p->K * es, nv = Ttot * p->H * p->V * es, ns = Ttot * p->H * 4;
+    // A dense batch is cut into its sequences (they are independent problems): while one sequence is
+    // computed the next one's inputs arrive and the previous one's results leave, on two copy streams
+    // that fork from and join `cuda_stream`.  Packed batches and single sequences go in one piece.
+    const int pieces = (p->nseq == 0 && p->B > 1) ? p->B : 1;
+    const size_t Tp = p->nseq > 0 ? (size_t)p->T : (size_t)(p->B / pieces) * p->T;   // tokens per piece
+    const size_t nk = Tp * p->H * p->K * es, nv = Tp * p->H * p->V * es, ns = Tp * p->H * 4;
+    HostPipe* hp = pieces > 1 ? host_pipe(pieces) : nullptr;
+    if (pieces > 1 && !hp) return OSDN_CUDA_ERROR;
+    cudaStream_t sin = hp ? hp->in : st, sout = hp ? hp->out : st;
     bool ok = true;
-    auto h2d = [&](size_t off, const void* src, size_t n) {
-        ok = ok && cudaMemcpyAsync(d + off, src, n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    auto cpy = [&](void* dst, const void* src, size_t n, cudaMemcpyKind kind, cudaStream_t on) {
+        ok = ok && cudaMemcpyAsync(dst, src, n, kind, on) == cudaSuccess;
     };
-    auto d2h = [&](void* dst, size_t off, size_t n) {
-        ok = ok && cudaMemcpyAsync(dst, d + off, n, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    };
-    h2d(s.q, q_host, nk); h2d(s.k, k_host, nk); h2d(s.v, v_host, nv);
-    h2d(s.beta, beta_host, ns); h2d(s.gate, gate_host, ns);
-    if (bwd) h2d(s.dout, dout_host, nv);
+    auto hoff = [](const void* base, size_t off) { return static_cast<const char*>(base) + off; };
+    auto hoffw = [](void* base, size_t off) { return static_cast<char*>(base) + off; };
+    if (hp) {
+        ok = ok && cudaEventRecord(hp->fork, st) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(sin, hp->fork, 0) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(sout, hp->fork, 0) == cudaSuccess;
+    }
+    for (int b = 0; b < pieces; ++b) {
+        cpy(d + s.q + b * nk, hoff(q_host, b * nk), nk, cudaMemcpyHostToDevice, sin);
+        cpy(d + s.k + b * nk, hoff(k_host, b * nk), nk, cudaMemcpyHostToDevice, sin);
+        cpy(d + s.v + b * nv, hoff(v_host, b * nv), nv, cudaMemcpyHostToDevice, sin);
+        cpy(d + s.beta + b * ns, hoff(beta_host, b * ns), ns, cudaMemcpyHostToDevice, sin);
+        cpy(d + s.gate + b * ns, hoff(gate_host, b * ns), ns, cudaMemcpyHostToDevice, sin);
+        if (bwd) cpy(d + s.dout + b * nv, hoff(dout_host, b * nv), nv, cudaMemcpyHostToDevice, sin);
+        if (hp) ok = ok && cudaEventRecord(hp->arrived[b], sin) == cudaSuccess;
+    }
     if (!ok) return OSDN_CUDA_ERROR;
     osdn_params pp = *p;
-    pp.flags = (p->flags & OSDN_FLAG_FORCE_SIMT) | (bwd ? OSDN_FLAG_SAVE_RESIDUALS : 0);
-    rc = osdn_fwd(&pp, d + s.q, d + s.k, d + s.v, reinterpret_cast<float*>(d + s.beta),
-                  reinterpret_cast<float*>(d + s.gate), nullptr, nullptr, nullptr, d + s.out, nullptr, nullptr,
-                  d + s.ws, s.ws_bytes, cuda_stream);
-    if (rc != OSDN_OK) return rc;
-    int launches = g_last_launches;
-    if (bwd) {
-        pp.flags |= OSDN_FLAG_RESIDUALS_VALID;
-        rc = osdn_bwd(&pp, d + s.q, d + s.k, d + s.v, reinterpret_cast<float*>(d + s.beta),
-                      reinterpret_cast<float*>(d + s.gate), nullptr, nullptr, nullptr, d + s.dout, nullptr,
-                      nullptr, d + s.dq, d + s.dk, d + s.dv, reinterpret_cast<float*>(d + s.dbeta),
-                      reinterpret_cast<float*>(d + s.dgate), nullptr, nullptr, nullptr, d + s.ws, s.ws_bytes,
+    if (pieces > 1) pp.B = 1;
+    int launches = 0;
+    for (int b = 0; b < pieces; ++b) {
+        if (hp && cudaStreamWaitEvent(st, hp->arrived[b], 0) != cudaSuccess) return OSDN_CUDA_ERROR;
+        pp.flags = (p->flags & OSDN_FLAG_FORCE_SIMT) | (bwd ? OSDN_FLAG_SAVE_RESIDUALS : 0);
+        rc = osdn_fwd(&pp, d + s.q + b * nk, d + s.k + b * nk, d + s.v + b * nv,
+                      reinterpret_cast<float*>(d + s.beta + b * ns), reinterpret_cast<float*>(d + s.gate + b * ns),
+                      nullptr, nullptr, nullptr, d + s.out + b * nv, nullptr, nullptr, d + s.ws, s.ws_bytes,
                       cuda_stream);
         if (rc != OSDN_OK) return rc;
         launches += g_last_launches;
+        if (bwd) {
+            pp.flags |= OSDN_FLAG_RESIDUALS_VALID;
+            rc = osdn_bwd(&pp, d + s.q + b * nk, d + s.k + b * nk, d + s.v + b * nv,
+                          reinterpret_cast<float*>(d + s.beta + b * ns),
+                          reinterpret_cast<float*>(d + s.gate + b * ns), nullptr, nullptr, nullptr,
+                          d + s.dout + b * nv, nullptr, nullptr, d + s.dq + b * nk, d + s.dk + b * nk,
+                          d + s.dv + b * nv, reinterpret_cast<float*>(d + s.dbeta + b * ns),
+                          reinterpret_cast<float*>(d + s.dgate + b * ns), nullptr, nullptr, nullptr, d + s.ws,
+                          s.ws_bytes, cuda_stream);
+            if (rc != OSDN_OK) return rc;
+            launches += g_last_launches;
+        }
+        if (hp) {
+            ok = ok && cudaEventRecord(hp->computed[b], st) == cudaSuccess;
+            ok = ok && cudaStreamWaitEvent(sout, hp->computed[b], 0) == cudaSuccess;
+        }
+        cpy(hoffw(out_host, b * nv), d + s.out + b * nv, nv, cudaMemcpyDeviceToHost, sout);
+        if (bwd) {
+            cpy(hoffw(dq_host, b * nk), d + s.dq + b * nk, nk, cudaMemcpyDeviceToHost, sout);
+            cpy(hoffw(dk_host, b * nk), d + s.dk + b * nk, nk, cudaMemcpyDeviceToHost, sout);
+            cpy(hoffw(dv_host, b * nv), d + s.dv + b * nv, nv, cudaMemcpyDeviceToHost, sout);
+            cpy(hoffw(dbeta_host, b * ns), d + s.dbeta + b * ns, ns, cudaMemcpyDeviceToHost, sout);
+            cpy(hoffw(dgate_host, b * ns), d + s.dgate + b * ns, ns, cudaMemcpyDeviceToHost, sout);
+        }
     }
-    d2h(out_host, s.out, nv);
-    if (bwd) {
-        d2h(dq_host, s.dq, nk); d2h(dk_host, s.dk, nk); d2h(dv_host, s.dv, nv);
-        d2h(dbeta_host, s.dbeta, ns); d2h(dgate_host, s.dgate, ns);
+    if (hp) {   // everything the copy streams did is ordered before what follows on the caller's stream
+        ok = ok && cudaEventRecord(hp->join, sout) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(st, hp->join, 0) == cudaSuccess;
+        ok = ok && cudaEventRecord(hp->join, sin) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(st, hp->join, 0) == cudaSuccess;
     }
     g_last_launches = launches;
     return ok ? OSDN_OK : OSDN_CUDA_ERROR;
