@@ -23,6 +23,17 @@
 
 namespace osdn {
 
+#ifdef OSDN_PHASE_CLOCKS
+__device__ long long g_clk_p1[64];
+__device__ int g_clk_p1_n;
+#define P1_STAMP(cond)                                                     \
+    do {                                                                   \
+        if ((cond) && p1_stamp_n < 64) g_clk_p1[p1_stamp_n++] = clock64();  \
+    } while (0)
+#else
+#define P1_STAMP(cond)
+#endif
+
 namespace {
 
 __device__ __forceinline__ float warp_sum(float x)
@@ -293,6 +304,16 @@ __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
     if (lane == 0) a.r.flags[tile * 2 + half] = word;
 }
 
+__device__ __forceinline__ void prefetch_l2(const void* p)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+// Warms L2 (and the address translation) for a row of `bytes` bytes that starts on a 128-byte line.
+__device__ __forceinline__ void prefetch_row(const void* p, int bytes)
+{
+    for (int o = 0; o < bytes; o += 128) prefetch_l2(static_cast<const char*>(p) + o);
+}
+
 template <int R> __device__ __forceinline__ bool on_lower_face(const float (&d)[R], const Hyper& hy)
 {
     bool f = hy.clamp != 0;
@@ -330,6 +351,22 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
             const size_t tl = (size_t)(cbase + lane) * H + h;
             w0 = a.r.flags[tl * 2];
             w1 = a.r.flags[tl * 2 + 1];
+            // Sparse work: unflagged tokens are processed for certain; warm L2 with their rows now.
+            const int cl = cbase + lane;
+            const int lenl = min(CH, seq_len - (cl - c0) * CH);
+            unsigned long long m = ~((unsigned long long)w0 | ((unsigned long long)w1 << 32)) &
+                                   (lenl >= 64 ? ~0ull : ((1ull << lenl) - 1ull));
+            if (__popcll(m) <= 16) {
+                while (m) {
+                    const int t = __ffsll((long long)m) - 1;
+                    m &= m - 1;
+                    const size_t th = (size_t)(seq_t0 + (cl - c0) * CH + t) * H + h;
+                    prefetch_row(kp + th * K, K * (int)sizeof(TI));
+                    prefetch_l2(a.r.n + th);
+                    prefetch_l2(a.r.rho + th);
+                    prefetch_l2(a.beta + th);
+                }
+            }
         }
         const int cend = min(cbase + 32, c1);
         // chunks of this group whose every token is flagged (lane = chunk)
@@ -501,6 +538,10 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
 #pragma unroll
         for (int r = 0; r < R; ++r) lam[r] = 0.f;
     }
+#ifdef OSDN_PHASE_CLOCKS
+    int p1_stamp_n = 0;
+#endif
+    P1_STAMP(chain == 0 && lane == 0);
     bool lam_valid = true;     // lam holds dL/dd_{t+1} for the token about to be processed
     long src = -1;             // otherwise it is k (.) dktil of this (skipped) token
     auto restart = [&](long tsrc) {
@@ -520,6 +561,32 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
             const size_t tl = (size_t)(ctop - 1 - lane) * H + h;
             w0 = a.r.skipw[tl * 2];
             w1 = a.r.skipw[tl * 2 + 1];
+            // Sparse work (a few processed tokens per chunk): each lane warms L2 with the rows its
+            // chunk's tokens will need, long before the sequential walk gets there.  These rows sit in
+            // large arrays that were last touched several kernels ago; a cold access costs microseconds.
+            const int cl = ctop - 1 - lane;
+            const int lenl = min(CH, seq_len - (cl - c0) * CH);
+            unsigned long long m = ~((unsigned long long)w0 | ((unsigned long long)w1 << 32)) &
+                                   (lenl >= 64 ? ~0ull : ((1ull << lenl) - 1ull));
+            if (__popcll(m) <= 16) {
+                while (m) {
+                    const int t = __ffsll((long long)m) - 1;
+                    m &= m - 1;
+                    const size_t th = (size_t)(seq_t0 + (cl - c0) * CH + t) * H + h;
+                    prefetch_row(kp + th * K, K * (int)sizeof(T));
+                    prefetch_row(a.r.dtraj + th * K, K * 4);
+                    prefetch_row(a.dktil + th * K, K * 4);
+                    prefetch_row(a.dkread + th * K, K * 4);
+                    prefetch_l2(a.r.pmask + th * R);
+                    prefetch_l2(a.r.n + th);
+                    prefetch_l2(a.r.rho + th);
+                    prefetch_l2(a.beta + th);
+                    if (t + 1 < lenl) {   // rows a restart above this token would read
+                        prefetch_row(kp + (th + H) * K, K * (int)sizeof(T));
+                        prefetch_row(a.dktil + (th + H) * K, K * 4);
+                    }
+                }
+            }
         }
         const int cbot = max(ctop - 32, c0);
         for (int c = ctop - 1; c >= cbot; --c) {
@@ -533,12 +600,25 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                 src = tok0;
                 continue;
             }
+            // The tokens to process are known up front (the clear bits of the skip word), so the rows of
+            // the next PF of them are always in flight, across runs of skipped tokens.  Where the
+            // recurrence restarts before a token (its upper neighbour was skipped), the two rows the
+            // restart needs travel with that token's rows.
             constexpr int PF = 4;
             float kb[PF][R], db[PF][R], tb[PF][R], rb[PF][R], nb[PF], hb[PF], bb[PF];
+            float sk_k[PF][R], sk_t[PF][R];
             unsigned mb[PF];
+            bool needr[PF];
+            const unsigned long long todo = ~sk & valid;
+            const bool valid_in = lam_valid;
+            const long src_in = src;
+            auto pop_top = [](unsigned long long& m) {
+                const int t = 63 - __clzll((long long)m);
+                m &= ~(1ull << t);
+                return t;
+            };
             auto fetch = [&](int i, int slot) {
-                const int ii = max(i, 0);
-                const size_t th = (size_t)(tok0 + ii) * H + h;
+                const size_t th = (size_t)(tok0 + i) * H + h;
                 load_row<R>(kp + th * K, lane, kb[slot]);
                 load_row<R>(a.r.dtraj + th * K, lane, db[slot]);
                 load_row<R>(a.dktil + th * K, lane, tb[slot]);
@@ -547,83 +627,83 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                 nb[slot] = a.r.n[th];
                 hb[slot] = a.r.rho[th];
                 bb[slot] = hy.beta_aware ? a.beta[th] : 1.0f;
-            };
-            int i = len - 1;
-            while (i >= 0) {
-                if ((sk >> i) & 1ull) {
-                    // run of skipped tokens: the recurrence restarts at its lowest token
-                    const unsigned long long below = i >= 63 ? ~0ull : ((1ull << (i + 1)) - 1ull);
-                    const unsigned long long real = ~sk & valid & below;
-                    lam_valid = false;
-                    if (!real) {
-                        src = tok0;
-                        break;
-                    }
-                    const int j = 63 - __clzll((long long)real);
-                    src = tok0 + j + 1;
-                    i = j;
+                const bool top = i == len - 1;
+                const bool need = top ? !valid_in : (((sk >> (i + 1)) & 1ull) != 0ull);
+                needr[slot] = need;
+                if (need) {   // lambda restarts at the lowest token of the skipped run above
+                    const size_t ts = (size_t)(top ? src_in : (long)(tok0 + i + 1)) * H + h;
+                    load_row<R>(kp + ts * K, lane, sk_k[slot]);
+                    load_row<R>(a.dktil + ts * K, lane, sk_t[slot]);
                 }
+            };
+            unsigned long long pfm = todo, rem = todo;
+            P1_STAMP(chain == 0 && lane == 0);
 #pragma unroll
-                for (int u = 0; u < PF; ++u) fetch(i - u, u);
-                bool stop = false;
-                while (i >= 0 && !stop) {
+            for (int u = 0; u < PF; ++u)
+                if (pfm) fetch(pop_top(pfm), u);
+            while (rem) {
 #pragma unroll
-                    for (int u = 0; u < PF; ++u) {
-                        if (i >= 0 && !stop) {
-                            float kk[R], kap[R], dt[R], dkt[R], dkr[R], drho = 0.f, dc = 0.f, al = 0.f;
+                for (int u = 0; u < PF; ++u) {
+                    if (rem) {
+                        const int i = pop_top(rem);
+                        float kk[R], kap[R], dt[R], dkt[R], dkr[R], drho = 0.f, dc = 0.f, al = 0.f;
 #pragma unroll
-                            for (int r = 0; r < R; ++r) {
-                                kk[r] = kb[u][r]; dt[r] = db[u][r]; dkt[r] = tb[u][r]; dkr[r] = rb[u][r];
-                            }
-                            const unsigned mw = mb[u];
-                            const float ns = nb[u], n = fabsf(ns), rho = hb[u], b = bb[u];
-                            fetch(i - PF, u);
-                            if (!lam_valid) {
-                                restart(src);
-                                lam_valid = true;
-                            }
-                            const size_t th = (size_t)(tok0 + i) * H + h;
-#pragma unroll
-                            for (int r = 0; r < R; ++r) {
-                                kap[r] = kk[r] * kk[r];
-                                const unsigned wr = __shfl_sync(0xffffffffu, mw, r);
-                                if (!((wr >> lane) & 1u)) lam[r] = 0.f;
-                                drho = fmaf(lam[r], dt[r], drho);
-                                dc = fmaf(lam[r], kap[r], dc);
-                                al = fmaf(dt[r], kap[r], al);
-                            }
-                            drho = warp_sum(drho);
-                            dc = warp_sum(dc);
-                            al = warp_sum(al);
-                            const float cc = hy.eta * b * (1.0f - b * al) / n;
-                            const float da = -hy.eta * b * b / n * dc;
-                            const float dbt = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
-                            const float dn = ns > 0.f ? -cc / n * dc : 0.f;
-                            float out[R];
-#pragma unroll
-                            for (int r = 0; r < R; ++r) {
-                                const float dkap = cc * lam[r] + da * dt[r] + dn;
-                                out[r] = dkr[r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
-                                lam[r] = rho * lam[r] + da * kap[r] + kk[r] * dkt[r];
-                            }
-                            store_row<R>(dkp + th * K, lane, out);
-                            if (lane == 0) {
-                                if (hy.beta_aware) a.dbeta[th] += dbt;
-                                if (hy.apf_mode == 1) a.dgate[th] += rho * drho;
-                                if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
-                            }
-                            --i;
-                            stop = i >= 0 && ((sk >> i) & 1ull);
+                        for (int r = 0; r < R; ++r) {
+                            kk[r] = kb[u][r]; dt[r] = db[u][r]; dkt[r] = tb[u][r]; dkr[r] = rb[u][r];
+                            if (needr[u]) lam[r] = sk_k[u][r] * sk_t[u][r];
                         }
+                        const unsigned mw = mb[u];
+                        const float ns = nb[u], n = fabsf(ns), rho = hb[u], b = bb[u];
+                        if (pfm) fetch(pop_top(pfm), u);
+                        const size_t th = (size_t)(tok0 + i) * H + h;
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            kap[r] = kk[r] * kk[r];
+                            const unsigned wr = __shfl_sync(0xffffffffu, mw, r);
+                            if (!((wr >> lane) & 1u)) lam[r] = 0.f;
+                            drho = fmaf(lam[r], dt[r], drho);
+                            dc = fmaf(lam[r], kap[r], dc);
+                            al = fmaf(dt[r], kap[r], al);
+                        }
+                        drho = warp_sum(drho);
+                        dc = warp_sum(dc);
+                        al = warp_sum(al);
+                        const float cc = hy.eta * b * (1.0f - b * al) / n;
+                        const float da = -hy.eta * b * b / n * dc;
+                        const float dbt = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
+                        const float dn = ns > 0.f ? -cc / n * dc : 0.f;
+                        float out[R];
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            const float dkap = cc * lam[r] + da * dt[r] + dn;
+                            out[r] = dkr[r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
+                            lam[r] = rho * lam[r] + da * kap[r] + kk[r] * dkt[r];
+                        }
+                        store_row<R>(dkp + th * K, lane, out);
+                        if (lane == 0) {
+                            // added on top of what the chunk-local backward wrote; as reductions
+                            // without a return value, so that the sweep does not wait for memory
+                            if (hy.beta_aware) atomicAdd(&a.dbeta[th], dbt);
+                            if (hy.apf_mode == 1) atomicAdd(&a.dgate[th], rho * drho);
+                            if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
+                        }
+                        P1_STAMP(chain == 0 && lane == 0);
                     }
                 }
             }
+            // state handed to the chunk below: lambda is live iff the chunk's first token was processed
+            lam_valid = (todo & 1ull) != 0ull;
+            if (!lam_valid) src = tok0;
         }
     }
     if (a.dprecond_in) {
         if (!lam_valid) restart(src);
         store_row<R>(a.dprecond_in + ((size_t)s * H + h) * K, lane, lam);
     }
+    P1_STAMP(chain == 0 && lane == 0);
+#ifdef OSDN_PHASE_CLOCKS
+    if (chain == 0 && lane == 0) g_clk_p1_n = p1_stamp_n;
+#endif
 }
 
 template <typename TI, typename TO, int K>
@@ -708,3 +788,11 @@ int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const fl
 }
 
 }  // namespace osdn
+
+#ifdef OSDN_PHASE_CLOCKS
+extern "C" int osdn_debug_clocks_p1(long long* out, int* n)
+{
+    if (cudaMemcpyFromSymbol(out, osdn::g_clk_p1, sizeof(long long) * 64) != cudaSuccess) return -1;
+    return cudaMemcpyFromSymbol(n, osdn::g_clk_p1_n, sizeof(int)) == cudaSuccess ? 0 : -1;
+}
+#endif
