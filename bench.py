@@ -100,6 +100,20 @@ def kernel_model(name, inp, NT):
     return m.get(name)
 
 
+def load_traffic(workload, kernel):
+    """DRAM bytes (read + write) of one launch of `kernel`, from the committed ncu summary of this
+    workload (a line "- traffic_bytes <kernel> = <bytes>"), or None when there is no capture."""
+    path = os.path.join(ROOT, "profiles", f"osdn_step_{workload}.md")
+    try:
+        for line in open(path):
+            parts = line.split()
+            if len(parts) >= 5 and parts[0] == "-" and parts[1] == "traffic_bytes" and parts[2] == kernel:
+                return float(parts[4])
+    except OSError:
+        pass
+    return None
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -252,7 +266,6 @@ def main():
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
-    binding.stage_timing_enable(True)
     sync_all()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches = 0
@@ -262,6 +275,13 @@ def main():
     e1.record()
     sync_all()
     ms_total = e0.elapsed_time(e1)
+    # Per-kernel durations: the same K steps once more, now with an event between every two launches
+    # (the events cost a few percent of a step, so they stay out of the region `value` is timed on).
+    binding.stage_timing_enable(True)
+    sync_all()
+    for _ in range(steps):
+        step()
+    sync_all()
     stages = binding.stage_timing_collect()
     binding.stage_timing_enable(False)
     clocks = sampler.stop()
@@ -335,7 +355,7 @@ def main():
             else:
                 ach, peak, unit = nbytes / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
             roofline = dict(kernel=dom, bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak,
-                            traffic=None, peak_source=peaks["source"], avg_us=avg_s * 1e6,
+                            traffic=load_traffic(args.workload, dom), peak_source=peaks["source"], avg_us=avg_s * 1e6,
                             algorithmic_bytes=nbytes, algorithmic_flops=flops)
     # whole-step roofline (the slower of the step's flops at tensor peak and its bytes at HBM peak)
     es = 2 if inp.io_dtype == "bf16" else 4
@@ -374,7 +394,8 @@ def main():
         "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if inp.io_dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": w["desc"], "l2": "inputs + workspace exceed L2 (no flush)",
-                   "path": "simt" if args.simt else "auto", "tokens_per_step_per_gpu": tokens},
+                   "path": "simt" if args.simt else "auto", "tokens_per_step_per_gpu": tokens,
+                   "kernel_timing": "second pass of the same steps with an event between launches"},
         "clocks": clocks, "gpu_launches": launches,
         "e2e": ({"value": total_tokens / (e2e["ms"] * 1e-3), "unit": "tokens/s",
                  "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"]} if e2e else None),
