@@ -46,6 +46,8 @@ def load_peaks():
 
 def make_inputs(name):
     from paper_2605_13473_b200.synth import OsdnHyper, config, draw
+    if name == "decode":
+        return draw("decode_b512", 21, [1] * 512, 8, 128, 128, "bf16", dense_B=512, hyper=OsdnHyper(), with_state=True)
     w = WORKLOADS[name]
     if w["idx"] >= 0:
         return config(w["idx"])
@@ -171,7 +173,8 @@ def run_reference(args):
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     import oracle
     inp = make_inputs(args.workload)
-    w = WORKLOADS[args.workload]
+    w = WORKLOADS.get(args.workload) or dict(bwd=False, desc="decode: 512 sequences x 1 new token, H=8 dk=dv=128, "
+                                                               "bf16 activations, fp32 state")
     tokens = inp.T_total
 
     def step():
@@ -190,7 +193,9 @@ def run_reference(args):
     val = tokens * steps / dt
     cores = oracle.threads()
     line = {
-        "impl": "reference", "metric": "fwd+bwd tokens/s per layer", "value": val, "unit": "tokens/s",
+        "impl": "reference",
+        "metric": ("decode tokens/s per layer" if args.workload == "decode" else
+                   "fwd+bwd tokens/s per layer" if w["bwd"] else "fwd tokens/s per layer"), "value": val, "unit": "tokens/s",
         "n_gpus": 0, "steps": steps, "warmup": args.warmup if args.warmup is not None else 1,
         "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
@@ -202,18 +207,141 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_decode(args):
+    """`--workload decode`: the recurrent step (osdn_decode_step) on a serving-sized cache: one new token
+    for each of 512 sequences, H=8, dk=dv=128, bf16 activations, fp32 state (268 MB, larger than L2).
+    Bound by reading and writing the state once per token."""
+    import torch
+    import torch.distributed as dist
+    from paper_2605_13473_b200 import binding
+    from paper_2605_13473_b200.build import build
+    from paper_2605_13473_b200.sharding import aggregate_throughput
+    from paper_2605_13473_b200.synth import OsdnHyper, draw
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    steps = args.steps if args.steps is not None else 50
+    warmup = max(args.warmup if args.warmup is not None else 5, 3)
+    B, H, D = 512, 8, 128
+    hy = OsdnHyper()
+    inp = draw("decode_b512", 21 + rank, [1] * B, H, D, D, "bf16", dense_B=B, hyper=hy, with_state=True)
+    p = binding.make_params(B=B, T=1, H=H, K=D, V=D, io_dtype="bf16", hyper=hy)
+    hq, hk, hv = (x.to(torch.bfloat16).contiguous().pin_memory() for x in (inp.q, inp.k, inp.v))
+    hb, hg = inp.beta.float().pin_memory(), inp.gate.float().pin_memory()
+    q, k, v, beta, gate = (x.to(dev) for x in (hq, hk, hv, hb, hg))
+    state, precond = inp.init_state.float().to(dev).contiguous(), inp.precond_in.float().to(dev).contiguous()
+    out = torch.empty(B, H, D, device=dev, dtype=torch.bfloat16)
+    hout = torch.empty(B, H, D, dtype=torch.bfloat16).pin_memory()
+
+    def step():
+        binding.osdn_decode_step(p, q, k, v, beta, gate, None, state, precond, out)
+
+    def host_step():
+        for dst, src in ((q, hq), (k, hk), (v, hv), (beta, hb), (gate, hg)):
+            dst.copy_(src, non_blocking=True)
+        step()
+        hout.copy_(out, non_blocking=True)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn):
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        sync_all()
+        return e0.elapsed_time(e1)
+
+    for _ in range(warmup):
+        step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    ms_total = timed(step)
+    binding.stage_timing_enable(True)
+    timed(step)
+    stages = binding.stage_timing_collect()
+    binding.stage_timing_enable(False)
+    clocks = sampler.stop()
+    for _ in range(2):
+        host_step()
+    ms_host = timed(host_step)
+    total_tokens, ms_total, _ = aggregate_throughput(B * steps, ms_total, dev)
+    _, ms_host, _ = aggregate_throughput(B * steps, ms_host, dev)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peaks = load_peaks()
+    durs = stages.get("decode_step", [])
+    avg_s = (sum(durs) / len(durs) * 1e-3) if durs else ms_total / steps * 1e-3
+    nbytes = B * H * (2 * D * D * 4 + 2 * D * 4 + (2 * D + 2 * D) * 2 + 8)   # state and d in+out, q k v out, beta gate
+    ach = nbytes / avg_s / 1e9
+    roofline = dict(kernel="decode_step", bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=ach / peaks["hbm_gbs"], traffic=load_traffic("decode", "decode_step"),
+                    peak_source=peaks["source"], avg_us=avg_s * 1e6, algorithmic_bytes=nbytes)
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import oracle
+        oracle.build()
+        t0, reps = time.perf_counter(), 0
+        while time.perf_counter() - t0 < 10.0 and reps < 200:
+            oracle.fwd_inputs(inp)
+            reps += 1
+        dt = time.perf_counter() - t0
+        cpu_baseline = dict(value=B * reps / dt, unit="tokens/s", cores=oracle.threads(), kind="oracle",
+                            sample=f"whole workload ({B} sequences x {H} heads, one token each), {reps} repetitions, {dt:.1f} s")
+    nb = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))
+    line = {
+        "metric": "decode tokens/s per layer", "value": total_tokens / (ms_total * 1e-3), "unit": "tokens/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_total / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "decode: 512 sequences x 1 new token, H=8 dk=dv=128, bf16 activations, fp32 state",
+                   "l2": "state (268 MB) exceeds L2 (no flush)", "tokens_per_step_per_gpu": B,
+                   "kernel_timing": "second pass of the same steps with an event between launches"},
+        "clocks": clocks, "gpu_launches": steps,
+        "e2e": {"value": total_tokens / (ms_host * 1e-3), "unit": "tokens/s",
+                "h2d_bytes_per_step": nb(hq, hk, hv, hb, hg), "d2h_bytes_per_step": nb(hout),
+                "note": "activations from and to pinned host memory every step; the state stays in its device cache"},
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=list(WORKLOADS))
+    ap.add_argument("--workload", default="cfg2", choices=list(WORKLOADS) + ["decode"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core fp32 kernels")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload == "decode":
+        run_decode(args)
         return
     steps = args.steps if args.steps is not None else 20
     warmup = max(args.warmup if args.warmup is not None else 5, 3)

@@ -135,6 +135,26 @@ int osdn_precond_update(const osdn_params* p, const void* k, const float* beta,
                         void* k_tilde_out, float* precond_out, void* cuda_stream);
 
 /*
+ * Recurrent (decode) step (appendix paragraph "Single-token recurrence kernel for OSGDN", stated
+ * for q_len <= 64): for the p->T new tokens of each of the p->B sequences, in order,
+ *     alpha_t = exp(g_t);  ktil_t = d_t (.) k_t;  d_{t+1} as in osdn_fwd (Algorithm 1 with APF and the
+ *     box projection);  S_t = alpha_t S_{t-1} + beta_t (v_t - alpha_t S_{t-1} k_t) ktil_t^T;
+ *     o_t = scale S_t q_t,
+ * in one launch.  It is the recurrence osdn_fwd evaluates chunk by chunk, so a prefill with osdn_fwd
+ * (final_state, precond_out) followed by this call continues the same sequence.
+ *   in    : q, k [B,T,H,K], v [B,T,H,V] io_dtype; beta, gate [B,T,H] fp32; apf_log_ret [B,T,H]
+ *           (required iff apf_mode == SEPARATE).  Dense batches only (p->nseq == 0).
+ *   in/out: state [B,H,V,K] fp32 and precond [B,H,K] fp32, the caller's cache, updated in place.
+ *   out   : out [B,T,H,V] io_dtype.
+ * All pointers are DEVICE pointers, 16-byte aligned.  No workspace, nothing is allocated.  Any T >= 1
+ * is accepted; the call is sequential over T, so long prompts belong to osdn_fwd.  Errors as for
+ * osdn_fwd (nothing is launched on an argument error).
+ */
+int osdn_decode_step(const osdn_params* p, const void* q, const void* k, const void* v,
+                     const float* beta, const float* gate, const float* apf_log_ret,
+                     float* state, float* precond, void* out, void* cuda_stream);
+
+/*
  * Forward pass for callers that cannot provide a workspace.  (The paper has no counterpart to
  * this call; it exists for deployment reasons only.)
  *

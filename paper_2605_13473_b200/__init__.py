@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     osdn_bwd,
     osdn_fwd,
     osdn_fwd_static,
+    osdn_decode_step,
     osdn_precond_update,
     osdn_step_host,
     osdn_workspace_bytes,

@@ -19,7 +19,7 @@ EXPORTS = [
     "osdn_workspace_bytes", "osdn_fwd", "osdn_bwd", "osdn_precond_update", "osdn_host_staging_bytes",
     "osdn_step_host", "osdn_read_device_status", "osdn_status_string", "osdn_last_launch_count",
     "osdn_stage_timing_enable", "osdn_stage_timing_read", "osdn_workspace_region",
-    "osdn_fwd_static",
+    "osdn_fwd_static", "osdn_decode_step",
 ]
 
 
@@ -58,6 +58,8 @@ def load_library(path: Optional[str] = None):
     lib.osdn_bwd.argtypes = [pp] + [vp] * 19 + [vp, sz, vp]
     lib.osdn_precond_update.restype = ci
     lib.osdn_precond_update.argtypes = [pp] + [vp] * 6 + [vp]
+    lib.osdn_decode_step.restype = ci
+    lib.osdn_decode_step.argtypes = [pp] + [vp] * 9 + [vp]
     lib.osdn_step_host.restype = ci
     lib.osdn_step_host.argtypes = [pp] + [vp] * 12 + [vp, sz, vp]
     lib.osdn_read_device_status.restype = ci
@@ -208,6 +210,14 @@ def osdn_precond_update(p: OsdnParams, k, beta, gate_or_log_ret, precond_in, k_t
     rc = lib.osdn_precond_update(ctypes.byref(p), _ptr(k), _ptr(beta), _ptr(gate_or_log_ret), _ptr(precond_in),
                                  _ptr(k_tilde_out), _ptr(precond_out), _stream_ptr())
     _check(rc, "osdn_precond_update")
+
+
+def osdn_decode_step(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, state, precond, out):
+    """``state`` [B,H,V,K] and ``precond`` [B,H,K] (fp32, device) are updated in place."""
+    lib = load_library()
+    rc = lib.osdn_decode_step(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gate), _ptr(apf_log_ret),
+                              _ptr(state), _ptr(precond), _ptr(out), _stream_ptr())
+    _check(rc, "osdn_decode_step")
 
 
 def osdn_step_host(p: OsdnParams, q, k, v, beta, gate, dout, out, dq, dk, dv, dbeta, dgate,

@@ -224,6 +224,26 @@ int osdn_precond_update(const osdn_params* p, const void* k, const float* beta, 
     return OSDN_OK;
 }
 
+int osdn_decode_step(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                     const float* gate, const float* apf_log_ret, float* state, float* precond, void* out,
+                     void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (p->nseq != 0) return OSDN_INVALID_ARG;   // a dense [B, T, H, *] block of new tokens
+    if (!q || !k || !v || !beta || !gate || !state || !precond || !out) return OSDN_INVALID_ARG;
+    if (p->apf_mode == OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, state, precond, out};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    const int n = decode_step(*p, make_hyper(*p), q, k, v, beta, gate, apf_log_ret, state, precond, out,
+                              static_cast<cudaStream_t>(cuda_stream));
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = n;
+    return OSDN_OK;
+}
+
 // ---- host-buffer convenience --------------------------------------------------------------
 namespace {
 struct Staging {

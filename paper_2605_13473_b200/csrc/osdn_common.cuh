@@ -174,6 +174,12 @@ int phase1_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, vo
                     const float* dktil, const float* dkread, bool bulk, cudaStream_t st);
 int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta, const float* retsrc,
                   const float* precond_in, void* ktil_out, float* precond_out, cudaStream_t st);
+
+// Recurrent step over p.T tokens per sequence on cached state and preconditioner (both updated in
+// place); one launch.
+int decode_step(const osdn_params& p, const Hyper& hy, const void* q, const void* k, const void* v,
+                const float* beta, const float* gate, const float* log_ret, float* state, float* precond,
+                void* out, cudaStream_t st);
 int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st);
 
 // Optional per-kernel timing (off by default): when enabled through osdn_stage_timing_enable, every
