@@ -69,6 +69,19 @@ def test_calls_reject_bad_arguments_before_any_launch(lib):
     rc = lib.osdn_precond_update(ctypes.byref(p), fake, fake, fake, null, null, fake, null)
     assert rc == -1
     assert osdn.status_string(-2) == "unsupported shape"
+    # the recurrent step: missing cache, misaligned pointer, missing separate retention, packed batch
+    p = osdn.make_params(B=2, T=1, H=1, K=128, V=128, io_dtype="bf16", hyper=hy)
+    rc = lib.osdn_decode_step(ctypes.byref(p), fake, fake, fake, fake, fake, null, null, fake, fake, null)
+    assert rc == -1
+    rc = lib.osdn_decode_step(ctypes.byref(p), fake, fake, fake, fake, fake, null, odd, fake, fake, null)
+    assert rc == -3
+    p.apf_mode = 2
+    rc = lib.osdn_decode_step(ctypes.byref(p), fake, fake, fake, fake, fake, null, fake, fake, fake, null)
+    assert rc == -1
+    p.apf_mode = 1
+    p.K = 96
+    rc = lib.osdn_decode_step(ctypes.byref(p), fake, fake, fake, fake, fake, null, fake, fake, fake, null)
+    assert rc == -2
 
 
 def test_missing_library_fails_loudly(tmp_path):
