@@ -22,13 +22,31 @@ struct Hyper {
 // Sequence / chunk table built on the device from cu_seqlens (or from B, T for dense input).
 // Chunks never straddle sequences; chunk_len < 64 marks a ragged tail; entries beyond the
 // realised chunk count have chunk_len == 0.
+// Chunk table.  For a dense batch (every sequence T tokens long) the entries are pure arithmetic and
+// nothing is read; for a packed batch they were written by build_table_kernel from cu_seqlens.
 struct Table {
-    int* seq_tok0;    // [S]    first packed token of the sequence
-    int* seq_len;     // [S]
-    int* seq_chunk0;  // [S+1]  first chunk of the sequence; [S] = number of chunks
-    int* chunk_tok0;  // [NTmax]
-    int* chunk_len;   // [NTmax]
-    int* chunk_seq;   // [NTmax]
+    int* seq_tok0_;    // [S]    first packed token of the sequence
+    int* seq_len_;     // [S]
+    int* seq_chunk0_;  // [S+1]  first chunk of the sequence; [S] = number of chunks
+    int* chunk_tok0_;  // [NTmax]
+    int* chunk_len_;   // [NTmax]
+    int* chunk_seq_;   // [NTmax]
+    int dense_T;       // > 0: dense batch with sequences of this length
+    int dense_nc;      //      and this many chunks per sequence
+    __device__ __forceinline__ int seq_tok0(int s) const { return dense_T ? s * dense_T : seq_tok0_[s]; }
+    __device__ __forceinline__ int seq_len(int s) const { return dense_T ? dense_T : seq_len_[s]; }
+    __device__ __forceinline__ int seq_chunk0(int s) const { return dense_T ? s * dense_nc : seq_chunk0_[s]; }
+    __device__ __forceinline__ int chunk_tok0(int c) const
+    {
+        return dense_T ? (c / dense_nc) * dense_T + (c % dense_nc) * CH : chunk_tok0_[c];
+    }
+    __device__ __forceinline__ int chunk_len(int c) const
+    {
+        if (!dense_T) return chunk_len_[c];
+        const int rem = dense_T - (c % dense_nc) * CH;
+        return rem < CH ? rem : CH;
+    }
+    __device__ __forceinline__ int chunk_seq(int c) const { return dense_T ? c / dense_nc : chunk_seq_[c]; }
 };
 
 // Byte offsets of every region inside the caller's workspace.
@@ -58,6 +76,7 @@ struct WsLayout {
     size_t out_scratch; // [T,H,V]        f32   forward output when the backward recomputes the forward
     size_t total;
     int S, NTmax;
+    int dense_T;        // > 0 for a dense batch (see Table)
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -70,6 +89,7 @@ inline WsLayout make_layout(const osdn_params& p, bool need_bwd)
     const int NTmax = p.nseq > 0 ? (int)(Ttot / CH) + S : p.B * ((p.T + CH - 1) / CH);
     L.S = S;
     L.NTmax = NTmax;
+    L.dense_T = p.nseq > 0 ? 0 : p.T;
     const size_t H = p.H, K = p.K, V = p.V, NT = NTmax;
     const size_t D = K > V ? K : V;
     size_t off = 0;
@@ -107,12 +127,14 @@ inline Table carve_table(void* ws, const WsLayout& L)
 {
     int* base = reinterpret_cast<int*>(static_cast<char*>(ws) + L.table);
     Table t;
-    t.seq_tok0 = base;
-    t.seq_len = base + L.S;
-    t.seq_chunk0 = base + 2 * L.S;
-    t.chunk_tok0 = base + 3 * L.S + 1;
-    t.chunk_len = t.chunk_tok0 + L.NTmax;
-    t.chunk_seq = t.chunk_len + L.NTmax;
+    t.seq_tok0_ = base;
+    t.seq_len_ = base + L.S;
+    t.seq_chunk0_ = base + 2 * L.S;
+    t.chunk_tok0_ = base + 3 * L.S + 1;
+    t.chunk_len_ = t.chunk_tok0_ + L.NTmax;
+    t.chunk_seq_ = t.chunk_len_ + L.NTmax;
+    t.dense_T = L.dense_T;
+    t.dense_nc = L.dense_T ? (L.dense_T + CH - 1) / CH : 0;
     return t;
 }
 

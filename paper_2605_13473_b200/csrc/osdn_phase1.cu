@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
     const int half = (int)(w & 1);
     if (tile >= (long)a.NT * a.H) return;
     const int c = (int)(tile / a.H), h = (int)(tile % a.H);
-    const int len = a.tab.chunk_len[c], tok0 = a.tab.chunk_tok0[c];
+    const int len = a.tab.chunk_len(c), tok0 = a.tab.chunk_tok0(c);
     const Hyper hy = a.hy;
     const TI* kbase = static_cast<const TI*>(a.k);
     TO* tbase = static_cast<TO*>(a.ktil);
@@ -343,8 +343,8 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
         for (int r = 0; r < R; ++r) d[r] = 1.0f;
     }
     bool face = on_lower_face<R>(d, hy);
-    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
-    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
+    const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
+    const int seq_t0 = a.tab.seq_tok0(s), seq_len = a.tab.seq_len(s);
     for (int cbase = c0; cbase < c1; cbase += 32) {
         unsigned w0 = 0, w1 = 0;
         if (cbase + lane < c1) {
@@ -503,7 +503,7 @@ __global__ void __launch_bounds__(128) phase1_bwd_bulk_kernel(P1Bwd a)
     const int half = (int)(w & 1);
     if (tile >= (long)a.NT * a.H) return;
     const int c = (int)(tile / a.H), h = (int)(tile % a.H);
-    const int len = a.tab.chunk_len[c], tok0 = a.tab.chunk_tok0[c];
+    const int len = a.tab.chunk_len(c), tok0 = a.tab.chunk_tok0(c);
     const unsigned word = a.r.skipw[tile * 2 + half];
     T* dkp = static_cast<T*>(a.dk);
     for (int j = 0; j < 32; ++j) {
@@ -552,8 +552,8 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
 #pragma unroll
         for (int r = 0; r < R; ++r) lam[r] = kk[r] * dk[r];
     };
-    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
-    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
+    const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
+    const int seq_t0 = a.tab.seq_tok0(s), seq_len = a.tab.seq_len(s);
     for (int ctop = c1; ctop > c0; ctop -= 32) {
         // lane j holds the words of chunk ctop - 1 - j
         unsigned w0 = 0, w1 = 0;

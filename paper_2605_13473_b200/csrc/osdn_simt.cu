@@ -59,9 +59,9 @@ build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Ta
         const int carry = s_carry;
         if (s < S) {
             const int c = min(carry + s_scan[tid] - nc, NTmax);
-            t.seq_tok0[s] = t0;
-            t.seq_len[s] = len;
-            t.seq_chunk0[s] = c;
+            t.seq_tok0_[s] = t0;
+            t.seq_len_[s] = len;
+            t.seq_chunk0_[s] = c;
             if (s <= TBL_SMEM_SEQ) s_c0[s] = c;
         }
         __syncthreads();
@@ -70,34 +70,34 @@ build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Ta
     }
     const int total = min(s_carry, NTmax);
     if (tid == 0) {
-        t.seq_chunk0[S] = total;
+        t.seq_chunk0_[S] = total;
         if (S <= TBL_SMEM_SEQ) s_c0[S] = total;
     }
     __syncthreads();
     const bool in_smem = S <= TBL_SMEM_SEQ;
     for (int j = tid; j < NTmax; j += TBL_THREADS) {
         if (j >= total) {
-            t.chunk_tok0[j] = 0;
-            t.chunk_len[j] = 0;
-            t.chunk_seq[j] = 0;
+            t.chunk_tok0_[j] = 0;
+            t.chunk_len_[j] = 0;
+            t.chunk_seq_[j] = 0;
             continue;
         }
         int lo = 0, hi = S - 1;   // last sequence whose first chunk is <= j (empty sequences share an offset)
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
-            const int c = in_smem ? s_c0[mid] : t.seq_chunk0[mid];
+            const int c = in_smem ? s_c0[mid] : t.seq_chunk0_[mid];
             if (c <= j) lo = mid;
             else hi = mid - 1;
         }
         const int s = lo;
-        const int c0 = in_smem ? s_c0[s] : t.seq_chunk0[s];
+        const int c0 = in_smem ? s_c0[s] : t.seq_chunk0_[s];
         const int t0 = cu ? cu[s] : s * T_dense;
         int len = cu ? cu[s + 1] - cu[s] : T_dense;
         if (len < 0) len = 0;
         const int rem = len - (j - c0) * CH;
-        t.chunk_tok0[j] = t0 + (j - c0) * CH;
-        t.chunk_len[j] = rem < CH ? rem : CH;
-        t.chunk_seq[j] = s;
+        t.chunk_tok0_[j] = t0 + (j - c0) * CH;
+        t.chunk_len_[j] = rem < CH ? rem : CH;
+        t.chunk_seq_[j] = s;
     }
 }
 
@@ -236,9 +236,9 @@ __global__ void __launch_bounds__(NTH) chunk_local_fwd_kernel(ChunkArgs a)
     __shared__ GateVecs gv;
 
     const int c = blockIdx.x, h = blockIdx.y, H = a.H;
-    const int len = a.tab.chunk_len[c];
+    const int len = a.tab.chunk_len(c);
     if (len == 0) return;
-    const int tok0 = a.tab.chunk_tok0[c];
+    const int tok0 = a.tab.chunk_tok0(c);
     const size_t tile = (size_t)c * H + h;
 
     load_tile<T, K>(sK, LD, static_cast<const T*>(a.k), tok0, len, H, h);
@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(NTH) chain_fwd_kernel(ChainArgs a)
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
     const int v0 = blockIdx.y * VS;
-    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
     const float scale = a.hy.scale;
 
     for (int e = threadIdx.x; e < VS * K; e += NTH) {
@@ -334,7 +334,7 @@ __global__ void __launch_bounds__(NTH) chain_fwd_kernel(ChainArgs a)
     }
     T* outp = static_cast<T*>(a.out);
     for (int c = c0; c < c1; ++c) {
-        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+        const int tok0 = a.tab.chunk_tok0(c), len = a.tab.chunk_len(c);
         const size_t tile = (size_t)c * H + h;
         __syncthreads();
         for (int e = threadIdx.x; e < CH * K; e += NTH) sW[(e / K) * LD + e % K] = a.W[tile * CH * K + e];
@@ -400,7 +400,7 @@ __global__ void __launch_bounds__(NTH) chain_bwd_kernel(ChainArgs a)
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
     const int v0 = blockIdx.y * VS;
-    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
+    const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
     const float scale = a.hy.scale;
 
     for (int e = threadIdx.x; e < VS * K; e += NTH) {
@@ -409,7 +409,7 @@ __global__ void __launch_bounds__(NTH) chain_bwd_kernel(ChainArgs a)
     }
     const T* dop = static_cast<const T*>(a.dout);
     for (int c = c1 - 1; c >= c0; --c) {
-        const int tok0 = a.tab.chunk_tok0[c], len = a.tab.chunk_len[c];
+        const int tok0 = a.tab.chunk_tok0(c), len = a.tab.chunk_len(c);
         const size_t tile = (size_t)c * H + h;
         __syncthreads();
         for (int e = threadIdx.x; e < CH * K; e += NTH) sW[(e / K) * LD + e % K] = a.W[tile * CH * K + e];
@@ -464,9 +464,9 @@ __global__ void __launch_bounds__(NTH) chunk_local_bwd_kernel(ChunkArgs a)
     __shared__ float sdG[CH], sdB[CH], sR[CH], sRed[NTH / 32];
 
     const int c = blockIdx.x, h = blockIdx.y, H = a.H;
-    const int len = a.tab.chunk_len[c];
+    const int len = a.tab.chunk_len(c);
     if (len == 0) return;
-    const int tok0 = a.tab.chunk_tok0[c];
+    const int tok0 = a.tab.chunk_tok0(c);
     const size_t tile = (size_t)c * H + h;
     const float scale = a.hy.scale;
 
@@ -728,8 +728,9 @@ int bwd_impl(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws,
 int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st)
 {
     Table tab = carve_table(ws, L);
+    if (L.dense_T) return 0;   // dense batch: the table is arithmetic, nothing to build
     stage_mark(st, "build_table");
-    build_table_kernel<<<1, TBL_THREADS, 0, st>>>(L.S, p.T, p.nseq > 0 ? p.cu_seqlens : nullptr, L.NTmax, tab);
+    build_table_kernel<<<1, TBL_THREADS, 0, st>>>(L.S, p.T, p.cu_seqlens, L.NTmax, tab);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -333,9 +333,9 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     __shared__ __align__(16) float sG[CH], sBeta[CH];
 
     const int c = blockIdx.x, h = blockIdx.y, H = a.H;
-    const int len = a.tab.chunk_len[c];
+    const int len = a.tab.chunk_len(c);
     if (len == 0) return;
-    const int tok0 = a.tab.chunk_tok0[c];
+    const int tok0 = a.tab.chunk_tok0(c);
     const size_t tile = (size_t)c * H + h;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, half = warp >> 2;
@@ -632,8 +632,8 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
-    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
-    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
+    const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
+    const int seq_t0 = a.tab.seq_tok0(s), seq_len = a.tab.seq_len(s);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, colq = (warp >> 2) & 3;
     const int v = quad * 32 + lane;             // state row owned by a state-warp thread
@@ -1059,8 +1059,8 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
 
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
-    const int c0 = a.tab.seq_chunk0[s], c1 = a.tab.seq_chunk0[s + 1];
-    const int seq_t0 = a.tab.seq_tok0[s], seq_len = a.tab.seq_len[s];
+    const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
+    const int seq_t0 = a.tab.seq_tok0(s), seq_len = a.tab.seq_len(s);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, colq = (warp >> 2) & 3;
     const int v = quad * 32 + lane;
@@ -1402,7 +1402,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // are requested in two batches as soon as the shared-memory regions they land in are dead, and
     // its per-token scalars are fetched into registers one tile ahead.
     auto next_tile = [&](int t) {   // first non-empty tile of this CTA at or after t
-        while (t < a.ntiles && a.tab.chunk_len[(int)(t / H)] == 0) t += (int)gridDim.x;
+        while (t < a.ntiles && a.tab.chunk_len((int)(t / H)) == 0) t += (int)gridDim.x;
         return t;
     };
     // The copies of a tile arrive on one barrier phase; the transaction count is announced with the
@@ -1440,8 +1440,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     int tok0 = 0, len = 0;
     float g_cur = 0.f, b_cur = 0.f;
     if (tile_l < a.ntiles) {
-        tok0 = a.tab.chunk_tok0[(int)(tile_l / H)];
-        len = a.tab.chunk_len[(int)(tile_l / H)];
+        tok0 = a.tab.chunk_tok0((int)(tile_l / H));
+        len = a.tab.chunk_len((int)(tile_l / H));
         if (tid == 0) {
             expect_all();
             issue_first(tile_l, tok0);
@@ -1469,8 +1469,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     int tok0_next = 0, len_next = 0;
     float g_next = 0.f, b_next = 0.f;
     if (tile_next < a.ntiles) {
-        tok0_next = a.tab.chunk_tok0[(int)(tile_next / H)];
-        len_next = a.tab.chunk_len[(int)(tile_next / H)];
+        tok0_next = a.tab.chunk_tok0((int)(tile_next / H));
+        len_next = a.tab.chunk_len((int)(tile_next / H));
         fetch_scalars(tile_next, tok0_next, len_next, g_next, b_next);
     }
 
