@@ -23,17 +23,6 @@
 
 namespace osdn {
 
-#ifdef OSDN_PHASE_CLOCKS
-__device__ long long g_clk_p1[64];
-__device__ int g_clk_p1_n;
-#define P1_STAMP(cond)                                                     \
-    do {                                                                   \
-        if ((cond) && p1_stamp_n < 64) g_clk_p1[p1_stamp_n++] = clock64();  \
-    } while (0)
-#else
-#define P1_STAMP(cond)
-#endif
-
 namespace {
 
 __device__ __forceinline__ float warp_sum(float x)
@@ -538,10 +527,6 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
 #pragma unroll
         for (int r = 0; r < R; ++r) lam[r] = 0.f;
     }
-#ifdef OSDN_PHASE_CLOCKS
-    int p1_stamp_n = 0;
-#endif
-    P1_STAMP(chain == 0 && lane == 0);
     bool lam_valid = true;     // lam holds dL/dd_{t+1} for the token about to be processed
     long src = -1;             // otherwise it is k (.) dktil of this (skipped) token
     auto restart = [&](long tsrc) {
@@ -637,7 +622,6 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                 }
             };
             unsigned long long pfm = todo, rem = todo;
-            P1_STAMP(chain == 0 && lane == 0);
 #pragma unroll
             for (int u = 0; u < PF; ++u)
                 if (pfm) fetch(pop_top(pfm), u);
@@ -687,7 +671,6 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                             if (hy.apf_mode == 1) atomicAdd(&a.dgate[th], rho * drho);
                             if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
                         }
-                        P1_STAMP(chain == 0 && lane == 0);
                     }
                 }
             }
@@ -700,10 +683,6 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
         if (!lam_valid) restart(src);
         store_row<R>(a.dprecond_in + ((size_t)s * H + h) * K, lane, lam);
     }
-    P1_STAMP(chain == 0 && lane == 0);
-#ifdef OSDN_PHASE_CLOCKS
-    if (chain == 0 && lane == 0) g_clk_p1_n = p1_stamp_n;
-#endif
 }
 
 template <typename TI, typename TO, int K>
@@ -788,11 +767,3 @@ int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const fl
 }
 
 }  // namespace osdn
-
-#ifdef OSDN_PHASE_CLOCKS
-extern "C" int osdn_debug_clocks_p1(long long* out, int* n)
-{
-    if (cudaMemcpyFromSymbol(out, osdn::g_clk_p1, sizeof(long long) * 64) != cudaSuccess) return -1;
-    return cudaMemcpyFromSymbol(n, osdn::g_clk_p1_n, sizeof(int)) == cudaSuccess ? 0 : -1;
-}
-#endif

@@ -31,22 +31,14 @@ namespace osdn {
 using namespace umma;
 
 // Developer aid (compiled only with -DOSDN_PHASE_CLOCKS): clock64 stamps of one CTA at the phase
-// boundaries of each tensor-core kernel, read back with osdn_debug_clocks.
+// boundaries of each tensor-core kernel, and accumulated waiting times of single threads, read back
+// with osdn_debug_clocks.  The stamps are kept in shared memory until the kernel ends: a global store
+// inside a loop would itself delay the tensor-memory loads that follow it.
 #ifdef OSDN_PHASE_CLOCKS
 __device__ long long g_clk[4][32];
-#define OSDN_CLK(k, i, cond)                                          \
-    do {                                                              \
-        if ((cond) && threadIdx.x == 0) g_clk[k][i] = clock64();      \
-    } while (0)
 #ifndef OSDN_CLK_MASK
 #define OSDN_CLK_MASK 0xffffffffu
 #endif
-#define OSDN_CLKW(k, i, cond)                                         \
-    do {                                                              \
-        if (((OSDN_CLK_MASK >> (i)) & 1u) && (cond)) g_clk[k][i] = clock64(); \
-    } while (0)
-// stamps kept in shared memory until the kernel ends (a global store in the loop would itself stall
-// the tensor-memory loads that follow it)
 #define OSDN_CLKS(i, cond)                                            \
     do {                                                              \
         if (((OSDN_CLK_MASK >> (i)) & 1u) && (cond)) s_clk[i] = clock64(); \
@@ -59,14 +51,16 @@ __device__ long long g_clk[4][32];
         stmt;                                                         \
         acc_clk[slot] += clock64() - t_acc0;                          \
     } while (0)
+#ifdef OSDN_ACC_OFF   // the sums share the stamp slots: build with one or the other
+#define OSDN_ACC_DUMP(base, count, cond)
+#else
 #define OSDN_ACC_DUMP(base, count, cond)                              \
     do {                                                              \
         if (cond)                                                     \
             for (int i_acc = 0; i_acc < (count); ++i_acc) s_clk[(base) + i_acc] = acc_clk[i_acc]; \
     } while (0)
+#endif
 #else
-#define OSDN_CLK(k, i, cond)
-#define OSDN_CLKW(k, i, cond)
 #define OSDN_CLKS(i, cond)
 #define OSDN_ACC_DECL
 #define OSDN_ACC(slot, stmt) stmt
