@@ -1433,7 +1433,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     int tile_l = next_tile((int)blockIdx.x);
     int tok0 = 0, len = 0;
     float g_cur = 0.f, b_cur = 0.f;
+    unsigned long long sk_cur = 0ull;
     if (tile_l < a.ntiles) {
+        sk_cur = (unsigned long long)a.skipw[(size_t)tile_l * 2] | ((unsigned long long)a.skipw[(size_t)tile_l * 2 + 1] << 32);
         tok0 = a.tab.chunk_tok0((int)(tile_l / H));
         len = a.tab.chunk_len((int)(tile_l / H));
         if (tid == 0) {
@@ -1445,7 +1447,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fetch_scalars(tile_l, tok0, len, g_cur, b_cur);
     }
     while (tile_l < a.ntiles) {
-    const size_t tile = (size_t)tile_l;
     const int h = (int)(tile_l % H);
     const bool clk = tile_l == 1603;
     (void)clk;
@@ -1468,9 +1469,13 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fetch_scalars(tile_next, tok0_next, len_next, g_next, b_next);
     }
 
-    // skip words of this tile (every thread reads the same two words; used in the final epilogue)
-    const unsigned long long sk =
-        (unsigned long long)a.skipw[tile * 2] | ((unsigned long long)a.skipw[tile * 2 + 1] << 32);
+    // skip words (every thread reads the same two words), like the scalars fetched one tile ahead so
+    // that nothing at the top of a tile waits for memory
+    const unsigned long long sk = sk_cur;
+    unsigned long long sk_next = 0ull;
+    if (tile_next < a.ntiles)
+        sk_next = (unsigned long long)a.skipw[(size_t)tile_next * 2] |
+                  ((unsigned long long)a.skipw[(size_t)tile_next * 2 + 1] << 32);
     // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's preconditioner
     // step was skipped); ragged or mixed chunks are copied row by row.  In the all-skipped case the
     // space of each chain tile is not reused by the output staging, so the next tile's copy of it
@@ -1478,30 +1483,21 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const bool full = len == CH;
     const bool dk_tile = full && sk == ~0ull;
     const bool early = dk_tile && tile_next < a.ntiles;
-    if (tid == 64 && tile_next < a.ntiles) {   // warm L2 with everything the next tile will ask for
-        const int hh = (int)(tile_next % H);
-        for (int hf = 0; hf < 2; ++hf) {
-            tma_prefetch_2d(&tmQ, hh * KD + hf * 64, tok0_next);
-            tma_prefetch_2d(&tmK, hh * KD + hf * 64, tok0_next);
-            tma_prefetch_2d(&tmKt, hh * KD + hf * 64, tok0_next);
-            tma_prefetch_2d(&tmV, hh * KD + hf * 64, tok0_next);
-            tma_prefetch_2d(&tmDO, hh * KD + hf * 64, tok0_next);
+    if (warp == 0) {   // in-chunk gate prefix G_i and the decay vectors (lane: tokens l and l + 32)
+        float sa = sg[lane], sb = sg[lane + 32];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float ua = __shfl_up_sync(0xffffffffu, sa, o), ub = __shfl_up_sync(0xffffffffu, sb, o);
+            if (lane >= o) { sa += ua; sb += ub; }
         }
-        bulk_prefetch(a.dUT + (size_t)tile_next * 16384, 16384);
-        bulk_prefetch(a.ddUT + (size_t)tile_next * 16384, 16384);
-        bulk_prefetch(a.Tm + (size_t)tile_next * 8192, 8192);
-        bulk_prefetch(a.Sn + (size_t)tile_next * 32768, 32768);
-        bulk_prefetch(a.dSn + (size_t)tile_next * 32768, 32768);
-    }
-    if (tid < CH) {
-        float acc = 0.f, tot = 0.f;
-        for (int j = 0; j < CH; ++j) {
-            tot += sg[j];
-            if (j <= tid) acc += sg[j];
-        }
-        sG[tid] = acc;
-        sGam[tid] = __expf(acc);
-        sRho[tid] = __expf(tot - acc);
+        sb += __shfl_sync(0xffffffffu, sa, 31);
+        const float tot = __shfl_sync(0xffffffffu, sb, 31);
+        sG[lane] = sa;
+        sG[lane + 32] = sb;
+        sGam[lane] = __expf(sa);
+        sGam[lane + 32] = __expf(sb);
+        sRho[lane] = __expf(tot - sa);
+        sRho[lane + 32] = __expf(tot - sb);
     }
     bool ok = mbar_wait(&bar_tma, ph, a.status, ERR_TMA);
     OSDN_CLKS(1, threadIdx.x == 0 && clk);
@@ -1994,6 +1990,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     len = len_next;
     g_cur = g_next;
     b_cur = b_next;
+    sk_cur = sk_next;
     }   // tile loop
     if (tid == 0) bulk_wait_all();
     tc_fence_before();
