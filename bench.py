@@ -30,6 +30,8 @@ WORKLOADS = {
     "cfg2": dict(idx=2, bwd=True, desc="cfg2 340M layer train step (fwd+bwd): B=8 T=2048 H=8 dk=dv=128 bf16"),
     "cfg3": dict(idx=3, bwd=True, desc="cfg3 1.3B layer fwd+bwd: B=4 T=4096 H=16 dk=dv=128 bf16, mixture gates"),
     "cfg4": dict(idx=4, bwd=True, desc="cfg4 varlen fwd+bwd: 8 packed sequences, 131072 tokens, H=8 dk=dv=128 bf16"),
+    "osdn_1p3b": dict(idx=-3, bwd=True, desc="ungated 1.3B OSDN setting (g = 0, separate retention near 0.999, "
+                                             "non-beta-aware step): B=4 T=4096 H=16 dk=dv=128 bf16"),
     "cfg2_lively": dict(idx=-2, bwd=True, desc="cfg2 shape with a moving preconditioner (eta=0.3, sparse keys, "
                                                "separate retention): B=8 T=2048 H=8 dk=dv=128 bf16"),
 }
@@ -51,6 +53,10 @@ def make_inputs(name):
     w = WORKLOADS[name]
     if w["idx"] >= 0:
         return config(w["idx"])
+    if w["idx"] == -3:
+        hy = OsdnHyper(eta=0.003, apf_mode=2, beta_aware=0)
+        return draw("osdn_1p3b", 13, [4096] * 4, 16, 128, 128, "bf16", dense_B=4, hyper=hy, gate_kind="zero",
+                    with_dout=True, with_log_ret=True, log_ret_shift=7.0)
     hy = OsdnHyper(eta=0.3, apf_mode=2)
     return draw("cfg2_lively", 12, [2048] * 8, 8, 128, 128, "bf16", dense_B=8, hyper=hy, key_kind="sparse",
                 with_dout=True, with_log_ret=True)

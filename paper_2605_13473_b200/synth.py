@@ -105,6 +105,7 @@ def draw(
     with_state: bool = False,
     with_log_ret: bool = False,
     with_state_cotangents: bool = False,
+    log_ret_shift: float = 5.0,
 ) -> OsdnInputs:
     """Draw one input set.  Draw order: q, k, v, beta, gate, then optionals."""
     hyper = hyper or OsdnHyper()
@@ -168,7 +169,7 @@ def draw(
     if with_dout:
         out.dout = _round_io(randn(T, H, V), io_dtype)
     if with_log_ret:
-        out.log_ret = torch.nn.functional.logsigmoid(randn(T, H) + 5.0).contiguous()
+        out.log_ret = torch.nn.functional.logsigmoid(randn(T, H) + log_ret_shift).contiguous()
     if with_state:
         out.init_state = 0.5 * randn(nseq, H, V, K)
         out.precond_in = hyper.d_min + (hyper.d_max - hyper.d_min) * rand(nseq, H, K)
@@ -265,4 +266,8 @@ def lively(idx: int, *, T: int = 200, B: int = 2, H: int = 2, D: int = 128,
         hy = OsdnHyper(eta=0.2, apf_mode=2, beta_aware=0)
         return draw("lively5_rawkeys", 105, lens, H, D, D, io_dtype, dense_B=B, hyper=hy,
                     key_kind="raw", with_dout=True, with_log_ret=True)
+    if idx == 6:  # the ungated 1.3B OSDN setting: g = 0, separate retention near 0.999, non-beta-aware step
+        hy = OsdnHyper(eta=0.003, apf_mode=2, beta_aware=0)
+        return draw("lively6_ungated_osdn", 106, lens, H, D, D, io_dtype, dense_B=B, hyper=hy,
+                    gate_kind="zero", with_dout=True, with_log_ret=True, log_ret_shift=7.0)
     raise ValueError(idx)

@@ -57,7 +57,7 @@ def test_benchmark_configs_reduced(idx, path, flags):
 
 @pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])
 @pytest.mark.parametrize("io", ["fp32", "bf16"])
-@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5, 6])
 def test_lively_sets(idx, io, path, flags):
     if io == "fp32" and path == "auto":
         pytest.skip("fp32 I/O always runs the CUDA-core kernels")
