@@ -82,7 +82,9 @@ def fwd(hy, seq_lens, q, k, v, beta, gate, log_ret=None, init_state=None, precon
     nseq = len(seq_lens)
     assert cu[-1] == T
     if hy.apf_mode == 2:
-        assert log_ret is not None
+        assert log_ret is not None and log_ret.shape == (T, H)
+    if hy.apf_mode == 3:
+        assert log_ret is not None and log_ret.shape == (T, H, K)
     out = np.zeros((T, H, V))
     S = np.zeros((nseq, H, V, K))
     d = np.zeros((nseq, H, K))
@@ -134,7 +136,8 @@ def bwd(hy, seq_lens, q, k, v, beta, gate, dout, log_ret=None, init_state=None, 
     cu = _cu(seq_lens)
     nseq = len(seq_lens)
     dq, dk, dv = np.zeros((T, H, K)), np.zeros((T, H, K)), np.zeros((T, H, V))
-    dbeta, dgate, dlr = np.zeros((T, H)), np.zeros((T, H)), np.zeros((T, H))
+    dbeta, dgate = np.zeros((T, H)), np.zeros((T, H))
+    dlr = np.zeros((T, H, K)) if hy.apf_mode == 3 else np.zeros((T, H))
     dS0, dd0 = np.zeros((nseq, H, V, K)), np.zeros((nseq, H, K))
     hp = _hyper(hy, K)
     mo = None if mask_override is None else np.ascontiguousarray(mask_override, dtype=np.uint8)

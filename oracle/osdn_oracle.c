@@ -17,6 +17,8 @@
  *       c      = eta * b * (1 - b a) / n
  *       rho    = 1 | exp(g_t) | exp(l_t)           (no APF | aliased | separate)
  *       dbar   = rho d_t + c kap ;  d_{t+1} = clip(dbar, d_min, d_max)
+ *   apf_mode 3, the vector-retention extension of the affine form of the update
+ *   (diag(r_t) in place of r_t I): dbar = exp(l_t) (.) d_t + c kap with l_t in R^K.
  *
  *   phase 2 (gated, online-scaled delta rule of the backbone-extension
  *   appendix, post-gate residual):
@@ -63,10 +65,17 @@ int osdn_oracle_threads(void)
 #endif
 }
 
+/* Retention inputs of token-head th: apf_mode 2 reads one log-retention per
+ * token-head, apf_mode 3 (vector retention, diag(r_t) in place of r_t I in the
+ * affine form of the update) one per coordinate. */
+#define LRET_S(hp, lr, th) (((lr) && (hp)->apf_mode != 3) ? (lr)[th] : 0.0)
+#define LRET_V(hp, lr, th, K) (((lr) && (hp)->apf_mode == 3) ? (lr) + (th) * (size_t)(K) : (const double *)0)
+
 /* One phase-1 step.  Reads d (length K) and overwrites it with d_{t+1}.
- * Optionally reports ktil, the scalar c and the pass-through mask. */
+ * Optionally reports ktil, the scalar c and the pass-through mask.
+ * lret_vec (apf_mode 3 only): K log-retentions, one per coordinate. */
 static void phase1_step(const oracle_hyper *hp, int K, const double *k, double beta,
-                        double g, double lret, double *d, double *ktil,
+                        double g, double lret, const double *lret_vec, double *d, double *ktil,
                         double *c_out, double *rho_out, double *a_out, double *n_out,
                         int *raw_norm_above_eps, unsigned char *mask, double *margin)
 {
@@ -84,7 +93,8 @@ static void phase1_step(const oracle_hyper *hp, int K, const double *k, double b
     if (hp->apf_mode == 1) rho = exp(g);
     else if (hp->apf_mode == 2) rho = exp(lret);
     for (int i = 0; i < K; ++i) {
-        double dbar = rho * d[i] + c * k[i] * k[i];
+        double ri = (hp->apf_mode == 3 && lret_vec) ? exp(lret_vec[i]) : rho;
+        double dbar = ri * d[i] + c * k[i] * k[i];
         unsigned char m = 1;
         if (margin) {
             double lo = fabs(dbar - hp->d_min), hi = fabs(dbar - hp->d_max);
@@ -125,7 +135,7 @@ static void phase2_step(int K, int V, const double *k, const double *ktil, const
 }
 
 /*
- * Forward.  Nullable: log_ret (unless apf_mode 2), S0 (zeros), d0 (ones),
+ * Forward.  Nullable: log_ret (needed for apf_mode 2: [T,H]; 3: [T,H,K]), S0 (zeros), d0 (ones),
  * ktil_out, d_traj_out ([T_total, H, K], the PRE-update d_t of every token).
  */
 void osdn_oracle_fwd(int nseq, const int *cu, int H, int K, int V, const oracle_hyper *hp,
@@ -150,7 +160,7 @@ void osdn_oracle_fwd(int nseq, const int *cu, int H, int K, int V, const oracle_
             size_t th = (size_t)t * H + h;
             const double *kt = k + th * K, *qt = q + th * K, *vt = v + th * V;
             if (d_traj_out) memcpy(d_traj_out + th * K, d, sizeof(double) * K);
-            phase1_step(hp, K, kt, beta[th], gate[th], log_ret ? log_ret[th] : 0.0, d, ktil,
+            phase1_step(hp, K, kt, beta[th], gate[th], LRET_S(hp, log_ret, th), LRET_V(hp, log_ret, th, K), d, ktil,
                         0, 0, 0, 0, 0, mask_out ? mask_out + th * K : 0, margin_out ? margin_out + th * K : 0);
             if (ktil_out) memcpy(ktil_out + th * K, ktil, sizeof(double) * K);
             phase2_step(K, V, kt, ktil, vt, beta[th], gate[th], S, 0);
@@ -182,7 +192,7 @@ void osdn_oracle_precond_update(int nseq, const int *cu, int H, int K, const ora
         for (int t = cu[s]; t < cu[s + 1]; ++t) {
             size_t th = (size_t)t * H + h;
             phase1_step(hp, K, k + th * K, beta[th], gate ? gate[th] : 0.0,
-                        log_ret ? log_ret[th] : 0.0, d, ktil, 0, 0, 0, 0, 0, 0, 0);
+                        LRET_S(hp, log_ret, th), LRET_V(hp, log_ret, th, K), d, ktil, 0, 0, 0, 0, 0, 0, 0);
             if (ktil_out) memcpy(ktil_out + th * K, ktil, sizeof(double) * K);
         }
         memcpy(d_final + ((size_t)s * H + h) * K, d, sizeof(double) * K);
@@ -195,7 +205,7 @@ void osdn_oracle_precond_update(int nseq, const int *cu, int H, int K, const ora
  *
  * Cotangents in: dout [T,H,V]; dS_final, dd_final nullable (zeros).
  * Gradients out: dq, dk [T,H,K], dv [T,H,V], dbeta, dgate [T,H],
- * dlog_ret [T,H] (nullable; written only for apf_mode 2), dS0, dd0 (nullable).
+ * dlog_ret [T,H] for apf_mode 2, [T,H,K] for apf_mode 3 (nullable), dS0, dd0 (nullable).
  *
  * S_{t-1} and d_t are needed in reverse order.  Each chain keeps S and d at
  * every SEG-token boundary during a forward sweep, then walks the segments
@@ -257,8 +267,8 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
             int a0 = t0 + sg * SEG, a1 = a0 + SEG < t1 ? a0 + SEG : t1;
             for (int t = a0; t < a1; ++t) {
                 size_t th = (size_t)t * H + h;
-                phase1_step(hp, K, k + th * K, beta[th], gate[th], log_ret ? log_ret[th] : 0.0,
-                            d, ktil, 0, 0, 0, 0, 0, 0, 0);
+                phase1_step(hp, K, k + th * K, beta[th], gate[th], LRET_S(hp, log_ret, th),
+                            LRET_V(hp, log_ret, th, K), d, ktil, 0, 0, 0, 0, 0, 0, 0);
                 phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
             }
         }
@@ -276,8 +286,8 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 size_t th = (size_t)t * H + h;
                 memcpy(Shist + (size_t)(t - a0) * VK, S, sizeof(double) * VK);
                 memcpy(dhist + (size_t)(t - a0) * K, d, sizeof(double) * K);
-                phase1_step(hp, K, k + th * K, beta[th], gate[th], log_ret ? log_ret[th] : 0.0,
-                            d, ktil, 0, 0, 0, 0, 0, 0, 0);
+                phase1_step(hp, K, k + th * K, beta[th], gate[th], LRET_S(hp, log_ret, th),
+                            LRET_V(hp, log_ret, th, K), d, ktil, 0, 0, 0, 0, 0, 0, 0);
                 phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
             }
             for (int t = a1 - 1; t >= a0; --t) {
@@ -286,13 +296,14 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 const double *dot = dout + th * V;
                 const double *Sprev = Shist + (size_t)(t - a0) * VK;
                 const double *dt = dhist + (size_t)(t - a0) * K;
-                double bt = beta[th], gt = gate[th], lt = log_ret ? log_ret[th] : 0.0;
+                double bt = beta[th], gt = gate[th], lt = LRET_S(hp, log_ret, th);
+                const double *lv = LRET_V(hp, log_ret, th, K);
                 double alpha = exp(gt);
 
                 /* recompute this token's forward quantities */
                 double c, rho, a, n; int above;
                 memcpy(dnew, dt, sizeof(double) * K);
-                phase1_step(hp, K, kt, bt, gt, lt, dnew, ktil, &c, &rho, &a, &n, &above, mask, 0);
+                phase1_step(hp, K, kt, bt, gt, lt, lv, dnew, ktil, &c, &rho, &a, &n, &above, mask, 0);
                 if (mask_override)
                     for (int i = 0; i < K; ++i)
                         if (mask_override[th * K + i] != 255) mask[i] = mask_override[th * K + i];
@@ -357,10 +368,13 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                     double kap = kt[i] * kt[i];
                     double dkap = c * lam[i] + da * dt[i] + dn;
                     dk[th * K + i] += dt[i] * dktil[i] + 2.0 * kt[i] * dkap;
-                    lam[i] = rho * lam[i] + da * kap + kt[i] * dktil[i];   /* dL/dd_t */
+                    double ri = lv ? exp(lv[i]) : rho;
+                    /* vector retention: d(dbar_i)/d(l_i) = r_i d_i, one gradient per coordinate */
+                    if (lv && dlog_ret) dlog_ret[th * K + i] = ri * lam[i] * dt[i];
+                    lam[i] = ri * lam[i] + da * kap + kt[i] * dktil[i];   /* dL/dd_t */
                 }
                 if (hp->apf_mode == 1) dg_t += rho * drho;
-                if (dlog_ret) dlog_ret[th] = hp->apf_mode == 2 ? rho * drho : 0.0;
+                if (dlog_ret && !lv) dlog_ret[th] = hp->apf_mode == 2 ? rho * drho : 0.0;
                 dbeta[th] = dbeta_t;
                 dgate[th] = dg_t;
             }
