@@ -59,7 +59,10 @@ typedef enum osdn_status {
 } osdn_status;
 
 enum { OSDN_FP32 = 0, OSDN_BF16 = 1 };
-enum { OSDN_APF_NONE = 0, OSDN_APF_ALIAS_GATE = 1, OSDN_APF_SEPARATE = 2 };
+/* Retention of the preconditioner (Eq. "dt_update_apf"): none, the layer's gate, a separate
+ * log-retention per (token, head), or one per coordinate (the vector-retention extension of the
+ * update's affine form: diag(r_t) in place of r_t I). */
+enum { OSDN_APF_NONE = 0, OSDN_APF_ALIAS_GATE = 1, OSDN_APF_SEPARATE = 2, OSDN_APF_VECTOR = 3 };
 enum {
     OSDN_FLAG_SAVE_RESIDUALS = 1,  /* osdn_fwd: keep chunk residuals in the workspace for osdn_bwd */
     OSDN_FLAG_RESIDUALS_VALID = 2, /* osdn_bwd: the workspace holds the residuals of the matching
@@ -90,7 +93,8 @@ size_t osdn_workspace_bytes(const osdn_params* p, int need_bwd);
 /*
  * Forward (Algorithm 1 + the gated chunk form).
  *   in : q,k [T,H,K], v [T,H,V] io_dtype; beta, gate [T,H] fp32;
- *        apf_log_ret [T,H] fp32 (required iff apf_mode == SEPARATE, else may be NULL);
+ *        apf_log_ret fp32: [T,H] for apf_mode == SEPARATE, [T,H,K] for VECTOR (required for
+ *        these two modes, else may be NULL);
  *        init_state [S,H,V,K] (NULL = zeros); precond_in [S,H,K] (NULL = ones).
  *   out: out [T,H,V] io_dtype; final_state [S,H,V,K] and precond_out [S,H,K] fp32 (either may
  *        be NULL; precond_out may alias precond_in).
@@ -107,7 +111,8 @@ int osdn_fwd(const osdn_params* p, const void* q, const void* k, const void* v,
  * sum(precond_out*dprecond_out) with respect to every forward input.
  *   in : the forward inputs; dout [T,H,V] io_dtype; dfinal_state, dprecond_out (NULL = zeros).
  *   out: dq, dk [T,H,K], dv [T,H,V] io_dtype; dbeta, dgate [T,H] fp32;
- *        dapf_log_ret [T,H] (written iff apf_mode == SEPARATE; may be NULL otherwise);
+ *        dapf_log_ret, shaped like apf_log_ret (written iff apf_mode is SEPARATE or VECTOR; may be
+ *        NULL otherwise);
  *        dinit_state [S,H,V,K], dprecond_in [S,H,K] (either may be NULL).
  *   The projection passes gradient where d_min <= pre-projection value <= d_max;
  *   max(|k|^2, eps) passes gradient where |k|^2 > eps.
@@ -124,9 +129,9 @@ int osdn_bwd(const osdn_params* p, const void* q, const void* k, const void* v,
 /*
  * Phase 1 alone (Algorithm 1 as its own pass; Section 3.5 "Phase 1"): advances the
  * preconditioner over the given tokens and optionally emits the write keys.
- *   in : k [T,H,K] io_dtype; beta [T,H]; gate_or_log_ret [T,H] (the log-retention source:
- *        the gate for ALIAS_GATE, the separate log-retention for SEPARATE; may be NULL for
- *        APF_NONE); precond_in [S,H,K] (NULL = ones).
+ *   in : k [T,H,K] io_dtype; beta [T,H]; gate_or_log_ret (the log-retention source: the gate
+ *        [T,H] for ALIAS_GATE, the separate log-retention [T,H] for SEPARATE or [T,H,K] for VECTOR;
+ *        may be NULL for APF_NONE); precond_in [S,H,K] (NULL = ones).
  *   out: k_tilde_out [T,H,K] io_dtype (may be NULL); precond_out [S,H,K] (required; may alias
  *        precond_in).  Needs no workspace for dense batches; var-len reads cu_seqlens directly.
  */
@@ -143,7 +148,7 @@ int osdn_precond_update(const osdn_params* p, const void* k, const float* beta,
  * in one launch.  It is the recurrence osdn_fwd evaluates chunk by chunk, so a prefill with osdn_fwd
  * (final_state, precond_out) followed by this call continues the same sequence.
  *   in    : q, k [B,T,H,K], v [B,T,H,V] io_dtype; beta, gate [B,T,H] fp32; apf_log_ret [B,T,H]
- *           (required iff apf_mode == SEPARATE).  Dense batches only (p->nseq == 0).
+ *           (apf_mode == SEPARATE) or [B,T,H,K] (VECTOR), required for these two modes.  Dense batches only (p->nseq == 0).
  *   in/out: state [B,H,V,K] fp32 and precond [B,H,K] fp32, the caller's cache, updated in place.
  *   out   : out [B,T,H,V] io_dtype.
  * All pointers are DEVICE pointers, 16-byte aligned.  No workspace, nothing is allocated.  Any T >= 1

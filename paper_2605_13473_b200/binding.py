@@ -280,7 +280,11 @@ class DeviceBundle:
             self.dv = torch.empty(T, H, V, device=dev, dtype=dt)
             self.dbeta = torch.empty(T, H, device=dev, dtype=torch.float32)
             self.dgate = torch.empty(T, H, device=dev, dtype=torch.float32)
-            self.dlog_ret = torch.zeros(T, H, device=dev, dtype=torch.float32)
+            mode = int(self.params.apf_mode)
+            if mode >= 2:   # written in full by osdn_bwd ([T,H], or [T,H,K] for the vector retention)
+                self.dlog_ret = torch.full((T, H, K) if mode == 3 else (T, H), float("nan"), device=dev)
+            else:           # not touched by the library
+                self.dlog_ret = torch.zeros(T, H, device=dev, dtype=torch.float32)
             self.dinit_state = torch.empty(S, H, V, K, device=dev, dtype=torch.float32)
             self.dprecond_in = torch.empty(S, H, K, device=dev, dtype=torch.float32)
 

@@ -53,7 +53,7 @@ int validate(const osdn_params* p)
 {
     if (!p) return OSDN_INVALID_ARG;
     if (p->io_dtype != OSDN_FP32 && p->io_dtype != OSDN_BF16) return OSDN_INVALID_ARG;
-    if (p->apf_mode < 0 || p->apf_mode > 2) return OSDN_INVALID_ARG;
+    if (p->apf_mode < 0 || p->apf_mode > 3) return OSDN_INVALID_ARG;
     if (p->B <= 0 || p->H <= 0) return OSDN_INVALID_ARG;
     if (p->T <= 0) return OSDN_UNSUPPORTED_SHAPE;
     if (p->chunk != CH) return OSDN_UNSUPPORTED_SHAPE;
@@ -138,7 +138,7 @@ int osdn_fwd(const osdn_params* p, const void* q, const void* k, const void* v, 
     int rc = validate(p);
     if (rc != OSDN_OK) return rc;
     if (!q || !k || !v || !beta || !gate || !out || !workspace) return OSDN_INVALID_ARG;
-    if (p->apf_mode == OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
+    if (p->apf_mode >= OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
     const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, init_state, precond_in, out, final_state,
                           precond_out};
     for (const void* x : ptrs)
@@ -171,7 +171,7 @@ int osdn_bwd(const osdn_params* p, const void* q, const void* k, const void* v, 
     if (rc != OSDN_OK) return rc;
     if (!q || !k || !v || !beta || !gate || !dout || !dq || !dk || !dv || !dbeta || !dgate || !workspace)
         return OSDN_INVALID_ARG;
-    if (p->apf_mode == OSDN_APF_SEPARATE && (!apf_log_ret || !dapf_log_ret)) return OSDN_INVALID_ARG;
+    if (p->apf_mode >= OSDN_APF_SEPARATE && (!apf_log_ret || !dapf_log_ret)) return OSDN_INVALID_ARG;
     const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, init_state, precond_in, dout, dfinal_state,
                           dprecond_out, dq, dk, dv, dbeta, dgate, dapf_log_ret, dinit_state, dprecond_in};
     for (const void* x : ptrs)
@@ -233,7 +233,7 @@ int osdn_decode_step(const osdn_params* p, const void* q, const void* k, const v
     if (rc != OSDN_OK) return rc;
     if (p->nseq != 0) return OSDN_INVALID_ARG;   // a dense [B, T, H, *] block of new tokens
     if (!q || !k || !v || !beta || !gate || !state || !precond || !out) return OSDN_INVALID_ARG;
-    if (p->apf_mode == OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
+    if (p->apf_mode >= OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
     const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, state, precond, out};
     for (const void* x : ptrs)
         if (x && !aligned16(x)) return OSDN_MISALIGNED;
@@ -318,7 +318,7 @@ int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host,
     const bool bwd = dout_host != nullptr;
     if (!q_host || !k_host || !v_host || !beta_host || !gate_host || !out_host || !staging) return OSDN_INVALID_ARG;
     if (bwd && (!dq_host || !dk_host || !dv_host || !dbeta_host || !dgate_host)) return OSDN_INVALID_ARG;
-    if (p->apf_mode == OSDN_APF_SEPARATE) return OSDN_INVALID_ARG;
+    if (p->apf_mode >= OSDN_APF_SEPARATE) return OSDN_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(staging) & 255u) return OSDN_MISALIGNED;
     const Staging s = make_staging(*p, bwd);
     if (staging_bytes < s.total) return OSDN_WORKSPACE_TOO_SMALL;
@@ -435,7 +435,7 @@ int osdn_fwd_static(const osdn_params* p, const void* q, const void* k, const vo
     int rc = validate(p);
     if (rc != OSDN_OK) return rc;
     if (!q || !k || !v || !beta || !gate || !out) return OSDN_INVALID_ARG;
-    if (p->apf_mode == OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
+    if (p->apf_mode >= OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
     const void* ptrs[] = {q, k, v, beta, gate, apf_log_ret, init_state, precond_in, out, final_state,
                           precond_out};
     for (const void* x : ptrs)

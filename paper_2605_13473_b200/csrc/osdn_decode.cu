@@ -5,6 +5,7 @@
 //   alpha_t = exp(g_t)
 //   ktil_t  = d_t (.) k_t                               (write key from the PRE-update d)
 //   d_{t+1} = clip(rho_t d_t + c_t k_t^2)                c_t = eta b_t (1 - b_t <d_t, k_t^2>) / max(|k_t|^2, eps)
+//             (rho_t a scalar, or one retention per coordinate in the vector-retention mode)
 //   S_t     = alpha_t S_{t-1} + beta_t (v_t - alpha_t S_{t-1} k_t) ktil_t^T ,   o_t = scale S_t q_t
 //
 // exactly the recurrence the chunk path evaluates chunk by chunk, so that a prefill with osdn_fwd
@@ -92,7 +93,9 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
     dec_load<R>(a.precond + (size_t)chain * K, lane, d);
 
     // inputs of a token, fetched one token ahead
-    float kk[R], qq[R], vv[DEC_RW], bt, gt, lr;
+    float kk[R], qq[R], vv[DEC_RW], bt, gt, lr, lrv[R];
+#pragma unroll
+    for (int j = 0; j < R; ++j) lrv[j] = 0.f;
     auto fetch = [&](int t) {
         const size_t th = ((size_t)b * a.L + t) * a.H + h;
         dec_load<R>(kp + th * K, lane, kk);
@@ -102,6 +105,7 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
         bt = a.beta[th];
         gt = a.gate[th];
         lr = hy.apf_mode == 2 ? a.log_ret[th] : 0.f;
+        if (hy.apf_mode == 3) dec_load<R>(a.log_ret + th * K, lane, lrv);   // one log-retention per coordinate
     };
     fetch(0);
     for (int t = 0; t < a.L; ++t) {
@@ -111,7 +115,10 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
 #pragma unroll
         for (int r = 0; r < DEC_RW; ++r) v1[r] = vv[r];
         const float beta = bt, alpha = expf(gt);
-        const float rho = hy.apf_mode == 0 ? 1.0f : (hy.apf_mode == 1 ? alpha : expf(lr));
+        const float rho1 = hy.apf_mode == 0 ? 1.0f : (hy.apf_mode == 1 ? alpha : expf(lr));
+        float rho[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) rho[j] = hy.apf_mode == 3 ? expf(lrv[j]) : rho1;
         if (t + 1 < a.L) fetch(t + 1);
 
         // preconditioner step
@@ -130,7 +137,7 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
         const float c = hy.eta * bb * (1.0f - bb * al) / n;
 #pragma unroll
         for (int j = 0; j < R; ++j) {
-            float x = fmaf(c, kap[j], rho * d[j]);
+            float x = fmaf(c, kap[j], rho[j] * d[j]);
             if (hy.clamp) x = fminf(fmaxf(x, hy.d_min), hy.d_max);
             d[j] = x;
         }

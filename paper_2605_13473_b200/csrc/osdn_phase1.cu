@@ -34,11 +34,12 @@ __device__ __forceinline__ float warp_sum(float x)
 
 // One step of the recurrence on the warp-distributed vector d (lane l owns coordinates R l + r).
 //   c = eta b (1 - b <d, kap>) / n ;  x = rho d + c kap ;  d <- clip(x)
+// rho is given per owned coordinate (all equal unless the retention is a vector).
 // n_signed: max(sum kap, eps), negated when the floor eps is active.  pass[r]: ballot of the
 // coordinates whose projection passes gradient; all_low: every x strictly below d_min.
 template <int R>
-__device__ __forceinline__ void p1_step(float (&d)[R], const float (&kap)[R], float n, float b, float rho,
-                                        const Hyper& hy, unsigned (&pass)[R], bool& all_low, float& c_out,
+__device__ __forceinline__ void p1_step(float (&d)[R], const float (&kap)[R], float n, float b,
+                                        const float (&rho)[R], const Hyper& hy, unsigned (&pass)[R], bool& all_low, float& c_out,
                                         float& al_out)
 {
     float al = 0.f;
@@ -49,7 +50,7 @@ __device__ __forceinline__ void p1_step(float (&d)[R], const float (&kap)[R], fl
     bool low = true;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        float x = fmaf(c, kap[r], rho * d[r]);
+        float x = fmaf(c, kap[r], rho[r] * d[r]);
         bool p = true;
         if (hy.clamp) {
             p = (x >= hy.d_min) && (x <= hy.d_max);
@@ -134,7 +135,8 @@ struct P1Args {
     Hyper hy;
 };
 
-template <typename TI, typename TO, int K>
+// VEC: vector retention, retsrc is [T,H,K] (one log-retention per coordinate).
+template <typename TI, typename TO, int K, bool VEC>
 __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
 {
     constexpr int R = K / 32;
@@ -165,7 +167,16 @@ __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
         }
         const float n = fmaxf(sumk, hy.eps);
         const float b = hy.beta_aware ? a.beta[th] : 1.0f;
-        const float rho = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
+        float rho[R];
+        if constexpr (VEC) {
+            load_row<R>(a.retsrc + th * K, lane, rho);
+#pragma unroll
+            for (int r = 0; r < R; ++r) rho[r] = expf(rho[r]);
+        } else {
+            const float r1 = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
+#pragma unroll
+            for (int r = 0; r < R; ++r) rho[r] = r1;
+        }
         unsigned pass[R];
         bool low;
         float c, al;
@@ -224,7 +235,8 @@ __device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&x)[8])
 // read in full 128-byte lines and the sums need three shuffle rounds.  The step is taken from
 // d = d_min 1: then <d, k^2> = d_min sum k^2, and since x_r = rho d_min + c k_r^2 is monotone in k_r^2
 // for a fixed c, "every x_r below d_min" is decided by the largest (c >= 0) or smallest (c < 0) k_r^2.
-template <typename TI, typename TO, int K>
+// With a vector retention (VEC) rho differs per coordinate and every x_r is formed.
+template <typename TI, typename TO, int K, bool VEC>
 __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
 {
     constexpr int NV = K / 64;   // 8-value vectors per lane
@@ -248,7 +260,7 @@ __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
         float x[NV][8];
 #pragma unroll
         for (int v = 0; v < NV; ++v) load8(kbase + th * K + v * 64 + l8 * 8, x[v]);
-        const float ret = (in && hy.apf_mode != 0) ? a.retsrc[th] : 0.f;
+        const float ret = (!VEC && in && hy.apf_mode != 0) ? a.retsrc[th] : 0.f;
         const float b = (in && hy.beta_aware) ? a.beta[th] : 1.0f;
         float sumk = 0.f, kmax = 0.f, kmin = 3.0e38f;
 #pragma unroll
@@ -272,8 +284,23 @@ __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
         if (hy.clamp) {
             const float al = hy.d_min * sumk;
             const float cc = hy.eta * b * (1.0f - b * al) / n;
-            const float xtop = fmaf(cc, cc >= 0.f ? kmax : kmin, rho * hy.d_min);
-            low = in && xtop < hy.d_min;
+            if constexpr (VEC) {
+                bool below = true;
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    float lr[8];
+                    load8(a.retsrc + th * K + v * 64 + l8 * 8, lr);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        below = below && fmaf(cc, x[v][e] * x[v][e], expf(lr[e]) * hy.d_min) < hy.d_min;
+                }
+#pragma unroll
+                for (int o = 4; o > 0; o >>= 1) below = __shfl_xor_sync(0xffffffffu, (int)below, o) && below;
+                low = in && below;
+            } else {
+                const float xtop = fmaf(cc, cc >= 0.f ? kmax : kmin, rho * hy.d_min);
+                low = in && xtop < hy.d_min;
+            }
         }
         if (in && l8 == 0) {
             a.r.n[th] = sumk > hy.eps ? n : -n;
@@ -313,7 +340,7 @@ template <int R> __device__ __forceinline__ bool on_lower_face(const float (&d)[
 
 // one warp per chain.  Flag words are fetched for 32 chunks at a time (one chunk per lane); the
 // rows of the tokens that are really processed are prefetched a few tokens ahead.
-template <typename TI, typename TO, int K>
+template <typename TI, typename TO, int K, bool VEC>
 __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
 {
     constexpr int R = K / 32;
@@ -351,6 +378,7 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
                     m &= m - 1;
                     const size_t th = (size_t)(seq_t0 + (cl - c0) * CH + t) * H + h;
                     prefetch_row(kp + th * K, K * (int)sizeof(TI));
+                    if constexpr (VEC) prefetch_row(a.retsrc + th * K, K * 4);
                     prefetch_l2(a.r.n + th);
                     prefetch_l2(a.r.rho + th);
                     prefetch_l2(a.beta + th);
@@ -397,10 +425,12 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
             } else {
                 // ring of prefetched rows and scalars
                 float kbuf[PF][R], nbuf[PF], rbuf[PF], bbuf[PF];
+                float lbuf[VEC ? PF : 1][R];   // log-retention rows (vector retention only)
                 auto fetch = [&](int i, int slot) {
                     const int ii = min(i, len - 1);
                     const size_t th = (size_t)(tok0 + ii) * H + h;
                     load_row<R>(kp + th * K, lane, kbuf[slot]);
+                    if constexpr (VEC) load_row<R>(a.retsrc + th * K, lane, lbuf[slot]);
                     nbuf[slot] = a.r.n[th];
                     rbuf[slot] = a.r.rho[th];
                     bbuf[slot] = hy.beta_aware ? a.beta[th] : 1.0f;
@@ -428,7 +458,13 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
                                 float kk[R];
 #pragma unroll
                                 for (int r = 0; r < R; ++r) kk[r] = kbuf[u][r];
-                                const float n = fabsf(nbuf[u]), rho = rbuf[u], b = bbuf[u];
+                                const float n = fabsf(nbuf[u]), b = bbuf[u];
+                                float rho[R];
+#pragma unroll
+                                for (int r = 0; r < R; ++r) {
+                                    if constexpr (VEC) rho[r] = expf(lbuf[u][r]);
+                                    else rho[r] = rbuf[u];
+                                }
                                 fetch(i + PF, u);
                                 const size_t th = (size_t)(tok0 + i) * H + h;
                                 float kap[R], wk[R];
@@ -475,6 +511,7 @@ struct P1Bwd {
     Table tab;
     const void* k;
     const float *beta, *dktil, *dkread, *dprecond_out;
+    const float* log_ret;   // [T,H,K], vector retention only
     void* dk;
     float *dbeta, *dgate, *dlog_ret, *dprecond_in;
     P1Regions r;
@@ -510,7 +547,7 @@ __global__ void __launch_bounds__(128) phase1_bwd_bulk_kernel(P1Bwd a)
 }
 
 // processed tokens, in reverse; one warp per chain.  Skip words are fetched for 32 chunks at a time.
-template <typename T, int K>
+template <typename T, int K, bool VEC>
 __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
 {
     constexpr int R = K / 32;
@@ -562,6 +599,7 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                     prefetch_row(a.r.dtraj + th * K, K * 4);
                     prefetch_row(a.dktil + th * K, K * 4);
                     prefetch_row(a.dkread + th * K, K * 4);
+                    if constexpr (VEC) prefetch_row(a.log_ret + th * K, K * 4);
                     prefetch_l2(a.r.pmask + th * R);
                     prefetch_l2(a.r.n + th);
                     prefetch_l2(a.r.rho + th);
@@ -592,6 +630,7 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
             constexpr int PF = 4;
             float kb[PF][R], db[PF][R], tb[PF][R], rb[PF][R], nb[PF], hb[PF], bb[PF];
             float sk_k[PF][R], sk_t[PF][R];
+            float lb[VEC ? PF : 1][R];   // log-retention rows (vector retention only)
             unsigned mb[PF];
             bool needr[PF];
             const unsigned long long todo = ~sk & valid;
@@ -608,6 +647,7 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                 load_row<R>(a.r.dtraj + th * K, lane, db[slot]);
                 load_row<R>(a.dktil + th * K, lane, tb[slot]);
                 load_row<R>(a.dkread + th * K, lane, rb[slot]);
+                if constexpr (VEC) load_row<R>(a.log_ret + th * K, lane, lb[slot]);
                 mb[slot] = lane < R ? a.r.pmask[th * R + lane] : 0u;
                 nb[slot] = a.r.n[th];
                 hb[slot] = a.r.rho[th];
@@ -638,6 +678,12 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                         }
                         const unsigned mw = mb[u];
                         const float ns = nb[u], n = fabsf(ns), rho = hb[u], b = bb[u];
+                        float rv[R];
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            if constexpr (VEC) rv[r] = expf(lb[u][r]);
+                            else rv[r] = rho;
+                        }
                         if (pfm) fetch(pop_top(pfm), u);
                         const size_t th = (size_t)(tok0 + i) * H + h;
 #pragma unroll
@@ -657,11 +703,19 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                         const float dbt = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
                         const float dn = ns > 0.f ? -cc / n * dc : 0.f;
                         float out[R];
+                        if constexpr (VEC) {   // one gradient per coordinate: r_i lambda_i d_i
+                            if (a.dlog_ret) {
+                                float dl[R];
+#pragma unroll
+                                for (int r = 0; r < R; ++r) dl[r] = rv[r] * lam[r] * dt[r];
+                                store_row<R>(a.dlog_ret + th * K, lane, dl);
+                            }
+                        }
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
                             const float dkap = cc * lam[r] + da * dt[r] + dn;
                             out[r] = dkr[r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
-                            lam[r] = rho * lam[r] + da * kap[r] + kk[r] * dkt[r];
+                            lam[r] = rv[r] * lam[r] + da * kap[r] + kk[r] * dkt[r];
                         }
                         store_row<R>(dkp + th * K, lane, out);
                         if (lane == 0) {
@@ -689,10 +743,13 @@ template <typename TI, typename TO, int K>
 int fwd_launch(const P1Fwd& a, cudaStream_t st)
 {
     const long warps = (long)a.NT * a.H * 2;
+    const unsigned gspec = (unsigned)((warps + 3) / 4), gseq = (unsigned)((a.S * a.H + 3) / 4);
     stage_mark(st, "phase1_spec");
-    phase1_spec_kernel<TI, TO, K><<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(a);
+    if (a.hy.apf_mode == 3) phase1_spec_kernel<TI, TO, K, true><<<gspec, 128, 0, st>>>(a);
+    else phase1_spec_kernel<TI, TO, K, false><<<gspec, 128, 0, st>>>(a);
     stage_mark(st, "phase1_seq");
-    phase1_seq_kernel<TI, TO, K><<<(a.S * a.H + 3) / 4, 128, 0, st>>>(a);
+    if (a.hy.apf_mode == 3) phase1_seq_kernel<TI, TO, K, true><<<gseq, 128, 0, st>>>(a);
+    else phase1_seq_kernel<TI, TO, K, false><<<gseq, 128, 0, st>>>(a);
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
@@ -707,7 +764,8 @@ int bwd_launch(const P1Bwd& a, bool bulk, cudaStream_t st)
         ++n;
     }
     stage_mark(st, "phase1_bwd_seq");
-    phase1_bwd_seq_kernel<T, K><<<(a.S * a.H + 3) / 4, 128, 0, st>>>(a);
+    if (a.hy.apf_mode == 3) phase1_bwd_seq_kernel<T, K, true><<<(a.S * a.H + 3) / 4, 128, 0, st>>>(a);
+    else phase1_bwd_seq_kernel<T, K, false><<<(a.S * a.H + 3) / 4, 128, 0, st>>>(a);
     ++n;
     return cudaGetLastError() == cudaSuccess ? n : -1;
 }
@@ -719,7 +777,7 @@ int phase1_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, voi
 {
     P1Fwd f{};
     f.S = L.S; f.H = p.H; f.NT = L.NTmax; f.tab = carve_table(ws, L);
-    f.k = a.k; f.beta = a.beta; f.retsrc = p.apf_mode == 2 ? a.log_ret : a.gate; f.d0 = a.precond_in;
+    f.k = a.k; f.beta = a.beta; f.retsrc = p.apf_mode >= 2 ? a.log_ret : a.gate; f.d0 = a.precond_in;
     f.ktil = ktil; f.d_final = a.precond_out; f.r = carve_p1(ws, L); f.save = save ? 1 : 0; f.hy = hy;
     if (p.io_dtype == OSDN_FP32) {
         if (ktil_bf16) return -1;
@@ -738,7 +796,14 @@ int phase1_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, vo
     b.S = L.S; b.H = p.H; b.NT = L.NTmax; b.tab = carve_table(ws, L);
     b.k = a.k; b.beta = a.beta; b.dktil = dktil; b.dkread = dkread; b.dprecond_out = a.dprecond_out;
     b.dk = a.dk; b.dbeta = a.dbeta; b.dgate = a.dgate; b.dlog_ret = a.dlog_ret; b.dprecond_in = a.dprecond_in;
-    b.r = carve_p1(ws, L); b.hy = hy;
+    b.r = carve_p1(ws, L); b.hy = hy; b.log_ret = a.log_ret;
+    // retention gradients are written for processed tokens only; a skipped token (projection mask all
+    // zero) has none
+    if (p.apf_mode >= 2 && a.dlog_ret) {
+        const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
+        const size_t nb = Ttot * p.H * (p.apf_mode == 3 ? (size_t)p.K : 1) * sizeof(float);
+        if (cudaMemsetAsync(a.dlog_ret, 0, nb, st) != cudaSuccess) return -1;
+    }
     if (p.io_dtype == OSDN_FP32)
         return p.K == 64 ? bwd_launch<float, 64>(b, bulk, st) : bwd_launch<float, 128>(b, bulk, st);
     return p.K == 64 ? bwd_launch<__nv_bfloat16, 64>(b, bulk, st) : bwd_launch<__nv_bfloat16, 128>(b, bulk, st);
@@ -755,12 +820,23 @@ int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const fl
     const int chains = pa.S * pa.H;
     const unsigned grid = (chains + 3) / 4;
     stage_mark(st, "phase1_stream");
+    const bool vec = hy.apf_mode == 3;
     if (p.io_dtype == OSDN_FP32) {
-        if (p.K == 64) phase1_stream_kernel<float, float, 64><<<grid, 128, 0, st>>>(pa);
-        else phase1_stream_kernel<float, float, 128><<<grid, 128, 0, st>>>(pa);
+        if (p.K == 64) {
+            if (vec) phase1_stream_kernel<float, float, 64, true><<<grid, 128, 0, st>>>(pa);
+            else phase1_stream_kernel<float, float, 64, false><<<grid, 128, 0, st>>>(pa);
+        } else {
+            if (vec) phase1_stream_kernel<float, float, 128, true><<<grid, 128, 0, st>>>(pa);
+            else phase1_stream_kernel<float, float, 128, false><<<grid, 128, 0, st>>>(pa);
+        }
     } else {
-        if (p.K == 64) phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 64><<<grid, 128, 0, st>>>(pa);
-        else phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 128><<<grid, 128, 0, st>>>(pa);
+        if (p.K == 64) {
+            if (vec) phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 64, true><<<grid, 128, 0, st>>>(pa);
+            else phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 64, false><<<grid, 128, 0, st>>>(pa);
+        } else {
+            if (vec) phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 128, true><<<grid, 128, 0, st>>>(pa);
+            else phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 128, false><<<grid, 128, 0, st>>>(pa);
+        }
     }
     stage_end(st);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;

@@ -33,7 +33,7 @@ class OsdnHyper:
     eps: float = 1e-6
     scale: float = 0.0  # <= 0 means K ** -0.5
     beta_aware: int = 1
-    apf_mode: int = 1  # 0 none, 1 retention aliased to the gate, 2 separate log-retention
+    apf_mode: int = 1  # 0 none, 1 retention aliased to the gate, 2 separate log-retention, 3 one per coordinate
     clamp: int = 1
     chunk: int = 64
 
@@ -169,7 +169,9 @@ def draw(
     if with_dout:
         out.dout = _round_io(randn(T, H, V), io_dtype)
     if with_log_ret:
-        out.log_ret = torch.nn.functional.logsigmoid(randn(T, H) + log_ret_shift).contiguous()
+        # one log-retention per (token, head); per coordinate for the vector-retention mode
+        shape = (T, H, K) if hyper.apf_mode == 3 else (T, H)
+        out.log_ret = torch.nn.functional.logsigmoid(randn(*shape) + log_ret_shift).contiguous()
     if with_state:
         out.init_state = 0.5 * randn(nseq, H, V, K)
         out.precond_in = hyper.d_min + (hyper.d_max - hyper.d_min) * rand(nseq, H, K)
@@ -270,4 +272,9 @@ def lively(idx: int, *, T: int = 200, B: int = 2, H: int = 2, D: int = 128,
         hy = OsdnHyper(eta=0.003, apf_mode=2, beta_aware=0)
         return draw("lively6_ungated_osdn", 106, lens, H, D, D, io_dtype, dense_B=B, hyper=hy,
                     gate_kind="zero", with_dout=True, with_log_ret=True, log_ret_shift=7.0)
+    if idx == 7:  # vector retention: one log-retention per coordinate
+        hy = OsdnHyper(eta=0.3, apf_mode=3)
+        return draw("lively7_vector_ret", 107, lens, H, D, D, io_dtype, dense_B=B, hyper=hy,
+                    key_kind="sparse", with_dout=True, with_log_ret=True, with_state=True,
+                    with_state_cotangents=True, log_ret_shift=3.0)
     raise ValueError(idx)

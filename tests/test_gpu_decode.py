@@ -55,6 +55,8 @@ CASES = [
     ("bf16", 128, 128, 2, 2, 1, 1, 1, 1, 0.003),
     ("bf16", 128, 128, 2, 2, 33, 1, 1, 1, 0.3),
     ("bf16", 64, 64, 1, 4, 64, 2, 1, 1, 0.3),
+    ("fp32", 128, 128, 2, 2, 9, 3, 1, 1, 0.3),    # vector retention
+    ("bf16", 64, 128, 2, 2, 40, 3, 1, 0, 0.3),
 ]
 
 
@@ -62,7 +64,7 @@ CASES = [
 def test_decode_matches_oracle(io, K, V, B, H, L, apf, clamp, ba, eta):
     hy = OsdnHyper(eta=eta, apf_mode=apf, clamp=clamp, beta_aware=ba)
     inp = draw(f"decode_{io}_{K}_{V}_{L}", 900 + L + K, [L] * B, H, K, V, io, dense_B=B, hyper=hy,
-               with_log_ret=(apf == 2), with_state=True)
+               with_log_ret=(apf >= 2), with_state=True)
     got_out, got_S, got_d = _decode(inp, inp.init_state, inp.precond_in)
     ref = oracle.fwd_inputs(inp)
     assert parity.err(got_S, ref["final_state"]) <= 1e-4

@@ -57,7 +57,7 @@ def test_benchmark_configs_reduced(idx, path, flags):
 
 @pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])
 @pytest.mark.parametrize("io", ["fp32", "bf16"])
-@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5, 6, 7])
 def test_lively_sets(idx, io, path, flags):
     if io == "fp32" and path == "auto":
         pytest.skip("fp32 I/O always runs the CUDA-core kernels")
@@ -113,6 +113,27 @@ def test_precond_update_alone():
                                 d_mid, None, d_mid)
     torch.cuda.synchronize()
     assert torch.equal(d_mid, d_all)
+
+
+@pytest.mark.parametrize("io,K", [("bf16", 128), ("fp32", 64)])
+def test_precond_update_vector_retention(io, K):
+    """One log-retention per coordinate ([T,H,K]), packed batch with ragged sequences."""
+    hy = OsdnHyper(eta=0.3, apf_mode=3)
+    inp = draw(f"pu_vec_{io}", 952, [150, 64, 7], 3, K, K, io, hyper=hy, with_log_ret=True, with_state=True,
+               key_kind="sparse", log_ret_shift=3.0)
+    assert tuple(inp.log_ret.shape) == (221, 3, K)
+    dev = torch.device("cuda:0")
+    b = binding.DeviceBundle(inp, dev, need_bwd=False)
+    ktil = torch.empty_like(b.k)
+    dout = torch.empty_like(b.precond_in)
+    binding.osdn_precond_update(b.params, b.k, b.beta, b.log_ret, b.precond_in, ktil, dout)
+    torch.cuda.synchronize()
+    ref = oracle.precond_update(hy, inp.seq_lens, inp.k, inp.beta, None, inp.log_ret, inp.precond_in)
+    assert parity.err(dout.cpu().numpy(), ref["precond_out"], "fp32") <= 1e-5
+    assert parity.err(ktil.float().cpu().numpy(), ref["ktil"], io) <= parity.TOL[io]
+    # the sweep of osdn_fwd and the stand-alone update agree on the final preconditioner
+    full = run_inputs_fwd(inp)
+    assert parity.err(full["precond_out"].numpy(), dout.cpu().numpy(), "fp32") <= 1e-6
 
 
 def test_split_sequence_state_carry_on_gpu():

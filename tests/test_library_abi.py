@@ -64,6 +64,12 @@ def test_calls_reject_bad_arguments_before_any_launch(lib):
     rc = lib.osdn_fwd(ctypes.byref(p), fake, fake, fake, fake, fake, null, null, null, fake, null, null,
                       fake, ctypes.c_size_t(1 << 30), null)
     assert rc == -1                     # separate retention requested but not given
+    p.apf_mode = 3
+    rc = lib.osdn_fwd(ctypes.byref(p), fake, fake, fake, fake, fake, null, null, null, fake, null, null,
+                      fake, ctypes.c_size_t(1 << 30), null)
+    assert rc == -1                     # vector retention requested but not given
+    p.apf_mode = 4
+    assert osdn.osdn_workspace_bytes(p, False) == 0   # no such retention mode
     p.apf_mode = 1
     p.nseq = 3                          # var-len without cu_seqlens
     rc = lib.osdn_precond_update(ctypes.byref(p), fake, fake, fake, null, null, fake, null)
