@@ -1382,7 +1382,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     if (tid == 0) {
         mbar_init(&bar_tma, 1);
-        for (int i = 0; i < 5; ++i) mbar_init(&bar_mma[i], 1);
+        // the independent products of a phase are issued by different warps (the issue rate of one
+        // thread, not the tensor pipe, limits these small shapes); each issuer commits for itself
+        const uint32_t issuers[5] = {5, 6, 1, 1, 2};
+        for (int i = 0; i < 5; ++i) mbar_init(&bar_mma[i], issuers[i]);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(&tmem_base, 512);
@@ -1519,32 +1522,34 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t cDKB = 256, cDVB = 64, cDQ2 = 0, cY = 320, cZ = 384, cDKR = 320;
 
     // ---- phase A -------------------------------------------------------------------------------
-    if (tid == 0 && ok) {
+    if (lane == 0 && warp < 5 && ok) {
         tc_fence_after();
+        if (warp == 0) {
         for (int k = 0; k < 8; ++k) {   // rawkk[i][j] = <k_i, ktil_j>          (M = 64)
             mma_ss(tb + cRAW, desc_advance(desc_kmajor(sm + R_K + (k >> 2) * BOX), 32 * (k & 3)),
                    desc_advance(desc_kmajor(sm + R_KT + (k >> 2) * BOX), 32 * (k & 3)), make_idesc(64, 64), k > 0);
         }
-        {   // dP'[i][j] = sum_v dO[i][v] dU[j][v]                               (M = 64)
+        }
+        if (warp == 1) {   // dP'[i][j] = sum_v dO[i][v] dU[j][v]                               (M = 64)
             const uint64_t db0 = desc_mnmajor(sm + R_DU, 0);
             for (int k = 0; k < 8; ++k)
                 mma_ss(tb + cDP, desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
                        desc_advance(db0, 2048 * k), make_idesc(64, 64, IDESC_B_MN), k > 0);
         }
-        {   // dQ1^T[k][i] = sum_v S[v][k] dO[i][v]
+        if (warp == 2) {   // dQ1^T[k][i] = sum_v S[v][k] dO[i][v]
             const uint64_t da0 = desc_mnmajor(sm + R_S, 16384);
             for (int k = 0; k < 8; ++k)
                 mma_ss(tb + cDQ1, desc_advance(da0, 2048 * k),
                        desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
                        make_idesc(128, 64, IDESC_A_MN), k > 0);
         }
-        {   // dKtr^T[k][j] = sum_v dS[v][k] dU[j][v]
+        if (warp == 3) {   // dKtr^T[k][j] = sum_v dS[v][k] dU[j][v]
             const uint64_t da0 = desc_mnmajor(sm + R_DS, 16384), db0 = desc_mnmajor(sm + R_DU, 0);
             for (int k = 0; k < 8; ++k)
                 mma_ss(tb + cDKTR, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
                        make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
         }
-        {   // dW^T[k][i] = -sum_v S[v][k] ddU[i][v]
+        if (warp == 4) {   // dW^T[k][i] = -sum_v S[v][k] ddU[i][v]
             const uint64_t da0 = desc_mnmajor(sm + R_S, 16384), db0 = desc_mnmajor(sm + R_DDU, 0);
             for (int k = 0; k < 8; ++k)
                 mma_ss(tb + cDW, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
@@ -1622,44 +1627,48 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     OSDN_CLKS(4, threadIdx.x == 0 && clk);
 
     // ---- phase B -------------------------------------------------------------------------------
-    if (tid == 0 && ok) {
+    if (lane == 0 && warp < 6 && ok) {
         tc_fence_after();
-        {   // dT_a[i][j] = sum_k dW[i][k] K[j][k]                               (M = 64)
+        if (warp == 0) {   // dT_a[i][j] = sum_k dW[i][k] K[j][k]                               (M = 64)
             const uint64_t da0 = desc_mnmajor(sm + R_DWT, 0);
             for (int k = 0; k < 8; ++k)
                 mma_ss(tb + cDTA, desc_advance(da0, 2048 * k),
                        desc_advance(desc_kmajor(sm + R_K + (k >> 2) * BOX), 32 * (k & 3)),
                        make_idesc(64, 64, IDESC_A_MN), k > 0);
         }
-        {   // dT_b[i][j] = sum_v ddU[i][v] V[j][v]                              (M = 64)
+        if (warp == 1) {   // dT_b[i][j] = sum_v ddU[i][v] V[j][v]                              (M = 64)
             const uint64_t da0 = desc_mnmajor(sm + R_DDU, 0);
             for (int k = 0; k < 8; ++k)
                 mma_ss(tb + cDTB, desc_advance(da0, 2048 * k),
                        desc_advance(desc_kmajor(sm + R_V + (k >> 2) * BOX), 32 * (k & 3)),
                        make_idesc(64, 64, IDESC_A_MN), k > 0);
         }
-        {   // dKb^T[k][j] = sum_i dW^T[k][i] T[i][j] ;  dVb^T[v][j] = sum_i ddU^T[v][i] T[i][j]
+        if (warp == 2 || warp == 3) {   // dKb^T[k][j] = sum_i dW^T[k][i] T[i][j] ;  dVb^T[v][j] = sum_i ddU^T[v][i] T[i][j]
             const uint64_t db0 = desc_mnmajor(sm + R_T, 0);
             const uint64_t da0 = desc_kmajor(sm + R_DWT), da1 = desc_kmajor(sm + R_DDU);
-            for (int k = 0; k < 4; ++k)
-                mma_ss(tb + cDKB, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k),
-                       make_idesc(128, 64, IDESC_B_MN), k > 0);
-            for (int k = 0; k < 4; ++k)
-                mma_ss(tb + cDVB, desc_advance(da1, 32 * k), desc_advance(db0, 2048 * k),
-                       make_idesc(128, 64, IDESC_B_MN), k > 0);
+            if (warp == 2)
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tb + cDKB, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k),
+                           make_idesc(128, 64, IDESC_B_MN), k > 0);
+            else
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tb + cDVB, desc_advance(da1, 32 * k), desc_advance(db0, 2048 * k),
+                           make_idesc(128, 64, IDESC_B_MN), k > 0);
         }
-        {   // dq2^T[k][i] = sum_j Ktil[j][k] M1[i][j] ;  dktil^T[k][j] = sum_i Q[i][k] M1[i][j]
+        if (warp == 4 || warp == 5) {   // dq2^T[k][i] = sum_j Ktil[j][k] M1[i][j] ;  dktil^T[k][j] = sum_i Q[i][k] M1[i][j]
             const uint64_t da0 = desc_mnmajor(sm + R_KT, BOX), da1 = desc_mnmajor(sm + R_Q, BOX);
             const uint64_t dbk = desc_kmajor(sm + R_M1), dbm = desc_mnmajor(sm + R_M1, 0);
-            for (int k = 0; k < 4; ++k)
-                mma_ss(tb + cDQ2, desc_advance(da0, 2048 * k), desc_advance(dbk, 32 * k),
-                       make_idesc(128, 64, IDESC_A_MN), k > 0);
-            for (int k = 0; k < 4; ++k)
-                mma_ss(tb + cDKT, desc_advance(da1, 2048 * k), desc_advance(dbm, 2048 * k),
-                       make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
+            if (warp == 4)
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tb + cDQ2, desc_advance(da0, 2048 * k), desc_advance(dbk, 32 * k),
+                           make_idesc(128, 64, IDESC_A_MN), k > 0);
+            else
+                for (int k = 0; k < 4; ++k)
+                    mma_ss(tb + cDKT, desc_advance(da1, 2048 * k), desc_advance(dbm, 2048 * k),
+                           make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
         }
         mma_commit(&bar_mma[1]);
-        if (early) {   // phase A has finished: dU and dS are dead
+        if (early && warp == 0) {   // phase A has finished: dU and dS are dead
             expect_all();
             bulk_load(sm + R_DU, a.dUT + (size_t)tile_next * 16384, 16384, &bar_tma);
             bulk_load(sm + R_DS, a.dSn + (size_t)tile_next * 32768, 32768, &bar_tma);
@@ -1776,18 +1785,20 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     OSDN_CLKS(10, threadIdx.x == 0 && clk);
 
     // ---- phase E: dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T -----------------------------------------
-    if (tid == 0 && ok) {
+    if (lane == 0 && warp < 2 && ok) {
         tc_fence_after();
         const uint64_t da0 = desc_mnmajor(sm + R_K, BOX), da1 = desc_mnmajor(sm + R_KT, BOX);
         const uint64_t dbm = desc_mnmajor(sm + R_M2, 0), dbk = desc_kmajor(sm + R_M2);
-        for (int k = 0; k < 4; ++k)
-            mma_ss(tb + cDKT, desc_advance(da0, 2048 * k), desc_advance(dbm, 2048 * k),
-                   make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), 1);
-        for (int k = 0; k < 4; ++k)
-            mma_ss(tb + cDKR, desc_advance(da1, 2048 * k), desc_advance(dbk, 32 * k),
-                   make_idesc(128, 64, IDESC_A_MN), k > 0);
+        if (warp == 0)
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tb + cDKT, desc_advance(da0, 2048 * k), desc_advance(dbm, 2048 * k),
+                       make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), 1);
+        else
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tb + cDKR, desc_advance(da1, 2048 * k), desc_advance(dbk, 32 * k),
+                       make_idesc(128, 64, IDESC_A_MN), k > 0);
         mma_commit(&bar_mma[4]);
-        if (early) bulk_load(sm + R_T, a.Tm + (size_t)tile_next * 8192, 8192, &bar_tma);   // phase D done
+        if (early && warp == 0) bulk_load(sm + R_T, a.Tm + (size_t)tile_next * 8192, 8192, &bar_tma);   // phase D done
     }
     ok = ok && mbar_wait(&bar_mma[4], ph, a.status, ERR_MMA2);
     OSDN_CLKS(11, threadIdx.x == 0 && clk);
