@@ -108,6 +108,23 @@ def fwd(hy, seq_lens, q, k, v, beta, gate, log_ret=None, init_state=None, precon
     return res
 
 
+def residual_ratio(hy, seq_lens, k, v, beta, gate, log_ret=None, init_state=None, precond_in=None) -> np.ndarray:
+    """q_t = f_t(S_t) / f_t(exp(g_t) S_{t-1}) with f_t(S) = |S k_t - v_t|^2 / 2, from the states
+    themselves (the definition; not the closed form).  Returns [T, H]."""
+    lib = _load()
+    k, v, beta, gate = map(_f64, (k, v, beta, gate))
+    log_ret, init_state, precond_in = map(_f64, (log_ret, init_state, precond_in))
+    T, H, K = k.shape
+    V = v.shape[-1]
+    cu = _cu(seq_lens)
+    out = np.zeros((T, H))
+    hp = _hyper(hy, K)
+    lib.osdn_oracle_residual_ratio(ctypes.c_int(len(seq_lens)), _p(cu), ctypes.c_int(H), ctypes.c_int(K),
+                                   ctypes.c_int(V), ctypes.byref(hp), _p(k), _p(v), _p(beta), _p(gate),
+                                   _p(log_ret), _p(init_state), _p(precond_in), _p(out))
+    return out
+
+
 def precond_update(hy, seq_lens, k, beta, gate=None, log_ret=None, precond_in=None) -> dict:
     lib = _load()
     k, beta, gate, log_ret, precond_in = map(_f64, (k, beta, gate, log_ret, precond_in))

@@ -176,6 +176,50 @@ void osdn_oracle_fwd(int nseq, const int *cu, int H, int K, int V, const oracle_
     }
 }
 
+/*
+ * Residual ratio of the mechanism diagnostic, by its definition: with the
+ * per-token loss f_t(S) = 1/2 |S k_t - v_t|^2,
+ *     q_t = f_t(S_t) / f_t(Sbar_{t-1}),      Sbar_{t-1} = exp(g_t) S_{t-1},
+ * the loss after the write over the loss before it (the state the write starts
+ * from is the gated one).  0/0 is read as 1 (no residual, nothing to reduce).
+ * The closed form (1 - beta_t <d_t, k_t^2>)^2 of the token-local theorem is NOT
+ * used here; it is what the tests and the CUDA path are compared with.
+ * ratio_out [T_total, H].
+ */
+void osdn_oracle_residual_ratio(int nseq, const int *cu, int H, int K, int V, const oracle_hyper *hp,
+                                const double *k, const double *v, const double *beta, const double *gate,
+                                const double *log_ret, const double *S0, const double *d0, double *ratio_out)
+{
+    int nchain = nseq * H;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int ch = 0; ch < nchain; ++ch) {
+        int s = ch / H, h = ch % H;
+        double *S = (double *)malloc(sizeof(double) * V * K);
+        double *d = (double *)malloc(sizeof(double) * K);
+        double *ktil = (double *)malloc(sizeof(double) * K);
+        double *u = (double *)malloc(sizeof(double) * V);
+        if (S0) memcpy(S, S0 + ((size_t)s * H + h) * V * K, sizeof(double) * V * K);
+        else memset(S, 0, sizeof(double) * V * K);
+        for (int i = 0; i < K; ++i) d[i] = d0 ? d0[((size_t)s * H + h) * K + i] : 1.0;
+        for (int t = cu[s]; t < cu[s + 1]; ++t) {
+            size_t th = (size_t)t * H + h;
+            const double *kt = k + th * K, *vt = v + th * V;
+            phase1_step(hp, K, kt, beta[th], gate[th], LRET_S(hp, log_ret, th), LRET_V(hp, log_ret, th, K), d, ktil,
+                        0, 0, 0, 0, 0, 0, 0);
+            phase2_step(K, V, kt, ktil, vt, beta[th], gate[th], S, u);   /* u = v - Sbar k */
+            double before = 0.0, after = 0.0;
+            for (int r = 0; r < V; ++r) {
+                double acc = 0.0;
+                for (int i = 0; i < K; ++i) acc += S[(size_t)r * K + i] * kt[i];
+                after += (acc - vt[r]) * (acc - vt[r]);
+                before += u[r] * u[r];
+            }
+            ratio_out[th] = before > 0.0 ? after / before : 1.0;
+        }
+        free(S); free(d); free(ktil); free(u);
+    }
+}
+
 /* Phase 1 alone (the stand-alone preconditioner update). */
 void osdn_oracle_precond_update(int nseq, const int *cu, int H, int K, const oracle_hyper *hp,
                                 const double *k, const double *beta, const double *gate,

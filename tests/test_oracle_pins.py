@@ -283,3 +283,39 @@ def test_phase1_order_write_key_uses_pre_update_d():
     np.testing.assert_allclose(res4["d_traj"][3, 0],
                                np.clip(np.exp(g[2, 0]) * res4["d_traj"][2, 0], 0.5, 2.0), atol=1e-15)
     assert np.isfinite(res4["out"]).all()
+
+
+# ---------------------------------------------------------------- residual ratio of the mechanism diagnostic
+def test_residual_ratio_definition_equals_token_local_closed_form():
+    """The oracle forms q_t = f_t(S_t) / f_t(exp(g_t) S_{t-1}) from the states; the proof of the
+    token-local theorem gives q_t = (1 - beta_t <d_t, k_t^2>)^2, which involves neither S nor v."""
+    hy = OsdnHyper(eta=0.3, apf_mode=1)
+    L, H, K, V = 40, 2, 6, 5
+    q, k, v, beta, g = _small(4, L, H, K, V, unit=False)
+    r = _rng(9)
+    S0 = r.standard_normal((2, H, V, K))
+    d0 = r.uniform(hy.d_min, hy.d_max, size=(2, H, K))
+    lens = [25, 15]
+    got = oracle.residual_ratio(hy, lens, k, v, beta, g, None, S0, d0)
+    dtr = oracle.fwd(hy, lens, q, k, v, beta, g, None, S0, d0, want_dtraj=True)["d_traj"]
+    want = (1.0 - beta * np.einsum("thk,thk->th", dtr, k ** 2)) ** 2
+    np.testing.assert_allclose(got, want, rtol=1e-9, atol=1e-12)
+    # other values change nothing: the ratio does not depend on v or on the state
+    got2 = oracle.residual_ratio(hy, lens, k, 3.0 * v[::-1].copy(), beta, g, None, -S0, d0)
+    np.testing.assert_allclose(got2, want, rtol=1e-8, atol=1e-12)
+
+
+def test_residual_ratio_special_cases():
+    L, H, K, V = 9, 1, 4, 3
+    q, k, v, beta, g = _small(6, L, H, K, V, unit=True)
+    # beta = 0: nothing is written, the loss does not move
+    hy = OsdnHyper(eta=0.3, apf_mode=0)
+    assert np.array_equal(oracle.residual_ratio(hy, [L], k, v, 0 * beta, g), np.ones((L, H)))
+    # plain delta rule (eta = 0, d = 1) with unit keys: q_t = (1 - beta_t)^2, an exact overwrite at beta = 1
+    hy0 = OsdnHyper(eta=0.0, apf_mode=0)
+    np.testing.assert_allclose(oracle.residual_ratio(hy0, [L], k, v, beta, g), (1 - beta) ** 2, rtol=1e-9, atol=1e-15)
+    np.testing.assert_allclose(oracle.residual_ratio(hy0, [L], k, v, np.ones_like(beta), g), 0.0, atol=1e-25)
+    # a preconditioner of 2 on unit keys doubles the step: q_t = (1 - 2 beta_t)^2
+    d2 = np.full((1, H, K), 2.0)
+    np.testing.assert_allclose(oracle.residual_ratio(hy0, [L], k, v, beta, g, None, None, d2), (1 - 2 * beta) ** 2,
+                               rtol=1e-9, atol=1e-15)
