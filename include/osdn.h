@@ -140,6 +140,23 @@ int osdn_precond_update(const osdn_params* p, const void* k, const float* beta,
                         void* k_tilde_out, float* precond_out, void* cuda_stream);
 
 /*
+ * Residual ratio of the paper's mechanism diagnostic (Section "Mechanism diagnostic"; Eq. "qt_form" in
+ * the proof of the token-local theorem), a by-product of the same sweep: for every token-head
+ *     q_t = f_t(S_t) / f_t(S_{t-1}) = (1 - beta_t <d_t, k_t^2>)^2,   f_t(S) = |S k_t - v_t|^2 / 2,
+ * the factor by which the write of token t shrinks its own loss (with the gate, S_{t-1} is the gated
+ * state the write starts from), where d_t is the preconditioner the write key of token t is formed
+ * with; it needs neither the state nor the values.  eta = 0 with precond_in = NULL gives the ratio of
+ * the unscaled delta rule.
+ *   in : k, beta, gate_or_log_ret, precond_in as for osdn_precond_update.
+ *   out: ratio_out [T,H] fp32 (may be NULL); log_ratio_sum [S,H] fp32 = sum over the sequence of
+ *        log(max(q_t, FLT_MIN)) (may be NULL; the geometric mean of a chain is exp(sum / length));
+ *        at least one of the two; precond_out [S,H,K] (may be NULL; may alias precond_in).
+ */
+int osdn_residual_ratio(const osdn_params* p, const void* k, const float* beta,
+                        const float* gate_or_log_ret, const float* precond_in,
+                        float* ratio_out, float* log_ratio_sum, float* precond_out, void* cuda_stream);
+
+/*
  * Recurrent (decode) step (appendix paragraph "Single-token recurrence kernel for OSGDN", stated
  * for q_len <= 64): for the p->T new tokens of each of the p->B sequences, in order,
  *     alpha_t = exp(g_t);  ktil_t = d_t (.) k_t;  d_{t+1} as in osdn_fwd (Algorithm 1 with APF and the

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     osdn_fwd_static,
     osdn_decode_step,
     osdn_precond_update,
+    osdn_residual_ratio,
     osdn_step_host,
     osdn_workspace_bytes,
     osdn_host_staging_bytes,

@@ -19,7 +19,7 @@ EXPORTS = [
     "osdn_workspace_bytes", "osdn_fwd", "osdn_bwd", "osdn_precond_update", "osdn_host_staging_bytes",
     "osdn_step_host", "osdn_read_device_status", "osdn_status_string", "osdn_last_launch_count",
     "osdn_stage_timing_enable", "osdn_stage_timing_read", "osdn_workspace_region",
-    "osdn_fwd_static", "osdn_decode_step",
+    "osdn_fwd_static", "osdn_decode_step", "osdn_residual_ratio",
 ]
 
 
@@ -58,6 +58,8 @@ def load_library(path: Optional[str] = None):
     lib.osdn_bwd.argtypes = [pp] + [vp] * 19 + [vp, sz, vp]
     lib.osdn_precond_update.restype = ci
     lib.osdn_precond_update.argtypes = [pp] + [vp] * 6 + [vp]
+    lib.osdn_residual_ratio.restype = ci
+    lib.osdn_residual_ratio.argtypes = [pp] + [vp] * 7 + [vp]
     lib.osdn_decode_step.restype = ci
     lib.osdn_decode_step.argtypes = [pp] + [vp] * 9 + [vp]
     lib.osdn_step_host.restype = ci
@@ -210,6 +212,13 @@ def osdn_precond_update(p: OsdnParams, k, beta, gate_or_log_ret, precond_in, k_t
     rc = lib.osdn_precond_update(ctypes.byref(p), _ptr(k), _ptr(beta), _ptr(gate_or_log_ret), _ptr(precond_in),
                                  _ptr(k_tilde_out), _ptr(precond_out), _stream_ptr())
     _check(rc, "osdn_precond_update")
+
+
+def osdn_residual_ratio(p: OsdnParams, k, beta, gate_or_log_ret, precond_in, ratio_out, log_ratio_sum, precond_out=None):
+    lib = load_library()
+    rc = lib.osdn_residual_ratio(ctypes.byref(p), _ptr(k), _ptr(beta), _ptr(gate_or_log_ret), _ptr(precond_in),
+                                 _ptr(ratio_out), _ptr(log_ratio_sum), _ptr(precond_out), _stream_ptr())
+    _check(rc, "osdn_residual_ratio")
 
 
 def osdn_decode_step(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, state, precond, out):

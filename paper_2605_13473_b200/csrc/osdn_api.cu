@@ -218,7 +218,26 @@ int osdn_precond_update(const osdn_params* p, const void* k, const float* beta, 
     for (const void* x : ptrs)
         if (x && !aligned16(x)) return OSDN_MISALIGNED;
     const int n = phase1_update(*p, make_hyper(*p), k, beta, gate_or_log_ret, precond_in, k_tilde_out,
-                                      precond_out, static_cast<cudaStream_t>(cuda_stream));
+                                      precond_out, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream));
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = n;
+    return OSDN_OK;
+}
+
+int osdn_residual_ratio(const osdn_params* p, const void* k, const float* beta, const float* gate_or_log_ret,
+                        const float* precond_in, float* ratio_out, float* log_ratio_sum, float* precond_out,
+                        void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (!k || !beta || (!ratio_out && !log_ratio_sum)) return OSDN_INVALID_ARG;
+    if (p->apf_mode != OSDN_APF_NONE && !gate_or_log_ret) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {k, beta, gate_or_log_ret, precond_in, ratio_out, log_ratio_sum, precond_out};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    const int n = phase1_update(*p, make_hyper(*p), k, beta, gate_or_log_ret, precond_in, nullptr, precond_out,
+                                ratio_out, log_ratio_sum, static_cast<cudaStream_t>(cuda_stream));
     if (n < 0) return OSDN_CUDA_ERROR;
     g_last_launches = n;
     return OSDN_OK;

@@ -195,7 +195,8 @@ int phase1_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, voi
 int phase1_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
                     const float* dktil, const float* dkread, bool bulk, cudaStream_t st);
 int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta, const float* retsrc,
-                  const float* precond_in, void* ktil_out, float* precond_out, cudaStream_t st);
+                  const float* precond_in, void* ktil_out, float* precond_out, float* ratio_out,
+                  float* log_sum_out, cudaStream_t st);
 
 // Recurrent step over p.T tokens per sequence on cached state and preconditioner (both updated in
 // place); one launch.

@@ -132,6 +132,8 @@ struct P1Args {
     const float *beta, *retsrc, *d0;
     void* ktil;
     float* d_final;
+    float* ratio;      // nullable: residual ratio q_t per token-head
+    float* log_sum;    // nullable: sum_t log q_t per chain
     Hyper hy;
 };
 
@@ -155,6 +157,7 @@ __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
         for (int r = 0; r < R; ++r) d[r] = 1.0f;
     }
     const Hyper hy = a.hy;
+    float lsum = 0.f;
     for (int i = 0; i < len; ++i) {
         const size_t th = (size_t)(t0 + i) * a.H + h;
         float kk[R], kap[R], w[R];
@@ -181,8 +184,18 @@ __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
         bool low;
         float c, al;
         p1_step<R>(d, kap, n, b, rho, hy, pass, low, c, al);
+        if (a.ratio || a.log_sum) {
+            // residual ratio of the write of this token (token-local theorem): the loss |S k - v|^2 after
+            // the write over the loss before it is (1 - beta <d_t, k^2>)^2, with the write strength beta
+            // itself (whether or not the step of d is beta-aware) and the d the write key was formed with
+            const float fac = 1.0f - a.beta[th] * al;
+            const float qt = fac * fac;
+            if (a.ratio && lane == 0) a.ratio[th] = qt;
+            lsum += logf(fmaxf(qt, 1.17549435e-38f));
+        }
     }
-    store_row<R>(a.d_final + ((size_t)s * a.H + h) * K, lane, d);
+    if (a.d_final) store_row<R>(a.d_final + ((size_t)s * a.H + h) * K, lane, d);
+    if (a.log_sum && lane == 0) a.log_sum[(size_t)s * a.H + h] = lsum;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -810,13 +823,14 @@ int phase1_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, vo
 }
 
 int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const float* beta, const float* retsrc,
-                  const float* precond_in, void* ktil_out, float* precond_out, cudaStream_t st)
+                  const float* precond_in, void* ktil_out, float* precond_out, float* ratio_out,
+                  float* log_sum_out, cudaStream_t st)
 {
     P1Args pa{};
     pa.S = p.nseq > 0 ? p.nseq : p.B;
     pa.H = p.H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
     pa.k = k; pa.beta = beta; pa.retsrc = retsrc; pa.d0 = precond_in; pa.ktil = ktil_out;
-    pa.d_final = precond_out; pa.hy = hy;
+    pa.d_final = precond_out; pa.ratio = ratio_out; pa.log_sum = log_sum_out; pa.hy = hy;
     const int chains = pa.S * pa.H;
     const unsigned grid = (chains + 3) / 4;
     stage_mark(st, "phase1_stream");

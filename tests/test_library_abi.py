@@ -75,6 +75,12 @@ def test_calls_reject_bad_arguments_before_any_launch(lib):
     rc = lib.osdn_precond_update(ctypes.byref(p), fake, fake, fake, null, null, fake, null)
     assert rc == -1
     assert osdn.status_string(-2) == "unsupported shape"
+    # the residual-ratio diagnostic: no output requested, misaligned output
+    pr = osdn.make_params(B=1, T=64, H=1, K=64, V=64, io_dtype="fp32", hyper=hy)
+    rc = lib.osdn_residual_ratio(ctypes.byref(pr), fake, fake, fake, null, null, null, null, null)
+    assert rc == -1
+    rc = lib.osdn_residual_ratio(ctypes.byref(pr), fake, fake, fake, null, odd, null, null, null)
+    assert rc == -3
     # the recurrent step: missing cache, misaligned pointer, missing separate retention, packed batch
     p = osdn.make_params(B=2, T=1, H=1, K=128, V=128, io_dtype="bf16", hyper=hy)
     rc = lib.osdn_decode_step(ctypes.byref(p), fake, fake, fake, fake, fake, null, null, fake, fake, null)
