@@ -231,7 +231,7 @@ int osdn_step_host(const osdn_params* p, const void* q_host, const void* k_host,
  * Location of a named region inside a workspace laid out for (p, need_bwd): "p1_skip"
  * ([chunks, H, 2] uint32: bit i of the 64-bit pair = token i of the chunk was skipped by the
  * sequential preconditioner pass, i.e. it was entered on the lower face of the box and its
- * projection mask is all zero) and "p1_mask" ([T, H, R] uint32 with R = K/32: bit l of word r =
+ * projection mask is all zero) and "p1_mask" ([T, H, 32] uint32, with R = K/32: bit r of word l =
  * the projection passed gradient for coordinate R l + r; valid for tokens that were not skipped).
  * Chunks are numbered sequence by sequence, ceil(len / 64) per sequence.  Filled by osdn_fwd with
  * OSDN_FLAG_SAVE_RESIDUALS.  For inspection and tests; returns 0 or OSDN_INVALID_ARG.

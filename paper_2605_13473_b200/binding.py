@@ -320,11 +320,11 @@ class DeviceBundle:
         o1, n1 = workspace_region(self.params, "p1_skip")
         o2, n2 = workspace_region(self.params, "p1_mask")
         skip = self.workspace[o1:o1 + n1].view(torch.int32).cpu().numpy().astype("uint32").reshape(-1, H, 2)
-        words = self.workspace[o2:o2 + n2].view(torch.int32).cpu().numpy().astype("uint32").reshape(T, H, K // 32)
+        words = self.workspace[o2:o2 + n2].view(torch.int32).cpu().numpy().astype("uint32").reshape(T, H, 32)
         import numpy as np
-        R = K // 32   # bit l of word r <-> coordinate R * l + r
-        bits = ((words[..., None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8)   # [T,H,R,32]
-        bits = np.ascontiguousarray(bits.transpose(0, 1, 3, 2)).reshape(T, H, K)
+        R = K // 32   # bit r of word l <-> coordinate R * l + r
+        bits = ((words[..., None] >> np.arange(R, dtype=np.uint32)) & 1).astype(np.uint8)   # [T,H,32,R]
+        bits = np.ascontiguousarray(bits).reshape(T, H, K)
         skipped = np.zeros((T, H), dtype=bool)
         c = 0
         t0 = 0

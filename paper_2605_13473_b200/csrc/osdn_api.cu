@@ -490,7 +490,7 @@ int osdn_workspace_region(const osdn_params* p, int need_bwd, const char* name, 
     }
     if (!std::strcmp(name, "p1_mask")) {
         *offset = L.pmask;
-        *bytes = 4 * Ttot * p->H * (p->K / 32);
+        *bytes = 4 * Ttot * p->H * 32;
         return OSDN_OK;
     }
     return OSDN_INVALID_ARG;

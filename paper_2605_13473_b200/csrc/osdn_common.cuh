@@ -58,7 +58,8 @@ struct WsLayout {
     size_t p1rho;       // [T,H]          f32   retention of the preconditioner
     size_t p1flags;     // [NT,H,2]       u32   per token: the step maps d_min*1 to d_min*1, mask all zero
     size_t p1skip;      // [NT,H,2]       u32   tokens the sequential pass skipped           (save only)
-    size_t pmask;       // [T,H,K/32]     u32   projection pass masks of processed tokens    (save only)
+    size_t pmask;       // [T,H,32]       u32   projection pass masks of processed tokens: word of lane l,
+                        //                      bit r = coordinate (K/32) l + r passes gradient    (save only)
     size_t dtraj;       // [T,H,K]        f32   d_t of processed tokens                      (save only)
     size_t ktil;        // [T,H,K]        f32   write keys
     size_t Tm;          // [NT,H,64,64]   f32   UT inverse
@@ -101,7 +102,7 @@ inline WsLayout make_layout(const osdn_params& p, bool need_bwd)
     L.p1flags = take(4 * NT * H * 2);
     if (need_bwd) {
         L.p1skip = take(4 * NT * H * 2);
-        L.pmask = take(4 * Ttot * H * (K / 32));
+        L.pmask = take(4 * Ttot * H * 32);
         L.dtraj = take(4 * Ttot * H * K);
     }
     L.ktil = take(4 * Ttot * H * K);

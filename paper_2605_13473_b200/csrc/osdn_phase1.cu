@@ -111,6 +111,55 @@ template <int R> __device__ __forceinline__ void store_row(__nv_bfloat16* p, int
     }
 }
 
+// A row as it sits in memory: loading it does not wait for the data (a conversion right after the
+// load would stall the warp until the load returns, which defeats fetching rows ahead of their use).
+template <typename T, int R> struct RawRow;
+template <> struct RawRow<float, 4> { float4 v; };
+template <> struct RawRow<float, 2> { float2 v; };
+template <> struct RawRow<__nv_bfloat16, 4> { uint2 v; };
+template <> struct RawRow<__nv_bfloat16, 2> { uint32_t v; };
+template <int R> __device__ __forceinline__ void load_raw(const float* p, int lane, RawRow<float, R>& x)
+{
+    if constexpr (R == 4) x.v = *reinterpret_cast<const float4*>(p + 4 * lane);
+    else x.v = *reinterpret_cast<const float2*>(p + 2 * lane);
+}
+template <int R> __device__ __forceinline__ void load_raw(const __nv_bfloat16* p, int lane, RawRow<__nv_bfloat16, R>& x)
+{
+    if constexpr (R == 4) x.v = *reinterpret_cast<const uint2*>(p + 4 * lane);
+    else x.v = *reinterpret_cast<const uint32_t*>(p + 2 * lane);
+}
+template <int R> __device__ __forceinline__ void unpack(const RawRow<float, R>& x, float (&y)[R])
+{
+    if constexpr (R == 4) { y[0] = x.v.x; y[1] = x.v.y; y[2] = x.v.z; y[3] = x.v.w; }
+    else { y[0] = x.v.x; y[1] = x.v.y; }
+}
+template <int R> __device__ __forceinline__ void unpack(const RawRow<__nv_bfloat16, R>& x, float (&y)[R])
+{
+    if constexpr (R == 4) {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.v.x));
+        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.v.y));
+        y[0] = a.x; y[1] = a.y; y[2] = b.x; y[3] = b.y;
+    } else {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.v));
+        y[0] = a.x; y[1] = a.y;
+    }
+}
+
+// Asynchronous copies into a shared-memory ring: completion is counted per committed group (first in,
+// first out), so a row fetched PF tokens ahead can be waited for without waiting for the more recent
+// ones.  Rows fetched into registers cannot do that: the hardware tracks outstanding loads with a
+// handful of counters per warp, and a counter shared with a load issued one token ago holds back the
+// use of a row issued eight tokens ago (measured: about 300 cycles per token).
+template <int BYTES> __device__ __forceinline__ void cp_async(void* smem, const void* gmem)
+{
+    static_assert(BYTES == 4 || BYTES == 8 || BYTES == 16, "cp.async copies 4, 8 or 16 bytes");
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem),
+                 "n"(BYTES)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 template <int R> __device__ __forceinline__ float square_sum(const float (&kk)[R], float (&kap)[R])
 {
     float sumk = 0.f;
@@ -358,6 +407,13 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
 {
     constexpr int R = K / 32;
     constexpr int PF = 8;   // prefetch distance in tokens
+    struct RingSlot {
+        RawRow<TI, R> k[32];
+        RawRow<float, R> lr[VEC ? 32 : 1];
+        float n[32], rho[32], beta[32];
+    };
+    __shared__ __align__(16) RingSlot ring_all[4][PF];
+    RingSlot* ring = ring_all[threadIdx.x >> 5];
     const int lane = threadIdx.x & 31;
     const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (chain >= a.S * a.H) return;
@@ -436,17 +492,18 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
             if (face && (bits & valid) == valid) {
                 skipped = valid;
             } else {
-                // ring of prefetched rows and scalars
-                float kbuf[PF][R], nbuf[PF], rbuf[PF], bbuf[PF];
-                float lbuf[VEC ? PF : 1][R];   // log-retention rows (vector retention only)
+                // ring of prefetched rows and scalars in shared memory (every lane copies and later reads
+                // its own bytes, the three scalars included, so no lane waits for another)
                 auto fetch = [&](int i, int slot) {
                     const int ii = min(i, len - 1);
                     const size_t th = (size_t)(tok0 + ii) * H + h;
-                    load_row<R>(kp + th * K, lane, kbuf[slot]);
-                    if constexpr (VEC) load_row<R>(a.retsrc + th * K, lane, lbuf[slot]);
-                    nbuf[slot] = a.r.n[th];
-                    rbuf[slot] = a.r.rho[th];
-                    bbuf[slot] = hy.beta_aware ? a.beta[th] : 1.0f;
+                    RingSlot& rs = ring[slot];
+                    cp_async<R * (int)sizeof(TI)>(&rs.k[lane], kp + th * K + R * lane);
+                    if constexpr (VEC) cp_async<R * 4>(&rs.lr[VEC ? lane : 0], a.retsrc + th * K + R * lane);
+                    cp_async<4>(&rs.n[lane], a.r.n + th);
+                    cp_async<4>(&rs.rho[lane], a.r.rho + th);
+                    cp_async<4>(&rs.beta[lane], a.beta + th);
+                    cp_async_commit();
                 };
                 int i = 0;
                 while (i < len) {
@@ -461,6 +518,7 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
                         }
                     }
                     // process tokens i, i+1, ... until d is back on the face (or the chunk ends)
+                    cp_async_wait<0>();   // nothing of an earlier run is still on its way into the ring
 #pragma unroll
                     for (int u = 0; u < PF; ++u) fetch(i + u, u);
                     bool stop = false;
@@ -468,37 +526,55 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
 #pragma unroll
                         for (int u = 0; u < PF; ++u) {
                             if (i < len && !stop) {
+                                cp_async_wait<PF - 1>();   // the oldest group, this token's, has landed
+                                const RingSlot& rs = ring[u];
                                 float kk[R];
-#pragma unroll
-                                for (int r = 0; r < R; ++r) kk[r] = kbuf[u][r];
-                                const float n = fabsf(nbuf[u]), b = bbuf[u];
+                                unpack<R>(rs.k[lane], kk);
+                                const float n = fabsf(rs.n[lane]), b = hy.beta_aware ? rs.beta[lane] : 1.0f;
+                                // c = e - a2 <d, k^2>: e and a2 do not depend on d, so the division is off
+                                // the token-to-token path
+                                const float e = hy.eta * b / n, a2 = e * b;
                                 float rho[R];
+                                if constexpr (VEC) {
+                                    float lr[R];
+                                    unpack<R>(rs.lr[VEC ? lane : 0], lr);
 #pragma unroll
-                                for (int r = 0; r < R; ++r) {
-                                    if constexpr (VEC) rho[r] = expf(lbuf[u][r]);
-                                    else rho[r] = rbuf[u];
+                                    for (int r = 0; r < R; ++r) rho[r] = expf(lr[r]);
+                                } else {
+                                    const float r1 = rs.rho[lane];
+#pragma unroll
+                                    for (int r = 0; r < R; ++r) rho[r] = r1;
                                 }
                                 fetch(i + PF, u);
                                 const size_t th = (size_t)(tok0 + i) * H + h;
-                                float kap[R], wk[R];
+                                float kap[R], wk[R], rd[R], al = 0.f;
 #pragma unroll
                                 for (int r = 0; r < R; ++r) {
                                     kap[r] = kk[r] * kk[r];
                                     wk[r] = d[r] * kk[r];
+                                    rd[r] = rho[r] * d[r];
+                                    al = fmaf(d[r], kap[r], al);
                                 }
+                                al = warp_sum(al);
                                 store_row<R>(kt + th * K, lane, wk);
                                 if (a.save) store_row<R>(a.r.dtraj + th * K, lane, d);
-                                unsigned pass[R];
-                                bool low;
-                                float cc, al;
-                                p1_step<R>(d, kap, n, b, rho, hy, pass, low, cc, al);
-                                if (a.save && lane < R) {
-                                    unsigned wv = 0;
+                                const float cc = fmaf(-a2, al, e);
+                                unsigned mybits = 0;         // bit r: the projection passes gradient for coordinate R lane + r
+                                bool at_min = hy.clamp != 0;
 #pragma unroll
-                                    for (int r = 0; r < R; ++r) wv = lane == r ? pass[r] : wv;
-                                    a.r.pmask[th * R + lane] = wv;
+                                for (int r = 0; r < R; ++r) {
+                                    float x = fmaf(cc, kap[r], rd[r]);
+                                    bool pz = true;
+                                    if (hy.clamp) {
+                                        pz = (x >= hy.d_min) && (x <= hy.d_max);
+                                        x = fminf(fmaxf(x, hy.d_min), hy.d_max);
+                                    }
+                                    mybits |= pz ? (1u << r) : 0u;
+                                    at_min = at_min && (x == hy.d_min);
+                                    d[r] = x;
                                 }
-                                face = on_lower_face<R>(d, hy);
+                                if (a.save) a.r.pmask[th * 32 + lane] = mybits;
+                                face = __all_sync(0xffffffffu, at_min);
                                 ++i;
                                 // back on the face with a flagged token next: leave the run
                                 stop = face && i < len && ((bits >> i) & 1ull);
@@ -613,7 +689,7 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                     prefetch_row(a.dktil + th * K, K * 4);
                     prefetch_row(a.dkread + th * K, K * 4);
                     if constexpr (VEC) prefetch_row(a.log_ret + th * K, K * 4);
-                    prefetch_l2(a.r.pmask + th * R);
+                    prefetch_l2(a.r.pmask + th * 32);
                     prefetch_l2(a.r.n + th);
                     prefetch_l2(a.r.rho + th);
                     prefetch_l2(a.beta + th);
@@ -641,8 +717,9 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
             // recurrence restarts before a token (its upper neighbour was skipped), the two rows the
             // restart needs travel with that token's rows.
             constexpr int PF = 4;
-            float kb[PF][R], db[PF][R], tb[PF][R], rb[PF][R], nb[PF], hb[PF], bb[PF];
-            float sk_k[PF][R], sk_t[PF][R];
+            RawRow<T, R> kb[PF], sk_k[PF];
+            float db[PF][R], tb[PF][R], rb[PF][R], nb[PF], hb[PF], bb[PF];
+            float sk_t[PF][R];
             float lb[VEC ? PF : 1][R];   // log-retention rows (vector retention only)
             unsigned mb[PF];
             bool needr[PF];
@@ -656,21 +733,21 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
             };
             auto fetch = [&](int i, int slot) {
                 const size_t th = (size_t)(tok0 + i) * H + h;
-                load_row<R>(kp + th * K, lane, kb[slot]);
+                load_raw<R>(kp + th * K, lane, kb[slot]);
                 load_row<R>(a.r.dtraj + th * K, lane, db[slot]);
                 load_row<R>(a.dktil + th * K, lane, tb[slot]);
                 load_row<R>(a.dkread + th * K, lane, rb[slot]);
                 if constexpr (VEC) load_row<R>(a.log_ret + th * K, lane, lb[slot]);
-                mb[slot] = lane < R ? a.r.pmask[th * R + lane] : 0u;
+                mb[slot] = a.r.pmask[th * 32 + lane];
                 nb[slot] = a.r.n[th];
                 hb[slot] = a.r.rho[th];
-                bb[slot] = hy.beta_aware ? a.beta[th] : 1.0f;
+                bb[slot] = a.beta[th];
                 const bool top = i == len - 1;
                 const bool need = top ? !valid_in : (((sk >> (i + 1)) & 1ull) != 0ull);
                 needr[slot] = need;
                 if (need) {   // lambda restarts at the lowest token of the skipped run above
                     const size_t ts = (size_t)(top ? src_in : (long)(tok0 + i + 1)) * H + h;
-                    load_row<R>(kp + ts * K, lane, sk_k[slot]);
+                    load_raw<R>(kp + ts * K, lane, sk_k[slot]);
                     load_row<R>(a.dktil + ts * K, lane, sk_t[slot]);
                 }
             };
@@ -684,13 +761,19 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                     if (rem) {
                         const int i = pop_top(rem);
                         float kk[R], kap[R], dt[R], dkt[R], dkr[R], drho = 0.f, dc = 0.f, al = 0.f;
+                        unpack<R>(kb[u], kk);
+                        if (needr[u]) {
+                            float rk[R];
+                            unpack<R>(sk_k[u], rk);
+#pragma unroll
+                            for (int r = 0; r < R; ++r) lam[r] = rk[r] * sk_t[u][r];
+                        }
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
-                            kk[r] = kb[u][r]; dt[r] = db[u][r]; dkt[r] = tb[u][r]; dkr[r] = rb[u][r];
-                            if (needr[u]) lam[r] = sk_k[u][r] * sk_t[u][r];
+                            dt[r] = db[u][r]; dkt[r] = tb[u][r]; dkr[r] = rb[u][r];
                         }
                         const unsigned mw = mb[u];
-                        const float ns = nb[u], n = fabsf(ns), rho = hb[u], b = bb[u];
+                        const float ns = nb[u], n = fabsf(ns), rho = hb[u], b = hy.beta_aware ? bb[u] : 1.0f;
                         float rv[R];
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
@@ -702,8 +785,7 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
                             kap[r] = kk[r] * kk[r];
-                            const unsigned wr = __shfl_sync(0xffffffffu, mw, r);
-                            if (!((wr >> lane) & 1u)) lam[r] = 0.f;
+                            if (!((mw >> r) & 1u)) lam[r] = 0.f;
                             drho = fmaf(lam[r], dt[r], drho);
                             dc = fmaf(lam[r], kap[r], dc);
                             al = fmaf(dt[r], kap[r], al);
