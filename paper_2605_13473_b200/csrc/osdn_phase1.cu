@@ -636,10 +636,22 @@ __global__ void __launch_bounds__(128) phase1_bwd_bulk_kernel(P1Bwd a)
 }
 
 // processed tokens, in reverse; one warp per chain.  Skip words are fetched for 32 chunks at a time.
+constexpr int P1B_WARPS = 2;   // chains per CTA (the ring of a chain takes up to 14 KB of shared memory)
+
 template <typename T, int K, bool VEC>
-__global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
+__global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
 {
     constexpr int R = K / 32;
+    constexpr int PF = 4;   // prefetch distance in processed tokens
+    // ring of prefetched rows and scalars (cp.async; every lane copies and later reads its own bytes)
+    struct BSlot {
+        RawRow<T, R> k[32], sk_k[32];
+        RawRow<float, R> dt[32], dkt[32], dkr[32], sk_t[32], lr[VEC ? 32 : 1];
+        unsigned m[32];
+        float n[32], rho[32], beta[32];
+    };
+    __shared__ __align__(16) BSlot ring_all[P1B_WARPS][PF];
+    BSlot* ring = ring_all[threadIdx.x >> 5];
     const int lane = threadIdx.x & 31;
     const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (chain >= a.S * a.H) return;
@@ -716,13 +728,6 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
             // the next PF of them are always in flight, across runs of skipped tokens.  Where the
             // recurrence restarts before a token (its upper neighbour was skipped), the two rows the
             // restart needs travel with that token's rows.
-            constexpr int PF = 4;
-            RawRow<T, R> kb[PF], sk_k[PF];
-            float db[PF][R], tb[PF][R], rb[PF][R], nb[PF], hb[PF], bb[PF];
-            float sk_t[PF][R];
-            float lb[VEC ? PF : 1][R];   // log-retention rows (vector retention only)
-            unsigned mb[PF];
-            bool needr[PF];
             const unsigned long long todo = ~sk & valid;
             const bool valid_in = lam_valid;
             const long src_in = src;
@@ -731,72 +736,94 @@ __global__ void __launch_bounds__(128) phase1_bwd_seq_kernel(P1Bwd a)
                 m &= ~(1ull << t);
                 return t;
             };
+            // one committed group per ring slot use (an empty one when nothing is left to fetch), so
+            // that "all but the PF - 1 most recent groups" is always the slot about to be read
             auto fetch = [&](int i, int slot) {
                 const size_t th = (size_t)(tok0 + i) * H + h;
-                load_raw<R>(kp + th * K, lane, kb[slot]);
-                load_row<R>(a.r.dtraj + th * K, lane, db[slot]);
-                load_row<R>(a.dktil + th * K, lane, tb[slot]);
-                load_row<R>(a.dkread + th * K, lane, rb[slot]);
-                if constexpr (VEC) load_row<R>(a.log_ret + th * K, lane, lb[slot]);
-                mb[slot] = a.r.pmask[th * 32 + lane];
-                nb[slot] = a.r.n[th];
-                hb[slot] = a.r.rho[th];
-                bb[slot] = a.beta[th];
+                BSlot& rs = ring[slot];
+                cp_async<R * (int)sizeof(T)>(&rs.k[lane], kp + th * K + R * lane);
+                cp_async<R * 4>(&rs.dt[lane], a.r.dtraj + th * K + R * lane);
+                cp_async<R * 4>(&rs.dkt[lane], a.dktil + th * K + R * lane);
+                cp_async<R * 4>(&rs.dkr[lane], a.dkread + th * K + R * lane);
+                if constexpr (VEC) cp_async<R * 4>(&rs.lr[VEC ? lane : 0], a.log_ret + th * K + R * lane);
+                cp_async<4>(&rs.m[lane], a.r.pmask + th * 32 + lane);
+                cp_async<4>(&rs.n[lane], a.r.n + th);
+                cp_async<4>(&rs.rho[lane], a.r.rho + th);
+                cp_async<4>(&rs.beta[lane], a.beta + th);
                 const bool top = i == len - 1;
                 const bool need = top ? !valid_in : (((sk >> (i + 1)) & 1ull) != 0ull);
-                needr[slot] = need;
                 if (need) {   // lambda restarts at the lowest token of the skipped run above
                     const size_t ts = (size_t)(top ? src_in : (long)(tok0 + i + 1)) * H + h;
-                    load_raw<R>(kp + ts * K, lane, sk_k[slot]);
-                    load_row<R>(a.dktil + ts * K, lane, sk_t[slot]);
+                    cp_async<R * (int)sizeof(T)>(&rs.sk_k[lane], kp + ts * K + R * lane);
+                    cp_async<R * 4>(&rs.sk_t[lane], a.dktil + ts * K + R * lane);
                 }
+                cp_async_commit();
+                return need;
             };
+            bool needr[PF];
             unsigned long long pfm = todo, rem = todo;
+            cp_async_wait<0>();
 #pragma unroll
-            for (int u = 0; u < PF; ++u)
-                if (pfm) fetch(pop_top(pfm), u);
+            for (int u = 0; u < PF; ++u) {
+                needr[u] = false;
+                if (pfm) needr[u] = fetch(pop_top(pfm), u);
+                else cp_async_commit();
+            }
             while (rem) {
 #pragma unroll
                 for (int u = 0; u < PF; ++u) {
                     if (rem) {
                         const int i = pop_top(rem);
+                        cp_async_wait<PF - 1>();
+                        const BSlot& rs = ring[u];
                         float kk[R], kap[R], dt[R], dkt[R], dkr[R], drho = 0.f, dc = 0.f, al = 0.f;
-                        unpack<R>(kb[u], kk);
+                        unpack<R>(rs.k[lane], kk);
+                        unpack<R>(rs.dt[lane], dt);
+                        unpack<R>(rs.dkt[lane], dkt);
+                        unpack<R>(rs.dkr[lane], dkr);
                         if (needr[u]) {
-                            float rk[R];
-                            unpack<R>(sk_k[u], rk);
+                            float rk[R], rt[R];
+                            unpack<R>(rs.sk_k[lane], rk);
+                            unpack<R>(rs.sk_t[lane], rt);
 #pragma unroll
-                            for (int r = 0; r < R; ++r) lam[r] = rk[r] * sk_t[u][r];
+                            for (int r = 0; r < R; ++r) lam[r] = rk[r] * rt[r];
                         }
-#pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            dt[r] = db[u][r]; dkt[r] = tb[u][r]; dkr[r] = rb[u][r];
-                        }
-                        const unsigned mw = mb[u];
-                        const float ns = nb[u], n = fabsf(ns), rho = hb[u], b = hy.beta_aware ? bb[u] : 1.0f;
+                        const unsigned mw = rs.m[lane];
+                        const float ns = rs.n[lane], n = fabsf(ns), rho = rs.rho[lane];
+                        const float b = hy.beta_aware ? rs.beta[lane] : 1.0f;
                         float rv[R];
+                        if constexpr (VEC) {
+                            float lr[R];
+                            unpack<R>(rs.lr[VEC ? lane : 0], lr);
 #pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            if constexpr (VEC) rv[r] = expf(lb[u][r]);
-                            else rv[r] = rho;
+                            for (int r = 0; r < R; ++r) rv[r] = expf(lr[r]);
+                        } else {
+#pragma unroll
+                            for (int r = 0; r < R; ++r) rv[r] = rho;
                         }
-                        if (pfm) fetch(pop_top(pfm), u);
+                        if (pfm) needr[u] = fetch(pop_top(pfm), u);
+                        else cp_async_commit();
                         const size_t th = (size_t)(tok0 + i) * H + h;
+                        // what does not depend on lambda first: the step's own scalars
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
                             kap[r] = kk[r] * kk[r];
+                            al = fmaf(dt[r], kap[r], al);
+                        }
+                        al = warp_sum(al);
+                        const float e = hy.eta * b / n, a2 = e * b;
+                        const float cc = fmaf(-a2, al, e);
+                        const float g1 = hy.eta * (1.0f - 2.0f * b * al) / n;
+                        const float g2 = ns > 0.f ? -cc / n : 0.f;
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
                             if (!((mw >> r) & 1u)) lam[r] = 0.f;
                             drho = fmaf(lam[r], dt[r], drho);
                             dc = fmaf(lam[r], kap[r], dc);
-                            al = fmaf(dt[r], kap[r], al);
                         }
-                        drho = warp_sum(drho);
                         dc = warp_sum(dc);
-                        al = warp_sum(al);
-                        const float cc = hy.eta * b * (1.0f - b * al) / n;
-                        const float da = -hy.eta * b * b / n * dc;
-                        const float dbt = hy.eta * (1.0f - 2.0f * b * al) / n * dc;
-                        const float dn = ns > 0.f ? -cc / n * dc : 0.f;
+                        drho = warp_sum(drho);
+                        const float da = -a2 * dc, dbt = g1 * dc, dn = g2 * dc;
                         float out[R];
                         if constexpr (VEC) {   // one gradient per coordinate: r_i lambda_i d_i
                             if (a.dlog_ret) {
@@ -859,8 +886,9 @@ int bwd_launch(const P1Bwd& a, bool bulk, cudaStream_t st)
         ++n;
     }
     stage_mark(st, "phase1_bwd_seq");
-    if (a.hy.apf_mode == 3) phase1_bwd_seq_kernel<T, K, true><<<(a.S * a.H + 3) / 4, 128, 0, st>>>(a);
-    else phase1_bwd_seq_kernel<T, K, false><<<(a.S * a.H + 3) / 4, 128, 0, st>>>(a);
+    const unsigned gseq = (unsigned)((a.S * a.H + P1B_WARPS - 1) / P1B_WARPS);
+    if (a.hy.apf_mode == 3) phase1_bwd_seq_kernel<T, K, true><<<gseq, P1B_WARPS * 32, 0, st>>>(a);
+    else phase1_bwd_seq_kernel<T, K, false><<<gseq, P1B_WARPS * 32, 0, st>>>(a);
     ++n;
     return cudaGetLastError() == cudaSuccess ? n : -1;
 }
