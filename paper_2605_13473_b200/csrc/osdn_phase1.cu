@@ -207,42 +207,79 @@ __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
     }
     const Hyper hy = a.hy;
     float lsum = 0.f;
-    for (int i = 0; i < len; ++i) {
-        const size_t th = (size_t)(t0 + i) * a.H + h;
-        float kk[R], kap[R], w[R];
-        load_row<R>(kp + th * K, lane, kk);
-        const float sumk = square_sum<R>(kk, kap);
-        if (kt) {
-#pragma unroll
-            for (int r = 0; r < R; ++r) w[r] = d[r] * kk[r];
-            store_row<R>(kt + th * K, lane, w);
+    // rows and scalars a few tokens ahead, through a shared-memory ring (every lane copies and later
+    // reads its own bytes; one committed group per token)
+    constexpr int PF = 8;
+    struct Slot {
+        RawRow<TI, R> k[32];
+        RawRow<float, R> lr[VEC ? 32 : 1];
+        float beta[32], ret[32];
+    };
+    __shared__ __align__(16) Slot ring_all[4][PF];
+    Slot* ring = ring_all[threadIdx.x >> 5];
+    const bool scalar_ret = !VEC && hy.apf_mode != 0;
+    auto fetch = [&](int i, int slot) {
+        if (i < len) {
+            const size_t th = (size_t)(t0 + i) * a.H + h;
+            Slot& rs = ring[slot];
+            cp_async<R * (int)sizeof(TI)>(&rs.k[lane], kp + th * K + R * lane);
+            if constexpr (VEC) cp_async<R * 4>(&rs.lr[VEC ? lane : 0], a.retsrc + th * K + R * lane);
+            cp_async<4>(&rs.beta[lane], a.beta + th);
+            if (scalar_ret) cp_async<4>(&rs.ret[lane], a.retsrc + th);
         }
-        const float n = fmaxf(sumk, hy.eps);
-        const float b = hy.beta_aware ? a.beta[th] : 1.0f;
-        float rho[R];
-        if constexpr (VEC) {
-            load_row<R>(a.retsrc + th * K, lane, rho);
+        cp_async_commit();
+    };
 #pragma unroll
-            for (int r = 0; r < R; ++r) rho[r] = expf(rho[r]);
-        } else {
-            const float r1 = hy.apf_mode == 0 ? 1.0f : expf(a.retsrc[th]);
+    for (int u = 0; u < PF; ++u) fetch(u, u);
+    for (int i0 = 0; i0 < len; i0 += PF) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) rho[r] = r1;
-        }
-        unsigned pass[R];
-        bool low;
-        float c, al;
-        p1_step<R>(d, kap, n, b, rho, hy, pass, low, c, al);
-        if (a.ratio || a.log_sum) {
-            // residual ratio of the write of this token (token-local theorem): the loss |S k - v|^2 after
-            // the write over the loss before it is (1 - beta <d_t, k^2>)^2, with the write strength beta
-            // itself (whether or not the step of d is beta-aware) and the d the write key was formed with
-            const float fac = 1.0f - a.beta[th] * al;
-            const float qt = fac * fac;
-            if (a.ratio && lane == 0) a.ratio[th] = qt;
-            lsum += logf(fmaxf(qt, 1.17549435e-38f));
+        for (int u = 0; u < PF; ++u) {
+            const int i = i0 + u;
+            if (i < len) {
+                cp_async_wait<PF - 1>();
+                const Slot& rs = ring[u];
+                const size_t th = (size_t)(t0 + i) * a.H + h;
+                float kk[R], kap[R], w[R];
+                unpack<R>(rs.k[lane], kk);
+                const float beta = rs.beta[lane];
+                float rho[R];
+                if constexpr (VEC) {
+                    float lr[R];
+                    unpack<R>(rs.lr[VEC ? lane : 0], lr);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) rho[r] = expf(lr[r]);
+                } else {
+                    const float r1 = scalar_ret ? expf(rs.ret[lane]) : 1.0f;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) rho[r] = r1;
+                }
+                fetch(i + PF, u);
+                const float sumk = square_sum<R>(kk, kap);
+                if (kt) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) w[r] = d[r] * kk[r];
+                    store_row<R>(kt + th * K, lane, w);
+                }
+                const float n = fmaxf(sumk, hy.eps);
+                const float b = hy.beta_aware ? beta : 1.0f;
+                unsigned pass[R];
+                bool low;
+                float c, al;
+                p1_step<R>(d, kap, n, b, rho, hy, pass, low, c, al);
+                if (a.ratio || a.log_sum) {
+                    // residual ratio of the write of this token (token-local theorem): the loss |S k - v|^2
+                    // after the write over the loss before it is (1 - beta <d_t, k^2>)^2, with the write
+                    // strength beta itself (whether or not the step of d is beta-aware) and the d the write
+                    // key was formed with
+                    const float fac = 1.0f - beta * al;
+                    const float qt = fac * fac;
+                    if (a.ratio && lane == 0) a.ratio[th] = qt;
+                    lsum += logf(fmaxf(qt, 1.17549435e-38f));
+                }
+            }
         }
     }
+    cp_async_wait<0>();
     if (a.d_final) store_row<R>(a.d_final + ((size_t)s * a.H + h) * K, lane, d);
     if (a.log_sum && lane == 0) a.log_sum[(size_t)s * a.H + h] = lsum;
 }
