@@ -54,7 +54,7 @@ struct WsLayout {
     size_t status;      // int32 device status word (+ padding)
     size_t table;       // ints, see carve_table
     // phase 1 (shared by both kernel families)
-    size_t p1n;         // [T,H]          f32   max(|k|^2, eps), negated where the floor is active
+    size_t p1n;         // [T,H]          f32   1 / max(|k|^2, eps), negated where the floor is active
     size_t p1rho;       // [T,H]          f32   retention of the preconditioner
     size_t p1flags;     // [NT,H,2]       u32   per token: the step maps d_min*1 to d_min*1, mask all zero
     size_t p1skip;      // [NT,H,2]       u32   tokens the sequential pass skipped           (save only)

@@ -402,7 +402,7 @@ __global__ void __launch_bounds__(128) phase1_spec_kernel(P1Fwd a)
             }
         }
         if (in && l8 == 0) {
-            a.r.n[th] = sumk > hy.eps ? n : -n;
+            a.r.n[th] = sumk > hy.eps ? 1.0f / n : -1.0f / n;   // reciprocal of the normaliser, signed
             a.r.rho[th] = rho;
         }
         if (low) {   // the write key of a token entered on the face: d_min k
@@ -567,10 +567,10 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
                                 const RingSlot& rs = ring[u];
                                 float kk[R];
                                 unpack<R>(rs.k[lane], kk);
-                                const float n = fabsf(rs.n[lane]), b = hy.beta_aware ? rs.beta[lane] : 1.0f;
-                                // c = e - a2 <d, k^2>: e and a2 do not depend on d, so the division is off
-                                // the token-to-token path
-                                const float e = hy.eta * b / n, a2 = e * b;
+                                const float rn = fabsf(rs.n[lane]), b = hy.beta_aware ? rs.beta[lane] : 1.0f;
+                                // c = e - a2 <d, k^2>: e and a2 do not depend on d (1 / n comes from the
+                                // parallel pass), so nothing but one multiply-add follows the warp sum
+                                const float e = hy.eta * b * rn, a2 = e * b;
                                 float rho[R];
                                 if constexpr (VEC) {
                                     float lr[R];
@@ -826,7 +826,7 @@ __global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
                             for (int r = 0; r < R; ++r) lam[r] = rk[r] * rt[r];
                         }
                         const unsigned mw = rs.m[lane];
-                        const float ns = rs.n[lane], n = fabsf(ns), rho = rs.rho[lane];
+                        const float ns = rs.n[lane], rn = fabsf(ns), rho = rs.rho[lane];
                         const float b = hy.beta_aware ? rs.beta[lane] : 1.0f;
                         float rv[R];
                         if constexpr (VEC) {
@@ -848,10 +848,10 @@ __global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
                             al = fmaf(dt[r], kap[r], al);
                         }
                         al = warp_sum(al);
-                        const float e = hy.eta * b / n, a2 = e * b;
+                        const float e = hy.eta * b * rn, a2 = e * b;
                         const float cc = fmaf(-a2, al, e);
-                        const float g1 = hy.eta * (1.0f - 2.0f * b * al) / n;
-                        const float g2 = ns > 0.f ? -cc / n : 0.f;
+                        const float g1 = hy.eta * (1.0f - 2.0f * b * al) * rn;
+                        const float g2 = ns > 0.f ? -cc * rn : 0.f;
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
                             if (!((mw >> r) & 1u)) lam[r] = 0.f;
