@@ -71,7 +71,8 @@ template <int R> __device__ __forceinline__ void dec_store(float* p, int lane, c
     else *reinterpret_cast<float2*>(p + 2 * lane) = make_float2(x[0], x[1]);
 }
 
-template <typename T, int K, int V>
+// VEC: vector retention (one log-retention per coordinate, log_ret [B,T,H,K]).
+template <typename T, int K, int V, bool VEC>
 __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
 {
     constexpr int R = K / 32;
@@ -93,9 +94,7 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
     dec_load<R>(a.precond + (size_t)chain * K, lane, d);
 
     // inputs of a token, fetched one token ahead
-    float kk[R], qq[R], vv[DEC_RW], bt, gt, lr, lrv[R];
-#pragma unroll
-    for (int j = 0; j < R; ++j) lrv[j] = 0.f;
+    float kk[R], qq[R], vv[DEC_RW], bt, gt, lr, lrv[VEC ? R : 1];
     auto fetch = [&](int t) {
         const size_t th = ((size_t)b * a.L + t) * a.H + h;
         dec_load<R>(kp + th * K, lane, kk);
@@ -105,7 +104,7 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
         bt = a.beta[th];
         gt = a.gate[th];
         lr = hy.apf_mode == 2 ? a.log_ret[th] : 0.f;
-        if (hy.apf_mode == 3) dec_load<R>(a.log_ret + th * K, lane, lrv);   // one log-retention per coordinate
+        if constexpr (VEC) dec_load<R>(a.log_ret + th * K, lane, lrv);   // one log-retention per coordinate
     };
     fetch(0);
     for (int t = 0; t < a.L; ++t) {
@@ -118,7 +117,10 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
         const float rho1 = hy.apf_mode == 0 ? 1.0f : (hy.apf_mode == 1 ? alpha : expf(lr));
         float rho[R];
 #pragma unroll
-        for (int j = 0; j < R; ++j) rho[j] = hy.apf_mode == 3 ? expf(lrv[j]) : rho1;
+        for (int j = 0; j < R; ++j) {
+            if constexpr (VEC) rho[j] = expf(lrv[j]);
+            else rho[j] = rho1;
+        }
         if (t + 1 < a.L) fetch(t + 1);
 
         // preconditioner step
@@ -184,10 +186,17 @@ template <typename T> int launch_typed(const osdn_params& p, const DecArgs& a, c
     const unsigned chains = (unsigned)p.B * (unsigned)p.H;
     const unsigned grid = chains * (unsigned)(p.V / DEC_VB);
     const int threads = DEC_WARPS * 32;
-    if (p.K == 128 && p.V == 128) decode_kernel<T, 128, 128><<<grid, threads, 0, st>>>(a);
-    else if (p.K == 128 && p.V == 64) decode_kernel<T, 128, 64><<<grid, threads, 0, st>>>(a);
-    else if (p.K == 64 && p.V == 128) decode_kernel<T, 64, 128><<<grid, threads, 0, st>>>(a);
-    else decode_kernel<T, 64, 64><<<grid, threads, 0, st>>>(a);
+    if (a.hy.apf_mode == 3) {
+        if (p.K == 128 && p.V == 128) decode_kernel<T, 128, 128, true><<<grid, threads, 0, st>>>(a);
+        else if (p.K == 128 && p.V == 64) decode_kernel<T, 128, 64, true><<<grid, threads, 0, st>>>(a);
+        else if (p.K == 64 && p.V == 128) decode_kernel<T, 64, 128, true><<<grid, threads, 0, st>>>(a);
+        else decode_kernel<T, 64, 64, true><<<grid, threads, 0, st>>>(a);
+    } else {
+        if (p.K == 128 && p.V == 128) decode_kernel<T, 128, 128, false><<<grid, threads, 0, st>>>(a);
+        else if (p.K == 128 && p.V == 64) decode_kernel<T, 128, 64, false><<<grid, threads, 0, st>>>(a);
+        else if (p.K == 64 && p.V == 128) decode_kernel<T, 64, 128, false><<<grid, threads, 0, st>>>(a);
+        else decode_kernel<T, 64, 64, false><<<grid, threads, 0, st>>>(a);
+    }
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
