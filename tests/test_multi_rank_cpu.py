@@ -75,3 +75,89 @@ def test_shard_sequences_properties():
             assert tokens == sum(lens[i] for i in mine)
         assert sorted(seen) == list(range(len(lens)))
         assert max(loads) <= max(max(lens), -(-sum(lens) // world) + max(lens))
+
+
+# ---------------------------------------------------------------------------------------------
+# one sequence cut along T over the ranks: the state and the preconditioner are handed on
+# ---------------------------------------------------------------------------------------------
+def _seq_worker(rank, world, port, out):
+    from paper_2605_13473_b200.sharding import backward_handoff, forward_handoff, segment_bounds
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        B, T, H, K, V = 2, 150, 2, 8, 8
+        hy = OsdnHyper(eta=0.3, apf_mode=2)
+        inp = draw("seqshard", 77, [T] * B, H, K, V, "fp32", dense_B=B, hyper=hy, with_dout=True,
+                   with_log_ret=True, with_state=True, with_state_cotangents=True)
+        f64 = lambda t: None if t is None else t.double().numpy()
+        x = {n: f64(getattr(inp, n)) for n in ("q", "k", "v", "beta", "gate", "log_ret", "dout", "init_state",
+                                               "precond_in", "dfinal_state", "dprecond_out")}
+        lo, hi = segment_bounds(T, world)[rank]
+        ok = True
+        worst = 0.0
+        full_f = oracle.fwd(hy, [T] * B, x["q"], x["k"], x["v"], x["beta"], x["gate"], x["log_ret"],
+                            x["init_state"], x["precond_in"])
+        full_b = oracle.bwd(hy, [T] * B, x["q"], x["k"], x["v"], x["beta"], x["gate"], x["dout"], x["log_ret"],
+                            x["init_state"], x["precond_in"], x["dfinal_state"], x["dprecond_out"])
+        saved = []
+        for b in range(B):   # micro-batches: one sequence each, the ranks form a pipeline
+            sl = slice(b * T + lo, b * T + hi)
+            S_in = torch.from_numpy(x["init_state"][b:b + 1].copy())
+            d_in = torch.from_numpy(x["precond_in"][b:b + 1].copy())
+
+            def run(S, d):
+                if hi == lo:
+                    return None, S, d
+                r = oracle.fwd(hy, [hi - lo], x["q"][sl], x["k"][sl], x["v"][sl], x["beta"][sl], x["gate"][sl],
+                               x["log_ret"][sl], S.numpy(), d.numpy())
+                return r["out"], torch.from_numpy(r["final_state"]), torch.from_numpy(r["precond_out"])
+            res, S_out, d_out = forward_handoff(run, S_in, d_in, rank, world)
+            saved.append((S_in.clone(), d_in.clone()))
+            if res is not None:
+                worst = max(worst, float(np.abs(res - full_f["out"][sl]).max()))
+            if rank == world - 1:
+                worst = max(worst, float(np.abs(S_out.numpy() - full_f["final_state"][b:b + 1]).max()),
+                            float(np.abs(d_out.numpy() - full_f["precond_out"][b:b + 1]).max()))
+        for b in range(B):
+            sl = slice(b * T + lo, b * T + hi)
+            S_in, d_in = saved[b]
+            dS = torch.from_numpy(x["dfinal_state"][b:b + 1].copy())
+            dd = torch.from_numpy(x["dprecond_out"][b:b + 1].copy())
+
+            def run_bwd(dS_r, dd_r):
+                if hi == lo:
+                    return None, dS_r, dd_r
+                g = oracle.bwd(hy, [hi - lo], x["q"][sl], x["k"][sl], x["v"][sl], x["beta"][sl], x["gate"][sl],
+                               x["dout"][sl], x["log_ret"][sl], S_in.numpy(), d_in.numpy(), dS_r.numpy(), dd_r.numpy())
+                return g, torch.from_numpy(g["dinit_state"]), torch.from_numpy(g["dprecond_in"])
+            g, dS_in, dd_in = backward_handoff(run_bwd, dS, dd, rank, world)
+            if g is not None:
+                for name in ("dq", "dk", "dv", "dbeta", "dgate", "dlog_ret"):
+                    worst = max(worst, float(np.abs(g[name] - full_b[name][sl]).max()))
+            if rank == 0:
+                worst = max(worst, float(np.abs(dS_in.numpy() - full_b["dinit_state"][b:b + 1]).max()),
+                            float(np.abs(dd_in.numpy() - full_b["dprecond_in"][b:b + 1]).max()))
+        out.put((rank, ok, worst, hi - lo))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_sequence_cut_over_ranks_hands_state_and_cotangents_on():
+    from paper_2605_13473_b200.sharding import segment_bounds
+    assert segment_bounds(150, 3) == [(0, 64), (64, 128), (128, 150)]
+    assert segment_bounds(65, 3) == [(0, 64), (64, 65), (65, 65)]
+    assert segment_bounds(4096, 4)[2] == (2048, 3072)
+    world = 3
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_seq_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(q.get(timeout=180) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [r[3] for r in results] == [64, 64, 22]
+    for rank, ok, worst, n in results:
+        assert ok and worst <= 1e-9, (rank, worst)
