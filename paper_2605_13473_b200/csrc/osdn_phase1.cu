@@ -9,12 +9,17 @@
 //  * Once every coordinate of d sits on the lower face of the box, the step for token t maps
 //    d_min*1 to d_min*1 again iff every pre-projection value rho_t d_min + c_t k_t^2 is below d_min,
 //    a condition that involves token t alone.  phase1_spec evaluates that step for every token
-//    ("flag" bit), one thread per token; from the face the step has a closed form.  The sequential kernel
+//    ("flag" bit), eight lanes per token; from the face the step has a closed form.  The sequential kernel
 //    (phase1_seq) then only walks tokens where d is not on the face or the flag is clear; flagged
 //    tokens entered on the face are skipped (their write key d_min*k was already emitted, their
 //    projection mask is all zero).  On the benchmark distributions with the retention aliased to
 //    the gate this removes almost every token from the chain; on inputs where d really moves it
 //    degenerates to the plain sequential scan.
+//
+// The sequential kernels run one warp per chain, so only the warp's own look-ahead hides memory
+// latency: rows are fetched a few tokens ahead into a shared-memory ring with cp.async, whose
+// completion is counted per committed group, first in first out (rows prefetched into registers
+// are held back by the few counters a warp has for outstanding loads).
 //
 // For the backward pass the forward records, per processed token, d_t and the projection mask,
 // and per chunk which tokens were skipped.  A skipped token has an all-zero mask, so the reverse
