@@ -75,6 +75,17 @@ def test_shapes_and_ragged_tails(T, K, V, path, flags):
     _check(inp, True, f"shape_T{T}_K{K}_V{V}_{path}", flags=flags)
 
 
+@pytest.mark.parametrize("io", ["fp32", "bf16"])
+@pytest.mark.parametrize("K,V", [(64, 64), (64, 128)])
+def test_vector_retention_small_heads_and_ragged_batch(K, V, io):
+    """One log-retention per coordinate with K = 64 (two coordinates per lane), packed ragged batch
+    with an empty sequence, forward and backward."""
+    hy = OsdnHyper(eta=0.3, apf_mode=3)
+    inp = draw(f"vec_{K}_{V}_{io}", 990 + K + V, [130, 0, 65, 1], 2, K, V, io, hyper=hy, key_kind="sparse",
+               with_dout=True, with_log_ret=True, with_state=True, with_state_cotangents=True, log_ret_shift=3.0)
+    _check(inp, True, f"vector_ret_K{K}_V{V}_{io}")
+
+
 @pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])
 def test_degenerate_inputs(path, flags):
     hy = OsdnHyper(eta=0.3, apf_mode=1)
