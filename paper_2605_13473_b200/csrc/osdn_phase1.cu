@@ -632,6 +632,7 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
         }
     }
     if (a.d_final) store_row<R>(a.d_final + ((size_t)s * H + h) * K, lane, d);
+    cp_async_wait<0>();   // rows fetched past the last processed token are not used, but must have landed
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -901,6 +902,7 @@ __global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
         if (!lam_valid) restart(src);
         store_row<R>(a.dprecond_in + ((size_t)s * H + h) * K, lane, lam);
     }
+    cp_async_wait<0>();
 }
 
 template <typename TI, typename TO, int K>
