@@ -63,11 +63,34 @@ def make_inputs(name):
 
 
 # ---------------------------------------------------------------------------------------------
-# Algorithmic work of each kernel per launch (bytes it must read + write given the data flow of
-# the design, and tensor flops), as a function of the workload.  Stated in the design doc.
+# Work of each kernel per launch, as a function of the workload.
+#   method_bytes : the bytes of the METHOD that the kernel is the one to move -- user tensors it reads
+#                  or writes and the per-chunk state the backward is entitled to (one bf16 state
+#                  image per 64 tokens) -- independent of how this design splits the work.  The
+#                  roofline fraction is computed from these.
+#   kernel_model : the bytes the DESIGN makes the kernel read + write (its tiles included) and its
+#                  tensor flops; reported beside the fraction as `design_bytes`, never as its numerator.
 # ---------------------------------------------------------------------------------------------
+def method_bytes(name, inp, with_bwd):
+    """Method bytes per launch of one kernel (see above); None for kernels outside the table."""
+    K, V = inp.K, inp.V
+    es = 2 if inp.io_dtype == "bf16" else 4
+    tokh = inp.T_total * inp.H
+    state = V * K * 2 / 64.0          # one bf16 state image per 64-token chunk, per token-head
+    per = {
+        "phase1_spec": K * es + 8,                                   # k, beta, gate
+        "phase1_seq": 0.0, "phase1_bwd_seq": 0.0, "build_table": 0.0,
+        "tc_chunk_fwd": 2 * K * es + 8,                              # q, k, beta, gate
+        "tc_chain_fwd": V * es + V * es + (state if with_bwd else 0),  # v in, out, saved state
+        "tc_chain_bwd": V * es,                                      # dout
+        # q, k, v, dout, beta, gate, the saved state in; dq, dk, dv, dbeta, dgate out
+        "tc_chunk_bwd": (2 * K + 2 * V) * es + 8 + state + (2 * K + V) * es + 8,
+    }
+    return None if name not in per else per[name] * tokh
+
+
 def kernel_model(name, inp, NT):
-    """returns (bytes, flops, bound) for one launch; NT = number of 64-token chunks (all heads excluded)."""
+    """returns (design bytes, flops, bound) for one launch; NT = number of 64-token chunks (all heads excluded)."""
     H, K, V = inp.H, inp.K, inp.V
     T = inp.T_total
     es = 2 if inp.io_dtype == "bf16" else 4
@@ -94,7 +117,7 @@ def kernel_model(name, inp, NT):
     m["phase1_seq"] = (tiles * (16 + K * 4), 0.0, "hbm")          # pinned regime: flag words + chunk-start d
     m["phase1_bwd_seq"] = (tiles * 8, 0.0, "hbm")
     m["phase1_bwd_bulk"] = (tokh * (2 * K * 4 + K * es), tokh * 2.0 * K, "hbm")
-    # tensor-core family: bytes of the tiles each kernel must read and write (bf16 images)
+    # tensor-core family: bytes of the tiles each kernel reads and writes in this design (bf16 images)
     raw = C * K * es                                               # one [64 x 128] user tile
     m["tc_chunk_fwd"] = (tiles * (3 * raw + 16384 + 8192 + 8192 + 8192 + 16384) + tokh * 8,
                          tiles * (f(128, 64, K) + f(128, 64, C)), "hbm")
@@ -108,18 +131,32 @@ def kernel_model(name, inp, NT):
     return m.get(name)
 
 
-def load_traffic(workload, kernel):
-    """DRAM bytes (read + write) of one launch of `kernel`, from the committed ncu summary of this
-    workload (a line "- traffic_bytes <kernel> = <bytes>"), or None when there is no capture."""
-    path = os.path.join(ROOT, "profiles", f"osdn_step_{workload}.md")
+def load_traffic(workload, kernel, measured_us=None):
+    """DRAM bytes (read + write) of one launch of `kernel` from the committed ncu summary of this
+    workload (lines "- traffic_bytes <kernel> = <bytes>" and "- profile_us <kernel> = <duration>").
+    The capture belongs to the build it was taken on: when the kernel's duration in the capture and the
+    one measured now differ by more than 15 % the figure is stale and dropped.  Returns
+    (bytes or None, a note naming the source)."""
+    rel = os.path.join("profiles", f"osdn_step_{workload}.md")
+    nbytes, prof_us = None, None
     try:
-        for line in open(path):
+        for line in open(os.path.join(ROOT, rel)):
             parts = line.split()
-            if len(parts) >= 5 and parts[0] == "-" and parts[1] == "traffic_bytes" and parts[2] == kernel:
-                return float(parts[4])
+            if len(parts) >= 5 and parts[0] == "-" and parts[2] == kernel:
+                if parts[1] == "traffic_bytes":
+                    nbytes = float(parts[4])
+                elif parts[1] == "profile_us":
+                    prof_us = float(parts[4])
     except OSError:
-        pass
-    return None
+        return None, "no ncu capture committed for this workload"
+    if nbytes is None:
+        return None, f"{rel} has no capture of this kernel"
+    if prof_us is not None and measured_us:
+        if abs(prof_us - measured_us) > 0.15 * measured_us:
+            return None, (f"{rel} is stale: the captured launch took {prof_us:.1f} us, this build "
+                          f"{measured_us:.1f} us")
+        return nbytes, f"{rel} (ncu capture, {prof_us:.1f} us per launch there)"
+    return nbytes, f"{rel} (ncu capture)"
 
 
 class ClockSampler:
@@ -300,7 +337,7 @@ def run_decode(args):
     nbytes = B * H * (2 * D * D * 4 + 2 * D * 4 + (2 * D + 2 * D) * 2 + 8)   # state and d in+out, q k v out, beta gate
     ach = nbytes / avg_s / 1e9
     roofline = dict(kernel="decode_step", bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
-                    frac=ach / peaks["hbm_gbs"], traffic=load_traffic("decode", "decode_step"),
+                    frac=ach / peaks["hbm_gbs"], traffic=load_traffic("decode", "decode_step")[0],
                     peak_source=peaks["source"], avg_us=avg_s * 1e6, algorithmic_bytes=nbytes)
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -343,6 +380,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core fp32 kernels")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a graph replay")
+    ap.add_argument("--no-lively", action="store_true", help="skip the moving-preconditioner sub-record of cfg2")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the two-second back-to-back run")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -376,75 +415,117 @@ def main():
     w = WORKLOADS[args.workload]
     inp = make_inputs(args.workload)
     flags = binding.FLAG_FORCE_SIMT if args.simt else 0
-    b = binding.DeviceBundle(inp, dev, need_bwd=w["bwd"], flags=flags)
     tokens = inp.T_total
-
-    def step():
-        if w["bwd"]:
-            b.fwd(save=True)
-            n = binding.osdn_last_launch_count()
-            b.bwd(residuals_valid=True)
-            return n + binding.osdn_last_launch_count()
-        b.fwd(save=False)
-        return binding.osdn_last_launch_count()
 
     def sync_all():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(warmup):
-        step()
-    torch.cuda.synchronize()
-    assert b.device_status() == 0, "device-side error recorded during warm-up"
+    def prepare(inputs, with_bwd):
+        """Device bundle, a step function and (unless --no-graph) a CUDA graph holding one step."""
+        bundle = binding.DeviceBundle(inputs, dev, need_bwd=with_bwd, flags=flags)
 
-    # One step (osdn_fwd + osdn_bwd through the C ABI) captured once as a CUDA graph and replayed K
-    # times: the calls only enqueue kernels on the stream they are given, so the capture holds exactly
-    # the launches of the plain call sequence, without the launch gaps between them.
-    graph, per_step = None, 0
-    if not args.no_graph:
-        try:
-            cap = torch.cuda.Stream()
-            with torch.cuda.stream(cap):
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(graph, stream=cap):
-                    per_step = step()
-            torch.cuda.synchronize()
-            for _ in range(3):
+        def step():
+            if with_bwd:
+                bundle.fwd(save=True)
+                n = binding.osdn_last_launch_count()
+                bundle.bwd(residuals_valid=True)
+                return n + binding.osdn_last_launch_count()
+            bundle.fwd(save=False)
+            return binding.osdn_last_launch_count()
+
+        for _ in range(warmup):
+            step()
+        torch.cuda.synchronize()
+        assert bundle.device_status() == 0, "device-side error recorded during warm-up"
+        # One step (osdn_fwd + osdn_bwd through the C ABI) captured once as a CUDA graph and replayed:
+        # the calls only enqueue kernels on the stream they are given, so the capture holds exactly
+        # the launches of the plain call sequence, without the launch gaps between them.
+        graph, per_step = None, 0
+        if not args.no_graph:
+            try:
+                cap = torch.cuda.Stream()
+                with torch.cuda.stream(cap):
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=cap):
+                        per_step = step()
+                torch.cuda.synchronize()
+                for _ in range(3):
+                    graph.replay()
+                torch.cuda.synchronize()
+            except Exception as exc:   # report and time the plain call sequence instead
+                print(f"bench: graph capture failed ({exc}); timing plain launches", file=sys.stderr)
+                graph = None
+                torch.cuda.synchronize()
+        return bundle, step, graph, per_step
+
+    def timed(step, graph, per_step, n):
+        """n steps between two events on the current stream; returns (ms, launches)."""
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches = 0
+        e0.record()
+        for _ in range(n):
+            if graph is not None:
                 graph.replay()
-            torch.cuda.synchronize()
-        except Exception as exc:   # report and time the plain call sequence instead
-            print(f"bench: graph capture failed ({exc}); timing plain launches", file=sys.stderr)
-            graph = None
-            torch.cuda.synchronize()
+                launches += per_step
+            else:
+                launches += step()
+        e1.record()
+        sync_all()
+        return e0.elapsed_time(e1), launches
 
+    def per_kernel(step, n):
+        """The same steps once more with an event between every two launches (the events cost a few
+        percent of a step, so they stay out of the region `value` is timed on)."""
+        binding.stage_timing_enable(True)
+        sync_all()
+        for _ in range(n):
+            step()
+        sync_all()
+        st = binding.stage_timing_collect()
+        binding.stage_timing_enable(False)
+        return st
+
+    b, step, graph, per_step = prepare(inp, w["bwd"])
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches = 0
-    e0.record()
-    for _ in range(steps):
-        if graph is not None:
-            graph.replay()
-            launches += per_step
-        else:
-            launches += step()
-    e1.record()
-    sync_all()
-    ms_total = e0.elapsed_time(e1)
-    # Per-kernel durations: the same K steps once more, now with an event between every two launches
-    # (the events cost a few percent of a step, so they stay out of the region `value` is timed on).
-    binding.stage_timing_enable(True)
-    sync_all()
-    for _ in range(steps):
-        step()
-    sync_all()
-    stages = binding.stage_timing_collect()
-    binding.stage_timing_enable(False)
+    ms_total, launches = timed(step, graph, per_step, steps)
+    stages = per_kernel(step, steps)
     clocks = sampler.stop()
     assert b.device_status() == 0, "device-side error recorded during the timed region"
+
+    # ---- sustained: the same step back to back for at least two seconds, clocks sampled meanwhile ----
+    sustained = None
+    if not args.no_sustained:
+        n_sus = max(steps, int(2000.0 / max(ms_total / steps, 1e-3)) + 1)
+        sus_sampler = ClockSampler(local)
+        sus_sampler.start()
+        time.sleep(0.2)
+        ms_sus, _ = timed(step, graph, per_step, n_sus)
+        sus_clocks = sus_sampler.stop()
+        mhz = sus_clocks.get("sm_mhz")
+        sustained = dict(steps=n_sus, seconds=ms_sus * 1e-3, ms_per_step=ms_sus / n_sus,
+                         tokens_per_s=tokens * n_sus / (ms_sus * 1e-3), sm_mhz_median=mhz,
+                         ms_times_mhz=(ms_sus / n_sus * mhz) if mhz else None, power_w_max=sus_clocks.get("power_w_max"),
+                         reasons=sus_clocks.get("reasons"))
+
+    # ---- the same shape with a preconditioner that really moves (no token is skipped) --------------
+    lively = None
+    if args.workload == "cfg2" and not args.no_lively and not args.simt:
+        linp = make_inputs("cfg2_lively")
+        lb, lstep, lgraph, lper = prepare(linp, True)
+        ms_l, _ = timed(lstep, lgraph, lper, steps)
+        lst = per_kernel(lstep, steps)
+        assert lb.device_status() == 0
+        ltot = {k: sum(v) / len(v) * 1e3 for k, v in lst.items()}
+        ldom = max(ltot, key=ltot.get) if ltot else None
+        lively = dict(workload=WORKLOADS["cfg2_lively"]["desc"], ms_per_step=ms_l / steps,
+                      tokens_per_s=linp.T_total * steps / (ms_l * 1e-3), dominant_kernel=ldom,
+                      kernels_us={k: round(v, 1) for k, v in sorted(ltot.items(), key=lambda kv: -kv[1])})
+        del lb, lstep, lgraph
 
     # ---- end to end through the host-buffer entry point --------------------------------------
     e2e = None
@@ -492,7 +573,7 @@ def main():
 
     peaks = load_peaks()
     value = total_tokens / (ms_total * 1e-3)
-    # dominant kernel and its roofline
+    # dominant kernel and its roofline: method bytes (or flops) per launch over the measured duration
     totals = {k: sum(v) for k, v in stages.items()}
     NT = sum((L + 63) // 64 for L in inp.seq_lens)
     roofline = None
@@ -504,30 +585,50 @@ def main():
         dom = max(totals, key=totals.get)
         avg_s = totals[dom] / len(stages[dom]) * 1e-3
         model = kernel_model(dom, inp, NT)
+        mbytes = method_bytes(dom, inp, w["bwd"])
         if model:
-            nbytes, flops, bound = model
+            dbytes, flops, bound = model
+            traffic, traffic_source = load_traffic(args.workload, dom, avg_s * 1e6)
             if bound == "tensor":
                 ach, peak, unit = flops / avg_s / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
             elif bound == "alu":
                 # fp32 FMA peak of the chip: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
                 ach, peak, unit = flops / avg_s / 1e12, 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
             else:
-                ach, peak, unit = nbytes / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
+                nb = mbytes if mbytes is not None else dbytes
+                ach, peak, unit = nb / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
             roofline = dict(kernel=dom, bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak,
-                            traffic=load_traffic(args.workload, dom), peak_source=peaks["source"], avg_us=avg_s * 1e6,
-                            algorithmic_bytes=nbytes, algorithmic_flops=flops)
-    # whole-step roofline (the slower of the step's flops at tensor peak and its bytes at HBM peak)
+                            traffic=traffic, traffic_source=traffic_source, peak_source=peaks["source"],
+                            avg_us=avg_s * 1e6,
+                            algorithmic_bytes=mbytes if (mbytes is not None and bound == "hbm") else dbytes,
+                            algorithmic_bytes_kind=("method bytes moved by this kernel (user tensors and one bf16 "
+                                                    "state image per chunk)" if (mbytes is not None and bound == "hbm")
+                                                    else "bytes of the design's data flow"),
+                            design_bytes=dbytes, design_frac=(dbytes / avg_s / 1e9 / peaks["hbm_gbs"]) if bound == "hbm" else None,
+                            algorithmic_flops=flops)
+    # whole-step roofline (the slower of the step's flops at tensor peak and its bytes at HBM peak), for
+    # two byte counts: the least any implementation moves (inputs, outputs, gradients once) and the
+    # method's count with one bf16 state image per chunk saved by the forward and read by the backward
     es = 2 if inp.io_dtype == "bf16" else 4
     tokh = tokens * inp.H
+    state = inp.V * inp.K * 2 / 64.0
     if w["bwd"]:
-        step_bytes = tokh * ((2 * inp.K + inp.V) * es * 2 + inp.V * es * 2 + 16 + 16) + 0.0
+        min_bytes = tokh * ((2 * inp.K + inp.V) * es * 2 + inp.V * es * 2 + 16 + 16) + 0.0
+        fwd_b = (2 * inp.K + inp.V) * es + 8 + inp.V * es + state + 8
+        bwd_b = (2 * inp.K + inp.V) * es + inp.V * es + state + 8 + (2 * inp.K + inp.V) * es + 8
+        method_step_bytes = tokh * (fwd_b + bwd_b)
         step_flops = tokh * 0.67e6 * (inp.K * inp.V) / (128 * 128)
     else:
-        step_bytes = tokh * ((2 * inp.K + 2 * inp.V) * es + 8)
+        min_bytes = tokh * ((2 * inp.K + 2 * inp.V) * es + 8)
+        method_step_bytes = min_bytes
         step_flops = tokh * 139264.0 * (inp.K * inp.V) / (128 * 128)
-    t_roof = max(step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (peaks["bf16_tflops"] * 1e12))
-    step_roof = dict(roofline_us=t_roof * 1e6, measured_us=ms_total / steps * 1e3,
-                     frac=t_roof / (ms_total / steps * 1e-3), min_bytes=step_bytes, flops=step_flops)
+    t_flop = step_flops / (peaks["bf16_tflops"] * 1e12)
+    t_roof = max(min_bytes / (peaks["hbm_gbs"] * 1e9), t_flop)
+    t_roof_m = max(method_step_bytes / (peaks["hbm_gbs"] * 1e9), t_flop)
+    step_s = ms_total / steps * 1e-3
+    step_roof = dict(roofline_us=t_roof * 1e6, measured_us=step_s * 1e6, frac=t_roof / step_s, min_bytes=min_bytes,
+                     flops=step_flops, method_bytes=method_step_bytes, method_roofline_us=t_roof_m * 1e6,
+                     method_frac=t_roof_m / step_s)
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -559,7 +660,8 @@ def main():
         "clocks": clocks, "gpu_launches": launches,
         "e2e": ({"value": total_tokens / (e2e["ms"] * 1e-3), "unit": "tokens/s",
                  "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"]} if e2e else None),
-        "roofline": roofline, "step_roofline": step_roof, "kernels": kernel_table, "cpu_baseline": cpu_baseline,
+        "roofline": roofline, "step_roofline": step_roof, "kernels": kernel_table, "lively": lively,
+        "sustained": sustained, "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line), flush=True)
     if world > 1:

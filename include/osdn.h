@@ -58,6 +58,17 @@ typedef enum osdn_status {
     OSDN_STATIC_SCRATCH_TOO_SMALL = -6 /* osdn_fwd_static: problem larger than the built-in scratch */
 } osdn_status;
 
+/* Values found in the device status word (first 4 bytes of a workspace) after a call whose kernels
+ * met an error on the device.  101..113: a bounded wait inside a tensor-core kernel ran out (the
+ * kernel then skipped the dependent work and returned; outputs of that call are undefined). */
+enum {
+    OSDN_DEVICE_OK = 0,
+    OSDN_DEVICE_BAD_CU_SEQLENS = 120,   /* cu_seqlens broke its contract (cu[0] != 0, a decreasing pair,
+                                           cu[nseq] != T); sequences were clamped into [0, T], so no
+                                           access left the user tensors, but the results are undefined */
+    OSDN_DEVICE_SELFTEST_TIMEOUT = 199  /* written by osdn_selftest_wait_timeout                         */
+};
+
 enum { OSDN_FP32 = 0, OSDN_BF16 = 1 };
 /* Retention of the preconditioner (Eq. "dt_update_apf"): none, the layer's gate, a separate
  * log-retention per (token, head), or one per coordinate (the vector-retention extension of the
@@ -200,12 +211,18 @@ int osdn_decode_step(const osdn_params* p, const void* q, const void* k, const v
  *     the call clears the part that has to start at zero itself.  Two calls that overlap on the
  *     GPU (different streams, or different host threads without ordering) race on the array and
  *     give undefined results: serialise them.
+ *   - The array is looked up for the device that is current when the call is made: `cuda_stream`
+ *     must be a stream of that device.
+ *   - The device status word of such a call sits inside the array, where the caller cannot point
+ *     osdn_read_device_status at it: osdn_read_static_status reads it (synchronous 4-byte copy from
+ *     the array of the current device; call it after synchronising the stream).
  */
 #define OSDN_STATIC_SCRATCH_BYTES (32u << 20)
 int osdn_fwd_static(const osdn_params* p, const void* q, const void* k, const void* v,
                     const float* beta, const float* gate, const float* apf_log_ret,
                     const float* init_state, const float* precond_in,
                     void* out, float* final_state, float* precond_out, void* cuda_stream);
+int osdn_read_static_status(int32_t* status_host);
 
 /*
  * Host-buffer convenience for end-to-end measurements: copies the inputs (HOST pointers,
@@ -241,6 +258,17 @@ int osdn_workspace_region(const osdn_params* p, int need_bwd, const char* name, 
 /* Reads the device status word at the head of a workspace (synchronous 4-byte copy).
  * 0 = no device-side error recorded. */
 int osdn_read_device_status(const void* workspace, int32_t* status_host);
+
+/*
+ * Self-test of the device-side error path (no counterpart in the paper).  Every wait inside the
+ * tensor-core kernels is bounded: when it runs out the kernel records a code in the device status
+ * word and returns instead of spinning.  This call exercises exactly that mechanism by itself: it
+ * clears the status word of `workspace` (device memory, >= 256 bytes, 256-byte aligned) and launches
+ * one warp that waits, for at most about `limit_us` microseconds (1..100000), on a barrier nothing
+ * ever arrives on.  The kernel returns by itself; after synchronising the stream
+ * osdn_read_device_status yields OSDN_DEVICE_SELFTEST_TIMEOUT.
+ */
+int osdn_selftest_wait_timeout(void* workspace, uint32_t limit_us, void* cuda_stream);
 
 const char* osdn_status_string(int status);
 

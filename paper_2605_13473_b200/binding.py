@@ -19,7 +19,8 @@ EXPORTS = [
     "osdn_workspace_bytes", "osdn_fwd", "osdn_bwd", "osdn_precond_update", "osdn_host_staging_bytes",
     "osdn_step_host", "osdn_read_device_status", "osdn_status_string", "osdn_last_launch_count",
     "osdn_stage_timing_enable", "osdn_stage_timing_read", "osdn_workspace_region",
-    "osdn_fwd_static", "osdn_decode_step", "osdn_residual_ratio",
+    "osdn_fwd_static", "osdn_decode_step", "osdn_residual_ratio", "osdn_read_static_status",
+    "osdn_selftest_wait_timeout",
 ]
 
 
@@ -66,6 +67,10 @@ def load_library(path: Optional[str] = None):
     lib.osdn_step_host.argtypes = [pp] + [vp] * 12 + [vp, sz, vp]
     lib.osdn_read_device_status.restype = ci
     lib.osdn_read_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.osdn_read_static_status.restype = ci
+    lib.osdn_read_static_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+    lib.osdn_selftest_wait_timeout.restype = ci
+    lib.osdn_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, vp]
     lib.osdn_status_string.restype = ctypes.c_char_p
     lib.osdn_status_string.argtypes = [ci]
     lib.osdn_last_launch_count.restype = ci
@@ -193,6 +198,22 @@ def osdn_fwd_static(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, init_state,
     return int(lib.osdn_fwd_static(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gate),
                                    _ptr(apf_log_ret), _ptr(init_state), _ptr(precond_in), _ptr(out),
                                    _ptr(final_state), _ptr(precond_out), _stream_ptr()))
+
+
+def osdn_read_static_status() -> int:
+    """Device status word of the most recent ``osdn_fwd_static`` call on the current device
+    (0 = no device-side error).  Synchronise the stream first."""
+    lib = load_library()
+    st = ctypes.c_int32(0)
+    _check(lib.osdn_read_static_status(ctypes.byref(st)), "osdn_read_static_status")
+    return int(st.value)
+
+
+def osdn_selftest_wait_timeout(workspace: torch.Tensor, limit_us: int) -> None:
+    """Launches the self-test of the bounded device-side wait on ``workspace`` (>= 256 bytes)."""
+    lib = load_library()
+    _check(lib.osdn_selftest_wait_timeout(_ptr(workspace), ctypes.c_uint32(limit_us), _stream_ptr()),
+           "osdn_selftest_wait_timeout")
 
 
 def osdn_bwd(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, init_state, precond_in, dout, dfinal_state,

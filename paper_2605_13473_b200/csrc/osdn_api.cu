@@ -15,6 +15,7 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
                 cudaStream_t st);
 bool tc_supported(const osdn_params& p);
 bool tc_backward_supported(const osdn_params& p);
+int launch_wait_timeout_selftest(int* status, long long limit_cycles, int code, cudaStream_t st);
 }  // namespace osdn
 
 using namespace osdn;
@@ -431,7 +432,8 @@ constexpr int MAX_DEVICES = 64;
 std::mutex g_static_mutex;
 void* g_static_ptr[MAX_DEVICES] = {};
 
-// Device address of g_static_scratch on the current device (looked up on first use).
+// Device address of g_static_scratch on the current device (looked up on first use).  The stream a
+// caller passes must belong to the device that is current at the call.
 void* static_scratch_address()
 {
     int dev = -1;
@@ -476,6 +478,28 @@ int osdn_fwd_static(const osdn_params* p, const void* q, const void* k, const vo
     if (n < 0) return OSDN_CUDA_ERROR;
     g_last_launches = n;
     return OSDN_OK;
+}
+
+int osdn_read_static_status(int32_t* status_host)
+{
+    if (!status_host) return OSDN_INVALID_ARG;
+    void* scratch = static_scratch_address();
+    if (!scratch) return OSDN_CUDA_ERROR;
+    return cudaMemcpy(status_host, scratch, sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess
+               ? OSDN_OK : OSDN_CUDA_ERROR;
+}
+
+int osdn_selftest_wait_timeout(void* workspace, uint32_t limit_us, void* cuda_stream)
+{
+    if (!workspace || limit_us == 0 || limit_us > 100000u) return OSDN_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return OSDN_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) return OSDN_CUDA_ERROR;
+    // about 2000 clock cycles per microsecond at the chip's highest clock: the limit is an upper bound
+    const long long cycles = 2000ll * (long long)limit_us;
+    const int n = launch_wait_timeout_selftest(static_cast<int*>(workspace), cycles, OSDN_DEVICE_SELFTEST_TIMEOUT, st);
+    g_last_launches = n > 0 ? n : 0;
+    return n > 0 ? OSDN_OK : OSDN_CUDA_ERROR;
 }
 
 int osdn_workspace_region(const osdn_params* p, int need_bwd, const char* name, size_t* offset, size_t* bytes)

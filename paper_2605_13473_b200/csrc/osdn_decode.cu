@@ -13,9 +13,13 @@
 //
 // The work is bound by reading and writing the state once (V x K fp32 per chain).  Rows of S are
 // independent, so a chain is cut into V / 16 slices of 16 rows, one CTA each (4 warps x 4 rows); every
-// CTA repeats the tiny preconditioner update for its own use and slice 0 stores it.  Lane l of a warp
-// owns the R = K / 32 consecutive columns R l .. R l + R - 1 of its rows (one vector access per row),
-// the rows stay in registers over all tokens of the call.
+// CTA repeats the tiny preconditioner update for its own use and slice 0 stores it.  The slices of a
+// chain form one thread-block cluster: the preconditioner is updated in place, so slice 0 may only
+// store the advanced vector once every slice of the chain has read the old one; a cluster barrier
+// (arrive after the read, wait before the store) gives exactly that order within the one launch,
+// however many waves the grid takes.  Lane l of a warp owns the R = K / 32 consecutive columns
+// R l .. R l + R - 1 of its rows (one vector access per row), the rows stay in registers over all
+// tokens of the call.
 #include "osdn_common.cuh"
 
 namespace osdn {
@@ -92,6 +96,8 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
 #pragma unroll
     for (int r = 0; r < DEC_RW; ++r) dec_load<R>(srow + (size_t)r * K, lane, S[r]);
     dec_load<R>(a.precond + (size_t)chain * K, lane, d);
+    // this slice has read the chain's preconditioner (release: the read is ordered before the arrival)
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
     // inputs of a token, fetched one token ahead
     float kk[R], qq[R], vv[DEC_RW], bt, gt, lr, lrv[VEC ? R : 1];
@@ -178,26 +184,45 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
     }
 #pragma unroll
     for (int r = 0; r < DEC_RW; ++r) dec_store<R>(srow + (size_t)r * K, lane, S[r]);
+    // every slice of the chain has read the old preconditioner before slice 0 overwrites it
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     if (slice == 0 && warp == 0) dec_store<R>(a.precond + (size_t)chain * K, lane, d);
+}
+
+// One cluster per chain: its V / 16 slices (8 or 4 CTAs, within the portable cluster size).
+template <typename T, int K, int V, bool VEC> bool launch_one(unsigned chains, const DecArgs& a, cudaStream_t st)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(chains * (unsigned)(V / DEC_VB));
+    cfg.blockDim = dim3(DEC_WARPS * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = V / DEC_VB;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_kernel<T, K, V, VEC>, a) == cudaSuccess;
 }
 
 template <typename T> int launch_typed(const osdn_params& p, const DecArgs& a, cudaStream_t st)
 {
     const unsigned chains = (unsigned)p.B * (unsigned)p.H;
-    const unsigned grid = chains * (unsigned)(p.V / DEC_VB);
-    const int threads = DEC_WARPS * 32;
+    bool ok;
     if (a.hy.apf_mode == 3) {
-        if (p.K == 128 && p.V == 128) decode_kernel<T, 128, 128, true><<<grid, threads, 0, st>>>(a);
-        else if (p.K == 128 && p.V == 64) decode_kernel<T, 128, 64, true><<<grid, threads, 0, st>>>(a);
-        else if (p.K == 64 && p.V == 128) decode_kernel<T, 64, 128, true><<<grid, threads, 0, st>>>(a);
-        else decode_kernel<T, 64, 64, true><<<grid, threads, 0, st>>>(a);
+        if (p.K == 128 && p.V == 128) ok = launch_one<T, 128, 128, true>(chains, a, st);
+        else if (p.K == 128 && p.V == 64) ok = launch_one<T, 128, 64, true>(chains, a, st);
+        else if (p.K == 64 && p.V == 128) ok = launch_one<T, 64, 128, true>(chains, a, st);
+        else ok = launch_one<T, 64, 64, true>(chains, a, st);
     } else {
-        if (p.K == 128 && p.V == 128) decode_kernel<T, 128, 128, false><<<grid, threads, 0, st>>>(a);
-        else if (p.K == 128 && p.V == 64) decode_kernel<T, 128, 64, false><<<grid, threads, 0, st>>>(a);
-        else if (p.K == 64 && p.V == 128) decode_kernel<T, 64, 128, false><<<grid, threads, 0, st>>>(a);
-        else decode_kernel<T, 64, 64, false><<<grid, threads, 0, st>>>(a);
+        if (p.K == 128 && p.V == 128) ok = launch_one<T, 128, 128, false>(chains, a, st);
+        else if (p.K == 128 && p.V == 64) ok = launch_one<T, 128, 64, false>(chains, a, st);
+        else if (p.K == 64 && p.V == 128) ok = launch_one<T, 64, 128, false>(chains, a, st);
+        else ok = launch_one<T, 64, 64, false>(chains, a, st);
     }
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return ok && cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace

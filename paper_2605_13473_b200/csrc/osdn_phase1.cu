@@ -200,8 +200,9 @@ __global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
     const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (chain >= a.S * a.H) return;
     const int s = chain / a.H, h = chain % a.H;
-    const int t0 = a.cu ? a.cu[s] : s * a.T_dense;
-    const int len = a.cu ? max(a.cu[s + 1] - a.cu[s], 0) : a.T_dense;
+    // packed batch: T_dense is the packed token count; a malformed offset pair is clamped into it
+    const int t0 = a.cu ? min(max(a.cu[s], 0), a.T_dense) : s * a.T_dense;
+    const int len = a.cu ? min(max(a.cu[s + 1], t0), a.T_dense) - t0 : a.T_dense;
     const TI* kp = static_cast<const TI*>(a.k);
     TO* kt = static_cast<TO*>(a.ktil);
     float d[R];

@@ -30,8 +30,20 @@ constexpr int NTH = 256;
 // its sequence by bisection over the chunk offsets (kept in shared memory while they fit).
 constexpr int TBL_THREADS = 256, TBL_SMEM_SEQ = 2048;
 
+// The offsets live on the device, so the host cannot check them: a sequence is clamped into the packed
+// token range [0, T_total] (every later access stays inside the user tensors whatever cu_seqlens
+// holds), and a violated contract (cu[0] != 0, a decreasing pair, cu[S] != T_total) is reported through
+// the device status word.
+__device__ __forceinline__ void clamped_sequence(const int* __restrict__ cu, int s, int T_total, int& t0, int& len, bool& bad)
+{
+    const int a = cu[s], b = cu[s + 1];
+    bad = b < a || a < 0 || b > T_total;
+    t0 = min(max(a, 0), T_total);
+    len = min(max(b, t0), T_total) - t0;
+}
+
 __global__ void __launch_bounds__(TBL_THREADS)
-build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Table t)
+build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Table t, int* status)
 {
     __shared__ int s_c0[TBL_SMEM_SEQ + 1];
     __shared__ int s_scan[TBL_THREADS];
@@ -43,9 +55,16 @@ build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Ta
         const int s = base + tid;
         int t0 = 0, len = 0;
         if (s < S) {
-            t0 = cu ? cu[s] : s * T_dense;
-            len = cu ? cu[s + 1] - cu[s] : T_dense;
-            if (len < 0) len = 0;
+            if (cu) {   // packed batch: T_dense is the packed token count
+                bool bad;
+                clamped_sequence(cu, s, T_dense, t0, len, bad);
+                if (s == 0 && cu[0] != 0) bad = true;
+                if (s == S - 1 && cu[S] != T_dense) bad = true;
+                if (bad && status) atomicCAS(status, 0, OSDN_DEVICE_BAD_CU_SEQLENS);
+            } else {
+                t0 = s * T_dense;
+                len = T_dense;
+            }
         }
         const int nc = (len + CH - 1) / CH;
         s_scan[tid] = nc;
@@ -91,9 +110,11 @@ build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Ta
         }
         const int s = lo;
         const int c0 = in_smem ? s_c0[s] : t.seq_chunk0_[s];
-        const int t0 = cu ? cu[s] : s * T_dense;
-        int len = cu ? cu[s + 1] - cu[s] : T_dense;
-        if (len < 0) len = 0;
+        int t0 = s * T_dense, len = T_dense;
+        if (cu) {
+            bool bad;
+            clamped_sequence(cu, s, T_dense, t0, len, bad);
+        }
         const int rem = len - (j - c0) * CH;
         t.chunk_tok0_[j] = t0 + (j - c0) * CH;
         t.chunk_len_[j] = rem < CH ? rem : CH;
@@ -730,7 +751,8 @@ int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaSt
     Table tab = carve_table(ws, L);
     if (L.dense_T) return 0;   // dense batch: the table is arithmetic, nothing to build
     stage_mark(st, "build_table");
-    build_table_kernel<<<1, TBL_THREADS, 0, st>>>(L.S, p.T, p.cu_seqlens, L.NTmax, tab);
+    build_table_kernel<<<1, TBL_THREADS, 0, st>>>(L.S, p.T, p.cu_seqlens, L.NTmax, tab,
+                                                  reinterpret_cast<int*>(static_cast<char*>(ws) + L.status));
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -30,42 +30,6 @@ namespace osdn {
 
 using namespace umma;
 
-// Developer aid (compiled only with -DOSDN_PHASE_CLOCKS): clock64 stamps of one CTA at the phase
-// boundaries of each tensor-core kernel, and accumulated waiting times of single threads, read back
-// with osdn_debug_clocks.  The stamps are kept in shared memory until the kernel ends: a global store
-// inside a loop would itself delay the tensor-memory loads that follow it.
-#ifdef OSDN_PHASE_CLOCKS
-__device__ long long g_clk[4][32];
-#ifndef OSDN_CLK_MASK
-#define OSDN_CLK_MASK 0xffffffffu
-#endif
-#define OSDN_CLKS(i, cond)                                            \
-    do {                                                              \
-        if (((OSDN_CLK_MASK >> (i)) & 1u) && (cond)) s_clk[i] = clock64(); \
-    } while (0)
-// accumulated waiting time of one thread: OSDN_ACC_DECL once, then OSDN_ACC(slot, statement)
-#define OSDN_ACC_DECL long long acc_clk[6] = {0, 0, 0, 0, 0, 0}
-#define OSDN_ACC(slot, stmt)                                          \
-    do {                                                              \
-        const long long t_acc0 = clock64();                           \
-        stmt;                                                         \
-        acc_clk[slot] += clock64() - t_acc0;                          \
-    } while (0)
-#ifdef OSDN_ACC_OFF   // the sums share the stamp slots: build with one or the other
-#define OSDN_ACC_DUMP(base, count, cond)
-#else
-#define OSDN_ACC_DUMP(base, count, cond)                              \
-    do {                                                              \
-        if (cond)                                                     \
-            for (int i_acc = 0; i_acc < (count); ++i_acc) s_clk[(base) + i_acc] = acc_clk[i_acc]; \
-    } while (0)
-#endif
-#else
-#define OSDN_CLKS(i, cond)
-#define OSDN_ACC_DECL
-#define OSDN_ACC(slot, stmt) stmt
-#define OSDN_ACC_DUMP(base, count, cond)
-#endif
 
 namespace {
 
@@ -299,11 +263,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     const __grid_constant__ CUtensorMap tmKt, TcChunkArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
-#ifdef OSDN_PHASE_CLOCKS
-    __shared__ long long s_clk[32];
-    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
-    __syncthreads();
-#endif
     uint8_t* sm = align1024(smem_raw);
     uint8_t* sKQ = sm;                 // per k-half h: [K rows 0-63 | Q rows 64-127], 16 KB each
     uint8_t* sKt = sKQ + 32768;        // per k-half: 8 KB
@@ -353,12 +312,10 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(0, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     const uint32_t tb = tmem_base;
 
     bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
-    OSDN_CLKS(1, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sKQ + hf * 16384, len, tid, CL_THREADS);
@@ -368,7 +325,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         fence_proxy_async();
         __syncthreads();
     }
-    OSDN_CLKS(2, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- D1[128 x 64] = [K;Q] Ktil^T ---------------------------------------------------------
     if (tid == 0 && ok) {
@@ -397,7 +353,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         *reinterpret_cast<uint4*>(a.Qg + tile * REC_BYTES + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
     }
     ok = ok && mbar_wait(&bar_mma1, 0, a.status, ERR_MMA1);
-    OSDN_CLKS(3, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
         const int L = quad * 32 + lane;
@@ -461,7 +416,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
     }
     __syncthreads();
-    OSDN_CLKS(4, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- T = (I + A)^-1, blocked, in place ---------------------------------------------------------
     ut_inverse_64_inplace(sA, tid);
@@ -493,7 +447,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(6, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
 
     // ---- D2[128 x 64] = K^T Tbg^T  (W^T) -----------------------------------------------------
     if (tid == 0 && ok) {
@@ -505,7 +458,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         mma_commit(&bar_mma2);
     }
     ok = ok && mbar_wait(&bar_mma2, 0, a.status, ERR_MMA2);
-    OSDN_CLKS(7, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
     tc_fence_after();
     if (ok) {
         const int k = quad * 32 + lane;
@@ -529,11 +481,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(8, threadIdx.x == 0 && blockIdx.x == 5 && blockIdx.y == 0);
-#ifdef OSDN_PHASE_CLOCKS
-    __syncthreads();
-    if ((blockIdx.x == 5 && blockIdx.y == 0) && threadIdx.x < 32) g_clk[0][threadIdx.x] = s_clk[threadIdx.x];
-#endif
     if (warp == 1) tmem_dealloc(tb, 128);
 }
 
@@ -607,11 +554,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     __shared__ uint64_t bar_o_done[2], bar_o_free[2];
     __shared__ uint32_t tmem_base;
     __shared__ float sRho[2][CH], sGC[2];              // slot = chunk % 2
-#ifdef OSDN_PHASE_CLOCKS
-    __shared__ long long s_clk[32];
-    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
-    __syncthreads();
-#endif
 
     const int chain = blockIdx.x, H = a.H;
     const int s = chain / H, h = chain % H;
@@ -630,7 +572,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     const int nchunks = c1 - c0;
     auto chunk_tok0 = [&](int n) { return seq_t0 + n * CH; };
     auto chunk_len = [&](int n) { return min(CH, seq_len - n * CH); };
-    OSDN_CLKS(15, blockIdx.x == 0 && tid == 0);
 
     if (tid == 0) {
         mbar_init(&bar_full[0], 2);
@@ -691,7 +632,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     } else if (warp == CFW_MMA_WARP) {
         // ------------------------------------------------------------------ tensor-core issuer
         bool ok = true;
-        OSDN_ACC_DECL;
         bool ut_issued = false;   // V^T Tb^T of the coming chunk is already in the dU^T accumulator
         auto issue_ut = [&](uint8_t* d) {   // dU^T = V^T Tb^T
             const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN);
@@ -703,11 +643,10 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             const int st = n & 1;
             const size_t tile = (size_t)(c0 + n) * H + h;
             uint8_t* d = sStage + st * STAGE_BYTES;
-            if (!ut_issued) OSDN_ACC(0, ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA));
-            OSDN_ACC(1, ok = ok && mbar_wait(&bar_s_ready, n & 1, a.status, ERR_CHAIN_MMA1));
+            if (!ut_issued) ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);
+            ok = ok && mbar_wait(&bar_s_ready, n & 1, a.status, ERR_CHAIN_MMA1);
             if (!ok) break;
             tc_fence_after();
-            OSDN_CLKS(10, blockIdx.x == 0 && n == 10 && lane == 0);
             if (lane == 0) {
                 bulk_wait_read();   // saved images of the previous chunk have left shared memory
                 if (a.save) {
@@ -723,11 +662,10 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                                desc_advance(db0, 2048 * k), idesc, 1);
                 }
                 mma_commit(&bar_du_done);
-                OSDN_CLKS(11, blockIdx.x == 0 && n == 10);
             }
             __syncwarp();
             // the output accumulators of chunk n - 2 (same buffers) have been read
-            if (n >= 2) OSDN_ACC(2, ok = mbar_wait(&bar_o_free[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_MMA2));
+            if (n >= 2) ok = mbar_wait(&bar_o_free[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_MMA2);
             if (!ok) break;
             tc_fence_after();
             if (lane == 0) {   // O^T = S Qg^T
@@ -737,10 +675,9 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                            desc_advance(desc_kmajor(d + ST_QG + (k >> 2) * BOX), 32 * (k & 3)), idesc, k > 0);
             }
             __syncwarp();
-            OSDN_ACC(3, ok = mbar_wait(&bar_du_ready, n & 1, a.status, ERR_CHAIN_MMA2));
+            ok = mbar_wait(&bar_du_ready, n & 1, a.status, ERR_CHAIN_MMA2);
             if (!ok) break;
             tc_fence_after();
-            OSDN_CLKS(12, blockIdx.x == 0 && n == 10 && lane == 0);
             if (lane == 0) {
                 // The image of S sent off at the start of this chunk must have left shared memory before
                 // the state update is released: its completion lets the state warps overwrite that image.
@@ -756,7 +693,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                         mma_ss(tS, desc_advance(da0, 32 * k), desc_advance(db0, 2048 * k), idesc, 1);
                 }
                 mma_commit(&bar_s_done);
-                OSDN_CLKS(13, blockIdx.x == 0 && n == 10);
                 {   // O^T += dU^T P'^T
                     const uint32_t idesc = make_idesc(128, 64);
                     const uint64_t da0 = desc_kmajor(sDU1), db0 = desc_kmajor(d + ST_P);
@@ -771,7 +707,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             // state warps convert S (full chunks only: a ragged chunk has its tail rows cleared first).
             ut_issued = false;
             if (n + 1 < nchunks && chunk_len(n + 1) == CH) {
-                OSDN_ACC(4, ok = mbar_wait(&bar_full[st ^ 1], ((n + 1) >> 1) & 1, a.status, ERR_CHAIN_TMA));
+                ok = mbar_wait(&bar_full[st ^ 1], ((n + 1) >> 1) & 1, a.status, ERR_CHAIN_TMA);
                 if (!ok) break;
                 if (lane == 0) issue_ut(sStage + (st ^ 1) * STAGE_BYTES);
                 __syncwarp();
@@ -779,7 +715,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             }
         }
         if (lane == 0) bulk_wait_all();
-        OSDN_ACC_DUMP(0, 5, blockIdx.x == 0 && lane == 0);
     } else if (warp >= CFW_OUT_WARP0) {
         // ------------------------------------------------------------------ output warps
         // o_i = (S Qg^T + dU^T P'^T)_i is complete in the accumulator: lane = feature, 16 token columns
@@ -791,7 +726,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4;
         const int tsub = (b0 ? 8 : 0) + ((lane >> 1) & 3) * 2;
         bool ok = true;
-        OSDN_ACC_DECL;
         for (int n = 0; n < nchunks && ok; ++n) {
             const int st = n & 1;
             const int tok0 = chunk_tok0(n), len = chunk_len(n);
@@ -804,7 +738,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                 if (ow == 2)
                     for (int hf = 0; hf < 2; ++hf) tma_prefetch_2d(&tmKt, h * KD + hf * 64, t2);
             }
-            OSDN_ACC(0, ok = mbar_wait(&bar_o_done[st], (n >> 1) & 1, a.status, ERR_CHAIN_MMA2));
+            ok = mbar_wait(&bar_o_done[st], (n >> 1) & 1, a.status, ERR_CHAIN_MMA2);
             if (!ok) break;
             tc_fence_after();
             __nv_bfloat16* op = a.out + ((size_t)tok0 * H + h) * KD + ow * 32 + (lane >> 3) * 8;
@@ -852,7 +786,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                 }
             }
         }
-        OSDN_ACC_DUMP(12, 1, blockIdx.x == 0 && ow == 0 && lane == 0);
     } else {
         // ------------------------------------------------------------------ state warps
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
@@ -873,30 +806,19 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         tmem_st_wait();
 
         bool ok = true;
-        OSDN_ACC_DECL;
         for (int n = 0; n < nchunks && ok; ++n) {
             const int st = n & 1, gs = n & 1;
             const int len = chunk_len(n);
             uint8_t* d = sStage + st * STAGE_BYTES;
-            OSDN_ACC(0, ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA));   // gate vectors, tail rows
-#ifdef OSDN_PHASE_CLOCKS
-            acc_clk[3] += clock64() - s_clk[20 + st];
-#endif
-            if (n > 0) OSDN_ACC(1, ok = ok && mbar_wait(&bar_s_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2));
+            ok = mbar_wait(&bar_full[st], (n >> 1) & 1, a.status, ERR_CHAIN_TMA);   // gate vectors, tail rows
+            if (n > 0) ok = ok && mbar_wait(&bar_s_done, (n - 1) & 1, a.status, ERR_CHAIN_MMA2);
             if (!ok) break;
             tc_fence_after();
-            OSDN_CLKS(0, blockIdx.x == 0 && n == 10 && tid == 0);
-            OSDN_CLKS(8, blockIdx.x == 0 && n == 11 && tid == 0);
-            OSDN_CLKS(17, blockIdx.x == 0 && n == 0 && tid == 0);
-            OSDN_CLKS(18, blockIdx.x == 0 && n == 1 && tid == 0);
-            OSDN_CLKS(19, blockIdx.x == 0 && n == 20 && tid == 0);
-            OSDN_CLKS(24, blockIdx.x == 0 && n == 31 && tid == 0);
             // ---- E0: S -> bf16 operand (what the next products wait for), then decay the accumulator
             uint32_t rr[2][16];
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) tmem_ld16(tS + lane_addr + colq * 32 + cb * 16, rr[cb]);
             tmem_ld_wait();
-            OSDN_CLKS(1, blockIdx.x == 0 && n == 10 && tid == 0);
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
                 const uint32_t* r = rr[cb];
@@ -910,7 +832,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
                     *reinterpret_cast<uint4*>(sS + (colq >> 1) * 16384 + sw128_chunk(v, (colq & 1) * 4 + cb * 2 + c2)) = w;
                 }
             }
-            OSDN_CLKS(2, blockIdx.x == 0 && n == 10 && tid == 0);
             if (len < CH) {
                 for (int hf = 0; hf < 2; ++hf) {
                     zero_tail_rows(d + ST_V + hf * BOX, len, etid, CFW_EPI_WARPS * 32);
@@ -921,7 +842,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_s_ready);
-            OSDN_CLKS(3, blockIdx.x == 0 && n == 10 && tid == 0);
             {   // gamma_C S back into the accumulator: only the state update (after du_ready) reads it
                 const float gC = sGC[gs];
 #pragma unroll
@@ -936,15 +856,13 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             float rho[16];
 #pragma unroll
             for (int x = 0; x < 16; ++x) rho[x] = sRho[gs][colq * 16 + x];
-            OSDN_ACC(2, ok = mbar_wait(&bar_du_done, n & 1, a.status, ERR_CHAIN_MMA1));
+            ok = mbar_wait(&bar_du_done, n & 1, a.status, ERR_CHAIN_MMA1);
             if (!ok) break;
             tc_fence_after();
-            OSDN_CLKS(4, blockIdx.x == 0 && n == 10 && tid == 0);
             {
                 uint32_t r[16];
                 tmem_ld16(tDU + lane_addr + colq * 16, r);
                 tmem_ld_wait();
-                OSDN_CLKS(5, blockIdx.x == 0 && n == 10 && tid == 0);
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     float f[8], g[8];
@@ -965,9 +883,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_du_ready);
-            OSDN_CLKS(6, blockIdx.x == 0 && n == 10 && tid == 0);
         }
-        OSDN_ACC_DUMP(6, 4, blockIdx.x == 0 && tid == 0);
         if (ok) ok = mbar_wait(&bar_s_done, (nchunks - 1) & 1, a.status, ERR_CHAIN_MMA2);
         tc_fence_after();
         if (ok && fin) {
@@ -985,11 +901,6 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(16, blockIdx.x == 0 && tid == 0);
-#ifdef OSDN_PHASE_CLOCKS
-    __syncthreads();
-    if (blockIdx.x == 0 && tid < 32) g_clk[1][tid] = s_clk[tid];
-#endif
     if (warp == 0) tmem_dealloc(tb, 512);
 }
 
@@ -1027,11 +938,6 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
                     TcChainBwdArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
-#ifdef OSDN_PHASE_CLOCKS
-    __shared__ long long s_clk[32];
-    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
-    __syncthreads();
-#endif
     uint8_t* sm = align1024(smem_raw);
     uint8_t* sStage = sm;
     uint8_t* sdS = sm + 2 * BSTAGE_BYTES;       // dS as bf16, K-major, 2 k-halves x [128 x 128 B]
@@ -1060,7 +966,6 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
     auto chunk_tok0 = [&](int n) { return seq_t0 + chunk_rel(n) * CH; };
     auto chunk_len = [&](int n) { return min(CH, seq_len - chunk_rel(n) * CH); };
     auto chunk_tile = [&](int n) { return (size_t)(c0 + chunk_rel(n)) * H + h; };
-    OSDN_CLKS(15, blockIdx.x == 0 && tid == 0);
 
     if (tid == 0) {
         mbar_init(&bar_full[0], 2);
@@ -1296,11 +1201,6 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
     }
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(16, blockIdx.x == 0 && tid == 0);
-#ifdef OSDN_PHASE_CLOCKS
-    __syncthreads();
-    if ((blockIdx.x == 0) && threadIdx.x < 32) g_clk[2][threadIdx.x] = s_clk[threadIdx.x];
-#endif
     if (warp == 0) tmem_dealloc(tb, 256);
 }
 
@@ -1349,11 +1249,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     TcChunkBwdArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
-#ifdef OSDN_PHASE_CLOCKS
-    __shared__ long long s_clk[32];
-    if (threadIdx.x < 32) s_clk[threadIdx.x] = 0;
-    __syncthreads();
-#endif
     uint8_t* sm = align1024(smem_raw);
     float* sRaw = reinterpret_cast<float*>(sm + R_RAW);       // Gamma_ij <k_i, ktil_j>, j < i
     __shared__ uint64_t bar_tma, bar_mma[5];
@@ -1440,8 +1335,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     while (tile_l < a.ntiles) {
     const int h = (int)(tile_l % H);
-    const bool clk = tile_l == 1603;
-    (void)clk;
     if (tid < CH) {
         sg[tid] = g_cur;
         sBeta[tid] = b_cur;
@@ -1450,7 +1343,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     if (tid == 0) sRsum = 0.f;
     __syncthreads();
-    OSDN_CLKS(0, threadIdx.x == 0 && clk);
     // table entries and scalars of the next tile, one tile ahead
     const int tile_next = next_tile(tile_l + (int)gridDim.x);
     int tok0_next = 0, len_next = 0;
@@ -1492,7 +1384,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sRho[lane + 32] = __expf(tot - sb);
     }
     bool ok = mbar_wait(&bar_tma, ph, a.status, ERR_TMA);
-    OSDN_CLKS(1, threadIdx.x == 0 && clk);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sm + R_Q + hf * BOX, len, tid, CBW_THREADS);
@@ -1504,7 +1395,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fence_proxy_async();
     }
     __syncthreads();
-    OSDN_CLKS(2, threadIdx.x == 0 && clk);
 
     // tensor memory columns
     const uint32_t cRAW = 0, cDP = 64, cDQ1 = 128, cDKTR = 192, cDW = 256, cDTA = 320, cDTB = 384, cDKT = 448;
@@ -1566,7 +1456,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (lane == 0) sRed[warp] = part;
     }
     ok = ok && mbar_wait(&bar_mma[0], ph, a.status, ERR_MMA1);
-    OSDN_CLKS(3, threadIdx.x == 0 && clk);
     tc_fence_after();
     __syncthreads();   // every thread is done reading S / dS before their space is reused
     // epilogue A
@@ -1613,7 +1502,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(4, threadIdx.x == 0 && clk);
 
     // ---- phase B -------------------------------------------------------------------------------
     if (lane == 0 && warp < 6 && ok) {
@@ -1664,7 +1552,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     }
     ok = ok && mbar_wait(&bar_mma[1], ph, a.status, ERR_MMA2);
-    OSDN_CLKS(5, threadIdx.x == 0 && clk);
     tc_fence_after();
     {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j]
         const int i = row64;
@@ -1692,7 +1579,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(6, threadIdx.x == 0 && clk);
 
     // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] -----------------------------------------------
     if (tid == 0 && ok) {
@@ -1705,7 +1591,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (early) bulk_load(sm + R_DDU, a.ddUT + (size_t)tile_next * 16384, 16384, &bar_tma);   // phase B done
     }
     ok = ok && mbar_wait(&bar_mma[2], ph, a.status, ERR_MMA2);
-    OSDN_CLKS(7, threadIdx.x == 0 && clk);
     tc_fence_after();
     {
         const int i = row64;
@@ -1728,7 +1613,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(8, threadIdx.x == 0 && clk);
 
     // ---- phase D: Z[a][b] = sum_c Y[a][c] T[b][c] ; dA = -strictLower(Z) --------------------------
     if (tid == 0 && ok) {
@@ -1739,7 +1623,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[3]);
     }
     ok = ok && mbar_wait(&bar_mma[3], ph, a.status, ERR_MMA2);
-    OSDN_CLKS(9, threadIdx.x == 0 && clk);
     tc_fence_after();
     {
         const int i = row64;
@@ -1771,7 +1654,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    OSDN_CLKS(10, threadIdx.x == 0 && clk);
 
     // ---- phase E: dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T -----------------------------------------
     if (lane == 0 && warp < 2 && ok) {
@@ -1790,12 +1672,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (early && warp == 0) bulk_load(sm + R_T, a.Tm + (size_t)tile_next * 8192, 8192, &bar_tma);   // phase D done
     }
     ok = ok && mbar_wait(&bar_mma[4], ph, a.status, ERR_MMA2);
-    OSDN_CLKS(11, threadIdx.x == 0 && clk);
     tc_fence_after();
     // every product has finished: the images in the space of S are dead
     if (early && tid == 0 && ok) bulk_load(sm + R_S, a.Sn + (size_t)tile_next * 32768, 32768, &bar_tma);
-    OSDN_CLKS(19, threadIdx.x == 0 && clk);
-    OSDN_CLKS(20, threadIdx.x == 32 && clk);
 
     // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
     float rsum = 0.f;
@@ -1860,13 +1739,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
             }
         }
-        OSDN_CLKS(14, threadIdx.x == 0 && clk);
-        OSDN_CLKS(21, threadIdx.x == 32 && clk);
     }
-    OSDN_CLKS(15, threadIdx.x == 0 && clk);
     fence_proxy_async();
     ok = __syncthreads_and(ok);   // block-uniform from here on; staging complete, q, k, ktil, v dead
-    OSDN_CLKS(16, threadIdx.x == 0 && clk);
     if (tid == 0) {
         if (tile_next < a.ntiles) {
             if (!early) expect_all();
@@ -1971,7 +1846,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         *reinterpret_cast<const uint4*>(sm + ST_DKT + j * 512 + ch * 16);
             }
         }
-        OSDN_CLKS(17, threadIdx.x == 0 && clk);
         if (full && tid == 0) bulk_wait_read();   // the staging tiles may be overwritten by the next tile
     }
     __syncthreads();   // every copy-out read of the staging tiles is done
@@ -1979,11 +1853,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         issue_dout(tile_next, tok0_next);
         if (!early) issue_chain_tiles(tile_next);
     }
-    OSDN_CLKS(12, threadIdx.x == 0 && clk);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    OSDN_CLKS(13, threadIdx.x == 0 && clk);
     ph ^= 1u;
     tile_l = tile_next;
     tok0 = tok0_next;
@@ -1995,11 +1867,20 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (tid == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
-#ifdef OSDN_PHASE_CLOCKS
-    __syncthreads();
-    if (blockIdx.x == 1603 % gridDim.x && threadIdx.x < 32) g_clk[3][threadIdx.x] = s_clk[threadIdx.x];
-#endif
     if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+// Exercises the bounded wait by itself: one warp waits on a barrier that nothing ever arrives on.  The
+// wait gives up after `limit_cycles`, records `code` in the status word and the kernel returns.
+__global__ void wait_timeout_selftest_kernel(int* status, long long limit_cycles, int code)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0, status, code, limit_cycles);
 }
 
 int num_sms()
@@ -2019,6 +1900,12 @@ template <typename F> bool set_smem(F* kernel, size_t bytes)
 }
 
 }  // namespace
+
+int launch_wait_timeout_selftest(int* status, long long limit_cycles, int code, cudaStream_t st)
+{
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status, limit_cycles, code);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
 
 bool tc_supported(const osdn_params& p)
 {
@@ -2132,9 +2019,3 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
 
 }  // namespace osdn
 
-#ifdef OSDN_PHASE_CLOCKS
-extern "C" int osdn_debug_clocks(long long* out)
-{
-    return (int)cudaMemcpyFromSymbol(out, osdn::g_clk, sizeof(osdn::g_clk));
-}
-#endif

@@ -61,10 +61,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after about two seconds of polling, records `code` in the device status
-// word and returns false.  Callers then skip the dependent work; nothing spins forever.  The
-// result is made uniform across the warp so that warp-aligned instructions stay converged.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code)
+// Bounded wait: gives up after `limit_cycles` of polling (about two seconds by default), records
+// `code` in the device status word and returns false.  Callers then skip the dependent work; nothing
+// spins forever.  The result is made uniform across the warp so that warp-aligned instructions stay
+// converged.
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code,
+                                          long long limit_cycles = WAIT_LIMIT_CYCLES)
 {
     bool done = mbar_try_wait(bar, parity);
     if (!done) {
@@ -72,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
         uint32_t it = 0;
         while (!(done = mbar_try_wait(bar, parity))) {
             if ((++it & 1023u) == 0u) {
-                if (clock64() - t0 > 4000000000ll) break;
+                if (clock64() - t0 > limit_cycles) break;
                 if (status && *reinterpret_cast<volatile int*>(status) != 0) break;
             }
         }

@@ -8,30 +8,95 @@ import torch
 
 import oracle
 
-# Tolerances of the parity gate: per tensor, max|x - y| / max|y| (the maximum absolute error after
-# the reference tensor is scaled to unit magnitude)
-#   fp32 I/O : <= 1e-4
-#   bf16 I/O : <= 2e-2   (bf16 operands, fp32 accumulation)
-# The report also records max|x - y| / rms(y), which is stricter by the tensor's crest factor.
+# Three measures per tensor, all of them gated (x = CUDA path, y = fp64 oracle):
+#   max_norm  max|x - y| / max|y|      fp32 I/O <= 1e-4, bf16 I/O <= 2e-2
+#   l2_rel    |x - y|_2 / |y|_2        bf16 I/O <= 7e-3: the bound the paper reports between its own
+#                                      bf16 chunk path and its token recurrence (appendix "Numerical
+#                                      equivalence with the chunk forward"); fp32 I/O <= 1e-4
+#   rms_norm  max|x - y| / rms(y)      bf16 I/O <= 2e-2 on results the library stores in fp32.  For a
+#             result stored in bf16 the reference is the oracle value rounded to bf16 and one unit in
+#             the last place of that value is allowed on top: two correctly rounded programs may
+#             land on neighbouring bf16 numbers, and at the magnitude of the largest elements (eight
+#             times the rms here) one such step alone is 3e-2 rms.
+# Where the tensor-core path is known to exceed the rms_norm bound on an fp32-stored result, the
+# excess is a recorded shortfall, not a reading: RMS_SHORTFALL lists the tensor, the ceiling that is
+# asserted instead, and the report carries the measured figure.
 TOL = {"fp32": 1e-4, "bf16": 2e-2}
+L2_TOL = {"fp32": 1e-4, "bf16": 7e-3}
+RMS_TOL = {"fp32": None, "bf16": 2e-2}   # fp32 I/O: recorded, not gated (its bound is max_norm)
+BF16_STORED = ("out", "dq", "dk", "dv")
+# tensor-core path (bf16 operand images of the state, the UT inverse, the pseudo keys and the chunk
+# updates, i.e. more than one bf16 rounding per contraction): largest max|x - y| / rms(y) measured over
+# the parity suite and the full-size configurations, plus a margin of a quarter; asserted so that the
+# figures cannot grow unnoticed.  The relative Euclidean error of the same tensors is 2e-3 .. 4.5e-3.
+RMS_SHORTFALL = {"out": 5e-2, "dq": 8e-2, "dk": 7.5e-2, "dv": 6e-2, "final_state": 6e-2, "dinit_state": 3.5e-2,
+                 "dbeta": 3.5e-2, "dgate": 3.7e-2, "dlog_ret": 1.6e-1, "dprecond_in": 2.8e-2}
 
 FWD_KEYS = ("out", "final_state", "precond_out")
 BWD_KEYS = ("dq", "dk", "dv", "dbeta", "dgate", "dlog_ret", "dinit_state", "dprecond_in")
+NEAR_TIE_CEILING = 2e-3   # largest admissible fraction of projection decisions taken over from the CUDA path
 
 
 def err(x, y, io_dtype=None, norm="max"):
-    """max|x - y| normalised by max|y| (default) or rms(y); absolute if the reference is all zero."""
+    """max|x - y| normalised by max|y| (default) or rms(y), or the relative Euclidean error
+    (norm="l2"); absolute if the reference is all zero."""
     x = np.asarray(x, dtype=np.float64)
     y = np.asarray(y, dtype=np.float64)
     if y.size == 0:
         return 0.0
     if not np.isfinite(x).all():
         return float("inf")
-    diff = np.abs(x - y).max()
-    den = np.abs(y).max() if norm == "max" else np.sqrt(np.mean(y * y))
+    if norm == "l2":
+        num, den = np.sqrt(np.sum((x - y) ** 2)), np.sqrt(np.sum(y * y))
+    else:
+        num = np.abs(x - y).max()
+        den = np.abs(y).max() if norm == "max" else np.sqrt(np.mean(y * y))
     if den < 1e-30:
-        return float(diff)
-    return float(diff / den)
+        return float(num)
+    return float(num / den)
+
+
+def _bf16_round(y):
+    return torch.as_tensor(np.asarray(y, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def _bf16_ulp(y):
+    """Spacing of bf16 numbers at |y| (8 significant bits)."""
+    a = np.maximum(np.abs(np.asarray(y, dtype=np.float64)), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(a)) - 7)
+
+
+def err_rms_stored_bf16(x, y):
+    """max over elements of (|x - bf16(y)| - ulp(y))_+ / rms(y): the rms_norm measure for a result that
+    is stored in bf16."""
+    x = np.asarray(x, dtype=np.float64)
+    y = np.asarray(y, dtype=np.float64)
+    if y.size == 0:
+        return 0.0
+    if not np.isfinite(x).all():
+        return float("inf")
+    yb = _bf16_round(y)
+    excess = np.maximum(np.abs(x - yb) - _bf16_ulp(yb), 0.0).max()
+    den = np.sqrt(np.mean(y * y))
+    return float(excess if den < 1e-30 else excess / den)
+
+
+def write_report(report, env="OSDN_PARITY_REPORT", suffix=""):
+    """Writes a report dict as JSON to the file the environment variable names (if it is set)."""
+    import json
+    import os
+    path = os.environ.get(env)
+    if not path:
+        return
+    if suffix:
+        root, ext = os.path.splitext(path)
+        path = root + suffix + ext
+    try:
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+        with open(path, "w") as f:
+            json.dump(report, f, indent=1)
+    except OSError:
+        pass
 
 
 def subset(inp, seqs, heads):
@@ -79,11 +144,14 @@ def oracle_all(inp, bwd: bool, gpu_masks=None):
     """Oracle forward (and backward).  The gradient is discontinuous where a pre-projection value of
     the preconditioner touches a face of the box.  Where the oracle's fp64 value is within TIE of a
     face the decision is not unique at fp32 resolution: there (and only there) the oracle's reverse
-    sweep takes the decision the CUDA path took (`gpu_masks`); everywhere else the two must agree."""
+    sweep takes the decision the CUDA path took (`gpu_masks`); everywhere else the two must agree.
+    How many decisions were taken over is returned (`near_ties`, `near_tie_fraction`) and bounded by
+    NEAR_TIE_CEILING.  With gpu_masks=None nothing is taken over."""
     if not bwd:
         return oracle.fwd_inputs(inp)
     ref = oracle.fwd_inputs(inp, want_margin=True)
     override = None
+    ref["near_ties"], ref["near_tie_fraction"] = 0, 0.0
     if gpu_masks is not None and inp.hyper.clamp:
         gm = np.asarray(gpu_masks, dtype=np.uint8)
         near = ref["margin"] <= TIE
@@ -91,20 +159,45 @@ def oracle_all(inp, bwd: bool, gpu_masks=None):
         assert not disagree.any(), f"{int(disagree.sum())} projection decisions differ away from any tie"
         override = np.where(near, gm, 255).astype(np.uint8)
         ref["near_ties"] = int(near.sum())
+        ref["near_tie_fraction"] = float(near.mean()) if near.size else 0.0
+        assert ref["near_tie_fraction"] <= NEAR_TIE_CEILING, (
+            f"{ref['near_ties']} of {near.size} projection decisions lie within {TIE} of a face")
     ref.update(oracle.bwd_inputs(inp, mask_override=override))
     return ref
 
 
-def compare(got, ref, io_dtype, keys, label="", tol=None, report=None):
+def compare(got, ref, io_dtype, keys, label="", tol=None, report=None, tensor_core=False):
+    """Gates every tensor on the three measures of the header.  `tensor_core`: the case ran on the
+    tcgen05 kernels (RMS_SHORTFALL applies)."""
     tol = TOL[io_dtype] if tol is None else tol
-    worst = {}
+    worst, l2, rms = {}, {}, {}
     for k in keys:
         if k not in ref or k not in got:
             continue
         worst[k] = err(got[k], ref[k], io_dtype)
+        l2[k] = err(got[k], ref[k], io_dtype, "l2")
+        if io_dtype == "bf16" and k in BF16_STORED:
+            rms[k] = err_rms_stored_bf16(got[k], ref[k])
+        else:
+            rms[k] = err(got[k], ref[k], io_dtype, "rms")
     if report is not None:
         report[label] = dict(worst)
-        report[label + "/rms_normalised"] = {k: err(got[k], ref[k], io_dtype, "rms") for k in worst}
+        report[label + "/l2_relative"] = dict(l2)
+        report[label + "/rms_normalised"] = dict(rms)
+        if "near_ties" in ref:
+            report[label + "/near_ties"] = dict(count=ref["near_ties"], fraction=ref["near_tie_fraction"])
     bad = {k: e for k, e in worst.items() if not (e <= tol)}
-    assert not bad, f"{label}: parity failed {bad} (tol {tol}); all: {worst}"
+    assert not bad, f"{label}: parity failed {bad} (max_norm tol {tol}); all: {worst}"
+    bad = {k: e for k, e in l2.items() if not (e <= L2_TOL[io_dtype])}
+    assert not bad, f"{label}: parity failed {bad} (l2_rel tol {L2_TOL[io_dtype]}); all: {l2}"
+    bad = {}
+    for k, e in rms.items():
+        lim = RMS_TOL[io_dtype]
+        if lim is None:
+            continue
+        if tensor_core and k in RMS_SHORTFALL:
+            lim = max(lim, RMS_SHORTFALL[k])
+        if not (e <= lim):
+            bad[k] = e
+    assert not bad, f"{label}: parity failed {bad} (rms_norm); all: {rms}"
     return worst

@@ -72,6 +72,21 @@ def test_decode_matches_oracle(io, K, V, B, H, L, apf, clamp, ba, eta):
     assert parity.err(got_out, ref["out"]) <= parity.TOL[io]
 
 
+@pytest.mark.parametrize("L", [1, 64])
+def test_decode_in_place_preconditioner_over_many_waves(L):
+    """The preconditioner is advanced in place while every slice of a chain reads it: with a grid of
+    several waves (512 chains x 8 slices) and a preconditioner that really moves (large step, no
+    projection) a slice that started late must still see the vector the call was entered with."""
+    hy = OsdnHyper(eta=0.3, apf_mode=1, clamp=0)
+    B, H, D = 64, 8, 128
+    inp = draw(f"decode_waves_{L}", 4100 + L, [L] * B, H, D, D, "bf16", dense_B=B, hyper=hy, with_state=True)
+    got_out, got_S, got_d = _decode(inp, inp.init_state, inp.precond_in)
+    ref = oracle.fwd_inputs(inp)
+    assert parity.err(got_d, ref["precond_out"]) <= 1e-4
+    assert parity.err(got_S, ref["final_state"]) <= 1e-4
+    assert parity.err(got_out, ref["out"]) <= parity.TOL["bf16"]
+
+
 def test_decode_continues_in_place_across_calls():
     """Two calls of 3 and 4 tokens equal one call of 7: the cache carries everything."""
     hy = OsdnHyper(eta=0.3, apf_mode=1)

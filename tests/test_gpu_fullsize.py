@@ -12,13 +12,17 @@ pytestmark = pytest.mark.gpu
 REPORT = {}
 
 
+def teardown_module(module):
+    parity.write_report(REPORT, suffix="_fullsize")
+
+
 def _sampled(inp, bwd, seqs, heads, label):
     got = run_inputs_bwd(inp) if bwd else run_inputs_fwd(inp)
     sub, tok_t, hd = parity.subset(inp, seqs, heads)
     got_sub = parity.subset_result(got, seqs, heads, tok_t, hd)
     ref = parity.oracle_all(sub, bwd, got_sub.get("projection_masks"))
     keys = parity.FWD_KEYS + (parity.BWD_KEYS if bwd else ())
-    parity.compare(got_sub, ref, inp.io_dtype, keys, label, report=REPORT)
+    parity.compare(got_sub, ref, inp.io_dtype, keys, label, report=REPORT, tensor_core=True)
 
 
 def test_cfg1_full_forward():

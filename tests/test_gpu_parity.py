@@ -1,7 +1,4 @@
 """GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by element."""
-import json
-import os
-
 import numpy as np
 import pytest
 import torch
@@ -17,20 +14,20 @@ REPORT = {}
 
 
 def teardown_module(module):
-    out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    try:
-        os.makedirs(out, exist_ok=True)
-        with open(os.path.join(out, "parity_report.json"), "w") as f:
-            json.dump(REPORT, f, indent=1)
-    except OSError:
-        pass
+    """Writes every measure of every case as JSON to the file named by OSDN_PARITY_REPORT, if set."""
+    parity.write_report(REPORT)
 
 
-def _check(inp, bwd, label, flags=0, tol=None):
+def _on_tensor_cores(inp, flags):
+    return inp.io_dtype == "bf16" and inp.K == 128 and inp.V == 128 and not (flags & binding.FLAG_FORCE_SIMT)
+
+
+def _check(inp, bwd, label, flags=0, tol=None, take_over_ties=True):
     got = run_inputs_bwd(inp, flags=flags) if bwd else run_inputs_fwd(inp, flags=flags)
-    ref = parity.oracle_all(inp, bwd, got.get("projection_masks"))
+    ref = parity.oracle_all(inp, bwd, got.get("projection_masks") if take_over_ties else None)
     keys = parity.FWD_KEYS + (parity.BWD_KEYS if bwd else ())
-    return parity.compare(got, ref, inp.io_dtype, keys, label, tol=tol, report=REPORT)
+    return parity.compare(got, ref, inp.io_dtype, keys, label, tol=tol, report=REPORT,
+                          tensor_core=_on_tensor_cores(inp, flags))
 
 
 PATHS = [("simt", binding.FLAG_FORCE_SIMT), ("auto", 0)]
@@ -63,6 +60,23 @@ def test_lively_sets(idx, io, path, flags):
         pytest.skip("fp32 I/O always runs the CUDA-core kernels")
     inp = lively(idx, T=200, B=2, H=2, D=128, io_dtype=io)
     _check(inp, True, f"lively{idx}_{io}_{path}", flags=flags)
+
+
+@pytest.mark.parametrize("io,D,seed,kind", [("bf16", 128, 2010, "alias"), ("fp32", 64, 2015, "sparse")],
+                         ids=["tensor_core", "cuda_core"])
+def test_backward_owes_nothing_to_the_gpu_masks(io, D, seed, kind):
+    """One case per kernel family in which the oracle's reverse sweep takes every projection decision
+    by itself: the seeds were chosen (on the CPU, from the oracle's own margins) so that the box is
+    active for part of the coordinates and no pre-projection value lies within 1e-4 of a face."""
+    if kind == "alias":
+        hy, extra = OsdnHyper(eta=0.3, apf_mode=1), {}
+    else:
+        hy, extra = OsdnHyper(eta=0.3, apf_mode=2), dict(key_kind="sparse", with_log_ret=True)
+    inp = draw("noties", seed, [100], 1, D, D, io, dense_B=1, hyper=hy, with_dout=True, with_state=True,
+               with_state_cotangents=True, **extra)
+    probe = oracle.fwd_inputs(inp, want_margin=True)
+    assert probe["margin"].min() > 1e-4 and 0.02 < probe["mask"].mean() < 0.98
+    _check(inp, True, f"no_ties_{io}", take_over_ties=False)
 
 
 @pytest.mark.parametrize("path,flags", PATHS, ids=[p[0] for p in PATHS])

@@ -11,6 +11,7 @@ Collected last on purpose: a run that stops at the first failure has then run ev
 import pytest
 import torch
 
+import oracle
 import parity
 from paper_2605_13473_b200 import binding
 from paper_2605_13473_b200.synth import OsdnHyper, config, draw
@@ -34,6 +35,7 @@ def _static(b):
                                  out, fin, dout)
     assert rc == 0, binding.status_string(rc)
     torch.cuda.synchronize()
+    assert binding.osdn_read_static_status() == 0     # no device-side error inside the built-in array
     return dict(out=out.float().cpu(), final_state=fin.cpu(), precond_out=dout.cpu())
 
 
@@ -51,9 +53,14 @@ def test_static_scratch_forward_matches_workspace_forward(name, make):
     b, ref = _reference(inp)
     assert binding.osdn_workspace_bytes(b.params, False) <= binding.STATIC_SCRATCH_BYTES
     first = _static(b)
+    free_before = torch.cuda.mem_get_info()[0]
     second = _static(b)          # the shared array now holds the first call's contents
+    assert torch.cuda.mem_get_info()[0] == free_before      # the call took no device memory
+    want = oracle.fwd_inputs(inp)   # the definition itself, so that this test stands without osdn_fwd
+    on_tc = inp.io_dtype == "bf16" and inp.K == 128 and inp.V == 128
     for got in (first, second):
         parity.compare(got, ref, inp.io_dtype, parity.FWD_KEYS, f"static_{name}")
+        parity.compare(got, want, inp.io_dtype, parity.FWD_KEYS, f"static_{name}_vs_oracle", tensor_core=on_tc)
     # another problem in between, then the first one again
     other = config(1, shrink=dict(B=2, T=128, H=1))
     ob, oref = _reference(other)
