@@ -1206,13 +1206,16 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
 
 // ---------------------------------------------------------------------------------------------
 // chunk-local backward.  Feature-major ("transposed") accumulators: lane = feature, column = token.
-//   phase A : rawkk = K Ktil^T ; dP' = dO dU^T ; dQ1^T = S^T dO^T ; dKtr^T = dS^T dU ; dW^T = -S^T ddU
+//   phase A : dP' = dO dU^T ; dQ1^T = S^T dO^T ; dKtr^T = dS^T dU ; dW^T = -S^T ddU
+//             (reads only what the chain kernels and the caller wrote: issued a tile ahead)
 //   phase B : dT = (dW K^T) beta gamma + (ddU V^T) beta ; dKb^T = dW^T T ; dVb^T = ddU^T T ;
 //             dq2^T = Ktil^T M1^T ; dktil^T = Q^T M1            (M1 = scale Gamma (.) lower(dP'))
-//   phase C : Y = T^T dT        phase D : Z = Y T^T, dA = -strictLower(Z), M2 = dA beta_i Gamma_ij
+//             dbeta_j += sum_i T_ij (gamma_j dW K^T + ddU V^T)_ij
+//   phase C : Y = T^T dT ; rawkk = K Ktil^T
+//   phase D : Z = Y T^T, dA = -strictLower(Z), M2 = dA beta_i Gamma_ij, dbeta_i += sum_j dA_ij Gamma_ij rawkk_ij
 //   phase E : dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T
 //   final   : dq = scale gamma dQ1 + dq2 ; dktil += rho dKtr ; dk_read = dkr + beta gamma dKb ;
-//             dv = beta dVb ; dbeta, dgate from the products of the gradients with their inputs
+//             dv = beta dVb ; dgate from the products of the gradients with their inputs
 // ---------------------------------------------------------------------------------------------
 struct TcChunkBwdArgs {
     int H, ntiles;
@@ -1230,16 +1233,20 @@ constexpr int CBW_THREADS = 512;   // 16 warps = 4 lane quadrants x 4 column gro
 constexpr uint32_t R_Q = 0, R_K = 16384, R_KT = 32768, R_V = 49152, R_DO = 65536, R_DU = 81920, R_DDU = 98304,
                    R_T = 114688, R_S = 122880, R_DS = 155648, R_RAW = 188416;
 constexpr uint32_t R_DWT = R_DO;                 // dW^T image replaces dO after phase A
-constexpr uint32_t R_M1 = R_S, R_M2 = R_S + 8192, R_DT = R_S + 16384, R_Y = R_S + 24576;
-// Output staging after the last product ([token][feature] tiles over dead space): dq and dv over the
-// fp32 scratch (dead after phase D), dk over dO / dW^T; the fp32 copies of dk_read and dL/dktil, needed
-// only when some token's preconditioner step was really taken, over T, S and dS.  When every token of a
-// full chunk was skipped, the space of dU, ddU, T, S and dS is therefore free during the final epilogue
-// and the next tile's copies of them start there.
-constexpr uint32_t ST_DQ = R_RAW, ST_DV = R_RAW + 16384, ST_DK = R_DO, ST_DKR = 114688, ST_DKT = 147456;
+// M1, dT, Y and M2 are live one after the other (each is written once the product that read its
+// predecessor has finished), so they share one 8 KB image behind the fp32 scratch.
+constexpr uint32_t R_IMG = R_RAW + 24576;
+// Output staging ([token][feature] tiles over dead space): dq over V (dead after phase B; dq is complete
+// then and is formed while phase C runs), dk and dv after the last product over the fp32 scratch (dead
+// after phase D) and the operand image; the fp32 copies of dk_read and dL/dktil, needed only when some
+// token's preconditioner step was really taken, over T, S and dS.  When every token of a full chunk was
+// skipped, the space of dO, dU, ddU, T, S and dS is therefore never reused inside a tile and the next
+// tile's copies of them start as soon as the last product reading the current ones has finished.
+constexpr uint32_t ST_DQ = R_V, ST_DV = R_RAW + 16384, ST_DK = R_RAW, ST_DKR = 114688, ST_DKT = 147456;
+constexpr int CBW_STORE_TID = 256;   // the thread that sends the output tiles off (and owns their bulk group)
 static_assert(ST_DKT + 32768 <= R_RAW, "fp32 staging tiles must fit below the fp32 scratch");
 constexpr size_t CBW_SMEM = R_RAW + 32768 + 1024;
-static_assert(CH * LC * 4 <= 32768, "fp32 scratch must fit in its region");
+static_assert(CH * LC * 4 <= 24576, "fp32 scratch must end before the shared operand image");
 
 __global__ void __launch_bounds__(CBW_THREADS, 1)
 tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -1250,10 +1257,16 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* sm = align1024(smem_raw);
-    float* sRaw = reinterpret_cast<float*>(sm + R_RAW);       // Gamma_ij <k_i, ktil_j>, j < i
-    __shared__ uint64_t bar_tma, bar_mma[5];
+    // bar_ct: dO and the tiles written by the chain kernels (everything phase A reads);
+    // bar_tok: q, k, ktil, v
+    __shared__ uint64_t bar_ct, bar_tok, bar_mma[5];
     __shared__ uint32_t tmem_base;
-    __shared__ __align__(16) float sG[CH], sBeta[CH], sg[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
+    __shared__ __align__(16) float sG[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
+    // per-token gate and beta and the two skip words of a tile, copied asynchronously one tile ahead
+    // (two buffers; values fetched into registers that early would be spilled, and the spill would wait
+    // for the load)
+    __shared__ __align__(16) float sScal[2][2][CH];
+    __shared__ unsigned sSkipW[2][2];
     __shared__ float sRsum;
     __shared__ __align__(16) float sFirstKt[KD];
 
@@ -1261,14 +1274,18 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, colq = warp >> 2;   // lane quadrant, column group (16 columns each)
     const int f = quad * 32 + lane;                 // feature (k or v) owned in 128-lane accumulators
-    const int row64 = quad * 16 + (lane & 15);      // token row owned in 64-row accumulators (lanes 0-15)
-    const bool row_active = lane < 16;
+    // 64-row accumulators keep their rows in lanes 0-15 of each quadrant: thread t reads row
+    // quad * 16 + (t & 15), eight columns (threads 16-31 the second eight of the warp's sixteen)
+    const int row64 = quad * 16 + (lane & 15);
+    const int jb = colq * 16 + (lane >> 4) * 8;     // first of the eight columns
+    const uint32_t addr64 = ((uint32_t)(quad * 32) << 16) + colq * 16;
 
     if (tid == 0) {
-        mbar_init(&bar_tma, 1);
+        mbar_init(&bar_ct, 1);
+        mbar_init(&bar_tok, 1);
         // the independent products of a phase are issued by different warps (the issue rate of one
         // thread, not the tensor pipe, limits these small shapes); each issuer commits for itself
-        const uint32_t issuers[5] = {5, 6, 1, 1, 2};
+        const uint32_t issuers[5] = {4, 6, 2, 1, 2};
         for (int i = 0; i < 5; ++i) mbar_init(&bar_mma[i], issuers[i]);
         fence_mbar_init();
     }
@@ -1279,94 +1296,166 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t tb = tmem_base;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
 
+    // tensor memory columns
+    const uint32_t cDP = 64, cDQ1 = 128, cDKTR = 192, cDW = 256;                       // phase A
+    const uint32_t cDTA = 320, cDTB = 384, cDKB = 256, cDVB = 64, cDQ2 = 0, cDKT = 448;   // phase B
+    const uint32_t cY = 320, cRAW = 384, cZ = 320, cDKR = 384;                          // phases C, D, E
+
     // persistent: one CTA per SM walks over the (chunk, head) tiles.  The operands of the next tile
-    // are requested in two batches as soon as the shared-memory regions they land in are dead, and
-    // its per-token scalars are fetched into registers one tile ahead.
-    auto next_tile = [&](int t) {   // first non-empty tile of this CTA at or after t
-        while (t < a.ntiles && a.tab.chunk_len((int)(t / H)) == 0) t += (int)gridDim.x;
-        return t;
+    // are requested as soon as the shared-memory regions they land in are dead, its per-token scalars
+    // are fetched into registers one tile ahead, and its first products (phase A, which reads only what
+    // the chain kernels and the caller wrote) are issued while the current tile's sums and stores
+    // are still being formed.
+    // A tile index t = chunk * H + head advances by the grid size; chunk, head and (for a dense batch)
+    // sequence and chunk within the sequence are carried along, so that no integer division sits on the
+    // tile-to-tile path.
+    struct TileAt { int t, c, h, seq, n; };
+    const int step_c = (int)gridDim.x / H, step_h = (int)gridDim.x % H;
+    const int dense_nc = a.tab.dense_nc, dense_T = a.tab.dense_T;
+    auto tile_len = [&](const TileAt& x) {
+        if (!dense_T) return a.tab.chunk_len_[x.c];
+        const int rem = dense_T - x.n * CH;
+        return rem < CH ? rem : CH;
     };
-    // The copies of a tile arrive on one barrier phase; the transaction count is announced with the
-    // first group that is issued (expect_all), whichever that is.
-    constexpr uint32_t TILE_TX = 10 * BOX + 16384 + 16384 + 8192 + 32768 + 32768;
-    auto expect_all = [&]() { mbar_expect_tx(&bar_tma, TILE_TX); };
-    auto issue_first = [&](int t, int t0) {   // q, k, ktil, v
-        const int hh = (int)(t % H);
-        for (int hf = 0; hf < 2; ++hf) {
-            tma_load_2d(sm + R_Q + hf * BOX, &tmQ, hh * KD + hf * 64, t0, &bar_tma);
-            tma_load_2d(sm + R_K + hf * BOX, &tmK, hh * KD + hf * 64, t0, &bar_tma);
-            tma_load_2d(sm + R_KT + hf * BOX, &tmKt, hh * KD + hf * 64, t0, &bar_tma);
-            tma_load_2d(sm + R_V + hf * BOX, &tmV, hh * KD + hf * 64, t0, &bar_tma);
+    auto tile_tok0 = [&](const TileAt& x) { return dense_T ? x.seq * dense_T + x.n * CH : a.tab.chunk_tok0_[x.c]; };
+    auto tile_step = [&](TileAt& x) {
+        int dc = step_c;
+        x.t += (int)gridDim.x;
+        x.h += step_h;
+        if (x.h >= H) { x.h -= H; ++dc; }
+        x.c += dc;
+        if (dense_T) {
+            x.n += dc;
+            while (x.n >= dense_nc) { x.n -= dense_nc; ++x.seq; }
         }
     };
-    auto issue_dout = [&](int t, int t0) {
-        const int hh = (int)(t % H);
-        for (int hf = 0; hf < 2; ++hf) tma_load_2d(sm + R_DO + hf * BOX, &tmDO, hh * KD + hf * 64, t0, &bar_tma);
+    auto next_tile = [&](TileAt x) {   // first non-empty tile of this CTA at or after x
+        while (x.t < a.ntiles && tile_len(x) == 0) tile_step(x);
+        return x;
     };
-    auto issue_chain_tiles = [&](int t) {   // dU, ddU, T, S, dS
-        bulk_load(sm + R_DU, a.dUT + (size_t)t * 16384, 16384, &bar_tma);
-        bulk_load(sm + R_DDU, a.ddUT + (size_t)t * 16384, 16384, &bar_tma);
-        bulk_load(sm + R_T, a.Tm + (size_t)t * 8192, 8192, &bar_tma);
-        bulk_load(sm + R_S, a.Sn + (size_t)t * 32768, 32768, &bar_tma);
-        bulk_load(sm + R_DS, a.dSn + (size_t)t * 32768, 32768, &bar_tma);
+    // The copies of a tile arrive on one phase of each barrier; the transaction count is announced with
+    // the first group that is issued, whichever that is.
+    constexpr uint32_t CT_TX = 2 * BOX + 16384 + 16384 + 8192 + 32768 + 32768, TOK_TX = 8 * BOX;
+    auto load_qkkt = [&](int hh, int t0) {
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_load_2d(sm + R_Q + hf * BOX, &tmQ, hh * KD + hf * 64, t0, &bar_tok);
+            tma_load_2d(sm + R_K + hf * BOX, &tmK, hh * KD + hf * 64, t0, &bar_tok);
+            tma_load_2d(sm + R_KT + hf * BOX, &tmKt, hh * KD + hf * 64, t0, &bar_tok);
+        }
     };
-    auto fetch_scalars = [&](int t, int t0, int ln, float& g, float& b) {
-        const int hh = (int)(t % H);
-        const bool in = tid < ln;
-        g = (tid < CH && in) ? a.gate[(size_t)(t0 + tid) * H + hh] : 0.f;
-        b = (tid < CH && in) ? a.beta[(size_t)(t0 + tid) * H + hh] : 0.f;
+    auto load_v = [&](int hh, int t0) {
+        for (int hf = 0; hf < 2; ++hf) tma_load_2d(sm + R_V + hf * BOX, &tmV, hh * KD + hf * 64, t0, &bar_tok);
+    };
+    auto load_dout = [&](int hh, int t0) {
+        for (int hf = 0; hf < 2; ++hf) tma_load_2d(sm + R_DO + hf * BOX, &tmDO, hh * KD + hf * 64, t0, &bar_ct);
+    };
+    auto load_du_ds_s = [&](int t) {
+        bulk_load(sm + R_DU, a.dUT + (size_t)t * 16384, 16384, &bar_ct);
+        bulk_load(sm + R_DS, a.dSn + (size_t)t * 32768, 32768, &bar_ct);
+        bulk_load(sm + R_S, a.Sn + (size_t)t * 32768, 32768, &bar_ct);
+    };
+    auto load_ddu = [&](int t) { bulk_load(sm + R_DDU, a.ddUT + (size_t)t * 16384, 16384, &bar_ct); };
+    auto load_t = [&](int t) { bulk_load(sm + R_T, a.Tm + (size_t)t * 8192, 8192, &bar_ct); };
+    auto fetch_scalars = [&](int t, int hh, int t0, int ln, int buf) {   // tokens beyond the chunk read as zero
+        if (tid < CH) {
+            const bool in = tid < ln;
+            const size_t th = (size_t)(t0 + (in ? tid : 0)) * H + hh;
+            cp_async4_zfill(&sScal[buf][0][tid], a.gate + th, in);
+            cp_async4_zfill(&sScal[buf][1][tid], a.beta + th, in);
+        } else if (tid < CH + 2) {
+            cp_async4_zfill(&sSkipW[buf][tid - CH], a.skipw + (size_t)t * 2 + (tid - CH), true);
+        }
+        cp_async_commit();
+    };
+    // phase A: dP' = dO dU^T ; dQ1^T = S^T dO^T ; dKtr^T = dS^T dU ; dW^T = -S^T ddU  (warps 0-3, one each)
+    auto issue_phase_a = [&](bool go) {
+        if (lane == 0 && warp < 4 && go) {
+            tc_fence_after();
+            if (warp == 0) {   // dP'[i][j] = sum_v dO[i][v] dU[j][v]                               (M = 64)
+                const uint64_t db0 = desc_mnmajor(sm + R_DU, 0);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tb + cDP, desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
+                           desc_advance(db0, 2048 * k), make_idesc(64, 64, IDESC_B_MN), k > 0);
+            }
+            if (warp == 1) {   // dQ1^T[k][i] = sum_v S[v][k] dO[i][v]
+                const uint64_t da0 = desc_mnmajor(sm + R_S, 16384);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tb + cDQ1, desc_advance(da0, 2048 * k),
+                           desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
+                           make_idesc(128, 64, IDESC_A_MN), k > 0);
+            }
+            if (warp == 2) {   // dKtr^T[k][j] = sum_v dS[v][k] dU[j][v]
+                const uint64_t da0 = desc_mnmajor(sm + R_DS, 16384), db0 = desc_mnmajor(sm + R_DU, 0);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tb + cDKTR, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
+                           make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
+            }
+            if (warp == 3) {   // dW^T[k][i] = -sum_v S[v][k] ddU[i][v]
+                const uint64_t da0 = desc_mnmajor(sm + R_S, 16384), db0 = desc_mnmajor(sm + R_DDU, 0);
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tb + cDW, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
+                           make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN | IDESC_A_NEG), k > 0);
+            }
+            mma_commit(&bar_mma[0]);
+        }
     };
     uint32_t ph = 0;   // barrier phase parity: number of tiles processed so far, mod 2
-    int tile_l = next_tile((int)blockIdx.x);
+    TileAt cur;
+    cur.t = (int)blockIdx.x;
+    cur.c = (int)blockIdx.x / H;
+    cur.h = (int)blockIdx.x % H;
+    cur.seq = dense_T ? cur.c / dense_nc : 0;
+    cur.n = dense_T ? cur.c % dense_nc : 0;
+    cur = cur.t < a.ntiles ? next_tile(cur) : cur;
     int tok0 = 0, len = 0;
-    float g_cur = 0.f, b_cur = 0.f;
-    unsigned long long sk_cur = 0ull;
-    if (tile_l < a.ntiles) {
-        sk_cur = (unsigned long long)a.skipw[(size_t)tile_l * 2] | ((unsigned long long)a.skipw[(size_t)tile_l * 2 + 1] << 32);
-        tok0 = a.tab.chunk_tok0((int)(tile_l / H));
-        len = a.tab.chunk_len((int)(tile_l / H));
+    bool a_issued = false;   // phase A of the current tile was issued at the end of the previous one
+    if (cur.t < a.ntiles) {
+        tok0 = tile_tok0(cur);
+        len = tile_len(cur);
         if (tid == 0) {
-            expect_all();
-            issue_first(tile_l, tok0);
-            issue_dout(tile_l, tok0);
-            issue_chain_tiles(tile_l);
+            mbar_expect_tx(&bar_ct, CT_TX);
+            load_dout(cur.h, tok0);
+            load_du_ds_s(cur.t);
+            load_ddu(cur.t);
+            load_t(cur.t);
+            mbar_expect_tx(&bar_tok, TOK_TX);
+            load_qkkt(cur.h, tok0);
+            load_v(cur.h, tok0);
         }
-        fetch_scalars(tile_l, tok0, len, g_cur, b_cur);
+        fetch_scalars(cur.t, cur.h, tok0, len, 0);
     }
-    while (tile_l < a.ntiles) {
-    const int h = (int)(tile_l % H);
+    while (cur.t < a.ntiles) {
+    const int h = cur.h;
+    const float* sg = sScal[ph][0];      // log-gates of the chunk's tokens
+    const float* sBeta = sScal[ph][1];
     if (tid < CH) {
-        sg[tid] = g_cur;
-        sBeta[tid] = b_cur;
         sdB[tid] = 0.f;
         sdG[tid] = 0.f;
     }
     if (tid == 0) sRsum = 0.f;
+    cp_async_wait_all();   // this tile's scalars and skip words (requested a tile ago) have landed
     __syncthreads();
-    // table entries and scalars of the next tile, one tile ahead
-    const int tile_next = next_tile(tile_l + (int)gridDim.x);
+    // table entries, scalars and skip words of the next tile, one tile ahead
+    TileAt nxt = cur;
+    tile_step(nxt);
+    nxt = next_tile(nxt);
+    const int tile_next = nxt.t, h_next = nxt.h;
     int tok0_next = 0, len_next = 0;
-    float g_next = 0.f, b_next = 0.f;
     if (tile_next < a.ntiles) {
-        tok0_next = a.tab.chunk_tok0((int)(tile_next / H));
-        len_next = a.tab.chunk_len((int)(tile_next / H));
-        fetch_scalars(tile_next, tok0_next, len_next, g_next, b_next);
+        tok0_next = tile_tok0(nxt);
+        len_next = tile_len(nxt);
+        fetch_scalars(tile_next, h_next, tok0_next, len_next, (int)(ph ^ 1u));
     }
-
-    // skip words (every thread reads the same two words), like the scalars fetched one tile ahead so
-    // that nothing at the top of a tile waits for memory
-    const unsigned long long sk = sk_cur;
-    unsigned long long sk_next = 0ull;
-    if (tile_next < a.ntiles)
-        sk_next = (unsigned long long)a.skipw[(size_t)tile_next * 2] |
-                  ((unsigned long long)a.skipw[(size_t)tile_next * 2 + 1] << 32);
+    const unsigned long long sk = (unsigned long long)sSkipW[ph][0] | ((unsigned long long)sSkipW[ph][1] << 32);
     // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's preconditioner
     // step was skipped); ragged or mixed chunks are copied row by row.  In the all-skipped case the
-    // space of each chain tile is not reused by the output staging, so the next tile's copy of it
-    // starts as soon as the last product reading it has finished (thread 0, below).
+    // space of dO and of each chain tile is not reused by the output staging, so the next tile's copy of
+    // it starts as soon as the last product reading it has finished ("early"), and when that tile is a
+    // full chunk its phase A is issued before this tile's sums are formed ("a_early").
     const bool full = len == CH;
     const bool dk_tile = full && sk == ~0ull;
     const bool early = dk_tile && tile_next < a.ntiles;
+    const bool a_early = early && len_next == CH;
     if (warp == 0) {   // in-chunk gate prefix G_i and the decay vectors (lane: tokens l and l + 32)
         float sa = sg[lane], sb = sg[lane + 32];
 #pragma unroll
@@ -1383,107 +1472,35 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sRho[lane] = __expf(tot - sa);
         sRho[lane + 32] = __expf(tot - sb);
     }
-    bool ok = mbar_wait(&bar_tma, ph, a.status, ERR_TMA);
-    if (len < CH) {
-        for (int hf = 0; hf < 2; ++hf) {
-            zero_tail_rows(sm + R_Q + hf * BOX, len, tid, CBW_THREADS);
-            zero_tail_rows(sm + R_K + hf * BOX, len, tid, CBW_THREADS);
-            zero_tail_rows(sm + R_KT + hf * BOX, len, tid, CBW_THREADS);
-            zero_tail_rows(sm + R_V + hf * BOX, len, tid, CBW_THREADS);
-            zero_tail_rows(sm + R_DO + hf * BOX, len, tid, CBW_THREADS);
-        }
+    bool ok = mbar_wait(&bar_ct, ph, a.status, ERR_TMA);
+    if (len < CH) {   // a ragged chunk never had its phase A issued ahead
+        for (int hf = 0; hf < 2; ++hf) zero_tail_rows(sm + R_DO + hf * BOX, len, tid, CBW_THREADS);
         fence_proxy_async();
     }
+    tc_fence_before();
     __syncthreads();
 
-    // tensor memory columns
-    const uint32_t cRAW = 0, cDP = 64, cDQ1 = 128, cDKTR = 192, cDW = 256, cDTA = 320, cDTB = 384, cDKT = 448;
-    const uint32_t cDKB = 256, cDVB = 64, cDQ2 = 0, cY = 320, cZ = 384, cDKR = 320;
-
     // ---- phase A -------------------------------------------------------------------------------
-    if (lane == 0 && warp < 5 && ok) {
-        tc_fence_after();
-        if (warp == 0) {
-        for (int k = 0; k < 8; ++k) {   // rawkk[i][j] = <k_i, ktil_j>          (M = 64)
-            mma_ss(tb + cRAW, desc_advance(desc_kmajor(sm + R_K + (k >> 2) * BOX), 32 * (k & 3)),
-                   desc_advance(desc_kmajor(sm + R_KT + (k >> 2) * BOX), 32 * (k & 3)), make_idesc(64, 64), k > 0);
-        }
-        }
-        if (warp == 1) {   // dP'[i][j] = sum_v dO[i][v] dU[j][v]                               (M = 64)
-            const uint64_t db0 = desc_mnmajor(sm + R_DU, 0);
-            for (int k = 0; k < 8; ++k)
-                mma_ss(tb + cDP, desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
-                       desc_advance(db0, 2048 * k), make_idesc(64, 64, IDESC_B_MN), k > 0);
-        }
-        if (warp == 2) {   // dQ1^T[k][i] = sum_v S[v][k] dO[i][v]
-            const uint64_t da0 = desc_mnmajor(sm + R_S, 16384);
-            for (int k = 0; k < 8; ++k)
-                mma_ss(tb + cDQ1, desc_advance(da0, 2048 * k),
-                       desc_advance(desc_kmajor(sm + R_DO + (k >> 2) * BOX), 32 * (k & 3)),
-                       make_idesc(128, 64, IDESC_A_MN), k > 0);
-        }
-        if (warp == 3) {   // dKtr^T[k][j] = sum_v dS[v][k] dU[j][v]
-            const uint64_t da0 = desc_mnmajor(sm + R_DS, 16384), db0 = desc_mnmajor(sm + R_DU, 0);
-            for (int k = 0; k < 8; ++k)
-                mma_ss(tb + cDKTR, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
-                       make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
-        }
-        if (warp == 4) {   // dW^T[k][i] = -sum_v S[v][k] ddU[i][v]
-            const uint64_t da0 = desc_mnmajor(sm + R_S, 16384), db0 = desc_mnmajor(sm + R_DDU, 0);
-            for (int k = 0; k < 8; ++k)
-                mma_ss(tb + cDW, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
-                       make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN | IDESC_A_NEG), k > 0);
-        }
-        mma_commit(&bar_mma[0]);
-    }
-    // <dS, S>_F while the tensor core works (both images share the same layout)
-    {
-        float part = 0.f;
-        for (int e = tid; e < 2048; e += CBW_THREADS) {
-            const uint4 x = *reinterpret_cast<const uint4*>(sm + R_S + e * 16);
-            const uint4 y = *reinterpret_cast<const uint4*>(sm + R_DS + e * 16);
-            const __nv_bfloat162* px = reinterpret_cast<const __nv_bfloat162*>(&x);
-            const __nv_bfloat162* py = reinterpret_cast<const __nv_bfloat162*>(&y);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float2 fx = __bfloat1622float2(px[q]), fy = __bfloat1622float2(py[q]);
-                part = fmaf(fx.x, fy.x, part);
-                part = fmaf(fx.y, fy.y, part);
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-        if (lane == 0) sRed[warp] = part;
-    }
+    if (!a_issued) issue_phase_a(ok);
     ok = ok && mbar_wait(&bar_mma[0], ph, a.status, ERR_MMA1);
     tc_fence_after();
-    __syncthreads();   // every thread is done reading S / dS before their space is reused
     // epilogue A
+    float gam8[8];   // Gamma_ij = exp(G_i - G_j) for this thread's row and columns, j <= i (else 0)
     {
-        // rawkk, dP' (64-row accumulators: rows in lanes 0-15 of each quadrant)
+        // dP' -> M1 = scale Gamma (.) lower(dP')
         const int i = row64;
         const float Gi = sG[i];
         {
-            uint32_t r1[16], r2[16];
-            const int j0 = colq * 16;
-            tmem_ld16(tb + cRAW + lane_addr + j0, r1);
-            tmem_ld16(tb + cDP + lane_addr + j0, r2);
+            uint32_t r2[8];
+            tmem_ld_half8(tb + cDP + addr64, r2);
+            float m1[8];
+#pragma unroll
+            for (int x = 0; x < 8; ++x) gam8[x] = jb + x <= i ? __expf(Gi - sG[jb + x]) : 0.f;
             tmem_ld_wait();
-            if (row_active) {
-                float m1[16];
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const int j = j0 + x;
-                    const float gm = j <= i ? __expf(Gi - sG[j]) : 0.f;
-                    sRaw[i * LC + j] = j < i ? gm * __uint_as_float(r1[x]) : 0.f;
-                    m1[x] = a.scale * gm * __uint_as_float(r2[x]);
-                }
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2)
-                    *reinterpret_cast<uint4*>(sm + R_M1 + sw128_chunk(i, (j0 >> 3) + c2)) =
-                        make_uint4(pack_bf16(m1[c2 * 8 + 0], m1[c2 * 8 + 1]), pack_bf16(m1[c2 * 8 + 2], m1[c2 * 8 + 3]),
-                                   pack_bf16(m1[c2 * 8 + 4], m1[c2 * 8 + 5]), pack_bf16(m1[c2 * 8 + 6], m1[c2 * 8 + 7]));
-            }
+            for (int x = 0; x < 8; ++x) m1[x] = a.scale * gam8[x] * __uint_as_float(r2[x]);
+            *reinterpret_cast<uint4*>(sm + R_IMG + sw128_chunk(i, jb >> 3)) =
+                make_uint4(pack_bf16(m1[0], m1[1]), pack_bf16(m1[2], m1[3]), pack_bf16(m1[4], m1[5]), pack_bf16(m1[6], m1[7]));
         }
         // dW^T -> bf16 image [rows k][cols i]
         {
@@ -1497,6 +1514,15 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3])),
                     pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5])),
                     pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7])));
+        }
+    }
+    ok = ok && mbar_wait(&bar_tok, ph, a.status, ERR_TMA);   // q, k, ktil, v have landed
+    if (len < CH) {
+        for (int hf = 0; hf < 2; ++hf) {
+            zero_tail_rows(sm + R_Q + hf * BOX, len, tid, CBW_THREADS);
+            zero_tail_rows(sm + R_K + hf * BOX, len, tid, CBW_THREADS);
+            zero_tail_rows(sm + R_KT + hf * BOX, len, tid, CBW_THREADS);
+            zero_tail_rows(sm + R_V + hf * BOX, len, tid, CBW_THREADS);
         }
     }
     fence_proxy_async();
@@ -1534,7 +1560,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         if (warp == 4 || warp == 5) {   // dq2^T[k][i] = sum_j Ktil[j][k] M1[i][j] ;  dktil^T[k][j] = sum_i Q[i][k] M1[i][j]
             const uint64_t da0 = desc_mnmajor(sm + R_KT, BOX), da1 = desc_mnmajor(sm + R_Q, BOX);
-            const uint64_t dbk = desc_kmajor(sm + R_M1), dbm = desc_mnmajor(sm + R_M1, 0);
+            const uint64_t dbk = desc_kmajor(sm + R_IMG), dbm = desc_mnmajor(sm + R_IMG, 0);
             if (warp == 4)
                 for (int k = 0; k < 4; ++k)
                     mma_ss(tb + cDQ2, desc_advance(da0, 2048 * k), desc_advance(dbk, 32 * k),
@@ -1545,79 +1571,159 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                            make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
         }
         mma_commit(&bar_mma[1]);
-        if (early && warp == 0) {   // phase A has finished: dU and dS are dead
-            expect_all();
-            bulk_load(sm + R_DU, a.dUT + (size_t)tile_next * 16384, 16384, &bar_tma);
-            bulk_load(sm + R_DS, a.dSn + (size_t)tile_next * 32768, 32768, &bar_tma);
+    }
+    // <dS, S>_F while the tensor core works on phase B (both images share the same layout)
+    {
+        float part = 0.f;
+        for (int e = tid; e < 2048; e += CBW_THREADS) {
+            const uint4 x = *reinterpret_cast<const uint4*>(sm + R_S + e * 16);
+            const uint4 y = *reinterpret_cast<const uint4*>(sm + R_DS + e * 16);
+            const __nv_bfloat162* px = reinterpret_cast<const __nv_bfloat162*>(&x);
+            const __nv_bfloat162* py = reinterpret_cast<const __nv_bfloat162*>(&y);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 fx = __bfloat1622float2(px[q]), fy = __bfloat1622float2(py[q]);
+                part = fmaf(fx.x, fy.x, part);
+                part = fmaf(fx.y, fy.y, part);
+            }
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        if (lane == 0) sRed[warp] = part;
+    }
+    __syncthreads();   // every thread is done reading S / dS: phase A has finished, dU, dS and S are dead
+    if (early && tid == 0 && ok) {
+        mbar_expect_tx(&bar_ct, CT_TX);
+        load_du_ds_s(tile_next);
     }
     ok = ok && mbar_wait(&bar_mma[1], ph, a.status, ERR_MMA2);
     tc_fence_after();
-    {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j]
+    {   // dT = dT_a beta_j gamma_j + dT_b beta_j  -> bf16 image [rows i][cols j];
+        // dbeta_j += sum_i T_ij (gamma_j dT_a + dT_b)_ij: beta enters W = T diag(beta gamma) K and
+        // U = T diag(beta) V column by column
         const int i = row64;
+        uint32_t r1[8], r2[8];
+        tmem_ld_half8(tb + cDTA + addr64, r1);
+        tmem_ld_half8(tb + cDTB + addr64, r2);
+        const uint4 tw = *reinterpret_cast<const uint4*>(sm + R_T + sw128_chunk(i, jb >> 3));
+        const float4 ba = *reinterpret_cast<const float4*>(&sBeta[jb]), bb = *reinterpret_cast<const float4*>(&sBeta[jb + 4]);
+        const float4 ga = *reinterpret_cast<const float4*>(&sGam[jb]), gb = *reinterpret_cast<const float4*>(&sGam[jb + 4]);
+        const float bj[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
+        const float gj[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+        float tij[8];
         {
-            uint32_t r1[16], r2[16];
-            const int j0 = colq * 16;
-            tmem_ld16(tb + cDTA + lane_addr + j0, r1);
-            tmem_ld16(tb + cDTB + lane_addr + j0, r2);
-            tmem_ld_wait();
-            if (row_active) {
-                float t[16];
+            const __nv_bfloat162* p0 = reinterpret_cast<const __nv_bfloat162*>(&tw);
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const int j = j0 + x;
-                    t[x] = sBeta[j] * (sGam[j] * __uint_as_float(r1[x]) + __uint_as_float(r2[x]));
-                }
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2)
-                    *reinterpret_cast<uint4*>(sm + R_DT + sw128_chunk(i, (j0 >> 3) + c2)) =
-                        make_uint4(pack_bf16(t[c2 * 8 + 0], t[c2 * 8 + 1]), pack_bf16(t[c2 * 8 + 2], t[c2 * 8 + 3]),
-                                   pack_bf16(t[c2 * 8 + 4], t[c2 * 8 + 5]), pack_bf16(t[c2 * 8 + 6], t[c2 * 8 + 7]));
+            for (int x = 0; x < 4; ++x) {
+                const float2 u0 = __bfloat1622float2(p0[x]);
+                tij[2 * x] = u0.x;
+                tij[2 * x + 1] = u0.y;
             }
         }
+        tmem_ld_wait();
+        float t[8], cs[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            const float u = gj[x] * __uint_as_float(r1[x]) + __uint_as_float(r2[x]);
+            t[x] = bj[x] * u;
+            cs[x] = tij[x] * u;
+        }
+        *reinterpret_cast<uint4*>(sm + R_IMG + sw128_chunk(i, jb >> 3)) =
+            make_uint4(pack_bf16(t[0], t[1]), pack_bf16(t[2], t[3]), pack_bf16(t[4], t[5]), pack_bf16(t[6], t[7]));
+        // column sums over the 16 rows of a half warp: in each of three steps a lane keeps one half of its
+        // columns and hands the other half to its partner; a last exchange joins the two lanes that end
+        // up with the same column
+#pragma unroll
+        for (int step = 0; step < 3; ++step) {
+            const int off = 8 >> step, n = 4 >> step;
+            const bool upper = (lane & off) != 0;
+#pragma unroll
+            for (int x = 0; x < n; ++x) {
+                const float send = upper ? cs[x] : cs[x + n], keep = upper ? cs[x + n] : cs[x];
+                cs[x] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            }
+        }
+        cs[0] += __shfl_xor_sync(0xffffffffu, cs[0], 1);
+        if ((lane & 1) == 0) atomicAdd(&sdB[jb + ((lane & 15) >> 1)], cs[0]);
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
 
-    // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] -----------------------------------------------
-    if (tid == 0 && ok) {
+    // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] ; rawkk[i][j] = <k_i, ktil_j> -------------------
+    if (lane == 0 && warp < 2 && ok) {
         tc_fence_after();
-        const uint64_t da0 = desc_mnmajor(sm + R_T, 0), db0 = desc_mnmajor(sm + R_DT, 0);
-        for (int k = 0; k < 4; ++k)
-            mma_ss(tb + cY, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
-                   make_idesc(64, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
+        if (warp == 0) {
+            const uint64_t da0 = desc_mnmajor(sm + R_T, 0), db0 = desc_mnmajor(sm + R_IMG, 0);
+            for (int k = 0; k < 4; ++k)
+                mma_ss(tb + cY, desc_advance(da0, 2048 * k), desc_advance(db0, 2048 * k),
+                       make_idesc(64, 64, IDESC_A_MN | IDESC_B_MN), k > 0);
+        } else {
+            for (int k = 0; k < 8; ++k)   // (M = 64)
+                mma_ss(tb + cRAW, desc_advance(desc_kmajor(sm + R_K + (k >> 2) * BOX), 32 * (k & 3)),
+                       desc_advance(desc_kmajor(sm + R_KT + (k >> 2) * BOX), 32 * (k & 3)), make_idesc(64, 64), k > 0);
+        }
         mma_commit(&bar_mma[2]);
-        if (early) bulk_load(sm + R_DDU, a.ddUT + (size_t)tile_next * 16384, 16384, &bar_tma);   // phase B done
+        if (early && warp == 0) {   // phase B has finished: ddU and the dW^T image (in the space of dO) are dead
+            load_ddu(tile_next);
+            load_dout(h_next, tok0_next);
+        }
+    }
+    // dq = scale gamma dQ1 + dq2 (both complete since phase B) while the tensor core works on phase C
+    // (lane = feature f, columns = tokens; four token columns at a time)
+    float gv[16];   // per column: gate contribution of this feature
+    const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
+    const uint32_t fc = f & 63;
+    {
+        __nv_bfloat16* stq = reinterpret_cast<__nv_bfloat16*>(sm + ST_DQ);
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+            const int j0 = colq * 16 + cb * 4;
+            uint32_t rq1[4], rq2[4];
+            tmem_ld4(tb + cDQ1 + lane_addr + j0, rq1);
+            tmem_ld4(tb + cDQ2 + lane_addr + j0, rq2);
+            float qv[4];
+            const float4 g4 = *reinterpret_cast<const float4*>(&sGam[j0]);
+            const float gj[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+                qv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_Q + boxf + sw128_elem(j0 + x, fc)));
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const float dq = a.scale * gj[x] * __uint_as_float(rq1[x]) + __uint_as_float(rq2[x]);
+                gv[cb * 4 + x] = dq * qv[x];
+                stq[(j0 + x) * KD + f] = __float2bfloat16_rn(dq);
+            }
+        }
     }
     ok = ok && mbar_wait(&bar_mma[2], ph, a.status, ERR_MMA2);
     tc_fence_after();
+    float rawg[8];   // Gamma_ij <k_i, ktil_j>, j < i (kept in registers for the beta gradient of phase D)
     {
         const int i = row64;
-        {
-            uint32_t r[16];
-            const int j0 = colq * 16;
-            tmem_ld16(tb + cY + lane_addr + j0, r);
-            tmem_ld_wait();
-            if (row_active) {
+        uint32_t r[8], r1[8];
+        tmem_ld_half8(tb + cY + addr64, r);
+        tmem_ld_half8(tb + cRAW + addr64, r1);
+        tmem_ld_wait();
 #pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2)
-                    *reinterpret_cast<uint4*>(sm + R_Y + sw128_chunk(i, (j0 >> 3) + c2)) = make_uint4(
-                        pack_bf16(__uint_as_float(r[c2 * 8 + 0]), __uint_as_float(r[c2 * 8 + 1])),
-                        pack_bf16(__uint_as_float(r[c2 * 8 + 2]), __uint_as_float(r[c2 * 8 + 3])),
-                        pack_bf16(__uint_as_float(r[c2 * 8 + 4]), __uint_as_float(r[c2 * 8 + 5])),
-                        pack_bf16(__uint_as_float(r[c2 * 8 + 6]), __uint_as_float(r[c2 * 8 + 7])));
-            }
-        }
+        for (int x = 0; x < 8; ++x) rawg[x] = jb + x < i ? gam8[x] * __uint_as_float(r1[x]) : 0.f;
+        *reinterpret_cast<uint4*>(sm + R_IMG + sw128_chunk(i, jb >> 3)) = make_uint4(
+            pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1])), pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3])),
+            pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5])), pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7])));
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
 
+    if (tid == CBW_STORE_TID && ok && full) {   // the dq tile is staged (fenced before the barrier above)
+        tma_store_2d(&tmDQ, h * KD, tok0, sm + ST_DQ);
+        bulk_commit();
+    }
     // ---- phase D: Z[a][b] = sum_c Y[a][c] T[b][c] ; dA = -strictLower(Z) --------------------------
     if (tid == 0 && ok) {
         tc_fence_after();
-        const uint64_t da0 = desc_kmajor(sm + R_Y), db0 = desc_kmajor(sm + R_T);
+        const uint64_t da0 = desc_kmajor(sm + R_IMG), db0 = desc_kmajor(sm + R_T);
         for (int k = 0; k < 4; ++k)
             mma_ss(tb + cZ, desc_advance(da0, 32 * k), desc_advance(db0, 32 * k), make_idesc(64, 64), k > 0);
         mma_commit(&bar_mma[3]);
@@ -1626,30 +1732,22 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_after();
     {
         const int i = row64;
-        const float bi = sBeta[i], Gi = sG[i];
+        const float bi = sBeta[i];
         float db = 0.f;
-        {
-            uint32_t r[16];
-            const int j0 = colq * 16;
-            tmem_ld16(tb + cZ + lane_addr + j0, r);
-            tmem_ld_wait();
-            if (row_active) {
-                float m2[16];
+        uint32_t r[8];
+        tmem_ld_half8(tb + cZ + addr64, r);
+        tmem_ld_wait();
+        float m2[8];
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const int j = j0 + x;
-                    const float da = j < i ? -__uint_as_float(r[x]) : 0.f;
-                    db = fmaf(da, sRaw[i * LC + j], db);
-                    m2[x] = j < i ? da * bi * __expf(Gi - sG[j]) : 0.f;
-                }
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2)
-                    *reinterpret_cast<uint4*>(sm + R_M2 + sw128_chunk(i, (j0 >> 3) + c2)) =
-                        make_uint4(pack_bf16(m2[c2 * 8 + 0], m2[c2 * 8 + 1]), pack_bf16(m2[c2 * 8 + 2], m2[c2 * 8 + 3]),
-                                   pack_bf16(m2[c2 * 8 + 4], m2[c2 * 8 + 5]), pack_bf16(m2[c2 * 8 + 6], m2[c2 * 8 + 7]));
-            }
+        for (int x = 0; x < 8; ++x) {
+            const float da = jb + x < i ? -__uint_as_float(r[x]) : 0.f;
+            db = fmaf(da, rawg[x], db);
+            m2[x] = da * bi * gam8[x];
         }
-        if (row_active) atomicAdd(&sdB[i], db);
+        *reinterpret_cast<uint4*>(sm + R_IMG + sw128_chunk(i, jb >> 3)) =
+            make_uint4(pack_bf16(m2[0], m2[1]), pack_bf16(m2[2], m2[3]), pack_bf16(m2[4], m2[5]), pack_bf16(m2[6], m2[7]));
+        db += __shfl_xor_sync(0xffffffffu, db, 16);   // the two halves of a row's sixteen columns
+        if (lane < 16) atomicAdd(&sdB[i], db);
     }
     fence_proxy_async();
     tc_fence_before();
@@ -1659,7 +1757,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (lane == 0 && warp < 2 && ok) {
         tc_fence_after();
         const uint64_t da0 = desc_mnmajor(sm + R_K, BOX), da1 = desc_mnmajor(sm + R_KT, BOX);
-        const uint64_t dbm = desc_mnmajor(sm + R_M2, 0), dbk = desc_kmajor(sm + R_M2);
+        const uint64_t dbm = desc_mnmajor(sm + R_IMG, 0), dbk = desc_kmajor(sm + R_IMG);
         if (warp == 0)
             for (int k = 0; k < 4; ++k)
                 mma_ss(tb + cDKT, desc_advance(da0, 2048 * k), desc_advance(dbm, 2048 * k),
@@ -1669,22 +1767,16 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 mma_ss(tb + cDKR, desc_advance(da1, 2048 * k), desc_advance(dbk, 32 * k),
                        make_idesc(128, 64, IDESC_A_MN), k > 0);
         mma_commit(&bar_mma[4]);
-        if (early && warp == 0) bulk_load(sm + R_T, a.Tm + (size_t)tile_next * 8192, 8192, &bar_tma);   // phase D done
+        if (early && warp == 0) load_t(tile_next);   // phase D has finished: T is dead
     }
     ok = ok && mbar_wait(&bar_mma[4], ph, a.status, ERR_MMA2);
     tc_fence_after();
-    // every product has finished: the images in the space of S are dead
-    if (early && tid == 0 && ok) bulk_load(sm + R_S, a.Sn + (size_t)tile_next * 32768, 32768, &bar_tma);
 
-    // ---- final epilogue (lane = feature f, columns = tokens) --------------------------------------
+    // ---- final epilogue (lane = feature f, columns = tokens): dv, dk ---------------------------------
     float rsum = 0.f;
-    float gv[16], bv[16];   // per column: gate and beta contributions of this feature
     if (ok) {
-        const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
-        const uint32_t fc = f & 63;
         // Results are staged in shared memory as [token][feature] tiles (the operand tiles of the
         // finished products are dead by now) and written out with 16-byte stores afterwards.
-        __nv_bfloat16* stq = reinterpret_cast<__nv_bfloat16*>(sm + ST_DQ);
         __nv_bfloat16* stv = reinterpret_cast<__nv_bfloat16*>(sm + ST_DV);
         __nv_bfloat16* stk = reinterpret_cast<__nv_bfloat16*>(sm + ST_DK);
         float* stkr = reinterpret_cast<float*>(sm + ST_DKR);
@@ -1693,15 +1785,13 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
             const int j0 = colq * 16 + cb * 4;
-            uint32_t rq1[4], rq2[4], rkt[4], rdk[4], rkb[4], rkr[4], rvb[4];
-            tmem_ld4(tb + cDQ1 + lane_addr + j0, rq1);
-            tmem_ld4(tb + cDQ2 + lane_addr + j0, rq2);
+            uint32_t rkt[4], rdk[4], rkb[4], rkr[4], rvb[4];
             tmem_ld4(tb + cDVB + lane_addr + j0, rvb);
             tmem_ld4(tb + cDKTR + lane_addr + j0, rkt);
             tmem_ld4(tb + cDKT + lane_addr + j0, rdk);
             tmem_ld4(tb + cDKB + lane_addr + j0, rkb);
             tmem_ld4(tb + cDKR + lane_addr + j0, rkr);
-            float qv[4], kv[4], ktv[4], vv[4];
+            float kv[4], ktv[4];
             const float4 b4 = *reinterpret_cast<const float4*>(&sBeta[j0]);
             const float4 g4 = *reinterpret_cast<const float4*>(&sGam[j0]);
             const float4 r4 = *reinterpret_cast<const float4*>(&sRho[j0]);
@@ -1710,25 +1800,20 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const uint32_t eo = boxf + sw128_elem(j0 + x, fc);
-                qv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_Q + eo));
                 kv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_K + eo));
                 ktv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_KT + eo));
-                vv[x] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(sm + R_V + eo));
             }
             tmem_ld_wait();
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int j = j0 + x;
-                const float dq = a.scale * gj[x] * __uint_as_float(rq1[x]) + __uint_as_float(rq2[x]);
                 const float dktr = rj[x] * __uint_as_float(rkt[x]);
                 const float dkt = dktr + __uint_as_float(rdk[x]);
                 const float dkb = __uint_as_float(rkb[x]);
                 const float dkr = bj[x] * gj[x] * dkb + __uint_as_float(rkr[x]);
                 const float dvb = __uint_as_float(rvb[x]);
-                gv[cb * 4 + x] = dq * qv[x] + dkr * kv[x] - dkt * ktv[x];
-                bv[cb * 4 + x] = gj[x] * dkb * kv[x] + dvb * vv[x];
+                gv[cb * 4 + x] += dkr * kv[x] - dkt * ktv[x];
                 rsum = fmaf(dktr, ktv[x], rsum);
-                stq[j * KD + f] = __float2bfloat16_rn(dq);
                 stv[j * KD + f] = __float2bfloat16_rn(bj[x] * dvb);
                 stk[j * KD + f] = __float2bfloat16_rn(dkr + a.d_min * dkt);
                 if (!dk_tile) {   // fp32 copies feed the preconditioner's reverse pass only
@@ -1741,18 +1826,22 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     }
     fence_proxy_async();
-    ok = __syncthreads_and(ok);   // block-uniform from here on; staging complete, q, k, ktil, v dead
-    if (tid == 0) {
-        if (tile_next < a.ntiles) {
-            if (!early) expect_all();
-            issue_first(tile_next, tok0_next);
-        }
-        if (ok && full) {   // the tiles leave while the per-token sums below are formed
-            tma_store_2d(&tmDQ, h * KD, tok0, sm + ST_DQ);
-            tma_store_2d(&tmDV, h * KD, tok0, sm + ST_DV);
-            if (dk_tile) tma_store_2d(&tmDK, h * KD, tok0, sm + ST_DK);
-            bulk_commit();
-        }
+    tc_fence_before();
+    ok = __syncthreads_and(ok);   // block-uniform from here on; staging complete, q, k, ktil dead, accumulators read
+    if (tid == 32 && early) {   // the next tile's q, k, ktil (v follows once the dq tile has left its space)
+        mbar_expect_tx(&bar_tok, TOK_TX);
+        load_qkkt(h_next, tok0_next);
+    }
+    if (tid == CBW_STORE_TID && ok && full) {   // the tiles leave while the per-token sums below are formed
+        tma_store_2d(&tmDV, h * KD, tok0, sm + ST_DV);
+        if (dk_tile) tma_store_2d(&tmDK, h * KD, tok0, sm + ST_DK);
+        bulk_commit();
+    }
+    if (a_early) {
+        // phase A of the next tile: everything it reads was requested before this tile's phase C ended
+        bool okn = true;
+        if (warp < 4 && ok) okn = mbar_wait(&bar_ct, ph ^ 1u, a.status, ERR_TMA);
+        issue_phase_a(ok && okn);
     }
     if (ok) {
         // Sum over the 32 features of the warp for all 16 columns at once: in each of four steps a
@@ -1765,17 +1854,11 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
             for (int i = 0; i < n; ++i) {
                 const float gs = upper ? gv[i] : gv[i + n], gk = upper ? gv[i + n] : gv[i];
-                const float bs = upper ? bv[i] : bv[i + n], bk = upper ? bv[i + n] : bv[i];
                 gv[i] = gk + __shfl_xor_sync(0xffffffffu, gs, off);
-                bv[i] = bk + __shfl_xor_sync(0xffffffffu, bs, off);
             }
         }
         gv[0] += __shfl_xor_sync(0xffffffffu, gv[0], 1);
-        bv[0] += __shfl_xor_sync(0xffffffffu, bv[0], 1);
-        if ((lane & 1) == 0) {
-            atomicAdd(&sdG[colq * 16 + (lane >> 1)], gv[0]);
-            atomicAdd(&sdB[colq * 16 + (lane >> 1)], bv[0]);
-        }
+        if ((lane & 1) == 0) atomicAdd(&sdG[colq * 16 + (lane >> 1)], gv[0]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
         if (lane == 0) atomicAdd(&sRsum, rsum);
@@ -1828,7 +1911,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             }
         }
         if (dk_tile) {
-            // only the first token's dL/dktil is needed (a reverse recurrence may restart there)
+            // only the first token's dL/dktil is needed (a reverse pass may restart there)
             for (int e = tid; e < 32; e += CBW_THREADS) {
                 const size_t g = ((size_t)tok0 * H + h) * KD + e * 4;
                 *reinterpret_cast<uint4*>(a.dktil + g) = *reinterpret_cast<const uint4*>(&sFirstKt[e * 4]);
@@ -1846,25 +1929,34 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         *reinterpret_cast<const uint4*>(sm + ST_DKT + j * 512 + ch * 16);
             }
         }
-        if (full && tid == 0) bulk_wait_read();   // the staging tiles may be overwritten by the next tile
+        if (full && tid == CBW_STORE_TID) {
+            bulk_wait_read();   // the staging tiles may be overwritten by the next tile
+            if (early) load_v(h_next, tok0_next);
+        }
     }
     __syncthreads();   // every copy-out read of the staging tiles is done
     if (tid == 0 && tile_next < a.ntiles) {
-        issue_dout(tile_next, tok0_next);
-        if (!early) issue_chain_tiles(tile_next);
+        if (!early) {
+            mbar_expect_tx(&bar_ct, CT_TX);
+            load_dout(h_next, tok0_next);
+            load_du_ds_s(tile_next);
+            load_ddu(tile_next);
+            load_t(tile_next);
+            mbar_expect_tx(&bar_tok, TOK_TX);
+            load_qkkt(h_next, tok0_next);
+            load_v(h_next, tok0_next);
+        }
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    a_issued = a_early && ok;
     ph ^= 1u;
-    tile_l = tile_next;
+    cur = nxt;
     tok0 = tok0_next;
     len = len_next;
-    g_cur = g_next;
-    b_cur = b_next;
-    sk_cur = sk_next;
     }   // tile loop
-    if (tid == 0) bulk_wait_all();
+    if (tid == CBW_STORE_TID) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tb, 512);

@@ -150,6 +150,16 @@ __device__ __forceinline__ void bulk_prefetch(const void* gsrc, uint32_t bytes)
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gsrc), "r"(bytes) : "memory");
 }
 
+// 4-byte asynchronous copy global -> shared by the calling thread (cp.async group of that thread);
+// with valid == false nothing is read and the destination is filled with zero.
+__device__ __forceinline__ void cp_async4_zfill(void* smem_dst, const void* gsrc, bool valid)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(valid ? 4 : 0)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void prefetch_tmap(const void* tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
@@ -263,6 +273,17 @@ __device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t* r)
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(taddr)
+                 : "memory");
+}
+// 16x32bx2 shape: two 16-lane accesses in one instruction.  Threads 0-15 of the warp read lanes
+// base .. base + 15 at columns [col, col + 8), threads 16-31 read the SAME 16 lanes at columns
+// [col + 8, col + 16).  A 64-row accumulator keeps its rows in lanes 0-15 of every lane quadrant, so this
+// form reads 16 of its columns with all 32 threads busy (8 columns each).
+__device__ __forceinline__ void tmem_ld_half8(uint32_t taddr, uint32_t* r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.16x32bx2.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8], 8;"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(taddr)
                  : "memory");
 }
