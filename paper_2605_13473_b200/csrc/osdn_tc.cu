@@ -1237,16 +1237,15 @@ constexpr uint32_t R_DWT = R_DO;                 // dW^T image replaces dO after
 // predecessor has finished), so they share one 8 KB image behind the fp32 scratch.
 constexpr uint32_t R_IMG = R_RAW + 24576;
 // Output staging ([token][feature] tiles over dead space): dq over V (dead after phase B; dq is complete
-// then and is formed while phase C runs), dk and dv after the last product over the fp32 scratch (dead
-// after phase D) and the operand image; the fp32 copies of dk_read and dL/dktil, needed only when some
-// token's preconditioner step was really taken, over T, S and dS.  When every token of a full chunk was
+// then and is formed while phase C runs), dv over Q (dead once dq is formed; dv is formed while phase E
+// runs), dk after the last product in a region of its own; the fp32 copies of dk_read and dL/dktil,
+// needed only when some token's preconditioner step was really taken, over T, S and dS.  When every token of a full chunk was
 // skipped, the space of dO, dU, ddU, T, S and dS is therefore never reused inside a tile and the next
 // tile's copies of them start as soon as the last product reading the current ones has finished.
-constexpr uint32_t ST_DQ = R_V, ST_DV = R_RAW + 16384, ST_DK = R_RAW, ST_DKR = 114688, ST_DKT = 147456;
+constexpr uint32_t ST_DQ = R_V, ST_DV = R_Q, ST_DK = R_RAW, ST_DKR = 114688, ST_DKT = 147456;
 constexpr int CBW_STORE_TID = 256;   // the thread that sends the output tiles off (and owns their bulk group)
 static_assert(ST_DKT + 32768 <= R_RAW, "fp32 staging tiles must fit below the fp32 scratch");
 constexpr size_t CBW_SMEM = R_RAW + 32768 + 1024;
-static_assert(CH * LC * 4 <= 24576, "fp32 scratch must end before the shared operand image");
 
 __global__ void __launch_bounds__(CBW_THREADS, 1)
 tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -1261,7 +1260,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // bar_tok: q, k, ktil, v
     __shared__ uint64_t bar_ct, bar_tok, bar_mma[5];
     __shared__ uint32_t tmem_base;
-    __shared__ __align__(16) float sG[CH], sGam[CH], sRho[CH], sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
+    __shared__ __align__(16) float sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
+    // in-chunk gate prefix G_i, gamma_i = exp(G_i), rho_i = exp(G_C - G_i): two buffers, the next tile's
+    // vectors are formed during this tile's last stretch
+    __shared__ __align__(16) float sGv[2][3][CH];
     // per-token gate and beta and the two skip words of a tile, copied asynchronously one tile ahead
     // (two buffers; values fetched into registers that early would be spilled, and the spill would wait
     // for the load)
@@ -1336,15 +1338,17 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // The copies of a tile arrive on one phase of each barrier; the transaction count is announced with
     // the first group that is issued, whichever that is.
     constexpr uint32_t CT_TX = 2 * BOX + 16384 + 16384 + 8192 + 32768 + 32768, TOK_TX = 8 * BOX;
-    auto load_qkkt = [&](int hh, int t0) {
+    auto load_kkt = [&](int hh, int t0) {
         for (int hf = 0; hf < 2; ++hf) {
-            tma_load_2d(sm + R_Q + hf * BOX, &tmQ, hh * KD + hf * 64, t0, &bar_tok);
             tma_load_2d(sm + R_K + hf * BOX, &tmK, hh * KD + hf * 64, t0, &bar_tok);
             tma_load_2d(sm + R_KT + hf * BOX, &tmKt, hh * KD + hf * 64, t0, &bar_tok);
         }
     };
-    auto load_v = [&](int hh, int t0) {
-        for (int hf = 0; hf < 2; ++hf) tma_load_2d(sm + R_V + hf * BOX, &tmV, hh * KD + hf * 64, t0, &bar_tok);
+    auto load_qv = [&](int hh, int t0) {
+        for (int hf = 0; hf < 2; ++hf) {
+            tma_load_2d(sm + R_Q + hf * BOX, &tmQ, hh * KD + hf * 64, t0, &bar_tok);
+            tma_load_2d(sm + R_V + hf * BOX, &tmV, hh * KD + hf * 64, t0, &bar_tok);
+        }
     };
     auto load_dout = [&](int hh, int t0) {
         for (int hf = 0; hf < 2; ++hf) tma_load_2d(sm + R_DO + hf * BOX, &tmDO, hh * KD + hf * 64, t0, &bar_ct);
@@ -1399,6 +1403,22 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mma_commit(&bar_mma[0]);
         }
     };
+    auto gate_vectors = [&](int buf) {   // one warp; lane: tokens l and l + 32
+        float sa = sScal[buf][0][lane], sb = sScal[buf][0][lane + 32];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float ua = __shfl_up_sync(0xffffffffu, sa, o), ub = __shfl_up_sync(0xffffffffu, sb, o);
+            if (lane >= o) { sa += ua; sb += ub; }
+        }
+        sb += __shfl_sync(0xffffffffu, sa, 31);
+        const float tot = __shfl_sync(0xffffffffu, sb, 31);
+        sGv[buf][0][lane] = sa;
+        sGv[buf][0][lane + 32] = sb;
+        sGv[buf][1][lane] = __expf(sa);
+        sGv[buf][1][lane + 32] = __expf(sb);
+        sGv[buf][2][lane] = __expf(tot - sa);
+        sGv[buf][2][lane + 32] = __expf(tot - sb);
+    };
     uint32_t ph = 0;   // barrier phase parity: number of tiles processed so far, mod 2
     TileAt cur;
     cur.t = (int)blockIdx.x;
@@ -1419,21 +1439,26 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             load_ddu(cur.t);
             load_t(cur.t);
             mbar_expect_tx(&bar_tok, TOK_TX);
-            load_qkkt(cur.h, tok0);
-            load_v(cur.h, tok0);
+            load_kkt(cur.h, tok0);
+            load_qv(cur.h, tok0);
         }
         fetch_scalars(cur.t, cur.h, tok0, len, 0);
+        cp_async_wait_all();
+        __syncthreads();
     }
     while (cur.t < a.ntiles) {
     const int h = cur.h;
     const float* sg = sScal[ph][0];      // log-gates of the chunk's tokens
     const float* sBeta = sScal[ph][1];
+    const float* sG = sGv[ph][0];
+    const float* sGam = sGv[ph][1];
+    const float* sRho = sGv[ph][2];
     if (tid < CH) {
         sdB[tid] = 0.f;
         sdG[tid] = 0.f;
     }
     if (tid == 0) sRsum = 0.f;
-    cp_async_wait_all();   // this tile's scalars and skip words (requested a tile ago) have landed
+    cp_async_wait_all();
     __syncthreads();
     // table entries, scalars and skip words of the next tile, one tile ahead
     TileAt nxt = cur;
@@ -1456,22 +1481,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const bool dk_tile = full && sk == ~0ull;
     const bool early = dk_tile && tile_next < a.ntiles;
     const bool a_early = early && len_next == CH;
-    if (warp == 0) {   // in-chunk gate prefix G_i and the decay vectors (lane: tokens l and l + 32)
-        float sa = sg[lane], sb = sg[lane + 32];
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float ua = __shfl_up_sync(0xffffffffu, sa, o), ub = __shfl_up_sync(0xffffffffu, sb, o);
-            if (lane >= o) { sa += ua; sb += ub; }
-        }
-        sb += __shfl_sync(0xffffffffu, sa, 31);
-        const float tot = __shfl_sync(0xffffffffu, sb, 31);
-        sG[lane] = sa;
-        sG[lane + 32] = sb;
-        sGam[lane] = __expf(sa);
-        sGam[lane + 32] = __expf(sb);
-        sRho[lane] = __expf(tot - sa);
-        sRho[lane + 32] = __expf(tot - sb);
-    }
+    if (warp == 0) gate_vectors((int)ph);
     bool ok = mbar_wait(&bar_ct, ph, a.status, ERR_TMA);
     if (len < CH) {   // a ragged chunk never had its phase A issued ahead
         for (int hf = 0; hf < 2; ++hf) zero_tail_rows(sm + R_DO + hf * BOX, len, tid, CBW_THREADS);
@@ -1574,8 +1584,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     // <dS, S>_F while the tensor core works on phase B (both images share the same layout)
     {
-        float part = 0.f;
-        for (int e = tid; e < 2048; e += CBW_THREADS) {
+        float p4[4] = {0.f, 0.f, 0.f, 0.f};   // independent partial sums: no chain of dependent multiply-adds
+#pragma unroll
+        for (int it = 0; it < 2048 / CBW_THREADS; ++it) {
+            const int e = tid + it * CBW_THREADS;
             const uint4 x = *reinterpret_cast<const uint4*>(sm + R_S + e * 16);
             const uint4 y = *reinterpret_cast<const uint4*>(sm + R_DS + e * 16);
             const __nv_bfloat162* px = reinterpret_cast<const __nv_bfloat162*>(&x);
@@ -1583,10 +1595,11 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const float2 fx = __bfloat1622float2(px[q]), fy = __bfloat1622float2(py[q]);
-                part = fmaf(fx.x, fy.x, part);
-                part = fmaf(fx.y, fy.y, part);
+                p4[q] = fmaf(fx.x, fy.x, p4[q]);
+                p4[q] = fmaf(fx.y, fy.y, p4[q]);
             }
         }
+        float part = (p4[0] + p4[1]) + (p4[2] + p4[3]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
         if (lane == 0) sRed[warp] = part;
@@ -1769,15 +1782,30 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         mma_commit(&bar_mma[4]);
         if (early && warp == 0) load_t(tile_next);   // phase D has finished: T is dead
     }
+    // dv = beta dVb (complete since phase B) while the tensor core works on phase E; staged over Q (every
+    // read of q ended before the barrier that followed phase C)
+    {
+        __nv_bfloat16* stv = reinterpret_cast<__nv_bfloat16*>(sm + ST_DV);
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+            const int j0 = colq * 16 + cb * 4;
+            uint32_t rvb[4];
+            tmem_ld4(tb + cDVB + lane_addr + j0, rvb);
+            const float4 b4 = *reinterpret_cast<const float4*>(&sBeta[j0]);
+            const float bj[4] = {b4.x, b4.y, b4.z, b4.w};
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 4; ++x) stv[(j0 + x) * KD + f] = __float2bfloat16_rn(bj[x] * __uint_as_float(rvb[x]));
+        }
+    }
     ok = ok && mbar_wait(&bar_mma[4], ph, a.status, ERR_MMA2);
     tc_fence_after();
 
-    // ---- final epilogue (lane = feature f, columns = tokens): dv, dk ---------------------------------
+    // ---- final epilogue (lane = feature f, columns = tokens): dk --------------------------------------
     float rsum = 0.f;
     if (ok) {
         // Results are staged in shared memory as [token][feature] tiles (the operand tiles of the
         // finished products are dead by now) and written out with 16-byte stores afterwards.
-        __nv_bfloat16* stv = reinterpret_cast<__nv_bfloat16*>(sm + ST_DV);
         __nv_bfloat16* stk = reinterpret_cast<__nv_bfloat16*>(sm + ST_DK);
         float* stkr = reinterpret_cast<float*>(sm + ST_DKR);
         float* stkt = reinterpret_cast<float*>(sm + ST_DKT);
@@ -1785,8 +1813,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
             const int j0 = colq * 16 + cb * 4;
-            uint32_t rkt[4], rdk[4], rkb[4], rkr[4], rvb[4];
-            tmem_ld4(tb + cDVB + lane_addr + j0, rvb);
+            uint32_t rkt[4], rdk[4], rkb[4], rkr[4];
             tmem_ld4(tb + cDKTR + lane_addr + j0, rkt);
             tmem_ld4(tb + cDKT + lane_addr + j0, rdk);
             tmem_ld4(tb + cDKB + lane_addr + j0, rkb);
@@ -1811,10 +1838,8 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const float dkt = dktr + __uint_as_float(rdk[x]);
                 const float dkb = __uint_as_float(rkb[x]);
                 const float dkr = bj[x] * gj[x] * dkb + __uint_as_float(rkr[x]);
-                const float dvb = __uint_as_float(rvb[x]);
                 gv[cb * 4 + x] += dkr * kv[x] - dkt * ktv[x];
                 rsum = fmaf(dktr, ktv[x], rsum);
-                stv[j * KD + f] = __float2bfloat16_rn(bj[x] * dvb);
                 stk[j * KD + f] = __float2bfloat16_rn(dkr + a.d_min * dkt);
                 if (!dk_tile) {   // fp32 copies feed the preconditioner's reverse pass only
                     stkr[j * KD + f] = dkr;
@@ -1828,9 +1853,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     ok = __syncthreads_and(ok);   // block-uniform from here on; staging complete, q, k, ktil dead, accumulators read
-    if (tid == 32 && early) {   // the next tile's q, k, ktil (v follows once the dq tile has left its space)
+    if (tid == CBW_STORE_TID && early) {   // the next tile's k, ktil (q, v follow once the dv, dq tiles have left their space)
         mbar_expect_tx(&bar_tok, TOK_TX);
-        load_qkkt(h_next, tok0_next);
+        load_kkt(h_next, tok0_next);
     }
     if (tid == CBW_STORE_TID && ok && full) {   // the tiles leave while the per-token sums below are formed
         tma_store_2d(&tmDV, h * KD, tok0, sm + ST_DV);
@@ -1931,7 +1956,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         if (full && tid == CBW_STORE_TID) {
             bulk_wait_read();   // the staging tiles may be overwritten by the next tile
-            if (early) load_v(h_next, tok0_next);
+            if (early) load_qv(h_next, tok0_next);
         }
     }
     __syncthreads();   // every copy-out read of the staging tiles is done
@@ -1943,13 +1968,10 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             load_ddu(tile_next);
             load_t(tile_next);
             mbar_expect_tx(&bar_tok, TOK_TX);
-            load_qkkt(h_next, tok0_next);
-            load_v(h_next, tok0_next);
+            load_kkt(h_next, tok0_next);
+            load_qv(h_next, tok0_next);
         }
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
     a_issued = a_early && ok;
     ph ^= 1u;
     cur = nxt;
