@@ -82,9 +82,8 @@ def method_bytes(name, inp, with_bwd):
         "phase1_seq": 0.0, "phase1_bwd_seq": 0.0, "build_table": 0.0,
         "tc_chunk_fwd": 2 * K * es + 8,                              # q, k, beta, gate
         "tc_chain_fwd": V * es + V * es + (state if with_bwd else 0),  # v in, out, saved state
-        "tc_chain_bwd": V * es,                                      # dout
         # q, k, v, dout, beta, gate, the saved state in; dq, dk, dv, dbeta, dgate out
-        "tc_chunk_bwd": (2 * K + 2 * V) * es + 8 + state + (2 * K + V) * es + 8,
+        "tc_bwd": (2 * K + 2 * V) * es + 8 + state + (2 * K + V) * es + 8,
     }
     return None if name not in per else per[name] * tokh
 
@@ -123,11 +122,13 @@ def kernel_model(name, inp, NT):
                          tiles * (f(128, 64, K) + f(128, 64, C)), "hbm")
     m["tc_chain_fwd"] = (tiles * (16384 + 8192 + 8192 + 3 * raw + raw + 32768 + 16384) + tokh * 4,
                          tiles * (f(128, 64, C) + 2 * f(128, 64, K) + f(128, 64, C) + f(128, 128, C)), "hbm")
-    m["tc_chain_bwd"] = (tiles * (2 * raw + 8192 + 16384 + 16384 + 32768 + 16384) + tokh * 4,
-                         tiles * (f(128, 64, C) + f(128, 64, K) + 2 * f(128, 128, C)), "hbm")
-    m["tc_chunk_bwd"] = (tiles * (5 * raw + 16384 + 16384 + 8192 + 32768 + 32768 + 3 * raw) + tokh * 24,
-                         tiles * (2 * f(64, 64, K) + 3 * f(128, 64, K) + 2 * f(64, 64, K) + 2 * f(128, 64, C)
-                                  + 2 * f(64, 64, C) + 4 * f(128, 64, C)), "hbm")
+    # one launch: the reverse state chains (dout, ktil, W^T, P', Qg in; dS_n, ddU^T out) and the chunk-local
+    # part (q, k, ktil, v, dout, dU^T, ddU^T, T, S_n, dS_n in; dq, dk, dv out)
+    m["tc_bwd"] = (tiles * (2 * raw + 8192 + 16384 + 16384 + 32768 + 16384) + tokh * 4
+                   + tiles * (5 * raw + 16384 + 16384 + 8192 + 32768 + 32768 + 3 * raw) + tokh * 24,
+                   tiles * (f(128, 64, C) + f(128, 64, K) + 2 * f(128, 128, C))
+                   + tiles * (2 * f(64, 64, K) + 3 * f(128, 64, K) + 2 * f(64, 64, K) + 2 * f(128, 64, C)
+                              + 2 * f(64, 64, C) + 4 * f(128, 64, C)), "hbm")
     return m.get(name)
 
 

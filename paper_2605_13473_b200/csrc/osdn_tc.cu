@@ -37,12 +37,12 @@ constexpr int KD = 128;  // K = V = 128 on this path
 constexpr uint32_t BOX = 8192;   // one [64 rows x 128 B] box
 
 // device status codes of bounded waits
-enum { ERR_TMA = 101, ERR_MMA1 = 102, ERR_MMA2 = 103, ERR_CHAIN_TMA = 111, ERR_CHAIN_MMA1 = 112, ERR_CHAIN_MMA2 = 113 };
+enum { ERR_QUEUE = 121, ERR_TMA = 101, ERR_MMA1 = 102, ERR_MMA2 = 103, ERR_CHAIN_TMA = 111, ERR_CHAIN_MMA1 = 112, ERR_CHAIN_MMA2 = 113 };
 
 constexpr uint32_t REC_BYTES = 49152;   // stride of the Tb | W^T | P' | Qg record of a tile
 
 struct TcLayout {
-    size_t ktil, WT, Tb, Tm, P, Qg, Sn, dUT, ddUT, dSn, dktil, dkread, total;
+    size_t ktil, WT, Tb, Tm, P, Qg, Sn, dUT, ddUT, dSn, dktil, dkread, queue, total;
 };
 
 TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
@@ -69,6 +69,7 @@ TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
         t.dSn = take(NT * H * 32768);
         t.dktil = take(Ttot * H * KD * 4);
         t.dkread = take(Ttot * H * KD * 4);
+        t.queue = take(sizeof(int) * (64 + NT * H));
     }
     t.total = off;
     return t;
@@ -933,20 +934,36 @@ constexpr size_t CB_SMEM = 2 * BSTAGE_BYTES + 32768 + 16384 + 1024;
 constexpr int CBK_EPI_WARPS = 16, CBK_MMA_WARP = 16, CBK_TMA_WARP = 17;
 constexpr int CBK_THREADS = 18 * 32;
 
-__global__ void __launch_bounds__(CBK_THREADS, 1)
-tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_constant__ CUtensorMap tmKt,
-                    TcChainBwdArgs a)
+// Queue of (chunk, head) tiles between the backward chains (producers) and the chunk-local backward
+// (consumers) inside one kernel: slot i holds tile + 1 once the i-th finished tile has been published
+// (0 = not yet); consumers draw tickets from `head`.  The whole array is cleared before the launch.
+struct TileQueue {
+    int* slots;
+    unsigned *head, *tail;
+    // Publishes `count` tiles first, first + stride, ... (one fence and one counter update for all).
+    __device__ __forceinline__ void push(int first, int stride, int count) const
+    {
+        if (count <= 0) return;
+        fence_proxy_async_all();   // the tiles' images were written through the async proxy
+        __threadfence();
+        const unsigned slot = atomicAdd(tail, (unsigned)count);
+        for (int i = 0; i < count; ++i) *reinterpret_cast<volatile int*>(slots + slot + i) = first + i * stride + 1;
+    }
+};
+
+// One chain (sequence, head) of the backward state recurrence, by all CBK_THREADS threads of the CTA.
+// `tb`: 256 free tensor-memory columns.  Every (chunk, head) tile whose cotangent images have reached
+// global memory is appended to the tile queue `tq`, in the order the chains produce them.
+__device__ __forceinline__ void chain_bwd_role(const CUtensorMap& tmDO, const CUtensorMap& tmKt, const TcChainBwdArgs& a,
+                                               int chain, uint8_t* sm, uint32_t tb, const TileQueue& tq)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* sm = align1024(smem_raw);
     uint8_t* sStage = sm;
     uint8_t* sdS = sm + 2 * BSTAGE_BYTES;       // dS as bf16, K-major, 2 k-halves x [128 x 128 B]
     uint8_t* sddU = sdS + 32768;                // ddU^T, K-major [v][i]
     __shared__ uint64_t bar_full[2], bar_empty[2], bar_s_ready, bar_a_done, bar_a_ready, bar_s_done;
-    __shared__ uint32_t tmem_base;
     __shared__ float sRho[2][CH], sGC[2];
 
-    const int chain = blockIdx.x, H = a.H;
+    const int H = a.H;
     const int s = chain / H, h = chain % H;
     const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
     const int seq_t0 = a.tab.seq_tok0(s), seq_len = a.tab.seq_len(s);
@@ -978,11 +995,9 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         mbar_init(&bar_s_done, 1);
         fence_mbar_init();
     }
-    if (warp == 0) tmem_alloc(&tmem_base, 256);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tb = tmem_base;
     const uint32_t tS = tb, tA1 = tb + 128, tA2 = tb + 192;
 
     if (warp == CBK_TMA_WARP) {
@@ -1031,6 +1046,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
         // ------------------------------------------------------------------ tensor-core issuer
         bool ok = true;
         bool a1_issued = false;   // dO^T P' of the coming chunk is already in its accumulator
+        int next_pub = 1, interval = 1, published = 0;   // publication of finished tiles (lane 0)
         auto issue_a1 = [&](uint8_t* d) {   // acc1 = dO^T P'
             const uint32_t idesc = make_idesc(128, 64, IDESC_A_MN | IDESC_B_MN);
             const uint64_t da0 = desc_mnmajor(d + BS_DO, BOX), db0 = desc_mnmajor(d + BS_P, 0);
@@ -1093,8 +1109,24 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
                 __syncwarp();
                 a1_issued = true;
             }
+            // Finished tiles go to the chunk-local workers in batches: a publication costs the issuing
+            // thread a fence and a round trip to memory, and the workers consume far more slowly than the
+            // chains produce, so the batches grow (1, 2, 4, ... up to 16 steps).  Only tiles whose two
+            // bulk groups were committed at least a whole step ago are included: waiting for this
+            // chunk's own stores would put their round trip on the chunk-to-chunk path.
+            if (lane == 0 && n >= next_pub) {
+                bulk_wait_all_but<2>();
+                tq.push((int)chunk_tile(n - 1), H, n - published);   // steps published .. n - 1 (tile ids rise by H per step back)
+                published = n;
+                interval = min(2 * interval, 16);
+                next_pub = n + interval;
+            }
+            __syncwarp();
         }
-        if (lane == 0) bulk_wait_all();
+        if (lane == 0) {
+            bulk_wait_all();
+            if (ok) tq.push((int)chunk_tile(nchunks - 1), H, nchunks - published);
+        }
     } else {
         // ------------------------------------------------------------------ state warps
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
@@ -1201,7 +1233,12 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tb, 256);
+    if (tid == 0) {   // the barrier words are initialised again for the CTA's next chain
+        mbar_inval(&bar_full[0]); mbar_inval(&bar_full[1]); mbar_inval(&bar_empty[0]); mbar_inval(&bar_empty[1]);
+        mbar_inval(&bar_s_ready); mbar_inval(&bar_a_done); mbar_inval(&bar_a_ready); mbar_inval(&bar_s_done);
+    }
+    __syncthreads();
+    tc_fence_after();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1218,7 +1255,7 @@ tc_chain_bwd_kernel(const __grid_constant__ CUtensorMap tmDO, const __grid_const
 //             dv = beta dVb ; dgate from the products of the gradients with their inputs
 // ---------------------------------------------------------------------------------------------
 struct TcChunkBwdArgs {
-    int H, ntiles;
+    int H, ntiles, nseq;
     Table tab;
     const float *beta, *gate;
     float scale, d_min;
@@ -1244,22 +1281,21 @@ constexpr uint32_t R_IMG = R_RAW + 24576;
 // tile's copies of them start as soon as the last product reading the current ones has finished.
 constexpr uint32_t ST_DQ = R_V, ST_DV = R_Q, ST_DK = R_RAW, ST_DKR = 114688, ST_DKT = 147456;
 constexpr int CBW_STORE_TID = 256;   // the thread that sends the output tiles off (and owns their bulk group)
+constexpr int CBW_QUEUE_TID = 480;   // the thread that talks to the tile queue (a warp that issues no products)
 static_assert(ST_DKT + 32768 <= R_RAW, "fp32 staging tiles must fit below the fp32 scratch");
 constexpr size_t CBW_SMEM = R_RAW + 32768 + 1024;
 
-__global__ void __launch_bounds__(CBW_THREADS, 1)
-tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                    const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmV,
-                    const __grid_constant__ CUtensorMap tmDO, const __grid_constant__ CUtensorMap tmDQ,
-                    const __grid_constant__ CUtensorMap tmDK, const __grid_constant__ CUtensorMap tmDV,
-                    TcChunkBwdArgs a)
+// The chunk-local backward of the tiles drawn from the queue, by the first CBW_THREADS threads of the CTA
+// (their barrier is hardware barrier 1).  `tb`: 512 tensor-memory columns.
+__device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmKt,
+                                               const CUtensorMap& tmV, const CUtensorMap& tmDO, const CUtensorMap& tmDQ,
+                                               const CUtensorMap& tmDK, const CUtensorMap& tmDV, const TcChunkBwdArgs& a,
+                                               uint8_t* sm, uint32_t tb, const TileQueue& tq)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* sm = align1024(smem_raw);
     // bar_ct: dO and the tiles written by the chain kernels (everything phase A reads);
     // bar_tok: q, k, ktil, v
     __shared__ uint64_t bar_ct, bar_tok, bar_mma[5];
-    __shared__ uint32_t tmem_base;
+    __shared__ int sNext[4];   // next tile of this CTA: {tile, head, first token, length}; tile -1: not published yet, -2: none left
     __shared__ __align__(16) float sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
     // in-chunk gate prefix G_i, gamma_i = exp(G_i), rho_i = exp(G_C - G_i): two buffers, the next tile's
     // vectors are formed during this tile's last stretch
@@ -1291,11 +1327,9 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int i = 0; i < 5; ++i) mbar_init(&bar_mma[i], issuers[i]);
         fence_mbar_init();
     }
-    if (warp == 0) tmem_alloc(&tmem_base, 512);
     tc_fence_before();
-    __syncthreads();
+    named_sync(1, CBW_THREADS);
     tc_fence_after();
-    const uint32_t tb = tmem_base;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
 
     // tensor memory columns
@@ -1308,32 +1342,32 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // are fetched into registers one tile ahead, and its first products (phase A, which reads only what
     // the chain kernels and the caller wrote) are issued while the current tile's sums and stores
     // are still being formed.
-    // A tile index t = chunk * H + head advances by the grid size; chunk, head and (for a dense batch)
-    // sequence and chunk within the sequence are carried along, so that no integer division sits on the
-    // tile-to-tile path.
-    struct TileAt { int t, c, h, seq, n; };
-    const int step_c = (int)gridDim.x / H, step_h = (int)gridDim.x % H;
-    const int dense_nc = a.tab.dense_nc, dense_T = a.tab.dense_T;
-    auto tile_len = [&](const TileAt& x) {
-        if (!dense_T) return a.tab.chunk_len_[x.c];
-        const int rem = dense_T - x.n * CH;
-        return rem < CH ? rem : CH;
+    // Tiles come from the queue the chains fill, in the order they were finished: thread 0 draws a ticket,
+    // looks the slot up (waiting, within a bound, only where nothing else is left to do) and leaves the
+    // tile's coordinates in shared memory for the others.
+    const int total = a.tab.seq_chunk0(a.nseq) * H;   // realised (chunk, head) tiles
+    auto resolve = [&](int v) {   // queue thread only: v = slot value (tile + 1) or 0 (not published)
+        if (!v) { sNext[0] = -1; return; }
+        const int t = v - 1, c = t / H;
+        sNext[0] = t;
+        sNext[1] = t - c * H;
+        sNext[2] = a.tab.chunk_tok0(c);
+        sNext[3] = a.tab.chunk_len(c);
+        fence_proxy_async_all();   // the tile's images are read through the async proxy
     };
-    auto tile_tok0 = [&](const TileAt& x) { return dense_T ? x.seq * dense_T + x.n * CH : a.tab.chunk_tok0_[x.c]; };
-    auto tile_step = [&](TileAt& x) {
-        int dc = step_c;
-        x.t += (int)gridDim.x;
-        x.h += step_h;
-        if (x.h >= H) { x.h -= H; ++dc; }
-        x.c += dc;
-        if (dense_T) {
-            x.n += dc;
-            while (x.n >= dense_nc) { x.n -= dense_nc; ++x.seq; }
+    auto lookup_blocking = [&](unsigned ticket) {   // queue thread only
+        if (ticket >= (unsigned)total) { sNext[0] = -2; return; }
+        int v = ld_acquire_gpu(tq.slots + ticket);
+        if (!v) {
+            const long long t0 = clock64();
+            while (!(v = ld_acquire_gpu(tq.slots + ticket))) {
+                if (clock64() - t0 > WAIT_LIMIT_CYCLES || *reinterpret_cast<volatile int*>(a.status) != 0) break;
+                __nanosleep(64);
+            }
+            if (!v) atomicCAS(a.status, 0, ERR_QUEUE);
         }
-    };
-    auto next_tile = [&](TileAt x) {   // first non-empty tile of this CTA at or after x
-        while (x.t < a.ntiles && tile_len(x) == 0) tile_step(x);
-        return x;
+        if (!v) { sNext[0] = -2; return; }
+        resolve(v);
     };
     // The copies of a tile arrive on one phase of each barrier; the transaction count is announced with
     // the first group that is issued, whichever that is.
@@ -1420,34 +1454,31 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sGv[buf][2][lane + 32] = __expf(tot - sb);
     };
     uint32_t ph = 0;   // barrier phase parity: number of tiles processed so far, mod 2
-    TileAt cur;
-    cur.t = (int)blockIdx.x;
-    cur.c = (int)blockIdx.x / H;
-    cur.h = (int)blockIdx.x % H;
-    cur.seq = dense_T ? cur.c / dense_nc : 0;
-    cur.n = dense_T ? cur.c % dense_nc : 0;
-    cur = cur.t < a.ntiles ? next_tile(cur) : cur;
-    int tok0 = 0, len = 0;
+    // queue thread: the ticket of the next tile is drawn a tile ahead and its slot is read at the top of
+    // the tile, long before the value is looked at, so that neither round trip to memory is waited for
+    unsigned ticket_next = 0, ticket_after = 0;
+    int slot_next = 0;
+    if (tid == CBW_QUEUE_TID) {
+        lookup_blocking(atomicAdd(tq.head, 1u));
+        ticket_next = atomicAdd(tq.head, 1u);
+    }
+    named_sync(1, CBW_THREADS);
+    int tile_l = sNext[0], h = sNext[1], tok0 = sNext[2], len = sNext[3];
     bool a_issued = false;   // phase A of the current tile was issued at the end of the previous one
-    if (cur.t < a.ntiles) {
-        tok0 = tile_tok0(cur);
-        len = tile_len(cur);
+    if (tile_l >= 0) {
         if (tid == 0) {
             mbar_expect_tx(&bar_ct, CT_TX);
-            load_dout(cur.h, tok0);
-            load_du_ds_s(cur.t);
-            load_ddu(cur.t);
-            load_t(cur.t);
+            load_dout(h, tok0);
+            load_du_ds_s(tile_l);
+            load_ddu(tile_l);
+            load_t(tile_l);
             mbar_expect_tx(&bar_tok, TOK_TX);
-            load_kkt(cur.h, tok0);
-            load_qv(cur.h, tok0);
+            load_kkt(h, tok0);
+            load_qv(h, tok0);
         }
-        fetch_scalars(cur.t, cur.h, tok0, len, 0);
-        cp_async_wait_all();
-        __syncthreads();
+        fetch_scalars(tile_l, h, tok0, len, 0);
     }
-    while (cur.t < a.ntiles) {
-    const int h = cur.h;
+    while (tile_l >= 0) {
     const float* sg = sScal[ph][0];      // log-gates of the chunk's tokens
     const float* sBeta = sScal[ph][1];
     const float* sG = sGv[ph][0];
@@ -1459,17 +1490,11 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     if (tid == 0) sRsum = 0.f;
     cp_async_wait_all();
-    __syncthreads();
-    // table entries, scalars and skip words of the next tile, one tile ahead
-    TileAt nxt = cur;
-    tile_step(nxt);
-    nxt = next_tile(nxt);
-    const int tile_next = nxt.t, h_next = nxt.h;
-    int tok0_next = 0, len_next = 0;
-    if (tile_next < a.ntiles) {
-        tok0_next = tile_tok0(nxt);
-        len_next = tile_len(nxt);
-        fetch_scalars(tile_next, h_next, tok0_next, len_next, (int)(ph ^ 1u));
+    named_sync(1, CBW_THREADS);
+    // the next tile's slot and the ticket of the tile after it (both values are used much later)
+    if (tid == CBW_QUEUE_TID) {
+        ticket_after = atomicAdd(tq.head, 1u);
+        slot_next = ticket_next < (unsigned)total ? ld_acquire_gpu(tq.slots + ticket_next) : 0;
     }
     const unsigned long long sk = (unsigned long long)sSkipW[ph][0] | ((unsigned long long)sSkipW[ph][1] << 32);
     // Full chunks leave through TMA tile stores (dq, dv always; dk when every token's preconditioner
@@ -1479,8 +1504,6 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // full chunk its phase A is issued before this tile's sums are formed ("a_early").
     const bool full = len == CH;
     const bool dk_tile = full && sk == ~0ull;
-    const bool early = dk_tile && tile_next < a.ntiles;
-    const bool a_early = early && len_next == CH;
     if (warp == 0) gate_vectors((int)ph);
     bool ok = mbar_wait(&bar_ct, ph, a.status, ERR_TMA);
     if (len < CH) {   // a ragged chunk never had its phase A issued ahead
@@ -1488,7 +1511,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         fence_proxy_async();
     }
     tc_fence_before();
-    __syncthreads();
+    named_sync(1, CBW_THREADS);
 
     // ---- phase A -------------------------------------------------------------------------------
     if (!a_issued) issue_phase_a(ok);
@@ -1537,7 +1560,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    named_sync(1, CBW_THREADS);
 
     // ---- phase B -------------------------------------------------------------------------------
     if (lane == 0 && warp < 6 && ok) {
@@ -1604,10 +1627,16 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
         if (lane == 0) sRed[warp] = part;
     }
-    __syncthreads();   // every thread is done reading S / dS: phase A has finished, dU, dS and S are dead
-    if (early && tid == 0 && ok) {
-        mbar_expect_tx(&bar_ct, CT_TX);
-        load_du_ds_s(tile_next);
+    named_sync(1, CBW_THREADS);   // every thread is done reading S / dS: phase A has finished, dU, dS and S are dead
+    // the next tile, if the chains have published it already (asked again at the end of this tile if not);
+    // the queue thread works this out while everybody waits for phase B, the others read it after the next barrier
+    if (tid == CBW_QUEUE_TID) {
+        if (ticket_next >= (unsigned)total) sNext[0] = -2;
+        else resolve(slot_next);
+        if (dk_tile && sNext[0] >= 0 && ok) {
+            mbar_expect_tx(&bar_ct, CT_TX);
+            load_du_ds_s(sNext[0]);
+        }
     }
     ok = ok && mbar_wait(&bar_mma[1], ph, a.status, ERR_MMA2);
     tc_fence_after();
@@ -1661,7 +1690,13 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    named_sync(1, CBW_THREADS);
+
+    int tile_next = sNext[0], h_next = sNext[1], tok0_next = sNext[2], len_next = sNext[3];
+    const bool next_known = tile_next >= 0;
+    if (next_known) fetch_scalars(tile_next, h_next, tok0_next, len_next, (int)(ph ^ 1u));
+    const bool early = dk_tile && next_known;
+    const bool a_early = early && len_next == CH;
 
     // ---- phase C: Y[a][b] = sum_i T[i][a] dT[i][b] ; rawkk[i][j] = <k_i, ktil_j> -------------------
     if (lane == 0 && warp < 2 && ok) {
@@ -1727,7 +1762,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    named_sync(1, CBW_THREADS);
 
     if (tid == CBW_STORE_TID && ok && full) {   // the dq tile is staged (fenced before the barrier above)
         tma_store_2d(&tmDQ, h * KD, tok0, sm + ST_DQ);
@@ -1764,7 +1799,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    named_sync(1, CBW_THREADS);
 
     // ---- phase E: dktil^T += K^T M2 ; dkr^T = Ktil^T M2^T -----------------------------------------
     if (lane == 0 && warp < 2 && ok) {
@@ -1852,7 +1887,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     fence_proxy_async();
     tc_fence_before();
-    ok = __syncthreads_and(ok);   // block-uniform from here on; staging complete, q, k, ktil dead, accumulators read
+    ok = named_sync_and(1, CBW_THREADS, ok);   // block-uniform from here on; staging complete, q, k, ktil dead, accumulators read
     if (tid == CBW_STORE_TID && early) {   // the next tile's k, ktil (q, v follow once the dv, dq tiles have left their space)
         mbar_expect_tx(&bar_tok, TOK_TX);
         load_kkt(h_next, tok0_next);
@@ -1888,7 +1923,7 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
         if (lane == 0) atomicAdd(&sRsum, rsum);
     }
-    __syncthreads();   // the per-token sums are complete
+    named_sync(1, CBW_THREADS);   // the per-token sums are complete
     if (ok && warp == 1) {
         // gate and beta gradients of the chunk: dgate_j is the suffix sum of the per-token terms (the
         // in-chunk prefix G_i collects every g_j with j <= i), by one warp while the tiles are sent off
@@ -1959,8 +1994,13 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (early) load_qv(h_next, tok0_next);
         }
     }
-    __syncthreads();   // every copy-out read of the staging tiles is done
-    if (tid == 0 && tile_next < a.ntiles) {
+    if (tile_next == -1 && tid == CBW_QUEUE_TID) lookup_blocking(ticket_next);   // not published when this tile began: wait for it now
+    named_sync(1, CBW_THREADS);   // every copy-out read of the staging tiles is done
+    if (!next_known) {
+        tile_next = sNext[0]; h_next = sNext[1]; tok0_next = sNext[2]; len_next = sNext[3];
+        if (tile_next >= 0) fetch_scalars(tile_next, h_next, tok0_next, len_next, (int)(ph ^ 1u));
+    }
+    if (tid == 0 && tile_next >= 0) {
         if (!early) {
             mbar_expect_tx(&bar_ct, CT_TX);
             load_dout(h_next, tok0_next);
@@ -1974,11 +2014,42 @@ tc_chunk_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     a_issued = a_early && ok;
     ph ^= 1u;
-    cur = nxt;
+    ticket_next = ticket_after;
+    tile_l = tile_next;
+    h = h_next;
     tok0 = tok0_next;
     len = len_next;
     }   // tile loop
     if (tid == CBW_STORE_TID) bulk_wait_all();
+    tc_fence_before();
+    named_sync(1, CBW_THREADS);
+}
+
+// Backward of the layer's second phase in one launch.  CTA b first walks the chains b, b + grid, ...
+// (reverse state recurrence), each of which publishes its finished tiles; then every CTA processes
+// chunk-local tiles from the queue until none is left.  CTAs beyond the number of chains start on the
+// queue at once, so the SMs the chains leave idle work on the tiles the chains have already finished.
+// Nothing in a chain waits for a consumer, and a consumer waits (within a bound) only for tiles whose
+// chain is running or has run: lower block indices are dispatched first.
+__global__ void __launch_bounds__(CBK_THREADS, 1)
+tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+              const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmV,
+              const __grid_constant__ CUtensorMap tmDO, const __grid_constant__ CUtensorMap tmDQ,
+              const __grid_constant__ CUtensorMap tmDK, const __grid_constant__ CUtensorMap tmDV,
+              TcChainBwdArgs ca, TcChunkBwdArgs cb, TileQueue tq, int nchains)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sm = align1024(smem_raw);
+    __shared__ uint32_t tmem_base;
+    const int warp = threadIdx.x >> 5;
+    if (warp == 0) tmem_alloc(&tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+    for (int chain = (int)blockIdx.x; chain < nchains; chain += (int)gridDim.x)
+        chain_bwd_role(tmDO, tmKt, ca, chain, sm, tb, tq);
+    if (threadIdx.x < CBW_THREADS) chunk_bwd_role(tmQ, tmK, tmKt, tmV, tmDO, tmDQ, tmDK, tmDV, cb, sm, tb, tq);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tb, 512);
@@ -2099,14 +2170,8 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
         ch.H = H; ch.tab = tab; ch.gate = a.gate; ch.dfinal_state = a.dfinal_state; ch.dinit_state = a.dinit_state;
         ch.WT = U8(t.WT); ch.P = U8(t.P); ch.Qg = U8(t.Qg); ch.dSn = U8(t.dSn); ch.ddUT = U8(t.ddUT);
         ch.status = status;
-        if (!set_smem(tc_chain_bwd_kernel, CB_SMEM)) return -1;
-        stage_mark(st, "tc_chain_bwd");
-        tc_chain_bwd_kernel<<<S * H, CBK_THREADS, CB_SMEM, st>>>(tmDO, tmKt, ch);
-        ++launches;
-    }
-    {
         TcChunkBwdArgs cb{};
-        cb.H = H; cb.ntiles = L.NTmax * H; cb.tab = tab; cb.beta = a.beta; cb.gate = a.gate; cb.scale = hy.scale; cb.d_min = hy.d_min;
+        cb.H = H; cb.ntiles = L.NTmax * H; cb.nseq = S; cb.tab = tab; cb.beta = a.beta; cb.gate = a.gate; cb.scale = hy.scale; cb.d_min = hy.d_min;
         cb.Tm = U8(t.Tm); cb.Sn = U8(t.Sn); cb.dSn = U8(t.dSn); cb.dUT = U8(t.dUT); cb.ddUT = U8(t.ddUT);
         cb.skipw = carve_p1(ws, L).skipw;
         cb.dq = static_cast<__nv_bfloat16*>(a.dq); cb.dk = static_cast<__nv_bfloat16*>(a.dk);
@@ -2117,10 +2182,17 @@ int tc_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* 
         if (!make_store_map(&tmDQ, a.dq, Ttot, H) || !make_store_map(&tmDK, a.dk, Ttot, H) ||
             !make_store_map(&tmDV, a.dv, Ttot, H))
             return -1;
-        if (!set_smem(tc_chunk_bwd_kernel, CBW_SMEM)) return -1;
-        stage_mark(st, "tc_chunk_bwd");
-        tc_chunk_bwd_kernel<<<std::min(cb.ntiles, num_sms()), CBW_THREADS, CBW_SMEM, st>>>(tmQ, tmK, tmKt, tmV, tmDO, tmDQ, tmDK,
-                                                                                tmDV, cb);
+        // tile queue between the chains and the chunk-local workers: two counters, then one slot per tile
+        const size_t qbytes = sizeof(int) * (64 + (size_t)L.NTmax * H);
+        if (cudaMemsetAsync(w + t.queue, 0, qbytes, st) != cudaSuccess) return -1;
+        TileQueue tq{};
+        tq.head = reinterpret_cast<unsigned*>(w + t.queue);
+        tq.tail = tq.head + 32;
+        tq.slots = reinterpret_cast<int*>(w + t.queue) + 64;
+        const size_t smem = std::max(CB_SMEM, CBW_SMEM);
+        if (!set_smem(tc_bwd_kernel, smem)) return -1;
+        stage_mark(st, "tc_bwd");
+        tc_bwd_kernel<<<num_sms(), CBK_THREADS, smem, st>>>(tmQ, tmK, tmKt, tmV, tmDO, tmDQ, tmDK, tmDV, ch, cb, tq, S * H);
         ++launches;
     }
     const int n1 = phase1_backward(p, hy, L, ws, a, reinterpret_cast<float*>(w + t.dktil),

@@ -32,6 +32,12 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
 
+// Invalidates a barrier so that its shared-memory word may be initialised again.
+__device__ __forceinline__ void mbar_inval(uint64_t* bar)
+{
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
 __device__ __forceinline__ void fence_mbar_init()
 {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -138,6 +144,8 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // ... and have completed
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// ... all but the N most recently committed groups of this thread have completed
+template <int N> __device__ __forceinline__ void bulk_wait_all_but() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Requests that only warm the L2 cache (no shared-memory destination, nothing to wait for).
 __device__ __forceinline__ void tma_prefetch_2d(const void* tmap, int x, int y)
@@ -168,6 +176,40 @@ __device__ __forceinline__ void prefetch_tmap(const void* tmap)
 // ---------------------------------------------------------------------------------------------
 // tensor memory
 // ---------------------------------------------------------------------------------------------
+// Generic-proxy and async-proxy accesses to global memory are ordered by this fence (a tile written by
+// bulk stores is published with a plain store; a tile found through a plain load is read by bulk copies).
+__device__ __forceinline__ void fence_proxy_async_all()
+{
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int* p, int v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Barrier over the first `nthreads` threads of the CTA (a multiple of 32), hardware barrier `id` (1..15).
+__device__ __forceinline__ void named_sync(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// ... that also ANDs a predicate over the participating threads.
+__device__ __forceinline__ bool named_sync_and(int id, int nthreads, bool pred)
+{
+    int out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %3, 0;\n\t"
+        "bar.red.and.pred p, %1, %2, q;\n\tselp.s32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(id), "r"(nthreads), "r"((int)pred)
+        : "memory");
+    return out != 0;
+}
+
 // One full warp allocates `ncols` (power of two >= 32) columns; the base address lands in *dst_smem.
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols)
 {
