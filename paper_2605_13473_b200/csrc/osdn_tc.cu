@@ -1296,7 +1296,8 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
     // bar_tok: q, k, ktil, v
     __shared__ uint64_t bar_ct, bar_tok, bar_mma[5];
     __shared__ int sNext[4];   // next tile of this CTA: {tile, head, first token, length}; tile -1: not published yet, -2: none left
-    __shared__ __align__(16) float sdB[CH], sdG[CH], sRed[CBW_THREADS / 32];
+    // per-token sums of a tile (two buffers: the sums of a tile are finished while the next tile's phase B runs)
+    __shared__ __align__(16) float sdBv[2][CH], sdGv[2][CH], sRedv[2][CBW_THREADS / 32];
     // in-chunk gate prefix G_i, gamma_i = exp(G_i), rho_i = exp(G_C - G_i): two buffers, the next tile's
     // vectors are formed during this tile's last stretch
     __shared__ __align__(16) float sGv[2][3][CH];
@@ -1305,7 +1306,7 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
     // for the load)
     __shared__ __align__(16) float sScal[2][2][CH];
     __shared__ unsigned sSkipW[2][2];
-    __shared__ float sRsum;
+    __shared__ float sRsumv[2];
     __shared__ __align__(16) float sFirstKt[KD];
 
     const int H = a.H;
@@ -1453,6 +1454,57 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
         sGv[buf][2][lane] = __expf(tot - sa);
         sGv[buf][2][lane + 32] = __expf(tot - sb);
     };
+    // The per-token sums of a tile (gate and beta gradients) are finished one tile later, while the tensor
+    // core works on the next tile's phase B: the partial terms stay in registers until then.
+    float gv[16];       // per column: gate contribution of this thread's feature
+    float rsum = 0.f;
+    bool pend = false;  // the previous tile's sums are still to be finished
+    int p_tok0 = 0, p_h = 0, p_len = 0;
+    auto reduce_sums = [&](int buf) {   // all warps: 32 features of each warp, 16 columns at once
+#pragma unroll
+        for (int step = 0; step < 4; ++step) {   // a lane keeps one half of its columns, hands the other half over
+            const int off = 16 >> step, n = 8 >> step;
+            const bool upper = (lane & off) != 0;
+#pragma unroll
+            for (int i = 0; i < n; ++i) {
+                const float gs = upper ? gv[i] : gv[i + n], gk = upper ? gv[i + n] : gv[i];
+                gv[i] = gk + __shfl_xor_sync(0xffffffffu, gs, off);
+            }
+        }
+        gv[0] += __shfl_xor_sync(0xffffffffu, gv[0], 1);   // the two lanes that ended up with the same column
+        if ((lane & 1) == 0) atomicAdd(&sdGv[buf][colq * 16 + (lane >> 1)], gv[0]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
+        if (lane == 0) atomicAdd(&sRsumv[buf], rsum);
+    };
+    // one warp: dgate_j is the suffix sum of the per-token terms (the in-chunk prefix G_i collects every
+    // g_j with j <= i); the chunk-level term goes to the last token
+    auto finish_sums = [&](int buf, int t0, int hh, int ln) {
+        float s0 = sdGv[buf][lane], s1 = sdGv[buf][lane + 32];
+        float gl = sScal[buf][0][lane] + sScal[buf][0][lane + 32], tot = lane < CBW_THREADS / 32 ? sRedv[buf][lane] : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            gl += __shfl_xor_sync(0xffffffffu, gl, o);
+            tot += __shfl_xor_sync(0xffffffffu, tot, o);
+        }
+        if (lane == 31) s1 += sRsumv[buf] + __expf(gl) * tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float u0 = __shfl_down_sync(0xffffffffu, s0, o), u1 = __shfl_down_sync(0xffffffffu, s1, o);
+            if (lane + o < 32) { s0 += u0; s1 += u1; }
+        }
+        s0 += __shfl_sync(0xffffffffu, s1, 0);
+        if (lane < ln) {
+            const size_t th = (size_t)(t0 + lane) * H + hh;
+            a.dgate[th] = s0;
+            a.dbeta[th] = sdBv[buf][lane];
+        }
+        if (lane + 32 < ln) {
+            const size_t th = (size_t)(t0 + lane + 32) * H + hh;
+            a.dgate[th] = s1;
+            a.dbeta[th] = sdBv[buf][lane + 32];
+        }
+    };
     uint32_t ph = 0;   // barrier phase parity: number of tiles processed so far, mod 2
     // queue thread: the ticket of the next tile is drawn a tile ahead and its slot is read at the top of
     // the tile, long before the value is looked at, so that neither round trip to memory is waited for
@@ -1481,6 +1533,9 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
     while (tile_l >= 0) {
     const float* sg = sScal[ph][0];      // log-gates of the chunk's tokens
     const float* sBeta = sScal[ph][1];
+    float* sdB = sdBv[ph];
+    float* sdG = sdGv[ph];
+    float* sRed = sRedv[ph];
     const float* sG = sGv[ph][0];
     const float* sGam = sGv[ph][1];
     const float* sRho = sGv[ph][2];
@@ -1488,7 +1543,7 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
         sdB[tid] = 0.f;
         sdG[tid] = 0.f;
     }
-    if (tid == 0) sRsum = 0.f;
+    if (tid == 0) sRsumv[ph] = 0.f;
     cp_async_wait_all();
     named_sync(1, CBW_THREADS);
     // the next tile's slot and the ticket of the tile after it (both values are used much later)
@@ -1605,6 +1660,7 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
         }
         mma_commit(&bar_mma[1]);
     }
+    if (pend) reduce_sums((int)(ph ^ 1u));   // the previous tile's per-token sums
     // <dS, S>_F while the tensor core works on phase B (both images share the same layout)
     {
         float p4[4] = {0.f, 0.f, 0.f, 0.f};   // independent partial sums: no chain of dependent multiply-adds
@@ -1628,6 +1684,7 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
         if (lane == 0) sRed[warp] = part;
     }
     named_sync(1, CBW_THREADS);   // every thread is done reading S / dS: phase A has finished, dU, dS and S are dead
+    if (pend && warp == 1) finish_sums((int)(ph ^ 1u), p_tok0, p_h, p_len);
     // the next tile, if the chains have published it already (asked again at the end of this tile if not);
     // the queue thread works this out while everybody waits for phase B, the others read it after the next barrier
     if (tid == CBW_QUEUE_TID) {
@@ -1719,7 +1776,6 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
     }
     // dq = scale gamma dQ1 + dq2 (both complete since phase B) while the tensor core works on phase C
     // (lane = feature f, columns = tokens; four token columns at a time)
-    float gv[16];   // per column: gate contribution of this feature
     const uint32_t boxf = (uint32_t)(f >> 6) * BOX;
     const uint32_t fc = f & 63;
     {
@@ -1837,7 +1893,7 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
     tc_fence_after();
 
     // ---- final epilogue (lane = feature f, columns = tokens): dk --------------------------------------
-    float rsum = 0.f;
+    rsum = 0.f;
     if (ok) {
         // Results are staged in shared memory as [token][feature] tiles (the operand tiles of the
         // finished products are dead by now) and written out with 16-byte stores afterwards.
@@ -1904,55 +1960,6 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
         issue_phase_a(ok && okn);
     }
     if (ok) {
-        // Sum over the 32 features of the warp for all 16 columns at once: in each of four steps a
-        // lane keeps one half of its columns and hands the other half to its partner; a last exchange
-        // joins the two lanes that end up with the same column (16 shuffles per quantity).
-#pragma unroll
-        for (int step = 0; step < 4; ++step) {
-            const int off = 16 >> step, n = 8 >> step;   // n = columns kept after this step
-            const bool upper = (lane & off) != 0;
-#pragma unroll
-            for (int i = 0; i < n; ++i) {
-                const float gs = upper ? gv[i] : gv[i + n], gk = upper ? gv[i + n] : gv[i];
-                gv[i] = gk + __shfl_xor_sync(0xffffffffu, gs, off);
-            }
-        }
-        gv[0] += __shfl_xor_sync(0xffffffffu, gv[0], 1);
-        if ((lane & 1) == 0) atomicAdd(&sdG[colq * 16 + (lane >> 1)], gv[0]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
-        if (lane == 0) atomicAdd(&sRsum, rsum);
-    }
-    named_sync(1, CBW_THREADS);   // the per-token sums are complete
-    if (ok && warp == 1) {
-        // gate and beta gradients of the chunk: dgate_j is the suffix sum of the per-token terms (the
-        // in-chunk prefix G_i collects every g_j with j <= i), by one warp while the tiles are sent off
-        float s0 = sdG[lane], s1 = sdG[lane + 32];
-        float gl = sg[lane] + sg[lane + 32], tot = lane < CBW_THREADS / 32 ? sRed[lane] : 0.f;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            gl += __shfl_xor_sync(0xffffffffu, gl, o);
-            tot += __shfl_xor_sync(0xffffffffu, tot, o);
-        }
-        if (lane == 31) s1 += sRsum + __expf(gl) * tot;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float u0 = __shfl_down_sync(0xffffffffu, s0, o), u1 = __shfl_down_sync(0xffffffffu, s1, o);
-            if (lane + o < 32) { s0 += u0; s1 += u1; }
-        }
-        s0 += __shfl_sync(0xffffffffu, s1, 0);
-        if (lane < len) {
-            const size_t th = (size_t)(tok0 + lane) * H + h;
-            a.dgate[th] = s0;
-            a.dbeta[th] = sdB[lane];
-        }
-        if (lane + 32 < len) {
-            const size_t th = (size_t)(tok0 + lane + 32) * H + h;
-            a.dgate[th] = s1;
-            a.dbeta[th] = sdB[lane + 32];
-        }
-    }
-    if (ok) {
         if (!full) {
             for (int e = tid; e < len * 16; e += CBW_THREADS) {
                 const int j = e >> 4, ch = e & 15;
@@ -2013,6 +2020,10 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
         }
     }
     a_issued = a_early && ok;
+    pend = ok;
+    p_tok0 = tok0;
+    p_h = h;
+    p_len = len;
     ph ^= 1u;
     ticket_next = ticket_after;
     tile_l = tile_next;
@@ -2020,6 +2031,11 @@ __device__ __forceinline__ void chunk_bwd_role(const CUtensorMap& tmQ, const CUt
     tok0 = tok0_next;
     len = len_next;
     }   // tile loop
+    if (pend) {   // the last tile's sums
+        reduce_sums((int)(ph ^ 1u));
+        named_sync(1, CBW_THREADS);
+        if (warp == 1) finish_sums((int)(ph ^ 1u), p_tok0, p_h, p_len);
+    }
     if (tid == CBW_STORE_TID) bulk_wait_all();
     tc_fence_before();
     named_sync(1, CBW_THREADS);
