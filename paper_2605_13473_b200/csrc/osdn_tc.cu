@@ -37,12 +37,12 @@ constexpr int KD = 128;  // K = V = 128 on this path
 constexpr uint32_t BOX = 8192;   // one [64 rows x 128 B] box
 
 // device status codes of bounded waits
-enum { ERR_QUEUE = 121, ERR_TMA = 101, ERR_MMA1 = 102, ERR_MMA2 = 103, ERR_CHAIN_TMA = 111, ERR_CHAIN_MMA1 = 112, ERR_CHAIN_MMA2 = 113 };
+enum { ERR_QUEUE = 121, ERR_READY = 122, ERR_TMA = 101, ERR_MMA1 = 102, ERR_MMA2 = 103, ERR_CHAIN_TMA = 111, ERR_CHAIN_MMA1 = 112, ERR_CHAIN_MMA2 = 113 };
 
 constexpr uint32_t REC_BYTES = 49152;   // stride of the Tb | W^T | P' | Qg record of a tile
 
 struct TcLayout {
-    size_t ktil, WT, Tb, Tm, P, Qg, Sn, dUT, ddUT, dSn, dktil, dkread, queue, total;
+    size_t ktil, WT, Tb, Tm, P, Qg, Sn, dUT, ready, ddUT, dSn, dktil, dkread, queue, total;
 };
 
 TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
@@ -64,6 +64,7 @@ TcLayout make_tc_layout(const osdn_params& p, const WsLayout& L, bool need_bwd)
     t.Tm = take(NT * H * 8192);
     t.Sn = take(NT * H * 32768);
     t.dUT = take(NT * H * 16384);
+    t.ready = take(sizeof(int) * (64 + NT * H));   // ticket counter, then one flag per tile
     if (need_bwd) {
         t.ddUT = take(NT * H * 16384);
         t.dSn = take(NT * H * 32768);
@@ -199,7 +200,7 @@ __device__ __forceinline__ void block16_store_ld(float* C, const float (&acc)[2]
     }
 }
 
-__device__ __forceinline__ void ut_inverse_64_inplace(float* sA, int tid)
+template <typename Sync> __device__ __forceinline__ void ut_inverse_64_inplace(float* sA, int tid, Sync sync)
 {
     const int warp = tid >> 5, lane = tid & 31;
     {
@@ -215,13 +216,13 @@ __device__ __forceinline__ void ut_inverse_64_inplace(float* sA, int tid)
                 for (int i = j + 1; i < 16; ++i) x[i] = fmaf(-Ab[i * LCF + j], x[j], x[i]);
             }
         }
-        __syncthreads();   // every column has read the block before anyone overwrites it
+        sync();   // every column has read the block before anyone overwrites it
         if (tid < CH) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) Ab[i * LCF + col] = x[i];
         }
     }
-    __syncthreads();
+    sync();
     for (int b = 1; b < 4; ++b) {
         // warp c < b: X = sum_m A_bm T_mc, parked in block (c, b); then T_bc = -T_bb X
         float acc2[2][4] = {};
@@ -235,9 +236,9 @@ __device__ __forceinline__ void ut_inverse_64_inplace(float* sA, int tid)
             __syncwarp();
             block16_mma_ld<LCF>(acc2, sA + (16 * b) * LCF + 16 * b, X, lane);
         }
-        __syncthreads();   // row b of A has been read by every warp that needs it
+        sync();   // row b of A has been read by every warp that needs it
         if (warp < b) block16_store_ld<LCF>(sA + (16 * b) * LCF + 16 * warp, acc2, -1.f, lane);
-        __syncthreads();
+        sync();
     }
 }
 
@@ -246,6 +247,7 @@ __device__ __forceinline__ void ut_inverse_64_inplace(float* sA, int tid)
 // ---------------------------------------------------------------------------------------------
 struct TcChunkArgs {
     int H;
+    int* ready;   // merged forward launch: per (chunk, head) tile, set to 1 once the tile's images are in global memory
     Table tab;
     const float *beta, *gate;
     float scale;
@@ -259,35 +261,42 @@ struct TcChunkArgs {
 constexpr int CL_THREADS = 256;
 constexpr size_t CL_SMEM = 32768 + CH * LCF * 4 + 1024;
 
-__global__ void __launch_bounds__(CL_THREADS, 4)
-tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
-                    const __grid_constant__ CUtensorMap tmKt, TcChunkArgs a)
+// Small per-group state of the chunk-local forward that lives in shared memory.
+struct ClGroupShared {
+    uint64_t bar_tma, bar_mma1, bar_mma2;
+    int ticket;
+    int pad;
+    float sG[CH], sBeta[CH];
+};
+
+// One (chunk, head) tile by a group of CL_THREADS threads (local index `tid`) that synchronise on hardware
+// barrier `bar_id`; `sm`: CL_SMEM - 1024 bytes, 1024-byte aligned; `tb`: 128 tensor-memory columns;
+// `ph`: parity of the group's three barriers (they complete once per tile).
+__device__ __forceinline__ void chunk_fwd_tile(const CUtensorMap& tmK, const CUtensorMap& tmQ, const CUtensorMap& tmKt,
+                                               const TcChunkArgs& a, int c, int h, uint8_t* sm, ClGroupShared& gs,
+                                               uint32_t tb, int tid, int bar_id, uint32_t ph, int* publish)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* sm = align1024(smem_raw);
+    auto sync = [&]() { named_sync(bar_id, CL_THREADS); };
+    uint64_t& bar_tma = gs.bar_tma;
+    uint64_t& bar_mma1 = gs.bar_mma1;
+    uint64_t& bar_mma2 = gs.bar_mma2;
+    float* sG = gs.sG;
+    float* sBeta = gs.sBeta;
     uint8_t* sKQ = sm;                 // per k-half h: [K rows 0-63 | Q rows 64-127], 16 KB each
     uint8_t* sKt = sKQ + 32768;        // per k-half: 8 KB
     // A, then T (fp32, in place) take over the space of Ktil once the first product has consumed it;
     // the T diag(beta gamma) operand image takes over the first Q box once Qg has been written.
     float* sA = reinterpret_cast<float*>(sKt);
     uint8_t* sTb = sKQ + BOX;          // K-major [i][j]
-    __shared__ uint64_t bar_tma, bar_mma1, bar_mma2;
-    __shared__ uint32_t tmem_base;
-    __shared__ __align__(16) float sG[CH], sBeta[CH];
-
-    const int c = blockIdx.x, h = blockIdx.y, H = a.H;
+    const int H = a.H;
     const int len = a.tab.chunk_len(c);
     if (len == 0) return;
     const int tok0 = a.tab.chunk_tok0(c);
     const size_t tile = (size_t)c * H + h;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int warp = tid >> 5, lane = tid & 31;
     const int quad = warp & 3, half = warp >> 2;
 
     if (tid == 0) {
-        mbar_init(&bar_tma, 1);
-        mbar_init(&bar_mma1, 1);
-        mbar_init(&bar_mma2, 1);
-        fence_mbar_init();
         mbar_expect_tx(&bar_tma, 6 * BOX);
         for (int hf = 0; hf < 2; ++hf) {
             tma_load_2d(sKQ + hf * 16384, &tmK, h * KD + hf * 64, tok0, &bar_tma);
@@ -295,7 +304,6 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             tma_load_2d(sKt + hf * BOX, &tmKt, h * KD + hf * 64, tok0, &bar_tma);
         }
     }
-    if (warp == 1) tmem_alloc(&tmem_base, 128);
     if (warp == 2) {   // per-token scalars and the in-chunk gate prefix G_i
         const bool in0 = lane < len, in1 = lane + 32 < len;
         float sa = in0 ? a.gate[(size_t)(tok0 + lane) * H + h] : 0.f;
@@ -311,12 +319,15 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         sG[lane] = sa;
         sG[lane + 32] = sb;
     }
+    // The group's previous tile is published here: by now its stores have drained, so the fence is cheap,
+    // and the barrier that follows is needed anyway.
+    if (publish) __threadfence();
     tc_fence_before();
-    __syncthreads();
+    sync();
     tc_fence_after();
-    const uint32_t tb = tmem_base;
+    if (publish && tid == 0) st_release_gpu(publish, 1);
 
-    bool ok = mbar_wait(&bar_tma, 0, a.status, ERR_TMA);
+    bool ok = mbar_wait(&bar_tma, ph, a.status, ERR_TMA);
     if (len < CH) {
         for (int hf = 0; hf < 2; ++hf) {
             zero_tail_rows(sKQ + hf * 16384, len, tid, CL_THREADS);
@@ -324,7 +335,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             zero_tail_rows(sKt + hf * BOX, len, tid, CL_THREADS);
         }
         fence_proxy_async();
-        __syncthreads();
+        sync();
     }
 
     // ---- D1[128 x 64] = [K;Q] Ktil^T ---------------------------------------------------------
@@ -353,7 +364,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
         *reinterpret_cast<uint4*>(a.Qg + tile * REC_BYTES + hf * BOX + off) = make_uint4(o[0], o[1], o[2], o[3]);
     }
-    ok = ok && mbar_wait(&bar_mma1, 0, a.status, ERR_MMA1);
+    ok = ok && mbar_wait(&bar_mma1, ph, a.status, ERR_MMA1);
     tc_fence_after();
     if (ok) {
         const int L = quad * 32 + lane;
@@ -416,10 +427,10 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             }
         }
     }
-    __syncthreads();
+    sync();
 
     // ---- T = (I + A)^-1, blocked, in place ---------------------------------------------------------
-    ut_inverse_64_inplace(sA, tid);
+    ut_inverse_64_inplace(sA, tid, sync);
 
     // ---- operand images: Tbg (shared), Tb and T (HBM) -----------------------------------------
     for (int e = tid; e < CH * 8; e += CL_THREADS) {
@@ -447,7 +458,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    sync();
 
     // ---- D2[128 x 64] = K^T Tbg^T  (W^T) -----------------------------------------------------
     if (tid == 0 && ok) {
@@ -458,7 +469,7 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         for (int s = 0; s < 4; ++s) mma_ss(tb + 64, desc_advance(da0, 2048 * s), desc_advance(db0, 32 * s), idesc, s > 0);
         mma_commit(&bar_mma2);
     }
-    ok = ok && mbar_wait(&bar_mma2, 0, a.status, ERR_MMA2);
+    ok = ok && mbar_wait(&bar_mma2, ph, a.status, ERR_MMA2);
     tc_fence_after();
     if (ok) {
         const int k = quad * 32 + lane;
@@ -481,8 +492,32 @@ tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             }
     }
     tc_fence_before();
+    sync();
+}
+
+// Stand-alone launch: one tile per CTA, four CTAs per SM.
+__global__ void __launch_bounds__(CL_THREADS, 4)
+tc_chunk_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
+                    const __grid_constant__ CUtensorMap tmKt, TcChunkArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ ClGroupShared gs;
+    __shared__ uint32_t tmem_base;
+    const int tid = threadIdx.x;
+    if (a.tab.chunk_len(blockIdx.x) == 0) return;
+    if (tid == 0) {
+        mbar_init(&gs.bar_tma, 1);
+        mbar_init(&gs.bar_mma1, 1);
+        mbar_init(&gs.bar_mma2, 1);
+        fence_mbar_init();
+    }
+    if ((tid >> 5) == 1) tmem_alloc(&tmem_base, 128);
+    tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tb, 128);
+    tc_fence_after();
+    chunk_fwd_tile(tmK, tmQ, tmKt, a, blockIdx.x, blockIdx.y, align1024(smem_raw), gs, tmem_base, tid, 1, 0u, nullptr);
+    __syncthreads();
+    if ((tid >> 5) == 1) tmem_dealloc(tmem_base, 128);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -499,6 +534,7 @@ struct TcChainArgs {
     float scale;
     int save;
     int* status;
+    const int* ready;   // nullable: per (chunk, head) tile, nonzero once the chunk-local pass has written it
 };
 
 constexpr uint32_t STAGE_BYTES = 8192 + 16384 + 8192 + 3 * 16384;   // Tb, WT, P, Qg, V, Ktil = 81920
@@ -542,21 +578,21 @@ constexpr int CFW_EPI_WARPS = 16, CFW_OUT_WARPS = 4;
 constexpr int CFW_OUT_WARP0 = 16, CFW_MMA_WARP = 20, CFW_TMA_WARP = 21;
 constexpr int CFW_THREADS = 22 * 32;
 
-__global__ void __launch_bounds__(CFW_THREADS, 1)
-tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
+// One chain by the first CFW_THREADS threads of the CTA (all threads of the CTA must call: the function
+// synchronises the CTA).  `sm`: CF_SMEM - 1024 bytes, 1024-byte aligned; `tb`: 512 tensor-memory columns.
+// With `a.ready` set, the loads of a chunk wait until the chunk-local pass has published it.
+__device__ __forceinline__ void chain_fwd_role(const CUtensorMap& tmV, const CUtensorMap& tmKt, const TcChainArgs& a,
+                                               int chain, uint8_t* sm, uint32_t tb)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* sm = align1024(smem_raw);
     uint8_t* sStage = sm;                       // 2 stages
     uint8_t* sS = sm + 2 * STAGE_BYTES;         // S as bf16, K-major: 2 k-halves x [128 rows x 128 B]
     uint8_t* sDU1 = sS + 32768;                 // dU^T, K-major [v][i]
     uint8_t* sDU2 = sDU1 + 16384;               // (rho dU)^T
     __shared__ uint64_t bar_full[2], bar_empty[2], bar_s_ready, bar_du_done, bar_du_ready, bar_s_done;
     __shared__ uint64_t bar_o_done[2], bar_o_free[2];
-    __shared__ uint32_t tmem_base;
     __shared__ float sRho[2][CH], sGC[2];              // slot = chunk % 2
 
-    const int chain = blockIdx.x, H = a.H;
+    const int H = a.H;
     const int s = chain / H, h = chain % H;
     const int c0 = a.tab.seq_chunk0(s), c1 = a.tab.seq_chunk0(s + 1);
     const int seq_t0 = a.tab.seq_tok0(s), seq_len = a.tab.seq_len(s);
@@ -570,6 +606,9 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             for (int x = 0; x < 32; ++x) fin[x] = ini ? ini[x] : 0.f;
         return;
     }
+    uint64_t* const all_bars[] = {&bar_full[0], &bar_full[1], &bar_empty[0], &bar_empty[1], &bar_s_ready, &bar_du_done,
+                                  &bar_du_ready, &bar_s_done, &bar_o_done[0], &bar_o_done[1], &bar_o_free[0],
+                                  &bar_o_free[1]};
     const int nchunks = c1 - c0;
     auto chunk_tok0 = [&](int n) { return seq_t0 + n * CH; };
     auto chunk_len = [&](int n) { return min(CH, seq_len - n * CH); };
@@ -589,14 +628,14 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         mbar_init(&bar_o_free[1], CFW_OUT_WARPS);
         fence_mbar_init();
     }
-    if (warp == 0) tmem_alloc(&tmem_base, 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tb = tmem_base;
     const uint32_t tS = tb, tDU = tb + 128, tO = tb + 192;   // O^T: two buffers of 64 columns
 
-    if (warp == CFW_TMA_WARP) {
+    if (warp >= CFW_THREADS / 32) {
+        // not part of the chain
+    } else if (warp == CFW_TMA_WARP) {
         // ------------------------------------------------------------------ producer
         // A stage is complete when its copies have landed (transaction count, first arrival) and the
         // gate vectors of the chunk are written (second arrival).  The gates are read a chunk ahead.
@@ -615,6 +654,21 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             if (n + 1 < nchunks) load_gates(n + 1, ga_next, gb_next);
             if (n >= 2) ok = mbar_wait(&bar_empty[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_TMA);
             if (!ok) break;
+            if (a.ready) {   // the chunk-local pass runs beside the chains: wait until the record is written
+                const int* flag = a.ready + (size_t)(c0 + n) * H + h;
+                const long long t0 = clock64();
+                bool seen = false;
+                while (!(seen = ld_acquire_gpu(flag) != 0)) {
+                    if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+                    __nanosleep(64);
+                }
+                if (!seen) {
+                    if (lane == 0) atomicCAS(a.status, 0, ERR_READY);
+                    ok = false;
+                    break;
+                }
+                fence_proxy_async_all();
+            }
             if (lane == 0) {
                 const size_t tile = (size_t)(c0 + n) * H + h;
                 uint8_t* d = sStage + st * STAGE_BYTES;
@@ -733,7 +787,7 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             // Warm L2 with the operands of chunk n + 2 (the stage copies can only run one chunk ahead).
             if (lane == 0 && n + 2 < nchunks) {
                 const int t2 = chunk_tok0(n + 2);
-                if (ow == 0) bulk_prefetch(a.Tb + ((size_t)(c0 + n + 2) * H + h) * REC_BYTES, REC_BYTES);
+                if (ow == 0 && !a.ready) bulk_prefetch(a.Tb + ((size_t)(c0 + n + 2) * H + h) * REC_BYTES, REC_BYTES);
                 if (ow == 1)
                     for (int hf = 0; hf < 2; ++hf) tma_prefetch_2d(&tmV, h * KD + hf * 64, t2);
                 if (ow == 2)
@@ -902,7 +956,124 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tb, 512);
+    if (tid == 0)
+        for (uint64_t* b : all_bars) mbar_inval(b);
+    __syncthreads();
+}
+
+// Stand-alone launch: one chain per CTA.
+__global__ void __launch_bounds__(CFW_THREADS, 1)
+tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKt, TcChainArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_base;
+    if (threadIdx.x < 32) tmem_alloc(&tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    chain_fwd_role(tmV, tmKt, a, blockIdx.x, align1024(smem_raw), tmem_base);
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_dealloc(tmem_base, 512);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Forward of phase 2 in one launch.  Every CTA starts as three groups that take (chunk, head) tiles of
+// the chunk-local pass from a ticket counter, chunk position by chunk position across the chains, and
+// publish each finished tile with a flag.  Once `switch_at` tickets are out, the first `nchains` CTAs
+// turn into the state chains, whose loads wait for those flags; the other CTAs keep producing, and a CTA
+// whose chain is finished joins them again.  No worker ever waits, so the chains always make progress.
+// ---------------------------------------------------------------------------------------------
+struct FwdSched {
+    int* tickets;     // zero at launch
+    int ntickets;     // chunk positions x chains
+    int nchains;
+    int nchunks;      // chunk positions per chain (sequences of equal length)
+    int switch_at;
+};
+constexpr int FWD_GROUPS = 4;
+constexpr int FWD_THREADS = FWD_GROUPS * CL_THREADS;
+constexpr uint32_t FWD_GROUP_SMEM = (uint32_t)CL_SMEM - 1024;
+static_assert(FWD_GROUPS * FWD_GROUP_SMEM + FWD_GROUPS * sizeof(ClGroupShared) <= CF_SMEM - 1024, "worker groups fit");
+static_assert(FWD_THREADS >= CFW_THREADS, "the chain fits into the CTA");
+
+__device__ __forceinline__ void chunk_fwd_workers(const CUtensorMap& tmK, const CUtensorMap& tmQ,
+                                                  const CUtensorMap& tmKt, const TcChunkArgs& cl, const FwdSched& sc,
+                                                  int limit, uint8_t* sm, uint32_t tb)
+{
+    const int tid = threadIdx.x, g = tid / CL_THREADS, ltid = tid % CL_THREADS;
+    ClGroupShared& gs = reinterpret_cast<ClGroupShared*>(sm + FWD_GROUPS * FWD_GROUP_SMEM)[g];
+    auto gsync = [&]() { named_sync(1 + g, CL_THREADS); };
+    if (ltid == 0) {
+        mbar_init(&gs.bar_tma, 1);
+        mbar_init(&gs.bar_mma1, 1);
+        mbar_init(&gs.bar_mma2, 1);
+        fence_mbar_init();
+    }
+    gsync();
+    // The group's leader draws tickets one tile ahead, so the round trip of the atomic is hidden by the
+    // tile in progress.  A ticket that has been drawn is always worked off before the group stops.
+    auto draw = [&]() {
+        int t = -1;
+        if (*reinterpret_cast<volatile int*>(sc.tickets) < limit) {
+            t = atomicAdd(sc.tickets, 1);
+            if (t >= sc.ntickets) t = -1;
+        }
+        return t;
+    };
+    uint32_t ph = 0;
+    int* publish = nullptr;   // flag of the tile the group finished last
+    int next = ltid == 0 ? draw() : -1;
+    while (true) {
+        if (ltid == 0) gs.ticket = next;
+        gsync();
+        const int t = gs.ticket;
+        if (t < 0) break;
+        if (ltid == 0) next = draw();
+        const int n = t / sc.nchains, chain = t - n * sc.nchains;
+        const int s = chain / cl.H, h = chain - s * cl.H;
+        const int c = s * sc.nchunks + n;
+        chunk_fwd_tile(tmK, tmQ, tmKt, cl, c, h, sm + g * FWD_GROUP_SMEM, gs, tb + g * 128, ltid, 1 + g, ph, publish);
+        publish = cl.ready + (size_t)c * cl.H + h;
+        ph ^= 1;
+    }
+    if (publish) {
+        __threadfence();
+        gsync();
+        if (ltid == 0) st_release_gpu(publish, 1);
+    }
+    gsync();
+    if (ltid == 0) {
+        mbar_inval(&gs.bar_tma);
+        mbar_inval(&gs.bar_mma1);
+        mbar_inval(&gs.bar_mma2);
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(FWD_THREADS, 1)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
+              const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmV, TcChunkArgs cl,
+              TcChainArgs ch, FwdSched sc)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sm = align1024(smem_raw);
+    __shared__ uint32_t tmem_base;
+    if (threadIdx.x < 32) tmem_alloc(&tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_base;
+    const bool chain_cta = (int)blockIdx.x < sc.nchains;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {   // one copy of the worker code: it has to stay in the instruction cache
+        chunk_fwd_workers(tmK, tmQ, tmKt, cl, sc, chain_cta && pass == 0 ? sc.switch_at : sc.ntickets, sm, tb);
+        if (!chain_cta || pass == 1) break;
+        chain_fwd_role(tmV, tmKt, ch, blockIdx.x, sm, tb);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_dealloc(tb, 512);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -2102,6 +2273,11 @@ template <typename F> bool set_smem(F* kernel, size_t bytes)
 
 }  // namespace
 
+// Merged forward launch: SMs that must be left over to feed the chains, and the cost of one chain step in
+// units of the time one SM needs for a tile of the chunk-local pass (measured: 0.6 to 0.75 are equally good).
+constexpr int FWD_MIN_FEEDERS = 32;
+constexpr double FWD_STEP_OVER_TILE = 0.65;
+
 int launch_wait_timeout_selftest(int* status, long long limit_cycles, int code, cudaStream_t st)
 {
     wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status, limit_cycles, code);
@@ -2134,25 +2310,45 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
     if (!make_token_map(&tmK, a.k, Ttot, H) || !make_token_map(&tmQ, a.q, Ttot, H) ||
         !make_token_map(&tmKt, w + t.ktil, Ttot, H) || !make_token_map(&tmV, a.v, Ttot, H))
         return -1;
-    {
-        TcChunkArgs ca{};
-        ca.H = H; ca.tab = tab; ca.beta = a.beta; ca.gate = a.gate; ca.scale = hy.scale;
-        ca.WT = reinterpret_cast<uint8_t*>(w + t.WT); ca.Tb = reinterpret_cast<uint8_t*>(w + t.Tb);
-        ca.Tm = reinterpret_cast<uint8_t*>(w + t.Tm); ca.P = reinterpret_cast<uint8_t*>(w + t.P);
-        ca.Qg = reinterpret_cast<uint8_t*>(w + t.Qg); ca.save = save ? 1 : 0; ca.status = status;
+    TcChunkArgs ca{};
+    ca.H = H; ca.tab = tab; ca.beta = a.beta; ca.gate = a.gate; ca.scale = hy.scale;
+    ca.WT = reinterpret_cast<uint8_t*>(w + t.WT); ca.Tb = reinterpret_cast<uint8_t*>(w + t.Tb);
+    ca.Tm = reinterpret_cast<uint8_t*>(w + t.Tm); ca.P = reinterpret_cast<uint8_t*>(w + t.P);
+    ca.Qg = reinterpret_cast<uint8_t*>(w + t.Qg); ca.save = save ? 1 : 0; ca.status = status;
+    TcChainArgs ch{};
+    ch.H = H; ch.tab = tab; ch.gate = a.gate; ch.init_state = a.init_state;
+    ch.out = static_cast<__nv_bfloat16*>(a.out); ch.final_state = a.final_state;
+    ch.WT = reinterpret_cast<uint8_t*>(w + t.WT); ch.Tb = reinterpret_cast<uint8_t*>(w + t.Tb);
+    ch.P = reinterpret_cast<uint8_t*>(w + t.P); ch.Sn = reinterpret_cast<uint8_t*>(w + t.Sn);
+    ch.dUT = reinterpret_cast<uint8_t*>(w + t.dUT); ch.scale = hy.scale; ch.save = save ? 1 : 0;
+    ch.status = status;
+    // One launch for both passes when the batch is dense (equal chunk counts give the tile order the
+    // chains want) and enough SMs are left over to feed the chains.
+    const int grid = num_sms(), nchains = S * H;
+    const int nchunks = p.nseq > 0 ? 0 : (p.T + CH - 1) / CH;
+    if (p.nseq == 0 && nchunks > 0 && nchains + FWD_MIN_FEEDERS <= grid) {
+        const size_t rbytes = sizeof(int) * (64 + (size_t)L.NTmax * H);
+        if (cudaMemsetAsync(w + t.ready, 0, rbytes, st) != cudaSuccess) return -1;
+        FwdSched sc{};
+        sc.tickets = reinterpret_cast<int*>(w + t.ready);
+        sc.nchains = nchains;
+        sc.nchunks = nchunks;
+        sc.ntickets = nchunks * nchains;
+        // The chains start once the feeders alone can keep up with them to the end: a chain step costs
+        // about FWD_STEP_OVER_TILE of the time one SM needs for a tile.
+        const double fed = (double)(grid - nchains) * nchunks * FWD_STEP_OVER_TILE;
+        sc.switch_at = (int)std::max(0.0, (double)sc.ntickets - fed);
+        ca.ready = sc.tickets + 64;
+        ch.ready = sc.tickets + 64;
+        if (!set_smem(tc_fwd_kernel, CF_SMEM)) return -1;
+        stage_mark(st, "tc_fwd");
+        tc_fwd_kernel<<<grid, FWD_THREADS, CF_SMEM, st>>>(tmK, tmQ, tmKt, tmV, ca, ch, sc);
+        ++launches;
+    } else {
         if (!set_smem(tc_chunk_fwd_kernel, CL_SMEM)) return -1;
         stage_mark(st, "tc_chunk_fwd");
         tc_chunk_fwd_kernel<<<dim3(L.NTmax, H), CL_THREADS, CL_SMEM, st>>>(tmK, tmQ, tmKt, ca);
         ++launches;
-    }
-    {
-        TcChainArgs ch{};
-        ch.H = H; ch.tab = tab; ch.gate = a.gate; ch.init_state = a.init_state;
-        ch.out = static_cast<__nv_bfloat16*>(a.out); ch.final_state = a.final_state;
-        ch.WT = reinterpret_cast<uint8_t*>(w + t.WT); ch.Tb = reinterpret_cast<uint8_t*>(w + t.Tb);
-        ch.P = reinterpret_cast<uint8_t*>(w + t.P); ch.Sn = reinterpret_cast<uint8_t*>(w + t.Sn);
-        ch.dUT = reinterpret_cast<uint8_t*>(w + t.dUT); ch.scale = hy.scale; ch.save = save ? 1 : 0;
-        ch.status = status;
         if (!set_smem(tc_chain_fwd_kernel, CF_SMEM)) return -1;
         stage_mark(st, "tc_chain_fwd");
         tc_chain_fwd_kernel<<<S * H, CFW_THREADS, CF_SMEM, st>>>(tmV, tmKt, ch);
