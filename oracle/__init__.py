@@ -26,7 +26,8 @@ _lib = None
 class _Hyper(ctypes.Structure):
     _fields_ = [("eta", ctypes.c_double), ("d_min", ctypes.c_double), ("d_max", ctypes.c_double),
                 ("eps", ctypes.c_double), ("scale", ctypes.c_double),
-                ("beta_aware", ctypes.c_int), ("apf_mode", ctypes.c_int), ("clamp", ctypes.c_int)]
+                ("beta_aware", ctypes.c_int), ("apf_mode", ctypes.c_int), ("clamp", ctypes.c_int),
+                ("channel_gate", ctypes.c_int)]
 
 
 def build(force: bool = False) -> str:
@@ -51,7 +52,14 @@ def threads() -> int:
 def _hyper(hy, K: int) -> _Hyper:
     scale = float(hy.scale) if hy.scale and hy.scale > 0 else float(K) ** -0.5
     return _Hyper(float(hy.eta), float(hy.d_min), float(hy.d_max), float(hy.eps), scale,
-                  int(hy.beta_aware), int(hy.apf_mode), int(hy.clamp))
+                  int(hy.beta_aware), int(hy.apf_mode), int(hy.clamp), int(_channel_gate(hy)))
+
+
+def _channel_gate(hy) -> bool:
+    """OSKDA: `gate` holds one log-gate per key channel, [T, H, K]; the aliased retention mode is undefined."""
+    cg = bool(getattr(hy, "channel_gate", False))
+    assert not (cg and hy.apf_mode == 1), "the preconditioner's retention is separate from a channel gate"
+    return cg
 
 
 def _f64(x) -> Optional[np.ndarray]:
@@ -81,6 +89,7 @@ def fwd(hy, seq_lens, q, k, v, beta, gate, log_ret=None, init_state=None, precon
     cu = _cu(seq_lens)
     nseq = len(seq_lens)
     assert cu[-1] == T
+    assert gate.shape == ((T, H, K) if _channel_gate(hy) else (T, H))
     if hy.apf_mode == 2:
         assert log_ret is not None and log_ret.shape == (T, H)
     if hy.apf_mode == 3:
@@ -116,6 +125,7 @@ def residual_ratio(hy, seq_lens, k, v, beta, gate, log_ret=None, init_state=None
     log_ret, init_state, precond_in = map(_f64, (log_ret, init_state, precond_in))
     T, H, K = k.shape
     V = v.shape[-1]
+    assert not _channel_gate(hy)
     cu = _cu(seq_lens)
     out = np.zeros((T, H))
     hp = _hyper(hy, K)
@@ -153,7 +163,8 @@ def bwd(hy, seq_lens, q, k, v, beta, gate, dout, log_ret=None, init_state=None, 
     cu = _cu(seq_lens)
     nseq = len(seq_lens)
     dq, dk, dv = np.zeros((T, H, K)), np.zeros((T, H, K)), np.zeros((T, H, V))
-    dbeta, dgate = np.zeros((T, H)), np.zeros((T, H))
+    assert gate.shape == ((T, H, K) if _channel_gate(hy) else (T, H))
+    dbeta, dgate = np.zeros((T, H)), np.zeros((T, H, K) if _channel_gate(hy) else (T, H))
     dlr = np.zeros((T, H, K)) if hy.apf_mode == 3 else np.zeros((T, H))
     dS0, dd0 = np.zeros((nseq, H, V, K)), np.zeros((nseq, H, K))
     hp = _hyper(hy, K)

@@ -27,6 +27,16 @@
  *       S_t  = Sbar + beta_t u ktil_t^T            write with the scaled key
  *       o_t  = scale * S_t q_t                     read after the write
  *
+ *   channel gate (OSKDA, backbone-extension appendix "Kimi Delta Attention with
+ *   Online Scaling"): the scalar exp(g_t) becomes one gate per key channel,
+ *       Sbar = S_{t-1} Diag(alpha_t),   alpha_t = exp(g_t) in (0,1]^K,
+ *   everything else unchanged.  The paper writes the state as K x V with the
+ *   gate, the read key and the scaled write key on the left,
+ *       S'_t = (I - beta ktil k^T) Diag(alpha_t) S'_{t-1} + beta ktil v^T,  o = S'^T q;
+ *   with S' = S^T these are the lines above (S is kept V x K here as well).  The
+ *   preconditioner's retention stays separate from the channel gate, so the
+ *   aliased mode (apf_mode 1) is not defined for it.
+ *
  * The backward pass is the hand-derived adjoint of exactly these lines
  * (Section 3.5 only states its factorisation); it is validated against
  * central finite differences in the tests.
@@ -37,6 +47,11 @@
  * form of the preconditioner recurrence, the K=V=1 alternating example, the
  * WY product identity and the chunkwise form (an independent numpy program),
  * APF with unit retention, split-sequence carry, finite differences.
+ * Channel gate (tests/test_oracle_oskda.py): equal gates in every channel give
+ * the scalar-gate result, an independent numpy program of the paper's chunk
+ * equations (cumulative channel decays, suffix-gated write key) gives the same
+ * outputs and state, the K x V left-multiplied form written out in numpy gives
+ * the transpose, finite differences for the gradients.
  * Absolute output values for random inputs have no printed example in the
  * paper: beyond those pins they are "parity unpinned".
  *
@@ -54,6 +69,7 @@
 typedef struct {
     double eta, d_min, d_max, eps, scale;
     int beta_aware, apf_mode, clamp;
+    int channel_gate;   /* gate is [T,H,K]: one log-gate per key channel (OSKDA) */
 } oracle_hyper;
 
 int osdn_oracle_threads(void)
@@ -70,6 +86,9 @@ int osdn_oracle_threads(void)
  * affine form of the update) one per coordinate. */
 #define LRET_S(hp, lr, th) (((lr) && (hp)->apf_mode != 3) ? (lr)[th] : 0.0)
 #define LRET_V(hp, lr, th, K) (((lr) && (hp)->apf_mode == 3) ? (lr) + (th) * (size_t)(K) : (const double *)0)
+/* Gate inputs of token-head th: one log-gate, or K of them with a channel gate. */
+#define GATE_S(hp, g, th) ((hp)->channel_gate ? 0.0 : (g)[th])
+#define GATE_V(hp, g, th, K) ((hp)->channel_gate ? (g) + (th) * (size_t)(K) : (const double *)0)
 
 /* One phase-1 step.  Reads d (length K) and overwrites it with d_{t+1}.
  * Optionally reports ktil, the scalar c and the pass-through mask.
@@ -114,17 +133,16 @@ static void phase1_step(const oracle_hyper *hp, int K, const double *k, double b
     if (raw_norm_above_eps) *raw_norm_above_eps = sumk > hp->eps;
 }
 
-/* One phase-2 step on S (V x K, row-major).  u_out (length V) receives the
+/* One phase-2 step on S (V x K, row-major); gvec (nullable): K channel log-gates in place of g.  u_out (length V) receives the
  * post-gate residual v - Sbar k; S is overwritten by S_t. */
 static void phase2_step(int K, int V, const double *k, const double *ktil, const double *v,
-                        double beta, double g, double *S, double *u_out)
+                        double beta, double g, const double *gvec, double *S, double *u_out)
 {
-    double alpha = exp(g);
     for (int r = 0; r < V; ++r) {
         double *row = S + (size_t)r * K;
         double acc = 0.0;
         for (int i = 0; i < K; ++i) {
-            row[i] *= alpha;
+            row[i] *= exp(gvec ? gvec[i] : g);
             acc += row[i] * k[i];
         }
         double u = v[r] - acc;
@@ -160,10 +178,10 @@ void osdn_oracle_fwd(int nseq, const int *cu, int H, int K, int V, const oracle_
             size_t th = (size_t)t * H + h;
             const double *kt = k + th * K, *qt = q + th * K, *vt = v + th * V;
             if (d_traj_out) memcpy(d_traj_out + th * K, d, sizeof(double) * K);
-            phase1_step(hp, K, kt, beta[th], gate[th], LRET_S(hp, log_ret, th), LRET_V(hp, log_ret, th, K), d, ktil,
+            phase1_step(hp, K, kt, beta[th], GATE_S(hp, gate, th), LRET_S(hp, log_ret, th), LRET_V(hp, log_ret, th, K), d, ktil,
                         0, 0, 0, 0, 0, mask_out ? mask_out + th * K : 0, margin_out ? margin_out + th * K : 0);
             if (ktil_out) memcpy(ktil_out + th * K, ktil, sizeof(double) * K);
-            phase2_step(K, V, kt, ktil, vt, beta[th], gate[th], S, 0);
+            phase2_step(K, V, kt, ktil, vt, beta[th], GATE_S(hp, gate, th), GATE_V(hp, gate, th, K), S, 0);
             for (int r = 0; r < V; ++r) {
                 double acc = 0.0;
                 for (int i = 0; i < K; ++i) acc += S[(size_t)r * K + i] * qt[i];
@@ -206,7 +224,7 @@ void osdn_oracle_residual_ratio(int nseq, const int *cu, int H, int K, int V, co
             const double *kt = k + th * K, *vt = v + th * V;
             phase1_step(hp, K, kt, beta[th], gate[th], LRET_S(hp, log_ret, th), LRET_V(hp, log_ret, th, K), d, ktil,
                         0, 0, 0, 0, 0, 0, 0);
-            phase2_step(K, V, kt, ktil, vt, beta[th], gate[th], S, u);   /* u = v - Sbar k */
+            phase2_step(K, V, kt, ktil, vt, beta[th], gate[th], 0, S, u);   /* u = v - Sbar k */
             double before = 0.0, after = 0.0;
             for (int r = 0; r < V; ++r) {
                 double acc = 0.0;
@@ -311,9 +329,10 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
             int a0 = t0 + sg * SEG, a1 = a0 + SEG < t1 ? a0 + SEG : t1;
             for (int t = a0; t < a1; ++t) {
                 size_t th = (size_t)t * H + h;
-                phase1_step(hp, K, k + th * K, beta[th], gate[th], LRET_S(hp, log_ret, th),
+                phase1_step(hp, K, k + th * K, beta[th], GATE_S(hp, gate, th), LRET_S(hp, log_ret, th),
                             LRET_V(hp, log_ret, th, K), d, ktil, 0, 0, 0, 0, 0, 0, 0);
-                phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
+                phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], GATE_S(hp, gate, th),
+                            GATE_V(hp, gate, th, K), S, 0);
             }
         }
 
@@ -330,9 +349,10 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 size_t th = (size_t)t * H + h;
                 memcpy(Shist + (size_t)(t - a0) * VK, S, sizeof(double) * VK);
                 memcpy(dhist + (size_t)(t - a0) * K, d, sizeof(double) * K);
-                phase1_step(hp, K, k + th * K, beta[th], gate[th], LRET_S(hp, log_ret, th),
+                phase1_step(hp, K, k + th * K, beta[th], GATE_S(hp, gate, th), LRET_S(hp, log_ret, th),
                             LRET_V(hp, log_ret, th, K), d, ktil, 0, 0, 0, 0, 0, 0, 0);
-                phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], gate[th], S, 0);
+                phase2_step(K, V, k + th * K, ktil, v + th * V, beta[th], GATE_S(hp, gate, th),
+                            GATE_V(hp, gate, th, K), S, 0);
             }
             for (int t = a1 - 1; t >= a0; --t) {
                 size_t th = (size_t)t * H + h;
@@ -340,9 +360,10 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 const double *dot = dout + th * V;
                 const double *Sprev = Shist + (size_t)(t - a0) * VK;
                 const double *dt = dhist + (size_t)(t - a0) * K;
-                double bt = beta[th], gt = gate[th], lt = LRET_S(hp, log_ret, th);
+                double bt = beta[th], gt = GATE_S(hp, gate, th), lt = LRET_S(hp, log_ret, th);
                 const double *lv = LRET_V(hp, log_ret, th, K);
-                double alpha = exp(gt);
+                const double *gv = GATE_V(hp, gate, th, K);
+#define ALPHA(i) exp(gv ? gv[i] : gt)
 
                 /* recompute this token's forward quantities */
                 double c, rho, a, n; int above;
@@ -354,7 +375,7 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 for (int r = 0; r < V; ++r) {
                     double acc = 0.0;
                     for (int i = 0; i < K; ++i) {
-                        Sbar[(size_t)r * K + i] = alpha * Sprev[(size_t)r * K + i];
+                        Sbar[(size_t)r * K + i] = ALPHA(i) * Sprev[(size_t)r * K + i];
                         acc += Sbar[(size_t)r * K + i] * kt[i];
                     }
                     u[r] = vt[r] - acc;
@@ -385,14 +406,17 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 /* u = v - Sbar k ; Sbar = alpha S_{t-1} */
                 double dg_t = 0.0;
                 for (int i = 0; i < K; ++i) dk[th * K + i] = 0.0;
+                if (gv)
+                    for (int i = 0; i < K; ++i) dgate[th * K + i] = 0.0;
                 for (int r = 0; r < V; ++r) {
                     dv[th * V + r] = du[r];
                     for (int i = 0; i < K; ++i) {
                         size_t id = (size_t)r * K + i;
                         dk[th * K + i] -= Sbar[id] * du[r];
                         double dSbar = Shat[id] - du[r] * kt[i];
-                        dg_t += dSbar * Sbar[id];
-                        Shat[id] = alpha * dSbar;          /* now dL/dS_{t-1} */
+                        if (gv) dgate[th * K + i] += dSbar * Sbar[id];   /* d/dg_i of exp(g_i) S[:, i] */
+                        else dg_t += dSbar * Sbar[id];
+                        Shat[id] = ALPHA(i) * dSbar;       /* now dL/dS_{t-1} */
                     }
                 }
                 /* phase-1 adjoint of this step; lam holds dL/dd_{t+1} */
@@ -420,7 +444,8 @@ void osdn_oracle_bwd(int nseq, const int *cu, int H, int K, int V, const oracle_
                 if (hp->apf_mode == 1) dg_t += rho * drho;
                 if (dlog_ret && !lv) dlog_ret[th] = hp->apf_mode == 2 ? rho * drho : 0.0;
                 dbeta[th] = dbeta_t;
-                dgate[th] = dg_t;
+                if (!gv) dgate[th] = dg_t;
+#undef ALPHA
             }
         }
         if (dS0) memcpy(dS0 + ((size_t)s * H + h) * VK, Shat, sizeof(double) * VK);

@@ -36,6 +36,7 @@ class OsdnHyper:
     apf_mode: int = 1  # 0 none, 1 retention aliased to the gate, 2 separate log-retention, 3 one per coordinate
     clamp: int = 1
     chunk: int = 64
+    channel_gate: int = 0  # 1: `gate` is [T, H, K], one log-gate per key channel (OSKDA extension)
 
 
 @dataclass
@@ -159,6 +160,10 @@ def draw(
         gate = torch.zeros(T, H)
     else:
         raise ValueError(gate_kind)
+
+    if hyper.channel_gate:
+        # one log-gate per key channel: the token's gate spread over the channels by a factor in [0.25, 1.75]
+        gate = gate.unsqueeze(-1) * (0.25 + 1.5 * rand(T, H, K))
 
     out = OsdnInputs(
         name=name, H=H, K=K, V=V, io_dtype=io_dtype, seq_lens=[int(x) for x in seq_lens],
