@@ -188,6 +188,37 @@ int osdn_decode_step(const osdn_params* p, const void* q, const void* k, const v
                      float* state, float* precond, void* out, void* cuda_stream);
 
 /*
+ * Channel-gate variant of the layer: the OSKDA backbone extension (appendix "Kimi Delta Attention with
+ * Online Scaling").  The scalar gate of osdn_fwd becomes one gate per key channel,
+ *     Sbar = S_{t-1} Diag(alpha_t),  alpha_t = exp(gate_k[t]) in (0,1]^K,
+ *     u = v_t - Sbar k_t,   S_t = Sbar + beta_t u ktil_t^T,   o_t = scale S_t q_t,
+ * with ktil_t = d_t (.) k_t and d_{t+1} exactly as in osdn_fwd (the beta-aware phase 1 of that appendix;
+ * the preconditioner's retention is its own input and never the channel gate, so OSDN_APF_ALIAS_GATE is
+ * rejected with OSDN_INVALID_ARG).  The paper writes the state as K x V with the gate, the read key and
+ * the scaled write key acting from the left; that state is the transpose of the [S,H,V,K] state used
+ * here and by every other call of this library.
+ *   gate_k   [T,H,K] fp32 DEVICE, log of the channel gates (<= 0); every other argument, the layouts,
+ *            the flags, the alignment rules, ownership and the error codes are those of osdn_fwd / osdn_bwd.
+ *   dgate_k  [T,H,K] fp32, written in full.
+ *   workspace: osdn_kda_workspace_bytes(p, need_bwd) bytes (0 is returned for rejected parameters); for
+ *            the backward it includes, beside the regions of osdn_workspace_bytes, one row history of a
+ *            chunk per state row (S * H * V * 64 * K floats) and an fp32 accumulator for dq.
+ * This path runs on CUDA cores in fp32 for both io_dtypes (one warp per state row, sequential over the
+ * tokens of a sequence): it is the extension's reference implementation on the device, not a tuned one.
+ */
+size_t osdn_kda_workspace_bytes(const osdn_params* p, int need_bwd);
+int osdn_kda_fwd(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                 const float* gate_k, const float* apf_log_ret, const float* init_state,
+                 const float* precond_in, void* out, float* final_state, float* precond_out,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+int osdn_kda_bwd(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                 const float* gate_k, const float* apf_log_ret, const float* init_state,
+                 const float* precond_in, const void* dout, const float* dfinal_state,
+                 const float* dprecond_out, void* dq, void* dk, void* dv, float* dbeta, float* dgate_k,
+                 float* dapf_log_ret, float* dinit_state, float* dprecond_in, void* workspace,
+                 size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Forward pass for callers that cannot provide a workspace.  (The paper has no counterpart to
  * this call; it exists for deployment reasons only.)
  *

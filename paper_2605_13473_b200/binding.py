@@ -20,7 +20,7 @@ EXPORTS = [
     "osdn_step_host", "osdn_read_device_status", "osdn_status_string", "osdn_last_launch_count",
     "osdn_stage_timing_enable", "osdn_stage_timing_read", "osdn_workspace_region",
     "osdn_fwd_static", "osdn_decode_step", "osdn_residual_ratio", "osdn_read_static_status",
-    "osdn_selftest_wait_timeout",
+    "osdn_selftest_wait_timeout", "osdn_kda_workspace_bytes", "osdn_kda_fwd", "osdn_kda_bwd",
 ]
 
 
@@ -186,6 +186,35 @@ def osdn_fwd(p: OsdnParams, q, k, v, beta, gate, apf_log_ret, init_state, precon
     _check(rc, "osdn_fwd")
 
 
+def osdn_kda_workspace_bytes(p: OsdnParams, need_bwd: bool) -> int:
+    lib = load_library()
+    lib.osdn_kda_workspace_bytes.restype = ctypes.c_size_t
+    return int(lib.osdn_kda_workspace_bytes(ctypes.byref(p), ctypes.c_int(1 if need_bwd else 0)))
+
+
+def osdn_kda_fwd(p: OsdnParams, q, k, v, beta, gate_k, apf_log_ret, init_state, precond_in, out, final_state,
+                 precond_out, workspace: torch.Tensor):
+    """Channel-gate variant (OSKDA extension): ``gate_k`` is [T,H,K] fp32; the rest as for ``osdn_fwd``."""
+    lib = load_library()
+    rc = lib.osdn_kda_fwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gate_k), _ptr(apf_log_ret),
+                          _ptr(init_state), _ptr(precond_in), _ptr(out), _ptr(final_state), _ptr(precond_out),
+                          _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                          _stream_ptr())
+    _check(rc, "osdn_kda_fwd")
+
+
+def osdn_kda_bwd(p: OsdnParams, q, k, v, beta, gate_k, apf_log_ret, init_state, precond_in, dout, dfinal_state,
+                 dprecond_out, dq, dk, dv, dbeta, dgate_k, dapf_log_ret, dinit_state, dprecond_in,
+                 workspace: torch.Tensor):
+    lib = load_library()
+    rc = lib.osdn_kda_bwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(gate_k), _ptr(apf_log_ret),
+                          _ptr(init_state), _ptr(precond_in), _ptr(dout), _ptr(dfinal_state), _ptr(dprecond_out),
+                          _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dbeta), _ptr(dgate_k), _ptr(dapf_log_ret),
+                          _ptr(dinit_state), _ptr(dprecond_in), _ptr(workspace),
+                          ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream_ptr())
+    _check(rc, "osdn_kda_bwd")
+
+
 STATIC_SCRATCH_BYTES = 32 << 20
 
 
@@ -300,7 +329,8 @@ class DeviceBundle:
         self.out = torch.empty(T, H, V, device=dev, dtype=dt)
         self.final_state = torch.empty(S, H, V, K, device=dev, dtype=torch.float32)
         self.precond_out = torch.empty(S, H, K, device=dev, dtype=torch.float32)
-        nbytes = osdn_workspace_bytes(self.params, need_bwd)
+        self.channel_gate = bool(getattr(inp.hyper, "channel_gate", 0))   # OSKDA extension: gate is [T,H,K]
+        nbytes = (osdn_kda_workspace_bytes if self.channel_gate else osdn_workspace_bytes)(self.params, need_bwd)
         if nbytes == 0:
             raise RuntimeError("osdn_workspace_bytes rejected the parameters")
         self.workspace = torch.empty(nbytes, device=dev, dtype=torch.uint8)
@@ -309,7 +339,7 @@ class DeviceBundle:
             self.dk = torch.empty(T, H, K, device=dev, dtype=dt)
             self.dv = torch.empty(T, H, V, device=dev, dtype=dt)
             self.dbeta = torch.empty(T, H, device=dev, dtype=torch.float32)
-            self.dgate = torch.empty(T, H, device=dev, dtype=torch.float32)
+            self.dgate = torch.empty((T, H, K) if self.channel_gate else (T, H), device=dev, dtype=torch.float32)
             mode = int(self.params.apf_mode)
             if mode >= 2:   # written in full by osdn_bwd ([T,H], or [T,H,K] for the vector retention)
                 self.dlog_ret = torch.full((T, H, K) if mode == 3 else (T, H), float("nan"), device=dev)
@@ -321,15 +351,17 @@ class DeviceBundle:
     def fwd(self, save: bool = False):
         base = self.params.flags & FLAG_FORCE_SIMT
         self.params.flags = base | (FLAG_SAVE_RESIDUALS if save else 0)
-        osdn_fwd(self.params, self.q, self.k, self.v, self.beta, self.gate, self.log_ret, self.init_state,
-                 self.precond_in, self.out, self.final_state, self.precond_out, self.workspace)
+        (osdn_kda_fwd if self.channel_gate else osdn_fwd)(
+            self.params, self.q, self.k, self.v, self.beta, self.gate, self.log_ret, self.init_state,
+            self.precond_in, self.out, self.final_state, self.precond_out, self.workspace)
 
     def bwd(self, residuals_valid: bool = False):
         base = self.params.flags & FLAG_FORCE_SIMT
         self.params.flags = base | (FLAG_RESIDUALS_VALID if residuals_valid else 0)
-        osdn_bwd(self.params, self.q, self.k, self.v, self.beta, self.gate, self.log_ret, self.init_state,
-                 self.precond_in, self.dout, self.dfinal_state, self.dprecond_out, self.dq, self.dk, self.dv,
-                 self.dbeta, self.dgate, self.dlog_ret, self.dinit_state, self.dprecond_in, self.workspace)
+        (osdn_kda_bwd if self.channel_gate else osdn_bwd)(
+            self.params, self.q, self.k, self.v, self.beta, self.gate, self.log_ret, self.init_state,
+            self.precond_in, self.dout, self.dfinal_state, self.dprecond_out, self.dq, self.dk, self.dv,
+            self.dbeta, self.dgate, self.dlog_ret, self.dinit_state, self.dprecond_in, self.workspace)
 
     def device_status(self) -> int:
         return osdn_read_device_status(self.workspace)

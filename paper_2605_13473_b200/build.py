@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libosdn.so")
-SOURCES = ["osdn_api.cu", "osdn_phase1.cu", "osdn_simt.cu", "osdn_tc.cu", "osdn_decode.cu"]
+SOURCES = ["osdn_api.cu", "osdn_phase1.cu", "osdn_simt.cu", "osdn_tc.cu", "osdn_decode.cu", "osdn_kda.cu"]
 
 
 def _newest(paths):

@@ -207,6 +207,88 @@ int osdn_bwd(const osdn_params* p, const void* q, const void* k, const void* v, 
     return OSDN_OK;
 }
 
+size_t osdn_kda_workspace_bytes(const osdn_params* p, int need_bwd)
+{
+    if (validate(p) != OSDN_OK || p->apf_mode == OSDN_APF_ALIAS_GATE) return 0;
+    const WsLayout L = make_layout(*p, need_bwd != 0);
+    return align_up(L.total, 256) + kda_extra_bytes(*p, L, need_bwd != 0);
+}
+
+int osdn_kda_fwd(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                 const float* gate_k, const float* apf_log_ret, const float* init_state, const float* precond_in,
+                 void* out, float* final_state, float* precond_out, void* workspace, size_t workspace_bytes,
+                 void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (p->apf_mode == OSDN_APF_ALIAS_GATE) return OSDN_INVALID_ARG;   // the retention is separate from a channel gate
+    if (!q || !k || !v || !beta || !gate_k || !out || !workspace) return OSDN_INVALID_ARG;
+    if (p->apf_mode >= OSDN_APF_SEPARATE && !apf_log_ret) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, beta, gate_k, apf_log_ret, init_state, precond_in, out, final_state, precond_out};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return OSDN_MISALIGNED;
+    const bool save = (p->flags & OSDN_FLAG_SAVE_RESIDUALS) != 0;
+    const WsLayout L = make_layout(*p, save);
+    if (workspace_bytes < align_up(L.total, 256) + kda_extra_bytes(*p, L, save)) return OSDN_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(static_cast<char*>(workspace) + L.status, 0, 256, st) != cudaSuccess) return OSDN_CUDA_ERROR;
+    Pointers a{};
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.gate = gate_k; a.log_ret = apf_log_ret;
+    a.init_state = init_state; a.precond_in = precond_in; a.out = out; a.final_state = final_state;
+    a.precond_out = precond_out;
+    const int n = kda_forward(*p, make_hyper(*p), L, workspace, a, save, st);
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = n;
+    return OSDN_OK;
+}
+
+int osdn_kda_bwd(const osdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                 const float* gate_k, const float* apf_log_ret, const float* init_state, const float* precond_in,
+                 const void* dout, const float* dfinal_state, const float* dprecond_out, void* dq, void* dk,
+                 void* dv, float* dbeta, float* dgate_k, float* dapf_log_ret, float* dinit_state,
+                 float* dprecond_in, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != OSDN_OK) return rc;
+    if (p->apf_mode == OSDN_APF_ALIAS_GATE) return OSDN_INVALID_ARG;
+    if (!q || !k || !v || !beta || !gate_k || !dout || !dq || !dk || !dv || !dbeta || !dgate_k || !workspace)
+        return OSDN_INVALID_ARG;
+    if (p->apf_mode >= OSDN_APF_SEPARATE && (!apf_log_ret || !dapf_log_ret)) return OSDN_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, beta, gate_k, apf_log_ret, init_state, precond_in, dout, dfinal_state,
+                          dprecond_out, dq, dk, dv, dbeta, dgate_k, dapf_log_ret, dinit_state, dprecond_in};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return OSDN_MISALIGNED;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return OSDN_MISALIGNED;
+    const WsLayout L = make_layout(*p, true);
+    if (workspace_bytes < align_up(L.total, 256) + kda_extra_bytes(*p, L, true)) return OSDN_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Hyper hy = make_hyper(*p);
+    Pointers a{};
+    a.q = q; a.k = k; a.v = v; a.beta = beta; a.gate = gate_k; a.log_ret = apf_log_ret;
+    a.init_state = init_state; a.precond_in = precond_in;
+    a.dout = dout; a.dfinal_state = dfinal_state; a.dprecond_out = dprecond_out;
+    a.dq = dq; a.dk = dk; a.dv = dv; a.dbeta = dbeta; a.dgate = dgate_k; a.dlog_ret = dapf_log_ret;
+    a.dinit_state = dinit_state; a.dprecond_in = dprecond_in;
+    int total = 0;
+    if (!(p->flags & OSDN_FLAG_RESIDUALS_VALID)) {
+        if (cudaMemsetAsync(static_cast<char*>(workspace) + L.status, 0, 256, st) != cudaSuccess) return OSDN_CUDA_ERROR;
+        Pointers f = a;
+        f.out = static_cast<char*>(workspace) + L.out_scratch;
+        f.final_state = nullptr;
+        f.precond_out = nullptr;
+        const int n = kda_forward(*p, hy, L, workspace, f, true, st);
+        if (n < 0) return OSDN_CUDA_ERROR;
+        total += n;
+    }
+    const int n = kda_backward(*p, hy, L, workspace, a, st);
+    if (n < 0) return OSDN_CUDA_ERROR;
+    g_last_launches = total + n;
+    return OSDN_OK;
+}
+
 int osdn_precond_update(const osdn_params* p, const void* k, const float* beta, const float* gate_or_log_ret,
                         const float* precond_in, void* k_tilde_out, float* precond_out, void* cuda_stream)
 {

@@ -205,6 +205,13 @@ int decode_step(const osdn_params& p, const Hyper& hy, const void* q, const void
                 const float* beta, const float* gate, const float* log_ret, float* state, float* precond,
                 void* out, cudaStream_t st);
 int launch_build_table(const osdn_params& p, const WsLayout& L, void* ws, cudaStream_t st);
+// Channel-gate variant of the layer (osdn_kda.cu): a.gate is [T,H,K].  The backward needs
+// kda_extra_bytes of workspace behind the common layout.
+size_t kda_extra_bytes(const osdn_params& p, const WsLayout& L, bool need_bwd);
+int kda_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a, bool save,
+                cudaStream_t st);
+int kda_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                 cudaStream_t st);
 
 // Optional per-kernel timing (off by default): when enabled through osdn_stage_timing_enable, every
 // launch site records a CUDA event on the launching stream before its kernel; stage_end closes the

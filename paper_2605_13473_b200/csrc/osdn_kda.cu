@@ -1,0 +1,347 @@
+// Online-scaled delta rule with a channel gate (the OSKDA backbone extension: Kimi Delta Attention with
+// Online Scaling).  The scalar gate exp(g_t) of the layer becomes one gate per key channel,
+//     Sbar = S_{t-1} Diag(alpha_t),  u = v_t - Sbar k_t,  S_t = Sbar + beta_t u ktil_t^T,  o_t = scale S_t q_t,
+// with the state kept V x K as everywhere in this library (the paper's K x V state is its transpose).
+// Phase 1 (preconditioner, write keys, their adjoint) is the layer's own and is reused unchanged; this
+// file holds phase 2 and its adjoint as token-recurrent CUDA-core kernels in fp32: the rows of S do not
+// interact in the forward, so one warp owns one row (a lane holds K / 32 of its columns) and walks the
+// sequence; the dot products along a row are warp reductions.  The backward walks the chunks in
+// reverse: it replays a chunk from the row checkpoint the forward left at its start, keeping the row
+// before every token, then takes the adjoint steps; the sums over rows (dq, dk, d ktil, d gate, d beta)
+// are formed per CTA in shared memory and added to global fp32 accumulators.
+#include "osdn_common.cuh"
+
+namespace osdn {
+namespace {
+
+constexpr int KF_WARPS = 8;    // forward: state rows per CTA
+constexpr int KB_WARPS = 32;   // backward: state rows per CTA
+
+template <int R> struct Vec {
+    float x[R];
+};
+
+template <int R> __device__ __forceinline__ Vec<R> load_vec(const float* p)
+{
+    Vec<R> r;
+    if constexpr (R == 4) {
+        const float4 f = *reinterpret_cast<const float4*>(p);
+        r.x[0] = f.x; r.x[1] = f.y; r.x[2] = f.z; r.x[3] = f.w;
+    } else {
+        const float2 f = *reinterpret_cast<const float2*>(p);
+        r.x[0] = f.x; r.x[1] = f.y;
+    }
+    return r;
+}
+template <int R> __device__ __forceinline__ Vec<R> load_vec(const __nv_bfloat16* p)
+{
+    Vec<R> r;
+    if constexpr (R == 4) {
+        const uint2 w = *reinterpret_cast<const uint2*>(p);
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w.x));
+        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w.y));
+        r.x[0] = a.x; r.x[1] = a.y; r.x[2] = b.x; r.x[3] = b.y;
+    } else {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+        r.x[0] = a.x; r.x[1] = a.y;
+    }
+    return r;
+}
+template <int R> __device__ __forceinline__ void store_vec(float* p, const Vec<R>& v)
+{
+    if constexpr (R == 4) *reinterpret_cast<float4*>(p) = make_float4(v.x[0], v.x[1], v.x[2], v.x[3]);
+    else *reinterpret_cast<float2*>(p) = make_float2(v.x[0], v.x[1]);
+}
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+struct KdaArgs {
+    int H, V;
+    Table tab;
+    const void *q, *k, *v;
+    const float *beta, *gate;     // gate: [T,H,K] channel log-gates
+    const float* ktil;            // [T,H,K] write keys of phase 1
+    const float* init_state;      // nullable
+    void* out;
+    float* final_state;           // nullable
+    float* ckpt;                  // nullable: [chunk, H, V, K] rows at every chunk start
+    float scale;
+    // backward
+    const void* dout;
+    const float* dfinal_state;    // nullable
+    void* dv;
+    float *dq_acc, *dkread, *dktil, *dgate, *dbeta;   // zeroed accumulators
+    float* dinit_state;           // nullable
+    float* hist;                  // [chain, V, CH, K] rows before every token of the chunk in progress
+};
+
+// What a row needs of one token.
+template <int R> struct Tok {
+    Vec<R> k, kt, g;
+    float v, beta;
+};
+
+template <typename T, int R>
+__device__ __forceinline__ Tok<R> load_tok(const KdaArgs& a, size_t th, int K, int row, int lane)
+{
+    Tok<R> t;
+    t.k = load_vec<R>(static_cast<const T*>(a.k) + th * K + R * lane);
+    t.kt = load_vec<R>(a.ktil + th * K + R * lane);
+    t.g = load_vec<R>(a.gate + th * K + R * lane);
+    t.v = ldf(static_cast<const T*>(a.v) + th * a.V + row);
+    t.beta = a.beta[th];
+    return t;
+}
+
+// One forward step of a row: S <- S Diag(alpha) + beta u ktil^T; returns u, leaves Sbar in `sbar`.
+template <int R> __device__ __forceinline__ float row_step(Vec<R>& S, const Tok<R>& t, Vec<R>* sbar)
+{
+    float acc = 0.f;
+#pragma unroll
+    for (int x = 0; x < R; ++x) {
+        S.x[x] *= __expf(t.g.x[x]);
+        acc = fmaf(S.x[x], t.k.x[x], acc);
+    }
+    if (sbar) *sbar = S;
+    const float u = t.v - warp_sum(acc);
+    const float bu = t.beta * u;
+#pragma unroll
+    for (int x = 0; x < R; ++x) S.x[x] = fmaf(bu, t.kt.x[x], S.x[x]);
+    return u;
+}
+
+template <typename T, int K>
+__global__ void __launch_bounds__(KF_WARPS * 32) kda_fwd_kernel(KdaArgs a)
+{
+    constexpr int R = K / 32;
+    const int H = a.H, V = a.V;
+    const int chain = blockIdx.y, s = chain / H, h = chain - s * H;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * KF_WARPS + warp;
+    const int t0 = a.tab.seq_tok0(s), len = a.tab.seq_len(s), c0 = a.tab.seq_chunk0(s);
+    const size_t srow = (((size_t)s * H + h) * V + row) * K + R * lane;
+    Vec<R> S;
+    if (a.init_state) S = load_vec<R>(a.init_state + srow);
+    else
+#pragma unroll
+        for (int x = 0; x < R; ++x) S.x[x] = 0.f;
+    if (len > 0) {
+        Tok<R> cur = load_tok<T, R>(a, (size_t)t0 * H + h, K, row, lane);
+        Vec<R> qc = load_vec<R>(static_cast<const T*>(a.q) + ((size_t)t0 * H + h) * K + R * lane);
+        for (int t = 0; t < len; ++t) {
+            const size_t th = (size_t)(t0 + t) * H + h;
+            Tok<R> nxt = cur;
+            Vec<R> qn = qc;
+            if (t + 1 < len) {   // the next token's operands are in flight while this one is worked on
+                nxt = load_tok<T, R>(a, th + H, K, row, lane);
+                qn = load_vec<R>(static_cast<const T*>(a.q) + (th + H) * K + R * lane);
+            }
+            if (a.ckpt && (t % CH) == 0)
+                store_vec<R>(a.ckpt + (((size_t)(c0 + t / CH) * H + h) * V + row) * K + R * lane, S);
+            row_step<R>(S, cur, nullptr);
+            float o = 0.f;
+#pragma unroll
+            for (int x = 0; x < R; ++x) o = fmaf(S.x[x], qc.x[x], o);
+            o = a.scale * warp_sum(o);
+            if (lane == 0) stf(static_cast<T*>(a.out) + th * V + row, o);
+            cur = nxt;
+            qc = qn;
+        }
+    }
+    if (a.final_state) store_vec<R>(a.final_state + srow, S);
+}
+
+template <typename T, int K>
+__global__ void __launch_bounds__(KB_WARPS * 32) kda_bwd_kernel(KdaArgs a)
+{
+    constexpr int R = K / 32;
+    extern __shared__ float red[];                 // [2][KB_WARPS][4][K]: per-row terms of dq, dk, d ktil, d gate
+    __shared__ float red_beta[2][KB_WARPS];
+    const int H = a.H, V = a.V;
+    const int chain = blockIdx.y, s = chain / H, h = chain - s * H;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int row = blockIdx.x * KB_WARPS + warp;
+    const int t0 = a.tab.seq_tok0(s), len = a.tab.seq_len(s), c0 = a.tab.seq_chunk0(s);
+    const int nchunks = (len + CH - 1) / CH;
+    const size_t srow = (((size_t)s * H + h) * V + row) * K + R * lane;
+    float* hist = a.hist + ((size_t)chain * V + row) * CH * K + R * lane;
+    Vec<R> Shat;
+    if (a.dfinal_state) Shat = load_vec<R>(a.dfinal_state + srow);
+    else
+#pragma unroll
+        for (int x = 0; x < R; ++x) Shat.x[x] = 0.f;
+    int it = 0;
+    for (int n = nchunks - 1; n >= 0; --n) {
+        const int clen = min(CH, len - n * CH);
+        const size_t th0 = (size_t)(t0 + n * CH) * H + h;
+        // replay the chunk from its checkpoint, keeping the row before every token
+        {
+            Vec<R> S = load_vec<R>(a.ckpt + (((size_t)(c0 + n) * H + h) * V + row) * K + R * lane);
+            for (int j = 0; j < clen; ++j) {
+                store_vec<R>(hist + (size_t)j * K, S);
+                const Tok<R> tk = load_tok<T, R>(a, th0 + (size_t)j * H, K, row, lane);
+                row_step<R>(S, tk, nullptr);
+            }
+        }
+        for (int j = clen - 1; j >= 0; --j, ++it) {
+            const size_t th = th0 + (size_t)j * H;
+            const Tok<R> tk = load_tok<T, R>(a, th, K, row, lane);
+            const Vec<R> q = load_vec<R>(static_cast<const T*>(a.q) + th * K + R * lane);
+            const float sdo = a.scale * ldf(static_cast<const T*>(a.dout) + th * V + row);
+            Vec<R> St = load_vec<R>(hist + (size_t)j * K), Sbar;
+            const float u = row_step<R>(St, tk, &Sbar);
+            float* buf = red + ((size_t)(it & 1) * KB_WARPS + warp) * 4 * K + R * lane;
+            Vec<R> part;
+            // o_t = scale S_t q_t
+            float w = 0.f;
+#pragma unroll
+            for (int x = 0; x < R; ++x) {
+                part.x[x] = sdo * St.x[x];
+                Shat.x[x] = fmaf(sdo, q.x[x], Shat.x[x]);
+                w = fmaf(Shat.x[x], tk.kt.x[x], w);
+            }
+            store_vec<R>(buf, part);                              // dq
+            // S_t = Sbar + beta u ktil^T
+            w = warp_sum(w);
+            const float du = tk.beta * w;
+#pragma unroll
+            for (int x = 0; x < R; ++x) part.x[x] = tk.beta * u * Shat.x[x];
+            store_vec<R>(buf + 2 * K, part);                      // d ktil
+            // u = v - Sbar k ; Sbar = S_{t-1} Diag(alpha)
+            Vec<R> dkp, dgp;
+#pragma unroll
+            for (int x = 0; x < R; ++x) {
+                dkp.x[x] = -Sbar.x[x] * du;
+                const float dsb = fmaf(-du, tk.k.x[x], Shat.x[x]);
+                dgp.x[x] = dsb * Sbar.x[x];
+                Shat.x[x] = __expf(tk.g.x[x]) * dsb;
+            }
+            store_vec<R>(buf + K, dkp);                           // dk (read key)
+            store_vec<R>(buf + 3 * K, dgp);                       // d gate
+            if (lane == 0) {
+                red_beta[it & 1][warp] = u * w;
+                stf(static_cast<T*>(a.dv) + th * V + row, du);
+            }
+            __syncthreads();
+            // sums over the CTA's rows; the buffers alternate, so one barrier per token is enough
+            if (tid < 4 * K) {
+                const float* src = red + (size_t)(it & 1) * KB_WARPS * 4 * K + tid;
+                float sum = 0.f;
+#pragma unroll 8
+                for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += src[(size_t)w2 * 4 * K];
+                const int m = tid / K, i = tid - m * K;
+                float* dst = m == 0 ? a.dq_acc : m == 1 ? a.dkread : m == 2 ? a.dktil : a.dgate;
+                atomicAdd(dst + th * K + i, sum);
+            } else if (tid == 4 * K) {
+                float sum = 0.f;
+                for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += red_beta[it & 1][w2];
+                atomicAdd(a.dbeta + th, sum);
+            }
+        }
+    }
+    if (a.dinit_state) store_vec<R>(a.dinit_state + srow, Shat);
+}
+
+template <typename T> __global__ void cast_rows_kernel(const float* src, T* dst, size_t n)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) stf(dst + i, src[i]);
+}
+
+}  // namespace
+
+size_t kda_extra_bytes(const osdn_params& p, const WsLayout& L, bool need_bwd)
+{
+    if (!need_bwd) return 0;
+    const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
+    const size_t hist = align_up((size_t)L.S * p.H * p.V * CH * p.K * 4, 256);
+    const size_t dq = align_up(Ttot * p.H * p.K * 4, 256);
+    return hist + dq;
+}
+
+namespace {
+KdaArgs base_args(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a)
+{
+    char* w = static_cast<char*>(ws);
+    KdaArgs k{};
+    k.H = p.H; k.V = p.V; k.tab = carve_table(ws, L);
+    k.q = a.q; k.k = a.k; k.v = a.v; k.beta = a.beta; k.gate = a.gate;
+    k.ktil = reinterpret_cast<const float*>(w + L.ktil);
+    k.init_state = a.init_state; k.scale = hy.scale;
+    k.ckpt = reinterpret_cast<float*>(w + L.Sn);
+    return k;
+}
+}  // namespace
+
+int kda_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a, bool save,
+                cudaStream_t st)
+{
+    int launches = launch_build_table(p, L, ws, st);
+    if (launches < 0) return -1;
+    char* w = static_cast<char*>(ws);
+    const int n1 = phase1_forward(p, hy, L, ws, a, w + L.ktil, false, save, st);
+    if (n1 < 0) return -1;
+    launches += n1;
+    KdaArgs k = base_args(p, hy, L, ws, a);
+    k.out = a.out; k.final_state = a.final_state;
+    if (!save) k.ckpt = nullptr;
+    const dim3 grid(p.V / KF_WARPS, L.S * p.H);
+    stage_mark(st, "kda_fwd");
+    if (p.io_dtype == OSDN_FP32) {
+        if (p.K == 64) kda_fwd_kernel<float, 64><<<grid, KF_WARPS * 32, 0, st>>>(k);
+        else kda_fwd_kernel<float, 128><<<grid, KF_WARPS * 32, 0, st>>>(k);
+    } else {
+        if (p.K == 64) kda_fwd_kernel<__nv_bfloat16, 64><<<grid, KF_WARPS * 32, 0, st>>>(k);
+        else kda_fwd_kernel<__nv_bfloat16, 128><<<grid, KF_WARPS * 32, 0, st>>>(k);
+    }
+    stage_end(st);
+    return cudaGetLastError() == cudaSuccess ? launches + 1 : -1;
+}
+
+int kda_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* ws, const Pointers& a,
+                 cudaStream_t st)
+{
+    char* w = static_cast<char*>(ws);
+    const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
+    const size_t nK = Ttot * p.H * p.K;
+    KdaArgs k = base_args(p, hy, L, ws, a);
+    k.dout = a.dout; k.dfinal_state = a.dfinal_state; k.dv = a.dv; k.dinit_state = a.dinit_state;
+    k.hist = reinterpret_cast<float*>(w + align_up(L.total, 256));
+    k.dq_acc = reinterpret_cast<float*>(w + align_up(L.total, 256) +
+                                        align_up((size_t)L.S * p.H * p.V * CH * p.K * 4, 256));
+    k.dkread = reinterpret_cast<float*>(w + L.dkread);
+    k.dktil = reinterpret_cast<float*>(w + L.dktil);
+    k.dgate = a.dgate; k.dbeta = a.dbeta;
+    if (cudaMemsetAsync(k.dq_acc, 0, nK * 4, st) != cudaSuccess || cudaMemsetAsync(k.dkread, 0, nK * 4, st) != cudaSuccess ||
+        cudaMemsetAsync(k.dktil, 0, nK * 4, st) != cudaSuccess || cudaMemsetAsync(k.dgate, 0, nK * 4, st) != cudaSuccess ||
+        cudaMemsetAsync(k.dbeta, 0, Ttot * p.H * 4, st) != cudaSuccess)
+        return -1;
+    const dim3 grid(p.V / KB_WARPS, L.S * p.H);
+    const size_t smem = (size_t)2 * KB_WARPS * 4 * p.K * sizeof(float);
+    stage_mark(st, "kda_bwd");
+    auto launch = [&](auto kernel) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        kernel<<<grid, KB_WARPS * 32, smem, st>>>(k);
+        return true;
+    };
+    bool ok;
+    if (p.io_dtype == OSDN_FP32) ok = p.K == 64 ? launch(kda_bwd_kernel<float, 64>) : launch(kda_bwd_kernel<float, 128>);
+    else ok = p.K == 64 ? launch(kda_bwd_kernel<__nv_bfloat16, 64>) : launch(kda_bwd_kernel<__nv_bfloat16, 128>);
+    if (!ok) return -1;
+    stage_mark(st, "kda_cast_dq");
+    const unsigned blocks = (unsigned)((nK + 255) / 256);
+    if (p.io_dtype == OSDN_FP32) cast_rows_kernel<float><<<blocks, 256, 0, st>>>(k.dq_acc, static_cast<float*>(a.dq), nK);
+    else cast_rows_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(k.dq_acc, static_cast<__nv_bfloat16*>(a.dq), nK);
+    // phase-1 adjoint: dk = dk(read key) + d_t (.) d ktil + preconditioner terms; adds its share to d beta
+    const int n1 = phase1_backward(p, hy, L, ws, a, k.dktil, k.dkread, true, st);
+    if (n1 < 0) return -1;
+    stage_end(st);
+    return cudaGetLastError() == cudaSuccess ? 2 + n1 : -1;
+}
+
+}  // namespace osdn
