@@ -82,6 +82,7 @@ def method_bytes(name, inp, with_bwd):
         "phase1_seq": 0.0, "phase1_bwd_seq": 0.0, "build_table": 0.0,
         "tc_chunk_fwd": 2 * K * es + 8,                              # q, k, beta, gate
         "tc_chain_fwd": V * es + V * es + (state if with_bwd else 0),  # v in, out, saved state
+        "tc_fwd": 2 * K * es + 8 + V * es + V * es + (state if with_bwd else 0),   # both passes in one launch
         # q, k, v, dout, beta, gate, the saved state in; dq, dk, dv, dbeta, dgate out
         "tc_bwd": (2 * K + 2 * V) * es + 8 + state + (2 * K + V) * es + 8,
     }
@@ -122,6 +123,7 @@ def kernel_model(name, inp, NT):
                          tiles * (f(128, 64, K) + f(128, 64, C)), "hbm")
     m["tc_chain_fwd"] = (tiles * (16384 + 8192 + 8192 + 3 * raw + raw + 32768 + 16384) + tokh * 4,
                          tiles * (f(128, 64, C) + 2 * f(128, 64, K) + f(128, 64, C) + f(128, 128, C)), "hbm")
+    m["tc_fwd"] = (m["tc_chunk_fwd"][0] + m["tc_chain_fwd"][0], m["tc_chunk_fwd"][1] + m["tc_chain_fwd"][1], "hbm")
     # one launch: the reverse state chains (dout, ktil, W^T, P', Qg in; dS_n, ddU^T out) and the chunk-local
     # part (q, k, ktil, v, dout, dU^T, ddU^T, T, S_n, dS_n in; dq, dk, dv out)
     m["tc_bwd"] = (tiles * (2 * raw + 8192 + 16384 + 16384 + 32768 + 16384) + tokh * 4
