@@ -93,11 +93,18 @@ __global__ void __launch_bounds__(DEC_WARPS * 32) decode_kernel(DecArgs a)
 
     float S[DEC_RW][R], d[R];
     float* srow = a.state + ((size_t)chain * V + v0) * K;
+    dec_load<R>(a.precond + (size_t)chain * K, lane, d);
 #pragma unroll
     for (int r = 0; r < DEC_RW; ++r) dec_load<R>(srow + (size_t)r * K, lane, S[r]);
-    dec_load<R>(a.precond + (size_t)chain * K, lane, d);
-    // this slice has read the chain's preconditioner (release: the read is ordered before the arrival)
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    // This slice has read the chain's preconditioner: the arrival takes the loaded values as an operand, so
+    // it cannot issue before they have come back, and a load that has returned cannot see a later store.
+    // (A releasing arrival would also wait for the state rows, which are still in flight here.)
+    {
+        float seen = d[0];
+#pragma unroll
+        for (int j = 1; j < R; ++j) seen += d[j];
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::"f"(seen) : "memory");
+    }
 
     // inputs of a token, fetched one token ahead
     float kk[R], qq[R], vv[DEC_RW], bt, gt, lr, lrv[VEC ? R : 1];
