@@ -134,13 +134,13 @@ def kernel_model(name, inp, NT):
     return m.get(name)
 
 
-def load_traffic(workload, kernel, measured_us=None):
+def load_traffic(workload, kernel, measured_us=None, summary=None):
     """DRAM bytes (read + write) of one launch of `kernel` from the committed ncu summary of this
     workload (lines "- traffic_bytes <kernel> = <bytes>" and "- profile_us <kernel> = <duration>").
     The capture belongs to the build it was taken on: when the kernel's duration in the capture and the
     one measured now differ by more than 15 % the figure is stale and dropped.  Returns
     (bytes or None, a note naming the source)."""
-    rel = os.path.join("profiles", f"osdn_step_{workload}.md")
+    rel = os.path.join("profiles", summary or f"osdn_step_{workload}.md")
     nbytes, prof_us = None, None
     try:
         for line in open(os.path.join(ROOT, rel)):
@@ -340,7 +340,7 @@ def run_decode(args):
     nbytes = B * H * (2 * D * D * 4 + 2 * D * 4 + (2 * D + 2 * D) * 2 + 8)   # state and d in+out, q k v out, beta gate
     ach = nbytes / avg_s / 1e9
     roofline = dict(kernel="decode_step", bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
-                    frac=ach / peaks["hbm_gbs"], traffic=load_traffic("decode", "decode_step")[0],
+                    frac=ach / peaks["hbm_gbs"], traffic=load_traffic("decode", "decode_step", avg_s * 1e6, "osdn_decode_b512.md")[0],
                     peak_source=peaks["source"], avg_us=avg_s * 1e6, algorithmic_bytes=nbytes)
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
