@@ -68,7 +68,7 @@ def make_inputs(name):
 #                  or writes and the per-chunk state the backward is entitled to (one bf16 state
 #                  image per 64 tokens) -- independent of how this design splits the work.  The
 #                  roofline fraction is computed from these.
-#   kernel_model : the bytes the DESIGN makes the kernel read + write (its tiles included) and its
+#   kernel_model : the bytes this design makes the kernel read + write (its tiles included) and its
 #                  tensor flops; reported beside the fraction as `design_bytes`, never as its numerator.
 # ---------------------------------------------------------------------------------------------
 def method_bytes(name, inp, with_bwd):

@@ -31,6 +31,10 @@ struct Table {
     int* chunk_tok0_;  // [NTmax]
     int* chunk_len_;   // [NTmax]
     int* chunk_seq_;   // [NTmax]
+    int* order_;       // [NTmax]  packed batches: the chunks sorted by the step at which their chain needs them
+                       //          when all chains are to end together (see build_table_kernel)
+    int* pos_;         // [2 NTmax + 4] scratch of the sort; pos_[0] = chunks of the longest sequence
+    int* seq_first_;   // [S]      rank of the sequence's first chunk in order_
     int dense_T;       // > 0: dense batch with sequences of this length
     int dense_nc;      //      and this many chunks per sequence
     __device__ __forceinline__ int seq_tok0(int s) const { return dense_T ? s * dense_T : seq_tok0_[s]; }
@@ -96,7 +100,7 @@ inline WsLayout make_layout(const osdn_params& p, bool need_bwd)
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     L.status = take(256);
-    L.table = take(sizeof(int) * (3 * (size_t)S + 1 + 3 * NT));
+    L.table = take(sizeof(int) * (4 * (size_t)S + 1 + 6 * NT + 4));
     L.p1n = take(4 * Ttot * H);
     L.p1rho = take(4 * Ttot * H);
     L.p1flags = take(4 * NT * H * 2);
@@ -134,6 +138,9 @@ inline Table carve_table(void* ws, const WsLayout& L)
     t.chunk_tok0_ = base + 3 * L.S + 1;
     t.chunk_len_ = t.chunk_tok0_ + L.NTmax;
     t.chunk_seq_ = t.chunk_len_ + L.NTmax;
+    t.order_ = t.chunk_seq_ + L.NTmax;
+    t.pos_ = t.order_ + L.NTmax;
+    t.seq_first_ = t.pos_ + 2 * L.NTmax + 4;
     t.dense_T = L.dense_T;
     t.dense_nc = L.dense_T ? (L.dense_T + CH - 1) / CH : 0;
     return t;

@@ -120,6 +120,56 @@ build_table_kernel(int S, int T_dense, const int* __restrict__ cu, int NTmax, Ta
         t.chunk_len_[j] = rem < CH ? rem : CH;
         t.chunk_seq_[j] = s;
     }
+    // The chunks sorted by the step at which their chain needs them when every chain is to END at the same
+    // time: chunk n of a sequence of nc chunks has the key longest - nc + n, so a short sequence starts
+    // late and the longest ones are served first (a counting sort; the order among chunks of equal key
+    // is whatever the atomics give).  pos_: [0] longest sequence in chunks, [2 + key] number of chunks
+    // with that key, then its running offset, [2 + NTmax + 1 + key] fill counter.
+    int* cnt = t.pos_ + 2;
+    int* fill = t.pos_ + 3 + NTmax;
+    for (int j = tid; j <= NTmax; j += TBL_THREADS) {
+        cnt[j] = 0;
+        if (j < NTmax) fill[j] = 0;
+    }
+    if (tid == 0) t.pos_[0] = 0;
+    __syncthreads();
+    for (int s = tid; s < S; s += TBL_THREADS) atomicMax(&t.pos_[0], t.seq_chunk0_[s + 1] - t.seq_chunk0_[s]);
+    __syncthreads();
+    const int maxn = t.pos_[0];
+    auto key_of = [&](int j) {
+        const int s = t.chunk_seq_[j];
+        const int c0 = in_smem ? s_c0[s] : t.seq_chunk0_[s], c1 = in_smem ? s_c0[s + 1] : t.seq_chunk0_[s + 1];
+        return maxn - (c1 - c0) + (j - c0);
+    };
+    for (int j = tid; j < total; j += TBL_THREADS) atomicAdd(&cnt[key_of(j)], 1);
+    __syncthreads();
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (int base = 0; base < maxn; base += TBL_THREADS) {   // exclusive scan of the counts, in place
+        const int n = base + tid;
+        const int v = n < maxn ? cnt[n] : 0;
+        s_scan[tid] = v;
+        __syncthreads();
+        for (int o = 1; o < TBL_THREADS; o <<= 1) {
+            const int u = tid >= o ? s_scan[tid - o] : 0;
+            __syncthreads();
+            s_scan[tid] += u;
+            __syncthreads();
+        }
+        const int carry = s_carry;
+        if (n < maxn) cnt[n] = carry + s_scan[tid] - v;
+        __syncthreads();
+        if (tid == TBL_THREADS - 1) s_carry = carry + s_scan[tid];
+        __syncthreads();
+    }
+    for (int j = tid; j < total; j += TBL_THREADS) {
+        const int n = key_of(j);
+        t.order_[cnt[n] + atomicAdd(&fill[n], 1)] = j;
+    }
+    for (int s = tid; s < S; s += TBL_THREADS) {
+        const int nc = t.seq_chunk0_[s + 1] - t.seq_chunk0_[s];
+        t.seq_first_[s] = nc > 0 ? cnt[maxn - nc] : 0;
+    }
 }
 
 __device__ __forceinline__ float warp_sum(float x)

@@ -652,8 +652,8 @@ __device__ __forceinline__ void chain_fwd_role(const CUtensorMap& tmV, const CUt
             const int tok0 = chunk_tok0(n);
             float ga_next = 0.f, gb_next = 0.f;
             if (n + 1 < nchunks) load_gates(n + 1, ga_next, gb_next);
-            if (n >= 2) ok = mbar_wait(&bar_empty[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_TMA);
-            if (!ok) break;
+            // The record's flag is looked at before the stage is waited for: its round trip to memory then
+            // runs while the products of the chunk before last still read the stage.
             if (a.ready) {   // the chunk-local pass runs beside the chains: wait until the record is written
                 const int* flag = a.ready + (size_t)(c0 + n) * H + h;
                 const long long t0 = clock64();
@@ -669,6 +669,8 @@ __device__ __forceinline__ void chain_fwd_role(const CUtensorMap& tmV, const CUt
                 }
                 fence_proxy_async_all();
             }
+            if (n >= 2) ok = mbar_wait(&bar_empty[st], ((n >> 1) - 1) & 1, a.status, ERR_CHAIN_TMA);
+            if (!ok) break;
             if (lane == 0) {
                 const size_t tile = (size_t)(c0 + n) * H + h;
                 uint8_t* d = sStage + st * STAGE_BYTES;
@@ -984,19 +986,35 @@ tc_chain_fwd_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
 // turn into the state chains, whose loads wait for those flags; the other CTAs keep producing, and a CTA
 // whose chain is finished joins them again.  No worker ever waits, so the chains always make progress.
 // ---------------------------------------------------------------------------------------------
+constexpr float FWD_STEP_OVER_TILE_F = 0.65f;   // cost of a chain step in units of the time one SM needs for a tile
 struct FwdSched {
     int* tickets;     // zero at launch
-    int ntickets;     // chunk positions x chains
+    int ntickets;     // number of (chunk, head) tiles
     int nchains;
-    int nchunks;      // chunk positions per chain (sequences of equal length)
+    int nchunks;      // dense batch: chunk positions per chain (sequences of equal length)
     int switch_at;
+    const int* order; // packed batch: the chunks sorted by position inside their sequence (else null); then
+                      // ntickets and switch_at are worked out on the device from the chunk table
+    const int* longest;   // packed batch: chunks of the longest sequence
+    int nseq, feeders;
 };
-constexpr int FWD_GROUPS = 4;
-constexpr int FWD_THREADS = FWD_GROUPS * CL_THREADS;
-constexpr uint32_t FWD_GROUP_SMEM = (uint32_t)CL_SMEM - 1024;
-static_assert(FWD_GROUPS * FWD_GROUP_SMEM + FWD_GROUPS * sizeof(ClGroupShared) <= CF_SMEM - 1024, "worker groups fit");
-static_assert(FWD_THREADS >= CFW_THREADS, "the chain fits into the CTA");
 
+// Packed batches: the realised number of tiles and the longest chain are only known on the device.
+__device__ __forceinline__ void fwd_sched_resolve(FwdSched& sc, const Table& tab, int H)
+{
+    if (!sc.order) return;
+    sc.ntickets = tab.seq_chunk0(sc.nseq) * H;
+    const float fed = (float)sc.feeders * (float)(*sc.longest) * FWD_STEP_OVER_TILE_F;
+    sc.switch_at = max(0, sc.ntickets - (int)fed);
+}
+// Worker groups per CTA: four (1024 threads, 64 registers: the chain role loses about a tenth of its speed)
+// when the chunk-local tiles are the larger part of the work, three (768 threads, 80 registers) when the
+// longest chain is.
+constexpr uint32_t FWD_GROUP_SMEM = (uint32_t)CL_SMEM - 1024;
+static_assert(4 * FWD_GROUP_SMEM + 4 * sizeof(ClGroupShared) <= CF_SMEM - 1024, "worker groups fit");
+static_assert(3 * CL_THREADS >= CFW_THREADS, "the chain fits into the CTA");
+
+template <int FWD_GROUPS>
 __device__ __forceinline__ void chunk_fwd_workers(const CUtensorMap& tmK, const CUtensorMap& tmQ,
                                                   const CUtensorMap& tmKt, const TcChunkArgs& cl, const FwdSched& sc,
                                                   int limit, uint8_t* sm, uint32_t tb)
@@ -1030,9 +1048,17 @@ __device__ __forceinline__ void chunk_fwd_workers(const CUtensorMap& tmK, const 
         const int t = gs.ticket;
         if (t < 0) break;
         if (ltid == 0) next = draw();
-        const int n = t / sc.nchains, chain = t - n * sc.nchains;
-        const int s = chain / cl.H, h = chain - s * cl.H;
-        const int c = s * sc.nchunks + n;
+        int c, h;
+        if (sc.order) {   // packed batch: position-major order from the sorted list, heads innermost
+            const int j = t / cl.H;
+            h = t - j * cl.H;
+            c = sc.order[j];
+        } else {
+            const int n = t / sc.nchains, chain = t - n * sc.nchains;
+            const int s = chain / cl.H;
+            h = chain - s * cl.H;
+            c = s * sc.nchunks + n;
+        }
         chunk_fwd_tile(tmK, tmQ, tmKt, cl, c, h, sm + g * FWD_GROUP_SMEM, gs, tb + g * 128, ltid, 1 + g, ph, publish);
         publish = cl.ready + (size_t)c * cl.H + h;
         ph ^= 1;
@@ -1051,11 +1077,13 @@ __device__ __forceinline__ void chunk_fwd_workers(const CUtensorMap& tmK, const 
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(FWD_THREADS, 1)
+template <int FWD_GROUPS>
+__global__ void __launch_bounds__(FWD_GROUPS * CL_THREADS, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
               const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmV, TcChunkArgs cl,
-              TcChainArgs ch, FwdSched sc)
+              TcChainArgs ch, FwdSched sched)
 {
+    FwdSched sc = sched;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* sm = align1024(smem_raw);
     __shared__ uint32_t tmem_base;
@@ -1064,10 +1092,13 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_base;
+    fwd_sched_resolve(sc, cl.tab, cl.H);
     const bool chain_cta = (int)blockIdx.x < sc.nchains;
+    // packed batch: a chain starts when the tickets reach its own first tile (short sequences start late)
+    if (chain_cta && sc.order) sc.switch_at = max(sc.switch_at, cl.tab.seq_first_[blockIdx.x / cl.H] * cl.H);
 #pragma unroll 1
     for (int pass = 0; pass < 2; ++pass) {   // one copy of the worker code: it has to stay in the instruction cache
-        chunk_fwd_workers(tmK, tmQ, tmKt, cl, sc, chain_cta && pass == 0 ? sc.switch_at : sc.ntickets, sm, tb);
+        chunk_fwd_workers<FWD_GROUPS>(tmK, tmQ, tmKt, cl, sc, chain_cta && pass == 0 ? sc.switch_at : sc.ntickets, sm, tb);
         if (!chain_cta || pass == 1) break;
         chain_fwd_role(tmV, tmKt, ch, blockIdx.x, sm, tb);
     }
@@ -2276,7 +2307,7 @@ template <typename F> bool set_smem(F* kernel, size_t bytes)
 // Merged forward launch: SMs that must be left over to feed the chains, and the cost of one chain step in
 // units of the time one SM needs for a tile of the chunk-local pass (measured: 0.6 to 0.75 are equally good).
 constexpr int FWD_MIN_FEEDERS = 32;
-constexpr double FWD_STEP_OVER_TILE = 0.65;
+constexpr double FWD_STEP_OVER_TILE = FWD_STEP_OVER_TILE_F;
 
 int launch_wait_timeout_selftest(int* status, long long limit_cycles, int code, cudaStream_t st)
 {
@@ -2326,7 +2357,7 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
     // chains want) and enough SMs are left over to feed the chains.
     const int grid = num_sms(), nchains = S * H;
     const int nchunks = p.nseq > 0 ? 0 : (p.T + CH - 1) / CH;
-    if (p.nseq == 0 && nchunks > 0 && nchains + FWD_MIN_FEEDERS <= grid) {
+    if (nchains + FWD_MIN_FEEDERS <= grid) {
         const size_t rbytes = sizeof(int) * (64 + (size_t)L.NTmax * H);
         if (cudaMemsetAsync(w + t.ready, 0, rbytes, st) != cudaSuccess) return -1;
         FwdSched sc{};
@@ -2334,15 +2365,29 @@ int tc_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void* w
         sc.nchains = nchains;
         sc.nchunks = nchunks;
         sc.ntickets = nchunks * nchains;
+        sc.nseq = S;
+        sc.feeders = grid - nchains;
         // The chains start once the feeders alone can keep up with them to the end: a chain step costs
         // about FWD_STEP_OVER_TILE of the time one SM needs for a tile.
         const double fed = (double)(grid - nchains) * nchunks * FWD_STEP_OVER_TILE;
         sc.switch_at = (int)std::max(0.0, (double)sc.ntickets - fed);
+        if (p.nseq > 0) {   // both are worked out on the device from the chunk table
+            sc.order = tab.order_;
+            sc.longest = tab.pos_;
+        }
         ca.ready = sc.tickets + 64;
         ch.ready = sc.tickets + 64;
-        if (!set_smem(tc_fwd_kernel, CF_SMEM)) return -1;
+        // Three worker groups when the longest chain outweighs the tiles (packed batches: their longest
+        // sequence is not known here, and a long tail is what packing produces), four otherwise.
+        const bool chain_bound = p.nseq > 0 || (double)nchunks * 2.3 > 1.5 * (double)sc.ntickets * 5.5 / grid;
         stage_mark(st, "tc_fwd");
-        tc_fwd_kernel<<<grid, FWD_THREADS, CF_SMEM, st>>>(tmK, tmQ, tmKt, tmV, ca, ch, sc);
+        if (chain_bound) {
+            if (!set_smem(tc_fwd_kernel<3>, CF_SMEM)) return -1;
+            tc_fwd_kernel<3><<<grid, 3 * CL_THREADS, CF_SMEM, st>>>(tmK, tmQ, tmKt, tmV, ca, ch, sc);
+        } else {
+            if (!set_smem(tc_fwd_kernel<4>, CF_SMEM)) return -1;
+            tc_fwd_kernel<4><<<grid, 4 * CL_THREADS, CF_SMEM, st>>>(tmK, tmQ, tmKt, tmV, ca, ch, sc);
+        }
         ++launches;
     } else {
         if (!set_smem(tc_chunk_fwd_kernel, CL_SMEM)) return -1;
