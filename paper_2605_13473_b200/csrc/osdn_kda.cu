@@ -14,7 +14,7 @@
 namespace osdn {
 namespace {
 
-constexpr int KF_WARPS = 8;    // forward: state rows per CTA
+constexpr int KF_WARPS = 16;   // forward: state rows per CTA
 constexpr int KB_WARPS = 32;   // backward: state rows per CTA
 
 template <int R> struct Vec {
@@ -115,13 +115,61 @@ template <int R> __device__ __forceinline__ float row_step(Vec<R>& S, const Tok<
     return u;
 }
 
+// A block of KTB tokens of one chain in shared memory, filled with cp.async by the whole CTA: every row-warp
+// of the CTA needs the same k, ktil, gate and q of a token, so they are fetched once per CTA instead of once
+// per warp (which made the forward bound by L2 bandwidth: 1.5 KB per token and warp).
+constexpr int KTB = 8;
+template <typename T, int K> struct TokBlock {
+    T k[KTB][K];
+    T q[KTB][K];
+    float kt[KTB][K];
+    float g[KTB][K];
+};
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit_group() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// tokens [t, t + n) of the chain, n <= KTB; th0: token-head index of token t
+template <typename T, int K>
+__device__ __forceinline__ void fill_block(TokBlock<T, K>& blk, const KdaArgs& a, size_t th0, int H, int n, int tid, int nthreads)
+{
+    constexpr int PT = K * sizeof(T) / 16, PF = K * 4 / 16;   // 16-byte pieces per row
+    constexpr int PER = 2 * PT + 2 * PF;
+    for (int p = tid; p < n * PER; p += nthreads) {
+        const int j = p / PER, r = p - j * PER;
+        const size_t row = (th0 + (size_t)j * H) * K;
+        if (r < PT) cp_async16(reinterpret_cast<char*>(blk.k[j]) + r * 16, reinterpret_cast<const char*>(static_cast<const T*>(a.k) + row) + r * 16);
+        else if (r < 2 * PT) cp_async16(reinterpret_cast<char*>(blk.q[j]) + (r - PT) * 16, reinterpret_cast<const char*>(static_cast<const T*>(a.q) + row) + (r - PT) * 16);
+        else if (r < 2 * PT + PF) cp_async16(reinterpret_cast<char*>(blk.kt[j]) + (r - 2 * PT) * 16, reinterpret_cast<const char*>(a.ktil + row) + (r - 2 * PT) * 16);
+        else cp_async16(reinterpret_cast<char*>(blk.g[j]) + (r - 2 * PT - PF) * 16, reinterpret_cast<const char*>(a.gate + row) + (r - 2 * PT - PF) * 16);
+    }
+}
+
+template <typename T, int K, int R>
+__device__ __forceinline__ Tok<R> tok_from_block(const TokBlock<T, K>& blk, int j, int lane, float v, float beta)
+{
+    Tok<R> t;
+    t.k = load_vec<R>(blk.k[j] + R * lane);
+    t.kt = load_vec<R>(blk.kt[j] + R * lane);
+    t.g = load_vec<R>(blk.g[j] + R * lane);
+    t.v = v;
+    t.beta = beta;
+    return t;
+}
+
 template <typename T, int K>
 __global__ void __launch_bounds__(KF_WARPS * 32) kda_fwd_kernel(KdaArgs a)
 {
     constexpr int R = K / 32;
+    __shared__ __align__(16) TokBlock<T, K> blk[2];
     const int H = a.H, V = a.V;
     const int chain = blockIdx.y, s = chain / H, h = chain - s * H;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int row = blockIdx.x * KF_WARPS + warp;
     const int t0 = a.tab.seq_tok0(s), len = a.tab.seq_len(s), c0 = a.tab.seq_chunk0(s);
     const size_t srow = (((size_t)s * H + h) * V + row) * K + R * lane;
@@ -130,28 +178,45 @@ __global__ void __launch_bounds__(KF_WARPS * 32) kda_fwd_kernel(KdaArgs a)
     else
 #pragma unroll
         for (int x = 0; x < R; ++x) S.x[x] = 0.f;
-    if (len > 0) {
-        Tok<R> cur = load_tok<T, R>(a, (size_t)t0 * H + h, K, row, lane);
-        Vec<R> qc = load_vec<R>(static_cast<const T*>(a.q) + ((size_t)t0 * H + h) * K + R * lane);
-        for (int t = 0; t < len; ++t) {
+    const int nblk = (len + KTB - 1) / KTB;
+    // per-row scalars of a block (lane j < KTB: v of token j for this row; lane KTB + j: beta), one block ahead
+    auto scalars = [&](int bi) {
+        const int j = lane & (KTB - 1), t = bi * KTB + j;
+        float x = 0.f;
+        if (bi < nblk && t < len && lane < 2 * KTB) {
             const size_t th = (size_t)(t0 + t) * H + h;
-            Tok<R> nxt = cur;
-            Vec<R> qn = qc;
-            if (t + 1 < len) {   // the next token's operands are in flight while this one is worked on
-                nxt = load_tok<T, R>(a, th + H, K, row, lane);
-                qn = load_vec<R>(static_cast<const T*>(a.q) + (th + H) * K + R * lane);
-            }
+            x = lane < KTB ? ldf(static_cast<const T*>(a.v) + th * V + row) : a.beta[th];
+        }
+        return x;
+    };
+    if (nblk > 0) fill_block<T, K>(blk[0], a, (size_t)t0 * H + h, H, min(KTB, len), tid, KF_WARPS * 32);
+    cp_async_commit_group();
+    float sc = scalars(0);
+    for (int bi = 0; bi < nblk; ++bi) {
+        const int tb0 = bi * KTB, n = min(KTB, len - tb0);
+        if (bi + 1 < nblk)
+            fill_block<T, K>(blk[(bi + 1) & 1], a, (size_t)(t0 + tb0 + KTB) * H + h, H, min(KTB, len - tb0 - KTB), tid, KF_WARPS * 32);
+        cp_async_commit_group();
+        const float sc_next = scalars(bi + 1);
+        cp_async_wait_group<1>();
+        __syncthreads();   // the block has landed for every warp
+        const TokBlock<T, K>& B = blk[bi & 1];
+        for (int j = 0; j < n; ++j) {
+            const int t = tb0 + j;
+            const size_t th = (size_t)(t0 + t) * H + h;
             if (a.ckpt && (t % CH) == 0)
                 store_vec<R>(a.ckpt + (((size_t)(c0 + t / CH) * H + h) * V + row) * K + R * lane, S);
+            const Tok<R> cur = tok_from_block<T, K, R>(B, j, lane, __shfl_sync(0xffffffffu, sc, j), __shfl_sync(0xffffffffu, sc, KTB + j));
+            const Vec<R> qc = load_vec<R>(B.q[j] + R * lane);
             row_step<R>(S, cur, nullptr);
             float o = 0.f;
 #pragma unroll
             for (int x = 0; x < R; ++x) o = fmaf(S.x[x], qc.x[x], o);
             o = a.scale * warp_sum(o);
             if (lane == 0) stf(static_cast<T*>(a.out) + th * V + row, o);
-            cur = nxt;
-            qc = qn;
         }
+        sc = sc_next;
+        __syncthreads();   // everybody is done with the block before it is refilled
     }
     if (a.final_state) store_vec<R>(a.final_state + srow, S);
 }
