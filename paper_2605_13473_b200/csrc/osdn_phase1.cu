@@ -303,6 +303,7 @@ struct P1Fwd {
     P1Regions r;
     int save;
     Hyper hy;
+    int* status;         // device status word (bounded waits of the pipelined stretches report here)
 };
 
 // Eight consecutive values of a row as floats (one 16-byte load for bf16, two for fp32).
@@ -443,10 +444,199 @@ template <int R> __device__ __forceinline__ bool on_lower_face(const float (&d)[
     return __all_sync(0xffffffffu, f);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Pipelined stretches of the sequential pass.  Where nearly every token is processed (a preconditioner
+// that really moves), the walk of a chain is bound by the instructions one warp issues per token, most
+// of which do not depend on d: fetching and squaring the key, the step's scalars, forming and storing
+// the write key, the records for the backward.  For such a stretch three warps share the chain:
+//   pre   fetches a block of PB tokens and leaves k, k^2 and the scalars (e, a2, rho) in shared memory;
+//   core  carries d through the block: <d, k^2>, the step, the projection; leaves d_t and the mask;
+//   post  forms ktil_t = d_t (.) k_t and writes ktil, d_t and the mask words to global memory.
+// Blocks go round a ring of PN buffers; the roles meet at mbarriers (full: pre -> core and post,
+// done: core -> post, free: post -> pre).  Every token of a stretch is processed (none is skipped: for a
+// flagged token entered on the face the step returns to the face by construction, so the values are
+// the ones the skipping walk leaves), which keeps the core free of any bookkeeping.
+// ---------------------------------------------------------------------------------------------
+constexpr int PB = 16, PN = 3;
+constexpr int P1_ERR_PIPE = 131;
+constexpr long long P1_WAIT_LIMIT = 4000000000ll;   // about two seconds
+
+__device__ __forceinline__ void p1_mbar_init(uint64_t* b, int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(b)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void p1_mbar_arrive(uint64_t* b)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"((uint32_t)__cvta_generic_to_shared(b)) : "memory");
+}
+// Bounded: gives up after P1_WAIT_LIMIT cycles, records the error and returns false.
+__device__ __forceinline__ bool p1_mbar_wait(uint64_t* b, uint32_t parity, int* status)
+{
+    const uint32_t addr = (uint32_t)__cvta_generic_to_shared(b);
+    const long long t0 = clock64();
+    while (true) {
+        uint32_t ok;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(ok)
+                     : "r"(addr), "r"(parity)
+                     : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > P1_WAIT_LIMIT) {
+            if (status) atomicCAS(status, 0, P1_ERR_PIPE);
+            return false;
+        }
+    }
+}
+
+template <typename TI, int K, bool VEC> struct PipeBuf {
+    static constexpr int R = K / 32;
+    float kap[PB][K];                       // k^2
+    RawRow<TI, R> kraw[PB][32];             // k as it sits in memory
+    float dt[PB][K];                        // d_t (pre-update), written by the core
+    float rhov[VEC ? PB : 1][VEC ? K : 1];  // vector retention: exp(l_t) per coordinate
+    float4 scal[PB];                        // e = eta b / n, a2 = e b, rho, -
+    unsigned mask[PB][32];                  // projection pass bits of lane l's coordinates
+};
+struct PipeBars {
+    uint64_t full[PN], done[PN], free_[PN];
+};
+
+// tokens [t_a, t_b) of the chain (packed token indices), all three roles; d: the core's registers
+template <typename TI, typename TO, int K, bool VEC>
+__device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int t_b, float (&d)[K / 32],
+                                             PipeBuf<TI, K, VEC>* buf, PipeBars& bars, uint32_t& round0, int role, int lane)
+{
+    constexpr int R = K / 32;
+    const int H = a.H;
+    const Hyper hy = a.hy;
+    const int nblk = (t_b - t_a + PB - 1) / PB;
+    const TI* kp = static_cast<const TI*>(a.k);
+    bool ok = true;
+    // block b uses buffer b % PN; its barriers complete once per use: parity of the use count
+    const uint32_t base = round0;   // uses of the ring before this stretch (a multiple of PN blocks is not required)
+    if (role == 1) {
+        // ------------------------------------------------------------------ pre
+        for (int b = 0; b < nblk && ok; ++b) {
+            const uint32_t use = base + b;
+            const int bi = use % PN;
+            if (use >= PN) ok = p1_mbar_wait(&bars.free_[bi], ((use / PN) - 1) & 1, a.status);
+            if (!ok) break;
+            PipeBuf<TI, K, VEC>& B = buf[bi];
+            const int t0 = t_a + b * PB, n = min(PB, t_b - t0);
+            RawRow<TI, R> raw[PB];
+#pragma unroll
+            for (int j = 0; j < PB; ++j) {
+                const size_t th = (size_t)(t0 + min(j, n - 1)) * H + h;
+                load_raw<R>(kp + th * K, lane, raw[j]);
+            }
+            if (lane < n) {
+                const size_t th = (size_t)(t0 + lane) * H + h;
+                const float rn = fabsf(a.r.n[th]), bb = hy.beta_aware ? a.beta[th] : 1.0f;
+                const float e = hy.eta * bb * rn;
+                B.scal[lane] = make_float4(e, e * bb, a.r.rho[th], 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < PB; ++j) {
+                float kk[R], kap[R];
+                unpack<R>(raw[j], kk);
+#pragma unroll
+                for (int r = 0; r < R; ++r) kap[r] = kk[r] * kk[r];
+                store_row<R>(B.kap[j], lane, kap);
+                B.kraw[j][lane] = raw[j];
+            }
+            if constexpr (VEC) {
+                for (int j = 0; j < n; ++j) {
+                    const size_t th = (size_t)(t0 + j) * H + h;
+                    float lr[R];
+                    load_row<R>(a.retsrc + th * K, lane, lr);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) lr[r] = expf(lr[r]);
+                    store_row<R>(B.rhov[VEC ? j : 0], lane, lr);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.full[bi]);
+        }
+    } else if (role == 0) {
+        // ------------------------------------------------------------------ core
+        for (int b = 0; b < nblk && ok; ++b) {
+            const uint32_t use = base + b;
+            const int bi = use % PN;
+            ok = p1_mbar_wait(&bars.full[bi], (use / PN) & 1, a.status);
+            if (!ok) break;
+            PipeBuf<TI, K, VEC>& B = buf[bi];
+            const int n = min(PB, t_b - (t_a + b * PB));
+            for (int j = 0; j < n; ++j) {
+                const float4 sc = B.scal[j];
+                float kap[R], rho[R];
+                load_row<R>(B.kap[j], lane, kap);
+                if constexpr (VEC) load_row<R>(B.rhov[VEC ? j : 0], lane, rho);
+                else {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) rho[r] = sc.z;
+                }
+                float al = 0.f;
+#pragma unroll
+                for (int r = 0; r < R; ++r) al = fmaf(d[r], kap[r], al);
+                store_row<R>(B.dt[j], lane, d);
+                al = warp_sum(al);
+                const float cc = fmaf(-sc.y, al, sc.x);
+                unsigned mybits = 0;
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float x = fmaf(cc, kap[r], rho[r] * d[r]);
+                    bool pz = true;
+                    if (hy.clamp) {
+                        pz = (x >= hy.d_min) && (x <= hy.d_max);
+                        x = fminf(fmaxf(x, hy.d_min), hy.d_max);
+                    }
+                    mybits |= pz ? (1u << r) : 0u;
+                    d[r] = x;
+                }
+                B.mask[j][lane] = mybits;
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.done[bi]);
+        }
+    } else {
+        // ------------------------------------------------------------------ post
+        TO* kt = static_cast<TO*>(a.ktil);
+        for (int b = 0; b < nblk && ok; ++b) {
+            const uint32_t use = base + b;
+            const int bi = use % PN;
+            ok = p1_mbar_wait(&bars.done[bi], (use / PN) & 1, a.status);
+            if (!ok) break;
+            const PipeBuf<TI, K, VEC>& B = buf[bi];
+            const int t0 = t_a + b * PB, n = min(PB, t_b - t0);
+            for (int j = 0; j < n; ++j) {
+                const size_t th = (size_t)(t0 + j) * H + h;
+                float dd[R], kk[R], wk[R];
+                load_row<R>(B.dt[j], lane, dd);
+                unpack<R>(B.kraw[j][lane], kk);
+#pragma unroll
+                for (int r = 0; r < R; ++r) wk[r] = dd[r] * kk[r];
+                store_row<R>(kt + th * K, lane, wk);
+                if (a.save) {
+                    store_row<R>(a.r.dtraj + th * K, lane, dd);
+                    a.r.pmask[th * 32 + lane] = B.mask[j][lane];
+                }
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.free_[bi]);
+        }
+    }
+    round0 = base + nblk;
+    return ok;
+}
+
 // one warp per chain.  Flag words are fetched for 32 chunks at a time (one chunk per lane); the
 // rows of the tokens that are really processed are prefetched a few tokens ahead.
+// A chunk of which at least PIPE_TRIGGER tokens had to be processed starts a pipelined stretch of up to
+// PIPE_CHUNKS chunks; stretches follow one another while d stays off the lower face.
+constexpr int PIPE_TRIGGER = 32, PIPE_CHUNKS = 8;
+
 template <typename TI, typename TO, int K, bool VEC>
-__global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
+__global__ void __launch_bounds__(96) phase1_seq_kernel(P1Fwd a)
 {
     constexpr int R = K / 32;
     constexpr int PF = 8;   // prefetch distance in tokens
@@ -455,12 +645,36 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
         RawRow<float, R> lr[VEC ? 32 : 1];
         float n[32], rho[32], beta[32];
     };
-    __shared__ __align__(16) RingSlot ring_all[4][PF];
-    RingSlot* ring = ring_all[threadIdx.x >> 5];
-    const int lane = threadIdx.x & 31;
-    const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (chain >= a.S * a.H) return;
+    extern __shared__ __align__(16) uint8_t p1_dyn[];   // PipeBuf[PN]
+    PipeBuf<TI, K, VEC>* pbuf = reinterpret_cast<PipeBuf<TI, K, VEC>*>(p1_dyn);
+    __shared__ __align__(16) RingSlot ring[PF];
+    __shared__ PipeBars bars;
+    __shared__ int cmd[2];   // token range of the next pipelined stretch; empty: the chain is finished
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chain = blockIdx.x;
     const int s = chain / a.H, h = chain % a.H, H = a.H;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < PN; ++i) {
+            p1_mbar_init(&bars.full[i], 1);
+            p1_mbar_init(&bars.done[i], 1);
+            p1_mbar_init(&bars.free_[i], 1);
+        }
+    }
+    __syncthreads();
+    uint32_t pipe_uses = 0;   // blocks that have gone through the ring so far (the same in all three warps)
+    if (warp != 0) {
+        // helper warps (1: pre, 2: post) serve the stretches warp 0 announces
+        float none[R];
+        while (true) {
+            asm volatile("bar.sync 1, 96;" ::: "memory");
+            const int t_a = cmd[0], t_b = cmd[1];
+            if (t_b <= t_a) break;
+            pipe_stretch<TI, TO, K, VEC>(a, h, t_a, t_b, none, pbuf, bars, pipe_uses, warp, lane);
+            asm volatile("bar.sync 2, 96;" ::: "memory");
+        }
+        return;
+    }
+    bool pipe_next = false;
     const TI* kp = static_cast<const TI*>(a.k);
     TO* kt = static_cast<TO*>(a.ktil);
     const Hyper hy = a.hy;
@@ -508,6 +722,29 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
             allflag = __ballot_sync(0xffffffffu, cl < c1 && (bl & vl) == vl);
         }
         for (int c = cbase; c < cend; ++c) {
+            if (pipe_next) {
+                // a pipelined stretch: every token of the next chunks (of this group) is processed
+                const int np = min(PIPE_CHUNKS, cend - c);
+                const int nrel = c - c0;
+                const int t_a = seq_t0 + nrel * CH, t_b = seq_t0 + min(seq_len, (nrel + np) * CH);
+                if (lane == 0) {
+                    cmd[0] = t_a;
+                    cmd[1] = t_b;
+                }
+                cp_async_wait<0>();   // nothing of the token-by-token walk is still on its way
+                asm volatile("bar.sync 1, 96;" ::: "memory");
+                const bool okp = pipe_stretch<TI, TO, K, VEC>(a, h, t_a, t_b, d, pbuf, bars, pipe_uses, 0, lane);
+                asm volatile("bar.sync 2, 96;" ::: "memory");
+                if (a.save && lane < np) {
+                    const size_t tl = (size_t)(c + lane) * H + h;
+                    a.r.skipw[tl * 2] = 0u;
+                    a.r.skipw[tl * 2 + 1] = 0u;
+                }
+                face = on_lower_face<R>(d, hy);
+                pipe_next = okp && !face;
+                c += np - 1;
+                continue;
+            }
             if (face) {
                 // a run of fully flagged chunks entered on the face is skipped in one go
                 const unsigned rest = ~allflag >> (c - cbase);
@@ -532,6 +769,7 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
                                             ((unsigned long long)__shfl_sync(0xffffffffu, w1, c - cbase) << 32);
             const unsigned long long valid = len >= 64 ? ~0ull : ((1ull << len) - 1ull);
             unsigned long long skipped = 0ull;
+            int processed = 0;
             if (face && (bits & valid) == valid) {
                 skipped = valid;
             } else {
@@ -619,6 +857,7 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
                                 if (a.save) a.r.pmask[th * 32 + lane] = mybits;
                                 face = __all_sync(0xffffffffu, at_min);
                                 ++i;
+                                ++processed;
                                 // back on the face with a flagged token next: leave the run
                                 stop = face && i < len && ((bits >> i) & 1ull);
                             }
@@ -630,10 +869,16 @@ __global__ void __launch_bounds__(128) phase1_seq_kernel(P1Fwd a)
                 a.r.skipw[tile * 2] = (unsigned)(skipped & 0xffffffffull);
                 a.r.skipw[tile * 2 + 1] = (unsigned)(skipped >> 32);
             }
+            pipe_next = processed >= PIPE_TRIGGER && !face;
         }
     }
     if (a.d_final) store_row<R>(a.d_final + ((size_t)s * H + h) * K, lane, d);
     cp_async_wait<0>();   // rows fetched past the last processed token are not used, but must have landed
+    if (lane == 0) {      // release the helper warps
+        cmd[0] = 0;
+        cmd[1] = 0;
+    }
+    asm volatile("bar.sync 1, 96;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -915,8 +1160,15 @@ int fwd_launch(const P1Fwd& a, cudaStream_t st)
     if (a.hy.apf_mode == 3) phase1_spec_kernel<TI, TO, K, true><<<gspec, 128, 0, st>>>(a);
     else phase1_spec_kernel<TI, TO, K, false><<<gspec, 128, 0, st>>>(a);
     stage_mark(st, "phase1_seq");
-    if (a.hy.apf_mode == 3) phase1_seq_kernel<TI, TO, K, true><<<gseq, 128, 0, st>>>(a);
-    else phase1_seq_kernel<TI, TO, K, false><<<gseq, 128, 0, st>>>(a);
+    const unsigned chains = (unsigned)(a.S * a.H);
+    auto launch_seq = [&](auto kernel, size_t smem) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        kernel<<<chains, 96, smem, st>>>(a);
+        return true;
+    };
+    const bool okl = a.hy.apf_mode == 3 ? launch_seq(phase1_seq_kernel<TI, TO, K, true>, PN * sizeof(PipeBuf<TI, K, true>))
+                                        : launch_seq(phase1_seq_kernel<TI, TO, K, false>, PN * sizeof(PipeBuf<TI, K, false>));
+    if (!okl) return -1;
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
@@ -947,6 +1199,7 @@ int phase1_forward(const osdn_params& p, const Hyper& hy, const WsLayout& L, voi
     f.S = L.S; f.H = p.H; f.NT = L.NTmax; f.tab = carve_table(ws, L);
     f.k = a.k; f.beta = a.beta; f.retsrc = p.apf_mode >= 2 ? a.log_ret : a.gate; f.d0 = a.precond_in;
     f.ktil = ktil; f.d_final = a.precond_out; f.r = carve_p1(ws, L); f.save = save ? 1 : 0; f.hy = hy;
+    f.status = reinterpret_cast<int*>(static_cast<char*>(ws) + L.status);
     if (p.io_dtype == OSDN_FP32) {
         if (ktil_bf16) return -1;
         return p.K == 64 ? fwd_launch<float, float, 64>(f, st) : fwd_launch<float, float, 128>(f, st);
