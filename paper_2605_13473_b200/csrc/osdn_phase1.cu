@@ -894,6 +894,7 @@ struct P1Bwd {
     float *dbeta, *dgate, *dlog_ret, *dprecond_in;
     P1Regions r;
     Hyper hy;
+    int* status;
 };
 
 // skipped tokens: dk = dk_read + d_min dL/dktil (one warp per (chunk, head, 32-token half))
@@ -924,11 +925,204 @@ __global__ void __launch_bounds__(128) phase1_bwd_bulk_kernel(P1Bwd a)
     }
 }
 
-// processed tokens, in reverse; one warp per chain.  Skip words are fetched for 32 chunks at a time.
-constexpr int P1B_WARPS = 2;   // chains per CTA (the ring of a chain takes up to 14 KB of shared memory)
+// ---------------------------------------------------------------------------------------------
+// Pipelined stretches of the reverse pass, the mirror image of the forward ones: over chunks in which
+// every token was processed, lambda = dL/dd flows without a restart, and of a token's work only
+//     lambda <- mask (.) lambda ;  dc = <lambda, k^2> ;  lambda <- rho lambda - a2 dc k^2 + k (.) dL/dktil
+// depends on lambda.  Three warps share the chain:
+//   pre   fetches a block of QB tokens (k, d_t, dL/dktil, dk_read, mask, scalars) and recomputes the
+//         step's own scalars (<d_t, k^2>, c, the factors of the beta and normaliser gradients);
+//   core  carries lambda through the block (top token first) and leaves the masked lambda and dc;
+//   post  forms dk, the retention and beta gradients from those and writes them out.
+// ---------------------------------------------------------------------------------------------
+constexpr int QB = 8, QN = 3;
+
+template <typename T, int K, bool VEC> struct RevBuf {
+    static constexpr int R = K / 32;
+    RawRow<T, R> kraw[QB][32];
+    float dt[QB][K], dkt[QB][K], dkr[QB][K];
+    float lam[QB][K];                       // masked lambda of the token, written by the core
+    float rv[VEC ? QB : 1][VEC ? K : 1];    // vector retention: exp(l_t)
+    unsigned mask[QB][32];
+    float4 sc0[QB];                         // a2, rho, cc, g1
+    float4 sc1[QB];                         // g2, dc (written by the core), -, -
+};
+
+// tokens [t_lo, t_hi) of the chain in reverse, all three roles; lam: the core's registers
+template <typename T, int K, bool VEC>
+__device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int t_hi, float (&lam)[K / 32],
+                                            RevBuf<T, K, VEC>* buf, PipeBars& bars, uint32_t& round0, int role, int lane)
+{
+    constexpr int R = K / 32;
+    const int H = a.H;
+    const Hyper hy = a.hy;
+    const int nblk = (t_hi - t_lo + QB - 1) / QB;
+    const T* kp = static_cast<const T*>(a.k);
+    bool ok = true;
+    const uint32_t base = round0;
+    // block b: tokens t_hi - 1 - (b QB + j), j = 0 .. n - 1 (slot j of the buffer)
+    if (role == 1) {
+        for (int b = 0; b < nblk && ok; ++b) {
+            const uint32_t use = base + b;
+            const int bi = use % QN;
+            if (use >= QN) ok = p1_mbar_wait(&bars.free_[bi], ((use / QN) - 1) & 1, a.status);
+            if (!ok) break;
+            RevBuf<T, K, VEC>& B = buf[bi];
+            const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
+            RawRow<T, R> rk[QB];
+            RawRow<float, R> rdt[QB], rdkt[QB], rdkr[QB];
+#pragma unroll
+            for (int j = 0; j < QB; ++j) {
+                const size_t th = (size_t)(ttop - min(j, n - 1)) * H + h;
+                load_raw<R>(kp + th * K, lane, rk[j]);
+                load_raw<R>(a.r.dtraj + th * K, lane, rdt[j]);
+                load_raw<R>(a.dktil + th * K, lane, rdkt[j]);
+                load_raw<R>(a.dkread + th * K, lane, rdkr[j]);
+            }
+            float ns = 0.f, rho = 0.f, bb = 1.f;
+            if (lane < n) {
+                const size_t th = (size_t)(ttop - lane) * H + h;
+                ns = a.r.n[th];
+                rho = a.r.rho[th];
+                bb = hy.beta_aware ? a.beta[th] : 1.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < QB; ++j) {
+                const size_t th = (size_t)(ttop - min(j, n - 1)) * H + h;
+                B.mask[j][lane] = a.r.pmask[th * 32 + lane];
+            }
+            float alv = 0.f;   // lane j keeps <d_t, k^2> of slot j
+#pragma unroll
+            for (int j = 0; j < QB; ++j) {
+                float kk[R], dd[R], al = 0.f;
+                unpack<R>(rk[j], kk);
+                unpack<R>(rdt[j], dd);
+#pragma unroll
+                for (int r = 0; r < R; ++r) al = fmaf(dd[r], kk[r] * kk[r], al);
+                al = warp_sum(al);
+                if (lane == j) alv = al;
+                B.kraw[j][lane] = rk[j];
+                *reinterpret_cast<RawRow<float, R>*>(&B.dt[j][R * lane]) = rdt[j];
+                *reinterpret_cast<RawRow<float, R>*>(&B.dkt[j][R * lane]) = rdkt[j];
+                *reinterpret_cast<RawRow<float, R>*>(&B.dkr[j][R * lane]) = rdkr[j];
+            }
+            if (lane < n) {
+                const float rn = fabsf(ns);
+                const float e = hy.eta * bb * rn, a2 = e * bb;
+                const float cc = fmaf(-a2, alv, e);
+                const float g1 = hy.eta * (1.0f - 2.0f * bb * alv) * rn;
+                const float g2 = ns > 0.f ? -cc * rn : 0.f;
+                B.sc0[lane] = make_float4(a2, rho, cc, g1);
+                B.sc1[lane].x = g2;
+            }
+            if constexpr (VEC) {
+                for (int j = 0; j < n; ++j) {
+                    const size_t th = (size_t)(ttop - j) * H + h;
+                    float lr[R];
+                    load_row<R>(a.log_ret + th * K, lane, lr);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) lr[r] = expf(lr[r]);
+                    store_row<R>(B.rv[VEC ? j : 0], lane, lr);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.full[bi]);
+        }
+    } else if (role == 0) {
+        for (int b = 0; b < nblk && ok; ++b) {
+            const uint32_t use = base + b;
+            const int bi = use % QN;
+            ok = p1_mbar_wait(&bars.full[bi], (use / QN) & 1, a.status);
+            if (!ok) break;
+            RevBuf<T, K, VEC>& B = buf[bi];
+            const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
+            for (int j = 0; j < n; ++j) {
+                const float4 s0 = B.sc0[j];
+                const unsigned mw = B.mask[j][lane];
+                float kk[R], dkt[R], rv[R];
+                unpack<R>(B.kraw[j][lane], kk);
+                load_row<R>(B.dkt[j], lane, dkt);
+                if constexpr (VEC) load_row<R>(B.rv[VEC ? j : 0], lane, rv);
+                else {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) rv[r] = s0.y;
+                }
+                float kap[R], dc = 0.f;
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    kap[r] = kk[r] * kk[r];
+                    if (!((mw >> r) & 1u)) lam[r] = 0.f;
+                    dc = fmaf(lam[r], kap[r], dc);
+                }
+                store_row<R>(B.lam[j], lane, lam);
+                dc = warp_sum(dc);
+                const float da = -s0.x * dc;
+#pragma unroll
+                for (int r = 0; r < R; ++r) lam[r] = fmaf(rv[r], lam[r], fmaf(da, kap[r], kk[r] * dkt[r]));
+                if (lane == 0) B.sc1[j].y = dc;
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.done[bi]);
+        }
+    } else {
+        T* dkp = static_cast<T*>(a.dk);
+        for (int b = 0; b < nblk && ok; ++b) {
+            const uint32_t use = base + b;
+            const int bi = use % QN;
+            ok = p1_mbar_wait(&bars.done[bi], (use / QN) & 1, a.status);
+            if (!ok) break;
+            const RevBuf<T, K, VEC>& B = buf[bi];
+            const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
+            for (int j = 0; j < n; ++j) {
+                const size_t th = (size_t)(ttop - j) * H + h;
+                const float4 s0 = B.sc0[j], s1 = B.sc1[j];
+                const float a2 = s0.x, rho = s0.y, cc = s0.z, g1 = s0.w, g2 = s1.x, dc = s1.y;
+                float kk[R], dt[R], dkt[R], dkr[R], lm[R];
+                unpack<R>(B.kraw[j][lane], kk);
+                load_row<R>(B.dt[j], lane, dt);
+                load_row<R>(B.dkt[j], lane, dkt);
+                load_row<R>(B.dkr[j], lane, dkr);
+                load_row<R>(B.lam[j], lane, lm);
+                float drho = 0.f;
+#pragma unroll
+                for (int r = 0; r < R; ++r) drho = fmaf(lm[r], dt[r], drho);
+                drho = warp_sum(drho);
+                const float da = -a2 * dc, dbt = g1 * dc, dn = g2 * dc;
+                if constexpr (VEC) {
+                    if (a.dlog_ret) {
+                        float rv[R], dl[R];
+                        load_row<R>(B.rv[VEC ? j : 0], lane, rv);
+#pragma unroll
+                        for (int r = 0; r < R; ++r) dl[r] = rv[r] * lm[r] * dt[r];
+                        store_row<R>(a.dlog_ret + th * K, lane, dl);
+                    }
+                }
+                float out[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float dkap = cc * lm[r] + da * dt[r] + dn;
+                    out[r] = dkr[r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
+                }
+                store_row<R>(dkp + th * K, lane, out);
+                if (lane == 0) {
+                    if (hy.beta_aware) atomicAdd(&a.dbeta[th], dbt);
+                    if (hy.apf_mode == 1) atomicAdd(&a.dgate[th], rho * drho);
+                    if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.free_[bi]);
+        }
+    }
+    round0 = base + nblk;
+    return ok;
+}
+
+// processed tokens, in reverse; one chain per CTA: warp 0 walks the chain, warps 1 and 2 serve its
+// pipelined stretches.  Skip words are fetched for 32 chunks at a time.
 
 template <typename T, int K, bool VEC>
-__global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
+__global__ void __launch_bounds__(96) phase1_bwd_seq_kernel(P1Bwd a)
 {
     constexpr int R = K / 32;
     constexpr int PF = 4;   // prefetch distance in processed tokens
@@ -939,15 +1133,37 @@ __global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
         unsigned m[32];
         float n[32], rho[32], beta[32];
     };
-    __shared__ __align__(16) BSlot ring_all[P1B_WARPS][PF];
-    BSlot* ring = ring_all[threadIdx.x >> 5];
-    const int lane = threadIdx.x & 31;
-    const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (chain >= a.S * a.H) return;
+    extern __shared__ __align__(16) uint8_t p1_dyn[];   // RevBuf[QN]
+    RevBuf<T, K, VEC>* rbuf = reinterpret_cast<RevBuf<T, K, VEC>*>(p1_dyn);
+    __shared__ __align__(16) BSlot ring[PF];
+    __shared__ PipeBars bars;
+    __shared__ int cmd[2];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chain = blockIdx.x;
     const int s = chain / a.H, h = chain % a.H, H = a.H;
     const Hyper hy = a.hy;
     const T* kp = static_cast<const T*>(a.k);
     T* dkp = static_cast<T*>(a.dk);
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < QN; ++i) {
+            p1_mbar_init(&bars.full[i], 1);
+            p1_mbar_init(&bars.done[i], 1);
+            p1_mbar_init(&bars.free_[i], 1);
+        }
+    }
+    __syncthreads();
+    uint32_t pipe_uses = 0;
+    if (warp != 0) {
+        float none[R];
+        while (true) {
+            asm volatile("bar.sync 1, 96;" ::: "memory");
+            const int t_lo = cmd[0], t_hi = cmd[1];
+            if (t_hi <= t_lo) break;
+            rev_stretch<T, K, VEC>(a, h, t_lo, t_hi, none, rbuf, bars, pipe_uses, warp, lane);
+            asm volatile("bar.sync 2, 96;" ::: "memory");
+        }
+        return;
+    }
     float lam[R];
     if (a.dprecond_out) load_row<R>(a.dprecond_out + ((size_t)s * H + h) * K, lane, lam);
     else {
@@ -1011,6 +1227,31 @@ __global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
             if ((sk & valid) == valid) {
                 lam_valid = false;
                 src = tok0;
+                continue;
+            }
+            if ((sk & valid) == 0ull) {
+                // every token of the chunk was processed: a pipelined stretch over this chunk and the ones
+                // below it of which the same holds (within this group of skip words, at most PIPE_CHUNKS)
+                int np = 1;
+                while (np < PIPE_CHUNKS && c - np >= cbot) {
+                    const int cc2 = c - np;
+                    const unsigned long long s2 = (unsigned long long)__shfl_sync(0xffffffffu, w0, ctop - 1 - cc2) |
+                                                  ((unsigned long long)__shfl_sync(0xffffffffu, w1, ctop - 1 - cc2) << 32);
+                    if (s2 != 0ull) break;   // chunks below the top one of a sequence are full
+                    ++np;
+                }
+                const int t_hi = tok0 + len, t_lo = seq_t0 + (nrel - (np - 1)) * CH;
+                if (!lam_valid) restart(src);
+                if (lane == 0) {
+                    cmd[0] = t_lo;
+                    cmd[1] = t_hi;
+                }
+                cp_async_wait<0>();
+                asm volatile("bar.sync 1, 96;" ::: "memory");
+                rev_stretch<T, K, VEC>(a, h, t_lo, t_hi, lam, rbuf, bars, pipe_uses, 0, lane);
+                asm volatile("bar.sync 2, 96;" ::: "memory");
+                lam_valid = true;
+                c -= np - 1;
                 continue;
             }
             // The tokens to process are known up front (the clear bits of the skip word), so the rows of
@@ -1149,6 +1390,11 @@ __global__ void __launch_bounds__(P1B_WARPS * 32) phase1_bwd_seq_kernel(P1Bwd a)
         store_row<R>(a.dprecond_in + ((size_t)s * H + h) * K, lane, lam);
     }
     cp_async_wait<0>();
+    if (lane == 0) {   // release the helper warps
+        cmd[0] = 0;
+        cmd[1] = 0;
+    }
+    asm volatile("bar.sync 1, 96;" ::: "memory");
 }
 
 template <typename TI, typename TO, int K>
@@ -1183,9 +1429,15 @@ int bwd_launch(const P1Bwd& a, bool bulk, cudaStream_t st)
         ++n;
     }
     stage_mark(st, "phase1_bwd_seq");
-    const unsigned gseq = (unsigned)((a.S * a.H + P1B_WARPS - 1) / P1B_WARPS);
-    if (a.hy.apf_mode == 3) phase1_bwd_seq_kernel<T, K, true><<<gseq, P1B_WARPS * 32, 0, st>>>(a);
-    else phase1_bwd_seq_kernel<T, K, false><<<gseq, P1B_WARPS * 32, 0, st>>>(a);
+    const unsigned chains = (unsigned)(a.S * a.H);
+    auto launch_seq = [&](auto kernel, size_t smem) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        kernel<<<chains, 96, smem, st>>>(a);
+        return true;
+    };
+    if (!(a.hy.apf_mode == 3 ? launch_seq(phase1_bwd_seq_kernel<T, K, true>, QN * sizeof(RevBuf<T, K, true>))
+                             : launch_seq(phase1_bwd_seq_kernel<T, K, false>, QN * sizeof(RevBuf<T, K, false>))))
+        return -1;
     ++n;
     return cudaGetLastError() == cudaSuccess ? n : -1;
 }
@@ -1218,6 +1470,7 @@ int phase1_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, vo
     b.k = a.k; b.beta = a.beta; b.dktil = dktil; b.dkread = dkread; b.dprecond_out = a.dprecond_out;
     b.dk = a.dk; b.dbeta = a.dbeta; b.dgate = a.dgate; b.dlog_ret = a.dlog_ret; b.dprecond_in = a.dprecond_in;
     b.r = carve_p1(ws, L); b.hy = hy; b.log_ret = a.log_ret;
+    b.status = reinterpret_cast<int*>(static_cast<char*>(ws) + L.status);
     // retention gradients are written for processed tokens only; a skipped token (projection mask all
     // zero) has none
     if (p.apf_mode >= 2 && a.dlog_ret) {
