@@ -60,6 +60,7 @@ struct WsLayout {
     // phase 1 (shared by both kernel families)
     size_t p1n;         // [T,H]          f32   1 / max(|k|^2, eps), negated where the floor is active
     size_t p1rho;       // [T,H]          f32   retention of the preconditioner
+    size_t p1al;        // [T,H]          f32   <d_t, k_t^2> of processed tokens                (save only)
     size_t p1flags;     // [NT,H,2]       u32   per token: the step maps d_min*1 to d_min*1, mask all zero
     size_t p1skip;      // [NT,H,2]       u32   tokens the sequential pass skipped           (save only)
     size_t pmask;       // [T,H,32]       u32   projection pass masks of processed tokens: word of lane l,
@@ -106,6 +107,7 @@ inline WsLayout make_layout(const osdn_params& p, bool need_bwd)
     L.p1flags = take(4 * NT * H * 2);
     if (need_bwd) {
         L.p1skip = take(4 * NT * H * 2);
+        L.p1al = take(4 * Ttot * H);
         L.pmask = take(4 * Ttot * H * 32);
         L.dtraj = take(4 * Ttot * H * K);
     }
@@ -147,7 +149,7 @@ inline Table carve_table(void* ws, const WsLayout& L)
 }
 
 struct P1Regions {
-    float *n, *rho, *dtraj;
+    float *n, *rho, *dtraj, *al;
     unsigned *flags, *skipw, *pmask;
 };
 
@@ -157,6 +159,7 @@ inline P1Regions carve_p1(void* ws, const WsLayout& L)
     P1Regions r;
     r.n = reinterpret_cast<float*>(w + L.p1n);
     r.rho = reinterpret_cast<float*>(w + L.p1rho);
+    r.al = reinterpret_cast<float*>(w + L.p1al);
     r.flags = reinterpret_cast<unsigned*>(w + L.p1flags);
     r.skipw = reinterpret_cast<unsigned*>(w + L.p1skip);
     r.pmask = reinterpret_cast<unsigned*>(w + L.pmask);

@@ -594,6 +594,7 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
                     d[r] = x;
                 }
                 B.mask[j][lane] = mybits;
+                if (lane == 0) B.scal[j].w = al;
             }
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.done[bi]);
@@ -619,6 +620,7 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
                 if (a.save) {
                     store_row<R>(a.r.dtraj + th * K, lane, dd);
                     a.r.pmask[th * 32 + lane] = B.mask[j][lane];
+                    if (lane == 0) a.r.al[th] = B.scal[j].w;
                 }
             }
             __syncwarp();
@@ -854,7 +856,10 @@ __global__ void __launch_bounds__(96) phase1_seq_kernel(P1Fwd a)
                                     at_min = at_min && (x == hy.d_min);
                                     d[r] = x;
                                 }
-                                if (a.save) a.r.pmask[th * 32 + lane] = mybits;
+                                if (a.save) {
+                                    a.r.pmask[th * 32 + lane] = mybits;
+                                    if (lane == 0) a.r.al[th] = al;
+                                }
                                 face = __all_sync(0xffffffffu, at_min);
                                 ++i;
                                 ++processed;
@@ -979,28 +984,21 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
                 load_raw<R>(a.dktil + th * K, lane, rdkt[j]);
                 load_raw<R>(a.dkread + th * K, lane, rdkr[j]);
             }
-            float ns = 0.f, rho = 0.f, bb = 1.f;
+            float ns = 0.f, rho = 0.f, bb = 1.f, alv = 0.f;   // lane j: the scalars of slot j
             if (lane < n) {
                 const size_t th = (size_t)(ttop - lane) * H + h;
                 ns = a.r.n[th];
                 rho = a.r.rho[th];
                 bb = hy.beta_aware ? a.beta[th] : 1.0f;
+                alv = a.r.al[th];   // <d_t, k^2>, recorded by the forward pass
             }
 #pragma unroll
             for (int j = 0; j < QB; ++j) {
                 const size_t th = (size_t)(ttop - min(j, n - 1)) * H + h;
                 B.mask[j][lane] = a.r.pmask[th * 32 + lane];
             }
-            float alv = 0.f;   // lane j keeps <d_t, k^2> of slot j
 #pragma unroll
             for (int j = 0; j < QB; ++j) {
-                float kk[R], dd[R], al = 0.f;
-                unpack<R>(rk[j], kk);
-                unpack<R>(rdt[j], dd);
-#pragma unroll
-                for (int r = 0; r < R; ++r) al = fmaf(dd[r], kk[r] * kk[r], al);
-                al = warp_sum(al);
-                if (lane == j) alv = al;
                 B.kraw[j][lane] = rk[j];
                 *reinterpret_cast<RawRow<float, R>*>(&B.dt[j][R * lane]) = rdt[j];
                 *reinterpret_cast<RawRow<float, R>*>(&B.dkt[j][R * lane]) = rdkt[j];
@@ -1073,7 +1071,25 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
             if (!ok) break;
             const RevBuf<T, K, VEC>& B = buf[bi];
             const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
-            for (int j = 0; j < n; ++j) {
+            // <lambda, d_t> of the block's tokens first, all slots at once: the shuffle rounds of the eight
+            // sums overlap instead of following one another
+            float drv[QB];
+#pragma unroll
+            for (int j = 0; j < QB; ++j) {
+                float dt[R], lm[R];
+                load_row<R>(B.dt[j], lane, dt);
+                load_row<R>(B.lam[j], lane, lm);
+                drv[j] = 0.f;
+#pragma unroll
+                for (int r = 0; r < R; ++r) drv[j] = fmaf(lm[r], dt[r], drv[j]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                for (int j = 0; j < QB; ++j) drv[j] += __shfl_xor_sync(0xffffffffu, drv[j], o);
+#pragma unroll
+            for (int j = 0; j < QB; ++j) {
+                if (j >= n) break;
                 const size_t th = (size_t)(ttop - j) * H + h;
                 const float4 s0 = B.sc0[j], s1 = B.sc1[j];
                 const float a2 = s0.x, rho = s0.y, cc = s0.z, g1 = s0.w, g2 = s1.x, dc = s1.y;
@@ -1083,10 +1099,7 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
                 load_row<R>(B.dkt[j], lane, dkt);
                 load_row<R>(B.dkr[j], lane, dkr);
                 load_row<R>(B.lam[j], lane, lm);
-                float drho = 0.f;
-#pragma unroll
-                for (int r = 0; r < R; ++r) drho = fmaf(lm[r], dt[r], drho);
-                drho = warp_sum(drho);
+                const float drho = drv[j];
                 const float da = -a2 * dc, dbt = g1 * dc, dn = g2 * dc;
                 if constexpr (VEC) {
                     if (a.dlog_ret) {
@@ -1131,7 +1144,7 @@ __global__ void __launch_bounds__(96) phase1_bwd_seq_kernel(P1Bwd a)
         RawRow<T, R> k[32], sk_k[32];
         RawRow<float, R> dt[32], dkt[32], dkr[32], sk_t[32], lr[VEC ? 32 : 1];
         unsigned m[32];
-        float n[32], rho[32], beta[32];
+        float n[32], rho[32], beta[32], al[32];
     };
     extern __shared__ __align__(16) uint8_t p1_dyn[];   // RevBuf[QN]
     RevBuf<T, K, VEC>* rbuf = reinterpret_cast<RevBuf<T, K, VEC>*>(p1_dyn);
@@ -1280,6 +1293,7 @@ __global__ void __launch_bounds__(96) phase1_bwd_seq_kernel(P1Bwd a)
                 cp_async<4>(&rs.n[lane], a.r.n + th);
                 cp_async<4>(&rs.rho[lane], a.r.rho + th);
                 cp_async<4>(&rs.beta[lane], a.beta + th);
+                cp_async<4>(&rs.al[lane], a.r.al + th);
                 const bool top = i == len - 1;
                 const bool need = top ? !valid_in : (((sk >> (i + 1)) & 1ull) != 0ull);
                 if (need) {   // lambda restarts at the lowest token of the skipped run above
@@ -1334,13 +1348,11 @@ __global__ void __launch_bounds__(96) phase1_bwd_seq_kernel(P1Bwd a)
                         if (pfm) needr[u] = fetch(pop_top(pfm), u);
                         else cp_async_commit();
                         const size_t th = (size_t)(tok0 + i) * H + h;
-                        // what does not depend on lambda first: the step's own scalars
+                        // what does not depend on lambda first: the step's own scalars (<d_t, k^2> was
+                        // recorded by the forward pass)
 #pragma unroll
-                        for (int r = 0; r < R; ++r) {
-                            kap[r] = kk[r] * kk[r];
-                            al = fmaf(dt[r], kap[r], al);
-                        }
-                        al = warp_sum(al);
+                        for (int r = 0; r < R; ++r) kap[r] = kk[r] * kk[r];
+                        al = rs.al[lane];
                         const float e = hy.eta * b * rn, a2 = e * b;
                         const float cc = fmaf(-a2, al, e);
                         const float g1 = hy.eta * (1.0f - 2.0f * b * al) * rn;
