@@ -566,7 +566,7 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
             if (!ok) break;
             PipeBuf<TI, K, VEC>& B = buf[bi];
             const int n = min(PB, t_b - (t_a + b * PB));
-            for (int j = 0; j < n; ++j) {
+            auto token = [&](int j) {
                 const float4 sc = B.scal[j];
                 float kap[R], rho[R];
                 load_row<R>(B.kap[j], lane, kap);
@@ -575,26 +575,32 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
 #pragma unroll
                     for (int r = 0; r < R; ++r) rho[r] = sc.z;
                 }
-                float al = 0.f;
+                float al0 = d[0] * kap[0], al1 = d[1] * kap[1];   // two short chains instead of one long one
 #pragma unroll
-                for (int r = 0; r < R; ++r) al = fmaf(d[r], kap[r], al);
+                for (int r = 2; r < R; r += 2) {
+                    al0 = fmaf(d[r], kap[r], al0);
+                    al1 = fmaf(d[r + 1], kap[r + 1], al1);
+                }
                 store_row<R>(B.dt[j], lane, d);
-                al = warp_sum(al);
+                const float al = warp_sum(al0 + al1);
                 const float cc = fmaf(-sc.y, al, sc.x);
                 unsigned mybits = 0;
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    float x = fmaf(cc, kap[r], rho[r] * d[r]);
-                    bool pz = true;
-                    if (hy.clamp) {
-                        pz = (x >= hy.d_min) && (x <= hy.d_max);
-                        x = fminf(fmaxf(x, hy.d_min), hy.d_max);
-                    }
-                    mybits |= pz ? (1u << r) : 0u;
-                    d[r] = x;
+                    const float x = fmaf(cc, kap[r], rho[r] * d[r]);
+                    // inside the box (faces included) exactly when clamping leaves the value alone
+                    const float xc = hy.clamp ? fminf(fmaxf(x, hy.d_min), hy.d_max) : x;
+                    mybits |= xc == x ? (1u << r) : 0u;
+                    d[r] = xc;
                 }
                 B.mask[j][lane] = mybits;
                 if (lane == 0) B.scal[j].w = al;
+            };
+            if (n == PB) {   // unrolled: the shared-memory reads of later tokens are issued under the shuffles of earlier ones
+#pragma unroll
+                for (int j = 0; j < PB; ++j) token(j);
+            } else {
+                for (int j = 0; j < n; ++j) token(j);
             }
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.done[bi]);
@@ -1034,7 +1040,7 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
             if (!ok) break;
             RevBuf<T, K, VEC>& B = buf[bi];
             const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
-            for (int j = 0; j < n; ++j) {
+            auto token = [&](int j) {
                 const float4 s0 = B.sc0[j];
                 const unsigned mw = B.mask[j][lane];
                 float kk[R], dkt[R], rv[R];
@@ -1058,6 +1064,12 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
 #pragma unroll
                 for (int r = 0; r < R; ++r) lam[r] = fmaf(rv[r], lam[r], fmaf(da, kap[r], kk[r] * dkt[r]));
                 if (lane == 0) B.sc1[j].y = dc;
+            };
+            if (n == QB) {
+#pragma unroll
+                for (int j = 0; j < QB; ++j) token(j);
+            } else {
+                for (int j = 0; j < n; ++j) token(j);
             }
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.done[bi]);
