@@ -191,105 +191,6 @@ struct P1Args {
     Hyper hy;
 };
 
-// VEC: vector retention, retsrc is [T,H,K] (one log-retention per coordinate).
-template <typename TI, typename TO, int K, bool VEC>
-__global__ void __launch_bounds__(128) phase1_stream_kernel(P1Args a)
-{
-    constexpr int R = K / 32;
-    const int lane = threadIdx.x & 31;
-    const int chain = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (chain >= a.S * a.H) return;
-    const int s = chain / a.H, h = chain % a.H;
-    // packed batch: T_dense is the packed token count; a malformed offset pair is clamped into it
-    const int t0 = a.cu ? min(max(a.cu[s], 0), a.T_dense) : s * a.T_dense;
-    const int len = a.cu ? min(max(a.cu[s + 1], t0), a.T_dense) - t0 : a.T_dense;
-    const TI* kp = static_cast<const TI*>(a.k);
-    TO* kt = static_cast<TO*>(a.ktil);
-    float d[R];
-    if (a.d0) load_row<R>(a.d0 + ((size_t)s * a.H + h) * K, lane, d);
-    else {
-#pragma unroll
-        for (int r = 0; r < R; ++r) d[r] = 1.0f;
-    }
-    const Hyper hy = a.hy;
-    float lsum = 0.f;
-    // rows and scalars a few tokens ahead, through a shared-memory ring (every lane copies and later
-    // reads its own bytes; one committed group per token)
-    constexpr int PF = 8;
-    struct Slot {
-        RawRow<TI, R> k[32];
-        RawRow<float, R> lr[VEC ? 32 : 1];
-        float beta[32], ret[32];
-    };
-    __shared__ __align__(16) Slot ring_all[4][PF];
-    Slot* ring = ring_all[threadIdx.x >> 5];
-    const bool scalar_ret = !VEC && hy.apf_mode != 0;
-    auto fetch = [&](int i, int slot) {
-        if (i < len) {
-            const size_t th = (size_t)(t0 + i) * a.H + h;
-            Slot& rs = ring[slot];
-            cp_async<R * (int)sizeof(TI)>(&rs.k[lane], kp + th * K + R * lane);
-            if constexpr (VEC) cp_async<R * 4>(&rs.lr[VEC ? lane : 0], a.retsrc + th * K + R * lane);
-            cp_async<4>(&rs.beta[lane], a.beta + th);
-            if (scalar_ret) cp_async<4>(&rs.ret[lane], a.retsrc + th);
-        }
-        cp_async_commit();
-    };
-#pragma unroll
-    for (int u = 0; u < PF; ++u) fetch(u, u);
-    for (int i0 = 0; i0 < len; i0 += PF) {
-#pragma unroll
-        for (int u = 0; u < PF; ++u) {
-            const int i = i0 + u;
-            if (i < len) {
-                cp_async_wait<PF - 1>();
-                const Slot& rs = ring[u];
-                const size_t th = (size_t)(t0 + i) * a.H + h;
-                float kk[R], kap[R], w[R];
-                unpack<R>(rs.k[lane], kk);
-                const float beta = rs.beta[lane];
-                float rho[R];
-                if constexpr (VEC) {
-                    float lr[R];
-                    unpack<R>(rs.lr[VEC ? lane : 0], lr);
-#pragma unroll
-                    for (int r = 0; r < R; ++r) rho[r] = expf(lr[r]);
-                } else {
-                    const float r1 = scalar_ret ? expf(rs.ret[lane]) : 1.0f;
-#pragma unroll
-                    for (int r = 0; r < R; ++r) rho[r] = r1;
-                }
-                fetch(i + PF, u);
-                const float sumk = square_sum<R>(kk, kap);
-                if (kt) {
-#pragma unroll
-                    for (int r = 0; r < R; ++r) w[r] = d[r] * kk[r];
-                    store_row<R>(kt + th * K, lane, w);
-                }
-                const float n = fmaxf(sumk, hy.eps);
-                const float b = hy.beta_aware ? beta : 1.0f;
-                unsigned pass[R];
-                bool low;
-                float c, al;
-                p1_step<R>(d, kap, n, b, rho, hy, pass, low, c, al);
-                if (a.ratio || a.log_sum) {
-                    // residual ratio of the write of this token (token-local theorem): the loss |S k - v|^2
-                    // after the write over the loss before it is (1 - beta <d_t, k^2>)^2, with the write
-                    // strength beta itself (whether or not the step of d is beta-aware) and the d the write
-                    // key was formed with
-                    const float fac = 1.0f - beta * al;
-                    const float qt = fac * fac;
-                    if (a.ratio && lane == 0) a.ratio[th] = qt;
-                    lsum += logf(fmaxf(qt, 1.17549435e-38f));
-                }
-            }
-        }
-    }
-    cp_async_wait<0>();
-    if (a.d_final) store_row<R>(a.d_final + ((size_t)s * a.H + h) * K, lane, d);
-    if (a.log_sum && lane == 0) a.log_sum[(size_t)s * a.H + h] = lsum;
-}
-
 // ---------------------------------------------------------------------------------------------
 // forward: parallel speculative pass, then the sequential pass over what is left
 // ---------------------------------------------------------------------------------------------
@@ -501,6 +402,50 @@ struct PipeBars {
     uint64_t full[PN], done[PN], free_[PN];
 };
 
+// The core's work on one block: carries d through n tokens; reads kap, the scalars (and the retention
+// vector), leaves d_t, the mask bits and <d_t, k^2> (in scal.w).
+template <typename TI, int K, bool VEC>
+__device__ __forceinline__ void pipe_core_block(PipeBuf<TI, K, VEC>& B, int n, float (&d)[K / 32], const Hyper& hy, int lane)
+{
+    constexpr int R = K / 32;
+                auto token = [&](int j) {
+                    const float4 sc = B.scal[j];
+                    float kap[R], rho[R];
+                    load_row<R>(B.kap[j], lane, kap);
+                    if constexpr (VEC) load_row<R>(B.rhov[VEC ? j : 0], lane, rho);
+                    else {
+    #pragma unroll
+                        for (int r = 0; r < R; ++r) rho[r] = sc.z;
+                    }
+                    float al0 = d[0] * kap[0], al1 = d[1] * kap[1];   // two short chains instead of one long one
+    #pragma unroll
+                    for (int r = 2; r < R; r += 2) {
+                        al0 = fmaf(d[r], kap[r], al0);
+                        al1 = fmaf(d[r + 1], kap[r + 1], al1);
+                    }
+                    store_row<R>(B.dt[j], lane, d);
+                    const float al = warp_sum(al0 + al1);
+                    const float cc = fmaf(-sc.y, al, sc.x);
+                    unsigned mybits = 0;
+    #pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const float x = fmaf(cc, kap[r], rho[r] * d[r]);
+                        // inside the box (faces included) exactly when clamping leaves the value alone
+                        const float xc = hy.clamp ? fminf(fmaxf(x, hy.d_min), hy.d_max) : x;
+                        mybits |= xc == x ? (1u << r) : 0u;
+                        d[r] = xc;
+                    }
+                    B.mask[j][lane] = mybits;
+                    if (lane == 0) B.scal[j].w = al;
+                };
+                if (n == PB) {   // unrolled: the shared-memory reads of later tokens are issued under the shuffles of earlier ones
+    #pragma unroll
+                    for (int j = 0; j < PB; ++j) token(j);
+                } else {
+                    for (int j = 0; j < n; ++j) token(j);
+                }
+}
+
 // tokens [t_a, t_b) of the chain (packed token indices), all three roles; d: the core's registers
 template <typename TI, typename TO, int K, bool VEC>
 __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int t_b, float (&d)[K / 32],
@@ -564,44 +509,8 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
             const int bi = use % PN;
             ok = p1_mbar_wait(&bars.full[bi], (use / PN) & 1, a.status);
             if (!ok) break;
-            PipeBuf<TI, K, VEC>& B = buf[bi];
             const int n = min(PB, t_b - (t_a + b * PB));
-            auto token = [&](int j) {
-                const float4 sc = B.scal[j];
-                float kap[R], rho[R];
-                load_row<R>(B.kap[j], lane, kap);
-                if constexpr (VEC) load_row<R>(B.rhov[VEC ? j : 0], lane, rho);
-                else {
-#pragma unroll
-                    for (int r = 0; r < R; ++r) rho[r] = sc.z;
-                }
-                float al0 = d[0] * kap[0], al1 = d[1] * kap[1];   // two short chains instead of one long one
-#pragma unroll
-                for (int r = 2; r < R; r += 2) {
-                    al0 = fmaf(d[r], kap[r], al0);
-                    al1 = fmaf(d[r + 1], kap[r + 1], al1);
-                }
-                store_row<R>(B.dt[j], lane, d);
-                const float al = warp_sum(al0 + al1);
-                const float cc = fmaf(-sc.y, al, sc.x);
-                unsigned mybits = 0;
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float x = fmaf(cc, kap[r], rho[r] * d[r]);
-                    // inside the box (faces included) exactly when clamping leaves the value alone
-                    const float xc = hy.clamp ? fminf(fmaxf(x, hy.d_min), hy.d_max) : x;
-                    mybits |= xc == x ? (1u << r) : 0u;
-                    d[r] = xc;
-                }
-                B.mask[j][lane] = mybits;
-                if (lane == 0) B.scal[j].w = al;
-            };
-            if (n == PB) {   // unrolled: the shared-memory reads of later tokens are issued under the shuffles of earlier ones
-#pragma unroll
-                for (int j = 0; j < PB; ++j) token(j);
-            } else {
-                for (int j = 0; j < n; ++j) token(j);
-            }
+            pipe_core_block<TI, K, VEC>(buf[bi], n, d, hy, lane);
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.done[bi]);
         }
@@ -635,6 +544,146 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
     }
     round0 = base + nblk;
     return ok;
+}
+
+// The stand-alone sweep processes every token: the whole sequence is one pipelined stretch (see the
+// forward's stretches below the parallel pass).  pre also forms the normaliser here (there is no parallel
+// pass before this kernel); post forms the write keys and the residual ratios.
+template <typename TI, typename TO, int K, bool VEC>
+__global__ void __launch_bounds__(96) phase1_stream_kernel(P1Args a)
+{
+    constexpr int R = K / 32;
+    extern __shared__ __align__(16) uint8_t p1_dyn[];   // PipeBuf[PN], then the write strengths beta[PN][PB]
+    PipeBuf<TI, K, VEC>* buf = reinterpret_cast<PipeBuf<TI, K, VEC>*>(p1_dyn);
+    float(*sbeta)[PB] = reinterpret_cast<float(*)[PB]>(p1_dyn + PN * sizeof(PipeBuf<TI, K, VEC>));
+    __shared__ PipeBars bars;
+    const int lane = threadIdx.x & 31, role = threadIdx.x >> 5;   // 0 core, 1 pre, 2 post
+    const int chain = blockIdx.x;
+    const int s = chain / a.H, h = chain % a.H, H = a.H;
+    // packed batch: T_dense is the packed token count; a malformed offset pair is clamped into it
+    const int t0 = a.cu ? min(max(a.cu[s], 0), a.T_dense) : s * a.T_dense;
+    const int len = a.cu ? min(max(a.cu[s + 1], t0), a.T_dense) - t0 : a.T_dense;
+    const TI* kp = static_cast<const TI*>(a.k);
+    const Hyper hy = a.hy;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < PN; ++i) {
+            p1_mbar_init(&bars.full[i], 1);
+            p1_mbar_init(&bars.done[i], 1);
+            p1_mbar_init(&bars.free_[i], 1);
+        }
+    }
+    __syncthreads();
+    const int nblk = (len + PB - 1) / PB;
+    const bool scalar_ret = !VEC && hy.apf_mode != 0;
+    bool ok = true;
+    if (role == 1) {
+        for (int b = 0; b < nblk && ok; ++b) {
+            const int bi = b % PN;
+            if (b >= PN) ok = p1_mbar_wait(&bars.free_[bi], ((b / PN) - 1) & 1, nullptr);
+            if (!ok) break;
+            PipeBuf<TI, K, VEC>& B = buf[bi];
+            const int tb0 = t0 + b * PB, n = min(PB, len - b * PB);
+            RawRow<TI, R> raw[PB];
+#pragma unroll
+            for (int j = 0; j < PB; ++j) load_raw<R>(kp + ((size_t)(tb0 + min(j, n - 1)) * H + h) * K, lane, raw[j]);
+            float beta = 0.f, ret = 0.f;
+            if (lane < n) {
+                const size_t th = (size_t)(tb0 + lane) * H + h;
+                beta = a.beta[th];
+                if (scalar_ret) ret = a.retsrc[th];
+            }
+            float sums[PB];
+#pragma unroll
+            for (int j = 0; j < PB; ++j) {
+                float kk[R], kap[R];
+                unpack<R>(raw[j], kk);
+                sums[j] = 0.f;
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    kap[r] = kk[r] * kk[r];
+                    sums[j] += kap[r];
+                }
+                store_row<R>(B.kap[j], lane, kap);
+                B.kraw[j][lane] = raw[j];
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)   // the sixteen sums together: their shuffle rounds overlap
+#pragma unroll
+                for (int j = 0; j < PB; ++j) sums[j] += __shfl_xor_sync(0xffffffffu, sums[j], o);
+            float mine = 0.f;
+#pragma unroll
+            for (int j = 0; j < PB; ++j) mine = lane == j ? sums[j] : mine;
+            if (lane < n) {
+                const float nn = fmaxf(mine, hy.eps), bb = hy.beta_aware ? beta : 1.0f;
+                const float e = hy.eta * bb / nn;
+                B.scal[lane] = make_float4(e, e * bb, scalar_ret ? expf(ret) : 1.0f, 0.f);
+                sbeta[bi][lane] = beta;
+            }
+            if constexpr (VEC) {
+                for (int j = 0; j < n; ++j) {
+                    float lr[R];
+                    load_row<R>(a.retsrc + ((size_t)(tb0 + j) * H + h) * K, lane, lr);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) lr[r] = expf(lr[r]);
+                    store_row<R>(B.rhov[VEC ? j : 0], lane, lr);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.full[bi]);
+        }
+    } else if (role == 0) {
+        float d[R];
+        if (a.d0) load_row<R>(a.d0 + ((size_t)s * H + h) * K, lane, d);
+        else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) d[r] = 1.0f;
+        }
+        for (int b = 0; b < nblk && ok; ++b) {
+            const int bi = b % PN;
+            ok = p1_mbar_wait(&bars.full[bi], (b / PN) & 1, nullptr);
+            if (!ok) break;
+            pipe_core_block<TI, K, VEC>(buf[bi], min(PB, len - b * PB), d, hy, lane);
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.done[bi]);
+        }
+        if (a.d_final && ok) store_row<R>(a.d_final + ((size_t)s * H + h) * K, lane, d);
+    } else {
+        TO* kt = static_cast<TO*>(a.ktil);
+        float lsum = 0.f;
+        for (int b = 0; b < nblk && ok; ++b) {
+            const int bi = b % PN;
+            ok = p1_mbar_wait(&bars.done[bi], (b / PN) & 1, nullptr);
+            if (!ok) break;
+            const PipeBuf<TI, K, VEC>& B = buf[bi];
+            const int tb0 = t0 + b * PB, n = min(PB, len - b * PB);
+            if (kt) {
+                for (int j = 0; j < n; ++j) {
+                    float dd[R], kk[R], wk[R];
+                    load_row<R>(B.dt[j], lane, dd);
+                    unpack<R>(B.kraw[j][lane], kk);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) wk[r] = dd[r] * kk[r];
+                    store_row<R>(kt + ((size_t)(tb0 + j) * H + h) * K, lane, wk);
+                }
+            }
+            if (a.ratio || a.log_sum) {
+                // residual ratio of the write of a token (token-local theorem): the loss |S k - v|^2 after the
+                // write over the loss before it is (1 - beta <d_t, k^2>)^2, with the write strength beta itself
+                // (whether or not the step of d is beta-aware) and the d the write key was formed with
+                float lq = 0.f;
+                if (lane < n) {
+                    const float fac = 1.0f - sbeta[bi][lane] * B.scal[lane].w;
+                    const float qt = fac * fac;
+                    if (a.ratio) a.ratio[(size_t)(tb0 + lane) * H + h] = qt;
+                    lq = logf(fmaxf(qt, 1.17549435e-38f));
+                }
+                lsum += warp_sum(lq);
+            }
+            __syncwarp();
+            if (lane == 0) p1_mbar_arrive(&bars.free_[bi]);
+        }
+        if (a.log_sum && lane == 0) a.log_sum[(size_t)s * H + h] = lsum;
+    }
 }
 
 // one warp per chain.  Flag words are fetched for 32 chunks at a time (one chunk per lane); the
@@ -1516,27 +1565,33 @@ int phase1_update(const osdn_params& p, const Hyper& hy, const void* k, const fl
     pa.H = p.H; pa.T_dense = p.T; pa.cu = p.nseq > 0 ? p.cu_seqlens : nullptr;
     pa.k = k; pa.beta = beta; pa.retsrc = retsrc; pa.d0 = precond_in; pa.ktil = ktil_out;
     pa.d_final = precond_out; pa.ratio = ratio_out; pa.log_sum = log_sum_out; pa.hy = hy;
-    const int chains = pa.S * pa.H;
-    const unsigned grid = (chains + 3) / 4;
+    const unsigned chains = (unsigned)(pa.S * pa.H);
     stage_mark(st, "phase1_stream");
     const bool vec = hy.apf_mode == 3;
+    auto launch = [&](auto kernel, size_t buf_bytes) {
+        const size_t smem = PN * buf_bytes + PN * PB * sizeof(float);
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        kernel<<<chains, 96, smem, st>>>(pa);
+        return true;
+    };
+    bool ok;
     if (p.io_dtype == OSDN_FP32) {
-        if (p.K == 64) {
-            if (vec) phase1_stream_kernel<float, float, 64, true><<<grid, 128, 0, st>>>(pa);
-            else phase1_stream_kernel<float, float, 64, false><<<grid, 128, 0, st>>>(pa);
-        } else {
-            if (vec) phase1_stream_kernel<float, float, 128, true><<<grid, 128, 0, st>>>(pa);
-            else phase1_stream_kernel<float, float, 128, false><<<grid, 128, 0, st>>>(pa);
-        }
+        if (p.K == 64)
+            ok = vec ? launch(phase1_stream_kernel<float, float, 64, true>, sizeof(PipeBuf<float, 64, true>))
+                     : launch(phase1_stream_kernel<float, float, 64, false>, sizeof(PipeBuf<float, 64, false>));
+        else
+            ok = vec ? launch(phase1_stream_kernel<float, float, 128, true>, sizeof(PipeBuf<float, 128, true>))
+                     : launch(phase1_stream_kernel<float, float, 128, false>, sizeof(PipeBuf<float, 128, false>));
     } else {
-        if (p.K == 64) {
-            if (vec) phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 64, true><<<grid, 128, 0, st>>>(pa);
-            else phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 64, false><<<grid, 128, 0, st>>>(pa);
-        } else {
-            if (vec) phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 128, true><<<grid, 128, 0, st>>>(pa);
-            else phase1_stream_kernel<__nv_bfloat16, __nv_bfloat16, 128, false><<<grid, 128, 0, st>>>(pa);
-        }
+        using B16 = __nv_bfloat16;
+        if (p.K == 64)
+            ok = vec ? launch(phase1_stream_kernel<B16, B16, 64, true>, sizeof(PipeBuf<B16, 64, true>))
+                     : launch(phase1_stream_kernel<B16, B16, 64, false>, sizeof(PipeBuf<B16, 64, false>));
+        else
+            ok = vec ? launch(phase1_stream_kernel<B16, B16, 128, true>, sizeof(PipeBuf<B16, 128, true>))
+                     : launch(phase1_stream_kernel<B16, B16, 128, false>, sizeof(PipeBuf<B16, 128, false>));
     }
+    if (!ok) return -1;
     stage_end(st);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
