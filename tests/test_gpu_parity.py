@@ -215,3 +215,43 @@ def test_forward_launch_variants_of_the_tensor_core_path(case):
     # ragged sets with carried-in states: the largest elements stand 15-30 times above the rms, so the
     # third measure (largest error over rms) gets its own ceiling here; the other two gates are the usual ones
     _check(inp, True, "fwd_variants/" + case, rms_ceiling=0.16)
+
+
+@pytest.mark.parametrize("case", ["k64_fp32", "two_groups_fp32", "packed_ragged_bf16", "vector_two_groups_fp32",
+                                  "update_only_k64"])
+def test_pipelined_stretches_of_the_sequential_passes(case):
+    """Where nearly every token is processed the sequential preconditioner kernels hand a chain to three
+    warps (stretches of up to eight chunks, blocks of 16 / 8 tokens through a ring).  Cases that the small
+    sets above do not reach: K = 64, sequences longer than one group of 32 chunks (stretches end at group
+    boundaries), packed sequences whose stretches start and end on ragged chunks, the vector retention,
+    and the stand-alone update (the same pipeline over a whole sequence) with a block tail."""
+    if case == "k64_fp32":
+        hy = OsdnHyper(eta=0.3, apf_mode=2)
+        inp = draw(case, 401, [333, 333], 2, 64, 64, "fp32", dense_B=2, hyper=hy, key_kind="sparse", with_dout=True,
+                   with_log_ret=True, with_state=True, with_state_cotangents=True)
+    elif case == "two_groups_fp32":
+        hy = OsdnHyper(eta=0.3, apf_mode=2)
+        inp = draw(case, 402, [2300], 1, 64, 64, "fp32", dense_B=1, hyper=hy, key_kind="sparse", with_dout=True,
+                   with_log_ret=True, with_state=True, with_state_cotangents=True)
+    elif case == "packed_ragged_bf16":
+        hy = OsdnHyper(eta=0.3, apf_mode=2)
+        inp = draw(case, 403, [700, 65, 130, 1, 577], 2, 128, 128, "bf16", hyper=hy, key_kind="sparse", with_dout=True,
+                   with_log_ret=True, with_state=True, with_state_cotangents=True)
+    elif case == "vector_two_groups_fp32":
+        hy = OsdnHyper(eta=0.3, apf_mode=3)
+        inp = draw(case, 404, [2100], 1, 64, 64, "fp32", dense_B=1, hyper=hy, key_kind="sparse", with_dout=True,
+                   with_log_ret=True, with_state=True, with_state_cotangents=True, log_ret_shift=3.0)
+    else:
+        hy = OsdnHyper(eta=0.3, apf_mode=2)
+        inp = draw(case, 405, [203, 16, 1], 3, 64, 64, "fp32", hyper=hy, key_kind="sparse", with_log_ret=True, with_state=True)
+        dev = "cuda:0"
+        b = binding.DeviceBundle(inp, dev, need_bwd=False)
+        ktil = torch.empty_like(b.k)
+        d_out = torch.empty_like(b.precond_in)
+        binding.osdn_precond_update(b.params, b.k, b.beta, b.log_ret, b.precond_in, ktil, d_out)
+        torch.cuda.synchronize()
+        ref = oracle.precond_update(hy, inp.seq_lens, inp.k, inp.beta, None, inp.log_ret, inp.precond_in)
+        assert parity.err(ktil.float().cpu().numpy(), ref["ktil"], "fp32") <= 1e-4
+        assert parity.err(d_out.cpu().numpy(), ref["precond_out"], "fp32") <= 1e-4
+        return
+    _check(inp, True, "pipelined/" + case, rms_ceiling=0.16 if inp.io_dtype == "bf16" else None)
