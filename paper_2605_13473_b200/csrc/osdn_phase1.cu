@@ -777,6 +777,12 @@ __global__ void __launch_bounds__(96) phase1_seq_kernel(P1Fwd a)
             const unsigned long long bl = (unsigned long long)w0 | ((unsigned long long)w1 << 32);
             const unsigned long long vl = lenl >= 64 ? ~0ull : ((1ull << lenl) - 1ull);
             allflag = __ballot_sync(0xffffffffu, cl < c1 && (bl & vl) == vl);
+            // The first chunk of a sequence that enters off the face with at least PIPE_TRIGGER tokens that
+            // are processed for certain (unflagged) starts pipelined right away.
+            if (cbase == c0 && !face) {
+                const int sure = __shfl_sync(0xffffffffu, __popcll(~bl & vl), 0);
+                pipe_next = sure >= PIPE_TRIGGER;
+            }
         }
         for (int c = cbase; c < cend; ++c) {
             if (pipe_next) {
