@@ -1012,6 +1012,7 @@ template <typename T, int K, bool VEC> struct RevBuf {
     unsigned mask[QB][32];
     float4 sc0[QB];                         // a2, rho, cc, g1
     float4 sc1[QB];                         // g2, dc (written by the core), -, -
+    float raw[4][QB];                       // n (signed), rho, beta, <d_t, k^2> as they sit in memory
 };
 
 // tokens [t_lo, t_hi) of the chain in reverse, all three roles; lam: the core's registers
@@ -1028,44 +1029,17 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
     const uint32_t base = round0;
     // block b: tokens t_hi - 1 - (b QB + j), j = 0 .. n - 1 (slot j of the buffer)
     if (role == 1) {
-        for (int b = 0; b < nblk && ok; ++b) {
+        // Rows go straight into the buffer with cp.async (nothing of them is converted here), one committed
+        // group per block and one block ahead: while block b is on its way, block b - 1 is finished (the
+        // step's own scalars formed from the raw ones, the retention vector exponentiated) and handed over.
+        auto finish = [&](int b) {
             const uint32_t use = base + b;
             const int bi = use % QN;
-            if (use >= QN) ok = p1_mbar_wait(&bars.free_[bi], ((use / QN) - 1) & 1, a.status);
-            if (!ok) break;
             RevBuf<T, K, VEC>& B = buf[bi];
             const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
-            RawRow<T, R> rk[QB];
-            RawRow<float, R> rdt[QB], rdkt[QB], rdkr[QB];
-#pragma unroll
-            for (int j = 0; j < QB; ++j) {
-                const size_t th = (size_t)(ttop - min(j, n - 1)) * H + h;
-                load_raw<R>(kp + th * K, lane, rk[j]);
-                load_raw<R>(a.r.dtraj + th * K, lane, rdt[j]);
-                load_raw<R>(a.dktil + th * K, lane, rdkt[j]);
-                load_raw<R>(a.dkread + th * K, lane, rdkr[j]);
-            }
-            float ns = 0.f, rho = 0.f, bb = 1.f, alv = 0.f;   // lane j: the scalars of slot j
             if (lane < n) {
-                const size_t th = (size_t)(ttop - lane) * H + h;
-                ns = a.r.n[th];
-                rho = a.r.rho[th];
-                bb = hy.beta_aware ? a.beta[th] : 1.0f;
-                alv = a.r.al[th];   // <d_t, k^2>, recorded by the forward pass
-            }
-#pragma unroll
-            for (int j = 0; j < QB; ++j) {
-                const size_t th = (size_t)(ttop - min(j, n - 1)) * H + h;
-                B.mask[j][lane] = a.r.pmask[th * 32 + lane];
-            }
-#pragma unroll
-            for (int j = 0; j < QB; ++j) {
-                B.kraw[j][lane] = rk[j];
-                *reinterpret_cast<RawRow<float, R>*>(&B.dt[j][R * lane]) = rdt[j];
-                *reinterpret_cast<RawRow<float, R>*>(&B.dkt[j][R * lane]) = rdkt[j];
-                *reinterpret_cast<RawRow<float, R>*>(&B.dkr[j][R * lane]) = rdkr[j];
-            }
-            if (lane < n) {
+                const float ns = B.raw[0][lane], rho = B.raw[1][lane], alv = B.raw[3][lane];
+                const float bb = hy.beta_aware ? B.raw[2][lane] : 1.0f;
                 const float rn = fabsf(ns);
                 const float e = hy.eta * bb * rn, a2 = e * bb;
                 const float cc = fmaf(-a2, alv, e);
@@ -1076,9 +1050,8 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
             }
             if constexpr (VEC) {
                 for (int j = 0; j < n; ++j) {
-                    const size_t th = (size_t)(ttop - j) * H + h;
                     float lr[R];
-                    load_row<R>(a.log_ret + th * K, lane, lr);
+                    load_row<R>(B.rv[VEC ? j : 0], lane, lr);
 #pragma unroll
                     for (int r = 0; r < R; ++r) lr[r] = expf(lr[r]);
                     store_row<R>(B.rv[VEC ? j : 0], lane, lr);
@@ -1086,7 +1059,41 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
             }
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.full[bi]);
+        };
+        for (int b = 0; b < nblk && ok; ++b) {
+            const uint32_t use = base + b;
+            const int bi = use % QN;
+            if (use >= QN) ok = p1_mbar_wait(&bars.free_[bi], ((use / QN) - 1) & 1, a.status);
+            if (!ok) break;
+            RevBuf<T, K, VEC>& B = buf[bi];
+            const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
+#pragma unroll
+            for (int j = 0; j < QB; ++j) {
+                const size_t th = (size_t)(ttop - min(j, n - 1)) * H + h;
+                cp_async<R * (int)sizeof(T)>(&B.kraw[j][lane], kp + th * K + R * lane);
+                cp_async<R * 4>(&B.dt[j][R * lane], a.r.dtraj + th * K + R * lane);
+                cp_async<R * 4>(&B.dkt[j][R * lane], a.dktil + th * K + R * lane);
+                cp_async<R * 4>(&B.dkr[j][R * lane], a.dkread + th * K + R * lane);
+                cp_async<4>(&B.mask[j][lane], a.r.pmask + th * 32 + lane);
+                if constexpr (VEC) cp_async<R * 4>(&B.rv[VEC ? j : 0][R * lane], a.log_ret + th * K + R * lane);
+            }
+            if (lane < n) {
+                const size_t th = (size_t)(ttop - lane) * H + h;
+                cp_async<4>(&B.raw[0][lane], a.r.n + th);
+                cp_async<4>(&B.raw[1][lane], a.r.rho + th);
+                cp_async<4>(&B.raw[2][lane], a.beta + th);
+                cp_async<4>(&B.raw[3][lane], a.r.al + th);
+            }
+            cp_async_commit();
+            if (b > 0) {
+                cp_async_wait<1>();   // block b - 1 has landed
+                __syncwarp();
+                finish(b - 1);
+            }
         }
+        cp_async_wait<0>();
+        __syncwarp();
+        if (ok && nblk > 0) finish(nblk - 1);
     } else if (role == 0) {
         for (int b = 0; b < nblk && ok; ++b) {
             const uint32_t use = base + b;
