@@ -398,8 +398,9 @@ template <typename TI, int K, bool VEC> struct PipeBuf {
     float4 scal[PB];                        // e = eta b / n, a2 = e b, rho, -
     unsigned mask[PB][32];                  // projection pass bits of lane l's coordinates
 };
+constexpr int RING_MAX = 6;   // the deeper of the two rings
 struct PipeBars {
-    uint64_t full[PN], done[PN], free_[PN];
+    uint64_t full[RING_MAX], done[RING_MAX], free_[RING_MAX];
 };
 
 // The core's work on one block: carries d through n tokens; reads kap, the scalars (and the retention
@@ -524,7 +525,7 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
             if (!ok) break;
             const PipeBuf<TI, K, VEC>& B = buf[bi];
             const int t0 = t_a + b * PB, n = min(PB, t_b - t0);
-            for (int j = 0; j < n; ++j) {
+            auto token = [&](int j) {
                 const size_t th = (size_t)(t0 + j) * H + h;
                 float dd[R], kk[R], wk[R];
                 load_row<R>(B.dt[j], lane, dd);
@@ -535,8 +536,14 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
                 if (a.save) {
                     store_row<R>(a.r.dtraj + th * K, lane, dd);
                     a.r.pmask[th * 32 + lane] = B.mask[j][lane];
-                    if (lane == 0) a.r.al[th] = B.scal[j].w;
                 }
+            };
+            if (a.save && lane < n) a.r.al[(size_t)(t0 + lane) * H + h] = B.scal[lane].w;   // lane j: token j
+            if (n == PB) {
+#pragma unroll
+                for (int j = 0; j < PB; ++j) token(j);
+            } else {
+                for (int j = 0; j < n; ++j) token(j);
             }
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.free_[bi]);
@@ -1001,7 +1008,9 @@ __global__ void __launch_bounds__(128) phase1_bwd_bulk_kernel(P1Bwd a)
 //   core  carries lambda through the block (top token first) and leaves the masked lambda and dc;
 //   post  forms dk, the retention and beta gradients from those and writes them out.
 // ---------------------------------------------------------------------------------------------
-constexpr int QB = 8, QN = 3;
+// Five buffers: the pre role holds two (one landing, one being finished), core and post one each, one spare.
+constexpr int QB = 8, QN = 5;
+static_assert(QN <= RING_MAX && PN <= RING_MAX, "barrier arrays");
 
 template <typename T, int K, bool VEC> struct RevBuf {
     static constexpr int R = K / 32;
@@ -1161,20 +1170,31 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
             for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
                 for (int j = 0; j < QB; ++j) drv[j] += __shfl_xor_sync(0xffffffffu, drv[j], o);
+            // the per-token scalars (beta and retention gradients): lane j takes token j
+            {
+                float mine = 0.f;
 #pragma unroll
-            for (int j = 0; j < QB; ++j) {
-                if (j >= n) break;
+                for (int j = 0; j < QB; ++j) mine = lane == j ? drv[j] : mine;
+                if (lane < n) {
+                    const size_t th = (size_t)(ttop - lane) * H + h;
+                    const float4 s0 = B.sc0[lane];
+                    const float dc = B.sc1[lane].y;
+                    if (hy.beta_aware) atomicAdd(&a.dbeta[th], s0.w * dc);
+                    if (hy.apf_mode == 1) atomicAdd(&a.dgate[th], s0.y * mine);
+                    if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = s0.y * mine;
+                }
+            }
+            auto token = [&](int j) {
                 const size_t th = (size_t)(ttop - j) * H + h;
                 const float4 s0 = B.sc0[j], s1 = B.sc1[j];
-                const float a2 = s0.x, rho = s0.y, cc = s0.z, g1 = s0.w, g2 = s1.x, dc = s1.y;
+                const float a2 = s0.x, cc = s0.z, g2 = s1.x, dc = s1.y;
                 float kk[R], dt[R], dkt[R], dkr[R], lm[R];
                 unpack<R>(B.kraw[j][lane], kk);
                 load_row<R>(B.dt[j], lane, dt);
                 load_row<R>(B.dkt[j], lane, dkt);
                 load_row<R>(B.dkr[j], lane, dkr);
                 load_row<R>(B.lam[j], lane, lm);
-                const float drho = drv[j];
-                const float da = -a2 * dc, dbt = g1 * dc, dn = g2 * dc;
+                const float da = -a2 * dc, dn = g2 * dc;
                 if constexpr (VEC) {
                     if (a.dlog_ret) {
                         float rv[R], dl[R];
@@ -1191,11 +1211,12 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
                     out[r] = dkr[r] + dt[r] * dkt[r] + 2.0f * kk[r] * dkap;
                 }
                 store_row<R>(dkp + th * K, lane, out);
-                if (lane == 0) {
-                    if (hy.beta_aware) atomicAdd(&a.dbeta[th], dbt);
-                    if (hy.apf_mode == 1) atomicAdd(&a.dgate[th], rho * drho);
-                    if (hy.apf_mode == 2 && a.dlog_ret) a.dlog_ret[th] = rho * drho;
-                }
+            };
+            if (n == QB) {   // unrolled without a branch between the tokens: their reads and products interleave
+#pragma unroll
+                for (int j = 0; j < QB; ++j) token(j);
+            } else {
+                for (int j = 0; j < n; ++j) token(j);
             }
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.free_[bi]);
