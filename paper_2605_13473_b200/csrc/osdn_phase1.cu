@@ -409,42 +409,42 @@ template <typename TI, int K, bool VEC>
 __device__ __forceinline__ void pipe_core_block(PipeBuf<TI, K, VEC>& B, int n, float (&d)[K / 32], const Hyper& hy, int lane)
 {
     constexpr int R = K / 32;
-                auto token = [&](int j) {
-                    const float4 sc = B.scal[j];
-                    float kap[R], rho[R];
-                    load_row<R>(B.kap[j], lane, kap);
-                    if constexpr (VEC) load_row<R>(B.rhov[VEC ? j : 0], lane, rho);
-                    else {
-    #pragma unroll
-                        for (int r = 0; r < R; ++r) rho[r] = sc.z;
-                    }
-                    float al0 = d[0] * kap[0], al1 = d[1] * kap[1];   // two short chains instead of one long one
-    #pragma unroll
-                    for (int r = 2; r < R; r += 2) {
-                        al0 = fmaf(d[r], kap[r], al0);
-                        al1 = fmaf(d[r + 1], kap[r + 1], al1);
-                    }
-                    store_row<R>(B.dt[j], lane, d);
-                    const float al = warp_sum(al0 + al1);
-                    const float cc = fmaf(-sc.y, al, sc.x);
-                    unsigned mybits = 0;
-    #pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        const float x = fmaf(cc, kap[r], rho[r] * d[r]);
-                        // inside the box (faces included) exactly when clamping leaves the value alone
-                        const float xc = hy.clamp ? fminf(fmaxf(x, hy.d_min), hy.d_max) : x;
-                        mybits |= xc == x ? (1u << r) : 0u;
-                        d[r] = xc;
-                    }
-                    B.mask[j][lane] = mybits;
-                    if (lane == 0) B.scal[j].w = al;
-                };
-                if (n == PB) {   // unrolled: the shared-memory reads of later tokens are issued under the shuffles of earlier ones
-    #pragma unroll
-                    for (int j = 0; j < PB; ++j) token(j);
-                } else {
-                    for (int j = 0; j < n; ++j) token(j);
-                }
+    auto token = [&](int j) {
+        const float4 sc = B.scal[j];
+        float kap[R], rho[R];
+        load_row<R>(B.kap[j], lane, kap);
+        if constexpr (VEC) load_row<R>(B.rhov[VEC ? j : 0], lane, rho);
+        else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) rho[r] = sc.z;
+        }
+        float al0 = d[0] * kap[0], al1 = d[1] * kap[1];   // two short chains instead of one long one
+#pragma unroll
+        for (int r = 2; r < R; r += 2) {
+            al0 = fmaf(d[r], kap[r], al0);
+            al1 = fmaf(d[r + 1], kap[r + 1], al1);
+        }
+        store_row<R>(B.dt[j], lane, d);
+        const float al = warp_sum(al0 + al1);
+        const float cc = fmaf(-sc.y, al, sc.x);
+        unsigned mybits = 0;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const float x = fmaf(cc, kap[r], rho[r] * d[r]);
+            // inside the box (faces included) exactly when clamping leaves the value alone
+            const float xc = hy.clamp ? fminf(fmaxf(x, hy.d_min), hy.d_max) : x;
+            mybits |= xc == x ? (1u << r) : 0u;
+            d[r] = xc;
+        }
+        B.mask[j][lane] = mybits;
+        if (lane == 0) B.scal[j].w = al;
+    };
+    if (n == PB) {   // partly unrolled: the shared-memory reads of later tokens are issued under the shuffles of earlier ones
+#pragma unroll 4
+        for (int j = 0; j < PB; ++j) token(j);
+    } else {
+        for (int j = 0; j < n; ++j) token(j);
+    }
 }
 
 // tokens [t_a, t_b) of the chain (packed token indices), all three roles; d: the core's registers
@@ -540,7 +540,7 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
             };
             if (a.save && lane < n) a.r.al[(size_t)(t0 + lane) * H + h] = B.scal[lane].w;   // lane j: token j
             if (n == PB) {
-#pragma unroll
+#pragma unroll 4
                 for (int j = 0; j < PB; ++j) token(j);
             } else {
                 for (int j = 0; j < n; ++j) token(j);
