@@ -59,8 +59,10 @@ typedef enum osdn_status {
 } osdn_status;
 
 /* Values found in the device status word (first 4 bytes of a workspace) after a call whose kernels
- * met an error on the device.  101..113: a bounded wait inside a tensor-core kernel ran out (the
- * kernel then skipped the dependent work and returned; outputs of that call are undefined). */
+ * met an error on the device.  101..113, 121, 122, 131: a bounded wait inside a kernel ran out (an
+ * mbarrier of the tensor-core kernels, the backward's tile queue, a ready flag of the merged forward
+ * launch, a ring barrier of the pipelined preconditioner pass); the kernel then skipped the dependent
+ * work and returned, and the outputs of that call are undefined. */
 enum {
     OSDN_DEVICE_OK = 0,
     OSDN_DEVICE_BAD_CU_SEQLENS = 120,   /* cu_seqlens broke its contract (cu[0] != 0, a decreasing pair,
