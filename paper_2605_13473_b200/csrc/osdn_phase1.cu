@@ -393,11 +393,25 @@ template <typename TI, int K, bool VEC> struct PipeBuf {
     static constexpr int R = K / 32;
     float kap[PB][K];                       // k^2
     RawRow<TI, R> kraw[PB][32];             // k as it sits in memory
-    float dt[PB][K];                        // d_t (pre-update), written by the core
+    float x[PB][K];                         // the step's value before the projection (d_{t+1} = clip(x_t)), by the core
+    float d0[K];                            // d on entry to the block, by the core
     float rhov[VEC ? PB : 1][VEC ? K : 1];  // vector retention: exp(l_t) per coordinate
-    float4 scal[PB];                        // e = eta b / n, a2 = e b, rho, -
-    unsigned mask[PB][32];                  // projection pass bits of lane l's coordinates
+    float4 scal[PB];                        // e = eta b / n, a2 = e b, rho, fixed-point scale -> <d_t, k^2>
 };
+
+// What the post role derives from the core's x: d_t of every token (the clipped x of the token before it,
+// the block's entry value for the first) and the projection's pass bits.  The core then carries nothing
+// but the recurrence itself.
+template <int R> __device__ __forceinline__ void clip_row(const float (&x)[R], const Hyper& hy, float (&d)[R], unsigned& bits)
+{
+    bits = 0;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        // inside the box (faces included) exactly when clamping leaves the value alone
+        d[r] = hy.clamp ? fminf(fmaxf(x[r], hy.d_min), hy.d_max) : x[r];
+        bits |= d[r] == x[r] ? (1u << r) : 0u;
+    }
+}
 constexpr int RING_MAX = 6;   // the deeper of the two rings
 struct PipeBars {
     uint64_t full[RING_MAX], done[RING_MAX], free_[RING_MAX];
@@ -409,6 +423,7 @@ template <typename TI, int K, bool VEC>
 __device__ __forceinline__ void pipe_core_block(PipeBuf<TI, K, VEC>& B, int n, float (&d)[K / 32], const Hyper& hy, int lane)
 {
     constexpr int R = K / 32;
+    store_row<R>(B.d0, lane, d);
     auto token = [&](int j) {
         const float4 sc = B.scal[j];
         float kap[R], rho[R];
@@ -424,19 +439,24 @@ __device__ __forceinline__ void pipe_core_block(PipeBuf<TI, K, VEC>& B, int n, f
             al0 = fmaf(d[r], kap[r], al0);
             al1 = fmaf(d[r + 1], kap[r + 1], al1);
         }
-        store_row<R>(B.dt[j], lane, d);
-        const float al = warp_sum(al0 + al1);
-        const float cc = fmaf(-sc.y, al, sc.x);
-        unsigned mybits = 0;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const float x = fmaf(cc, kap[r], rho[r] * d[r]);
-            // inside the box (faces included) exactly when clamping leaves the value alone
-            const float xc = hy.clamp ? fminf(fmaxf(x, hy.d_min), hy.d_max) : x;
-            mybits |= xc == x ? (1u << r) : 0u;
-            d[r] = xc;
+        float al;
+        if (hy.clamp) {
+            // With the projection on, 0 <= <d, k^2> <= d_max sum k^2: the lanes' partial sums are added as
+            // fixed-point integers with one warp-wide instruction instead of five shuffle-add rounds.
+            // sc.w = 2^26 / (d_max sum k^2) (from the pre role): the total stays below 2^27, a lane's
+            // rounding is 2^-27 of the bound, 32 of them 2^-22 of it.
+            const unsigned q = __float2uint_rn((al0 + al1) * sc.w);
+            al = __uint2float_rn(__reduce_add_sync(0xffffffffu, q)) * __frcp_rn(sc.w);
+        } else {
+            al = warp_sum(al0 + al1);
         }
-        B.mask[j][lane] = mybits;
+        const float cc = fmaf(-sc.y, al, sc.x);
+        float x[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) x[r] = fmaf(cc, kap[r], rho[r] * d[r]);
+        store_row<R>(B.x[j], lane, x);
+#pragma unroll
+        for (int r = 0; r < R; ++r) d[r] = hy.clamp ? fminf(fmaxf(x[r], hy.d_min), hy.d_max) : x[r];
         if (lane == 0) B.scal[j].w = al;
     };
     if (n == PB) {   // partly unrolled: the shared-memory reads of later tokens are issued under the shuffles of earlier ones
@@ -479,7 +499,9 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
                 const size_t th = (size_t)(t0 + lane) * H + h;
                 const float rn = fabsf(a.r.n[th]), bb = hy.beta_aware ? a.beta[th] : 1.0f;
                 const float e = hy.eta * bb * rn;
-                B.scal[lane] = make_float4(e, e * bb, a.r.rho[th], 0.f);
+                // .w: the fixed-point scale of the core's sum, 2^26 / (d_max max(sum k^2, eps)); the core
+                // replaces it by <d_t, k^2>
+                B.scal[lane] = make_float4(e, e * bb, a.r.rho[th], 67108864.0f * rn / hy.d_max);
             }
 #pragma unroll
             for (int j = 0; j < PB; ++j) {
@@ -525,18 +547,20 @@ __device__ __forceinline__ bool pipe_stretch(const P1Fwd& a, int h, int t_a, int
             if (!ok) break;
             const PipeBuf<TI, K, VEC>& B = buf[bi];
             const int t0 = t_a + b * PB, n = min(PB, t_b - t0);
+            float dd[R];   // d_t of the token in hand
+            load_row<R>(B.d0, lane, dd);
             auto token = [&](int j) {
                 const size_t th = (size_t)(t0 + j) * H + h;
-                float dd[R], kk[R], wk[R];
-                load_row<R>(B.dt[j], lane, dd);
+                float kk[R], wk[R], xx[R];
                 unpack<R>(B.kraw[j][lane], kk);
 #pragma unroll
                 for (int r = 0; r < R; ++r) wk[r] = dd[r] * kk[r];
                 store_row<R>(kt + th * K, lane, wk);
-                if (a.save) {
-                    store_row<R>(a.r.dtraj + th * K, lane, dd);
-                    a.r.pmask[th * 32 + lane] = B.mask[j][lane];
-                }
+                if (a.save) store_row<R>(a.r.dtraj + th * K, lane, dd);
+                load_row<R>(B.x[j], lane, xx);
+                unsigned bits;
+                clip_row<R>(xx, hy, dd, bits);   // the next token's d, this token's pass bits
+                if (a.save) a.r.pmask[th * 32 + lane] = bits;
             };
             if (a.save && lane < n) a.r.al[(size_t)(t0 + lane) * H + h] = B.scal[lane].w;   // lane j: token j
             if (n == PB) {
@@ -623,7 +647,7 @@ __global__ void __launch_bounds__(96) phase1_stream_kernel(P1Args a)
             if (lane < n) {
                 const float nn = fmaxf(mine, hy.eps), bb = hy.beta_aware ? beta : 1.0f;
                 const float e = hy.eta * bb / nn;
-                B.scal[lane] = make_float4(e, e * bb, scalar_ret ? expf(ret) : 1.0f, 0.f);
+                B.scal[lane] = make_float4(e, e * bb, scalar_ret ? expf(ret) : 1.0f, 67108864.0f / (nn * hy.d_max));
                 sbeta[bi][lane] = beta;
             }
             if constexpr (VEC) {
@@ -664,13 +688,17 @@ __global__ void __launch_bounds__(96) phase1_stream_kernel(P1Args a)
             const PipeBuf<TI, K, VEC>& B = buf[bi];
             const int tb0 = t0 + b * PB, n = min(PB, len - b * PB);
             if (kt) {
+                float dd[R];
+                load_row<R>(B.d0, lane, dd);
                 for (int j = 0; j < n; ++j) {
-                    float dd[R], kk[R], wk[R];
-                    load_row<R>(B.dt[j], lane, dd);
+                    float kk[R], wk[R], xx[R];
                     unpack<R>(B.kraw[j][lane], kk);
 #pragma unroll
                     for (int r = 0; r < R; ++r) wk[r] = dd[r] * kk[r];
                     store_row<R>(kt + ((size_t)(tb0 + j) * H + h) * K, lane, wk);
+                    load_row<R>(B.x[j], lane, xx);
+                    unsigned bits;
+                    clip_row<R>(xx, hy, dd, bits);
                 }
             }
             if (a.ratio || a.log_sum) {
