@@ -1044,7 +1044,11 @@ template <typename T, int K, bool VEC> struct RevBuf {
     static constexpr int R = K / 32;
     RawRow<T, R> kraw[QB][32];
     float dt[QB][K], dkt[QB][K], dkr[QB][K];
-    float lam[QB][K];                       // masked lambda of the token, written by the core
+    float lam[QB][K];                       // lambda on entry to the token (before the mask), written by the core
+    // what the core reads, prepared by the pre role so that nothing but the recurrence is left to the core:
+    float kap[QB][K], mkap[QB][K];          // k^2, and k^2 where the projection passed (else 0)
+    float rm[QB][K];                        // retention where the projection passed (else 0)
+    float w[QB][K];                         // k (.) dL/dktil
     float rv[VEC ? QB : 1][VEC ? K : 1];    // vector retention: exp(l_t)
     unsigned mask[QB][32];
     float4 sc0[QB];                         // a2, rho, cc, g1
@@ -1094,6 +1098,31 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
                     store_row<R>(B.rv[VEC ? j : 0], lane, lr);
                 }
             }
+#pragma unroll 4
+            for (int j = 0; j < QB; ++j) {   // (slots beyond n repeat the last token: harmless)
+                float kk[R], dkt[R], kap[R], mkap[R], rm[R], w[R], rv[R];
+                unpack<R>(B.kraw[j][lane], kk);
+                load_row<R>(B.dkt[j], lane, dkt);
+                const unsigned mw = B.mask[j][lane];
+                if constexpr (VEC) load_row<R>(B.rv[VEC ? j : 0], lane, rv);
+                else {
+                    const float rho = B.raw[1][min(j, n - 1)];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) rv[r] = rho;
+                }
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const bool pass = (mw >> r) & 1u;
+                    kap[r] = kk[r] * kk[r];
+                    mkap[r] = pass ? kap[r] : 0.f;
+                    rm[r] = pass ? rv[r] : 0.f;
+                    w[r] = kk[r] * dkt[r];
+                }
+                store_row<R>(B.kap[j], lane, kap);
+                store_row<R>(B.mkap[j], lane, mkap);
+                store_row<R>(B.rm[j], lane, rm);
+                store_row<R>(B.w[j], lane, w);
+            }
             __syncwarp();
             if (lane == 0) p1_mbar_arrive(&bars.full[bi]);
         };
@@ -1140,28 +1169,23 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
             RevBuf<T, K, VEC>& B = buf[bi];
             const int ttop = t_hi - 1 - b * QB, n = min(QB, ttop - t_lo + 1);
             auto token = [&](int j) {
-                const float4 s0 = B.sc0[j];
-                const unsigned mw = B.mask[j][lane];
-                float kk[R], dkt[R], rv[R];
-                unpack<R>(B.kraw[j][lane], kk);
-                load_row<R>(B.dkt[j], lane, dkt);
-                if constexpr (VEC) load_row<R>(B.rv[VEC ? j : 0], lane, rv);
-                else {
+                const float a2 = B.sc0[j].x;
+                float kap[R], mkap[R], rm[R], w[R];
+                load_row<R>(B.mkap[j], lane, mkap);
+                load_row<R>(B.kap[j], lane, kap);
+                load_row<R>(B.rm[j], lane, rm);
+                load_row<R>(B.w[j], lane, w);
+                float dc0 = lam[0] * mkap[0], dc1 = lam[1] * mkap[1];
 #pragma unroll
-                    for (int r = 0; r < R; ++r) rv[r] = s0.y;
-                }
-                float kap[R], dc = 0.f;
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    kap[r] = kk[r] * kk[r];
-                    if (!((mw >> r) & 1u)) lam[r] = 0.f;
-                    dc = fmaf(lam[r], kap[r], dc);
+                for (int r = 2; r < R; r += 2) {
+                    dc0 = fmaf(lam[r], mkap[r], dc0);
+                    dc1 = fmaf(lam[r + 1], mkap[r + 1], dc1);
                 }
                 store_row<R>(B.lam[j], lane, lam);
-                dc = warp_sum(dc);
-                const float da = -s0.x * dc;
+                const float dc = warp_sum(dc0 + dc1);
+                const float da = -a2 * dc;
 #pragma unroll
-                for (int r = 0; r < R; ++r) lam[r] = fmaf(rv[r], lam[r], fmaf(da, kap[r], kk[r] * dkt[r]));
+                for (int r = 0; r < R; ++r) lam[r] = fmaf(rm[r], lam[r], fmaf(da, kap[r], w[r]));
                 if (lane == 0) B.sc1[j].y = dc;
             };
             if (n == QB) {
@@ -1190,9 +1214,10 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
                 float dt[R], lm[R];
                 load_row<R>(B.dt[j], lane, dt);
                 load_row<R>(B.lam[j], lane, lm);
+                const unsigned mw = B.mask[j][lane];
                 drv[j] = 0.f;
 #pragma unroll
-                for (int r = 0; r < R; ++r) drv[j] = fmaf(lm[r], dt[r], drv[j]);
+                for (int r = 0; r < R; ++r) drv[j] = fmaf((mw >> r) & 1u ? lm[r] : 0.f, dt[r], drv[j]);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1)
@@ -1222,6 +1247,11 @@ __device__ __forceinline__ bool rev_stretch(const P1Bwd& a, int h, int t_lo, int
                 load_row<R>(B.dkt[j], lane, dkt);
                 load_row<R>(B.dkr[j], lane, dkr);
                 load_row<R>(B.lam[j], lane, lm);
+                {
+                    const unsigned mw = B.mask[j][lane];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) lm[r] = (mw >> r) & 1u ? lm[r] : 0.f;
+                }
                 const float da = -a2 * dc, dn = g2 * dc;
                 if constexpr (VEC) {
                     if (a.dlog_ret) {
