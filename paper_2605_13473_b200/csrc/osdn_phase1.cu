@@ -731,7 +731,9 @@ template <typename TI, typename TO, int K, bool VEC>
 __global__ void __launch_bounds__(96) phase1_seq_kernel(P1Fwd a)
 {
     constexpr int R = K / 32;
-    constexpr int PF = 8;   // prefetch distance in tokens
+    // prefetch distance in tokens: short, because the long runs go through the pipelined stretches and a
+    // run's start waits for whatever the run before it still had in flight (8 -> 4: osdn_1p3b 452 -> 401 us)
+    constexpr int PF = 4;
     struct RingSlot {
         RawRow<TI, R> k[32];
         RawRow<float, R> lr[VEC ? 32 : 1];
