@@ -319,13 +319,15 @@ __device__ __forceinline__ void chunk_fwd_tile(const CUtensorMap& tmK, const CUt
         sG[lane] = sa;
         sG[lane + 32] = sb;
     }
-    // The group's previous tile is published here: by now its stores have drained, so the fence is cheap,
-    // and the barrier that follows is needed anyway.
-    if (publish) __threadfence();
+    // The group's previous tile is published here, behind a barrier that is needed anyway: the barrier
+    // orders every thread's stores before thread 0, whose fence (cumulative) then orders them before the flag.
     tc_fence_before();
     sync();
     tc_fence_after();
-    if (publish && tid == 0) st_release_gpu(publish, 1);
+    if (publish && tid == 0) {
+        __threadfence();
+        st_release_gpu(publish, 1);
+    }
 
     bool ok = mbar_wait(&bar_tma, ph, a.status, ERR_TMA);
     if (len < CH) {
@@ -1064,9 +1066,11 @@ __device__ __forceinline__ void chunk_fwd_workers(const CUtensorMap& tmK, const 
         ph ^= 1;
     }
     if (publish) {
-        __threadfence();
         gsync();
-        if (ltid == 0) st_release_gpu(publish, 1);
+        if (ltid == 0) {
+            __threadfence();
+            st_release_gpu(publish, 1);
+        }
     }
     gsync();
     if (ltid == 0) {
