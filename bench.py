@@ -34,6 +34,8 @@ WORKLOADS = {
                                              "non-beta-aware step): B=4 T=4096 H=16 dk=dv=128 bf16"),
     "cfg2_lively": dict(idx=-2, bwd=True, desc="cfg2 shape with a moving preconditioner (eta=0.3, sparse keys, "
                                                "separate retention): B=8 T=2048 H=8 dk=dv=128 bf16"),
+    "oskda": dict(idx=-4, bwd=True, desc="OSKDA extension (one gate per key channel, constant retention 0.999) at the "
+                                         "cfg2 shape: B=8 T=2048 H=8 dk=dv=128 bf16, osdn_kda_fwd + osdn_kda_bwd"),
 }
 
 
@@ -57,6 +59,13 @@ def make_inputs(name):
         hy = OsdnHyper(eta=0.003, apf_mode=2, beta_aware=0)
         return draw("osdn_1p3b", 13, [4096] * 4, 16, 128, 128, "bf16", dense_B=4, hyper=hy, gate_kind="zero",
                     with_dout=True, with_log_ret=True, log_ret_shift=7.0)
+    if w["idx"] == -4:
+        import math
+        import torch
+        hy = OsdnHyper(eta=0.003, apf_mode=2, channel_gate=1)
+        inp = draw("oskda", 5, [2048] * 8, 8, 128, 128, "bf16", dense_B=8, hyper=hy, with_dout=True, with_log_ret=True)
+        inp.log_ret = torch.full_like(inp.log_ret, math.log(0.999))   # the paper's setting for this extension
+        return inp
     hy = OsdnHyper(eta=0.3, apf_mode=2)
     return draw("cfg2_lively", 12, [2048] * 8, 8, 128, 128, "bf16", dense_B=8, hyper=hy, key_kind="sparse",
                 with_dout=True, with_log_ret=True)
@@ -85,6 +94,10 @@ def method_bytes(name, inp, with_bwd):
         "tc_fwd": 2 * K * es + 8 + V * es + V * es + (state if with_bwd else 0),   # both passes in one launch
         # q, k, v, dout, beta, gate, the saved state in; dq, dk, dv, dbeta, dgate out
         "tc_bwd": (2 * K + 2 * V) * es + 8 + state + (2 * K + V) * es + 8,
+        # channel-gate extension: q, k, v, beta, K gates in, out; the backward reads them again with dout and
+        # writes dq, dk, dv, dbeta and K gate gradients
+        "kda_fwd": (2 * K + 2 * V) * es + 4 + 4 * K,
+        "kda_bwd": (2 * K + 2 * V) * es + 4 + 4 * K + (2 * K + V) * es + 4 + 4 * K,
     }
     return None if name not in per else per[name] * tokh
 
@@ -131,6 +144,11 @@ def kernel_model(name, inp, NT):
                    tiles * (f(128, 64, C) + f(128, 64, K) + 2 * f(128, 128, C))
                    + tiles * (2 * f(64, 64, K) + 3 * f(128, 64, K) + 2 * f(64, 64, K) + 2 * f(128, 64, C)
                               + 2 * f(64, 64, C) + 4 * f(128, 64, C)), "hbm")
+    # channel-gate extension, token-recurrent on CUDA cores: per token and state row K decays, K + K + K fused
+    # multiply-adds forward (read, write, output); the backward replays the forward's two and takes about
+    # seven more per element for the adjoint
+    m["kda_fwd"] = (tokh * ((2 * K + 2 * V) * es + 4 + 8 * K) + tiles * 4 * V * K, tokh * V * K * 8.0, "alu")
+    m["kda_bwd"] = (tokh * ((4 * K + 3 * V) * es + 8 + 24 * K) + tiles * 4 * V * K, tokh * V * K * 20.0, "alu")
     return m.get(name)
 
 
