@@ -264,11 +264,18 @@ __global__ void __launch_bounds__(KF_WARPS * 32) kda_fwd_kernel(KdaArgs a)
         if (a.final_state) store_vec<R>(a.final_state + srow + (size_t)r * K, S[r]);
 }
 
+// Backward: one warp per state row, KB_WARPS rows per CTA.  The token operands (k, q, ktil, gates) of a
+// block of KTB tokens are staged once per CTA in shared memory, one block ahead, for the replay (forward
+// order) as for the adjoint steps (reverse order); a row's per-token scalars (v, beta, dout) travel in one
+// register per block; the row before a token comes from the history one token ahead of its use.
 template <typename T, int K>
 __global__ void __launch_bounds__(KB_WARPS * 32) kda_bwd_kernel(KdaArgs a)
 {
     constexpr int R = K / 32;
-    extern __shared__ float red[];                 // [2][KB_WARPS][4][K]: per-row terms of dq, dk, d ktil, d gate
+    constexpr int NT = KB_WARPS * 32;
+    extern __shared__ __align__(16) uint8_t kda_dyn[];
+    float* red = reinterpret_cast<float*>(kda_dyn);   // [2][KB_WARPS][4][K]: per-row terms of dq, dk, d ktil, d gate
+    TokBlock<T, K>* blk = reinterpret_cast<TokBlock<T, K>*>(kda_dyn + (size_t)2 * KB_WARPS * 4 * K * sizeof(float));
     __shared__ float red_beta[2][KB_WARPS];
     const int H = a.H, V = a.V;
     const int chain = blockIdx.y, s = chain / H, h = chain - s * H;
@@ -285,72 +292,119 @@ __global__ void __launch_bounds__(KB_WARPS * 32) kda_bwd_kernel(KdaArgs a)
         for (int x = 0; x < R; ++x) Shat.x[x] = 0.f;
     int it = 0;
     for (int n = nchunks - 1; n >= 0; --n) {
-        const int clen = min(CH, len - n * CH);
-        const size_t th0 = (size_t)(t0 + n * CH) * H + h;
-        // replay the chunk from its checkpoint, keeping the row before every token
+        const int clen = min(CH, len - n * CH), nb = (clen + KTB - 1) / KTB;
+        const int tc0 = t0 + n * CH;                       // first token of the chunk
+        // lane j < KTB: v of token j of block b for this row; KTB + j: beta; 2 KTB + j: dout
+        auto scalars = [&](int b) {
+            float x = 0.f;
+            const int j = lane & (KTB - 1), t = b * KTB + j, kind = lane / KTB;
+            if (b >= 0 && b < nb && t < clen && kind < 3) {
+                const size_t th = (size_t)(tc0 + t) * H + h;
+                x = kind == 0 ? ldf(static_cast<const T*>(a.v) + th * V + row)
+                  : kind == 1 ? a.beta[th] : ldf(static_cast<const T*>(a.dout) + th * V + row);
+            }
+            return x;
+        };
+        auto fill = [&](int b, int slot) {
+            if (b >= 0 && b < nb)
+                fill_block<T, K>(blk[slot], a, (size_t)(tc0 + b * KTB) * H + h, H, min(KTB, clen - b * KTB), tid, NT);
+            cp_async_commit_group();
+        };
+        // ---- replay the chunk from its checkpoint, keeping the row before every token
         {
             Vec<R> S = load_vec<R>(a.ckpt + (((size_t)(c0 + n) * H + h) * V + row) * K + R * lane);
-            for (int j = 0; j < clen; ++j) {
-                store_vec<R>(hist + (size_t)j * K, S);
-                const Tok<R> tk = load_tok<T, R>(a, th0 + (size_t)j * H, K, row, lane);
-                row_step<R>(S, tk, nullptr);
+            fill(0, 0);
+            float sc = scalars(0);
+            for (int b = 0; b < nb; ++b) {
+                fill(b + 1, (b + 1) & 1);
+                const float sc_next = scalars(b + 1);
+                cp_async_wait_group<1>();
+                __syncthreads();
+                const TokBlock<T, K>& B = blk[b & 1];
+                const int nt = min(KTB, clen - b * KTB);
+                for (int j = 0; j < nt; ++j) {
+                    store_vec<R>(hist + (size_t)(b * KTB + j) * K, S);
+                    const Tok<R> tk = tok_from_block<T, K, R>(B, j, lane, __shfl_sync(0xffffffffu, sc, j),
+                                                              __shfl_sync(0xffffffffu, sc, KTB + j));
+                    row_step<R>(S, tk, nullptr);
+                }
+                sc = sc_next;
+                __syncthreads();
             }
         }
-        for (int j = clen - 1; j >= 0; --j, ++it) {
-            const size_t th = th0 + (size_t)j * H;
-            const Tok<R> tk = load_tok<T, R>(a, th, K, row, lane);
-            const Vec<R> q = load_vec<R>(static_cast<const T*>(a.q) + th * K + R * lane);
-            const float sdo = a.scale * ldf(static_cast<const T*>(a.dout) + th * V + row);
-            Vec<R> St = load_vec<R>(hist + (size_t)j * K), Sbar;
-            const float u = row_step<R>(St, tk, &Sbar);
-            float* buf = red + ((size_t)(it & 1) * KB_WARPS + warp) * 4 * K + R * lane;
-            Vec<R> part;
-            // o_t = scale S_t q_t
-            float w = 0.f;
-#pragma unroll
-            for (int x = 0; x < R; ++x) {
-                part.x[x] = sdo * St.x[x];
-                Shat.x[x] = fmaf(sdo, q.x[x], Shat.x[x]);
-                w = fmaf(Shat.x[x], tk.kt.x[x], w);
-            }
-            store_vec<R>(buf, part);                              // dq
-            // S_t = Sbar + beta u ktil^T
-            w = warp_sum(w);
-            const float du = tk.beta * w;
-#pragma unroll
-            for (int x = 0; x < R; ++x) part.x[x] = tk.beta * u * Shat.x[x];
-            store_vec<R>(buf + 2 * K, part);                      // d ktil
-            // u = v - Sbar k ; Sbar = S_{t-1} Diag(alpha)
-            Vec<R> dkp, dgp;
-#pragma unroll
-            for (int x = 0; x < R; ++x) {
-                dkp.x[x] = -Sbar.x[x] * du;
-                const float dsb = fmaf(-du, tk.k.x[x], Shat.x[x]);
-                dgp.x[x] = dsb * Sbar.x[x];
-                Shat.x[x] = __expf(tk.g.x[x]) * dsb;
-            }
-            store_vec<R>(buf + K, dkp);                           // dk (read key)
-            store_vec<R>(buf + 3 * K, dgp);                       // d gate
-            if (lane == 0) {
-                red_beta[it & 1][warp] = u * w;
-                stf(static_cast<T*>(a.dv) + th * V + row, du);
-            }
+        // ---- adjoint steps, last token first
+        fill(nb - 1, 0);
+        float sc = scalars(nb - 1);
+        Vec<R> Sprev = load_vec<R>(hist + (size_t)(clen - 1) * K);
+        for (int b = nb - 1, step = 0; b >= 0; --b, ++step) {
+            fill(b - 1, (step + 1) & 1);
+            const float sc_next = scalars(b - 1);
+            cp_async_wait_group<1>();
             __syncthreads();
-            // sums over the CTA's rows; the buffers alternate, so one barrier per token is enough
-            if (tid < 4 * K) {
-                const float* src = red + (size_t)(it & 1) * KB_WARPS * 4 * K + tid;
-                float sum = 0.f;
+            const TokBlock<T, K>& B = blk[step & 1];
+            const int nt = min(KTB, clen - b * KTB);
+            for (int j = nt - 1; j >= 0; --j, ++it) {
+                const int jj = b * KTB + j;
+                const size_t th = (size_t)(tc0 + jj) * H + h;
+                const Tok<R> tk = tok_from_block<T, K, R>(B, j, lane, __shfl_sync(0xffffffffu, sc, j),
+                                                          __shfl_sync(0xffffffffu, sc, KTB + j));
+                const Vec<R> q = load_vec<R>(B.q[j] + R * lane);
+                const float sdo = a.scale * __shfl_sync(0xffffffffu, sc, 2 * KTB + j);
+                Vec<R> St = Sprev, Sbar;
+                if (jj > 0) Sprev = load_vec<R>(hist + (size_t)(jj - 1) * K);   // the next step's row, a token ahead
+                const float u = row_step<R>(St, tk, &Sbar);
+                float* buf = red + ((size_t)(it & 1) * KB_WARPS + warp) * 4 * K + R * lane;
+                Vec<R> part;
+                // o_t = scale S_t q_t
+                float w = 0.f;
+#pragma unroll
+                for (int x = 0; x < R; ++x) {
+                    part.x[x] = sdo * St.x[x];
+                    Shat.x[x] = fmaf(sdo, q.x[x], Shat.x[x]);
+                    w = fmaf(Shat.x[x], tk.kt.x[x], w);
+                }
+                store_vec<R>(buf, part);                              // dq
+                // S_t = Sbar + beta u ktil^T
+                w = warp_sum(w);
+                const float du = tk.beta * w;
+#pragma unroll
+                for (int x = 0; x < R; ++x) part.x[x] = tk.beta * u * Shat.x[x];
+                store_vec<R>(buf + 2 * K, part);                      // d ktil
+                // u = v - Sbar k ; Sbar = S_{t-1} Diag(alpha)
+                Vec<R> dkp, dgp;
+#pragma unroll
+                for (int x = 0; x < R; ++x) {
+                    dkp.x[x] = -Sbar.x[x] * du;
+                    const float dsb = fmaf(-du, tk.k.x[x], Shat.x[x]);
+                    dgp.x[x] = dsb * Sbar.x[x];
+                    Shat.x[x] = __expf(tk.g.x[x]) * dsb;
+                }
+                store_vec<R>(buf + K, dkp);                           // dk (read key)
+                store_vec<R>(buf + 3 * K, dgp);                       // d gate
+                if (lane == 0) {
+                    red_beta[it & 1][warp] = u * w;
+                    stf(static_cast<T*>(a.dv) + th * V + row, du);
+                }
+                __syncthreads();
+                // sums over the CTA's rows; the buffers alternate, so one barrier per token is enough
+                if (tid < 4 * K) {
+                    const float* src = red + (size_t)(it & 1) * KB_WARPS * 4 * K + tid;
+                    float sum = 0.f;
 #pragma unroll 8
-                for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += src[(size_t)w2 * 4 * K];
-                const int m = tid / K, i = tid - m * K;
-                float* dst = m == 0 ? a.dq_acc : m == 1 ? a.dkread : m == 2 ? a.dktil : a.dgate;
-                atomicAdd(dst + th * K + i, sum);
-            } else if (tid == 4 * K) {
-                float sum = 0.f;
-                for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += red_beta[it & 1][w2];
-                atomicAdd(a.dbeta + th, sum);
+                    for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += src[(size_t)w2 * 4 * K];
+                    const int m = tid / K, i = tid - m * K;
+                    float* dst = m == 0 ? a.dq_acc : m == 1 ? a.dkread : m == 2 ? a.dktil : a.dgate;
+                    atomicAdd(dst + th * K + i, sum);
+                } else if (tid == 4 * K) {
+                    float sum = 0.f;
+                    for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += red_beta[it & 1][w2];
+                    atomicAdd(a.dbeta + th, sum);
+                }
             }
+            sc = sc_next;
+            __syncthreads();   // everybody is done with the block before it is refilled
         }
+        cp_async_wait_group<0>();
     }
     if (a.dinit_state) store_vec<R>(a.dinit_state + srow, Shat);
 }
@@ -430,7 +484,9 @@ int kda_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void*
         cudaMemsetAsync(k.dbeta, 0, Ttot * p.H * 4, st) != cudaSuccess)
         return -1;
     const dim3 grid(p.V / KB_WARPS, L.S * p.H);
-    const size_t smem = (size_t)2 * KB_WARPS * 4 * p.K * sizeof(float);
+    const size_t es = p.io_dtype == OSDN_BF16 ? 2 : 4;
+    // the row sums' double buffer, then two token blocks (k, q in the I/O type; ktil, gates fp32)
+    const size_t smem = (size_t)2 * KB_WARPS * 4 * p.K * sizeof(float) + 2 * (size_t)KTB * p.K * (2 * es + 8);
     stage_mark(st, "kda_bwd");
     auto launch = [&](auto kernel) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
