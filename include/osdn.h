@@ -203,8 +203,9 @@ int osdn_decode_step(const osdn_params* p, const void* q, const void* k, const v
  *            the flags, the alignment rules, ownership and the error codes are those of osdn_fwd / osdn_bwd.
  *   dgate_k  [T,H,K] fp32, written in full.
  *   workspace: osdn_kda_workspace_bytes(p, need_bwd) bytes (0 is returned for rejected parameters); for
- *            the backward it includes, beside the regions of osdn_workspace_bytes, one row history of a
- *            chunk per state row (S * H * V * 64 * K floats) and an fp32 accumulator for dq.
+ *            the backward it includes, beside the regions of osdn_workspace_bytes, one row history of 16
+ *            tokens and four row checkpoints per state row (S * H * V * 20 * K floats) and an fp32
+ *            accumulator for dq.
  * This path runs on CUDA cores in fp32 for both io_dtypes (one warp per state row, sequential over the
  * tokens of a sequence): it is the extension's reference implementation on the device, not a tuned one.
  */

@@ -15,7 +15,10 @@ namespace osdn {
 namespace {
 
 constexpr int KF_WARPS = 8, KF_RW = 4;   // forward: warps per CTA, state rows per warp
-constexpr int KB_WARPS = 32;   // backward: state rows per CTA
+constexpr int KB_WARPS = 16, KB_RW = 2;   // backward: warps per CTA, state rows per warp
+// The backward keeps the rows before the tokens of a SUB-token stretch only (the history then stays in L2): a
+// chunk is walked once to leave a row checkpoint at every stretch start, then stretch by stretch in reverse.
+constexpr int SUB = 16, NSUB = CH / SUB, HROWS = SUB + NSUB;   // history rows per state row: a stretch, then the checkpoints
 
 template <int R> struct Vec {
     float x[R];
@@ -77,7 +80,8 @@ struct KdaArgs {
     void* dv;
     float *dq_acc, *dkread, *dktil, *dgate, *dbeta;   // zeroed accumulators
     float* dinit_state;           // nullable
-    float* hist;                  // [chain, V, CH, K] rows before every token of the chunk in progress
+    float* hist;                  // [chain, V, HROWS, K] rows before every token of the stretch in progress, then
+                                  // the stretch checkpoints of the chunk in progress
 };
 
 // What a row needs of one token.
@@ -264,149 +268,206 @@ __global__ void __launch_bounds__(KF_WARPS * 32) kda_fwd_kernel(KdaArgs a)
         if (a.final_state) store_vec<R>(a.final_state + srow + (size_t)r * K, S[r]);
 }
 
-// Backward: one warp per state row, KB_WARPS rows per CTA.  The token operands (k, q, ktil, gates) of a
-// block of KTB tokens are staged once per CTA in shared memory, one block ahead, for the replay (forward
-// order) as for the adjoint steps (reverse order); a row's per-token scalars (v, beta, dout) travel in one
-// register per block; the row before a token comes from the history one token ahead of its use.
+// Backward: a warp owns KB_RW state rows, KB_WARPS warps per CTA.  The token operands (k, q, ktil, gates) of
+// a block of KTB tokens are staged once per CTA in shared memory, one block ahead, for the replay (forward
+// order) as for the adjoint steps (reverse order); the rows' per-token scalars (v, dout; beta) travel in
+// registers, one block at a time; the rows before a token come from the history one token ahead of their
+// use.  The rows' contributions to dq, dk, d ktil and d gate are added up inside the warp first.
 template <typename T, int K>
-__global__ void __launch_bounds__(KB_WARPS * 32) kda_bwd_kernel(KdaArgs a)
+__global__ void __launch_bounds__(KB_WARPS * 32, 2) kda_bwd_kernel(KdaArgs a)
 {
     constexpr int R = K / 32;
-    constexpr int NT = KB_WARPS * 32;
+    constexpr int NT = KB_WARPS * 32, RW = KB_RW;
+    static_assert(2 * KTB * RW <= 32, "one lane per (kind, token of the block, row of the warp)");
     extern __shared__ __align__(16) uint8_t kda_dyn[];
-    float* red = reinterpret_cast<float*>(kda_dyn);   // [2][KB_WARPS][4][K]: per-row terms of dq, dk, d ktil, d gate
+    float* red = reinterpret_cast<float*>(kda_dyn);   // [2][KB_WARPS][4][K]: per-warp terms of dq, dk, d ktil, d gate
     TokBlock<T, K>* blk = reinterpret_cast<TokBlock<T, K>*>(kda_dyn + (size_t)2 * KB_WARPS * 4 * K * sizeof(float));
     __shared__ float red_beta[2][KB_WARPS];
     const int H = a.H, V = a.V;
     const int chain = blockIdx.y, s = chain / H, h = chain - s * H;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int row = blockIdx.x * KB_WARPS + warp;
+    const int row0 = (blockIdx.x * KB_WARPS + warp) * RW;
     const int t0 = a.tab.seq_tok0(s), len = a.tab.seq_len(s), c0 = a.tab.seq_chunk0(s);
     const int nchunks = (len + CH - 1) / CH;
-    const size_t srow = (((size_t)s * H + h) * V + row) * K + R * lane;
-    float* hist = a.hist + ((size_t)chain * V + row) * CH * K + R * lane;
-    Vec<R> Shat;
-    if (a.dfinal_state) Shat = load_vec<R>(a.dfinal_state + srow);
-    else
+    const size_t srow = (((size_t)s * H + h) * V + row0) * K + R * lane;
+    float* hist = a.hist + ((size_t)chain * V + row0) * HROWS * K + R * lane;   // row r of the warp: + r HROWS K
+    Vec<R> Shat[RW];
 #pragma unroll
-        for (int x = 0; x < R; ++x) Shat.x[x] = 0.f;
+    for (int r = 0; r < RW; ++r) {
+        if (a.dfinal_state) Shat[r] = load_vec<R>(a.dfinal_state + srow + (size_t)r * K);
+        else
+#pragma unroll
+            for (int x = 0; x < R; ++x) Shat[r].x[x] = 0.f;
+    }
     int it = 0;
     for (int n = nchunks - 1; n >= 0; --n) {
         const int clen = min(CH, len - n * CH), nb = (clen + KTB - 1) / KTB;
         const int tc0 = t0 + n * CH;                       // first token of the chunk
-        // lane j < KTB: v of token j of block b for this row; KTB + j: beta; 2 KTB + j: dout
-        auto scalars = [&](int b) {
-            float x = 0.f;
-            const int j = lane & (KTB - 1), t = b * KTB + j, kind = lane / KTB;
-            if (b >= 0 && b < nb && t < clen && kind < 3) {
+        // lane (kind, j, r) = kind KTB RW + j RW + r: kind 0 the row's v of token j of block b, kind 1 its dout
+        auto scalars = [&](int b, float& sv, float& sbeta) {
+            sv = 0.f;
+            sbeta = 0.f;
+            const int kind = lane / (KTB * RW), j = (lane / RW) % KTB, r = lane % RW, t = b * KTB + j;
+            if (b >= 0 && b < nb && t < clen && kind < 2) {
                 const size_t th = (size_t)(tc0 + t) * H + h;
-                x = kind == 0 ? ldf(static_cast<const T*>(a.v) + th * V + row)
-                  : kind == 1 ? a.beta[th] : ldf(static_cast<const T*>(a.dout) + th * V + row);
+                sv = ldf(static_cast<const T*>(kind == 0 ? a.v : a.dout) + th * V + row0 + r);
             }
-            return x;
+            if (b >= 0 && b < nb && lane < KTB && b * KTB + lane < clen) sbeta = a.beta[(size_t)(tc0 + b * KTB + lane) * H + h];
         };
         auto fill = [&](int b, int slot) {
             if (b >= 0 && b < nb)
                 fill_block<T, K>(blk[slot], a, (size_t)(tc0 + b * KTB) * H + h, H, min(KTB, clen - b * KTB), tid, NT);
             cp_async_commit_group();
         };
-        // ---- replay the chunk from its checkpoint, keeping the row before every token
+        // forward steps of the warp's rows over one staged block (optionally keeping the rows before each token)
+        auto forward_block = [&](const TokBlock<T, K>& B, int nt, float sv, float sbeta, Vec<R> (&S)[RW], int hist_at) {
+            for (int j = 0; j < nt; ++j) {
+                const float beta = __shfl_sync(0xffffffffu, sbeta, j);
+#pragma unroll
+                for (int r = 0; r < RW; ++r) {
+                    if (hist_at >= 0) store_vec<R>(hist + ((size_t)r * HROWS + hist_at + j) * K, S[r]);
+                    const Tok<R> tk = tok_from_block<T, K, R>(B, j, lane, __shfl_sync(0xffffffffu, sv, j * RW + r), beta);
+                    row_step<R>(S[r], tk, nullptr);
+                }
+            }
+        };
+        // ---- once through the chunk: a row checkpoint at the start of every stretch of SUB tokens
         {
-            Vec<R> S = load_vec<R>(a.ckpt + (((size_t)(c0 + n) * H + h) * V + row) * K + R * lane);
+            Vec<R> S[RW];
+#pragma unroll
+            for (int r = 0; r < RW; ++r) S[r] = load_vec<R>(a.ckpt + (((size_t)(c0 + n) * H + h) * V + row0 + r) * K + R * lane);
             fill(0, 0);
-            float sc = scalars(0);
+            float sv, sbeta;
+            scalars(0, sv, sbeta);
             for (int b = 0; b < nb; ++b) {
                 fill(b + 1, (b + 1) & 1);
-                const float sc_next = scalars(b + 1);
+                float sv_next, sbeta_next;
+                scalars(b + 1, sv_next, sbeta_next);
                 cp_async_wait_group<1>();
                 __syncthreads();
-                const TokBlock<T, K>& B = blk[b & 1];
-                const int nt = min(KTB, clen - b * KTB);
-                for (int j = 0; j < nt; ++j) {
-                    store_vec<R>(hist + (size_t)(b * KTB + j) * K, S);
-                    const Tok<R> tk = tok_from_block<T, K, R>(B, j, lane, __shfl_sync(0xffffffffu, sc, j),
-                                                              __shfl_sync(0xffffffffu, sc, KTB + j));
-                    row_step<R>(S, tk, nullptr);
+                if ((b * KTB) % SUB == 0) {
+#pragma unroll
+                    for (int r = 0; r < RW; ++r) store_vec<R>(hist + ((size_t)r * HROWS + SUB + b * KTB / SUB) * K, S[r]);
                 }
-                sc = sc_next;
+                forward_block(blk[b & 1], min(KTB, clen - b * KTB), sv, sbeta, S, -1);
+                sv = sv_next;
+                sbeta = sbeta_next;
                 __syncthreads();
             }
         }
-        // ---- adjoint steps, last token first
-        fill(nb - 1, 0);
-        float sc = scalars(nb - 1);
-        Vec<R> Sprev = load_vec<R>(hist + (size_t)(clen - 1) * K);
-        for (int b = nb - 1, step = 0; b >= 0; --b, ++step) {
-            fill(b - 1, (step + 1) & 1);
-            const float sc_next = scalars(b - 1);
-            cp_async_wait_group<1>();
-            __syncthreads();
-            const TokBlock<T, K>& B = blk[step & 1];
-            const int nt = min(KTB, clen - b * KTB);
-            for (int j = nt - 1; j >= 0; --j, ++it) {
-                const int jj = b * KTB + j;
-                const size_t th = (size_t)(tc0 + jj) * H + h;
-                const Tok<R> tk = tok_from_block<T, K, R>(B, j, lane, __shfl_sync(0xffffffffu, sc, j),
-                                                          __shfl_sync(0xffffffffu, sc, KTB + j));
-                const Vec<R> q = load_vec<R>(B.q[j] + R * lane);
-                const float sdo = a.scale * __shfl_sync(0xffffffffu, sc, 2 * KTB + j);
-                Vec<R> St = Sprev, Sbar;
-                if (jj > 0) Sprev = load_vec<R>(hist + (size_t)(jj - 1) * K);   // the next step's row, a token ahead
-                const float u = row_step<R>(St, tk, &Sbar);
-                float* buf = red + ((size_t)(it & 1) * KB_WARPS + warp) * 4 * K + R * lane;
-                Vec<R> part;
-                // o_t = scale S_t q_t
-                float w = 0.f;
+        for (int sb = (clen - 1) / SUB; sb >= 0; --sb) {
+            const int b_lo = sb * (SUB / KTB), b_hi = min(nb, (sb + 1) * (SUB / KTB));   // token blocks of the stretch
+            const int s_tok0 = sb * SUB, s_len = min(SUB, clen - s_tok0);
+            // ---- replay the stretch from its checkpoint, keeping the rows before every token
+            {
+                Vec<R> S[RW];
 #pragma unroll
-                for (int x = 0; x < R; ++x) {
-                    part.x[x] = sdo * St.x[x];
-                    Shat.x[x] = fmaf(sdo, q.x[x], Shat.x[x]);
-                    w = fmaf(Shat.x[x], tk.kt.x[x], w);
-                }
-                store_vec<R>(buf, part);                              // dq
-                // S_t = Sbar + beta u ktil^T
-                w = warp_sum(w);
-                const float du = tk.beta * w;
-#pragma unroll
-                for (int x = 0; x < R; ++x) part.x[x] = tk.beta * u * Shat.x[x];
-                store_vec<R>(buf + 2 * K, part);                      // d ktil
-                // u = v - Sbar k ; Sbar = S_{t-1} Diag(alpha)
-                Vec<R> dkp, dgp;
-#pragma unroll
-                for (int x = 0; x < R; ++x) {
-                    dkp.x[x] = -Sbar.x[x] * du;
-                    const float dsb = fmaf(-du, tk.k.x[x], Shat.x[x]);
-                    dgp.x[x] = dsb * Sbar.x[x];
-                    Shat.x[x] = __expf(tk.g.x[x]) * dsb;
-                }
-                store_vec<R>(buf + K, dkp);                           // dk (read key)
-                store_vec<R>(buf + 3 * K, dgp);                       // d gate
-                if (lane == 0) {
-                    red_beta[it & 1][warp] = u * w;
-                    stf(static_cast<T*>(a.dv) + th * V + row, du);
-                }
-                __syncthreads();
-                // sums over the CTA's rows; the buffers alternate, so one barrier per token is enough
-                if (tid < 4 * K) {
-                    const float* src = red + (size_t)(it & 1) * KB_WARPS * 4 * K + tid;
-                    float sum = 0.f;
-#pragma unroll 8
-                    for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += src[(size_t)w2 * 4 * K];
-                    const int m = tid / K, i = tid - m * K;
-                    float* dst = m == 0 ? a.dq_acc : m == 1 ? a.dkread : m == 2 ? a.dktil : a.dgate;
-                    atomicAdd(dst + th * K + i, sum);
-                } else if (tid == 4 * K) {
-                    float sum = 0.f;
-                    for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += red_beta[it & 1][w2];
-                    atomicAdd(a.dbeta + th, sum);
+                for (int r = 0; r < RW; ++r) S[r] = load_vec<R>(hist + ((size_t)r * HROWS + SUB + sb) * K);
+                fill(b_lo, 0);
+                float sv, sbeta;
+                scalars(b_lo, sv, sbeta);
+                for (int b = b_lo, step = 0; b < b_hi; ++b, ++step) {
+                    if (b + 1 < b_hi) fill(b + 1, (step + 1) & 1);
+                    else cp_async_commit_group();
+                    float sv_next, sbeta_next;
+                    scalars(b + 1 < b_hi ? b + 1 : -1, sv_next, sbeta_next);
+                    cp_async_wait_group<1>();
+                    __syncthreads();
+                    forward_block(blk[step & 1], min(KTB, clen - b * KTB), sv, sbeta, S, b * KTB - s_tok0);
+                    sv = sv_next;
+                    sbeta = sbeta_next;
+                    __syncthreads();
                 }
             }
-            sc = sc_next;
-            __syncthreads();   // everybody is done with the block before it is refilled
+            // ---- adjoint steps of the stretch, last token first
+            fill(b_hi - 1, 0);
+            float sv, sbeta;
+            scalars(b_hi - 1, sv, sbeta);
+            Vec<R> Sprev[RW];
+#pragma unroll
+            for (int r = 0; r < RW; ++r) Sprev[r] = load_vec<R>(hist + ((size_t)r * HROWS + s_len - 1) * K);
+            for (int b = b_hi - 1, step = 0; b >= b_lo; --b, ++step) {
+                if (b - 1 >= b_lo) fill(b - 1, (step + 1) & 1);
+                else cp_async_commit_group();
+                float sv_next, sbeta_next;
+                scalars(b - 1 >= b_lo ? b - 1 : -1, sv_next, sbeta_next);
+                cp_async_wait_group<1>();
+                __syncthreads();
+                const TokBlock<T, K>& B = blk[step & 1];
+                const int nt = min(KTB, clen - b * KTB);
+                for (int j = nt - 1; j >= 0; --j, ++it) {
+                    const int jj = b * KTB + j;
+                    const size_t th = (size_t)(tc0 + jj) * H + h;
+                    const float beta = __shfl_sync(0xffffffffu, sbeta, j);
+                    const Vec<R> q = load_vec<R>(B.q[j] + R * lane);
+                    Vec<R> pq, pk, pkt, pg;   // the warp's rows added up: dq, dk (read key), d ktil, d gate
+#pragma unroll
+                    for (int x = 0; x < R; ++x) pq.x[x] = pk.x[x] = pkt.x[x] = pg.x[x] = 0.f;
+                    float pbeta = 0.f, myv = 0.f;
+#pragma unroll
+                    for (int r = 0; r < RW; ++r) {
+                        const Tok<R> tk = tok_from_block<T, K, R>(B, j, lane, __shfl_sync(0xffffffffu, sv, j * RW + r), beta);
+                        const float sdo = a.scale * __shfl_sync(0xffffffffu, sv, KTB * RW + j * RW + r);
+                        Vec<R> St = Sprev[r], Sbar;
+                        if (jj > s_tok0) Sprev[r] = load_vec<R>(hist + ((size_t)r * HROWS + jj - 1 - s_tok0) * K);   // the next step's row
+                        const float u = row_step<R>(St, tk, &Sbar);
+                        // o_t = scale S_t q_t
+                        float w = 0.f;
+#pragma unroll
+                        for (int x = 0; x < R; ++x) {
+                            pq.x[x] = fmaf(sdo, St.x[x], pq.x[x]);
+                            Shat[r].x[x] = fmaf(sdo, q.x[x], Shat[r].x[x]);
+                            w = fmaf(Shat[r].x[x], tk.kt.x[x], w);
+                        }
+                        // S_t = Sbar + beta u ktil^T
+                        w = warp_sum(w);
+                        const float du = beta * w, bu = beta * u;
+                        pbeta = fmaf(u, w, pbeta);
+                        // u = v - Sbar k ; Sbar = S_{t-1} Diag(alpha)
+#pragma unroll
+                        for (int x = 0; x < R; ++x) {
+                            pkt.x[x] = fmaf(bu, Shat[r].x[x], pkt.x[x]);
+                            pk.x[x] = fmaf(-Sbar.x[x], du, pk.x[x]);
+                            const float dsb = fmaf(-du, tk.k.x[x], Shat[r].x[x]);
+                            pg.x[x] = fmaf(dsb, Sbar.x[x], pg.x[x]);
+                            Shat[r].x[x] = __expf(tk.g.x[x]) * dsb;
+                        }
+                        myv = lane == r ? du : myv;
+                    }
+                    float* buf = red + ((size_t)(it & 1) * KB_WARPS + warp) * 4 * K + R * lane;
+                    store_vec<R>(buf, pq);
+                    store_vec<R>(buf + K, pk);
+                    store_vec<R>(buf + 2 * K, pkt);
+                    store_vec<R>(buf + 3 * K, pg);
+                    if (lane == 0) red_beta[it & 1][warp] = pbeta;
+                    if (lane < RW) stf(static_cast<T*>(a.dv) + th * V + row0 + lane, myv);
+                    __syncthreads();
+                    // sums over the CTA's warps; the buffers alternate, so one barrier per token is enough
+                    for (int o = tid; o < 4 * K; o += NT) {
+                        const float* src = red + (size_t)(it & 1) * KB_WARPS * 4 * K + o;
+                        float sum = 0.f;
+#pragma unroll 8
+                        for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += src[(size_t)w2 * 4 * K];
+                        const int m = o / K, i = o - m * K;
+                        float* dst = m == 0 ? a.dq_acc : m == 1 ? a.dkread : m == 2 ? a.dktil : a.dgate;
+                        atomicAdd(dst + th * K + i, sum);
+                    }
+                    if (tid == NT - 1) {
+                        float sum = 0.f;
+                        for (int w2 = 0; w2 < KB_WARPS; ++w2) sum += red_beta[it & 1][w2];
+                        atomicAdd(a.dbeta + th, sum);
+                    }
+                }
+                sv = sv_next;
+                sbeta = sbeta_next;
+                __syncthreads();   // everybody is done with the block before it is refilled
+            }
         }
         cp_async_wait_group<0>();
     }
-    if (a.dinit_state) store_vec<R>(a.dinit_state + srow, Shat);
+#pragma unroll
+    for (int r = 0; r < RW; ++r)
+        if (a.dinit_state) store_vec<R>(a.dinit_state + srow + (size_t)r * K, Shat[r]);
 }
 
 template <typename T> __global__ void cast_rows_kernel(const float* src, T* dst, size_t n)
@@ -421,7 +482,7 @@ size_t kda_extra_bytes(const osdn_params& p, const WsLayout& L, bool need_bwd)
 {
     if (!need_bwd) return 0;
     const size_t Ttot = p.nseq > 0 ? (size_t)p.T : (size_t)p.B * p.T;
-    const size_t hist = align_up((size_t)L.S * p.H * p.V * CH * p.K * 4, 256);
+    const size_t hist = align_up((size_t)L.S * p.H * p.V * HROWS * p.K * 4, 256);
     const size_t dq = align_up(Ttot * p.H * p.K * 4, 256);
     return hist + dq;
 }
@@ -475,7 +536,7 @@ int kda_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void*
     k.dout = a.dout; k.dfinal_state = a.dfinal_state; k.dv = a.dv; k.dinit_state = a.dinit_state;
     k.hist = reinterpret_cast<float*>(w + align_up(L.total, 256));
     k.dq_acc = reinterpret_cast<float*>(w + align_up(L.total, 256) +
-                                        align_up((size_t)L.S * p.H * p.V * CH * p.K * 4, 256));
+                                        align_up((size_t)L.S * p.H * p.V * HROWS * p.K * 4, 256));
     k.dkread = reinterpret_cast<float*>(w + L.dkread);
     k.dktil = reinterpret_cast<float*>(w + L.dktil);
     k.dgate = a.dgate; k.dbeta = a.dbeta;
@@ -483,7 +544,7 @@ int kda_backward(const osdn_params& p, const Hyper& hy, const WsLayout& L, void*
         cudaMemsetAsync(k.dktil, 0, nK * 4, st) != cudaSuccess || cudaMemsetAsync(k.dgate, 0, nK * 4, st) != cudaSuccess ||
         cudaMemsetAsync(k.dbeta, 0, Ttot * p.H * 4, st) != cudaSuccess)
         return -1;
-    const dim3 grid(p.V / KB_WARPS, L.S * p.H);
+    const dim3 grid(p.V / (KB_WARPS * KB_RW), L.S * p.H);
     const size_t es = p.io_dtype == OSDN_BF16 ? 2 : 4;
     // the row sums' double buffer, then two token blocks (k, q in the I/O type; ktil, gates fp32)
     const size_t smem = (size_t)2 * KB_WARPS * 4 * p.K * sizeof(float) + 2 * (size_t)KTB * p.K * (2 * es + 8);
