@@ -4,11 +4,12 @@
 // with the state kept V x K as everywhere in this library (the paper's K x V state is its transpose).
 // Phase 1 (preconditioner, write keys, their adjoint) is the layer's own and is reused unchanged; this
 // file holds phase 2 and its adjoint as token-recurrent CUDA-core kernels in fp32: the rows of S do not
-// interact in the forward, so one warp owns one row (a lane holds K / 32 of its columns) and walks the
-// sequence; the dot products along a row are warp reductions.  The backward walks the chunks in
-// reverse: it replays a chunk from the row checkpoint the forward left at its start, keeping the row
-// before every token, then takes the adjoint steps; the sums over rows (dq, dk, d ktil, d gate, d beta)
-// are formed per CTA in shared memory and added to global fp32 accumulators.
+// interact in the forward, so a warp owns a few rows (a lane holds K / 32 columns of each) and walks the
+// sequence; the dot products along a row are warp reductions.  The backward walks the chunks in reverse:
+// from the row checkpoint the forward left at a chunk's start it first leaves a checkpoint at every
+// stretch of SUB tokens, then replays stretch by stretch, keeping the rows before every token, and takes
+// the adjoint steps; the sums over rows (dq, dk, d ktil, d gate, d beta) are formed per warp, then per CTA
+// in shared memory, and added to global fp32 accumulators.
 #include "osdn_common.cuh"
 
 namespace osdn {
